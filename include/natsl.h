@@ -1,0 +1,146 @@
+/*
+ * natsl.h -- C ABI of the B200 (sm_100a) hybrid attention layer of NAtS-L.
+ *
+ * The layer, per (batch, head), for tokens i = 0..L-1 with route r_i in {0,1}
+ * (1 = softmax token, K/V retained; 0 = linear token, folded into the state):
+ *
+ *   linear branch  (Section 4.3, Gated DeltaNet equation; decay on every token, the
+ *                   "always apply the decay" equation; update only for linear tokens,
+ *                   Section 4.1 case equation for the chunk state):
+ *       Sbar = exp(g_i) S ;  S = r_i ? Sbar : Sbar + beta_i k_i^T (v_i - k_i Sbar)
+ *       o_la_i = scale_la * q_i S
+ *   softmax branch (Section 4.1, O_nla equation with column mask M^nla):
+ *       o_nla_i = sum_{j<=i, r_j=1} softmax_j(scale_sm * q_i.k_j) v_j    (0 if no such j)
+ *   combination    (Section 4.3, Norm equation):
+ *       out_i = w_nla_i RMSnorm(o_nla_i) + w_la_i RMSnorm(o_la_i),
+ *       RMSnorm(x) = x / sqrt(mean_d(x^2) + eps)
+ *
+ * Every pointer below is a DEVICE pointer unless it says "host".  The caller owns all
+ * buffers and the stream; the library allocates nothing, keeps no per-call state, and only
+ * enqueues kernels on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ * Calls are asynchronous.  All tensors are dense, row-major, innermost dimension
+ * contiguous, in the shapes given.  Base pointers of q,k,v,out,dout,dq,dk,dv, the caches
+ * and the workspace must be 16-byte aligned.
+ *
+ * Return value: NATSL_OK or a negative natsl_status.  Arguments are validated on the host
+ * before anything is launched; an invalid call launches nothing.  Conditions only the
+ * device can see (decode cache full) are written to a status word that
+ * natsl_device_status() reads back; kernels never trap.
+ */
+#ifndef NATSL_H_
+#define NATSL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum natsl_status {
+    NATSL_OK = 0,
+    NATSL_ERR_NULL = -1,        /* a required pointer is NULL */
+    NATSL_ERR_SHAPE = -2,       /* B,H,L <= 0, L % C != 0, d not in {64,128}, C != 64 */
+    NATSL_ERR_DTYPE = -3,       /* dtype not NATSL_F32 / NATSL_BF16 */
+    NATSL_ERR_ALIGN = -4,       /* a tensor base is not 16-byte aligned */
+    NATSL_ERR_WORKSPACE = -5,   /* workspace NULL or smaller than natsl_workspace_size */
+    NATSL_ERR_CUDA = -6,        /* a launch or runtime call failed */
+    NATSL_ERR_CACHE_FULL = -7,  /* decode: a retained-KV cache has no room (device-detected) */
+    NATSL_ERR_UNSUPPORTED = -8  /* valid request this build does not implement */
+} natsl_status;
+
+enum { NATSL_F32 = 0, NATSL_BF16 = 1 };
+enum { NATSL_OP_FWD = 0, NATSL_OP_BWD = 1, NATSL_OP_DECODE = 2, NATSL_OP_COMPACT = 3 };
+
+/* flags */
+enum {
+    NATSL_FORCE_SIMT = 1u << 0   /* use the fp32 CUDA-core kernels even for bf16 tensors */
+};
+
+typedef struct natsl_params {
+    int32_t B, H, L, d;     /* d = d_k = d_v in {64, 128}; L % C == 0; decode ignores L */
+    int32_t C;              /* chunk size; must be 64 (Section 5: NAtS chunk = GDN chunk = 64) */
+    int32_t dtype;          /* storage type of q,k,v,out,dout,dq,dk,dv and the KV caches */
+    float scale_la;         /* logit scale of the linear read-out */
+    float scale_sm;         /* logit scale of the softmax branch */
+    float eps;              /* RMS-norm epsilon, > 0 */
+    uint32_t flags;
+    const float *w;         /* [B,L,H,2] (decode: [B,H,2]) = (w_nla, w_la); NULL => (0.5, 0.5) */
+    const float *state_in;  /* [B,H,d,d] fp32, row = key dim, col = value dim; NULL => zeros */
+    float *state_out;       /* [B,H,d,d] fp32 or NULL */
+    float *o_la;            /* optional raw linear-branch output  [B,L,H,d] fp32, or NULL */
+    float *o_nla;           /* optional raw softmax-branch output [B,L,H,d] fp32, or NULL */
+    float *lse;             /* optional log-sum-exp of the softmax logits [B,H,L] fp32, or NULL */
+    void *k_sm, *v_sm;      /* optional compacted K/V of the retained tokens [B,H,sm_cap,d], */
+    int32_t *sm_len;        /*   in `dtype`, with their counts [B,H]; all three or none.     */
+    int32_t sm_cap;         /*   This is the decode cache layout (prefill -> decode handoff). */
+} natsl_params;
+
+/* Bytes of workspace `op` needs for these shapes (host call, launches nothing). */
+int natsl_workspace_size(const natsl_params *p, int op, size_t *bytes /* host */);
+
+/*
+ * Route compaction: the column masks M^nla / M^la of Section 4.1 as index lists, so that the
+ * softmax branch loads only retained tokens and the linear branch only linear tokens.
+ *   route           [B,L,H] u8
+ *   sm_idx          [B,H,L]      ascending positions with route=1 (entries >= n_sm untouched)
+ *   sm_chunk_prefix [B,H,L/C+1]  exclusive prefix of per-chunk softmax counts, last = n_sm
+ *   lin_idx         [B,H,L/C,C]  ascending in-chunk offsets with route=0, padded with C
+ *   n_lin           [B,H,L/C]
+ * Integer work; exactly one result is correct.  No workspace needed (ws may be NULL).
+ */
+int natsl_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk_prefix,
+                        int32_t *lin_idx, int32_t *n_lin, const natsl_params *p,
+                        void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Forward of the whole layer (header comment; Sections 4.1 and 4.3).
+ *   q,k,v [B,L,H,d] in p->dtype; g,beta [B,L,H] fp32 (g = log decay <= 0);
+ *   route [B,L,H] u8; out [B,L,H,d] in p->dtype.
+ * The linear branch is computed chunkwise (Section 3, chunkwise equations) with C = 64.
+ * Optional outputs are taken from `p`.  Errors: NULL, SHAPE, DTYPE, ALIGN, WORKSPACE, CUDA.
+ */
+int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g,
+                     const float *beta, const uint8_t *route, void *out,
+                     const natsl_params *p, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * Backward of natsl_hybrid_fwd's `out` (Section 4.2 states the properties: the softmax-branch
+ * logit gradient is p (dp - <do,o>), and k, v gradients of an operation vanish for tokens
+ * inactive for it).  Self-contained: recomputes what it needs from the inputs.
+ *   dout [B,L,H,d] in p->dtype; dq,dk,dv [B,L,H,d] in p->dtype;
+ *   dg,dbeta [B,L,H] fp32; dw [B,L,H,2] fp32 or NULL.
+ * p->state_in must be NULL (zero initial state).  Errors as forward.
+ */
+int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g,
+                     const float *beta, const uint8_t *route, const void *dout,
+                     void *dq, void *dk, void *dv, float *dg, float *dbeta, float *dw,
+                     const natsl_params *p, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * One generation step (Section 4.1, per-token generation; the new token's route is known, so
+ * no roll-back is needed): decay the state, apply the delta rule (route 0) or append the
+ * token's K/V to the retained cache (route 1), then read both branches and combine.
+ *   q,k,v [B,H,d] in p->dtype; g,beta [B,H] fp32; route [B,H] u8; p->w [B,H,2] or NULL;
+ *   state [B,H,d,d] fp32, updated in place;
+ *   k_cache,v_cache [B,H,cache_cap,d] in p->dtype; cache_len [B,H] i32, updated in place;
+ *   out [B,H,d] in p->dtype.
+ * A sequence whose cache is full and whose token is routed to softmax is left untouched,
+ * its out row is zero-filled and NATSL_ERR_CACHE_FULL is recorded in the status word at the
+ * start of the workspace.  ws must hold natsl_workspace_size(p, NATSL_OP_DECODE) bytes and be
+ * zero-filled once before its first use.
+ */
+int natsl_decode_step(const void *q, const void *k, const void *v, const float *g,
+                      const float *beta, const uint8_t *route, float *state,
+                      void *k_cache, void *v_cache, int32_t *cache_len, int32_t cache_cap,
+                      void *out, const natsl_params *p, void *ws, size_t ws_bytes, void *stream);
+
+/* Synchronises `stream`, returns (and clears) the status word kernels wrote at ws[0]. */
+int natsl_device_status(void *ws, void *stream);
+
+const char *natsl_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NATSL_H_ */

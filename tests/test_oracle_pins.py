@@ -1,0 +1,444 @@
+"""Pins of the fp64 oracle against things other than itself: closed forms, special cases that
+reduce to a library routine (torch scaled_dot_product_attention, torch autograd), brute force on
+tiny inputs, finite differences, and the mask structure of the paper's Fig. 1(c)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import bruteforce, chunkwise
+
+RNG = np.random.default_rng(1234)
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rand_inputs(B, L, H, d, p=0.3, seed=0, unit=True):
+    r = np.random.default_rng(seed)
+    q = r.standard_normal((B, L, H, d))
+    k = r.standard_normal((B, L, H, d))
+    if unit:
+        q /= np.linalg.norm(q, axis=-1, keepdims=True)
+        k /= np.linalg.norm(k, axis=-1, keepdims=True)
+    v = r.standard_normal((B, L, H, d))
+    g = -np.log1p(np.exp(r.standard_normal((B, L, H))))
+    beta = 1 / (1 + np.exp(-r.standard_normal((B, L, H))))
+    route = (r.random((B, L, H)) < p).astype(np.uint8)
+    wz = np.exp(r.standard_normal((B, L, H, 2)))
+    w = wz / wz.sum(-1, keepdims=True)
+    return dict(q=q, k=k, v=v, g=g, beta=beta, route=route, w=w)
+
+
+def fwd(x, scale_la=0.5, scale_sm=1.5, eps=1e-5, **kw):
+    return oracle.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x.get("w"),
+                             scale_la=scale_la, scale_sm=scale_sm, eps=eps, **kw)
+
+
+# ------------------------------------------------------------------ compaction
+def test_compaction_against_nonzero():
+    for (B, L, H, C, p) in [(2, 256, 3, 64, 0.25), (1, 128, 2, 64, 0.0), (1, 128, 2, 64, 1.0),
+                            (1, 24, 1, 4, 0.5)]:
+        route = (RNG.random((B, L, H)) < p).astype(np.uint8)
+        res = oracle.route_compact(route, C)
+        NC = L // C
+        for b in range(B):
+            for h in range(H):
+                col = route[b, :, h]
+                pos = np.nonzero(col)[0]
+                n_sm = len(pos)
+                assert res["sm_chunk_prefix"][b, h, NC] == n_sm
+                assert np.array_equal(res["sm_idx"][b, h, :n_sm], pos)
+                assert n_sm + res["n_lin"][b, h].sum() == L
+                cnt = col.reshape(NC, C).sum(1)
+                assert np.array_equal(np.diff(res["sm_chunk_prefix"][b, h]), cnt)
+                for c in range(NC):
+                    lin = np.nonzero(col[c * C:(c + 1) * C] == 0)[0]
+                    assert res["n_lin"][b, h, c] == len(lin)
+                    assert np.array_equal(res["lin_idx"][b, h, c, :len(lin)], lin)
+                    assert np.all(res["lin_idx"][b, h, c, len(lin):] == C)
+
+
+def test_compaction_single_bit_and_reject():
+    route = np.zeros((1, 128, 1), np.uint8)
+    route[0, 77, 0] = 1
+    res = oracle.route_compact(route, 64)
+    assert res["sm_idx"][0, 0, 0] == 77 and list(res["sm_chunk_prefix"][0, 0]) == [0, 0, 1]
+    assert list(res["n_lin"][0, 0]) == [64, 63]
+    with pytest.raises(ValueError):
+        oracle.route_compact(np.zeros((1, 100, 1), np.uint8), 64)
+
+
+# ------------------------------------------------------------------ linear branch
+def test_recurrent_equals_chunkwise():
+    x = rand_inputs(2, 192, 2, 16, p=0.3, seed=1)
+    S0 = RNG.standard_normal((2, 2, 16, 16))
+    r = fwd(x, state_in=S0)
+    for b in range(2):
+        for h in range(2):
+            o, S = chunkwise.gdn_chunkwise(x["q"][b, :, h], x["k"][b, :, h], x["v"][b, :, h],
+                                           x["g"][b, :, h], x["beta"][b, :, h], x["route"][b, :, h],
+                                           64, 0.5, state_in=S0[b, h])
+            np.testing.assert_allclose(o, r["o_la"][b, :, h], rtol=1e-10, atol=1e-12)
+            np.testing.assert_allclose(S, r["state_out"][b, h], rtol=1e-10, atol=1e-12)
+
+
+def test_bruteforce_tiny():
+    x = rand_inputs(1, 12, 2, 5, p=0.35, seed=2)
+    S0 = RNG.standard_normal((1, 2, 5, 5))
+    r = fwd(x, state_in=S0)
+    for h in range(2):
+        o_la, S = bruteforce.linear_branch(x["q"][0, :, h], x["k"][0, :, h], x["v"][0, :, h],
+                                           x["g"][0, :, h], x["beta"][0, :, h], x["route"][0, :, h],
+                                           0.5, state_in=S0[0, h])
+        o_nla = bruteforce.softmax_branch(x["q"][0, :, h], x["k"][0, :, h], x["v"][0, :, h],
+                                          x["route"][0, :, h], 1.5)
+        np.testing.assert_allclose(o_la, r["o_la"][0, :, h], rtol=1e-10, atol=1e-13)
+        np.testing.assert_allclose(S, r["state_out"][0, h], rtol=1e-10, atol=1e-13)
+        np.testing.assert_allclose(o_nla, r["o_nla"][0, :, h], rtol=1e-10, atol=1e-13)
+        out = bruteforce.combine(o_nla, o_la, x["w"][0, :, h], 1e-5)
+        np.testing.assert_allclose(out, r["out"][0, :, h], rtol=1e-10, atol=1e-13)
+
+
+def test_hybrid_equals_pure_gdn_with_masked_beta():
+    x = rand_inputs(1, 96, 2, 8, p=0.4, seed=3)
+    r = fwd(x)
+    y = dict(x)
+    y["beta"] = x["beta"] * (1 - x["route"])
+    y["route"] = np.zeros_like(x["route"])
+    r2 = fwd(y)
+    np.testing.assert_allclose(r["o_la"], r2["o_la"], rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(r["state_out"], r2["state_out"], rtol=1e-12, atol=1e-15)
+    assert np.all(r2["o_nla"] == 0) and np.all(np.isneginf(r2["lse"]))
+
+
+def test_alpha_one_reduces_to_deltanet_paper_orientation():
+    """g = 0, all-linear: the DeltaNet equation of Section 4.3 in the paper's own orientation,
+    S in R^{dv x dk}, S_t = S_{t-1}(I - beta k k^T) + beta v k^T, o = S q."""
+    x = rand_inputs(1, 40, 1, 6, p=0.0, seed=4)
+    x["g"] = np.zeros_like(x["g"])
+    r = fwd(x, scale_la=1.0)
+    d = 6
+    S = np.zeros((d, d))
+    for t in range(40):
+        k, v, b = x["k"][0, t, 0], x["v"][0, t, 0], x["beta"][0, t, 0]
+        S = S @ (np.eye(d) - b * np.outer(k, k)) + b * np.outer(v, k)
+        np.testing.assert_allclose(S @ x["q"][0, t, 0], r["o_la"][0, t, 0], rtol=1e-11, atol=1e-14)
+    np.testing.assert_allclose(S.T, r["state_out"][0, 0], rtol=1e-11, atol=1e-14)
+
+
+def test_gdn_paper_orientation_with_decay():
+    """All-linear, g != 0: S_t = S_{t-1} alpha_t (I - beta_t k k^T) + beta_t v k^T (Section 4.3)."""
+    x = rand_inputs(1, 30, 1, 5, p=0.0, seed=5)
+    r = fwd(x, scale_la=1.0)
+    S = np.zeros((5, 5))
+    for t in range(30):
+        k, v, b, a = x["k"][0, t, 0], x["v"][0, t, 0], x["beta"][0, t, 0], np.exp(x["g"][0, t, 0])
+        S = S @ (a * (np.eye(5) - b * np.outer(k, k))) + b * np.outer(v, k)
+        np.testing.assert_allclose(S @ x["q"][0, t, 0], r["o_la"][0, t, 0], rtol=1e-11, atol=1e-14)
+
+
+def test_state_invariants_beta_zero():
+    x = rand_inputs(1, 64, 1, 8, p=0.3, seed=6)
+    S0 = RNG.standard_normal((1, 1, 8, 8))
+    x["beta"] = np.zeros_like(x["beta"])
+    r = fwd(x, state_in=S0)
+    np.testing.assert_allclose(r["state_out"], np.exp(x["g"].sum()) * S0, rtol=1e-12)
+    x["g"] = np.zeros_like(x["g"])
+    r = fwd(x, state_in=S0)
+    assert np.array_equal(r["state_out"], S0)          # bit for bit
+
+
+def test_decay_always_on_softmax_tokens():
+    """All tokens routed to softmax: the state is never written, only decayed, and a softmax
+    token's linear read sees the state after its own decay."""
+    x = rand_inputs(1, 20, 1, 4, p=1.1, seed=7)
+    S0 = RNG.standard_normal((1, 1, 4, 4))
+    r = fwd(x, state_in=S0, scale_la=0.7)
+    G = np.cumsum(x["g"][0, :, 0])
+    np.testing.assert_allclose(r["state_out"][0, 0], np.exp(G[-1]) * S0[0, 0], rtol=1e-12)
+    for i in range(20):
+        np.testing.assert_allclose(r["o_la"][0, i, 0], 0.7 * np.exp(G[i]) * x["q"][0, i, 0] @ S0[0, 0],
+                                   rtol=1e-12)
+
+
+def test_delta_rule_writes_value():
+    """beta = 1 and |k| = 1: after the update, k_t S_t = v_t exactly (delta rule)."""
+    x = rand_inputs(1, 10, 1, 6, p=0.0, seed=8)
+    x["beta"] = np.ones_like(x["beta"])
+    y = dict(x)
+    y["q"] = x["k"]
+    r = fwd(y, scale_la=1.0)
+    np.testing.assert_allclose(r["o_la"], x["v"], rtol=1e-12, atol=1e-13)
+
+
+def test_orthonormal_keys_plain_linear_attention():
+    d = 8
+    Q, _ = np.linalg.qr(RNG.standard_normal((d, d)))
+    x = rand_inputs(1, d, 1, d, p=0.0, seed=9)
+    x["k"] = Q[None, :, None, :].copy()
+    x["beta"] = np.ones_like(x["beta"])
+    x["g"] = np.zeros_like(x["g"])
+    r = fwd(x)
+    S = sum(np.outer(Q[j], x["v"][0, j, 0]) for j in range(d))
+    np.testing.assert_allclose(r["state_out"][0, 0], S, rtol=1e-12, atol=1e-13)
+
+
+# ------------------------------------------------------------------ softmax branch
+def test_all_softmax_equals_library_causal_attention():
+    x = rand_inputs(2, 50, 3, 16, p=1.1, seed=10, unit=False)
+    r = fwd(x, scale_sm=0.3)
+    tq, tk, tv = (torch.from_numpy(x[n]).permute(0, 2, 1, 3) for n in ("q", "k", "v"))
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True, scale=0.3)
+    np.testing.assert_allclose(r["o_nla"], ref.permute(0, 2, 1, 3).numpy(), rtol=1e-10, atol=1e-12)
+    # independent double loop for the log-sum-exp
+    for i in (0, 7, 49):
+        s = 0.3 * x["k"][1, :i + 1, 2] @ x["q"][1, i, 2]
+        assert abs(np.log(np.exp(s).sum()) - r["lse"][1, 2, i]) < 1e-10
+
+
+def test_mixed_route_equals_library_masked_attention():
+    x = rand_inputs(1, 70, 2, 8, p=0.3, seed=11, unit=False)
+    x["route"][0, 0, :] = 1                               # no empty rows
+    r = fwd(x, scale_sm=0.9)
+    tq, tk, tv = (torch.from_numpy(x[n]).permute(0, 2, 1, 3) for n in ("q", "k", "v"))
+    L = 70
+    keep = torch.from_numpy(x["route"].astype(bool)).permute(0, 2, 1)[:, :, None, :]  # [B,H,1,L]
+    mask = torch.tril(torch.ones(L, L, dtype=torch.bool))[None, None] & keep
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, attn_mask=mask, scale=0.9)
+    np.testing.assert_allclose(r["o_nla"], ref.permute(0, 2, 1, 3).numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_single_retained_token_and_empty_rows():
+    x = rand_inputs(1, 16, 1, 4, p=0.0, seed=12)
+    x["route"][0, 5, 0] = 1
+    r = fwd(x)
+    assert np.all(r["o_nla"][0, :5] == 0) and np.all(np.isneginf(r["lse"][0, 0, :5]))
+    for i in range(5, 16):
+        np.testing.assert_allclose(r["o_nla"][0, i, 0], x["v"][0, 5, 0], rtol=1e-13)
+
+
+# ------------------------------------------------------------------ combination
+def test_combination_properties():
+    x = rand_inputs(1, 32, 2, 16, p=0.3, seed=13)
+    x["route"][0, 0, :] = 1
+    x["w"] = np.zeros_like(x["w"])
+    x["w"][..., 0] = 1.0
+    r = fwd(x, eps=1e-12)
+    np.testing.assert_allclose(np.sqrt((r["out"] ** 2).mean(-1)), 1.0, rtol=1e-8)
+    x["w"][..., 0], x["w"][..., 1] = 0.0, 1.0
+    r = fwd(x, eps=1e-12)
+    rms = np.sqrt((r["out"] ** 2).mean(-1))
+    nz = np.abs(r["o_la"]).max(-1) > 0                    # empty state: Norm(0) = 0
+    np.testing.assert_allclose(rms[nz], 1.0, rtol=1e-6)
+    assert np.all(rms[~nz] == 0) and nz.sum() > 50
+    # all-linear: out = w_la Norm(GDN), the softmax branch contributes Norm(0) = 0
+    y = rand_inputs(1, 32, 1, 8, p=0.0, seed=14)
+    r = fwd(y)
+    o = r["o_la"]
+    ref = y["w"][..., 1:2] * o / np.sqrt((o * o).mean(-1, keepdims=True) + 1e-5)
+    np.testing.assert_allclose(r["out"], ref, rtol=1e-12, atol=1e-15)
+    # w = None means (1/2, 1/2)
+    y2 = dict(y)
+    y2["w"] = None
+    y3 = dict(y)
+    y3["w"] = np.full_like(y["w"], 0.5)
+    assert np.array_equal(fwd(y2)["out"], fwd(y3)["out"])
+
+
+# ------------------------------------------------------------------ Fig. 1(c)
+def _influence(x, field, i_out, scale=1e-3):
+    """|d o[i_out] / d v_j| > 0 pattern by perturbing v_j, j = 0..L-1."""
+    base = fwd(x)[field][0, :, 0]
+    L = base.shape[0]
+    vis = np.zeros((L, L), bool)
+    for j in range(L):
+        y = {n: a.copy() if isinstance(a, np.ndarray) else a for n, a in x.items()}
+        y["v"][0, j, 0] += scale
+        vis[:, j] = np.abs(fwd(y)[field][0, :, 0] - base).max(-1) > 0
+    return vis
+
+
+def test_fig1c_visibility_pattern():
+    rows = [ln.strip() for ln in open(os.path.join(GOLDEN, "fig1c_visibility.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 12 and all(len(r) == 12 for r in rows)
+    fig = np.array([list(r) for r in rows])
+    C = 2
+    route = np.zeros(12, np.uint8)
+    route[[0, 1, 6, 7]] = 1                               # chunks 1 and 4 are softmax chunks
+    x = rand_inputs(1, 12, 1, 4, seed=15)
+    x["route"] = route[None, :, None].copy()
+    x["beta"] = np.full_like(x["beta"], 0.7)
+    sm = _influence(x, "o_nla", None)
+    la = _influence(x, "o_la", None)
+    chunk = np.arange(12) // C
+    earlier = chunk[:, None] > chunk[None, :]             # key in an earlier chunk than the query
+    # softmax branch: cross-chunk cells are exactly the figure's S cells
+    assert np.array_equal(sm & earlier, fig == "S")
+    # linear branch: the state a query reads from earlier chunks holds linear tokens up to the
+    # column where the figure draws its G cell, and nothing when the row has no G
+    for i in range(12):
+        cols = np.nonzero(la[i] & earlier[i])[0]
+        gcol = np.nonzero(fig[i] == "G")[0]
+        if len(gcol) == 0:
+            assert len(cols) == 0
+        else:
+            assert cols.max() == gcol[0]
+            assert np.all(route[cols] == 0)
+    # each token is visible in exactly one branch, causally
+    assert np.array_equal(sm | la, np.tril(np.ones((12, 12), bool)))
+    assert not np.any(sm & la)
+    m_nla, m_la = bruteforce.masks(route)
+    assert np.array_equal(sm, m_nla) and np.array_equal(la, m_la)
+
+
+# ------------------------------------------------------------------ decode
+def test_decode_from_empty_equals_forward_rows():
+    x = rand_inputs(2, 24, 2, 8, p=0.3, seed=16)
+    r = fwd(x)
+    B, L, H, d = x["q"].shape
+    state = np.zeros((B, H, d, d))
+    kc, vc = np.zeros((B, H, L, d)), np.zeros((B, H, L, d))
+    n = np.zeros((B, H), np.int32)
+    for t in range(L):
+        o = oracle.decode_step(x["q"][:, t], x["k"][:, t], x["v"][:, t], x["g"][:, t],
+                               x["beta"][:, t], x["route"][:, t], x["w"][:, t], state, kc, vc, n,
+                               scale_la=0.5, scale_sm=1.5)
+        np.testing.assert_allclose(o["out"], r["out"][:, t], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(state, r["state_out"], rtol=1e-12, atol=1e-15)
+    assert np.array_equal(n, x["route"].sum(1).astype(np.int32))
+
+
+def test_prefill_handoff_then_one_step():
+    x = rand_inputs(1, 33, 2, 8, p=0.3, seed=17)
+    full = fwd(x)
+    head = {n: (a[:, :32] if a is not None else None) for n, a in x.items()}
+    r = fwd(head, want_cache=True)
+    state = r["state_out"].copy()
+    cap = 40
+    kc, vc = np.zeros((1, 2, cap, 8)), np.zeros((1, 2, cap, 8))
+    kc[:, :, :32], vc[:, :, :32] = r["k_sm"], r["v_sm"]
+    n = r["n_sm"].copy()
+    o = oracle.decode_step(x["q"][:, 32], x["k"][:, 32], x["v"][:, 32], x["g"][:, 32],
+                           x["beta"][:, 32], x["route"][:, 32], x["w"][:, 32], state, kc, vc, n,
+                           scale_la=0.5, scale_sm=1.5)
+    np.testing.assert_allclose(o["out"], full["out"][:, 32], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(state, full["state_out"], rtol=1e-12, atol=1e-15)
+
+
+def test_decode_cache_full():
+    x = rand_inputs(1, 1, 1, 4, p=1.1, seed=18)
+    state = np.zeros((1, 1, 4, 4))
+    kc, vc = np.zeros((1, 1, 2, 4)), np.zeros((1, 1, 2, 4))
+    n = np.full((1, 1), 2, np.int32)
+    with pytest.raises(OverflowError):
+        oracle.decode_step(x["q"][:, 0], x["k"][:, 0], x["v"][:, 0], x["g"][:, 0], x["beta"][:, 0],
+                           x["route"][:, 0], None, state, kc, vc, n, scale_la=1.0, scale_sm=1.0)
+
+
+# ------------------------------------------------------------------ backward
+def _loss(x, dout, S0, dS):
+    r = fwd(x, state_in=S0)
+    return (r["out"] * dout).sum() + (r["state_out"] * dS).sum()
+
+
+def test_backward_finite_differences():
+    B, L, H, d = 1, 20, 2, 6
+    x = rand_inputs(B, L, H, d, p=0.3, seed=19, unit=False)
+    x["q"] *= 0.5
+    x["k"] *= 0.4
+    x["route"][0, 0, 0] = 1
+    x["route"][0, :3, 1] = 0                               # head 1 starts with empty softmax rows
+    dout = RNG.standard_normal((B, L, H, d))
+    S0 = RNG.standard_normal((B, H, d, d)) * 0.3
+    dS = RNG.standard_normal((B, H, d, d))
+    gr = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], dout,
+                           scale_la=0.5, scale_sm=1.5, state_in=S0, dstate_out=dS)
+    h = 1e-6
+    checks = [("q", "dq"), ("k", "dk"), ("v", "dv"), ("g", "dg"), ("beta", "dbeta"), ("w", "dw")]
+    pick = np.random.default_rng(5)
+    for name, gname in checks:
+        flat = x[name].reshape(-1)
+        for idx in pick.choice(flat.size, size=min(40, flat.size), replace=False):
+            old = flat[idx]
+            flat[idx] = old + h
+            lp = _loss(x, dout, S0, dS)
+            flat[idx] = old - h
+            lm = _loss(x, dout, S0, dS)
+            flat[idx] = old
+            fd = (lp - lm) / (2 * h)
+            an = gr[gname].reshape(-1)[idx]
+            assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)) + 1e-7, (name, idx, fd, an)
+    flat = S0.reshape(-1)
+    for idx in pick.choice(flat.size, size=20, replace=False):
+        old = flat[idx]
+        flat[idx] = old + h
+        lp = _loss(x, dout, S0, dS)
+        flat[idx] = old - h
+        lm = _loss(x, dout, S0, dS)
+        flat[idx] = old
+        assert abs((lp - lm) / (2 * h) - gr["dstate_in"].reshape(-1)[idx]) < 2e-6
+
+
+def _torch_forward(q, k, v, g, beta, route, w, scale_la, scale_sm, eps):
+    """Same layer written with torch ops (masked library attention + a python recurrence) so that
+    torch autograd differentiates it; one (batch, head)."""
+    L, d = q.shape
+    S = torch.zeros(d, d, dtype=torch.float64)
+    o_la = []
+    for i in range(L):
+        S = torch.exp(g[i]) * S
+        if not route[i]:
+            S = S + beta[i] * torch.outer(k[i], v[i] - k[i] @ S)
+        o_la.append(scale_la * (q[i] @ S))
+    o_la = torch.stack(o_la)
+    keep = torch.tensor(route.astype(bool))
+    mask = torch.tril(torch.ones(L, L, dtype=torch.bool)) & keep[None, :]
+    o_nla = torch.nn.functional.scaled_dot_product_attention(q[None], k[None], v[None],
+                                                             attn_mask=mask[None], scale=scale_sm)[0]
+    rows = mask.any(1)
+    o_nla = torch.where(rows[:, None], o_nla, torch.zeros_like(o_nla))
+
+    def norm(x):
+        return x * torch.rsqrt((x * x).mean(-1, keepdim=True) + eps)
+    return w[:, 0:1] * norm(o_nla) + w[:, 1:2] * norm(o_la)
+
+
+def test_backward_equals_autograd():
+    B, L, H, d = 1, 48, 1, 8
+    x = rand_inputs(B, L, H, d, p=0.3, seed=20)
+    x["route"][0, 0, 0] = 1
+    dout = RNG.standard_normal((B, L, H, d))
+    gr = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], dout,
+                           scale_la=0.35, scale_sm=2.8)
+    t = {n: torch.tensor(x[n][0, :, 0], dtype=torch.float64, requires_grad=True)
+         for n in ("q", "k", "v", "g", "beta", "w")}
+    out = _torch_forward(t["q"], t["k"], t["v"], t["g"], t["beta"], x["route"][0, :, 0], t["w"],
+                         0.35, 2.8, 1e-5)
+    np.testing.assert_allclose(out.detach().numpy(), fwd(x, 0.35, 2.8)["out"][0, :, 0], rtol=1e-10,
+                               atol=1e-12)
+    (out * torch.from_numpy(dout[0, :, 0])).sum().backward()
+    for n, gn in [("q", "dq"), ("k", "dk"), ("v", "dv"), ("g", "dg"), ("beta", "dbeta"), ("w", "dw")]:
+        np.testing.assert_allclose(gr[gn][0, :, 0], t[n].grad.numpy(), rtol=1e-8, atol=1e-11,
+                                   err_msg=n)
+
+
+def test_inactive_branch_gradients_vanish():
+    """k, v gradients of an operation vanish for tokens that are inactive for it (Section 4.2)."""
+    x = rand_inputs(1, 40, 2, 8, p=0.3, seed=21)
+    x["route"][0, 0, :] = 1
+    dout = RNG.standard_normal(x["q"].shape)
+    lin = x["route"] == 0
+    only_sm = dict(x)
+    only_sm["w"] = np.stack([np.ones_like(x["g"]), np.zeros_like(x["g"])], -1)
+    gs = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], only_sm["w"], dout,
+                           scale_la=0.5, scale_sm=1.5)
+    assert np.all(gs["dk"][lin] == 0) and np.all(gs["dv"][lin] == 0)
+    assert np.all(gs["dbeta"] == 0) and np.all(gs["dg"] == 0)
+    only_la = np.stack([np.zeros_like(x["g"]), np.ones_like(x["g"])], -1)
+    gl = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], only_la, dout,
+                           scale_la=0.5, scale_sm=1.5)
+    assert np.all(gl["dk"][~lin] == 0) and np.all(gl["dv"][~lin] == 0)
+    assert np.all(gl["dbeta"][~lin] == 0)
+    assert np.abs(gl["dk"][lin]).min() > 0
