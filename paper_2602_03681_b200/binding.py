@@ -1,0 +1,178 @@
+"""Thin ctypes binding of ``libnatsl.so`` -- same names as the C ABI (``include/natsl.h``).
+
+Argument marshalling only: torch supplies device memory and streams, every step of the path
+runs in the library's CUDA kernels.  There is no fallback of any kind: if the library is not
+built, importing the entry points raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnatsl.so")
+
+NATSL_F32, NATSL_BF16 = 0, 1
+OP_FWD, OP_BWD, OP_DECODE, OP_COMPACT = 0, 1, 2, 3
+FORCE_SIMT = 1
+ERR_CACHE_FULL = -7
+
+EXPORTS = ["natsl_workspace_size", "natsl_route_compact", "natsl_hybrid_fwd", "natsl_hybrid_bwd",
+           "natsl_decode_step", "natsl_device_status", "natsl_strerror"]
+
+
+class NatslError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"natsl status {status}: {msg}")
+        self.status = status
+
+
+class natsl_params(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("L", ctypes.c_int32),
+                ("d", ctypes.c_int32), ("C", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("scale_la", ctypes.c_float), ("scale_sm", ctypes.c_float),
+                ("eps", ctypes.c_float), ("flags", ctypes.c_uint32),
+                ("w", ctypes.c_void_p), ("state_in", ctypes.c_void_p),
+                ("state_out", ctypes.c_void_p), ("o_la", ctypes.c_void_p),
+                ("o_nla", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("k_sm", ctypes.c_void_p),
+                ("v_sm", ctypes.c_void_p), ("sm_len", ctypes.c_void_p),
+                ("sm_cap", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library; raise loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2602_03681_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        _lib = ctypes.CDLL(LIB_PATH)
+        _lib.natsl_strerror.restype = ctypes.c_char_p
+        _lib.natsl_strerror.argtypes = [ctypes.c_int]
+        for name in EXPORTS[:-1]:
+            getattr(_lib, name).restype = ctypes.c_int
+    return _lib
+
+
+def natsl_strerror(status: int) -> str:
+    return lib().natsl_strerror(int(status)).decode()
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise NatslError(rc, natsl_strerror(rc))
+
+
+def _ptr(t):
+    if t is None:
+        return ctypes.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t) -> int:
+    if t.dtype == torch.float32:
+        return NATSL_F32
+    if t.dtype == torch.bfloat16:
+        return NATSL_BF16
+    raise NatslError(-3, "dtype must be float32 or bfloat16")
+
+
+def make_params(B, H, L, d, dtype_code, scale_la, scale_sm, eps=1e-5, C=64, flags=0, w=None,
+                state_in=None, state_out=None, o_la=None, o_nla=None, lse=None, k_sm=None,
+                v_sm=None, sm_len=None, sm_cap=0) -> natsl_params:
+    p = natsl_params()
+    p.B, p.H, p.L, p.d, p.C, p.dtype = B, H, L, d, C, dtype_code
+    p.scale_la, p.scale_sm, p.eps, p.flags = scale_la, scale_sm, eps, flags
+    for name, t in dict(w=w, state_in=state_in, state_out=state_out, o_la=o_la, o_nla=o_nla,
+                        lse=lse, k_sm=k_sm, v_sm=v_sm, sm_len=sm_len).items():
+        setattr(p, name, _ptr(t).value)
+    p.sm_cap = sm_cap
+    return p
+
+
+def natsl_workspace_size(p: natsl_params, op: int) -> int:
+    n = ctypes.c_size_t(0)
+    _check(lib().natsl_workspace_size(ctypes.byref(p), op, ctypes.byref(n)))
+    return int(n.value)
+
+
+def alloc_workspace(p: natsl_params, op: int, device="cuda") -> torch.Tensor:
+    """Zero-filled byte tensor of the size the library asks for (at least 256 bytes)."""
+    return torch.zeros(max(natsl_workspace_size(p, op), 256), dtype=torch.uint8, device=device)
+
+
+def natsl_route_compact(route, sm_idx, sm_chunk_prefix, lin_idx, n_lin, p: natsl_params):
+    _check(lib().natsl_route_compact(_ptr(route), _ptr(sm_idx), _ptr(sm_chunk_prefix),
+                                     _ptr(lin_idx), _ptr(n_lin), ctypes.byref(p),
+                                     ctypes.c_void_p(0), ctypes.c_size_t(0), _stream()))
+
+
+def natsl_hybrid_fwd(q, k, v, g, beta, route, out, p: natsl_params, ws):
+    _check(lib().natsl_hybrid_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(route),
+                                  _ptr(out), ctypes.byref(p), _ptr(ws),
+                                  ctypes.c_size_t(ws.numel()), _stream()))
+
+
+def natsl_hybrid_bwd(q, k, v, g, beta, route, dout, dq, dk, dv, dg, dbeta, dw, p: natsl_params, ws):
+    _check(lib().natsl_hybrid_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(route),
+                                  _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dg), _ptr(dbeta),
+                                  _ptr(dw), ctypes.byref(p), _ptr(ws),
+                                  ctypes.c_size_t(ws.numel()), _stream()))
+
+
+def natsl_decode_step(q, k, v, g, beta, route, state, k_cache, v_cache, cache_len, out,
+                      p: natsl_params, ws):
+    cap = k_cache.shape[2]
+    _check(lib().natsl_decode_step(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(route),
+                                   _ptr(state), _ptr(k_cache), _ptr(v_cache), _ptr(cache_len),
+                                   ctypes.c_int32(cap), _ptr(out), ctypes.byref(p), _ptr(ws),
+                                   ctypes.c_size_t(ws.numel()), _stream()))
+
+
+def natsl_device_status(ws) -> int:
+    return int(lib().natsl_device_status(_ptr(ws), _stream()))
+
+
+# ---------------------------------------------------------------------------------------------
+# Convenience wrappers (allocation + marshalling; no arithmetic).
+# ---------------------------------------------------------------------------------------------
+def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5, state_in=None,
+               want=(), flags=0, sm_cap=0, ws=None):
+    """Allocate outputs and run natsl_hybrid_fwd.  `want` may name optional outputs:
+    "o_la", "o_nla", "lse", "state_out", "cache" (compacted K/V with capacity sm_cap or L)."""
+    B, L, H, d = q.shape
+    dev = q.device
+    out = torch.empty_like(q)
+    opt = {}
+    if "o_la" in want:
+        opt["o_la"] = torch.empty((B, L, H, d), dtype=torch.float32, device=dev)
+    if "o_nla" in want:
+        opt["o_nla"] = torch.empty((B, L, H, d), dtype=torch.float32, device=dev)
+    if "lse" in want:
+        opt["lse"] = torch.empty((B, H, L), dtype=torch.float32, device=dev)
+    if "state_out" in want:
+        opt["state_out"] = torch.empty((B, H, d, d), dtype=torch.float32, device=dev)
+    cap = 0
+    if "cache" in want:
+        cap = sm_cap or L
+        opt["k_sm"] = torch.zeros((B, H, cap, d), dtype=q.dtype, device=dev)
+        opt["v_sm"] = torch.zeros((B, H, cap, d), dtype=q.dtype, device=dev)
+        opt["sm_len"] = torch.zeros((B, H), dtype=torch.int32, device=dev)
+    p = make_params(B, H, L, d, _dtype_code(q), scale_la, scale_sm, eps, flags=flags, w=w,
+                    state_in=state_in, sm_cap=cap, **opt)
+    if ws is None:
+        ws = alloc_workspace(p, OP_FWD, dev)
+    natsl_hybrid_fwd(q, k, v, g, beta, route, out, p, ws)
+    res = dict(out=out, ws=ws, **opt)
+    return res
