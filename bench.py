@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the NAtS-L hybrid attention layer on B200.
+
+`python bench.py --gpus N --steps K --warmup W` times K forward passes of the whole hot path
+(route compaction -> chunkwise Gated DeltaNet -> sparse softmax -> combination) on the bf16
+prefill workload (B=4, H=16, L=4096, d=128, C=64, 10 % softmax tokens) per GPU and prints ONE
+JSON line.  With N > 1 (launched by torch.distributed.run) every rank runs its own batch
+(independent (batch, head) problems, no collective on the data path): weak scaling.
+
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2602_03681_b200 import inputs  # noqa: E402
+
+METRIC = "hybrid_layer_fwd_tokens_per_s"
+UNIT = "tokens/s"
+WORKLOAD = "cfg1_bf16_prefill"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+# ------------------------------------------------------------------------------------------
+# algorithmic work (counted from the realised routing masks)
+# ------------------------------------------------------------------------------------------
+def useful_flops(route: np.ndarray, d: int, C: int = 64):
+    """Useful FLOPs of one forward, per stage, from the compacted algorithm (1 FMA = 2 FLOPs).
+    GDN per chunk with n linear tokens:
+      prepare: 6 n^2 d [K K^T, T(beta V), T(beta gamma K)] + 2 C n d [Q K_lin^T]
+      scan   : 2 d^2 (2 n + C) [W S, K~^T U~, Q S] + 2 C n d [P U~]
+    softmax per (batch, head): 4 d sum_i |{j <= i : route_j = 1}|."""
+    B, L, H = route.shape
+    r = route.astype(np.int64)
+    n = (C - r.reshape(B, L // C, C, H).sum(2)).astype(np.float64)       # linear tokens per chunk
+    prepare = float((6 * n * n * d + 2 * C * n * d).sum())
+    scan = float((2 * d * d * (2 * n + C) + 2 * C * n * d).sum())
+    nvis = np.cumsum(r, axis=1)
+    softmax = float(4 * d * nvis.sum())
+    return {"gdn_prepare": prepare, "gdn_scan": scan, "softmax_combine": softmax}
+
+
+def min_hbm_bytes_fwd(wl, B):
+    """q, k, v read once + out written once + the small per-token tensors."""
+    e = 2 if wl.dtype == "bf16" else 4
+    tok = B * wl.L * wl.H
+    return tok * wl.d * e * 4 + tok * (4 + 4 + 1 + 8)
+
+
+def decode_bytes_per_step(B, H, d, cache_len_mean, e=2):
+    """state read + written (fp32), retained K and V read once, per (sequence, head)."""
+    return B * H * (2 * d * d * 4 + 2 * cache_len_mean * d * e)
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def load_traffic():
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f)
+    return {}
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                      "sw_power_cap"), f[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ------------------------------------------------------------------------------------------
+# reference arm: the fp64 CPU oracle on a bounded sample
+# ------------------------------------------------------------------------------------------
+def oracle_sample_inputs(wl, sample_B):
+    x = inputs.make_layer_inputs(wl, B=sample_B)
+    return x
+
+
+def time_oracle(wl, x, repeats):
+    import oracle
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        oracle.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"],
+                          scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+        times.append(time.perf_counter() - t0)
+    return times, oracle.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = inputs.WORKLOADS[WORKLOAD]
+    sample_B = 1
+    x = oracle_sample_inputs(wl, sample_B)
+    time_oracle(wl, x, 1)      # page in, spin up OpenMP
+    times, cores = time_oracle(wl, x, args.steps)
+    total = sum(times)
+    value = sample_B * wl.L * args.steps / total
+    sample = f"{sample_B} of {wl.B} sequences of the workload per step (all {wl.H} heads, L={wl.L})"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "B": sample_B, "H": wl.H, "L": wl.L, "d": wl.d, "C": wl.C,
+                   "p_softmax": wl.p_softmax, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2602_03681_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    binding.lib()   # fail loudly here if the CUDA library is missing
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    wl = inputs.WORKLOADS[WORKLOAD]
+    wl_rank = inputs.Workload(**{**wl.__dict__, "seed": wl.seed + 1000 * rank})
+    x = inputs.make_layer_inputs(wl_rank)
+    dt = torch.bfloat16
+    B, L, H, d = wl.B, wl.L, wl.H, wl.d
+
+    host = {n: torch.from_numpy(x[n]) for n in ("q", "k", "v", "g", "beta", "route", "w")}
+    for n in ("q", "k", "v"):
+        host[n] = host[n].to(dt)
+    host = {n: t.contiguous().pin_memory() for n, t in host.items()}
+    devt = {n: t.cuda() for n, t in host.items()}
+    out = torch.empty((B, L, H, d), dtype=dt, device="cuda")
+    out_host = torch.empty((B, L, H, d), dtype=dt).pin_memory()
+
+    p = binding.make_params(B, H, L, d, binding.NATSL_BF16, wl.scale_la, wl.scale_sm, w=devt["w"])
+    ws = binding.alloc_workspace(p, binding.OP_FWD)
+
+    def step():
+        binding.natsl_hybrid_fwd(devt["q"], devt["k"], devt["v"], devt["g"], devt["beta"],
+                                 devt["route"], out, p, ws)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(ws) == 0
+
+    # ---- timed region: K steps, inputs resident in HBM ----
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = binding.natsl_launch_count()
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    launches = binding.natsl_launch_count() - launches0
+    ms = max_over_ranks(e0.elapsed_time(e1))
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = ms / args.steps
+    value = world * B * L / (ms_per_step * 1e-3)
+
+    # ---- per-stage device times (events recorded by the library between its kernels) ----
+    names = binding.stage_names(binding.OP_FWD)
+    n_ev = len(names) + 1
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(args.steps)]
+    for row in evs:
+        for e in row:
+            e.record()
+    torch.cuda.synchronize()
+    for row in evs:
+        keep = binding.attach_stage_events(p, row)
+        step()
+        del keep
+    p.stage_events, p.n_stage_events = None, 0
+    torch.cuda.synchronize()
+    stage_ms = {nm: float(np.mean([row[i].elapsed_time(row[i + 1]) for row in evs]))
+                for i, nm in enumerate(names)}
+
+    # ---- end to end: pinned host buffers -> device -> layer -> host, every step ----
+    def e2e_step():
+        for n in devt:
+            devt[n].copy_(host[n], non_blocking=True)
+        step()
+        out_host.copy_(out, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    h2d = sum(host[n].numel() * host[n].element_size() for n in devt)
+    d2h = out_host.numel() * out_host.element_size()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel ----
+    peaks, peak_kind = load_peaks()
+    traffic = load_traffic()
+    flops = useful_flops(x["route"], d, wl.C)
+    dom = max((n for n in names if n in flops), key=lambda n: stage_ms[n])
+    tf = flops[dom] / (stage_ms[dom] * 1e-3) / 1e12
+    peak_tf = peaks["bf16_tflops_sustained"] if ms > 2000 else peaks["bf16_tflops"]
+    roofline = {"kernel": dom, "bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": tf / peak_tf, "peak_source": peak_kind,
+                "traffic": traffic.get(f"{dom}:{WORKLOAD}"),
+                "useful_flops_per_launch": flops[dom], "ms_per_launch": stage_ms[dom]}
+    total_flops = sum(flops.values())
+    step_tf = total_flops / (ms_per_step * 1e-3) / 1e12
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "B_per_gpu": B, "H": H, "L": L, "d": d, "C": wl.C,
+                   "p_softmax": wl.p_softmax, "sharding": "independent (batch, head) per GPU",
+                   "l2": "working set (q,k,v,out + workspace) > 126 MB L2; no flush between steps"},
+        "e2e": {"value": world * B * L / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "stages_ms": stage_ms,
+        "step": {"useful_tflops": step_tf, "frac_of_bf16_peak": step_tf / peak_tf,
+                 "useful_gflop": total_flops / 1e9, "min_hbm_bytes": min_hbm_bytes_fwd(wl, B),
+                 "hbm_floor_ms": min_hbm_bytes_fwd(wl, B) / (peaks["hbm_gbs"] * 1e9) * 1e3},
+    }
+
+    if world == 1 and not args.no_extras:
+        line["decode"] = bench_decode(args, peaks, peak_kind, traffic)
+    if world == 1 and not args.no_cpu:
+        xs = x if args.cpu_sample_B >= B else inputs.make_layer_inputs(wl_rank, B=args.cpu_sample_B)
+        sb = min(args.cpu_sample_B, B)
+        times, cores = time_oracle(wl, xs, 2)
+        line["cpu_baseline"] = {"value": sb * L / min(times), "unit": UNIT, "cores": cores,
+                                "kind": "oracle",
+                                "sample": f"{sb} of {B} sequences (all {H} heads, L={L}), best of 2"}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def bench_decode(args, peaks, peak_kind, traffic):
+    """Decode workload: batch 64, H=16, d=128, 256 steps, 1638 retained tokens per cache."""
+    import torch
+
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg3_bf16_decode"]
+    B, H, d, T = wl.B, wl.H, wl.d, wl.L
+    x = inputs.make_decode_inputs(wl)
+    dt = torch.bfloat16
+    state0 = torch.from_numpy(x["state"]).cuda()
+    state = state0.clone()
+    kc = torch.from_numpy(x["k_cache"]).to(dt).cuda()
+    vc = torch.from_numpy(x["v_cache"]).to(dt).cuda()
+    n0 = torch.from_numpy(x["cache_len"]).cuda()
+    n = n0.clone()
+    tok = {m: torch.from_numpy(x[m]).cuda() for m in ("g", "beta", "route", "w")}
+    for m in ("q", "k", "v"):
+        tok[m] = torch.from_numpy(x[m]).to(dt).cuda()
+    out = torch.empty((T, B, H, d), dtype=dt, device="cuda")
+    p = binding.make_params(B, H, 0, d, binding.NATSL_BF16, wl.scale_la, wl.scale_sm)
+    ws = binding.alloc_workspace(p, binding.OP_DECODE)
+
+    def trajectory():
+        for t in range(T):
+            p.w = tok["w"][t].data_ptr()
+            binding.natsl_decode_step(tok["q"][t], tok["k"][t], tok["v"][t], tok["g"][t],
+                                      tok["beta"][t], tok["route"][t], state, kc, vc, n, out[t], p, ws)
+
+    times = []
+    for rep in range(3):
+        state.copy_(state0)
+        n.copy_(n0)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        trajectory()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert binding.natsl_device_status(ws) == 0
+    ms = min(times[1:])
+    mean_len = float(x["cache_len"].mean()) + 0.5 * float(x["route"].mean()) * T
+    bytes_step = decode_bytes_per_step(B, H, d, mean_len)
+    gbs = bytes_step / (ms / T * 1e-3) / 1e9
+    return {"workload": wl.name, "value": B * T / (ms * 1e-3), "unit": "tokens/s",
+            "ms_per_step": ms / T, "steps": T,
+            "roofline": {"kernel": "decode_step", "bound": "hbm", "achieved": gbs,
+                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                         "peak_source": peak_kind, "algorithmic_bytes_per_launch": bytes_step,
+                         "traffic": traffic.get(f"decode_step:{wl.name}")}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the decode workload")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--cpu-sample-B", type=int, default=4)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -74,6 +74,9 @@ typedef struct natsl_params {
     void *k_sm, *v_sm;      /* optional compacted K/V of the retained tokens [B,H,sm_cap,d], */
     int32_t *sm_len;        /*   in `dtype`, with their counts [B,H]; all three or none.     */
     int32_t sm_cap;         /*   This is the decode cache layout (prefill -> decode handoff). */
+    void *const *stage_events; /* host array of cudaEvent_t owned by the caller, or NULL: the    */
+    int32_t n_stage_events;    /*   library records event[i] on `stream` before stage i and one  */
+                               /*   after the last stage (see natsl_stage_name); for profiling.  */
 } natsl_params;
 
 /* Bytes of workspace `op` needs for these shapes (host call, launches nothing). */
@@ -139,6 +142,13 @@ int natsl_decode_step(const void *q, const void *k, const void *v, const float *
 int natsl_device_status(void *ws, void *stream);
 
 const char *natsl_strerror(int status);
+
+/* Name of stage i of operation `op` (the interval between stage events i and i+1), or NULL
+ * when i is past the last stage.  Host call. */
+const char *natsl_stage_name(int op, int i);
+
+/* Number of kernels this library has launched in this process so far (host counter). */
+uint64_t natsl_launch_count(void);
 
 #ifdef __cplusplus
 }

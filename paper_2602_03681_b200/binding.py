@@ -20,7 +20,8 @@ FORCE_SIMT = 1
 ERR_CACHE_FULL = -7
 
 EXPORTS = ["natsl_workspace_size", "natsl_route_compact", "natsl_hybrid_fwd", "natsl_hybrid_bwd",
-           "natsl_decode_step", "natsl_device_status", "natsl_strerror"]
+           "natsl_decode_step", "natsl_device_status", "natsl_stage_name", "natsl_launch_count",
+           "natsl_strerror"]
 
 
 class NatslError(RuntimeError):
@@ -38,7 +39,8 @@ class natsl_params(ctypes.Structure):
                 ("state_out", ctypes.c_void_p), ("o_la", ctypes.c_void_p),
                 ("o_nla", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("k_sm", ctypes.c_void_p),
                 ("v_sm", ctypes.c_void_p), ("sm_len", ctypes.c_void_p),
-                ("sm_cap", ctypes.c_int32)]
+                ("sm_cap", ctypes.c_int32), ("stage_events", ctypes.c_void_p),
+                ("n_stage_events", ctypes.c_int32)]
 
 
 _lib = None
@@ -55,13 +57,42 @@ def lib() -> ctypes.CDLL:
         _lib = ctypes.CDLL(LIB_PATH)
         _lib.natsl_strerror.restype = ctypes.c_char_p
         _lib.natsl_strerror.argtypes = [ctypes.c_int]
-        for name in EXPORTS[:-1]:
+        _lib.natsl_stage_name.restype = ctypes.c_char_p
+        _lib.natsl_stage_name.argtypes = [ctypes.c_int, ctypes.c_int]
+        _lib.natsl_launch_count.restype = ctypes.c_uint64
+        for name in EXPORTS[:6]:
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
 
 def natsl_strerror(status: int) -> str:
     return lib().natsl_strerror(int(status)).decode()
+
+
+def natsl_stage_name(op: int, i: int):
+    s = lib().natsl_stage_name(op, i)
+    return None if s is None else s.decode()
+
+
+def natsl_launch_count() -> int:
+    return int(lib().natsl_launch_count())
+
+
+def stage_names(op: int):
+    names, i = [], 0
+    while natsl_stage_name(op, i) is not None:
+        names.append(natsl_stage_name(op, i))
+        i += 1
+    return names
+
+
+def attach_stage_events(p, events):
+    """Point p.stage_events at a list of recorded-once torch.cuda.Event(enable_timing=True).
+    Returns the ctypes array, which the caller must keep alive while `p` is used."""
+    arr = (ctypes.c_void_p * len(events))(*[ctypes.c_void_p(e.cuda_event) for e in events])
+    p.stage_events = ctypes.cast(arr, ctypes.c_void_p).value
+    p.n_stage_events = len(events)
+    return arr
 
 
 def _check(rc: int):

@@ -4,7 +4,14 @@
 
 #include "natsl_internal.h"
 
+#include <atomic>
+
 using namespace natsl;
+
+namespace natsl {
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+}  // namespace natsl
 
 namespace {
 
@@ -70,6 +77,16 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
 
 extern "C" {
 
+uint64_t natsl_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *natsl_stage_name(int op, int i) {
+    static const char *fwd[] = {"route_compact+gather_kv", "gdn_prepare", "gdn_scan",
+                                "softmax_combine"};
+    if (op == NATSL_OP_FWD && i >= 0 && i < 4) return fwd[i];
+    if (op == NATSL_OP_DECODE && i == 0) return "decode_step";
+    return nullptr;
+}
+
 const char *natsl_strerror(int status) {
     switch (status) {
         case NATSL_OK: return "ok";
@@ -125,19 +142,30 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     const Shape s = shape_of(p);
 
 #define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
+    int stage = 0;
+    auto mark = [&]() -> cudaError_t {
+        if (p->stage_events && stage < p->n_stage_events)
+            return cudaEventRecord(static_cast<cudaEvent_t>(p->stage_events[stage++]), st);
+        return cudaSuccess;
+    };
     NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
+    NATSL_TRY(mark());
     int32_t *sm_len = want_cache ? p->sm_len : f.sm_len;
     void *k_sm = want_cache ? p->k_sm : f.k_sm, *v_sm = want_cache ? p->v_sm : f.v_sm;
     const int32_t cap = want_cache ? p->sm_cap : p->L;
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, sm_len, p->B, p->L,
                                    p->H, st));
     NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
+    NATSL_TRY(mark());
     float *o_la = p->o_la ? p->o_la : f.o_la;
     NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P, s, st));
+    NATSL_TRY(mark());
     NATSL_TRY(launch_gdn_scan_simt(q, k, g, f.W, f.U, f.P, p->scale_la, p->state_in, p->state_out,
                                    nullptr, o_la, s, st));
+    NATSL_TRY(mark());
     NATSL_TRY(launch_softmax_combine_simt(q, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
                                           p->scale_sm, p->eps, out, p->o_nla, p->lse, s, st));
+    NATSL_TRY(mark());
 #undef NATSL_TRY
     return NATSL_OK;
 }

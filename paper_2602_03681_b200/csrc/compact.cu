@@ -125,6 +125,7 @@ cudaError_t launch_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t 
                                  int H, cudaStream_t st) {
     route_compact_kernel<<<B * H, kCompactThreads, 0, st>>>(route, sm_idx, sm_chunk_prefix, lin_idx,
                                                             n_lin, sm_len, L, H);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -137,6 +138,7 @@ static cudaError_t gather_impl(const void *k, const void *v, const int32_t *sm_i
     dim3 grid((max_rows + kRows - 1) / kRows, s.B * s.H);
     gather_kv_kernel<T, D><<<grid, 256, 0, st>>>((const T *)k, (const T *)v, sm_idx, pre, (T *)k_sm,
                                                  (T *)v_sm, cap, status, s.L, s.H);
+    count_launch();
     return cudaGetLastError();
 }
 

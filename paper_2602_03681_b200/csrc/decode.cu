@@ -245,6 +245,7 @@ static cudaError_t decode_impl(const void *q, const void *k, const void *v, cons
     decode_step_kernel<T, D><<<s.B * s.H, kThreads, 0, st>>>(
         (const T *)q, (const T *)k, (const T *)v, g, beta, route, w, state, (T *)k_cache,
         (T *)v_cache, cache_len, cap, (T *)out, scale_la, scale_sm, eps, status);
+    count_launch();
     return cudaGetLastError();
 }
 

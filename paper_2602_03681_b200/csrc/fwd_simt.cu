@@ -396,6 +396,7 @@ static cudaError_t prepare_impl(const void *q, const void *k, const void *v, con
     dim3 grid(s.L / kC, s.B * s.H);
     gdn_prepare_simt_kernel<T, D><<<grid, kThreads, smem, st>>>(
         (const T *)q, (const T *)k, (const T *)v, g, beta, route, scale_la, W, U, P, s.L, s.H);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -417,6 +418,7 @@ static cudaError_t scan_impl(const void *q, const void *k, const float *g, const
     gdn_scan_simt_kernel<T, D><<<grid, kThreads, smem, st>>>(
         (const T *)q, (const T *)k, g, W, U, P, scale_la, state_in, state_out, chunk_states, o_la,
         s.L, s.H);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -440,6 +442,7 @@ static cudaError_t softmax_impl(const void *q, const void *k_sm, const void *v_s
     softmax_combine_simt_kernel<T, D><<<grid, kThreads, smem, st>>>(
         (const T *)q, (const T *)k_sm, (const T *)v_sm, cap, sm_idx, pre, o_la, w, scale_sm, eps,
         (T *)out, o_nla, lse, s.L, s.H);
+    count_launch();
     return cudaGetLastError();
 }
 

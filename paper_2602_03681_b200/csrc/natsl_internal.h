@@ -10,6 +10,9 @@ namespace natsl {
 
 constexpr int kC = 64;  // chunk size (NAtS chunk = GDN chunk)
 
+// Every launch_* function calls this once per kernel it enqueues.
+void count_launch(int n = 1);
+
 struct Shape {
     int B, H, L, d;
     bool bf16;

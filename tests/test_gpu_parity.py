@@ -49,14 +49,36 @@ def run_oracle(wl, x, state_in=None, w="given", **kw):
                              scale_sm=wl.scale_sm, state_in=state_in, **kw)
 
 
+def half_ulp_bf16(x):
+    """Exact half unit-in-the-last-place of bf16 (8 significant bits) at |x|."""
+    x = np.abs(np.asarray(x, np.float64))
+    e = np.floor(np.log2(np.maximum(x, 2.0 ** -126)))
+    return 2.0 ** (e - 8)
+
+
+def check_stored(got, ref, tol, storage, name="out"):
+    """A tensor stored in the workload's storage type: the computed value must be within
+    tol * RMS of the oracle; storing it in bf16 adds at most half a bf16 ulp on top, which by
+    itself already exceeds 2e-2 * RMS for the few elements with |x| >= 4."""
+    ref = np.asarray(ref, np.float64)
+    err = np.abs(np.asarray(got, np.float64) - ref)
+    bound = tol * np.sqrt((ref ** 2).mean())
+    if storage == "bf16":
+        bound = bound + half_ulp_bf16(ref)
+    worst = (err / bound).max()
+    assert worst <= 1.0, (name, worst, rel_err(got, ref))
+
+
 def check_fwd(wl, got, ref, tol):
     lse_ok = np.isfinite(ref["lse"])
     assert np.array_equal(np.isneginf(got["lse"]), ~lse_ok)
-    assert np.abs(got["lse"][lse_ok] - ref["lse"][lse_ok]).max() <= max(tol, 1e-3) * 2
-    for name in ("o_la", "o_nla", "state_out", "out"):
+    if lse_ok.any():
+        assert np.abs(got["lse"][lse_ok] - ref["lse"][lse_ok]).max() <= max(tol, 1e-3) * 2
+    for name in ("o_la", "o_nla", "state_out"):       # fp32 tensors: no storage rounding
         if name in got:
             e = rel_err(got[name], ref[name])
             assert e <= tol, (name, e)
+    check_stored(got["out"], ref["out"], tol, wl.dtype)
 
 
 # ------------------------------------------------------------------ compaction (bit-exact)
@@ -105,7 +127,6 @@ def test_fwd_small_cases_simt(name, B, H, L):
     ref = run_oracle(wl, x, state_in=S0)
     # fp32 math throughout: only the bf16 rounding of `out` is left for bf16 storage
     check_fwd(wl, got, ref, 1e-4)
-    assert rel_err(got["out"], ref["out"]) <= (1e-4 if wl.dtype == "f32" else 1.2e-2)
 
 
 def test_fwd_degenerate_routes():
@@ -152,7 +173,6 @@ def run_decode(wl, B, H, steps, n0, cap=None):
     o_kc, o_vc = x["k_cache"].astype(np.float64), x["v_cache"].astype(np.float64)
     o_n = x["cache_len"].copy()
     tol = TOL[wl.dtype]
-    worst = 0.0
     for t in range(steps):
         w = dev(x["w"][t])
         p.w = w.data_ptr()
@@ -163,10 +183,9 @@ def run_decode(wl, B, H, steps, n0, cap=None):
         ref = oracle.decode_step(x["q"][t], x["k"][t], x["v"][t], x["g"][t], x["beta"][t],
                                  x["route"][t], x["w"][t], o_state, o_kc, o_vc, o_n,
                                  scale_la=wl.scale_la, scale_sm=wl.scale_sm)
-        worst = max(worst, rel_err(out.float().cpu().numpy(), ref["out"]))
+        check_stored(out.float().cpu().numpy(), ref["out"], tol, wl.dtype, f"step{t}")
     assert binding.natsl_device_status(ws) == 0
     assert np.array_equal(n.cpu().numpy(), o_n)
-    assert worst <= tol, worst
     assert rel_err(state.cpu().numpy(), o_state) <= 1e-4
     for b in range(B):
         for h in range(H):
