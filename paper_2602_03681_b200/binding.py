@@ -207,3 +207,18 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5,
     natsl_hybrid_fwd(q, k, v, g, beta, route, out, p, ws)
     res = dict(out=out, ws=ws, **opt)
     return res
+
+
+def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5, ws=None):
+    """Allocate gradients and run natsl_hybrid_bwd.  Returns dict(dq, dk, dv, dg, dbeta, dw, ws)."""
+    B, L, H, d = q.shape
+    dev = q.device
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    dg = torch.empty((B, L, H), dtype=torch.float32, device=dev)
+    dbeta = torch.empty((B, L, H), dtype=torch.float32, device=dev)
+    dw = torch.empty((B, L, H, 2), dtype=torch.float32, device=dev)
+    p = make_params(B, H, L, d, _dtype_code(q), scale_la, scale_sm, eps, w=w)
+    if ws is None:
+        ws = alloc_workspace(p, OP_BWD, dev)
+    natsl_hybrid_bwd(q, k, v, g, beta, route, dout, dq, dk, dv, dg, dbeta, dw, p, ws)
+    return dict(dq=dq, dk=dk, dv=dv, dg=dg, dbeta=dbeta, dw=dw, ws=ws)

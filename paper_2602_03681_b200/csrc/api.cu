@@ -73,6 +73,44 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
     return f;
 }
 
+struct BwdWs {
+    int32_t *status, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
+    float *k_sm32, *v_sm32;                                  // [B,H,L,d] compacted, fp32
+    float *q32, *k32, *v32;                                  // token-major fp32 copies
+    float *W, *U, *Ut, *o_la, *o_nla, *do_la, *do_nla;       // token-major
+    float *dUt, *dQg, *dW, *dKt, *dKb, *dVb, *X1p, *X2, *X3, *X4, *dq_sm, *dk_sm, *dv_sm;
+    float *P, *Abar, *M, *N, *Mg, *Ms, *Ns;                  // [B,H,NC,64,64]
+    float *S_c, *dS_c;                                       // [B,H,NC,d,d]
+    float *Gcum, *lse, *Dsm, *dGrow, *kappa, *gS;            // [B,H,L] (gS: [B,H,NC,d/32])
+    size_t bytes;
+};
+
+BwdWs carve_bwd(const natsl_params *p, void *ws) {
+    Carver c(ws);
+    BwdWs f;
+    const size_t B = p->B, H = p->H, L = p->L, d = p->d, NC = L / kC;
+    const size_t TM = B * L * H * d, CC = B * H * NC * kC * kC, ST = B * H * NC * d * d, BHL = B * H * L;
+    f.status = c.take<int32_t>(kStatusBytes / 4);
+    f.sm_idx = c.take<int32_t>(BHL);
+    f.prefix = c.take<int32_t>(B * H * (NC + 1));
+    f.lin_idx = c.take<int32_t>(BHL);
+    f.n_lin = c.take<int32_t>(B * H * NC);
+    f.sm_len = c.take<int32_t>(B * H);
+    float **tm[] = {&f.k_sm32, &f.v_sm32, &f.q32, &f.k32, &f.v32, &f.W, &f.U, &f.Ut, &f.o_la,
+                    &f.o_nla, &f.do_la, &f.do_nla, &f.dUt, &f.dQg, &f.dW, &f.dKt, &f.dKb, &f.dVb,
+                    &f.X1p, &f.X2, &f.X3, &f.X4, &f.dq_sm, &f.dk_sm, &f.dv_sm};
+    for (float **t : tm) *t = c.take<float>(TM);
+    float **cc[] = {&f.P, &f.Abar, &f.M, &f.N, &f.Mg, &f.Ms, &f.Ns};
+    for (float **t : cc) *t = c.take<float>(CC);
+    f.S_c = c.take<float>(ST);
+    f.dS_c = c.take<float>(ST);
+    float **sm[] = {&f.Gcum, &f.lse, &f.Dsm, &f.dGrow, &f.kappa};
+    for (float **t : sm) *t = c.take<float>(BHL);
+    f.gS = c.take<float>(B * H * NC * (d / 32));
+    f.bytes = c.off;
+    return f;
+}
+
 }  // namespace
 
 extern "C" {
@@ -108,6 +146,7 @@ int natsl_workspace_size(const natsl_params *p, int op, size_t *bytes) {
     if (rc != NATSL_OK) return rc;
     switch (op) {
         case NATSL_OP_FWD: *bytes = carve_fwd(p, nullptr).bytes; return NATSL_OK;
+        case NATSL_OP_BWD: *bytes = carve_bwd(p, nullptr).bytes; return NATSL_OK;
         case NATSL_OP_DECODE: *bytes = kStatusBytes; return NATSL_OK;
         case NATSL_OP_COMPACT: *bytes = 0; return NATSL_OK;
         default: return NATSL_ERR_UNSUPPORTED;
@@ -158,10 +197,11 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
     NATSL_TRY(mark());
     float *o_la = p->o_la ? p->o_la : f.o_la;
-    NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P, s, st));
+    NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P, nullptr,
+                                      nullptr, s, st));
     NATSL_TRY(mark());
     NATSL_TRY(launch_gdn_scan_simt(q, k, g, f.W, f.U, f.P, p->scale_la, p->state_in, p->state_out,
-                                   nullptr, o_la, s, st));
+                                   nullptr, nullptr, o_la, s, st));
     NATSL_TRY(mark());
     NATSL_TRY(launch_softmax_combine_simt(q, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
                                           p->scale_sm, p->eps, out, p->o_nla, p->lse, s, st));
@@ -170,10 +210,72 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     return NATSL_OK;
 }
 
-int natsl_hybrid_bwd(const void *, const void *, const void *, const float *, const float *,
-                     const uint8_t *, const void *, void *, void *, void *, float *, float *,
-                     float *, const natsl_params *, void *, size_t, void *) {
-    return NATSL_ERR_UNSUPPORTED;
+int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g,
+                     const float *beta, const uint8_t *route, const void *dout, void *dq, void *dk,
+                     void *dv, float *dg, float *dbeta, float *dw, const natsl_params *p, void *ws,
+                     size_t ws_bytes, void *stream) {
+    int rc = check_params(p, true);
+    if (rc != NATSL_OK) return rc;
+    if (!q || !k || !v || !g || !beta || !route || !dout || !dq || !dk || !dv || !dg || !dbeta)
+        return NATSL_ERR_NULL;
+    if (p->state_in) return NATSL_ERR_UNSUPPORTED;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) ||
+        !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
+        return NATSL_ERR_ALIGN;
+    BwdWs f = carve_bwd(p, ws);
+    if (!ws || ws_bytes < f.bytes) return NATSL_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const Shape s = shape_of(p);
+    Shape s32 = s;              // the same shapes with fp32 storage (the fp32 copies)
+    s32.bf16 = false;
+    const long long B = p->B, H = p->H, L = p->L, d = p->d, NC = L / kC;
+    (void)B;
+    auto TM = [&](const float *x) { return BMat{x, L * H * d, d, (long long)kC * H * d, (int)(H * d)}; };
+    auto CC = [&](const float *x) { return BMat{x, H * NC * kC * kC, NC * kC * kC, (long long)kC * kC, kC}; };
+    auto ST = [&](const float *x) { return BMat{x, H * NC * d * d, NC * d * d, d * d, (int)d}; };
+    const int di = p->d;
+
+#define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
+    NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
+    // ---- forward recomputation, keeping what the backward needs ----
+    NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, p->B,
+                                   p->L, p->H, st));
+    NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
+    NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L, f.status,
+                               s32, st));
+    NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
+                                      f.P, f.Abar, f.Gcum, s32, st));
+    NATSL_TRY(launch_gdn_scan_simt(f.q32, f.k32, g, f.W, f.U, f.P, p->scale_la, nullptr, nullptr,
+                                   f.S_c, f.Ut, f.o_la, s32, st));
+    NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
+                                          f.o_la, p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
+                                          s32, st));
+    // ---- combination and softmax branch ----
+    NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la, f.do_nla, dw, f.Dsm,
+                                 s, st));
+    NATSL_TRY(launch_softmax_bwd(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix, f.do_nla,
+                                 f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
+    // ---- linear branch: reverse scan, then chunk-parallel products ----
+    NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
+                               f.dS_c, f.gS, s, st));
+    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, s, st));
+    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, s, st));
+    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, s, st));
+    NATSL_TRY(launch_bgemm(false, true, 1, TM(f.do_la), TM(f.Ut), CC(f.N), kC, kC, di, 1.f, false, s, st));
+    NATSL_TRY(launch_gdn_tsolve(f.Abar, beta, route, f.dW, f.dUt, f.dKb, f.dVb, s, st));
+    NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dKb), TM(f.W), CC(f.M), kC, kC, di, -1.f, false, s, st));
+    NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dVb), TM(f.U), CC(f.M), kC, kC, di, -1.f, true, s, st));
+    NATSL_TRY(launch_mask_scale(f.M, f.N, f.Gcum, beta, route, p->scale_la, f.Mg, f.Ms, f.Ns, s, st));
+    NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Mg), TM(f.k32), TM(f.X1p), kC, di, kC, 1.f, false, s, st));
+    NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ms), TM(f.k32), TM(f.X2), kC, di, kC, 1.f, false, s, st));
+    NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Ns), TM(f.k32), TM(f.X3), kC, di, kC, 1.f, false, s, st));
+    NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ns), TM(f.q32), TM(f.X4), kC, di, kC, 1.f, false, s, st));
+    AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
+                   f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
+                   p->scale_la, f.dGrow, f.kappa, dbeta, dg};
+    NATSL_TRY(launch_gdn_assemble(a, dq, dk, dv, s, st));
+#undef NATSL_TRY
+    return NATSL_OK;
 }
 
 int natsl_decode_step(const void *q, const void *k, const void *v, const float *g,

@@ -1,0 +1,830 @@
+// fp32 CUDA-core backward of the hybrid layer.
+//
+// The paper states the properties the backward must have (Section 4.2: the softmax logit
+// gradient is P (dP - <do, o>); k, v gradients of an operation vanish for tokens inactive for
+// it) but gives no backward of the gated delta rule.  This file differentiates the chunkwise
+// forward of fwd_simt.cu.  Per chunk, with entry state S0, exit-state gradient dS1, output
+// gradient dO and the forward quantities W, U, P, U~ (same notation as fwd_simt.cu):
+//
+//   dU~ = P^T dO + K~ dS1                       K~ = diag(gamma_C / gamma) K
+//   dS0 = Qg^T dO + gamma_C dS1 - W^T dU~       Qg = scale_la diag(gamma) Q      (reverse scan)
+//   dQg = dO S0^T     dW = -dU~ S0^T     dK~ = U~ dS1^T     N = lower(dO U~^T)
+//   [dKb | dVb] = (I + A)^-T [dW | dU~]         Kb = diag(beta~ gamma) K, Vb = diag(beta~) V
+//   M  = -strict_lower(dKb W^T + dVb U^T)       (gradient w.r.t. A)
+//   dq = scale_la gamma dQg + (N . scale_la Gamma) K
+//   dk = beta~ gamma dKb + (gamma_C/gamma) dK~ + (M . beta~ Gamma) K + (M . beta~ Gamma)^T K
+//        + (N . scale_la Gamma)^T Q
+//   dv = beta~ dVb
+//   every gamma / Gamma factor contributes to dG_i (G = in-chunk cumulative log decay), and
+//   dg_j = sum_{i >= j} dG_i;  dbeta = (1 - route) dbeta~.
+//
+// The dense products run through one generic batched tile-GEMM kernel over (batch, head,
+// chunk); the sequential part is the reverse scan.  Softmax-branch gradients are formed over
+// the compacted K/V list only and scattered back to the retained tokens.
+#include "common.cuh"
+#include "natsl_internal.h"
+
+namespace natsl {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// ------------------------------------------------------------------------------------------
+// generic batched GEMM: C = alpha * op(A) op(B) (+ C), 64x64 output tiles, fp32
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ const float *mat_base(const BMat &m, int b, int h, int ch) {
+    return m.p + (size_t)b * m.sb + (size_t)h * m.sh + (size_t)ch * m.sc;
+}
+
+template <bool TA, bool TB, int MASK>
+__global__ void __launch_bounds__(kThreads)
+bgemm_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H, int NC) {
+    __shared__ __align__(16) float As[16][68];
+    __shared__ __align__(16) float Bs[16][68];
+    const int z = blockIdx.z, ch = z % NC, bh = z / NC, b = bh / H, h = bh % H;
+    const float *Ap = mat_base(A, b, h, ch), *Bp = mat_base(B, b, h, ch);
+    float *Cp = const_cast<float *>(mat_base(Cm, b, h, ch));
+    const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+    const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < K; k0 += 16) {
+        if (!TA) {   // A[m][k], k contiguous
+            const int r = t >> 2, kk = (t & 3) * 4;
+            const float4 x = *reinterpret_cast<const float4 *>(Ap + (size_t)(m0 + r) * A.ld + k0 + kk);
+            As[kk][r] = x.x; As[kk + 1][r] = x.y; As[kk + 2][r] = x.z; As[kk + 3][r] = x.w;
+        } else {     // A[k][m], m contiguous
+            const int kk = t >> 4, r4 = (t & 15) * 4;
+            *reinterpret_cast<float4 *>(&As[kk][r4]) =
+                *reinterpret_cast<const float4 *>(Ap + (size_t)(k0 + kk) * A.ld + m0 + r4);
+        }
+        if (!TB) {   // B[k][n], n contiguous
+            const int kk = t >> 4, c4 = (t & 15) * 4;
+            *reinterpret_cast<float4 *>(&Bs[kk][c4]) =
+                *reinterpret_cast<const float4 *>(Bp + (size_t)(k0 + kk) * B.ld + n0 + c4);
+        } else {     // B[n][k], k contiguous
+            const int c = t >> 2, kk = (t & 3) * 4;
+            const float4 x = *reinterpret_cast<const float4 *>(Bp + (size_t)(n0 + c) * B.ld + k0 + kk);
+            Bs[kk][c] = x.x; Bs[kk + 1][c] = x.y; Bs[kk + 2][c] = x.z; Bs[kk + 3][c] = x.w;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            const float4 a = *reinterpret_cast<const float4 *>(&As[kk][ty * 4]);
+            const float4 bb = *reinterpret_cast<const float4 *>(&Bs[kk][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = m0 + ty * 4 + i;
+        float *cr = Cp + (size_t)row * Cm.ld + n0 + tx * 4;
+        float o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int col = n0 + tx * 4 + j;
+            float val = alpha * acc[i][j];
+            if (MASK == 1 && col > row) val = 0.f;
+            if (MASK == 2 && col >= row) val = 0.f;
+            o[j] = val;
+        }
+        if (accumulate) {
+            const float4 old = *reinterpret_cast<const float4 *>(cr);
+            o[0] += old.x; o[1] += old.y; o[2] += old.z; o[3] += old.w;
+        }
+        *reinterpret_cast<float4 *>(cr) = make_float4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// storage type -> fp32 copies of q, k, v
+// ------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void to_f32_kernel(const T *__restrict__ a, const T *__restrict__ b, const T *__restrict__ c,
+                              float *__restrict__ a32, float *__restrict__ b32,
+                              float *__restrict__ c32, size_t n4) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
+         i += (size_t)gridDim.x * blockDim.x) {
+        store4(a32 + 4 * i, load4(a + 4 * i));
+        store4(b32 + 4 * i, load4(b + 4 * i));
+        store4(c32 + 4 * i, load4(c + 4 * i));
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// combination backward (row-local): do_la, do_nla, dw, Dsm = <do_nla, o_nla>
+// one warp per (token, head) row
+// ------------------------------------------------------------------------------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads)
+combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_nla,
+                   const T *__restrict__ dout, const float *__restrict__ w, float eps,
+                   float *__restrict__ do_la, float *__restrict__ do_nla, float *__restrict__ dw,
+                   float *__restrict__ Dsm, int B, int L, int H) {
+    constexpr int kCols = D / 32;
+    const int lane = threadIdx.x & 31;
+    const size_t row = (size_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (row >= (size_t)B * L * H) return;
+    const int h = row % H;
+    const size_t bl = row / H;
+    const int l = bl % L, b = bl / L;
+    float ol[kCols], on[kCols], dy[kCols], ssl = 0.f, ssn = 0.f;
+#pragma unroll
+    for (int x = 0; x < kCols; ++x) {
+        const size_t i = row * D + lane + 32 * x;
+        ol[x] = o_la[i]; on[x] = o_nla[i]; dy[x] = to_f32(dout[i]);
+        ssl = fmaf(ol[x], ol[x], ssl);
+        ssn = fmaf(on[x], on[x], ssn);
+    }
+    ssl = warp_sum(ssl); ssn = warp_sum(ssn);
+    const float fl = rsqrtf(ssl / D + eps), fn = rsqrtf(ssn / D + eps);
+    const float wn = w ? w[row * 2] : 0.5f, wl = w ? w[row * 2 + 1] : 0.5f;
+    float dwl = 0.f, dwn = 0.f;
+#pragma unroll
+    for (int x = 0; x < kCols; ++x) {
+        dwl = fmaf(dy[x], ol[x] * fl, dwl);
+        dwn = fmaf(dy[x], on[x] * fn, dwn);
+    }
+    dwl = warp_sum(dwl); dwn = warp_sum(dwn);
+    const float ml = wl * dwl / D, mn = wn * dwn / D;
+    float dsm = 0.f;
+#pragma unroll
+    for (int x = 0; x < kCols; ++x) {
+        const size_t i = row * D + lane + 32 * x;
+        const float dl = fl * (wl * dy[x] - ol[x] * fl * ml);
+        const float dn = fn * (wn * dy[x] - on[x] * fn * mn);
+        do_la[i] = dl;
+        do_nla[i] = dn;
+        dsm = fmaf(dn, on[x], dsm);
+    }
+    dsm = warp_sum(dsm);
+    if (lane == 0) {
+        if (dw) { dw[row * 2] = dwn; dw[row * 2 + 1] = dwl; }
+        Dsm[((size_t)b * H + h) * L + l] = dsm;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// softmax backward, query side: dq_sm.  grid = (L/64, B*H), same tiling as the forward.
+// ------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+softmax_bwd_dq_kernel(const float *__restrict__ q32, const float *__restrict__ k_sm32,
+                      const float *__restrict__ v_sm32, int cap, const int32_t *__restrict__ sm_idx,
+                      const int32_t *__restrict__ sm_chunk_prefix,
+                      const float *__restrict__ do_nla, const float *__restrict__ lse,
+                      const float *__restrict__ Dsm, float scale_sm, float *__restrict__ dq_sm,
+                      int L, int H) {
+    extern __shared__ float smem[];
+    float *Qs = smem;                      // [64][D]
+    float *dOs = Qs + kC * D;              // [64][D]
+    float *Kt = dOs + kC * D;              // [32][D+1]
+    float *Vt = Kt + 32 * (D + 1);         // [32][D+1]
+    int *pos = reinterpret_cast<int *>(Vt + 32 * (D + 1));
+
+    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int NC = L / kC;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t ts = (size_t)H * D;
+    const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
+    const int n_end = min(sm_chunk_prefix[(size_t)bh * (NC + 1) + c + 1], cap);
+
+    for (int idx = threadIdx.x; idx < kC * D / 4; idx += kThreads) {
+        const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
+        store4(Qs + r * D + c4, load4(q32 + tok0 * D + (size_t)r * ts + c4));
+        store4(dOs + r * D + c4, load4(do_nla + tok0 * D + (size_t)r * ts + c4));
+    }
+    constexpr int kQ = 8, kCols = D / 32;
+    float acc[kQ][kCols], lse_r[kQ], dsm_r[kQ];
+#pragma unroll
+    for (int r = 0; r < kQ; ++r) {
+        const int i = c * kC + warp * kQ + r;
+        lse_r[r] = lse[(size_t)bh * L + i];
+        dsm_r[r] = Dsm[(size_t)bh * L + i];
+#pragma unroll
+        for (int x = 0; x < kCols; ++x) acc[r][x] = 0.f;
+    }
+    const float *kb = k_sm32 + (size_t)bh * cap * D, *vb = v_sm32 + (size_t)bh * cap * D;
+    for (int j0 = 0; j0 < n_end; j0 += 32) {
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < 32 * D / 4; idx += kThreads) {
+            const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
+            float4 kx = make_float4(0.f, 0.f, 0.f, 0.f), vx = kx;
+            if (j0 + r < n_end) {
+                kx = load4(kb + (size_t)(j0 + r) * D + c4);
+                vx = load4(vb + (size_t)(j0 + r) * D + c4);
+            }
+            float *kp = Kt + r * (D + 1) + c4, *vp = Vt + r * (D + 1) + c4;
+            kp[0] = kx.x; kp[1] = kx.y; kp[2] = kx.z; kp[3] = kx.w;
+            vp[0] = vx.x; vp[1] = vx.y; vp[2] = vx.z; vp[3] = vx.w;
+        }
+        if (threadIdx.x < 32)
+            pos[threadIdx.x] = (j0 + threadIdx.x < n_end) ? sm_idx[(size_t)bh * L + j0 + threadIdx.x]
+                                                          : 0x7fffffff;
+        __syncthreads();
+        const int my_pos = pos[lane];
+        const float *kr = Kt + lane * (D + 1), *vr = Vt + lane * (D + 1);
+#pragma unroll
+        for (int r = 0; r < kQ; ++r) {
+            const int i = c * kC + warp * kQ + r;
+            const float *qr = Qs + (warp * kQ + r) * D, *dor = dOs + (warp * kQ + r) * D;
+            float s = 0.f, dp = 0.f;
+#pragma unroll 8
+            for (int x = 0; x < D; ++x) {
+                s = fmaf(qr[x], kr[x], s);
+                dp = fmaf(dor[x], vr[x], dp);
+            }
+            const float pj = (my_pos <= i) ? __expf(s * scale_sm - lse_r[r]) : 0.f;
+            const float ds = pj * (dp - dsm_r[r]);
+            for (int j = 0; j < 32; ++j) {
+                const float db = __shfl_sync(0xffffffffu, ds, j);
+#pragma unroll
+                for (int x = 0; x < kCols; ++x)
+                    acc[r][x] = fmaf(db, Kt[j * (D + 1) + lane + 32 * x], acc[r][x]);
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < kQ; ++r) {
+        const size_t t = tok0 + (size_t)(warp * kQ + r) * H;
+#pragma unroll
+        for (int x = 0; x < kCols; ++x) dq_sm[t * D + lane + 32 * x] = scale_sm * acc[r][x];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// softmax backward, key side: dk_sm, dv_sm per compacted key.  grid = (ceil(cap/32), B*H).
+// ------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ k_sm32,
+                       const float *__restrict__ v_sm32, int cap, const int32_t *__restrict__ sm_idx,
+                       const int32_t *__restrict__ sm_chunk_prefix,
+                       const float *__restrict__ do_nla, const float *__restrict__ lse,
+                       const float *__restrict__ Dsm, float scale_sm, float *__restrict__ dk_sm,
+                       float *__restrict__ dv_sm, int L, int H) {
+    extern __shared__ float smem[];
+    float *Kt = smem;                       // [32][D+1]
+    float *Vt = Kt + 32 * (D + 1);          // [32][D+1]
+    float *Qs = Vt + 32 * (D + 1);          // [64][D]
+    float *dOs = Qs + kC * D;               // [64][D]
+    float *Ps = dOs + kC * D;               // [64][33]
+    float *Dss = Ps + kC * 33;              // [64][33]
+    float *lse_s = Dss + kC * 33;           // [64]
+    float *dsm_s = lse_s + kC;              // [64]
+    int *pos = reinterpret_cast<int *>(dsm_s + kC);
+
+    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int NC = L / kC;
+    const int n_sm = min(sm_chunk_prefix[(size_t)bh * (NC + 1) + NC], cap);
+    const int j0 = blockIdx.x * 32;
+    if (j0 >= n_sm) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const size_t ts = (size_t)H * D;
+    const float *kb = k_sm32 + (size_t)bh * cap * D, *vb = v_sm32 + (size_t)bh * cap * D;
+
+    for (int idx = threadIdx.x; idx < 32 * D / 4; idx += kThreads) {
+        const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
+        float4 kx = make_float4(0.f, 0.f, 0.f, 0.f), vx = kx;
+        if (j0 + r < n_sm) {
+            kx = load4(kb + (size_t)(j0 + r) * D + c4);
+            vx = load4(vb + (size_t)(j0 + r) * D + c4);
+        }
+        float *kp = Kt + r * (D + 1) + c4, *vp = Vt + r * (D + 1) + c4;
+        kp[0] = kx.x; kp[1] = kx.y; kp[2] = kx.z; kp[3] = kx.w;
+        vp[0] = vx.x; vp[1] = vx.y; vp[2] = vx.z; vp[3] = vx.w;
+    }
+    if (threadIdx.x < 32)
+        pos[threadIdx.x] = (j0 + threadIdx.x < n_sm) ? sm_idx[(size_t)bh * L + j0 + threadIdx.x]
+                                                     : 0x7fffffff;
+    __syncthreads();
+    const int my_pos = pos[lane];
+    const int c_first = pos[0] / kC;
+    constexpr int kPer = D / 8;
+    const int kj = threadIdx.x >> 3, cs = threadIdx.x & 7;
+    float adk[kPer], adv[kPer];
+#pragma unroll
+    for (int x = 0; x < kPer; ++x) { adk[x] = 0.f; adv[x] = 0.f; }
+
+    for (int c = c_first; c < NC; ++c) {
+        const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < kC * D / 4; idx += kThreads) {
+            const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
+            store4(Qs + r * D + c4, load4(q32 + tok0 * D + (size_t)r * ts + c4));
+            store4(dOs + r * D + c4, load4(do_nla + tok0 * D + (size_t)r * ts + c4));
+        }
+        if (threadIdx.x < kC) {
+            lse_s[threadIdx.x] = lse[(size_t)bh * L + c * kC + threadIdx.x];
+            dsm_s[threadIdx.x] = Dsm[(size_t)bh * L + c * kC + threadIdx.x];
+        }
+        __syncthreads();
+        const float *kr = Kt + lane * (D + 1), *vr = Vt + lane * (D + 1);
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const int il = warp * 8 + r, i = c * kC + il;
+            const float *qr = Qs + il * D, *dor = dOs + il * D;
+            float s = 0.f, dp = 0.f;
+#pragma unroll 8
+            for (int x = 0; x < D; ++x) {
+                s = fmaf(qr[x], kr[x], s);
+                dp = fmaf(dor[x], vr[x], dp);
+            }
+            const float pj = (my_pos <= i) ? __expf(s * scale_sm - lse_s[il]) : 0.f;
+            Ps[il * 33 + lane] = pj;
+            Dss[il * 33 + lane] = pj * (dp - dsm_s[il]);
+        }
+        __syncthreads();
+        for (int il = 0; il < kC; ++il) {
+            const float pj = Ps[il * 33 + kj], ds = Dss[il * 33 + kj];
+            const float *dor = dOs + il * D + cs, *qr = Qs + il * D + cs;
+#pragma unroll
+            for (int x = 0; x < kPer; ++x) {
+                adv[x] = fmaf(pj, dor[8 * x], adv[x]);
+                adk[x] = fmaf(ds, qr[8 * x], adk[x]);
+            }
+        }
+    }
+    if (j0 + kj < n_sm) {
+        float *dkr = dk_sm + ((size_t)bh * cap + j0 + kj) * D + cs;
+        float *dvr = dv_sm + ((size_t)bh * cap + j0 + kj) * D + cs;
+#pragma unroll
+        for (int x = 0; x < kPer; ++x) { dkr[8 * x] = scale_sm * adk[x]; dvr[8 * x] = adv[x]; }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// reverse scan over chunks: dU~ (stored), chunk-exit dS (stored), <dS1, S0> partials.
+// grid = (D/32, B*H), mirrors gdn_scan_simt_kernel.
+// ------------------------------------------------------------------------------------------
+constexpr int kDvs = 32;
+
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+gdn_rscan_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
+                 const float *__restrict__ Gcum, const float *__restrict__ W,
+                 const float *__restrict__ P, const float *__restrict__ do_la,
+                 const float *__restrict__ chunk_states, float scale_la, float *__restrict__ dUt,
+                 float *__restrict__ dS_c, float *__restrict__ gS, int L, int H) {
+    extern __shared__ float smem[];
+    float *dSs = smem;                       // [D][32]
+    float *Ws = dSs + D * kDvs;              // [64][D+1]
+    float *Qs = Ws + kC * (D + 1);           // [64][D+1]
+    float *Ks = Qs + kC * (D + 1);           // [64][D+1]
+    float *Ps = Ks + kC * (D + 1);           // [64][65]
+    float *dOs = Ps + kC * (kC + 1);         // [64][33]
+    float *dUs = dOs + kC * (kDvs + 1);      // [64][33]
+    float *Gs = dUs + kC * (kDvs + 1);       // [64]
+    float *red = Gs + kC;                    // [8]
+
+    const int slice = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int NC = L / kC;
+    const size_t ts = (size_t)H * D;
+    const int c0 = slice * kDvs;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    for (int idx = threadIdx.x; idx < D * kDvs; idx += kThreads) dSs[idx] = 0.f;
+
+    for (int c = NC - 1; c >= 0; --c) {
+        const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
+        __syncthreads();
+        // store the chunk-exit gradient and the partial <dS1, S0>
+        {
+            float part = 0.f;
+            for (int idx = threadIdx.x; idx < D * kDvs; idx += kThreads) {
+                const int a = idx / kDvs, cc = idx % kDvs;
+                const size_t gi = (((size_t)bh * NC + c) * D + a) * D + c0 + cc;
+                dS_c[gi] = dSs[idx];
+                part = fmaf(dSs[idx], chunk_states[gi], part);
+            }
+            part = warp_sum(part);
+            if (lane == 0) red[warp] = part;
+        }
+        for (int idx = threadIdx.x; idx < kC * D / 4; idx += kThreads) {
+            const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
+            const float4 wv = load4(W + tok0 * D + (size_t)r * ts + c4);
+            const float4 qv = load4(q32 + tok0 * D + (size_t)r * ts + c4);
+            const float4 kv = load4(k32 + tok0 * D + (size_t)r * ts + c4);
+            float *wp = Ws + r * (D + 1) + c4, *qp = Qs + r * (D + 1) + c4, *kp = Ks + r * (D + 1) + c4;
+            wp[0] = wv.x; wp[1] = wv.y; wp[2] = wv.z; wp[3] = wv.w;
+            qp[0] = qv.x; qp[1] = qv.y; qp[2] = qv.z; qp[3] = qv.w;
+            kp[0] = kv.x; kp[1] = kv.y; kp[2] = kv.z; kp[3] = kv.w;
+        }
+        {
+            const float *Pc = P + ((size_t)bh * NC + c) * kC * kC;
+            for (int idx = threadIdx.x; idx < kC * kC; idx += kThreads)
+                Ps[(idx >> 6) * (kC + 1) + (idx & 63)] = Pc[idx];
+            for (int idx = threadIdx.x; idx < kC * kDvs; idx += kThreads) {
+                const int r = idx / kDvs, cc = idx % kDvs;
+                dOs[r * (kDvs + 1) + cc] = do_la[(tok0 + (size_t)r * H) * D + c0 + cc];
+            }
+            if (threadIdx.x < kC) Gs[threadIdx.x] = Gcum[(size_t)bh * L + c * kC + threadIdx.x];
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float tot = 0.f;
+            for (int wv = 0; wv < kThreads / 32; ++wv) tot += red[wv];
+            gS[((size_t)bh * NC + c) * (D / kDvs) + slice] = tot;
+        }
+        const float gl = Gs[kC - 1];
+        const int r = threadIdx.x >> 2, cb = (threadIdx.x & 3) * 8;
+        // dU~_r = sum_{i>=r} P[i][r] dO_i + (gamma_C/gamma_r) k_r dS
+        {
+            float acc[8], acc2[8];
+#pragma unroll
+            for (int x = 0; x < 8; ++x) { acc[x] = 0.f; acc2[x] = 0.f; }
+            for (int i = r; i < kC; ++i) {
+                const float pv = Ps[i * (kC + 1) + r];
+                const float *dr = dOs + i * (kDvs + 1) + cb;
+#pragma unroll
+                for (int x = 0; x < 8; ++x) acc[x] = fmaf(pv, dr[x], acc[x]);
+            }
+            const float *kr = Ks + r * (D + 1);
+            for (int a = 0; a < D; ++a) {
+                const float kv = kr[a];
+                const float *sr = dSs + a * kDvs + cb;
+#pragma unroll
+                for (int x = 0; x < 8; ++x) acc2[x] = fmaf(kv, sr[x], acc2[x]);
+            }
+            const float kt = __expf(gl - Gs[r]);
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+                acc[x] = fmaf(kt, acc2[x], acc[x]);
+                dUs[r * (kDvs + 1) + cb + x] = acc[x];
+            }
+            float *dst = dUt + (tok0 + (size_t)r * H) * D + c0 + cb;
+            store4(dst, make_float4(acc[0], acc[1], acc[2], acc[3]));
+            store4(dst + 4, make_float4(acc[4], acc[5], acc[6], acc[7]));
+        }
+        __syncthreads();
+        // dS0 = Qg^T dO + gamma_C dS1 - W^T dU~
+        {
+            constexpr int kPer = D / 8, kTpr = kDvs / kPer;
+            const int a = threadIdx.x / kTpr, cs = (threadIdx.x % kTpr) * kPer;
+            const float gC = __expf(gl);
+            float acc[kPer];
+#pragma unroll
+            for (int x = 0; x < kPer; ++x) acc[x] = gC * dSs[a * kDvs + cs + x];
+            for (int i = 0; i < kC; ++i) {
+                const float qg = scale_la * __expf(Gs[i]) * Qs[i * (D + 1) + a];
+                const float wv = Ws[i * (D + 1) + a];
+                const float *dor = dOs + i * (kDvs + 1) + cs, *dur = dUs + i * (kDvs + 1) + cs;
+#pragma unroll
+                for (int x = 0; x < kPer; ++x) acc[x] = fmaf(qg, dor[x], fmaf(-wv, dur[x], acc[x]));
+            }
+            __syncthreads();
+#pragma unroll
+            for (int x = 0; x < kPer; ++x) dSs[a * kDvs + cs + x] = acc[x];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// transposed triangular solve: [dKb | dVb] = (I + A)^-T [dW | dU~], A = diag(beta~) Abar.
+// grid = (L/C, B*H); one right-hand-side column per thread.
+// ------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+gdn_tsolve_kernel(const float *__restrict__ Abar, const float *__restrict__ beta,
+                  const uint8_t *__restrict__ route, const float *__restrict__ dW,
+                  const float *__restrict__ dUt, float *__restrict__ dKb, float *__restrict__ dVb,
+                  int L, int H) {
+    __shared__ float As[kC * kC];
+    __shared__ float bts[kC];
+    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    const size_t ts = (size_t)H * D;
+    const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
+    if (threadIdx.x < kC) {
+        const size_t t = tok0 + (size_t)threadIdx.x * H;
+        bts[threadIdx.x] = route[t] ? 0.f : beta[t];
+    }
+    __syncthreads();
+    const float *Ab = Abar + ((size_t)bh * (L / kC) + c) * kC * kC;
+    for (int idx = threadIdx.x; idx < kC * kC; idx += kThreads) As[idx] = bts[idx >> 6] * Ab[idx];
+    __syncthreads();
+    if (threadIdx.x < 2 * D) {
+        const bool first = threadIdx.x < D;
+        const int col = first ? threadIdx.x : threadIdx.x - D;
+        const float *src = (first ? dW : dUt) + tok0 * D + col;
+        float x[kC];
+#pragma unroll
+        for (int i = kC - 1; i >= 0; --i) {
+            float acc = src[(size_t)i * ts];
+#pragma unroll
+            for (int j = i + 1; j < kC; ++j) acc = fmaf(-As[j * kC + i], x[j], acc);
+            x[i] = acc;
+        }
+        float *dst = (first ? dKb : dVb) + tok0 * D + col;
+#pragma unroll
+        for (int i = 0; i < kC; ++i) dst[(size_t)i * ts] = x[i];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Mg = M . Gamma, Ms = diag(beta~) Mg, Ns = scale_la N . Gamma    (all 64x64 per chunk)
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+mask_scale_kernel(const float *__restrict__ M, const float *__restrict__ N,
+                  const float *__restrict__ Gcum, const float *__restrict__ beta,
+                  const uint8_t *__restrict__ route, float scale_la, float *__restrict__ Mg,
+                  float *__restrict__ Ms, float *__restrict__ Ns, int L, int H) {
+    __shared__ float Gs[kC], bts[kC];
+    const int NC = L / kC;
+    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    if (threadIdx.x < kC) {
+        const size_t t = ((size_t)b * L + (size_t)c * kC + threadIdx.x) * H + h;
+        bts[threadIdx.x] = route[t] ? 0.f : beta[t];
+        Gs[threadIdx.x] = Gcum[(size_t)bh * L + c * kC + threadIdx.x];
+    }
+    __syncthreads();
+    const size_t base = ((size_t)bh * NC + c) * kC * kC;
+    for (int idx = threadIdx.x; idx < kC * kC; idx += kThreads) {
+        const int i = idx >> 6, j = idx & 63;
+        const float gam = j <= i ? __expf(Gs[i] - Gs[j]) : 0.f;
+        const float mg = M[base + idx] * gam;
+        Mg[base + idx] = mg;
+        Ms[base + idx] = bts[i] * mg;
+        Ns[base + idx] = scale_la * N[base + idx] * gam;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// assembly: dq (all tokens), dk/dv (linear tokens), per-row dG, kappa, dbeta.
+// one warp per (token, head) row.
+// ------------------------------------------------------------------------------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads)
+gdn_assemble_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
+                    const float *__restrict__ v32, const float *__restrict__ Gcum,
+                    const float *__restrict__ beta, const uint8_t *__restrict__ route,
+                    const float *__restrict__ dQg, const float *__restrict__ dKb,
+                    const float *__restrict__ dVb, const float *__restrict__ dKt,
+                    const float *__restrict__ X1p, const float *__restrict__ X2,
+                    const float *__restrict__ X3, const float *__restrict__ X4,
+                    const float *__restrict__ dq_sm, float scale_la, T *__restrict__ dq,
+                    T *__restrict__ dk, T *__restrict__ dv, float *__restrict__ dGrow,
+                    float *__restrict__ kappa, float *__restrict__ dbeta, int B, int L, int H) {
+    constexpr int kCols = D / 32;
+    const int lane = threadIdx.x & 31;
+    const size_t row = (size_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    if (row >= (size_t)B * L * H) return;
+    const int h = row % H;
+    const size_t bl = row / H;
+    const int l = bl % L, b = bl / L;
+    const size_t bhl = ((size_t)b * H + h) * L;
+    const float Gi = Gcum[bhl + l], GC = Gcum[bhl + (l | (kC - 1))];
+    const bool lin = route[row] == 0;
+    const float bt = lin ? beta[row] : 0.f;
+    const float gam = __expf(Gi), kt = __expf(GC - Gi);
+    float kdKb = 0.f, qdQg = 0.f, kdKt = 0.f, kX1 = 0.f, kX2 = 0.f, qX3 = 0.f, kX4 = 0.f, vdVb = 0.f;
+#pragma unroll
+    for (int x = 0; x < kCols; ++x) {
+        const size_t i = row * D + lane + 32 * x;
+        const float qv = q32[i], kv = k32[i], vv = v32[i];
+        const float a_dQg = dQg[i], a_dKb = dKb[i], a_dVb = dVb[i], a_dKt = dKt[i];
+        const float x1 = X1p[i], x2 = X2[i], x3 = X3[i], x4 = X4[i];
+        kdKb = fmaf(kv, a_dKb, kdKb); qdQg = fmaf(qv, a_dQg, qdQg); kdKt = fmaf(kv, a_dKt, kdKt);
+        kX1 = fmaf(kv, x1, kX1); kX2 = fmaf(kv, x2, kX2); qX3 = fmaf(qv, x3, qX3);
+        kX4 = fmaf(kv, x4, kX4); vdVb = fmaf(vv, a_dVb, vdVb);
+        dq[i] = from_f32<T>(scale_la * gam * a_dQg + x3 + dq_sm[i]);
+        if (lin) {
+            dk[i] = from_f32<T>(bt * gam * a_dKb + kt * a_dKt + bt * x1 + x2 + x4);
+            dv[i] = from_f32<T>(bt * a_dVb);
+        }
+    }
+    kdKb = warp_sum(kdKb); qdQg = warp_sum(qdQg); kdKt = warp_sum(kdKt); kX1 = warp_sum(kX1);
+    kX2 = warp_sum(kX2); qX3 = warp_sum(qX3); kX4 = warp_sum(kX4); vdVb = warp_sum(vdVb);
+    if (lane == 0) {
+        const float kap = kt * kdKt;
+        dGrow[bhl + l] = bt * gam * kdKb + scale_la * gam * qdQg - kap + bt * kX1 - kX2 + qX3 - kX4;
+        kappa[bhl + l] = kap;
+        dbeta[row] = lin ? gam * kdKb + vdVb + kX1 : 0.f;
+    }
+}
+
+// dg_j = sum_{i>=j in chunk} dG_i, with the chunk-end extras added to the last row.
+__global__ void dg_kernel(const float *__restrict__ dGrow, const float *__restrict__ kappa,
+                          const float *__restrict__ gS, const float *__restrict__ Gcum, int n_slices,
+                          float *__restrict__ dg, int B, int L, int H) {
+    const int NC = L / kC;
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)B * H * NC) return;
+    const int c = idx % NC;
+    const size_t bh = idx / NC;
+    const int h = bh % H, b = bh / H;
+    const size_t base = bh * L + (size_t)c * kC;
+    float extra = 0.f;
+    for (int i = 0; i < kC; ++i) extra += kappa[base + i];
+    float gs = 0.f;
+    for (int s = 0; s < n_slices; ++s) gs += gS[idx * n_slices + s];
+    extra += __expf(Gcum[base + kC - 1]) * gs;
+    float run = extra;
+    for (int i = kC - 1; i >= 0; --i) {
+        run += dGrow[base + i];
+        dg[((size_t)b * L + (size_t)c * kC + i) * H + h] = run;
+    }
+}
+
+// dk, dv of the retained tokens: scatter the compacted softmax-branch gradients.
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads)
+scatter_sm_kernel(const float *__restrict__ dk_sm, const float *__restrict__ dv_sm, int cap,
+                  const int32_t *__restrict__ sm_idx, const int32_t *__restrict__ sm_chunk_prefix,
+                  T *__restrict__ dk, T *__restrict__ dv, int L, int H) {
+    constexpr int kVec = D / 4, kRows = kThreads / kVec;
+    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int NC = L / kC;
+    const int n = min(sm_chunk_prefix[(size_t)bh * (NC + 1) + NC], cap);
+    const int row = blockIdx.x * kRows + threadIdx.x / kVec, c4 = (threadIdx.x % kVec) * 4;
+    if (row >= n) return;
+    const int tok = sm_idx[(size_t)bh * L + row];
+    const size_t dst = (((size_t)b * L + tok) * H + h) * D + c4;
+    const size_t src = ((size_t)bh * cap + row) * D + c4;
+    store4(dk + dst, load4(dk_sm + src));
+    store4(dv + dst, load4(dv_sm + src));
+}
+
+template <typename Kn>
+cudaError_t set_smem(Kn kernel, size_t bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// host launchers
+// ------------------------------------------------------------------------------------------
+cudaError_t launch_bgemm(bool ta, bool tb, int mask, BMat A, BMat B, BMat C, int m, int n, int k,
+                         float alpha, bool accumulate, Shape s, cudaStream_t st) {
+    const int NC = s.L / kC;
+    dim3 grid(n / 64, m / 64, s.B * s.H * NC);
+#define NATSL_BG(TA, TB, MK) \
+    bgemm_kernel<TA, TB, MK><<<grid, kThreads, 0, st>>>(A, B, C, k, alpha, accumulate ? 1 : 0, s.H, NC)
+    if (!ta && !tb && mask == 0) NATSL_BG(false, false, 0);
+    else if (!ta && tb && mask == 0) NATSL_BG(false, true, 0);
+    else if (ta && !tb && mask == 0) NATSL_BG(true, false, 0);
+    else if (!ta && tb && mask == 1) NATSL_BG(false, true, 1);
+    else if (!ta && tb && mask == 2) NATSL_BG(false, true, 2);
+    else return cudaErrorInvalidValue;
+#undef NATSL_BG
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t to_f32_impl(const void *a, const void *b, const void *c, float *a32, float *b32,
+                               float *c32, size_t n, cudaStream_t st) {
+    to_f32_kernel<T><<<1184, 256, 0, st>>>((const T *)a, (const T *)b, (const T *)c, a32, b32, c32,
+                                           n / 4);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_to_f32(const void *a, const void *b, const void *c, float *a32, float *b32,
+                          float *c32, size_t n, bool bf16, cudaStream_t st) {
+    return bf16 ? to_f32_impl<__nv_bfloat16>(a, b, c, a32, b32, c32, n, st)
+                : to_f32_impl<float>(a, b, c, a32, b32, c32, n, st);
+}
+
+template <typename T, int D>
+static cudaError_t combine_bwd_impl(const float *o_la, const float *o_nla, const void *dout,
+                                    const float *w, float eps, float *do_la, float *do_nla,
+                                    float *dw, float *Dsm, Shape s, cudaStream_t st) {
+    const size_t rows = (size_t)s.B * s.L * s.H;
+    combine_bwd_kernel<T, D><<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
+        o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, s.B, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine_bwd(const float *o_la, const float *o_nla, const void *dout,
+                               const float *w, float eps, float *do_la, float *do_nla, float *dw,
+                               float *Dsm, Shape s, cudaStream_t st) {
+    if (s.bf16) {
+        if (s.d == 128) return combine_bwd_impl<__nv_bfloat16, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, s, st);
+        return combine_bwd_impl<__nv_bfloat16, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, s, st);
+    }
+    if (s.d == 128) return combine_bwd_impl<float, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, s, st);
+    return combine_bwd_impl<float, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, s, st);
+}
+
+template <int D>
+static cudaError_t softmax_bwd_impl(const float *q32, const float *k_sm32, const float *v_sm32,
+                                    int cap, const int32_t *sm_idx, const int32_t *pre,
+                                    const float *do_nla, const float *lse, const float *Dsm,
+                                    float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
+                                    Shape s, cudaStream_t st) {
+    const size_t smem_q = sizeof(float) * (2 * kC * D + 2 * 32 * (D + 1) + 32);
+    const size_t smem_k = sizeof(float) * (2 * 32 * (D + 1) + 2 * kC * D + 2 * kC * 33 + 2 * kC + 32);
+    cudaError_t e = set_smem(softmax_bwd_dq_kernel<D>, smem_q);
+    if (e != cudaSuccess) return e;
+    e = set_smem(softmax_bwd_dkv_kernel<D>, smem_k);
+    if (e != cudaSuccess) return e;
+    dim3 gq(s.L / kC, s.B * s.H);
+    softmax_bwd_dq_kernel<D><<<gq, kThreads, smem_q, st>>>(q32, k_sm32, v_sm32, cap, sm_idx, pre,
+                                                           do_nla, lse, Dsm, scale_sm, dq_sm, s.L, s.H);
+    count_launch();
+    dim3 gk((cap + 31) / 32, s.B * s.H);
+    softmax_bwd_dkv_kernel<D><<<gk, kThreads, smem_k, st>>>(q32, k_sm32, v_sm32, cap, sm_idx, pre,
+                                                            do_nla, lse, Dsm, scale_sm, dk_sm, dv_sm,
+                                                            s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const float *v_sm32, int cap,
+                               const int32_t *sm_idx, const int32_t *sm_chunk_prefix,
+                               const float *do_nla, const float *lse, const float *Dsm,
+                               float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm, Shape s,
+                               cudaStream_t st) {
+    if (s.d == 128) return softmax_bwd_impl<128>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, scale_sm, dq_sm, dk_sm, dv_sm, s, st);
+    return softmax_bwd_impl<64>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, scale_sm, dq_sm, dk_sm, dv_sm, s, st);
+}
+
+template <int D>
+static cudaError_t rscan_impl(const float *q32, const float *k32, const float *Gcum, const float *W,
+                              const float *P, const float *do_la, const float *chunk_states,
+                              float scale_la, float *dUt, float *dS_c, float *gS, Shape s,
+                              cudaStream_t st) {
+    const size_t smem = sizeof(float) * (D * kDvs + 3 * kC * (D + 1) + kC * (kC + 1) +
+                                         2 * kC * (kDvs + 1) + kC + 8);
+    cudaError_t e = set_smem(gdn_rscan_kernel<D>, smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid(D / kDvs, s.B * s.H);
+    gdn_rscan_kernel<D><<<grid, kThreads, smem, st>>>(q32, k32, Gcum, W, P, do_la, chunk_states,
+                                                      scale_la, dUt, dS_c, gS, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gdn_rscan(const float *q32, const float *k32, const float *Gcum, const float *W,
+                             const float *P, const float *do_la, const float *chunk_states,
+                             float scale_la, float *dUt, float *dS_c, float *gS, Shape s,
+                             cudaStream_t st) {
+    if (s.d == 128) return rscan_impl<128>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, s, st);
+    return rscan_impl<64>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, s, st);
+}
+
+cudaError_t launch_gdn_tsolve(const float *Abar, const float *beta, const uint8_t *route,
+                              const float *dW, const float *dUt, float *dKb, float *dVb, Shape s,
+                              cudaStream_t st) {
+    dim3 grid(s.L / kC, s.B * s.H);
+    if (s.d == 128)
+        gdn_tsolve_kernel<128><<<grid, kThreads, 0, st>>>(Abar, beta, route, dW, dUt, dKb, dVb, s.L, s.H);
+    else
+        gdn_tsolve_kernel<64><<<grid, kThreads, 0, st>>>(Abar, beta, route, dW, dUt, dKb, dVb, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mask_scale(const float *M, const float *N, const float *Gcum, const float *beta,
+                              const uint8_t *route, float scale_la, float *Mg, float *Ms, float *Ns,
+                              Shape s, cudaStream_t st) {
+    dim3 grid(s.L / kC, s.B * s.H);
+    mask_scale_kernel<<<grid, kThreads, 0, st>>>(M, N, Gcum, beta, route, scale_la, Mg, Ms, Ns, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <typename T, int D>
+static cudaError_t assemble_impl(const AssembleArgs &a, void *dq, void *dk, void *dv, Shape s,
+                                 cudaStream_t st) {
+    const size_t rows = (size_t)s.B * s.L * s.H;
+    gdn_assemble_kernel<T, D><<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
+        a.q32, a.k32, a.v32, a.Gcum, a.beta, a.route, a.dQg, a.dKb, a.dVb, a.dKt, a.X1p, a.X2, a.X3,
+        a.X4, a.dq_sm, a.scale_la, (T *)dq, (T *)dk, (T *)dv, a.dGrow, a.kappa, a.dbeta, s.B, s.L, s.H);
+    count_launch();
+    const int NC = s.L / kC;
+    const size_t nch = (size_t)s.B * s.H * NC;
+    dg_kernel<<<(unsigned)((nch + 127) / 128), 128, 0, st>>>(a.dGrow, a.kappa, a.gS, a.Gcum,
+                                                            s.d / kDvs, a.dg, s.B, s.L, s.H);
+    count_launch();
+    constexpr int kRows = kThreads / (D / 4);
+    dim3 grid((a.cap + kRows - 1) / kRows, s.B * s.H);
+    scatter_sm_kernel<T, D><<<grid, kThreads, 0, st>>>(a.dk_sm, a.dv_sm, a.cap, a.sm_idx, a.sm_prefix,
+                                                       (T *)dk, (T *)dv, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gdn_assemble(const AssembleArgs &a, void *dq, void *dk, void *dv, Shape s,
+                                cudaStream_t st) {
+    if (s.bf16) {
+        if (s.d == 128) return assemble_impl<__nv_bfloat16, 128>(a, dq, dk, dv, s, st);
+        return assemble_impl<__nv_bfloat16, 64>(a, dq, dk, dv, s, st);
+    }
+    if (s.d == 128) return assemble_impl<float, 128>(a, dq, dk, dv, s, st);
+    return assemble_impl<float, 64>(a, dq, dk, dv, s, st);
+}
+
+}  // namespace natsl

@@ -38,7 +38,8 @@ __global__ void __launch_bounds__(kThreads)
 gdn_prepare_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
                         const float *__restrict__ g, const float *__restrict__ beta,
                         const uint8_t *__restrict__ route, float scale_la, float *__restrict__ W,
-                        float *__restrict__ U, float *__restrict__ P, int L, int H) {
+                        float *__restrict__ U, float *__restrict__ P, float *__restrict__ Abar,
+                        float *__restrict__ Gcum, int L, int H) {
     extern __shared__ float smem[];
     float *Ks = smem;                       // [64][D+1]
     float *Vs = Ks + kC * (D + 1);          // [64][D+1]  (V, later Q)
@@ -63,20 +64,23 @@ gdn_prepare_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const 
         for (int i = 0; i < kC; ++i) { acc += Gs[i]; Gs[i] = acc; }
     }
     __syncthreads();
-    // A (strictly lower)
+    if (Gcum && threadIdx.x < kC) Gcum[(size_t)bh * L + c * kC + threadIdx.x] = Gs[threadIdx.x];
+    // A (strictly lower); Abar = A without the beta~ row factor (the backward needs it)
     {
         const int i = threadIdx.x >> 2;
+        float *Ab = Abar ? Abar + ((size_t)bh * (L / kC) + c) * kC * kC : nullptr;
         for (int m = 0; m < 16; ++m) {
             const int j = (threadIdx.x & 3) + 4 * m;
             float a = 0.f;
-            if (j < i && bts[i] != 0.f) {
+            if (j < i && (bts[i] != 0.f || Ab)) {
                 float dot = 0.f;
                 const float *ki = Ks + i * (D + 1), *kj = Ks + j * (D + 1);
 #pragma unroll 8
                 for (int x = 0; x < D; ++x) dot = fmaf(ki[x], kj[x], dot);
-                a = bts[i] * __expf(Gs[i] - Gs[j]) * dot;
+                a = __expf(Gs[i] - Gs[j]) * dot;
             }
-            As[i * kC + j] = a;
+            if (Ab) Ab[i * kC + j] = a;
+            As[i * kC + j] = bts[i] * a;
         }
     }
     __syncthreads();
@@ -131,7 +135,7 @@ gdn_scan_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const flo
                      const float *__restrict__ W, const float *__restrict__ U,
                      const float *__restrict__ P, float scale_la, const float *__restrict__ state_in,
                      float *__restrict__ state_out, float *__restrict__ chunk_states,
-                     float *__restrict__ o_la, int L, int H) {
+                     float *__restrict__ Ut, float *__restrict__ o_la, int L, int H) {
     extern __shared__ float smem[];
     float *Ss = smem;                        // [D][32]
     float *Ws = Ss + D * kDvs;               // [64][D+1]
@@ -195,6 +199,11 @@ gdn_scan_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const flo
             __syncthreads();
 #pragma unroll
             for (int x = 0; x < 8; ++x) Us[r * (kDvs + 1) + cb + x] = acc[x];
+            if (Ut) {
+                float *dst = Ut + (tok0 + (size_t)r * H) * D + c0 + cb;
+                store4(dst, make_float4(acc[0], acc[1], acc[2], acc[3]));
+                store4(dst + 4, make_float4(acc[4], acc[5], acc[6], acc[7]));
+            }
         }
         __syncthreads();
         // O = scale_la gamma_r q_r S + sum_{j<=r} P_rj U~_j
@@ -356,7 +365,7 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
         const float wn = w ? w[t * 2] : 0.5f, wl = w ? w[t * 2 + 1] : 0.5f;
 #pragma unroll
         for (int x = 0; x < kCols; ++x) {
-            out[t * D + lane + 32 * x] = from_f32<T>(wn * on[x] * fn + wl * ol[x] * fl);
+            if (out) out[t * D + lane + 32 * x] = from_f32<T>(wn * on[x] * fn + wl * ol[x] * fl);
             if (o_nla) o_nla[t * D + lane + 32 * x] = on[x];
         }
         if (lse && lane == 0) lse[(size_t)bh * L + i] = z[r] > 0.f ? m[r] + __logf(z[r]) : -INFINITY;
@@ -389,35 +398,38 @@ static size_t simt_softmax_smem(int d) { return sizeof(float) * (kC * d + 32 * (
 template <typename T, int D>
 static cudaError_t prepare_impl(const void *q, const void *k, const void *v, const float *g,
                                 const float *beta, const uint8_t *route, float scale_la, float *W,
-                                float *U, float *P, Shape s, cudaStream_t st) {
+                                float *U, float *P, float *Abar, float *Gcum, Shape s,
+                                cudaStream_t st) {
     const size_t smem = simt_prepare_smem(D);
     cudaError_t e = set_smem(gdn_prepare_simt_kernel<T, D>, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(s.L / kC, s.B * s.H);
     gdn_prepare_simt_kernel<T, D><<<grid, kThreads, smem, st>>>(
-        (const T *)q, (const T *)k, (const T *)v, g, beta, route, scale_la, W, U, P, s.L, s.H);
+        (const T *)q, (const T *)k, (const T *)v, g, beta, route, scale_la, W, U, P, Abar, Gcum, s.L,
+        s.H);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_gdn_prepare_simt(const void *q, const void *k, const void *v, const float *g,
                                     const float *beta, const uint8_t *route, float scale_la,
-                                    float *W, float *U, float *P, Shape s, cudaStream_t st) {
-    NATSL_DISPATCH(prepare_impl, q, k, v, g, beta, route, scale_la, W, U, P, s, st);
+                                    float *W, float *U, float *P, float *Abar, float *Gcum, Shape s,
+                                    cudaStream_t st) {
+    NATSL_DISPATCH(prepare_impl, q, k, v, g, beta, route, scale_la, W, U, P, Abar, Gcum, s, st);
 }
 
 template <typename T, int D>
 static cudaError_t scan_impl(const void *q, const void *k, const float *g, const float *W,
                              const float *U, const float *P, float scale_la, const float *state_in,
-                             float *state_out, float *chunk_states, float *o_la, Shape s,
+                             float *state_out, float *chunk_states, float *Ut, float *o_la, Shape s,
                              cudaStream_t st) {
     const size_t smem = simt_scan_smem(D);
     cudaError_t e = set_smem(gdn_scan_simt_kernel<T, D>, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(D / kDvs, s.B * s.H);
     gdn_scan_simt_kernel<T, D><<<grid, kThreads, smem, st>>>(
-        (const T *)q, (const T *)k, g, W, U, P, scale_la, state_in, state_out, chunk_states, o_la,
-        s.L, s.H);
+        (const T *)q, (const T *)k, g, W, U, P, scale_la, state_in, state_out, chunk_states, Ut,
+        o_la, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -425,9 +437,9 @@ static cudaError_t scan_impl(const void *q, const void *k, const float *g, const
 cudaError_t launch_gdn_scan_simt(const void *q, const void *k, const float *g, const float *W,
                                  const float *U, const float *P, float scale_la,
                                  const float *state_in, float *state_out, float *chunk_states,
-                                 float *o_la, Shape s, cudaStream_t st) {
-    NATSL_DISPATCH(scan_impl, q, k, g, W, U, P, scale_la, state_in, state_out, chunk_states, o_la, s,
-                   st);
+                                 float *Ut, float *o_la, Shape s, cudaStream_t st) {
+    NATSL_DISPATCH(scan_impl, q, k, g, W, U, P, scale_la, state_in, state_out, chunk_states, Ut, o_la,
+                   s, st);
 }
 
 template <typename T, int D>

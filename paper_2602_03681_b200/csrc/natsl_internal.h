@@ -31,16 +31,63 @@ size_t simt_prepare_smem(int d);
 size_t simt_scan_smem(int d);
 cudaError_t launch_gdn_prepare_simt(const void *q, const void *k, const void *v, const float *g,
                                     const float *beta, const uint8_t *route, float scale_la,
-                                    float *W, float *U, float *P, Shape s, cudaStream_t st);
+                                    float *W, float *U, float *P, float *Abar, float *Gcum, Shape s,
+                                    cudaStream_t st);
 cudaError_t launch_gdn_scan_simt(const void *q, const void *k, const float *g, const float *W,
                                  const float *U, const float *P, float scale_la,
                                  const float *state_in, float *state_out, float *chunk_states,
-                                 float *o_la, Shape s, cudaStream_t st);
+                                 float *Ut, float *o_la, Shape s, cudaStream_t st);
 cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const void *v_sm,
                                         int32_t cap, const int32_t *sm_idx,
                                         const int32_t *sm_chunk_prefix, const float *o_la,
                                         const float *w, float scale_sm, float eps, void *out,
                                         float *o_nla, float *lse, Shape s, cudaStream_t st);
+
+// bwd_simt.cu -- fp32 CUDA-core backward
+// A batched matrix operand: element (r, c) of batch (b, h, chunk) is
+// p[b*sb + h*sh + chunk*sc + r*ld + c].
+struct BMat {
+    const float *p;
+    long long sb, sh, sc;
+    int ld;
+};
+// C = alpha * op(A) op(B) (+ C) per (batch, head, chunk); m, n multiples of 64, k of 16.
+// mask: 0 none, 1 keep col <= row, 2 keep col < row (64x64 outputs).
+cudaError_t launch_bgemm(bool ta, bool tb, int mask, BMat A, BMat B, BMat C, int m, int n, int k,
+                         float alpha, bool accumulate, Shape s, cudaStream_t st);
+cudaError_t launch_to_f32(const void *a, const void *b, const void *c, float *a32, float *b32,
+                          float *c32, size_t n, bool bf16, cudaStream_t st);
+cudaError_t launch_combine_bwd(const float *o_la, const float *o_nla, const void *dout,
+                               const float *w, float eps, float *do_la, float *do_nla, float *dw,
+                               float *Dsm, Shape s, cudaStream_t st);
+cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const float *v_sm32, int cap,
+                               const int32_t *sm_idx, const int32_t *sm_chunk_prefix,
+                               const float *do_nla, const float *lse, const float *Dsm,
+                               float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm, Shape s,
+                               cudaStream_t st);
+cudaError_t launch_gdn_rscan(const float *q32, const float *k32, const float *Gcum, const float *W,
+                             const float *P, const float *do_la, const float *chunk_states,
+                             float scale_la, float *dUt, float *dS_c, float *gS, Shape s,
+                             cudaStream_t st);
+cudaError_t launch_gdn_tsolve(const float *Abar, const float *beta, const uint8_t *route,
+                              const float *dW, const float *dUt, float *dKb, float *dVb, Shape s,
+                              cudaStream_t st);
+cudaError_t launch_mask_scale(const float *M, const float *N, const float *Gcum, const float *beta,
+                              const uint8_t *route, float scale_la, float *Mg, float *Ms, float *Ns,
+                              Shape s, cudaStream_t st);
+struct AssembleArgs {
+    const float *q32, *k32, *v32, *Gcum, *beta;
+    const uint8_t *route;
+    const float *dQg, *dKb, *dVb, *dKt, *X1p, *X2, *X3, *X4, *dq_sm, *dk_sm, *dv_sm, *gS;
+    const int32_t *sm_idx, *sm_prefix;
+    int cap;
+    float scale_la;
+    float *dGrow, *kappa, *dbeta, *dg;
+};
+// dq (all tokens), dk/dv (linear tokens from the GDN branch, retained tokens scattered from the
+// compacted softmax-branch gradients), dbeta, dg.  Three kernels.
+cudaError_t launch_gdn_assemble(const AssembleArgs &a, void *dq, void *dk, void *dv, Shape s,
+                                cudaStream_t st);
 
 // decode.cu
 cudaError_t launch_decode_step(const void *q, const void *k, const void *v, const float *g,
