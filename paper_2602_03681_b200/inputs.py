@@ -65,9 +65,12 @@ def _rng(seed: int, stream: str) -> np.random.Generator:
 def round_bf16(x: np.ndarray) -> np.ndarray:
     """Round float32 to the nearest bf16 (ties to even) and return it widened to float32."""
     x = np.ascontiguousarray(x, np.float32)
-    u = x.view(np.uint32).astype(np.uint64)
-    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
-    return u.astype(np.uint32).view(np.float32).reshape(x.shape)
+    u = x.view(np.uint32)                       # finite inputs: the add below cannot wrap
+    r = (u >> np.uint32(16)) & np.uint32(1)
+    r += np.uint32(0x7FFF)
+    r += u
+    r &= np.uint32(0xFFFF0000)
+    return r.view(np.float32).reshape(x.shape)
 
 
 def _normal(seed, stream, shape):

@@ -1,0 +1,72 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times.
+The oracle is fast enough to check every element of the prefill / training workloads; for the
+decode workload it recomputes a sample of the sequences (each (sequence, head) is independent)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_03681_b200 import inputs
+from test_gpu_parity import TOL, check_bwd, check_fwd, check_stored, dev, run_bwd, run_fwd, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["cfg1_bf16_prefill", "cfg2_bf16_long_prefill"])
+def test_fwd_full_size(name):
+    wl = inputs.WORKLOADS[name]
+    x = inputs.make_layer_inputs(wl)
+    got = run_fwd(wl, x)
+    ref = run_oracle(wl, x)
+    check_fwd(wl, got, ref, TOL[wl.dtype])
+
+
+def test_fwd_bwd_full_size_training_workload():
+    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+    x = inputs.make_layer_inputs(wl)
+    got = run_fwd(wl, x)
+    ref = run_oracle(wl, x)
+    check_fwd(wl, got, ref, TOL[wl.dtype])
+    gb = run_bwd(wl, x)
+    rb = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                           scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+    check_bwd(wl, gb, rb, TOL[wl.dtype])
+    lin = x["route"] == 0
+    assert np.all(gb["dbeta"][~lin] == 0)
+
+
+def test_decode_full_size_sampled_sequences():
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg3_bf16_decode"]
+    steps = 12
+    x = inputs.make_decode_inputs(wl, steps=steps)
+    B, H, d = wl.B, wl.H, wl.d
+    dt = torch.bfloat16
+    state = dev(x["state"])
+    kc, vc = dev(x["k_cache"], dt), dev(x["v_cache"], dt)
+    n = dev(x["cache_len"])
+    p = binding.make_params(B, H, 0, d, binding.NATSL_BF16, wl.scale_la, wl.scale_sm)
+    ws = binding.alloc_workspace(p, binding.OP_DECODE)
+    sample = [0, 21, 42, 63]
+    o_state = x["state"][sample].astype(np.float64)
+    o_kc, o_vc = x["k_cache"][sample].astype(np.float64), x["v_cache"][sample].astype(np.float64)
+    o_n = np.ascontiguousarray(x["cache_len"][sample])
+    for t in range(steps):
+        w = dev(x["w"][t])
+        p.w = w.data_ptr()
+        out = torch.empty((B, H, d), dtype=dt, device="cuda")
+        binding.natsl_decode_step(dev(x["q"][t], dt), dev(x["k"][t], dt), dev(x["v"][t], dt),
+                                  dev(x["g"][t]), dev(x["beta"][t]), dev(x["route"][t]), state, kc,
+                                  vc, n, out, p, ws)
+        ref = oracle.decode_step(x["q"][t][sample], x["k"][t][sample], x["v"][t][sample],
+                                 x["g"][t][sample], x["beta"][t][sample], x["route"][t][sample],
+                                 x["w"][t][sample], o_state, o_kc, o_vc, o_n,
+                                 scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+        check_stored(out[sample].float().cpu().numpy(), ref["out"], TOL["bf16"], "bf16", f"step{t}")
+    assert binding.natsl_device_status(ws) == 0
+    assert np.array_equal(n.cpu().numpy()[sample], o_n)
+    # properties that hold for every sequence: lengths grow by the routed tokens, state finite
+    assert np.array_equal(n.cpu().numpy(), x["cache_len"] + x["route"].sum(0).astype(np.int32))
+    assert torch.isfinite(state).all()
+    err = np.abs(state[sample].cpu().numpy() - o_state).max() / np.sqrt((o_state ** 2).mean())
+    assert err <= 1e-4
