@@ -46,7 +46,8 @@ typedef enum natsl_status {
     NATSL_ERR_WORKSPACE = -5,   /* workspace NULL or smaller than natsl_workspace_size */
     NATSL_ERR_CUDA = -6,        /* a launch or runtime call failed */
     NATSL_ERR_CACHE_FULL = -7,  /* decode: a retained-KV cache has no room (device-detected) */
-    NATSL_ERR_UNSUPPORTED = -8  /* valid request this build does not implement */
+    NATSL_ERR_UNSUPPORTED = -8, /* valid request this build does not implement */
+    NATSL_ERR_TOO_LARGE = -9    /* natsl_hybrid_fwd_static: problem needs more than the built-in scratch */
 } natsl_status;
 
 enum { NATSL_F32 = 0, NATSL_BF16 = 1 };
@@ -106,6 +107,28 @@ int natsl_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk
 int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g,
                      const float *beta, const uint8_t *route, void *out,
                      const natsl_params *p, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * natsl_hybrid_fwd for callers that cannot allocate device memory (no counterpart in the paper;
+ * it computes exactly what natsl_hybrid_fwd computes).  A plug-in inside a server that owns the
+ * memory pool, or a latency-critical loop that must not hit the device-wide synchronisation of
+ * cudaMalloc, has no workspace to hand over.  Here the scratch is a fixed array of
+ * NATSL_STATIC_WS_BYTES inside the library (each GPU that loads the library holds it until the
+ * process exits); the caller passes only inputs and outputs, including the optional ones in `p`.
+ *   - Problems whose natsl_workspace_size(p, NATSL_OP_FWD) exceeds NATSL_STATIC_WS_BYTES are
+ *     rejected with NATSL_ERR_TOO_LARGE before anything is launched.
+ *   - The first call on each device looks up the array's device address (a host-side set-up
+ *     step); make that first call outside any stream capture.
+ *   - The call itself performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the
+ *     library re-initialises what it needs.  Two calls that overlap on the GPU (different
+ *     streams, no ordering between them) race on it: keep them on one stream or order them.
+ * Errors otherwise as natsl_hybrid_fwd.
+ */
+#define NATSL_STATIC_WS_BYTES (32u << 20)
+int natsl_hybrid_fwd_static(const void *q, const void *k, const void *v, const float *g,
+                            const float *beta, const uint8_t *route, void *out,
+                            const natsl_params *p, void *stream);
 
 /*
  * Backward of natsl_hybrid_fwd's `out` (Section 4.2 states the properties: the softmax-branch

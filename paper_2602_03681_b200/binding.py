@@ -20,8 +20,10 @@ FORCE_SIMT = 1
 ERR_CACHE_FULL = -7
 
 EXPORTS = ["natsl_workspace_size", "natsl_route_compact", "natsl_hybrid_fwd", "natsl_hybrid_bwd",
-           "natsl_decode_step", "natsl_device_status", "natsl_stage_name", "natsl_launch_count",
-           "natsl_strerror"]
+           "natsl_decode_step", "natsl_device_status", "natsl_hybrid_fwd_static",
+           "natsl_stage_name", "natsl_launch_count", "natsl_strerror"]
+ERR_TOO_LARGE = -9
+STATIC_WS_BYTES = 32 << 20
 
 
 class NatslError(RuntimeError):
@@ -60,7 +62,7 @@ def lib() -> ctypes.CDLL:
         _lib.natsl_stage_name.restype = ctypes.c_char_p
         _lib.natsl_stage_name.argtypes = [ctypes.c_int, ctypes.c_int]
         _lib.natsl_launch_count.restype = ctypes.c_uint64
-        for name in EXPORTS[:6]:
+        for name in EXPORTS[:7]:
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -153,6 +155,14 @@ def natsl_hybrid_fwd(q, k, v, g, beta, route, out, p: natsl_params, ws):
     _check(lib().natsl_hybrid_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(route),
                                   _ptr(out), ctypes.byref(p), _ptr(ws),
                                   ctypes.c_size_t(ws.numel()), _stream()))
+
+
+def natsl_hybrid_fwd_static(q, k, v, g, beta, route, out, p: natsl_params):
+    """natsl_hybrid_fwd without a caller workspace: the scratch is a fixed array inside the
+    library, for hosts that cannot allocate device memory.  Raises NatslError(-9) when the
+    problem needs more than STATIC_WS_BYTES of scratch."""
+    _check(lib().natsl_hybrid_fwd_static(_ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta),
+                                         _ptr(route), _ptr(out), ctypes.byref(p), _stream()))
 
 
 def natsl_hybrid_bwd(q, k, v, g, beta, route, dout, dq, dk, dv, dg, dbeta, dw, p: natsl_params, ws):

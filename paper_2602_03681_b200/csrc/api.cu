@@ -136,6 +136,7 @@ const char *natsl_strerror(int status) {
         case NATSL_ERR_CUDA: return "CUDA launch or runtime error";
         case NATSL_ERR_CACHE_FULL: return "retained-KV cache full";
         case NATSL_ERR_UNSUPPORTED: return "request not implemented in this build";
+        case NATSL_ERR_TOO_LARGE: return "problem needs more scratch than the library's built-in array (NATSL_STATIC_WS_BYTES)";
         default: return "unknown natsl status";
     }
 }
