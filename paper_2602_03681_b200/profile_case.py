@@ -1,0 +1,108 @@
+"""Run one operation of the library a few times on a chosen (possibly reduced) workload.
+
+Meant to be the command a profiler wraps: it draws the seeded synthetic inputs, runs `--iters`
+calls of `--op` on the current device and exits.  Nothing is timed or checked here.
+
+    python -m paper_2602_03681_b200.profile_case --op fwd --workload cfg1_bf16_prefill --B 1
+    python -m paper_2602_03681_b200.profile_case --op decode --workload cfg3_bf16_decode --B 8 --iters 4
+    python -m paper_2602_03681_b200.profile_case --op bwd --workload cfg4_bf16_train --B 1
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import binding, inputs
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--op", choices=["fwd", "bwd", "decode"], default="fwd")
+    ap.add_argument("--workload", default=None, choices=sorted(inputs.WORKLOADS),
+                    help="default: the workload that belongs to --op")
+    ap.add_argument("--B", type=int, default=None, help="batch override (smaller case)")
+    ap.add_argument("--L", type=int, default=None, help="sequence length override")
+    ap.add_argument("--iters", type=int, default=2)
+    ap.add_argument("--flags", type=int, default=0)
+    ap.add_argument("--report", action="store_true", help="print CUDA-event time of each call")
+    args = ap.parse_args()
+    if args.workload is None:
+        args.workload = {"fwd": "cfg1_bf16_prefill", "bwd": "cfg4_bf16_train",
+                         "decode": "cfg3_bf16_decode"}[args.op]
+    if (inputs.WORKLOADS[args.workload].call == "decode") != (args.op == "decode"):
+        ap.error(f"workload {args.workload} does not belong to --op {args.op}")
+
+    wl = inputs.WORKLOADS[args.workload]
+    dt = torch.float32 if wl.dtype == "f32" else torch.bfloat16
+    code = binding.NATSL_F32 if wl.dtype == "f32" else binding.NATSL_BF16
+    torch.cuda.set_device(0)
+    binding.lib()
+
+    def dev(a, t=None):
+        x = torch.from_numpy(a).cuda()
+        return x if t is None else x.to(t)
+
+    events = []
+
+    def timed(call):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        call()
+        e1.record()
+        events.append((e0, e1))
+
+    def finish(note=""):
+        torch.cuda.synchronize()
+        if args.report:
+            print(f"{args.op} {args.workload}: ms per call",
+                  [round(a.elapsed_time(b), 4) for a, b in events], note)
+
+    if args.op == "decode":
+        B = args.B or wl.B
+        x = inputs.make_decode_inputs(wl, B=B, steps=args.iters)
+        state, n = dev(x["state"]), dev(x["cache_len"])
+        kc, vc = dev(x["k_cache"], dt), dev(x["v_cache"], dt)
+        p = binding.make_params(B, wl.H, 0, wl.d, code, wl.scale_la, wl.scale_sm, flags=args.flags)
+        ws = binding.alloc_workspace(p, binding.OP_DECODE)
+        out = torch.empty((B, wl.H, wl.d), dtype=dt, device="cuda")
+        tok = {m: dev(x[m], dt if m in ("q", "k", "v") else None)
+               for m in ("q", "k", "v", "g", "beta", "route", "w")}
+        for t in range(args.iters):
+            p.w = tok["w"][t].data_ptr()
+            timed(lambda: binding.natsl_decode_step(
+                tok["q"][t], tok["k"][t], tok["v"][t], tok["g"][t], tok["beta"][t],
+                tok["route"][t], state, kc, vc, n, out, p, ws))
+        finish(f"cache_len {int(n.min())}..{int(n.max())}")
+        return
+
+    kw = {}
+    if args.B:
+        kw["B"] = args.B
+    if args.L:
+        kw["L"] = args.L
+    x = inputs.make_layer_inputs(wl, **kw)
+    q, k, v = (dev(x[m], dt) for m in ("q", "k", "v"))
+    g, beta, route, w = (dev(x[m]) for m in ("g", "beta", "route", "w"))
+    if args.op == "fwd":
+        ws = None
+        for _ in range(args.iters):
+            def call():
+                nonlocal ws
+                ws = binding.hybrid_fwd(q, k, v, g, beta, route, w, scale_la=wl.scale_la,
+                                        scale_sm=wl.scale_sm, flags=args.flags, ws=ws)["ws"]
+            timed(call)
+    else:
+        dout = dev(x["dout"], dt)
+        ws = None
+        for _ in range(args.iters):
+            def call():
+                nonlocal ws
+                ws = binding.hybrid_bwd(q, k, v, g, beta, route, w, dout, scale_la=wl.scale_la,
+                                        scale_sm=wl.scale_sm, ws=ws)["ws"]
+            timed(call)
+    finish()
+
+
+if __name__ == "__main__":
+    main()
