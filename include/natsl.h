@@ -47,7 +47,8 @@ typedef enum natsl_status {
     NATSL_ERR_CUDA = -6,        /* a launch or runtime call failed */
     NATSL_ERR_CACHE_FULL = -7,  /* decode: a retained-KV cache has no room (device-detected) */
     NATSL_ERR_UNSUPPORTED = -8, /* valid request this build does not implement */
-    NATSL_ERR_TOO_LARGE = -9    /* natsl_hybrid_fwd_static: problem needs more than the built-in scratch */
+    NATSL_ERR_TOO_LARGE = -9,   /* natsl_hybrid_fwd_static: problem needs more than the built-in scratch */
+    NATSL_ERR_TIMEOUT = -10     /* a bounded device-side wait expired (device-detected); kernel drained */
 } natsl_status;
 
 enum { NATSL_F32 = 0, NATSL_BF16 = 1 };
@@ -55,7 +56,8 @@ enum { NATSL_OP_FWD = 0, NATSL_OP_BWD = 1, NATSL_OP_DECODE = 2, NATSL_OP_COMPACT
 
 /* flags */
 enum {
-    NATSL_FORCE_SIMT = 1u << 0   /* use the fp32 CUDA-core kernels even for bf16 tensors */
+    NATSL_FORCE_SIMT = 1u << 0   /* use the fp32 CUDA-core kernels even for bf16 tensors (the
+                                    default for bf16 is the tcgen05 tensor-core path) */
 };
 
 typedef struct natsl_params {

@@ -47,7 +47,7 @@ Shape shape_of(const natsl_params *p) { return Shape{p->B, p->H, p->L, p->d, p->
 
 struct FwdWs {
     int32_t *status, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
-    void *k_sm, *v_sm;
+    void *k_sm, *v_sm, *v16;
     float *W, *U, *P, *o_la;
     size_t bytes;
 };
@@ -65,6 +65,7 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
     f.sm_len = c.take<int32_t>(B * H);
     f.k_sm = c.take<char>(B * H * L * d * esz);
     f.v_sm = c.take<char>(B * H * L * d * esz);
+    f.v16 = c.take<char>(p->dtype == NATSL_BF16 ? B * H * L * d * 2 : 0);   // fp16 V of the retained tokens
     f.W = c.take<float>(B * L * H * d);
     f.U = c.take<float>(B * L * H * d);
     f.P = c.take<float>(B * H * NC * kC * kC);
@@ -136,6 +137,7 @@ const char *natsl_strerror(int status) {
         case NATSL_ERR_CUDA: return "CUDA launch or runtime error";
         case NATSL_ERR_CACHE_FULL: return "retained-KV cache full";
         case NATSL_ERR_UNSUPPORTED: return "request not implemented in this build";
+        case NATSL_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case NATSL_ERR_TOO_LARGE: return "problem needs more scratch than the library's built-in array (NATSL_STATIC_WS_BYTES)";
         default: return "unknown natsl status";
     }
@@ -195,7 +197,12 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     const int32_t cap = want_cache ? p->sm_cap : p->L;
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, sm_len, p->B, p->L,
                                    p->H, st));
-    NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
+    const bool tensor_cores = s.bf16 && !(p->flags & NATSL_FORCE_SIMT);
+    if (tensor_cores)
+        NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
+                                      f.v16, cap, p->L, f.status, s, st));
+    else
+        NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
     NATSL_TRY(mark());
     float *o_la = p->o_la ? p->o_la : f.o_la;
     NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P, nullptr,
@@ -204,8 +211,13 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_gdn_scan_simt(q, k, g, f.W, f.U, f.P, p->scale_la, p->state_in, p->state_out,
                                    nullptr, nullptr, o_la, s, st));
     NATSL_TRY(mark());
-    NATSL_TRY(launch_softmax_combine_simt(q, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
-                                          p->scale_sm, p->eps, out, p->o_nla, p->lse, s, st));
+    if (tensor_cores)
+        NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, p->L, f.sm_idx, f.prefix, o_la, p->w,
+                                            p->scale_sm, p->eps, out, p->o_nla, p->lse, f.status, s,
+                                            st));
+    else
+        NATSL_TRY(launch_softmax_combine_simt(q, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
+                                              p->scale_sm, p->eps, out, p->o_nla, p->lse, s, st));
     NATSL_TRY(mark());
 #undef NATSL_TRY
     return NATSL_OK;

@@ -43,6 +43,18 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
                                         const float *w, float scale_sm, float eps, void *out,
                                         float *o_nla, float *lse, Shape s, cudaStream_t st);
 
+// softmax_tc.cu -- tensor-core softmax branch + combination (bf16 storage)
+cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
+                                const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
+                                int32_t cap, int32_t capv, int32_t *status, Shape s,
+                                cudaStream_t st);
+cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const void *v16, int32_t cap,
+                                      int32_t capv, const int32_t *sm_idx,
+                                      const int32_t *sm_chunk_prefix, const float *o_la,
+                                      const float *w, float scale_sm, float eps, void *out,
+                                      float *o_nla, float *lse, int32_t *status, Shape s,
+                                      cudaStream_t st);
+
 // bwd_simt.cu -- fp32 CUDA-core backward
 // A batched matrix operand: element (r, c) of batch (b, h, chunk) is
 // p[b*sb + h*sh + chunk*sc + r*ld + c].

@@ -1,0 +1,418 @@
+// Tensor-core softmax branch over the retained tokens (Section 4.1, O_nla with mask M^nla) with
+// the RMS-norm / weighted combination (Section 4.3, Norm equation) as its epilogue, for bf16
+// storage on sm_100a.
+//
+// One CTA owns 128 consecutive queries of one (batch, head) and walks the compacted K/V of that
+// head in tiles of 64 retained tokens: logits = Q K^T as a bf16 tcgen05 MMA into TMEM (q and k
+// are exact bf16 inputs), online softmax in registers (one thread per query row), probabilities
+// written to shared memory as fp16 and P V as an fp16 MMA (V is gathered as fp16: the bf16
+// inputs convert exactly, and an 11-bit probability keeps the branch output within ~2e-3 of
+// its RMS where an 8-bit one would not).  K/V tiles arrive by TMA into a two-stage ring.
+// Warp roles: warps 0-3 softmax/epilogue (thread r <-> query row r <-> TMEM lane r), warp 4 issues
+// the MMAs, warp 5 issues the TMA loads.
+#include "common.cuh"
+#include "natsl_internal.h"
+#include "tc_common.cuh"
+
+namespace natsl {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kBM = 128;        // queries per CTA
+constexpr int kBN = 64;         // retained tokens per K/V tile
+constexpr int kStages = 2;
+constexpr int kSoftmaxThreads = 128;
+constexpr int kThreadsTc = 192;
+constexpr int kMiscBytes = 1024;
+
+template <int D> struct SmLayout {
+    static constexpr int KB = D / 64;                    // 64-column blocks of the head dimension
+    static constexpr int kQBytes = KB * kBM * 128;
+    static constexpr int kKStage = KB * kBN * 128;
+    static constexpr int kVStage = KB * kBN * 128;
+    static constexpr int kPBytes = kBM * 128;
+    static constexpr int oQ = 0;
+    static constexpr int oK = oQ + kQBytes;
+    static constexpr int oV = oK + kStages * kKStage;
+    static constexpr int oP = oV + kStages * kVStage;
+    static constexpr int oMisc = oP + kPBytes;
+    static constexpr int kTotal = oMisc + kMiscBytes;
+};
+
+struct Misc {                    // lives in the last kMiscBytes of the CTA's shared memory
+    uint64_t barQ, full[kStages], empty[kStages], barS[2], barP, barO;
+    uint32_t tmem_base;
+    int abort_flag;
+    int pos[kBM];                // positions of the retained tokens inside the CTA's own chunks
+};
+static_assert(sizeof(Misc) <= kMiscBytes, "misc page too small");
+
+template <int D>
+__global__ void __launch_bounds__(kThreadsTc)
+softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
+                          const __grid_constant__ CUtensorMap map_k,
+                          const __grid_constant__ CUtensorMap map_v, int cap, int capv,
+                          const int32_t *__restrict__ sm_idx,
+                          const int32_t *__restrict__ sm_chunk_prefix,
+                          const float *__restrict__ o_la, const float *__restrict__ w,
+                          float scale_sm, float eps, __nv_bfloat16 *__restrict__ out,
+                          float *__restrict__ o_nla, float *__restrict__ lse, int32_t *status, int L,
+                          int H) {
+    using SL = SmLayout<D>;
+    constexpr int KB = SL::KB;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    Misc &ms = *reinterpret_cast<Misc *>(smem + SL::oMisc);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int NP = (L + kBM - 1) / kBM, NC = L / kC;
+    const int p = NP - 1 - (int)blockIdx.x;           // long rows first
+    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int c0 = 2 * p, c1 = min(2 * p + 2, NC);
+    const int32_t *pre = sm_chunk_prefix + (size_t)bh * (NC + 1);
+    const int n_full = min(pre[c0], cap);             // retained tokens before the CTA's chunks
+    const int n_end = min(pre[c1], cap);              // ... up to the end of the CTA's chunks
+    const int T = (n_end + kBN - 1) / kBN;
+
+    if ((smem_u32(smem) & 1023u) != 0) {              // operand tiles need 1024-byte alignment
+        if (tid == 0) atomicMin(status, (int)NATSL_ERR_CUDA);
+        return;
+    }
+    if (tid == 0) {
+        mbar_init(&ms.barQ, 1);
+        for (int s = 0; s < kStages; ++s) { mbar_init(&ms.full[s], 1); mbar_init(&ms.empty[s], 1); }
+        mbar_init(&ms.barS[0], 1);
+        mbar_init(&ms.barS[1], 1);
+        mbar_init(&ms.barP, kSoftmaxThreads);
+        mbar_init(&ms.barO, 1);
+        ms.abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (tid < kBM) {
+        const int jj = n_full + tid;
+        ms.pos[tid] = jj < n_end ? sm_idx[(size_t)bh * L + jj] : 0x7fffffff;
+    }
+    if (warp == 4) tmem_alloc(&ms.tmem_base, 256);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ms.tmem_base;
+    const uint32_t tS[2] = {tmem, tmem + 64}, tO = tmem + 128;
+    volatile int *abort_flag = &ms.abort_flag;
+
+    if (warp == 5) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
+            mbar_arrive_expect_tx(&ms.barQ, SL::kQBytes);
+            for (int kb = 0; kb < KB; ++kb)
+                tma_load_4d(smem + SL::oQ + kb * kBM * 128, &map_q, &ms.barQ, kb * 64, h, p * kBM, b);
+            int t = 0;
+            for (; t < T; ++t) {
+                const int s = t % kStages;
+                if (!mbar_wait(&ms.empty[s], ((t / kStages) & 1) ^ 1, abort_flag)) break;
+                mbar_arrive_expect_tx(&ms.full[s], SL::kKStage + SL::kVStage);
+                for (int kb = 0; kb < KB; ++kb) {
+                    tma_load_2d(smem + SL::oK + s * SL::kKStage + kb * kBN * 128, &map_k, &ms.full[s],
+                                kb * 64, bh * cap + t * kBN);
+                    tma_load_2d(smem + SL::oV + s * SL::kVStage + kb * kBN * 128, &map_v, &ms.full[s],
+                                kb * 64, bh * capv + t * kBN);
+                }
+            }
+            // on an aborted run: let the copies already issued land before the CTA retires
+            if (*abort_flag)
+                for (int u = max(0, t - kStages); u < t; ++u)
+                    mbar_wait(&ms.full[u % kStages], (u / kStages) & 1, abort_flag);
+        }
+    } else if (warp == 4) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0 && T > 0) {
+            constexpr uint32_t idesc_qk = make_idesc(kFmtBF16, kBM, kBN, false, false);
+            constexpr uint32_t idesc_pv = make_idesc(kFmtF16, kBM, D, false, true);
+            const uint32_t aQ = smem_u32(smem + SL::oQ), aP = smem_u32(smem + SL::oP);
+            auto issue_qk = [&](int t) {
+                const uint32_t aK = smem_u32(smem + SL::oK + (t % kStages) * SL::kKStage);
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                    for (int k16 = 0; k16 < 4; ++k16)
+                        mma_ss(tS[t & 1], desc_kmajor(aQ + kb * kBM * 128 + k16 * 32),
+                               desc_kmajor(aK + kb * kBN * 128 + k16 * 32), idesc_qk,
+                               (kb | k16) != 0);
+                mma_commit(&ms.barS[t & 1]);
+            };
+            bool ok = mbar_wait(&ms.barQ, 0, abort_flag) && mbar_wait(&ms.full[0], 0, abort_flag);
+            if (ok) {
+                tc_fence_after_sync();
+                issue_qk(0);
+            }
+            for (int t = 0; ok && t < T; ++t) {
+                if (t + 1 < T) {
+                    ok = mbar_wait(&ms.full[(t + 1) % kStages], ((t + 1) / kStages) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_qk(t + 1);
+                }
+                ok = mbar_wait(&ms.barP, t & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t aV = smem_u32(smem + SL::oV + (t % kStages) * SL::kVStage);
+#pragma unroll
+                for (int k16 = 0; k16 < 4; ++k16)
+                    mma_ss(tO, desc_kmajor(aP + k16 * 32), desc_mnmajor(aV + k16 * 2048, kBN * 128),
+                           idesc_pv, (t | k16) != 0);
+                mma_commit(&ms.empty[t % kStages]);
+                mma_commit(&ms.barO);
+            }
+        }
+    } else {
+        // ------------------------------ softmax + epilogue ------------------------------
+        const int r = tid;                              // query row inside the tile, TMEM lane
+        const int i_abs = p * kBM + r;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        const float sl2 = scale_sm * 1.4426950408889634f;
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int t = 0; t < T; ++t) {
+            ok = mbar_wait(&ms.barS[t & 1], (t >> 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            uint32_t sv[2][32];
+            tmem_ld32(tS[t & 1] + lane_base, sv[0]);
+            tmem_ld32(tS[t & 1] + lane_base + 32, sv[1]);
+            tmem_wait_ld();
+            float x[kBN];
+#pragma unroll
+            for (int c = 0; c < kBN; ++c) x[c] = __uint_as_float(sv[c >> 5][c & 31]) * sl2;
+            const int j0 = t * kBN;
+            if (j0 + kBN > n_full) {                    // tile reaches into the CTA's own chunks
+#pragma unroll
+                for (int c = 0; c < kBN; ++c) {
+                    const int jj = j0 + c;
+                    const bool vis = jj < n_full || (jj < n_end && ms.pos[jj - n_full] <= i_abs);
+                    x[c] = vis ? x[c] : -INFINITY;
+                }
+            }
+            float mx = x[0];
+#pragma unroll
+            for (int c = 1; c < kBN; ++c) mx = fmaxf(mx, x[c]);
+            const float m_new = fmaxf(m, mx);
+            const float m_use = m_new == -INFINITY ? 0.f : m_new;
+            const float corr = exp2f(m - m_use);        // m = -inf -> 0
+            float psum = 0.f;
+#pragma unroll
+            for (int c = 0; c < kBN; ++c) {
+                x[c] = exp2f(x[c] - m_use);
+                psum += x[c];
+            }
+            l = l * corr + psum;
+            m = m_new;
+            if (t > 0) {
+                ok = mbar_wait(&ms.barO, (t - 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (__any_sync(0xffffffffu, corr != 1.f)) {
+#pragma unroll
+                    for (int cb = 0; cb < D / 32; ++cb) {
+                        uint32_t ov[32];
+                        tmem_ld32(tO + lane_base + cb * 32, ov);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) ov[c] = __float_as_uint(__uint_as_float(ov[c]) * corr);
+                        tmem_st32(tO + lane_base + cb * 32, ov);
+                    }
+                    tmem_wait_st();
+                }
+            }
+            uint8_t *prow = smem + SL::oP;
+#pragma unroll
+            for (int pc = 0; pc < 8; ++pc) {
+                uint4 u;
+                u.x = pack_half2(x[8 * pc + 0], x[8 * pc + 1]);
+                u.y = pack_half2(x[8 * pc + 2], x[8 * pc + 3]);
+                u.z = pack_half2(x[8 * pc + 4], x[8 * pc + 5]);
+                u.w = pack_half2(x[8 * pc + 6], x[8 * pc + 7]);
+                *reinterpret_cast<uint4 *>(prow + sw128_offset(r, pc)) = u;
+            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&ms.barP);
+        }
+        if (ok && T > 0) {
+            ok = mbar_wait(&ms.barO, (T - 1) & 1, abort_flag);
+            tc_fence_after_sync();
+        }
+        if (ok && i_abs < L) {
+            const size_t tok = ((size_t)b * L + i_abs) * H + h;
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            const float *ol = o_la + tok * D;
+            float ssn = 0.f, ssl = 0.f;
+#pragma unroll
+            for (int cb = 0; cb < D / 32; ++cb) {
+                uint32_t ov[32];
+                if (T > 0) {
+                    tmem_ld32(tO + lane_base + cb * 32, ov);
+                    tmem_wait_ld();
+                }
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const float on = l > 0.f ? __uint_as_float(ov[c]) * inv : 0.f;
+                    ssn = fmaf(on, on, ssn);
+                }
+#pragma unroll
+                for (int c4 = 0; c4 < 8; ++c4) {
+                    const float4 a = __ldg(reinterpret_cast<const float4 *>(ol + cb * 32) + c4);
+                    ssl = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, ssl))));
+                }
+            }
+            const float fn = rsqrtf(ssn / D + eps), fl = rsqrtf(ssl / D + eps);
+            const float wn = (w ? w[tok * 2] : 0.5f) * fn, wl = (w ? w[tok * 2 + 1] : 0.5f) * fl;
+#pragma unroll
+            for (int cb = 0; cb < D / 32; ++cb) {
+                uint32_t ov[32];
+                if (T > 0) {
+                    tmem_ld32(tO + lane_base + cb * 32, ov);
+                    tmem_wait_ld();
+                }
+                float on[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) on[c] = l > 0.f ? __uint_as_float(ov[c]) * inv : 0.f;
+                if (o_nla) {
+#pragma unroll
+                    for (int c4 = 0; c4 < 8; ++c4)
+                        reinterpret_cast<float4 *>(o_nla + tok * D + cb * 32)[c4] =
+                            make_float4(on[4 * c4], on[4 * c4 + 1], on[4 * c4 + 2], on[4 * c4 + 3]);
+                }
+                if (out) {
+                    float4 a[8];
+#pragma unroll
+                    for (int c4 = 0; c4 < 8; ++c4)
+                        a[c4] = __ldg(reinterpret_cast<const float4 *>(ol + cb * 32) + c4);
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const float4 a0 = a[2 * q4], a1 = a[2 * q4 + 1];
+                        const float *o8 = on + 8 * q4;
+                        uint4 u;
+                        u.x = pack_bf162(fmaf(wn, o8[0], wl * a0.x), fmaf(wn, o8[1], wl * a0.y));
+                        u.y = pack_bf162(fmaf(wn, o8[2], wl * a0.z), fmaf(wn, o8[3], wl * a0.w));
+                        u.z = pack_bf162(fmaf(wn, o8[4], wl * a1.x), fmaf(wn, o8[5], wl * a1.y));
+                        u.w = pack_bf162(fmaf(wn, o8[6], wl * a1.z), fmaf(wn, o8[7], wl * a1.w));
+                        reinterpret_cast<uint4 *>(out + tok * D + cb * 32)[q4] = u;
+                    }
+                }
+            }
+            if (lse) lse[(size_t)bh * L + i_abs] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        }
+    }
+    // ------------------------------ teardown ------------------------------
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, 256);
+    }
+    if (tid == 0 && ms.abort_flag) atomicMin(status, (int)NATSL_ERR_TIMEOUT);
+}
+
+// Copy the retained tokens' K rows (bf16) and V rows (as fp16) into the compacted layouts
+// [B,H,cap,d] / [B,H,capv,d] and zero the V rows up to the next multiple of 64, so that a K/V
+// tile never multiplies a zero probability with an uninitialised value.  grid = (row blocks, B*H).
+template <int D>
+__global__ void __launch_bounds__(256)
+gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__restrict__ v,
+                    const int32_t *__restrict__ sm_idx, const int32_t *__restrict__ sm_chunk_prefix,
+                    __nv_bfloat16 *__restrict__ k_sm, __nv_bfloat16 *__restrict__ v_sm,
+                    __half *__restrict__ v16, int cap, int capv, int32_t *status, int L, int H) {
+    constexpr int kVecPerRow = D * 2 / 16;
+    constexpr int kRows = 256 / kVecPerRow;
+    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int NC = L / kC;
+    const int n_sm = sm_chunk_prefix[(size_t)bh * (NC + 1) + NC];
+    if (blockIdx.x == 0 && threadIdx.x == 0 && n_sm > cap) atomicMin(status, (int)NATSL_ERR_CACHE_FULL);
+    const int n = min(n_sm, cap);
+    const int n_pad = min((n + kBN - 1) / kBN * kBN, capv);
+    const int row = blockIdx.x * kRows + threadIdx.x / kVecPerRow;
+    const int piece = threadIdx.x % kVecPerRow;
+    if (row >= n_pad) return;
+    uint4 *dv16 = reinterpret_cast<uint4 *>(v16 + ((size_t)bh * capv + row) * D) + piece;
+    if (row >= n) {
+        *dv16 = make_uint4(0u, 0u, 0u, 0u);
+        return;
+    }
+    const int tok = sm_idx[(size_t)bh * L + row];
+    const size_t src = (((size_t)b * L + tok) * H + h) * D;
+    const size_t dst = ((size_t)bh * cap + row) * D;
+    reinterpret_cast<uint4 *>(k_sm + dst)[piece] = reinterpret_cast<const uint4 *>(k + src)[piece];
+    const uint4 vv = reinterpret_cast<const uint4 *>(v + src)[piece];
+    if (v_sm) reinterpret_cast<uint4 *>(v_sm + dst)[piece] = vv;
+    const uint32_t wv[4] = {vv.x, vv.y, vv.z, vv.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        o[i] = pack_half2(__uint_as_float(wv[i] << 16), __uint_as_float(wv[i] & 0xffff0000u));
+    *dv16 = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+}  // namespace
+
+template <int D>
+static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *v16, int32_t cap,
+                                   int32_t capv, const int32_t *sm_idx, const int32_t *pre,
+                                   const float *o_la, const float *w, float scale_sm, float eps,
+                                   void *out, float *o_nla, float *lse, int32_t *status, Shape s,
+                                   cudaStream_t st) {
+    using SL = SmLayout<D>;
+    CUtensorMap mq, mk, mv;
+    if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, kBM) ||
+        !tch::make_map_2d(&mk, k_sm, (uint64_t)s.B * s.H * cap, D, kBN) ||
+        !tch::make_map_2d(&mv, v16, (uint64_t)s.B * s.H * capv, D, kBN))
+        return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(softmax_combine_tc_kernel<D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal);
+    if (e != cudaSuccess) return e;
+    dim3 grid((s.L + kBM - 1) / kBM, s.B * s.H);
+    softmax_combine_tc_kernel<D><<<grid, kThreadsTc, SL::kTotal, st>>>(
+        mq, mk, mv, cap, capv, sm_idx, pre, o_la, w, scale_sm, eps, (__nv_bfloat16 *)out, o_nla, lse,
+        status, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const void *v16, int32_t cap,
+                                      int32_t capv, const int32_t *sm_idx,
+                                      const int32_t *sm_chunk_prefix, const float *o_la,
+                                      const float *w, float scale_sm, float eps, void *out,
+                                      float *o_nla, float *lse, int32_t *status, Shape s,
+                                      cudaStream_t st) {
+    if (s.d == 128)
+        return softmax_tc_impl<128>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la, w,
+                                    scale_sm, eps, out, o_nla, lse, status, s, st);
+    return softmax_tc_impl<64>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la, w, scale_sm,
+                               eps, out, o_nla, lse, status, s, st);
+}
+
+template <int D>
+static cudaError_t gather_tc_impl(const void *k, const void *v, const int32_t *sm_idx,
+                                  const int32_t *pre, void *k_sm, void *v_sm, void *v16, int cap,
+                                  int capv, int32_t *status, Shape s, cudaStream_t st) {
+    constexpr int kRows = 256 / (D * 2 / 16);
+    const int max_rows = s.L < capv ? s.L : capv;
+    dim3 grid((max_rows + kRows - 1) / kRows, s.B * s.H);
+    gather_kv_tc_kernel<D><<<grid, 256, 0, st>>>(
+        (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, sm_idx, pre, (__nv_bfloat16 *)k_sm,
+        (__nv_bfloat16 *)v_sm, (__half *)v16, cap, capv, status, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
+                                const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
+                                int32_t cap, int32_t capv, int32_t *status, Shape s,
+                                cudaStream_t st) {
+    if (s.d == 128)
+        return gather_tc_impl<128>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, cap, capv, status, s, st);
+    return gather_tc_impl<64>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, cap, capv, status, s, st);
+}
+
+}  // namespace natsl
