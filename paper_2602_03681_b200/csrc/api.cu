@@ -48,9 +48,14 @@ Shape shape_of(const natsl_params *p) { return Shape{p->B, p->H, p->L, p->d, p->
 struct FwdWs {
     int32_t *status, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
     void *k_sm, *v_sm, *v16;
-    float *W, *U, *P, *o_la;
+    float *W, *U, *P, *o_la;    // W, U, P: fp32 CUDA-core path only
+    GdnTcWs tc;                 // tensor-core path only
     size_t bytes;
 };
+
+bool use_tensor_cores(const natsl_params *p) {
+    return p->dtype == NATSL_BF16 && !(p->flags & NATSL_FORCE_SIMT);
+}
 
 FwdWs carve_fwd(const natsl_params *p, void *ws) {
     Carver c(ws);
@@ -65,10 +70,22 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
     f.sm_len = c.take<int32_t>(B * H);
     f.k_sm = c.take<char>(B * H * L * d * esz);
     f.v_sm = c.take<char>(B * H * L * d * esz);
-    f.v16 = c.take<char>(p->dtype == NATSL_BF16 ? B * H * L * d * 2 : 0);   // fp16 V of the retained tokens
-    f.W = c.take<float>(B * L * H * d);
-    f.U = c.take<float>(B * L * H * d);
-    f.P = c.take<float>(B * H * NC * kC * kC);
+    if (use_tensor_cores(p)) {
+        f.v16 = c.take<char>(B * H * L * d * 2);          // fp16 V of the retained tokens
+        f.tc.Qh = c.take<char>(B * H * L * d * 2);
+        f.tc.Kh = c.take<char>(B * H * L * d * 2);
+        f.tc.Wt = c.take<char>(B * H * L * d * 2);
+        f.tc.Ut = c.take<float>(B * H * L * d);
+        f.tc.Ph = c.take<char>(B * H * NC * kC * kC * 2);
+        f.tc.Gc = c.take<float>(B * H * L);
+        f.W = f.U = f.P = nullptr;
+    } else {
+        f.v16 = nullptr;
+        f.tc = GdnTcWs{};
+        f.W = c.take<float>(B * L * H * d);
+        f.U = c.take<float>(B * L * H * d);
+        f.P = c.take<float>(B * H * NC * kC * kC);
+    }
     f.o_la = c.take<float>(B * L * H * d);
     f.bytes = c.off;
     return f;
@@ -197,7 +214,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     const int32_t cap = want_cache ? p->sm_cap : p->L;
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, sm_len, p->B, p->L,
                                    p->H, st));
-    const bool tensor_cores = s.bf16 && !(p->flags & NATSL_FORCE_SIMT);
+    const bool tensor_cores = use_tensor_cores(p);
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
                                       f.v16, cap, p->L, f.status, s, st));
@@ -205,11 +222,18 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
     NATSL_TRY(mark());
     float *o_la = p->o_la ? p->o_la : f.o_la;
-    NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P, nullptr,
-                                      nullptr, s, st));
-    NATSL_TRY(mark());
-    NATSL_TRY(launch_gdn_scan_simt(q, k, g, f.W, f.U, f.P, p->scale_la, p->state_in, p->state_out,
-                                   nullptr, nullptr, o_la, s, st));
+    if (tensor_cores) {
+        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, f.status, s, st));
+        NATSL_TRY(mark());
+        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, p->state_out, o_la, f.status, s,
+                                     st));
+    } else {
+        NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P,
+                                          nullptr, nullptr, s, st));
+        NATSL_TRY(mark());
+        NATSL_TRY(launch_gdn_scan_simt(q, k, g, f.W, f.U, f.P, p->scale_la, p->state_in,
+                                       p->state_out, nullptr, nullptr, o_la, s, st));
+    }
     NATSL_TRY(mark());
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, p->L, f.sm_idx, f.prefix, o_la, p->w,

@@ -1,0 +1,699 @@
+// Tensor-core chunkwise Gated DeltaNet (Section 3, chunkwise equations, specialised to the gated
+// delta rule of Section 4.3; decay applied on every token, state update only for linear tokens)
+// for bf16 storage on sm_100a: a chunk-parallel "prepare" kernel and a sequential "scan" kernel.
+//
+// Notation per chunk of C = 64 tokens: beta~ = (1 - route) beta, G_i = inclusive cumulative log
+// decay, gamma_i = exp(G_i), Gamma_ij = exp(G_i - G_j) (j <= i):
+//   A_ij = beta~_i Gamma_ij (k_i.k_j) (j < i),  T = (I + A)^-1,
+//   U = T diag(beta~) V,  W = T diag(beta~ gamma) K,  P_ij = scale_la Gamma_ij (q_i.k_j) (j <= i)
+//   U~ = U - W S;  O = scale_la diag(gamma) Q S + P U~;  S <- gamma_C S + (diag(gamma_C/gamma) K)^T U~
+//
+// Precision.  q, k, v are exact bf16 inputs, but T, W, U~, P and S are computed quantities: an
+// 8-bit significand on them puts the layer output 1.4-2e-2 x RMS off (the whole error budget), so
+// every tensor-core operand here is fp16 (11-bit significand; the inputs convert exactly, all
+// magnitudes are O(1) and decay factors only shrink them), T is solved in fp32, and U, which is
+// only ever added to an accumulator, stays fp32.
+//
+// All products are laid out "transposed", with the head dimension on the MMA's M axis
+// (M = 128 rows = TMEM lanes = one thread each) and the 64 tokens of a chunk on N or K, so that
+// every operand a thread has to produce is one contiguous 128-byte row of a swizzled tile.
+#include "common.cuh"
+#include "natsl_internal.h"
+#include "tc_common.cuh"
+
+namespace natsl {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kRowThreads = 128;
+
+// bf16 -> fp16, 8 values in place
+__device__ __forceinline__ uint4 bf16x8_to_f16x8(uint4 u) {
+    const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        o[i] = pack_half2(__uint_as_float(wv[i] << 16), __uint_as_float(wv[i] & 0xffff0000u));
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// ==========================================================================================
+// Prepare: one CTA per pair of chunks of one (batch, head).  Threads 0..127 own one token each
+// (thread r <-> token r of the pair) up to the triangular solve, and one head-dimension row each
+// afterwards; warp 4 issues TMA and MMAs.
+// ==========================================================================================
+constexpr int kPrepThreads = 160;
+constexpr int kPrepMisc = 2048;
+
+template <int D> struct PrepLayout {
+    static constexpr int KB = D / 64;
+    static constexpr int kTile = KB * 128 * 128;           // 128 tokens x D 16-bit values
+    static constexpr int oV = 0;
+    static constexpr int oK = oV + kTile;                  // directly after V (D = 64 stacks them)
+    static constexpr int oX = oK + kTile;                  // Q tile, then A^T (fp32), then T operands
+    static constexpr int kX = kTile > 32768 ? kTile : 32768;
+    static constexpr int oMisc = oX + kX;
+    static constexpr int kTotal = oMisc + kPrepMisc;
+};
+
+struct PrepMisc {
+    uint64_t barLoad, barConv, barM, barXfree, barT, barUW;
+    uint32_t tmem_base;
+    int abort_flag;
+    float G[128], bt[128], wsum[4];
+};
+static_assert(sizeof(PrepMisc) <= kPrepMisc, "misc page too small");
+
+template <int D>
+__global__ void __launch_bounds__(kPrepThreads)
+gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
+                      const __grid_constant__ CUtensorMap map_k,
+                      const __grid_constant__ CUtensorMap map_v,
+                      const __grid_constant__ CUtensorMap map_qh,
+                      const __grid_constant__ CUtensorMap map_kh, const float *__restrict__ g,
+                      const float *__restrict__ beta, const uint8_t *__restrict__ route,
+                      float scale_la, __half *__restrict__ Wt, float *__restrict__ Ut,
+                      __half *__restrict__ Ph, float *__restrict__ Gc, int32_t *status, int L,
+                      int H) {
+    using PL = PrepLayout<D>;
+    constexpr int KB = PL::KB;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    PrepMisc &ms = *reinterpret_cast<PrepMisc *>(smem + PL::oMisc);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int NC = L / kC;
+    const int pr = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int tok_first = pr * 128;                    // first token of the pair
+    const bool second_valid = 2 * pr + 1 < NC;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (tid == 0) atomicMin(status, (int)NATSL_ERR_CUDA);
+        return;
+    }
+    if (tid == 0) {
+        mbar_init(&ms.barLoad, 1);
+        mbar_init(&ms.barConv, kRowThreads);
+        mbar_init(&ms.barM, 1);
+        mbar_init(&ms.barXfree, 1);
+        mbar_init(&ms.barT, kRowThreads);
+        mbar_init(&ms.barUW, 1);
+        ms.abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 4) tmem_alloc(&ms.tmem_base, 256);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ms.tmem_base;
+    volatile int *abort_flag = &ms.abort_flag;
+    uint8_t *sV = smem + PL::oV, *sK = smem + PL::oK, *sX = smem + PL::oX;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            // ---- loads ----
+            mbar_arrive_expect_tx(&ms.barLoad, 3 * PL::kTile);
+            for (int kb = 0; kb < KB; ++kb) {
+                tma_load_4d(sK + kb * 16384, &map_k, &ms.barLoad, kb * 64, h, tok_first, b);
+                tma_load_4d(sX + kb * 16384, &map_q, &ms.barLoad, kb * 64, h, tok_first, b);
+                tma_load_4d(sV + kb * 16384, &map_v, &ms.barLoad, kb * 64, h, tok_first, b);
+            }
+            bool ok = mbar_wait(&ms.barConv, 0, abort_flag);       // tiles converted to fp16
+            if (ok) {
+                // ---- fp16 copies of q and k for the scan kernel; K K^T and Q K^T ----
+                const int row0 = bh * L + tok_first;
+                for (int kb = 0; kb < KB; ++kb)
+                    for (int hf = 0; hf < (second_valid ? 2 : 1); ++hf) {
+                        tma_store_2d(&map_qh, sX + kb * 16384 + hf * 8192, kb * 64, row0 + hf * 64);
+                        tma_store_2d(&map_kh, sK + kb * 16384 + hf * 8192, kb * 64, row0 + hf * 64);
+                    }
+                tma_store_commit();
+                tc_fence_after_sync();
+                constexpr uint32_t idesc = make_idesc(kFmtF16, 128, 128, false, false);
+                const uint32_t aK = smem_u32(sK), aQ = smem_u32(sX);
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                    for (int k16 = 0; k16 < 4; ++k16) {
+                        const uint64_t dk = desc_kmajor(aK + kb * 16384 + k16 * 32);
+                        mma_ss(tmem, dk, dk, idesc, (kb | k16) != 0);
+                        mma_ss(tmem + 128, desc_kmajor(aQ + kb * 16384 + k16 * 32), dk, idesc,
+                               (kb | k16) != 0);
+                    }
+                mma_commit(&ms.barM);
+                tma_store_wait_read();                    // the q copy has left its tile
+                ok = mbar_wait(&ms.barM, 0, abort_flag);  // and Q K^T has read it
+                mbar_arrive(&ms.barXfree);
+            }
+            if (ok) ok = mbar_wait(&ms.barT, 0, abort_flag);
+            if (ok) {
+                // ---- U^T = V^T (T beta~)^T,  W^T = K^T (T beta~ gamma)^T, per chunk ----
+                tc_fence_after_sync();
+                const uint32_t aV = smem_u32(sV), aK = smem_u32(sK), aT = smem_u32(sX);
+                if (D == 128) {
+                    constexpr uint32_t idesc = make_idesc(kFmtF16, 128, 64, true, false);
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                        for (int k16 = 0; k16 < 4; ++k16) {
+                            mma_ss(tmem + 64 * hf,
+                                   desc_mnmajor(aV + hf * 8192 + k16 * 2048, 16384),
+                                   desc_kmajor(aT + hf * 16384 + k16 * 32), idesc, k16 != 0);
+                            mma_ss(tmem + 128 + 64 * hf,
+                                   desc_mnmajor(aK + hf * 8192 + k16 * 2048, 16384),
+                                   desc_kmajor(aT + hf * 16384 + 8192 + k16 * 32), idesc, k16 != 0);
+                        }
+                } else {
+                    // d = 64: rows 0-63 of M are V^T, rows 64-127 are K^T (the K tile follows the V
+                    // tile in shared memory); N = 128 = [T beta~ ; T beta~ gamma].
+                    constexpr uint32_t idesc = make_idesc(kFmtF16, 128, 128, true, false);
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                        for (int k16 = 0; k16 < 4; ++k16)
+                            mma_ss(tmem + 128 * hf,
+                                   desc_mnmajor(aV + hf * 8192 + k16 * 2048, 16384),
+                                   desc_kmajor(aT + hf * 16384 + k16 * 32), idesc, k16 != 0);
+                }
+                mma_commit(&ms.barUW);
+            }
+            tma_store_wait_all();
+        }
+    } else {
+        const int r = tid, hf = r >> 6, i = r & 63;
+        const int c = 2 * pr + hf;                         // this thread's chunk
+        const bool valid = hf == 0 || second_valid;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        // ---- gates: beta~, inclusive cumulative log decay within the chunk ----
+        float gv = 0.f, btv = 0.f;
+        if (valid) {
+            const size_t t = ((size_t)b * L + tok_first + r) * H + h;
+            gv = g[t];
+            btv = route[t] ? 0.f : beta[t];
+        }
+        float G = gv;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float y = __shfl_up_sync(0xffffffffu, G, o);
+            if (lane >= o) G += y;
+        }
+        if (lane == 31) ms.wsum[warp] = G;
+        named_barrier_sync(1, kRowThreads);
+        if (warp & 1) G += ms.wsum[warp - 1];
+        ms.G[r] = G;
+        ms.bt[r] = btv;
+        if (valid) Gc[(size_t)bh * L + tok_first + r] = G;
+        // ---- tiles to fp16, in place ----
+        bool ok = mbar_wait(&ms.barLoad, 0, abort_flag);
+        if (ok) {
+            for (int idx = r; idx < 3 * PL::kTile / 16; idx += kRowThreads) {
+                uint4 *pp = reinterpret_cast<uint4 *>(smem) + idx;   // V, K, Q tiles are contiguous
+                *pp = bf16x8_to_f16x8(*pp);
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&ms.barConv);
+            ok = mbar_wait(&ms.barXfree, 0, abort_flag);
+        }
+        float t[64];
+        if (ok) {
+            // ---- A (strictly lower) -> A^T in shared memory; P (lower) -> global ----
+            tc_fence_after_sync();
+            float *At = reinterpret_cast<float *>(sX) + hf * 4096;   // At[j][m] = A_mj
+            {
+                uint32_t d1[2][32];
+                tmem_ld32(tmem + lane_base + 64 * hf, d1[0]);
+                tmem_ld32(tmem + lane_base + 64 * hf + 32, d1[1]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 64; ++j) {
+                    const float a = j < i ? btv * __expf(G - ms.G[64 * hf + j]) *
+                                                __uint_as_float(d1[j >> 5][j & 31])
+                                          : 0.f;
+                    At[j * 64 + i] = a;
+                }
+            }
+            {
+                uint32_t d2[2][32];
+                tmem_ld32(tmem + 128 + lane_base + 64 * hf, d2[0]);
+                tmem_ld32(tmem + 128 + lane_base + 64 * hf + 32, d2[1]);
+                tmem_wait_ld();
+                uint4 *prow = reinterpret_cast<uint4 *>(Ph + (((size_t)bh * NC + c) * 64 + i) * 64);
+#pragma unroll
+                for (int pc = 0; pc < 8; ++pc) {
+                    float x[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int j = 8 * pc + e;
+                        x[e] = j <= i ? scale_la * __expf(G - ms.G[64 * hf + j]) *
+                                            __uint_as_float(d2[j >> 5][j & 31])
+                                      : 0.f;
+                    }
+                    if (valid)
+                        prow[pc] = make_uint4(pack_half2(x[0], x[1]), pack_half2(x[2], x[3]),
+                                              pack_half2(x[4], x[5]), pack_half2(x[6], x[7]));
+                }
+            }
+            tc_fence_before_sync();
+            named_barrier_sync(1, kRowThreads);
+            // ---- row i of T = (I + A)^-1 by back substitution: t_j = [j = i] - sum_{m > j} t_m A_mj
+#pragma unroll
+            for (int j = 0; j < 64; ++j) t[j] = 0.f;
+#pragma unroll
+            for (int j = 63; j >= 0; --j) {
+                const float4 *col = reinterpret_cast<const float4 *>(At + j * 64);
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                for (int m4 = (j + 1) / 4; m4 < 16; ++m4) {
+                    const float4 a = col[m4];
+                    a0 = fmaf(t[4 * m4], a.x, a0);
+                    a1 = fmaf(t[4 * m4 + 1], a.y, a1);
+                    a2 = fmaf(t[4 * m4 + 2], a.z, a2);
+                    a3 = fmaf(t[4 * m4 + 3], a.w, a3);
+                }
+                t[j] = (j == i ? 1.f : 0.f) - ((a0 + a1) + (a2 + a3));
+            }
+            named_barrier_sync(1, kRowThreads);          // everyone is done reading A^T
+            // ---- operands T diag(beta~) and T diag(beta~ gamma), fp16 rows ----
+            uint8_t *tb = sX + hf * 16384, *tg = tb + 8192;
+#pragma unroll
+            for (int pc = 0; pc < 8; ++pc) {
+                float xb[8], xg[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int j = 8 * pc + e;
+                    xb[e] = t[j] * ms.bt[64 * hf + j];
+                    xg[e] = xb[e] * __expf(ms.G[64 * hf + j]);
+                }
+                *reinterpret_cast<uint4 *>(tb + sw128_offset(i, pc)) =
+                    make_uint4(pack_half2(xb[0], xb[1]), pack_half2(xb[2], xb[3]),
+                               pack_half2(xb[4], xb[5]), pack_half2(xb[6], xb[7]));
+                *reinterpret_cast<uint4 *>(tg + sw128_offset(i, pc)) =
+                    make_uint4(pack_half2(xg[0], xg[1]), pack_half2(xg[2], xg[3]),
+                               pack_half2(xg[4], xg[5]), pack_half2(xg[6], xg[7]));
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&ms.barT);
+            ok = mbar_wait(&ms.barUW, 0, abort_flag);
+        }
+        if (ok) {
+            // ---- U^T (fp32) and W^T (fp16) rows to global; thread r <-> head-dimension row ----
+            tc_fence_after_sync();
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                if (hh == 1 && !second_valid) break;
+                const size_t chunk = (size_t)bh * NC + 2 * pr + hh;
+                const bool do_u = D == 128 || r < 64, do_w = D == 128 || r >= 64;
+                const int row = D == 128 ? r : (r & 63);
+                const int col_u = D == 128 ? 64 * hh : 128 * hh;
+                const int col_w = D == 128 ? 128 + 64 * hh : 128 * hh + 64;
+                uint32_t x[2][32];
+                if (do_u) {                                 // warp-uniform
+                    tmem_ld32(tmem + lane_base + col_u, x[0]);
+                    tmem_ld32(tmem + lane_base + col_u + 32, x[1]);
+                    tmem_wait_ld();
+                    uint4 *dst = reinterpret_cast<uint4 *>(Ut + (chunk * D + row) * 64);
+#pragma unroll
+                    for (int pc = 0; pc < 16; ++pc)
+                        dst[pc] = make_uint4(x[pc >> 3][(4 * pc) & 31], x[pc >> 3][(4 * pc + 1) & 31],
+                                             x[pc >> 3][(4 * pc + 2) & 31], x[pc >> 3][(4 * pc + 3) & 31]);
+                }
+                if (do_w) {
+                    tmem_ld32(tmem + lane_base + col_w, x[0]);
+                    tmem_ld32(tmem + lane_base + col_w + 32, x[1]);
+                    tmem_wait_ld();
+                    uint4 *dst = reinterpret_cast<uint4 *>(Wt + (chunk * D + row) * 64);
+#pragma unroll
+                    for (int pc = 0; pc < 8; ++pc) {
+                        const uint32_t *xx = &x[pc >> 2][(8 * pc) & 31];
+                        dst[pc] = make_uint4(
+                            pack_half2(__uint_as_float(xx[0]), __uint_as_float(xx[1])),
+                            pack_half2(__uint_as_float(xx[2]), __uint_as_float(xx[3])),
+                            pack_half2(__uint_as_float(xx[4]), __uint_as_float(xx[5])),
+                            pack_half2(__uint_as_float(xx[6]), __uint_as_float(xx[7])));
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, 256);
+    }
+    if (tid == 0 && ms.abort_flag) atomicMin(status, (int)NATSL_ERR_TIMEOUT);
+}
+
+// ==========================================================================================
+// Scan: one CTA per (batch, head), sequential over chunks.  Thread r of warps 0-3 owns value
+// column r of the state (row r of S^T, TMEM lane r); warp 4 issues MMAs, warp 5 issues TMA.
+// Per chunk:
+//   D1 = S^T [W ; Q]^T        (columns 0-63: (W S)^T, 64-127: (Q S)^T)
+//   U~^T = U^T - (W S)^T       in registers -> fp16 operands U~ and U~ diag(gamma_C / gamma)
+//   S^T <- gamma_C S^T + (U~ diag(gamma_C/gamma))^T-rows x K ;  D3 = U~^T P^T
+//   o_la^T = scale_la diag(gamma) (Q S)^T + D3
+// ==========================================================================================
+constexpr int kScanThreads = 192;
+constexpr int kScanStages = 2;
+constexpr int kScanMisc = 1024;
+
+template <int D> struct ScanLayout {
+    static constexpr int KB = D / 64;
+    static constexpr int kW = D * 128;                     // W^T tile: D rows x 64 tokens (fp16)
+    static constexpr int kQ = KB * 8192;                   // Q tile: 64 tokens x D
+    static constexpr int kK = KB * 8192;
+    static constexpr int kP = 8192;
+    static constexpr int kG = 256;
+    static constexpr int oW = 0, oQ = oW + kW, oK = oQ + kQ, oP = oK + kK, oG = oP + kP;
+    static constexpr int kStage = ((oG + kG + 1023) / 1024) * 1024;
+    static constexpr int kTx = kW + kQ + kK + kP + kG;
+    static constexpr int oS = kScanStages * kStage;        // S^T operand: 128 rows x D fp16
+    static constexpr int kS = KB * 16384;
+    static constexpr int oU = oS + kS;                     // U~ operand: 128 rows x 64 tokens
+    static constexpr int oUs = oU + 16384;                 // U~ diag(gamma_C / gamma)
+    static constexpr int oMisc = oUs + 16384;
+    static constexpr int kTotal = oMisc + kScanMisc;
+    static constexpr int kTmemCols = D == 128 ? 512 : 256;
+    static constexpr int cS = 0, cD1 = D, cD3 = D + 128;   // TMEM columns
+};
+
+struct ScanMisc {
+    uint64_t full[kScanStages], empty[kScanStages], barA, barD1, barB, barSU, barD3;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+static_assert(sizeof(ScanMisc) <= kScanMisc, "misc page too small");
+
+template <int D>
+__global__ void __launch_bounds__(kScanThreads)
+gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
+                   const __grid_constant__ CUtensorMap map_qh,
+                   const __grid_constant__ CUtensorMap map_kh,
+                   const __grid_constant__ CUtensorMap map_ph, const float *__restrict__ Ut,
+                   const float *__restrict__ Gc, float scale_la,
+                   const float *__restrict__ state_in, float *__restrict__ state_out,
+                   float *__restrict__ o_la, int32_t *status, int L, int H) {
+    using SL = ScanLayout<D>;
+    constexpr int KB = SL::KB;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    ScanMisc &ms = *reinterpret_cast<ScanMisc *>(smem + SL::oMisc);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int NC = L / kC;
+    const int bh = blockIdx.x, b = bh / H, h = bh % H;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (tid == 0) atomicMin(status, (int)NATSL_ERR_CUDA);
+        return;
+    }
+    if (tid == 0) {
+        for (int s = 0; s < kScanStages; ++s) {
+            mbar_init(&ms.full[s], 1);
+            mbar_init(&ms.empty[s], 1 + kRowThreads);   // MMAs done + every row thread done with the decays
+        }
+        mbar_init(&ms.barA, kRowThreads);
+        mbar_init(&ms.barD1, 1);
+        mbar_init(&ms.barB, kRowThreads);
+        mbar_init(&ms.barSU, 1);
+        mbar_init(&ms.barD3, 1);
+        ms.abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 4) tmem_alloc(&ms.tmem_base, SL::kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = ms.tmem_base;
+    volatile int *abort_flag = &ms.abort_flag;
+
+    if (warp == 5) {
+        if (lane == 0) {
+            int c = 0;
+            for (; c < NC; ++c) {
+                const int s = c % kScanStages;
+                if (!mbar_wait(&ms.empty[s], ((c / kScanStages) & 1) ^ 1, abort_flag)) break;
+                uint8_t *st = smem + s * SL::kStage;
+                mbar_arrive_expect_tx(&ms.full[s], SL::kTx);
+                tma_load_2d(st + SL::oW, &map_wt, &ms.full[s], 0, (bh * NC + c) * D);
+                for (int kb = 0; kb < KB; ++kb) {
+                    tma_load_2d(st + SL::oQ + kb * 8192, &map_qh, &ms.full[s], kb * 64, bh * L + c * 64);
+                    tma_load_2d(st + SL::oK + kb * 8192, &map_kh, &ms.full[s], kb * 64, bh * L + c * 64);
+                }
+                tma_load_2d(st + SL::oP, &map_ph, &ms.full[s], 0, (bh * NC + c) * 64);
+                bulk_load_1d(st + SL::oG, Gc + (size_t)bh * L + c * 64, SL::kG, &ms.full[s]);
+            }
+            if (*abort_flag)
+                for (int u = max(0, c - kScanStages); u < c; ++u)
+                    mbar_wait(&ms.full[u % kScanStages], (u / kScanStages) & 1, abort_flag);
+        }
+    } else if (warp == 4) {
+        if (lane == 0) {
+            constexpr uint32_t id_ws = make_idesc(kFmtF16, 128, 64, false, true);    // B = W^T (MN-major)
+            constexpr uint32_t id_qs = make_idesc(kFmtF16, 128, 64, false, false);   // B = Q
+            constexpr uint32_t id_su = make_idesc(kFmtF16, 128, D, false, true);     // B = K (MN-major)
+            constexpr uint32_t id_pu = make_idesc(kFmtF16, 128, 64, false, false);   // B = P
+            const uint32_t aS = smem_u32(smem + SL::oS), aU = smem_u32(smem + SL::oU),
+                           aUs = smem_u32(smem + SL::oUs);
+            for (int c = 0; c < NC; ++c) {
+                const int s = c % kScanStages;
+                const uint32_t st = smem_u32(smem + s * SL::kStage);
+                if (!mbar_wait(&ms.full[s], (c / kScanStages) & 1, abort_flag)) break;
+                if (!mbar_wait(&ms.barA, c & 1, abort_flag)) break;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                    for (int k16 = 0; k16 < 4; ++k16) {
+                        const uint64_t da = desc_kmajor(aS + kb * 16384 + k16 * 32);
+                        mma_ss(tmem + SL::cD1, da,
+                               desc_mnmajor(st + SL::oW + (kb * 4 + k16) * 2048, 0), id_ws,
+                               (kb | k16) != 0);
+                        mma_ss(tmem + SL::cD1 + 64, da,
+                               desc_kmajor(st + SL::oQ + kb * 8192 + k16 * 32), id_qs, (kb | k16) != 0);
+                    }
+                mma_commit(&ms.barD1);
+                if (!mbar_wait(&ms.barB, c & 1, abort_flag)) break;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int k16 = 0; k16 < 4; ++k16)
+                    mma_ss(tmem + SL::cS, desc_kmajor(aUs + k16 * 32),
+                           desc_mnmajor(st + SL::oK + k16 * 2048, 8192), id_su, true);
+                mma_commit(&ms.barSU);
+#pragma unroll
+                for (int k16 = 0; k16 < 4; ++k16)
+                    mma_ss(tmem + SL::cD3, desc_kmajor(aU + k16 * 32),
+                           desc_kmajor(st + SL::oP + k16 * 32), id_pu, k16 != 0);
+                mma_commit(&ms.barD3);
+                mma_commit(&ms.empty[s]);
+            }
+        }
+    } else {
+        const int r = tid;
+        const bool active = r < D;                        // d = 64: rows 64-127 are zero padding
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        float u[64];
+        auto load_u = [&](int c) {
+            if (active) {
+                const float4 *src = reinterpret_cast<const float4 *>(Ut + (((size_t)bh * NC + c) * D + r) * 64);
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const float4 a = __ldg(src + x);
+                    u[4 * x] = a.x; u[4 * x + 1] = a.y; u[4 * x + 2] = a.z; u[4 * x + 3] = a.w;
+                }
+            } else {
+#pragma unroll
+                for (int x = 0; x < 64; ++x) u[x] = 0.f;
+            }
+        };
+        load_u(0);
+        bool ok = true;
+        for (int c = 0; c < NC && ok; ++c) {
+            const int s = c % kScanStages;
+            const float *Gs = reinterpret_cast<const float *>(smem + s * SL::kStage + SL::oG);
+            ok = mbar_wait(&ms.full[s], (c / kScanStages) & 1, abort_flag);
+            if (!ok) break;
+            const float gl = Gs[63], gC = __expf(gl);
+            if (c > 0) {
+                ok = mbar_wait(&ms.barSU, (c - 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+            }
+            // ---- (a) state row -> fp16 operand; decayed row back to TMEM ----
+#pragma unroll
+            for (int cb = 0; cb < D / 32; ++cb) {
+                uint32_t sv[32];
+                if (c > 0) {
+                    tmem_ld32(tmem + SL::cS + lane_base + cb * 32, sv);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int x = 0; x < 32; ++x)
+                        sv[x] = (state_in && active)
+                                    ? __float_as_uint(state_in[((size_t)bh * D + cb * 32 + x) * D + r])
+                                    : 0u;
+                }
+                uint8_t *sub = smem + SL::oS + (cb >> 1) * 16384;
+#pragma unroll
+                for (int pc = 0; pc < 4; ++pc) {
+                    const uint32_t *xx = &sv[8 * pc];
+                    *reinterpret_cast<uint4 *>(sub + sw128_offset(r, (cb & 1) * 4 + pc)) = make_uint4(
+                        pack_half2(__uint_as_float(xx[0]), __uint_as_float(xx[1])),
+                        pack_half2(__uint_as_float(xx[2]), __uint_as_float(xx[3])),
+                        pack_half2(__uint_as_float(xx[4]), __uint_as_float(xx[5])),
+                        pack_half2(__uint_as_float(xx[6]), __uint_as_float(xx[7])));
+                }
+#pragma unroll
+                for (int x = 0; x < 32; ++x) sv[x] = __float_as_uint(__uint_as_float(sv[x]) * gC);
+                tmem_st32(tmem + SL::cS + lane_base + cb * 32, sv);
+            }
+            tmem_wait_st();
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&ms.barA);
+            // ---- (b) U~ = U - W S ----
+            ok = mbar_wait(&ms.barD1, c & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            {
+                uint32_t ws[2][32];
+                tmem_ld32(tmem + SL::cD1 + lane_base, ws[0]);
+                tmem_ld32(tmem + SL::cD1 + lane_base + 32, ws[1]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 64; ++j) u[j] -= __uint_as_float(ws[j >> 5][j & 31]);
+            }
+#pragma unroll
+            for (int pc = 0; pc < 8; ++pc) {
+                float xs[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) xs[e] = u[8 * pc + e] * __expf(gl - Gs[8 * pc + e]);
+                *reinterpret_cast<uint4 *>(smem + SL::oU + sw128_offset(r, pc)) =
+                    make_uint4(pack_half2(u[8 * pc], u[8 * pc + 1]), pack_half2(u[8 * pc + 2], u[8 * pc + 3]),
+                               pack_half2(u[8 * pc + 4], u[8 * pc + 5]), pack_half2(u[8 * pc + 6], u[8 * pc + 7]));
+                *reinterpret_cast<uint4 *>(smem + SL::oUs + sw128_offset(r, pc)) =
+                    make_uint4(pack_half2(xs[0], xs[1]), pack_half2(xs[2], xs[3]),
+                               pack_half2(xs[4], xs[5]), pack_half2(xs[6], xs[7]));
+            }
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&ms.barB);
+            // ---- (c) output rows of this chunk ----
+            float qs[64];
+            {
+                uint32_t x[2][32];
+                tmem_ld32(tmem + SL::cD1 + 64 + lane_base, x[0]);
+                tmem_ld32(tmem + SL::cD1 + 64 + lane_base + 32, x[1]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 64; ++i)
+                    qs[i] = scale_la * __expf(Gs[i]) * __uint_as_float(x[i >> 5][i & 31]);
+            }
+            mbar_arrive(&ms.empty[s]);                    // last read of this stage's decay values
+            if (c + 1 < NC) load_u(c + 1);                // next chunk's U row, hidden behind the rest
+            ok = mbar_wait(&ms.barD3, c & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
+            {
+                uint32_t x[2][32];
+                tmem_ld32(tmem + SL::cD3 + lane_base, x[0]);
+                tmem_ld32(tmem + SL::cD3 + lane_base + 32, x[1]);
+                tmem_wait_ld();
+                if (active) {
+                    float *dst = o_la + (((size_t)b * L + (size_t)c * 64) * H + h) * D + r;
+#pragma unroll
+                    for (int i = 0; i < 64; ++i)
+                        dst[(size_t)i * H * D] = qs[i] + __uint_as_float(x[i >> 5][i & 31]);
+                }
+            }
+            tc_fence_before_sync();
+        }
+        if (ok && state_out) {
+            ok = mbar_wait(&ms.barSU, (NC - 1) & 1, abort_flag);
+            if (ok) {
+                tc_fence_after_sync();
+#pragma unroll
+                for (int cb = 0; cb < D / 32; ++cb) {
+                    uint32_t sv[32];
+                    tmem_ld32(tmem + SL::cS + lane_base + cb * 32, sv);
+                    tmem_wait_ld();
+                    if (active) {
+#pragma unroll
+                        for (int x = 0; x < 32; ++x)
+                            state_out[((size_t)bh * D + cb * 32 + x) * D + r] = __uint_as_float(sv[x]);
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem, SL::kTmemCols);
+    }
+    if (tid == 0 && ms.abort_flag) atomicMin(status, (int)NATSL_ERR_TIMEOUT);
+}
+
+}  // namespace
+
+template <int D>
+static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, const float *g,
+                                   const float *beta, const uint8_t *route, float scale_la,
+                                   const GdnTcWs &ws, int32_t *status, Shape s, cudaStream_t st) {
+    const int NC = s.L / kC;
+    const uint64_t BH = (uint64_t)s.B * s.H;
+    CUtensorMap mq, mk, mv, mqh, mkh;
+    if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, 128) ||
+        !tch::make_map_blhd(&mk, k, s.B, s.L, s.H, D, 128) ||
+        !tch::make_map_blhd(&mv, v, s.B, s.L, s.H, D, 128) ||
+        !tch::make_map_2d(&mqh, ws.Qh, BH * s.L, D, 64) ||
+        !tch::make_map_2d(&mkh, ws.Kh, BH * s.L, D, 64))
+        return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(gdn_prepare_tc_kernel<D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         PrepLayout<D>::kTotal);
+    if (e != cudaSuccess) return e;
+    dim3 grid((NC + 1) / 2, s.B * s.H);
+    gdn_prepare_tc_kernel<D><<<grid, kPrepThreads, PrepLayout<D>::kTotal, st>>>(
+        mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut, (__half *)ws.Ph, ws.Gc,
+        status, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <int D>
+static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *state_in,
+                                float *state_out, float *o_la, int32_t *status, Shape s,
+                                cudaStream_t st) {
+    const int NC = s.L / kC;
+    const uint64_t BH = (uint64_t)s.B * s.H;
+    CUtensorMap mwt, mqh, mkh, mph;
+    if (!tch::make_map_2d(&mwt, ws.Wt, BH * NC * D, 64, D) ||
+        !tch::make_map_2d(&mqh, ws.Qh, BH * s.L, D, 64) ||
+        !tch::make_map_2d(&mkh, ws.Kh, BH * s.L, D, 64) ||
+        !tch::make_map_2d(&mph, ws.Ph, BH * NC * 64, 64, 64))
+        return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(gdn_scan_tc_kernel<D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         ScanLayout<D>::kTotal);
+    if (e != cudaSuccess) return e;
+    gdn_scan_tc_kernel<D><<<s.B * s.H, kScanThreads, ScanLayout<D>::kTotal, st>>>(
+        mwt, mqh, mkh, mph, ws.Ut, ws.Gc, scale_la, state_in, state_out, o_la, status, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, const float *g,
+                                  const float *beta, const uint8_t *route, float scale_la,
+                                  const GdnTcWs &ws, int32_t *status, Shape s, cudaStream_t st) {
+    if (s.d == 128) return prepare_tc_impl<128>(q, k, v, g, beta, route, scale_la, ws, status, s, st);
+    return prepare_tc_impl<64>(q, k, v, g, beta, route, scale_la, ws, status, s, st);
+}
+
+cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
+                               float *state_out, float *o_la, int32_t *status, Shape s,
+                               cudaStream_t st) {
+    if (s.d == 128) return scan_tc_impl<128>(ws, scale_la, state_in, state_out, o_la, status, s, st);
+    return scan_tc_impl<64>(ws, scale_la, state_in, state_out, o_la, status, s, st);
+}
+
+}  // namespace natsl

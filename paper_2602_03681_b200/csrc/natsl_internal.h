@@ -55,6 +55,21 @@ cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const voi
                                       float *o_nla, float *lse, int32_t *status, Shape s,
                                       cudaStream_t st);
 
+// gdn_tc.cu -- tensor-core chunkwise Gated DeltaNet (bf16 storage): intermediates in workspace
+struct GdnTcWs {
+    void *Qh, *Kh;   // fp16 copies of q, k              [B,H,L,d]
+    void *Wt;        // W^T per chunk, fp16              [B,H,L/C,d,64]
+    float *Ut;       // U^T per chunk, fp32              [B,H,L/C,d,64]
+    void *Ph;        // P per chunk, fp16                [B,H,L/C,64,64]
+    float *Gc;       // in-chunk cumulative log decay    [B,H,L]
+};
+cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, const float *g,
+                                  const float *beta, const uint8_t *route, float scale_la,
+                                  const GdnTcWs &ws, int32_t *status, Shape s, cudaStream_t st);
+cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
+                               float *state_out, float *o_la, int32_t *status, Shape s,
+                               cudaStream_t st);
+
 // bwd_simt.cu -- fp32 CUDA-core backward
 // A batched matrix operand: element (r, c) of batch (b, h, chunk) is
 // p[b*sb + h*sh + chunk*sc + r*ld + c].
