@@ -1,0 +1,134 @@
+"""GPU parity of the tensor-core (tcgen05) forward, the default path for bf16 storage, against the
+fp64 oracle: small and ragged shapes (one chunk, odd chunk counts, half-filled last query tile),
+both head sizes, degenerate routings, initial state, prefill -> decode cache hand-off, extreme
+decays, and agreement with the library's fp32 CUDA-core path."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_03681_b200 import inputs
+from test_gpu_parity import TOL, check_fwd, check_stored, dev, rel_err, run_fwd, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,B,H,L", [("cfg1_bf16_prefill", 1, 1, 64),      # a single chunk
+                                        ("cfg1_bf16_prefill", 2, 3, 192),     # odd number of chunks
+                                        ("cfg1_bf16_prefill", 1, 2, 1088),    # several K/V tiles + tail
+                                        ("cfg4_bf16_train", 1, 1, 64),
+                                        ("cfg4_bf16_train", 2, 2, 448),
+                                        ("cfg2_bf16_long_prefill", 1, 3, 1536)])
+def test_fwd_tensor_core_small_cases(name, B, H, L):
+    wl = inputs.WORKLOADS[name]
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L)
+    check_fwd(wl, run_fwd(wl, x), run_oracle(wl, x), TOL["bf16"])
+
+
+@pytest.mark.parametrize("name", ["cfg1_bf16_prefill", "cfg4_bf16_train"])
+def test_fwd_tensor_core_initial_state_and_default_weights(name):
+    wl = inputs.WORKLOADS[name]
+    B, H, L = 2, 2, 320
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L)
+    S0 = (0.1 * np.random.default_rng(5).standard_normal((B, H, wl.d, wl.d))).astype(np.float32)
+    check_fwd(wl, run_fwd(wl, x, state_in=S0, w=None), run_oracle(wl, x, state_in=S0, w=None),
+              TOL["bf16"])
+
+
+@pytest.mark.parametrize("name", ["cfg1_bf16_prefill", "cfg4_bf16_train"])
+def test_fwd_tensor_core_degenerate_routes(name):
+    wl = inputs.WORKLOADS[name]
+    B, H, L = 1, 2, 256
+    for fill in (0, 1):
+        x = inputs.make_layer_inputs(wl, B=B, H=H, L=L, route=np.full((B, L, H), fill, np.uint8))
+        got, ref = run_fwd(wl, x), run_oracle(wl, x)
+        check_fwd(wl, got, ref, TOL["bf16"])
+        if fill == 0:                      # nothing retained: the softmax branch is exactly empty
+            assert np.all(got["o_nla"] == 0) and np.all(np.isneginf(got["lse"]))
+        else:                              # nothing folded: the state only decays from zero
+            assert np.all(got["o_la"] == 0) and np.all(got["state_out"] == 0)
+
+
+def test_fwd_tensor_core_single_retained_token_and_late_first_token():
+    """Queries before the first retained token see an empty set; after it, exactly v of that token."""
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    B, H, L = 1, 2, 256
+    route = np.zeros((B, L, H), np.uint8)
+    route[0, 70, 0] = 1
+    route[0, 200, 1] = 1
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L, route=route)
+    got, ref = run_fwd(wl, x), run_oracle(wl, x)
+    check_fwd(wl, got, ref, TOL["bf16"])
+    for h, first in ((0, 70), (1, 200)):
+        assert np.all(got["o_nla"][0, :first, h] == 0)
+        assert np.allclose(got["o_nla"][0, first:, h], x["v"][0, first, h], rtol=2e-3, atol=1e-6)
+
+
+def test_fwd_tensor_core_cache_handoff_matches_oracle():
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    B, H, L = 2, 3, 512
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L)
+    dt = torch.bfloat16
+    cap = 160
+    res = binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]),
+                             dev(x["beta"]), dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la,
+                             scale_sm=wl.scale_sm, want=("cache", "o_nla", "lse"), sm_cap=cap)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(res["ws"]) == 0
+    ref = run_oracle(wl, x, want_cache=True)
+    n = res["sm_len"].cpu().numpy()
+    assert np.array_equal(n, ref["n_sm"]) and n.max() <= cap
+    for b in range(B):
+        for h in range(H):
+            m = n[b, h]
+            assert np.array_equal(res["k_sm"][b, h, :m].float().cpu().numpy(),
+                                  ref["k_sm"][b, h, :m].astype(np.float32))
+            assert np.array_equal(res["v_sm"][b, h, :m].float().cpu().numpy(),
+                                  ref["v_sm"][b, h, :m].astype(np.float32))
+    assert rel_err(res["o_nla"].cpu().numpy(), ref["o_nla"]) <= TOL["bf16"]
+    check_stored(res["out"].float().cpu().numpy(), ref["out"], TOL["bf16"], "bf16")
+
+
+def test_fwd_tensor_core_cache_too_small_is_reported():
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    x = inputs.make_layer_inputs(wl, B=1, H=1, L=256, route=np.ones((1, 256, 1), np.uint8))
+    dt = torch.bfloat16
+    res = binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]),
+                             dev(x["beta"]), dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la,
+                             scale_sm=wl.scale_sm, want=("cache",), sm_cap=64)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(res["ws"]) == binding.ERR_CACHE_FULL
+    assert torch.isfinite(res["out"].float()).all()
+
+
+@pytest.mark.parametrize("g_value", [0.0, -3.0])
+def test_fwd_tensor_core_decay_extremes(g_value):
+    """No decay at all, and a decay strong enough that in-chunk factors underflow to zero."""
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    B, H, L = 1, 2, 256
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L)
+    x["g"] = np.full((B, L, H), g_value, np.float32)
+    got, ref = run_fwd(wl, x), run_oracle(wl, x)
+    assert np.isfinite(got["out"]).all() and np.isfinite(got["o_la"]).all()
+    check_fwd(wl, got, ref, TOL["bf16"])
+
+
+def test_fwd_tensor_core_agrees_with_cuda_core_path():
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    x = inputs.make_layer_inputs(wl, B=1, H=4, L=768)
+    a = run_fwd(wl, x)
+    b = run_fwd(wl, x, flags=binding.FORCE_SIMT)
+    for name in ("o_la", "o_nla", "state_out"):
+        assert rel_err(a[name], b[name]) <= TOL["bf16"], name
+    assert np.array_equal(np.isneginf(a["lse"]), np.isneginf(b["lse"]))
+
+
+def test_fwd_tensor_core_is_deterministic():
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    x = inputs.make_layer_inputs(wl, B=1, H=2, L=512)
+    a, b = run_fwd(wl, x), run_fwd(wl, x)
+    for name in ("out", "o_la", "o_nla", "lse", "state_out"):
+        assert np.array_equal(a[name], b[name]), name
