@@ -77,7 +77,7 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
         f.tc.Wt = c.take<char>(B * H * L * d * 2);
         f.tc.Ut = c.take<float>(B * H * L * d);
         f.tc.Ph = c.take<char>(B * H * NC * kC * kC * 2);
-        f.tc.Gc = c.take<float>(B * H * L);
+        f.tc.Gd = c.take<float>(B * H * L * 2);
         f.W = f.U = f.P = nullptr;
     } else {
         f.v16 = nullptr;

@@ -75,7 +75,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                       const __grid_constant__ CUtensorMap map_kh, const float *__restrict__ g,
                       const float *__restrict__ beta, const uint8_t *__restrict__ route,
                       float scale_la, __half *__restrict__ Wt, float *__restrict__ Ut,
-                      __half *__restrict__ Ph, float *__restrict__ Gc, int32_t *status, int L,
+                      __half *__restrict__ Ph, float *__restrict__ Gd, int32_t *status, int L,
                       int H) {
     using PL = PrepLayout<D>;
     constexpr int KB = PL::KB;
@@ -202,7 +202,6 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         if (warp & 1) G += ms.wsum[warp - 1];
         ms.G[r] = G;
         ms.bt[r] = btv;
-        if (valid) Gc[(size_t)bh * L + tok_first + r] = G;
         // ---- tiles to fp16, in place ----
         bool ok = mbar_wait(&ms.barLoad, 0, abort_flag);
         if (ok) {
@@ -219,6 +218,11 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             // ---- A (strictly lower) -> A^T in shared memory; P (lower) -> global ----
             tc_fence_after_sync();
             float *At = reinterpret_cast<float *>(sX) + hf * 4096;   // At[j][m] = A_mj
+            if (valid) {      // decay factors the scan needs: gamma_i and gamma_C / gamma_i
+                float *gd = Gd + ((size_t)bh * NC + c) * 128;
+                gd[i] = __expf(G);
+                gd[64 + i] = __expf(ms.G[64 * hf + 63] - G);
+            }
             {
                 uint32_t d1[2][32];
                 tmem_ld32(tmem + lane_base + 64 * hf, d1[0]);
@@ -311,10 +315,12 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     tmem_ld32(tmem + lane_base + col_u, x[0]);
                     tmem_ld32(tmem + lane_base + col_u + 32, x[1]);
                     tmem_wait_ld();
-                    uint4 *dst = reinterpret_cast<uint4 *>(Ut + (chunk * D + row) * 64);
+                    // piece-major: 16-byte piece pc (4 tokens) of all D rows is contiguous, so that a
+                    // warp's stores here and its loads in the scan are fully coalesced
+                    uint4 *dst = reinterpret_cast<uint4 *>(Ut + chunk * D * 64) + row;
 #pragma unroll
                     for (int pc = 0; pc < 16; ++pc)
-                        dst[pc] = make_uint4(x[pc >> 3][(4 * pc) & 31], x[pc >> 3][(4 * pc + 1) & 31],
+                        dst[pc * D] = make_uint4(x[pc >> 3][(4 * pc) & 31], x[pc >> 3][(4 * pc + 1) & 31],
                                              x[pc >> 3][(4 * pc + 2) & 31], x[pc >> 3][(4 * pc + 3) & 31]);
                 }
                 if (do_w) {
@@ -345,17 +351,22 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 }
 
 // ==========================================================================================
-// Scan: one CTA per (batch, head), sequential over chunks.  Thread r of warps 0-3 owns value
-// column r of the state (row r of S^T, TMEM lane r); warp 4 issues MMAs, warp 5 issues TMA.
-// Per chunk:
-//   D1 = S^T [W ; Q]^T        (columns 0-63: (W S)^T, 64-127: (Q S)^T)
-//   U~^T = U^T - (W S)^T       in registers -> fp16 operands U~ and U~ diag(gamma_C / gamma)
-//   S^T <- gamma_C S^T + (U~ diag(gamma_C/gamma))^T-rows x K ;  D3 = U~^T P^T
-//   o_la^T = scale_la diag(gamma) (Q S)^T + D3
+// Scan: one CTA per (batch, head), sequential over chunks.  Value column r of the state (row r of
+// S^T, TMEM lane r) belongs to the two threads (r, half 0) and (r, half 1) of warps q and q + 4,
+// which split every row between them; warp 8 issues MMAs, warp 9 issues TMA.  The fp32 state
+// lives in the registers of its two threads (half a row each); per chunk c:
+//   (a) S_c (fp16 operand) -> shared memory;                 MMA: WS = S^T W^T, QS = S^T Q^T
+//   (b) U~^T = U^T - WS  -> operands U~ and U~ diag(gamma_C/gamma);
+//                                      MMA: dS = (U~ diag(gamma_C/gamma))^T-rows x K,  D3 = U~^T P^T
+//   (c) [for chunk c-1, behind the MMAs of (b)]  o_la^T = scale_la diag(gamma) QS + D3
+//   next chunk: S_{c+1} = gamma_C S_c + dS
+// QS and D3 are double-buffered in TMEM so that (c) of chunk c-1 runs behind the MMAs of chunk c.
 // ==========================================================================================
-constexpr int kScanThreads = 192;
+constexpr int kScanRowThreads = 256;
+constexpr int kScanThreads = 320;
 constexpr int kScanStages = 2;
 constexpr int kScanMisc = 1024;
+constexpr int kDecaySlots = 4;                             // ring of per-chunk decay factors
 
 template <int D> struct ScanLayout {
     static constexpr int KB = D / 64;
@@ -363,38 +374,40 @@ template <int D> struct ScanLayout {
     static constexpr int kQ = KB * 8192;                   // Q tile: 64 tokens x D
     static constexpr int kK = KB * 8192;
     static constexpr int kP = 8192;
-    static constexpr int kG = 256;
-    static constexpr int oW = 0, oQ = oW + kW, oK = oQ + kQ, oP = oK + kK, oG = oP + kP;
-    static constexpr int kStage = ((oG + kG + 1023) / 1024) * 1024;
-    static constexpr int kTx = kW + kQ + kK + kP + kG;
+    static constexpr int kG = 512;                         // gamma_i and gamma_C / gamma_i, 64 each
+    static constexpr int oW = 0, oQ = oW + kW, oK = oQ + kQ, oP = oK + kK;
+    static constexpr int kStage = oP + kP;
+    static constexpr int kTx = kStage + kG;
     static constexpr int oS = kScanStages * kStage;        // S^T operand: 128 rows x D fp16
     static constexpr int kS = KB * 16384;
     static constexpr int oU = oS + kS;                     // U~ operand: 128 rows x 64 tokens
     static constexpr int oUs = oU + 16384;                 // U~ diag(gamma_C / gamma)
-    static constexpr int oMisc = oUs + 16384;
+    static constexpr int oG = oUs + 16384;                 // decay ring
+    static constexpr int oMisc = oG + kDecaySlots * kG;
     static constexpr int kTotal = oMisc + kScanMisc;
-    static constexpr int kTmemCols = D == 128 ? 512 : 256;
-    static constexpr int cS = 0, cD1 = D, cD3 = D + 128;   // TMEM columns
+    static constexpr int kTmemCols = 512;
+    static constexpr int cS = 0, cWS = D, cQS = D + 64, cD3 = D + 192;   // TMEM columns
 };
 
 struct ScanMisc {
-    uint64_t full[kScanStages], empty[kScanStages], barA, barD1, barB, barSU, barD3;
+    uint64_t full[kScanStages], empty[kScanStages], barA, barWS, barQS[2], barB, barSU, barD3[2];
     uint32_t tmem_base;
     int abort_flag;
 };
 static_assert(sizeof(ScanMisc) <= kScanMisc, "misc page too small");
 
 template <int D>
-__global__ void __launch_bounds__(kScanThreads)
+__global__ void __launch_bounds__(kScanThreads, 1)
 gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                    const __grid_constant__ CUtensorMap map_qh,
                    const __grid_constant__ CUtensorMap map_kh,
                    const __grid_constant__ CUtensorMap map_ph, const float *__restrict__ Ut,
-                   const float *__restrict__ Gc, float scale_la,
+                   const float *__restrict__ Gd, float scale_la,
                    const float *__restrict__ state_in, float *__restrict__ state_out,
                    float *__restrict__ o_la, int32_t *status, int L, int H) {
     using SL = ScanLayout<D>;
     constexpr int KB = SL::KB;
+    constexpr int kHalfCols = D / 2;                       // state columns per thread
     extern __shared__ __align__(1024) uint8_t smem[];
     ScanMisc &ms = *reinterpret_cast<ScanMisc *>(smem + SL::oMisc);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -406,26 +419,23 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
         return;
     }
     if (tid == 0) {
-        for (int s = 0; s < kScanStages; ++s) {
-            mbar_init(&ms.full[s], 1);
-            mbar_init(&ms.empty[s], 1 + kRowThreads);   // MMAs done + every row thread done with the decays
-        }
-        mbar_init(&ms.barA, kRowThreads);
-        mbar_init(&ms.barD1, 1);
-        mbar_init(&ms.barB, kRowThreads);
+        for (int s = 0; s < kScanStages; ++s) { mbar_init(&ms.full[s], 1); mbar_init(&ms.empty[s], 1); }
+        mbar_init(&ms.barA, kScanRowThreads);
+        mbar_init(&ms.barB, kScanRowThreads);
+        mbar_init(&ms.barWS, 1);
         mbar_init(&ms.barSU, 1);
-        mbar_init(&ms.barD3, 1);
+        for (int s = 0; s < 2; ++s) { mbar_init(&ms.barQS[s], 1); mbar_init(&ms.barD3[s], 1); }
         ms.abort_flag = 0;
         fence_mbar_init();
     }
-    if (warp == 4) tmem_alloc(&ms.tmem_base, SL::kTmemCols);
+    if (warp == 8) tmem_alloc(&ms.tmem_base, SL::kTmemCols);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = ms.tmem_base;
     volatile int *abort_flag = &ms.abort_flag;
 
-    if (warp == 5) {
+    if (warp == 9) {
         if (lane == 0) {
             int c = 0;
             for (; c < NC; ++c) {
@@ -439,13 +449,16 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                     tma_load_2d(st + SL::oK + kb * 8192, &map_kh, &ms.full[s], kb * 64, bh * L + c * 64);
                 }
                 tma_load_2d(st + SL::oP, &map_ph, &ms.full[s], 0, (bh * NC + c) * 64);
-                bulk_load_1d(st + SL::oG, Gc + (size_t)bh * L + c * 64, SL::kG, &ms.full[s]);
+                // A decay slot is reused four chunks later, i.e. only after the stage of chunk c + 2
+                // has been released, which every row thread's work on chunk c precedes.
+                bulk_load_1d(smem + SL::oG + (c % kDecaySlots) * SL::kG,
+                             Gd + ((size_t)bh * NC + c) * 128, SL::kG, &ms.full[s]);
             }
             if (*abort_flag)
                 for (int u = max(0, c - kScanStages); u < c; ++u)
                     mbar_wait(&ms.full[u % kScanStages], (u / kScanStages) & 1, abort_flag);
         }
-    } else if (warp == 4) {
+    } else if (warp == 8) {
         if (lane == 0) {
             constexpr uint32_t id_ws = make_idesc(kFmtF16, 128, 64, false, true);    // B = W^T (MN-major)
             constexpr uint32_t id_qs = make_idesc(kFmtF16, 128, 64, false, false);   // B = Q
@@ -462,163 +475,178 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
-                    for (int k16 = 0; k16 < 4; ++k16) {
-                        const uint64_t da = desc_kmajor(aS + kb * 16384 + k16 * 32);
-                        mma_ss(tmem + SL::cD1, da,
+                    for (int k16 = 0; k16 < 4; ++k16)
+                        mma_ss(tmem + SL::cWS, desc_kmajor(aS + kb * 16384 + k16 * 32),
                                desc_mnmajor(st + SL::oW + (kb * 4 + k16) * 2048, 0), id_ws,
                                (kb | k16) != 0);
-                        mma_ss(tmem + SL::cD1 + 64, da,
+                mma_commit(&ms.barWS);
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                    for (int k16 = 0; k16 < 4; ++k16)
+                        mma_ss(tmem + SL::cQS + 64 * (c & 1), desc_kmajor(aS + kb * 16384 + k16 * 32),
                                desc_kmajor(st + SL::oQ + kb * 8192 + k16 * 32), id_qs, (kb | k16) != 0);
-                    }
-                mma_commit(&ms.barD1);
+                mma_commit(&ms.barQS[c & 1]);
                 if (!mbar_wait(&ms.barB, c & 1, abort_flag)) break;
                 tc_fence_after_sync();
 #pragma unroll
                 for (int k16 = 0; k16 < 4; ++k16)
                     mma_ss(tmem + SL::cS, desc_kmajor(aUs + k16 * 32),
-                           desc_mnmajor(st + SL::oK + k16 * 2048, 8192), id_su, true);
+                           desc_mnmajor(st + SL::oK + k16 * 2048, 8192), id_su, k16 != 0);
                 mma_commit(&ms.barSU);
 #pragma unroll
                 for (int k16 = 0; k16 < 4; ++k16)
-                    mma_ss(tmem + SL::cD3, desc_kmajor(aU + k16 * 32),
+                    mma_ss(tmem + SL::cD3 + 64 * (c & 1), desc_kmajor(aU + k16 * 32),
                            desc_kmajor(st + SL::oP + k16 * 32), id_pu, k16 != 0);
-                mma_commit(&ms.barD3);
+                mma_commit(&ms.barD3[c & 1]);
                 mma_commit(&ms.empty[s]);
             }
         }
     } else {
-        const int r = tid;
+        const int q = warp & 3, half = warp >> 2;
+        const int r = q * 32 + lane;                      // value column / TMEM lane
         const bool active = r < D;                        // d = 64: rows 64-127 are zero padding
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        float u[64];
-        auto load_u = [&](int c) {
-            if (active) {
-                const float4 *src = reinterpret_cast<const float4 *>(Ut + (((size_t)bh * NC + c) * D + r) * 64);
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        const int col0 = half * kHalfCols;                // this thread's state columns (key dim)
+        const int tk0 = half * 32;                        // ... and its tokens of every chunk
+        float S[kHalfCols];                               // fp32 state, already decayed to chunk entry
 #pragma unroll
-                for (int x = 0; x < 16; ++x) {
-                    const float4 a = __ldg(src + x);
+        for (int x = 0; x < kHalfCols; ++x)
+            S[x] = (state_in && active) ? state_in[((size_t)bh * D + col0 + x) * D + r] : 0.f;
+        // This thread's 8 pieces (4 tokens each) of row r of U^T of chunk c.
+        auto u_src = [&](int c) {
+            return reinterpret_cast<const float4 *>(Ut + ((size_t)bh * NC + c) * D * 64) + (tk0 / 4) * D + r;
+        };
+        // The U row of the next chunk is only pulled into L2 ahead of time and loaded into registers
+        // right before it is used: a global load left in flight across TMEM loads makes their
+        // consumers wait for it as well.
+        auto prefetch_u = [&](int c) {
+            if (active) {
+                const float4 *src = u_src(c);
+#pragma unroll
+                for (int x = 0; x < 8; ++x) prefetch_l2(src + x * D);
+            }
+        };
+        // (c): output rows of chunk c (its QS / D3 buffers and decay slot are still intact)
+        auto emit = [&](int c) -> bool {
+            const float *e1 = reinterpret_cast<const float *>(smem + SL::oG + (c % kDecaySlots) * SL::kG);
+            if (!mbar_wait(&ms.barQS[c & 1], (c >> 1) & 1, abort_flag)) return false;
+            if (!mbar_wait(&ms.barD3[c & 1], (c >> 1) & 1, abort_flag)) return false;
+            tc_fence_after_sync();
+            float *dst = o_la + (((size_t)b * L + (size_t)c * 64 + tk0) * H + h) * D + r;
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {        // 16 tokens at a time keeps registers low
+                uint32_t x[16], y[16];
+                tmem_ld16(tmem + SL::cQS + 64 * (c & 1) + tk0 + 16 * part + lane_base, x);
+                tmem_ld16(tmem + SL::cD3 + 64 * (c & 1) + tk0 + 16 * part + lane_base, y);
+                tmem_wait_ld();
+                if (active) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        dst[(size_t)(16 * part + i) * H * D] =
+                            fmaf(scale_la * e1[tk0 + 16 * part + i], __uint_as_float(x[i]),
+                                 __uint_as_float(y[i]));
+                }
+            }
+            tc_fence_before_sync();
+            return true;
+        };
+        prefetch_u(0);
+        bool ok = true;
+        for (int c = 0; c < NC && ok; ++c) {
+            const int s = c % kScanStages;
+            const float *e1 = reinterpret_cast<const float *>(smem + SL::oG + (c % kDecaySlots) * SL::kG);
+            const float *e2 = e1 + 64;
+            ok = mbar_wait(&ms.full[s], (c / kScanStages) & 1, abort_flag);
+            if (!ok) break;
+            if (c > 0) {                                   // S_c = gamma_C S_{c-1} + dS_{c-1}
+                ok = mbar_wait(&ms.barSU, (c - 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after_sync();
+#pragma unroll
+                for (int cb = 0; cb < kHalfCols / 32; ++cb) {
+                    uint32_t ds[32];
+                    tmem_ld32(tmem + SL::cS + col0 + cb * 32 + lane_base, ds);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) S[cb * 32 + x] += __uint_as_float(ds[x]);
+                }
+                tc_fence_before_sync();
+            }
+            // ---- (a) state row -> fp16 operand; decay the register copy to the next chunk entry
+            {
+                uint8_t *sub = smem + SL::oS + (col0 >> 6) * 16384;
+                const int piece0 = (col0 & 63) >> 3;
+#pragma unroll
+                for (int pc = 0; pc < kHalfCols / 8; ++pc)
+                    *reinterpret_cast<uint4 *>(sub + sw128_offset(r, piece0 + pc)) = make_uint4(
+                        pack_half2(S[8 * pc], S[8 * pc + 1]), pack_half2(S[8 * pc + 2], S[8 * pc + 3]),
+                        pack_half2(S[8 * pc + 4], S[8 * pc + 5]), pack_half2(S[8 * pc + 6], S[8 * pc + 7]));
+            }
+            fence_proxy_async_smem();
+            mbar_arrive(&ms.barA);
+            float u[32];                                   // from L2; lands while W S is computed
+            if (active) {
+                const float4 *src = u_src(c);
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    const float4 a = __ldg(src + x * D);
                     u[4 * x] = a.x; u[4 * x + 1] = a.y; u[4 * x + 2] = a.z; u[4 * x + 3] = a.w;
                 }
             } else {
 #pragma unroll
-                for (int x = 0; x < 64; ++x) u[x] = 0.f;
+                for (int x = 0; x < 32; ++x) u[x] = 0.f;
             }
-        };
-        load_u(0);
-        bool ok = true;
-        for (int c = 0; c < NC && ok; ++c) {
-            const int s = c % kScanStages;
-            const float *Gs = reinterpret_cast<const float *>(smem + s * SL::kStage + SL::oG);
-            ok = mbar_wait(&ms.full[s], (c / kScanStages) & 1, abort_flag);
-            if (!ok) break;
-            const float gl = Gs[63], gC = __expf(gl);
-            if (c > 0) {
-                ok = mbar_wait(&ms.barSU, (c - 1) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after_sync();
+            {
+                const float gC = e1[63];
+#pragma unroll
+                for (int x = 0; x < kHalfCols; ++x) S[x] *= gC;
             }
-            // ---- (a) state row -> fp16 operand; decayed row back to TMEM ----
-#pragma unroll
-            for (int cb = 0; cb < D / 32; ++cb) {
-                uint32_t sv[32];
-                if (c > 0) {
-                    tmem_ld32(tmem + SL::cS + lane_base + cb * 32, sv);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int x = 0; x < 32; ++x)
-                        sv[x] = (state_in && active)
-                                    ? __float_as_uint(state_in[((size_t)bh * D + cb * 32 + x) * D + r])
-                                    : 0u;
-                }
-                uint8_t *sub = smem + SL::oS + (cb >> 1) * 16384;
-#pragma unroll
-                for (int pc = 0; pc < 4; ++pc) {
-                    const uint32_t *xx = &sv[8 * pc];
-                    *reinterpret_cast<uint4 *>(sub + sw128_offset(r, (cb & 1) * 4 + pc)) = make_uint4(
-                        pack_half2(__uint_as_float(xx[0]), __uint_as_float(xx[1])),
-                        pack_half2(__uint_as_float(xx[2]), __uint_as_float(xx[3])),
-                        pack_half2(__uint_as_float(xx[4]), __uint_as_float(xx[5])),
-                        pack_half2(__uint_as_float(xx[6]), __uint_as_float(xx[7])));
-                }
-#pragma unroll
-                for (int x = 0; x < 32; ++x) sv[x] = __float_as_uint(__uint_as_float(sv[x]) * gC);
-                tmem_st32(tmem + SL::cS + lane_base + cb * 32, sv);
-            }
-            tmem_wait_st();
-            fence_proxy_async_smem();
-            tc_fence_before_sync();
-            mbar_arrive(&ms.barA);
-            // ---- (b) U~ = U - W S ----
-            ok = mbar_wait(&ms.barD1, c & 1, abort_flag);
+            // ---- (b) U~ = U - W S for this thread's 32 tokens ----
+            ok = mbar_wait(&ms.barWS, c & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
             {
-                uint32_t ws[2][32];
-                tmem_ld32(tmem + SL::cD1 + lane_base, ws[0]);
-                tmem_ld32(tmem + SL::cD1 + lane_base + 32, ws[1]);
+                uint32_t ws[32];
+                tmem_ld32(tmem + SL::cWS + tk0 + lane_base, ws);
                 tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 64; ++j) u[j] -= __uint_as_float(ws[j >> 5][j & 31]);
+                for (int j = 0; j < 32; ++j) u[j] -= __uint_as_float(ws[j]);
             }
 #pragma unroll
-            for (int pc = 0; pc < 8; ++pc) {
+            for (int pc = 0; pc < 4; ++pc) {
                 float xs[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) xs[e] = u[8 * pc + e] * __expf(gl - Gs[8 * pc + e]);
-                *reinterpret_cast<uint4 *>(smem + SL::oU + sw128_offset(r, pc)) =
+                for (int e = 0; e < 8; ++e) xs[e] = u[8 * pc + e] * e2[tk0 + 8 * pc + e];
+                *reinterpret_cast<uint4 *>(smem + SL::oU + sw128_offset(r, 4 * half + pc)) =
                     make_uint4(pack_half2(u[8 * pc], u[8 * pc + 1]), pack_half2(u[8 * pc + 2], u[8 * pc + 3]),
                                pack_half2(u[8 * pc + 4], u[8 * pc + 5]), pack_half2(u[8 * pc + 6], u[8 * pc + 7]));
-                *reinterpret_cast<uint4 *>(smem + SL::oUs + sw128_offset(r, pc)) =
+                *reinterpret_cast<uint4 *>(smem + SL::oUs + sw128_offset(r, 4 * half + pc)) =
                     make_uint4(pack_half2(xs[0], xs[1]), pack_half2(xs[2], xs[3]),
                                pack_half2(xs[4], xs[5]), pack_half2(xs[6], xs[7]));
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&ms.barB);
-            // ---- (c) output rows of this chunk ----
-            float qs[64];
-            {
-                uint32_t x[2][32];
-                tmem_ld32(tmem + SL::cD1 + 64 + lane_base, x[0]);
-                tmem_ld32(tmem + SL::cD1 + 64 + lane_base + 32, x[1]);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 64; ++i)
-                    qs[i] = scale_la * __expf(Gs[i]) * __uint_as_float(x[i >> 5][i & 31]);
-            }
-            mbar_arrive(&ms.empty[s]);                    // last read of this stage's decay values
-            if (c + 1 < NC) load_u(c + 1);                // next chunk's U row, hidden behind the rest
-            ok = mbar_wait(&ms.barD3, c & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after_sync();
-            {
-                uint32_t x[2][32];
-                tmem_ld32(tmem + SL::cD3 + lane_base, x[0]);
-                tmem_ld32(tmem + SL::cD3 + lane_base + 32, x[1]);
-                tmem_wait_ld();
-                if (active) {
-                    float *dst = o_la + (((size_t)b * L + (size_t)c * 64) * H + h) * D + r;
-#pragma unroll
-                    for (int i = 0; i < 64; ++i)
-                        dst[(size_t)i * H * D] = qs[i] + __uint_as_float(x[i >> 5][i & 31]);
-                }
-            }
-            tc_fence_before_sync();
+            // ---- behind the MMAs just released: next U row towards L2, previous chunk's output ----
+            if (c + 1 < NC) prefetch_u(c + 1);
+            if (c > 0) ok = emit(c - 1);
         }
+        if (ok) ok = emit(NC - 1);
         if (ok && state_out) {
             ok = mbar_wait(&ms.barSU, (NC - 1) & 1, abort_flag);
             if (ok) {
                 tc_fence_after_sync();
 #pragma unroll
-                for (int cb = 0; cb < D / 32; ++cb) {
-                    uint32_t sv[32];
-                    tmem_ld32(tmem + SL::cS + lane_base + cb * 32, sv);
+                for (int cb = 0; cb < kHalfCols / 32; ++cb) {
+                    uint32_t ds[32];
+                    tmem_ld32(tmem + SL::cS + col0 + cb * 32 + lane_base, ds);
                     tmem_wait_ld();
                     if (active) {
 #pragma unroll
                         for (int x = 0; x < 32; ++x)
-                            state_out[((size_t)bh * D + cb * 32 + x) * D + r] = __uint_as_float(sv[x]);
+                            state_out[((size_t)bh * D + col0 + cb * 32 + x) * D + r] =
+                                S[cb * 32 + x] + __uint_as_float(ds[x]);
                     }
                 }
             }
@@ -626,7 +654,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == 8) {
         tc_fence_after_sync();
         tmem_dealloc(tmem, SL::kTmemCols);
     }
@@ -654,7 +682,7 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
     if (e != cudaSuccess) return e;
     dim3 grid((NC + 1) / 2, s.B * s.H);
     gdn_prepare_tc_kernel<D><<<grid, kPrepThreads, PrepLayout<D>::kTotal, st>>>(
-        mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut, (__half *)ws.Ph, ws.Gc,
+        mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut, (__half *)ws.Ph, ws.Gd,
         status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
@@ -677,7 +705,7 @@ static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *
                                          ScanLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
     gdn_scan_tc_kernel<D><<<s.B * s.H, kScanThreads, ScanLayout<D>::kTotal, st>>>(
-        mwt, mqh, mkh, mph, ws.Ut, ws.Gc, scale_la, state_in, state_out, o_la, status, s.L, s.H);
+        mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, o_la, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }

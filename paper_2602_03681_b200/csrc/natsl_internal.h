@@ -59,9 +59,9 @@ cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const voi
 struct GdnTcWs {
     void *Qh, *Kh;   // fp16 copies of q, k              [B,H,L,d]
     void *Wt;        // W^T per chunk, fp16              [B,H,L/C,d,64]
-    float *Ut;       // U^T per chunk, fp32              [B,H,L/C,d,64]
+    float *Ut;       // U^T per chunk, fp32, in 4-token pieces   [B,H,L/C,16,d,4]
     void *Ph;        // P per chunk, fp16                [B,H,L/C,64,64]
-    float *Gc;       // in-chunk cumulative log decay    [B,H,L]
+    float *Gd;       // per chunk: gamma_i (64), gamma_C / gamma_i (64), fp32   [B,H,L/C,128]
 };
 cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, const float *g,
                                   const float *beta, const uint8_t *route, float scale_la,
