@@ -167,7 +167,7 @@ int natsl_workspace_size(const natsl_params *p, int op, size_t *bytes) {
     switch (op) {
         case NATSL_OP_FWD: *bytes = carve_fwd(p, nullptr).bytes; return NATSL_OK;
         case NATSL_OP_BWD: *bytes = carve_bwd(p, nullptr).bytes; return NATSL_OK;
-        case NATSL_OP_DECODE: *bytes = kStatusBytes; return NATSL_OK;
+        case NATSL_OP_DECODE: *bytes = decode_workspace_bytes(p->B, p->H, p->d); return NATSL_OK;
         case NATSL_OP_COMPACT: *bytes = 0; return NATSL_OK;
         default: return NATSL_ERR_UNSUPPORTED;
     }
@@ -328,10 +328,10 @@ int natsl_decode_step(const void *q, const void *k, const void *v, const float *
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(state) ||
         !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
         return NATSL_ERR_ALIGN;
-    if (!ws || ws_bytes < kStatusBytes) return NATSL_ERR_WORKSPACE;
+    if (!ws || ws_bytes < decode_workspace_bytes(p->B, p->H, p->d)) return NATSL_ERR_WORKSPACE;
     cudaError_t e = launch_decode_step(q, k, v, g, beta, route, p->w, state, k_cache, v_cache,
                                        cache_len, cache_cap, out, p->scale_la, p->scale_sm, p->eps,
-                                       static_cast<int32_t *>(ws), shape_of(p),
+                                       ws, shape_of(p),
                                        static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
 }

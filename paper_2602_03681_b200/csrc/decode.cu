@@ -1,30 +1,46 @@
-// Decode step (Section 4.1, per-token generation): one CTA per (batch, head) streams the fp32
-// d x d state once (decay, rank-1 gated delta update, read-out, write back) and the retained
-// K/V cache once (online softmax), then RMS-normalises and combines both branch outputs
-// (Section 4.3, Norm equation).  HBM-bound: every global access is a 16-byte vector, whole
-// rows per warp instruction, with several independent loads in flight per thread.
+// Decode step (Section 4.1, per-token generation): decay the fp32 d x d state, apply the gated
+// delta rule (linear token) or retain the token's K/V (softmax token), read both branches and
+// combine their RMS-normalised outputs (Section 4.3, Norm equation).
+//
+// HBM-bound: per (sequence, head) the state is read and written once (2 d^2 4 bytes) and the
+// retained K/V are read once.  To keep enough bytes in flight and the SMs evenly loaded, each
+// (sequence, head) is split over kDecodeParts + kStateParts CTAs: a "cache" CTA streams one slice
+// of the retained K/V through a four-stage ring of bulk asynchronous copies (16 KB per stage in
+// flight whatever the arithmetic is doing) and leaves a partial online-softmax result in the
+// workspace; a "state" CTA streams half of the state's value columns through registers (the
+// columns of the delta rule are independent) and leaves its part of the linear read-out there.
+// Whichever CTA of the head finishes last (an atomic ticket, nobody waits) merges the partials,
+// adds the new token's own term, normalises, combines, writes `out`, appends the token to the
+// cache and bumps its length.
 #include "common.cuh"
 #include "natsl_internal.h"
+#include "tc_common.cuh"
 
 namespace natsl {
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
+using namespace tc;
+
+constexpr int kWorkThreads = 256;
+constexpr int kWarps = kWorkThreads / 32;
+constexpr int kThreads = kWorkThreads + 32;      // + one warp that issues the bulk copies
+constexpr int kTileKeys = 32;
+constexpr int kStages = 4;
+constexpr int kStateParts = 2;
+constexpr int kCtasPerHead = kDecodeParts + kStateParts;
 
 template <typename T> struct Vec16;   // 16 bytes of T as fp32 values
 template <> struct Vec16<float> {
     static constexpr int kN = 4;
-    __device__ static void load(const float *p, float (&x)[4]) {
-        const float4 v = __ldg(reinterpret_cast<const float4 *>(p));
-        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    __device__ static void unpack(const uint4 u, float (&x)[4]) {
+        x[0] = __uint_as_float(u.x); x[1] = __uint_as_float(u.y);
+        x[2] = __uint_as_float(u.z); x[3] = __uint_as_float(u.w);
     }
 };
 template <> struct Vec16<__nv_bfloat16> {
     static constexpr int kN = 8;
-    __device__ static void load(const __nv_bfloat16 *p, float (&x)[8]) {
-        const uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
+    __device__ static void unpack(const uint4 u, float (&x)[8]) {
         const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -34,87 +50,192 @@ template <> struct Vec16<__nv_bfloat16> {
     }
 };
 
+// Workspace: [0,256) status word; then tickets [BH] i32; partials [BH][kDecodeParts][D+2] f32
+// (m, z, acc[D]); o_la [BH][D] f32.
+__host__ __device__ inline size_t dec_off_tickets() { return 256; }
+__host__ __device__ inline size_t dec_off_partials(size_t BH) {
+    return (256 + BH * 4 + 255) / 256 * 256;
+}
+__host__ __device__ inline size_t dec_off_ola(size_t BH, int D) {
+    return dec_off_partials(BH) + (BH * kDecodeParts * (D + 2) * 4 + 255) / 256 * 256;
+}
+
 template <typename T, int D>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
                    const float *__restrict__ g, const float *__restrict__ beta,
                    const uint8_t *__restrict__ route, const float *__restrict__ w,
                    float *__restrict__ state, T *__restrict__ k_cache, T *__restrict__ v_cache,
                    int32_t *__restrict__ cache_len, int cap, T *__restrict__ out, float scale_la,
-                   float scale_sm, float eps, int32_t *status) {
-    // state tiling: a lane owns 4 consecutive value columns; a warp instruction covers kRpl rows
-    constexpr int kLpr = D / 4;                 // lanes per state row
-    constexpr int kRpl = 32 / kLpr;             // rows per warp-wide load
-    constexpr int kSlots = kWarps * kRpl;       // row slots in the CTA
-    constexpr int kR = D / kSlots;              // rows per thread
-    // cache tiling: 16-byte pieces, kLpk lanes per key row, kStreams independent softmax streams
-    constexpr int kE = Vec16<T>::kN;
-    constexpr int kLpk = D / kE;
-    constexpr int kStreams = kThreads / kLpk;
-    constexpr int kUnroll = 4;
+                   float scale_sm, float eps, uint8_t *__restrict__ ws, int BH) {
+    constexpr int kE = Vec16<T>::kN;               // elements per 16-byte piece
+    constexpr int kRowBytes = D * (int)sizeof(T);
+    constexpr int kLpk = kRowBytes / 16;           // lanes per key row
+    constexpr int kStreams = kWorkThreads / kLpk;  // independent online-softmax streams
+    constexpr int kTileBytes = kTileKeys * kRowBytes;
+    static_assert(kStreams <= kTileKeys && kTileKeys % kStreams == 0, "tile / stream mismatch");
 
-    __shared__ float qs[D], ks[D], vs[D];
-    __shared__ float red[kSlots][D];
-    __shared__ float o_la_s[D], o_nla_s[D];
-    __shared__ float sm_m[kStreams], sm_z[kStreams];
-    __shared__ float sm_acc[kStreams][D];
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ uint64_t full[kStages], empty[kStages];
+    __shared__ __align__(16) float qs[D], ks[D], vs[D];
+    __shared__ float sm_m[kTileKeys], sm_z[kTileKeys];
     __shared__ float norm_red[2][kWarps];
+    __shared__ int s_last, s_abort;
 
-    const int bh = blockIdx.x;
+    const int part = blockIdx.x, bh = blockIdx.y;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    int32_t *status = reinterpret_cast<int32_t *>(ws);
+    int32_t *ticket = reinterpret_cast<int32_t *>(ws + dec_off_tickets()) + bh;
+    float *partials =
+        reinterpret_cast<float *>(ws + dec_off_partials(BH)) + (size_t)bh * kDecodeParts * (D + 2);
+    float *ola_ws = reinterpret_cast<float *>(ws + dec_off_ola(BH, D)) + (size_t)bh * D;
+
     const int r = route[bh] != 0;
     const int n_old = cache_len[bh];
-    if (r && n_old >= cap) {   // no room: leave the sequence untouched, report
-        if (tid < D) out[(size_t)bh * D + tid] = from_f32<T>(0.f);
-        if (tid == 0) atomicMin(status, (int)NATSL_ERR_CACHE_FULL);
-        return;
-    }
+    const bool cache_full = r && n_old >= cap;     // no room: the sequence is left untouched
     if (tid < D) {
         qs[tid] = to_f32(q[(size_t)bh * D + tid]);
         ks[tid] = to_f32(k[(size_t)bh * D + tid]);
         vs[tid] = to_f32(v[(size_t)bh * D + tid]);
     }
-    const float alpha = __expf(g[bh]);
-    const float bt = r ? 0.f : beta[bh];
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kWorkThreads); }
+        s_abort = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    volatile int *abort_flag = &s_abort;
 
-    // ---------------- linear branch: state in registers ----------------
-    const int slot = warp * kRpl + lane / kLpr;
-    const int col = (lane % kLpr) * 4;
-    float *sp = state + (size_t)bh * D * D;
-    float4 s[kR];
+    if (part < kDecodeParts) {
+        // ---------------- cache CTA: one slice of the retained K/V ----------------
+        const int tiles_total = cache_full ? 0 : (n_old + kTileKeys - 1) / kTileKeys;
+        const int tpp = (tiles_total + kDecodeParts - 1) / kDecodeParts;
+        const int t_begin = min(part * tpp, tiles_total), t_end = min(t_begin + tpp, tiles_total);
+        const uint8_t *kc = reinterpret_cast<const uint8_t *>(k_cache + (size_t)bh * cap * D);
+        const uint8_t *vc = reinterpret_cast<const uint8_t *>(v_cache + (size_t)bh * cap * D);
+        if (warp == kWarps) {
+            if (lane == 0) {
+                int t = t_begin;
+                for (; t < t_end; ++t) {
+                    const int i = t - t_begin, s = i % kStages;
+                    if (!mbar_wait(&empty[s], ((i / kStages) & 1) ^ 1, abort_flag)) break;
+                    const int rows = min(kTileKeys, n_old - t * kTileKeys);
+                    const uint32_t bytes = (uint32_t)rows * kRowBytes;
+                    mbar_arrive_expect_tx(&full[s], 2 * bytes);
+                    bulk_load_1d(smem + (2 * s) * kTileBytes, kc + (size_t)t * kTileBytes, bytes, &full[s]);
+                    bulk_load_1d(smem + (2 * s + 1) * kTileBytes, vc + (size_t)t * kTileBytes, bytes,
+                                 &full[s]);
+                }
+                if (*abort_flag)           // let the copies already issued land before the CTA retires
+                    for (int u = max(t_begin, t - kStages); u < t; ++u)
+                        mbar_wait(&full[(u - t_begin) % kStages], ((u - t_begin) / kStages) & 1,
+                                  abort_flag);
+            }
+        } else {
+            const int stream = tid / kLpk, piece = tid % kLpk;
+            float qf[kE];
 #pragma unroll
-    for (int rr = 0; rr < kR; ++rr)
-        s[rr] = *reinterpret_cast<const float4 *>(sp + (size_t)(slot * kR + rr) * D + col);
-    __syncthreads();   // qs/ks/vs visible
+            for (int x = 0; x < kE; ++x) qf[x] = qs[piece * kE + x] * scale_sm;
+            float m = -INFINITY, z = 0.f, acc[kE];
 #pragma unroll
-    for (int rr = 0; rr < kR; ++rr) {
-        s[rr].x *= alpha; s[rr].y *= alpha; s[rr].z *= alpha; s[rr].w *= alpha;
-    }
-    if (!r) {   // block-uniform
-        float4 p = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int x = 0; x < kE; ++x) acc[x] = 0.f;
+            for (int t = t_begin; t < t_end; ++t) {
+                const int i = t - t_begin, s = i % kStages;
+                if (!mbar_wait(&full[s], (i / kStages) & 1, abort_flag)) break;
+                const uint8_t *kt = smem + (2 * s) * kTileBytes, *vt = kt + kTileBytes;
+                const int rows = min(kTileKeys, n_old - t * kTileKeys);
+#pragma unroll
+                for (int u = 0; u < kTileKeys / kStreams; ++u) {
+                    const int j = u * kStreams + stream;       // trip count uniform over the warp
+                    float kx[kE], vx[kE];
+                    Vec16<T>::unpack(*reinterpret_cast<const uint4 *>(kt + j * kRowBytes + piece * 16), kx);
+                    Vec16<T>::unpack(*reinterpret_cast<const uint4 *>(vt + j * kRowBytes + piece * 16), vx);
+                    float sc = 0.f;
+#pragma unroll
+                    for (int x = 0; x < kE; ++x) sc = fmaf(qf[x], kx[x], sc);
+#pragma unroll
+                    for (int o = kLpk / 2; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                    if (j < rows) {                            // rows past the slice hold stale bytes
+                        const float m_new = fmaxf(m, sc);
+                        const float corr = __expf(m - m_new), pj = __expf(sc - m_new);
+                        z = fmaf(z, corr, pj);
+                        m = m_new;
+#pragma unroll
+                        for (int x = 0; x < kE; ++x) acc[x] = fmaf(acc[x], corr, pj * vx[x]);
+                    }
+                }
+                mbar_arrive(&empty[s]);
+            }
+            // merge the streams of this CTA -> one partial (m, z, acc[D]); the ring is free now
+            float *stage_acc = reinterpret_cast<float *>(smem);   // [kStreams][D]
+            named_barrier_sync(1, kWorkThreads);
+            if (piece == 0) { sm_m[stream] = m; sm_z[stream] = z; }
+#pragma unroll
+            for (int x = 0; x < kE; ++x) stage_acc[stream * D + piece * kE + x] = acc[x];
+            named_barrier_sync(1, kWorkThreads);
+            if (tid < D) {
+                float M = -INFINITY;
+                for (int st = 0; st < kStreams; ++st) M = fmaxf(M, sm_m[st]);
+                float Z = 0.f, o = 0.f;
+                if (M > -INFINITY) {
+                    for (int st = 0; st < kStreams; ++st) {
+                        const float f = __expf(sm_m[st] - M);
+                        Z = fmaf(sm_z[st], f, Z);
+                        o = fmaf(stage_acc[st * D + tid], f, o);
+                    }
+                }
+                float *pp = partials + (size_t)part * (D + 2);
+                pp[2 + tid] = o;
+                if (tid == 0) { pp[0] = M; pp[1] = Z; }
+            }
+        }
+    } else if (warp < kWarps && !cache_full) {
+        // ---------------- state CTA: half of the value columns, all rows ----------------
+        constexpr int kCols = D / kStateParts;      // value columns of this CTA
+        constexpr int kLpr = kCols / 4;             // lanes per (half) state row
+        constexpr int kRpl = 32 / kLpr;             // rows per warp-wide access
+        constexpr int kSlots = kWarps * kRpl;       // row slots in the CTA
+        constexpr int kR = D / kSlots;              // rows per thread
+        static_assert(kSlots <= 32, "reduction scratch too small");
+        float (*redv)[kCols] = reinterpret_cast<float (*)[kCols]>(smem);   // [kSlots][kCols]
+        const int c0 = (part - kDecodeParts) * kCols;
+        const float alpha = __expf(g[bh]);
+        const float bt = r ? 0.f : beta[bh];
+        const int slot = warp * kRpl + lane / kLpr;
+        const int col = (lane % kLpr) * 4;
+        float *sp = state + (size_t)bh * D * D + c0;
+        float4 s[kR];
+#pragma unroll
+        for (int rr = 0; rr < kR; ++rr)
+            s[rr] = *reinterpret_cast<const float4 *>(sp + (size_t)(slot * kR + rr) * D + col);
 #pragma unroll
         for (int rr = 0; rr < kR; ++rr) {
-            const float ka = ks[slot * kR + rr];
-            p.x = fmaf(ka, s[rr].x, p.x); p.y = fmaf(ka, s[rr].y, p.y);
-            p.z = fmaf(ka, s[rr].z, p.z); p.w = fmaf(ka, s[rr].w, p.w);
+            s[rr].x *= alpha; s[rr].y *= alpha; s[rr].z *= alpha; s[rr].w *= alpha;
         }
-        *reinterpret_cast<float4 *>(&red[slot][col]) = p;
-        __syncthreads();
-        float4 e = *reinterpret_cast<const float4 *>(&vs[col]);
+        if (!r) {   // block-uniform
+            float4 p = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int sl = 0; sl < kSlots; ++sl) {
-            const float4 t = *reinterpret_cast<const float4 *>(&red[sl][col]);
-            e.x -= t.x; e.y -= t.y; e.z -= t.z; e.w -= t.w;
-        }
+            for (int rr = 0; rr < kR; ++rr) {
+                const float ka = ks[slot * kR + rr];
+                p.x = fmaf(ka, s[rr].x, p.x); p.y = fmaf(ka, s[rr].y, p.y);
+                p.z = fmaf(ka, s[rr].z, p.z); p.w = fmaf(ka, s[rr].w, p.w);
+            }
+            *reinterpret_cast<float4 *>(&redv[slot][col]) = p;
+            named_barrier_sync(1, kWorkThreads);
+            float4 e = *reinterpret_cast<const float4 *>(&vs[c0 + col]);
 #pragma unroll
-        for (int rr = 0; rr < kR; ++rr) {
-            const float bk = bt * ks[slot * kR + rr];
-            s[rr].x = fmaf(bk, e.x, s[rr].x); s[rr].y = fmaf(bk, e.y, s[rr].y);
-            s[rr].z = fmaf(bk, e.z, s[rr].z); s[rr].w = fmaf(bk, e.w, s[rr].w);
+            for (int sl = 0; sl < kSlots; ++sl) {
+                const float4 t = *reinterpret_cast<const float4 *>(&redv[sl][col]);
+                e.x -= t.x; e.y -= t.y; e.z -= t.z; e.w -= t.w;
+            }
+#pragma unroll
+            for (int rr = 0; rr < kR; ++rr) {
+                const float bk = bt * ks[slot * kR + rr];
+                s[rr].x = fmaf(bk, e.x, s[rr].x); s[rr].y = fmaf(bk, e.y, s[rr].y);
+                s[rr].z = fmaf(bk, e.z, s[rr].z); s[rr].w = fmaf(bk, e.w, s[rr].w);
+            }
+            named_barrier_sync(1, kWorkThreads);   // redv is reused below
         }
-        __syncthreads();   // red is reused below
-    }
-    {
         float4 p = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int rr = 0; rr < kR; ++rr) {
@@ -123,106 +244,64 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
             p.z = fmaf(qa, s[rr].z, p.z); p.w = fmaf(qa, s[rr].w, p.w);
             *reinterpret_cast<float4 *>(sp + (size_t)(slot * kR + rr) * D + col) = s[rr];
         }
-        *reinterpret_cast<float4 *>(&red[slot][col]) = p;
-    }
-    __syncthreads();
-    if (tid < D) {
-        float acc = 0.f;
+        *reinterpret_cast<float4 *>(&redv[slot][col]) = p;
+        named_barrier_sync(1, kWorkThreads);
+        if (tid < kCols) {
+            float a = 0.f;
 #pragma unroll
-        for (int sl = 0; sl < kSlots; ++sl) acc += red[sl][tid];
-        o_la_s[tid] = scale_la * acc;
+            for (int sl = 0; sl < kSlots; ++sl) a += redv[sl][tid];
+            ola_ws[c0 + tid] = scale_la * a;
+        }
     }
 
-    // ---------------- softmax branch: stream the retained K/V once ----------------
-    if (r) {   // append the new token's K/V (the token attends to itself from shared memory)
-        if (tid < D) {
-            k_cache[((size_t)bh * cap + n_old) * D + tid] = k[(size_t)bh * D + tid];
-            v_cache[((size_t)bh * cap + n_old) * D + tid] = v[(size_t)bh * D + tid];
-        }
-        if (tid == 0) cache_len[bh] = n_old + 1;
-    }
-    const int stream = tid / kLpk, piece = tid % kLpk;
-    const T *kc = k_cache + (size_t)bh * cap * D + piece * kE;
-    const T *vc = v_cache + (size_t)bh * cap * D + piece * kE;
-    float qf[kE];
-#pragma unroll
-    for (int x = 0; x < kE; ++x) qf[x] = qs[piece * kE + x] * scale_sm;
-    float m = -INFINITY, z = 0.f, acc[kE];
-#pragma unroll
-    for (int x = 0; x < kE; ++x) acc[x] = 0.f;
-
-    // Trip count and shuffles are uniform over the CTA; only the state updates are predicated.
-    for (int base = 0; base < n_old; base += kStreams * kUnroll) {
-        float kx[kUnroll][kE], vx[kUnroll][kE];
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int j = base + u * kStreams + stream;
-            if (j < n_old) {
-                Vec16<T>::load(kc + (size_t)j * D, kx[u]);
-                Vec16<T>::load(vc + (size_t)j * D, vx[u]);
-            } else {
-#pragma unroll
-                for (int x = 0; x < kE; ++x) { kx[u][x] = 0.f; vx[u][x] = 0.f; }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            const int j = base + u * kStreams + stream;
-            float sc = 0.f;
-#pragma unroll
-            for (int x = 0; x < kE; ++x) sc = fmaf(qf[x], kx[u][x], sc);
-#pragma unroll
-            for (int o = kLpk / 2; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
-            if (j < n_old) {
-                const float m_new = fmaxf(m, sc);
-                const float corr = __expf(m - m_new), pj = __expf(sc - m_new);
-                z = fmaf(z, corr, pj);
-                m = m_new;
-#pragma unroll
-                for (int x = 0; x < kE; ++x) acc[x] = fmaf(acc[x], corr, pj * vx[u][x]);
-            }
-        }
-    }
-    if (r && warp == 0) {   // the token itself, from shared memory; stream 0 takes it
-        float sc = 0.f;
-#pragma unroll
-        for (int x = 0; x < kE; ++x) sc = fmaf(qf[x], ks[piece * kE + x], sc);
-#pragma unroll
-        for (int o = kLpk / 2; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
-        if (stream == 0) {
-            const float m_new = fmaxf(m, sc);
-            const float corr = __expf(m - m_new), pj = __expf(sc - m_new);
-            z = fmaf(z, corr, pj);
-            m = m_new;
-#pragma unroll
-            for (int x = 0; x < kE; ++x) acc[x] = fmaf(acc[x], corr, pj * vs[piece * kE + x]);
-        }
-    }
-    if (piece == 0) { sm_m[stream] = m; sm_z[stream] = z; }
-#pragma unroll
-    for (int x = 0; x < kE; ++x) sm_acc[stream][piece * kE + x] = acc[x];
+    // -------- ticket: the last CTA of this (sequence, head) to get here finishes the step --------
+    __threadfence();
     __syncthreads();
+    if (tid == 0) {
+        const int old = atomicAdd(ticket, 1);
+        s_last = old == kCtasPerHead - 1;
+        if (s_last) *ticket = 0;                      // ready for the next step
+        if (s_abort) atomicMin(status, (int)NATSL_ERR_TIMEOUT);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (cache_full) {
+        if (tid < D) out[(size_t)bh * D + tid] = from_f32<T>(0.f);
+        if (tid == 0) atomicMin(status, (int)NATSL_ERR_CACHE_FULL);
+        return;
+    }
+    float on = 0.f, ol = 0.f;
     if (tid < D) {
+        const volatile float *pv = partials;
         float M = -INFINITY;
-        for (int st = 0; st < kStreams; ++st) M = fmaxf(M, sm_m[st]);
-        float Z = 0.f, o = 0.f;
-        if (M > -INFINITY) {
-            for (int st = 0; st < kStreams; ++st) {
-                const float f = __expf(sm_m[st] - M);
-                Z = fmaf(sm_z[st], f, Z);
-                o = fmaf(sm_acc[st][tid], f, o);
-            }
-            o /= Z;
+        for (int pt = 0; pt < kDecodeParts; ++pt) M = fmaxf(M, pv[pt * (D + 2)]);
+        float sc_self = 0.f;
+        if (r) {                                       // the token attends to itself
+            for (int x = 0; x < D; ++x) sc_self = fmaf(qs[x] * scale_sm, ks[x], sc_self);
+            M = fmaxf(M, sc_self);
         }
-        o_nla_s[tid] = o;
+        float Z = 0.f;
+        if (M > -INFINITY) {
+            for (int pt = 0; pt < kDecodeParts; ++pt) {
+                const float mp = pv[pt * (D + 2)];
+                if (mp > -INFINITY) {
+                    const float f = __expf(mp - M);
+                    Z = fmaf(pv[pt * (D + 2) + 1], f, Z);
+                    on = fmaf(pv[pt * (D + 2) + 2 + tid], f, on);
+                }
+            }
+            if (r) {
+                const float f = __expf(sc_self - M);
+                Z += f;
+                on = fmaf(vs[tid], f, on);
+            }
+            on /= Z;
+        }
+        ol = reinterpret_cast<const volatile float *>(ola_ws)[tid];
     }
-    __syncthreads();
-    // ---------------- combination ----------------
-    float ssn = 0.f, ssl = 0.f;
-    if (tid < D) { ssn = o_nla_s[tid] * o_nla_s[tid]; ssl = o_la_s[tid] * o_la_s[tid]; }
-    ssn = warp_sum(ssn);
-    ssl = warp_sum(ssl);
-    if (lane == 0) { norm_red[0][warp] = ssn; norm_red[1][warp] = ssl; }
+    float ssn = warp_sum(on * on), ssl = warp_sum(ol * ol);
+    if (lane == 0 && warp < kWarps) { norm_red[0][warp] = ssn; norm_red[1][warp] = ssl; }
     __syncthreads();
     if (tid < D) {
         float tn = 0.f, tl = 0.f;
@@ -230,21 +309,38 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
         for (int wv = 0; wv < kWarps; ++wv) { tn += norm_red[0][wv]; tl += norm_red[1][wv]; }
         const float fn = rsqrtf(tn / D + eps), fl = rsqrtf(tl / D + eps);
         const float wn = w ? w[(size_t)bh * 2] : 0.5f, wl = w ? w[(size_t)bh * 2 + 1] : 0.5f;
-        out[(size_t)bh * D + tid] = from_f32<T>(wn * o_nla_s[tid] * fn + wl * o_la_s[tid] * fl);
+        out[(size_t)bh * D + tid] = from_f32<T>(wn * on * fn + wl * ol * fl);
+        if (r) {   // retain the token: every reader of the old length has finished
+            k_cache[((size_t)bh * cap + n_old) * D + tid] = k[(size_t)bh * D + tid];
+            v_cache[((size_t)bh * cap + n_old) * D + tid] = v[(size_t)bh * D + tid];
+        }
     }
+    if (r && tid == 0) cache_len[bh] = n_old + 1;
 }
 
 }  // namespace
+
+size_t decode_workspace_bytes(int B, int H, int d) {
+    return dec_off_ola((size_t)B * H, d) + ((size_t)B * H * d * 4 + 255) / 256 * 256;
+}
 
 template <typename T, int D>
 static cudaError_t decode_impl(const void *q, const void *k, const void *v, const float *g,
                                const float *beta, const uint8_t *route, const float *w,
                                float *state, void *k_cache, void *v_cache, int32_t *cache_len,
                                int32_t cap, void *out, float scale_la, float scale_sm, float eps,
-                               int32_t *status, Shape s, cudaStream_t st) {
-    decode_step_kernel<T, D><<<s.B * s.H, kThreads, 0, st>>>(
+                               void *ws, Shape s, cudaStream_t st) {
+    constexpr int kTileBytes = kTileKeys * D * (int)sizeof(T);
+    constexpr int kRing = 2 * kStages * kTileBytes;
+    constexpr int kRed = 32 * D * 4;               // per-stream / per-slot reduction scratch
+    constexpr int kSmem = kRing > kRed ? kRing : kRed;
+    cudaError_t e = cudaFuncSetAttribute(decode_step_kernel<T, D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return e;
+    dim3 grid(kCtasPerHead, s.B * s.H);
+    decode_step_kernel<T, D><<<grid, kThreads, kSmem, st>>>(
         (const T *)q, (const T *)k, (const T *)v, g, beta, route, w, state, (T *)k_cache,
-        (T *)v_cache, cache_len, cap, (T *)out, scale_la, scale_sm, eps, status);
+        (T *)v_cache, cache_len, cap, (T *)out, scale_la, scale_sm, eps, (uint8_t *)ws, s.B * s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -253,9 +349,9 @@ cudaError_t launch_decode_step(const void *q, const void *k, const void *v, cons
                                const float *beta, const uint8_t *route, const float *w,
                                float *state, void *k_cache, void *v_cache, int32_t *cache_len,
                                int32_t cache_cap, void *out, float scale_la, float scale_sm,
-                               float eps, int32_t *status, Shape s, cudaStream_t st) {
+                               float eps, void *ws, Shape s, cudaStream_t st) {
 #define ARGS q, k, v, g, beta, route, w, state, k_cache, v_cache, cache_len, cache_cap, out, \
-             scale_la, scale_sm, eps, status, s, st
+             scale_la, scale_sm, eps, ws, s, st
     if (s.bf16) {
         if (s.d == 128) return decode_impl<__nv_bfloat16, 128>(ARGS);
         return decode_impl<__nv_bfloat16, 64>(ARGS);

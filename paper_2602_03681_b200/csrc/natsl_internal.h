@@ -117,10 +117,14 @@ cudaError_t launch_gdn_assemble(const AssembleArgs &a, void *dq, void *dk, void 
                                 cudaStream_t st);
 
 // decode.cu
+constexpr int kDecodeParts = 4;   // CTAs that share the retained K/V of one (sequence, head)
+// Bytes of workspace of a decode step: status word, per-head tickets, partial softmax results and
+// linear read-outs.  Zero-filled once by the caller; the kernel leaves the tickets at zero.
+size_t decode_workspace_bytes(int B, int H, int d);
 cudaError_t launch_decode_step(const void *q, const void *k, const void *v, const float *g,
                                const float *beta, const uint8_t *route, const float *w,
                                float *state, void *k_cache, void *v_cache, int32_t *cache_len,
                                int32_t cache_cap, void *out, float scale_la, float scale_sm,
-                               float eps, int32_t *status, Shape s, cudaStream_t st);
+                               float eps, void *ws, Shape s, cudaStream_t st);
 
 }  // namespace natsl
