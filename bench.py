@@ -345,6 +345,7 @@ def run_ours(args):
 
     if world == 1 and not args.no_extras:
         line["decode"] = bench_decode(args, peaks, peak_kind, traffic)
+        line["other_workloads"] = bench_other_workloads(peaks)
     if world == 1 and not args.no_cpu:
         xs = x if args.cpu_sample_B >= B else inputs.make_layer_inputs(wl_rank, B=args.cpu_sample_B)
         sb = min(args.cpu_sample_B, B)
@@ -355,6 +356,57 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def bench_other_workloads(peaks):
+    """Forward of the long-context workload and forward + backward of the training workload
+    (device-resident inputs, CUDA events, best of 3 after a warm-up), with useful FLOPs."""
+    import torch
+
+    from paper_2602_03681_b200 import binding
+    res = {}
+    dt = torch.bfloat16
+    for name, ops in (("cfg2_bf16_long_prefill", ("fwd",)), ("cfg4_bf16_train", ("fwd", "bwd"))):
+        wl = inputs.WORKLOADS[name]
+        x = inputs.make_layer_inputs(wl)
+        d = {m: torch.from_numpy(x[m]).cuda() for m in ("g", "beta", "route", "w")}
+        for m in ("q", "k", "v", "dout"):
+            d[m] = torch.from_numpy(x[m]).cuda().to(dt)
+        ws = {"fwd": None, "bwd": None}
+
+        def call(op):
+            if op == "fwd":
+                ws["fwd"] = binding.hybrid_fwd(d["q"], d["k"], d["v"], d["g"], d["beta"], d["route"],
+                                               d["w"], scale_la=wl.scale_la, scale_sm=wl.scale_sm,
+                                               ws=ws["fwd"])["ws"]
+            else:
+                ws["bwd"] = binding.hybrid_bwd(d["q"], d["k"], d["v"], d["g"], d["beta"], d["route"],
+                                               d["w"], d["dout"], scale_la=wl.scale_la,
+                                               scale_sm=wl.scale_sm, ws=ws["bwd"])["ws"]
+
+        ms = {}
+        for op in ops:
+            call(op)
+            torch.cuda.synchronize()
+            best = float("inf")
+            for _ in range(3):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                call(op)
+                e1.record()
+                torch.cuda.synchronize()
+                best = min(best, e0.elapsed_time(e1))
+            ms[op] = best
+        fl = sum(useful_flops(x["route"], wl.d, wl.C).values())
+        total_ms = sum(ms.values())
+        entry = {"ms": ms, "tokens_per_s": wl.B * wl.L / (total_ms * 1e-3),
+                 "useful_fwd_gflop": fl / 1e9,
+                 "fwd_useful_tflops": fl / (ms["fwd"] * 1e-3) / 1e12,
+                 "fwd_frac_of_bf16_peak": fl / (ms["fwd"] * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+        res[name] = entry
+        del d, ws
+        torch.cuda.empty_cache()
+    return res
 
 
 def bench_decode(args, peaks, peak_kind, traffic):

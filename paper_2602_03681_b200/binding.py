@@ -219,7 +219,7 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5,
     return res
 
 
-def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5, ws=None):
+def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5, ws=None, flags=0):
     """Allocate gradients and run natsl_hybrid_bwd.  Returns dict(dq, dk, dv, dg, dbeta, dw, ws)."""
     B, L, H, d = q.shape
     dev = q.device
@@ -227,7 +227,7 @@ def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5
     dg = torch.empty((B, L, H), dtype=torch.float32, device=dev)
     dbeta = torch.empty((B, L, H), dtype=torch.float32, device=dev)
     dw = torch.empty((B, L, H, 2), dtype=torch.float32, device=dev)
-    p = make_params(B, H, L, d, _dtype_code(q), scale_la, scale_sm, eps, w=w)
+    p = make_params(B, H, L, d, _dtype_code(q), scale_la, scale_sm, eps, w=w, flags=flags)
     if ws is None:
         ws = alloc_workspace(p, OP_BWD, dev)
     natsl_hybrid_bwd(q, k, v, g, beta, route, dout, dq, dk, dv, dg, dbeta, dw, p, ws)

@@ -100,6 +100,7 @@ struct BwdWs {
     float *P, *Abar, *M, *N, *Mg, *Ms, *Ns;                  // [B,H,NC,64,64]
     float *S_c, *dS_c;                                       // [B,H,NC,d,d]
     float *Gcum, *lse, *Dsm, *dGrow, *kappa, *gS;            // [B,H,L] (gS: [B,H,NC,d/32])
+    void *k_smb, *k16, *v16, *Qh, *dO16;                     // tensor-core softmax branch: 16-bit [B,H,L,d]
     size_t bytes;
 };
 
@@ -125,6 +126,12 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     float **sm[] = {&f.Gcum, &f.lse, &f.Dsm, &f.dGrow, &f.kappa};
     for (float **t : sm) *t = c.take<float>(BHL);
     f.gS = c.take<float>(B * H * NC * (d / 32));
+    const size_t h16 = use_tensor_cores(p) ? TM * 2 : 0;
+    f.k_smb = c.take<char>(h16);
+    f.k16 = c.take<char>(h16);
+    f.v16 = c.take<char>(h16);
+    f.Qh = c.take<char>(h16);
+    f.dO16 = c.take<char>(h16);
     f.bytes = c.off;
     return f;
 }
@@ -217,7 +224,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     const bool tensor_cores = use_tensor_cores(p);
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
-                                      f.v16, cap, p->L, f.status, s, st));
+                                      f.v16, nullptr, cap, p->L, f.status, s, st));
     else
         NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
     NATSL_TRY(mark());
@@ -278,20 +285,34 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, p->B,
                                    p->L, p->H, st));
     NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
-    NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L, f.status,
-                               s32, st));
+    const bool tensor_cores = use_tensor_cores(p);   // softmax branch on tcgen05; GDN stays fp32
+    if (tensor_cores)
+        NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, f.k_smb, nullptr, f.v16, f.k16, p->L,
+                                      p->L, f.status, s, st));
+    else
+        NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
+                                   f.status, s32, st));
     NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
                                       f.P, f.Abar, f.Gcum, s32, st));
     NATSL_TRY(launch_gdn_scan_simt(f.q32, f.k32, g, f.W, f.U, f.P, p->scale_la, nullptr, nullptr,
                                    f.S_c, f.Ut, f.o_la, s32, st));
-    NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
-                                          f.o_la, p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
-                                          s32, st));
+    if (tensor_cores)
+        NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la,
+                                            p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
+                                            f.status, s, st));
+    else
+        NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
+                                              f.o_la, p->w, p->scale_sm, p->eps, nullptr, f.o_nla,
+                                              f.lse, s32, st));
     // ---- combination and softmax branch ----
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la, f.do_nla, dw, f.Dsm,
-                                 s, st));
-    NATSL_TRY(launch_softmax_bwd(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix, f.do_nla,
-                                 f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
+                                 tensor_cores ? f.dO16 : nullptr, s, st));
+    if (tensor_cores)
+        NATSL_TRY(launch_softmax_bwd_tc(q, f.Qh, f.dO16, f.k16, f.v16, p->L, f.sm_idx, f.prefix, f.lse,
+                                        f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, f.status, s, st));
+    else
+        NATSL_TRY(launch_softmax_bwd(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix, f.do_nla,
+                                     f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
     // ---- linear branch: reverse scan, then chunk-parallel products ----
     NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
                                f.dS_c, f.gS, s, st));

@@ -46,7 +46,7 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
 // softmax_tc.cu -- tensor-core softmax branch + combination (bf16 storage)
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
                                 const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
-                                int32_t cap, int32_t capv, int32_t *status, Shape s,
+                                void *k16, int32_t cap, int32_t capv, int32_t *status, Shape s,
                                 cudaStream_t st);
 cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const void *v16, int32_t cap,
                                       int32_t capv, const int32_t *sm_idx,
@@ -54,6 +54,15 @@ cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const voi
                                       const float *w, float scale_sm, float eps, void *out,
                                       float *o_nla, float *lse, int32_t *status, Shape s,
                                       cudaStream_t st);
+
+// softmax_bwd_tc.cu -- tensor-core backward of the softmax branch (bf16 storage).  Qh is scratch
+// for the fp16 copy of q [B,H,L,d]; dO16 the fp16 branch-output gradient [B,H,L,d]; k16, v16 the
+// fp16 retained K/V [B,H,cap,d]; dq_sm is token-major [B,L,H,d], dk_sm / dv_sm compacted.
+cudaError_t launch_softmax_bwd_tc(const void *q, void *Qh, const void *dO16, const void *k16,
+                                  const void *v16, int cap, const int32_t *sm_idx,
+                                  const int32_t *sm_chunk_prefix, const float *lse, const float *Dsm,
+                                  float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
+                                  int32_t *status, Shape s, cudaStream_t st);
 
 // gdn_tc.cu -- tensor-core chunkwise Gated DeltaNet (bf16 storage): intermediates in workspace
 struct GdnTcWs {
@@ -84,9 +93,10 @@ cudaError_t launch_bgemm(bool ta, bool tb, int mask, BMat A, BMat B, BMat C, int
                          float alpha, bool accumulate, Shape s, cudaStream_t st);
 cudaError_t launch_to_f32(const void *a, const void *b, const void *c, float *a32, float *b32,
                           float *c32, size_t n, bool bf16, cudaStream_t st);
+// do16: optional fp16 copy of do_nla in [B,H,L,d] layout (tensor-core softmax backward).
 cudaError_t launch_combine_bwd(const float *o_la, const float *o_nla, const void *dout,
                                const float *w, float eps, float *do_la, float *do_nla, float *dw,
-                               float *Dsm, Shape s, cudaStream_t st);
+                               float *Dsm, void *do16, Shape s, cudaStream_t st);
 cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const float *v_sm32, int cap,
                                const int32_t *sm_idx, const int32_t *sm_chunk_prefix,
                                const float *do_nla, const float *lse, const float *Dsm,

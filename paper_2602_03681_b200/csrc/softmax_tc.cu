@@ -103,7 +103,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 
     if (warp == 5) {
         // ------------------------------ TMA producer ------------------------------
-        if (lane == 0) {
+        if (lane == 0 && T > 0) {      // nothing is loaded for a tile that sees no retained key
             prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
             mbar_arrive_expect_tx(&ms.barQ, SL::kQBytes);
             for (int kb = 0; kb < KB; ++kb)
@@ -316,14 +316,15 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 }
 
 // Copy the retained tokens' K rows (bf16) and V rows (as fp16) into the compacted layouts
-// [B,H,cap,d] / [B,H,capv,d] and zero the V rows up to the next multiple of 64, so that a K/V
-// tile never multiplies a zero probability with an uninitialised value.  grid = (row blocks, B*H).
+// [B,H,cap,d] / [B,H,capv,d] (optionally K as fp16 too, for the backward) and zero the fp16 rows
+// up to the next multiple of 128, so that a K/V tile never multiplies a zero probability or a
+// zero logit gradient with an uninitialised value.  grid = (row blocks, B*H).
 template <int D>
 __global__ void __launch_bounds__(256)
 gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__restrict__ v,
                     const int32_t *__restrict__ sm_idx, const int32_t *__restrict__ sm_chunk_prefix,
                     __nv_bfloat16 *__restrict__ k_sm, __nv_bfloat16 *__restrict__ v_sm,
-                    __half *__restrict__ v16, int cap, int capv, int32_t *status, int L, int H) {
+                    __half *__restrict__ v16, __half *__restrict__ k16, int cap, int capv, int32_t *status, int L, int H) {
     constexpr int kVecPerRow = D * 2 / 16;
     constexpr int kRows = 256 / kVecPerRow;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
@@ -331,19 +332,30 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
     const int n_sm = sm_chunk_prefix[(size_t)bh * (NC + 1) + NC];
     if (blockIdx.x == 0 && threadIdx.x == 0 && n_sm > cap) atomicMin(status, (int)NATSL_ERR_CACHE_FULL);
     const int n = min(n_sm, cap);
-    const int n_pad = min((n + kBN - 1) / kBN * kBN, capv);
+    const int n_pad = min((n + 127) / 128 * 128, capv);
     const int row = blockIdx.x * kRows + threadIdx.x / kVecPerRow;
     const int piece = threadIdx.x % kVecPerRow;
     if (row >= n_pad) return;
     uint4 *dv16 = reinterpret_cast<uint4 *>(v16 + ((size_t)bh * capv + row) * D) + piece;
+    uint4 *dk16 = k16 ? reinterpret_cast<uint4 *>(k16 + ((size_t)bh * capv + row) * D) + piece : nullptr;
     if (row >= n) {
         *dv16 = make_uint4(0u, 0u, 0u, 0u);
+        if (dk16) *dk16 = make_uint4(0u, 0u, 0u, 0u);
         return;
     }
     const int tok = sm_idx[(size_t)bh * L + row];
     const size_t src = (((size_t)b * L + tok) * H + h) * D;
     const size_t dst = ((size_t)bh * cap + row) * D;
-    reinterpret_cast<uint4 *>(k_sm + dst)[piece] = reinterpret_cast<const uint4 *>(k + src)[piece];
+    const uint4 kk = reinterpret_cast<const uint4 *>(k + src)[piece];
+    reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
+    if (dk16) {
+        const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
+        uint32_t ko[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            ko[i] = pack_half2(__uint_as_float(kw[i] << 16), __uint_as_float(kw[i] & 0xffff0000u));
+        *dk16 = make_uint4(ko[0], ko[1], ko[2], ko[3]);
+    }
     const uint4 vv = reinterpret_cast<const uint4 *>(v + src)[piece];
     if (v_sm) reinterpret_cast<uint4 *>(v_sm + dst)[piece] = vv;
     const uint32_t wv[4] = {vv.x, vv.y, vv.z, vv.w};
@@ -394,25 +406,25 @@ cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const voi
 
 template <int D>
 static cudaError_t gather_tc_impl(const void *k, const void *v, const int32_t *sm_idx,
-                                  const int32_t *pre, void *k_sm, void *v_sm, void *v16, int cap,
-                                  int capv, int32_t *status, Shape s, cudaStream_t st) {
+                                  const int32_t *pre, void *k_sm, void *v_sm, void *v16, void *k16,
+                                  int cap, int capv, int32_t *status, Shape s, cudaStream_t st) {
     constexpr int kRows = 256 / (D * 2 / 16);
     const int max_rows = s.L < capv ? s.L : capv;
     dim3 grid((max_rows + kRows - 1) / kRows, s.B * s.H);
     gather_kv_tc_kernel<D><<<grid, 256, 0, st>>>(
         (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, sm_idx, pre, (__nv_bfloat16 *)k_sm,
-        (__nv_bfloat16 *)v_sm, (__half *)v16, cap, capv, status, s.L, s.H);
+        (__nv_bfloat16 *)v_sm, (__half *)v16, (__half *)k16, cap, capv, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
                                 const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
-                                int32_t cap, int32_t capv, int32_t *status, Shape s,
+                                void *k16, int32_t cap, int32_t capv, int32_t *status, Shape s,
                                 cudaStream_t st) {
     if (s.d == 128)
-        return gather_tc_impl<128>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, cap, capv, status, s, st);
-    return gather_tc_impl<64>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, cap, capv, status, s, st);
+        return gather_tc_impl<128>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, status, s, st);
+    return gather_tc_impl<64>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, status, s, st);
 }
 
 }  // namespace natsl

@@ -225,12 +225,13 @@ def test_decode_cache_full_is_reported_not_trapped():
 
 
 # ------------------------------------------------------------------ backward
-def run_bwd(wl, x, w="given"):
+def run_bwd(wl, x, w="given", flags=0):
     from paper_2602_03681_b200 import binding
     dt = tdtype(wl)
     res = binding.hybrid_bwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]),
                              dev(x["beta"]), dev(x["route"]), dev(x["w"]) if w == "given" else None,
-                             dev(x["dout"], dt), scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+                             dev(x["dout"], dt), scale_la=wl.scale_la, scale_sm=wl.scale_sm,
+                             flags=flags)
     torch.cuda.synchronize()
     assert binding.natsl_device_status(res["ws"]) == 0
     return {n: t.float().cpu().numpy() for n, t in res.items() if n != "ws"}
@@ -249,9 +250,12 @@ def check_bwd(wl, got, ref, tol):
                                         ("cfg4_bf16_train", 2, 3, 320),
                                         ("cfg1_bf16_prefill", 1, 2, 192)])
 def test_bwd_small_cases(name, B, H, L):
+    """The fp32 CUDA-core backward (forced for bf16 storage, whose default runs the softmax branch
+    on tensor cores)."""
+    from paper_2602_03681_b200 import binding
     wl = inputs.WORKLOADS[name]
     x = inputs.make_layer_inputs(wl, B=B, H=H, L=L)
-    got = run_bwd(wl, x)
+    got = run_bwd(wl, x, flags=binding.FORCE_SIMT)
     ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
                             scale_la=wl.scale_la, scale_sm=wl.scale_sm)
     # fp32 arithmetic throughout; bf16 storage only rounds dq, dk, dv

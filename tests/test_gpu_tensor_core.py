@@ -8,7 +8,8 @@ import torch
 
 import oracle
 from paper_2602_03681_b200 import inputs
-from test_gpu_parity import TOL, check_fwd, check_stored, dev, rel_err, run_fwd, run_oracle
+from test_gpu_parity import (TOL, check_bwd, check_fwd, check_stored, dev, rel_err, run_bwd, run_fwd,
+                             run_oracle)
 
 pytestmark = pytest.mark.gpu
 
@@ -132,3 +133,32 @@ def test_fwd_tensor_core_is_deterministic():
     a, b = run_fwd(wl, x), run_fwd(wl, x)
     for name in ("out", "o_la", "o_nla", "lse", "state_out"):
         assert np.array_equal(a[name], b[name]), name
+
+
+# ------------------------------------------------------------------ backward (softmax branch on tcgen05)
+@pytest.mark.parametrize("name,B,H,L,route", [("cfg4_bf16_train", 2, 3, 320, None),
+                                              ("cfg4_bf16_train", 1, 2, 64, None),
+                                              ("cfg1_bf16_prefill", 1, 2, 448, None),
+                                              ("cfg4_bf16_train", 1, 2, 384, "all_softmax"),
+                                              ("cfg1_bf16_prefill", 1, 2, 256, "all_linear"),
+                                              ("cfg4_bf16_train", 1, 1, 256, "late")])
+def test_bwd_tensor_core_softmax_branch(name, B, H, L, route):
+    wl = inputs.WORKLOADS[name]
+    r = None
+    if route == "all_softmax":
+        r = np.ones((B, L, H), np.uint8)
+    elif route == "all_linear":
+        r = np.zeros((B, L, H), np.uint8)
+    elif route == "late":                         # queries before token 100 see nothing
+        r = np.zeros((B, L, H), np.uint8)
+        r[:, 100, :] = 1
+        r[:, 101:, :] = (np.random.default_rng(1).random((B, L - 101, H)) < 0.3)
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L, route=r)
+    got = run_bwd(wl, x)
+    ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                            scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+    for name_ in ("dq", "dk", "dv", "dg", "dbeta", "dw"):
+        assert np.isfinite(got[name_]).all(), name_
+    check_bwd(wl, got, ref, TOL["bf16"])
+    lin = x["route"] == 0
+    assert np.all(got["dbeta"][~lin] == 0)
