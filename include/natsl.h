@@ -22,6 +22,11 @@
  * contiguous, in the shapes given.  Base pointers of q,k,v,out,dout,dq,dk,dv, the caches
  * and the workspace must be 16-byte aligned.
  *
+ * Precision of the default path for NATSL_BF16 (tcgen05 tensor cores): q, k, v are used as
+ * given; every computed tensor-core operand is held in fp16 with fp32 accumulation, and q, k, v
+ * are converted to fp16 on the way, so their magnitudes must stay below 65504 (values below
+ * 6e-8 in magnitude flush to zero).  NATSL_FORCE_SIMT selects fp32 arithmetic throughout.
+ *
  * Return value: NATSL_OK or a negative natsl_status.  Arguments are validated on the host
  * before anything is launched; an invalid call launches nothing.  Conditions only the
  * device can see (decode cache full) are written to a status word that
@@ -156,7 +161,9 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
  * A sequence whose cache is full and whose token is routed to softmax is left untouched,
  * its out row is zero-filled and NATSL_ERR_CACHE_FULL is recorded in the status word at the
  * start of the workspace.  ws must hold natsl_workspace_size(p, NATSL_OP_DECODE) bytes and be
- * zero-filled once before its first use.
+ * zero-filled once before its first use; besides the status word it holds per-head tickets and
+ * partial results of the step in flight, so two steps that use the same ws must not overlap on
+ * the GPU (successive steps on one stream are fine).
  */
 int natsl_decode_step(const void *q, const void *k, const void *v, const float *g,
                       const float *beta, const uint8_t *route, float *state,
