@@ -364,9 +364,9 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 // ==========================================================================================
 constexpr int kScanRowThreads = 256;
 constexpr int kScanThreads = 320;
-constexpr int kScanStages = 2;
+constexpr int kScanStages = 3;
 constexpr int kScanMisc = 1024;
-constexpr int kDecaySlots = 4;                             // ring of per-chunk decay factors
+constexpr int kDecaySlots = 8;                             // ring of per-chunk decay factors
 
 template <int D> struct ScanLayout {
     static constexpr int KB = D / 64;
@@ -378,15 +378,15 @@ template <int D> struct ScanLayout {
     static constexpr int oW = 0, oQ = oW + kW, oK = oQ + kQ, oP = oK + kK;
     static constexpr int kStage = oP + kP;
     static constexpr int kTx = kStage + kG;
-    static constexpr int oS = kScanStages * kStage;        // S^T operand: 128 rows x D fp16
-    static constexpr int kS = KB * 16384;
-    static constexpr int oU = oS + kS;                     // U~ operand: 128 rows x 64 tokens
-    static constexpr int oUs = oU + 16384;                 // U~ diag(gamma_C / gamma)
-    static constexpr int oG = oUs + 16384;                 // decay ring
+    static constexpr int oG = kScanStages * kStage;        // decay ring
     static constexpr int oMisc = oG + kDecaySlots * kG;
     static constexpr int kTotal = oMisc + kScanMisc;
     static constexpr int kTmemCols = 512;
-    static constexpr int cS = 0, cWS = D, cQS = D + 64, cD3 = D + 192;   // TMEM columns
+    // TMEM columns.  dS: fp32 state increment [D].  WS: fp32 W S [64], overwritten by each thread
+    // with its fp16 operands (U~ | U~ diag(gamma_C/gamma), 16 + 16 packed columns per 32 tokens).
+    // A: the fp16 state operand [D/2 packed].  QS, D3: double-buffered fp32 [64] each.
+    static constexpr int cS = 0, cWS = D, cA = D + 64, cQS = cA + D / 2, cD3 = cQS + 128;
+    static_assert(cD3 + 128 <= 512, "TMEM budget");
 };
 
 struct ScanMisc {
@@ -449,8 +449,9 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                     tma_load_2d(st + SL::oK + kb * 8192, &map_kh, &ms.full[s], kb * 64, bh * L + c * 64);
                 }
                 tma_load_2d(st + SL::oP, &map_ph, &ms.full[s], 0, (bh * NC + c) * 64);
-                // A decay slot is reused four chunks later, i.e. only after the stage of chunk c + 2
-                // has been released, which every row thread's work on chunk c precedes.
+                // A decay slot is reused kDecaySlots chunks later, i.e. only after the stages of the
+                // chunks up to c + kDecaySlots - kScanStages have been released, which every row
+                // thread's work on chunk c precedes.
                 bulk_load_1d(smem + SL::oG + (c % kDecaySlots) * SL::kG,
                              Gd + ((size_t)bh * NC + c) * 128, SL::kG, &ms.full[s]);
             }
@@ -464,8 +465,6 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             constexpr uint32_t id_qs = make_idesc(kFmtF16, 128, 64, false, false);   // B = Q
             constexpr uint32_t id_su = make_idesc(kFmtF16, 128, D, false, true);     // B = K (MN-major)
             constexpr uint32_t id_pu = make_idesc(kFmtF16, 128, 64, false, false);   // B = P
-            const uint32_t aS = smem_u32(smem + SL::oS), aU = smem_u32(smem + SL::oU),
-                           aUs = smem_u32(smem + SL::oUs);
             for (int c = 0; c < NC; ++c) {
                 const int s = c % kScanStages;
                 const uint32_t st = smem_u32(smem + s * SL::kStage);
@@ -473,32 +472,29 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 if (!mbar_wait(&ms.barA, c & 1, abort_flag)) break;
                 tc_fence_after_sync();
 #pragma unroll
-                for (int kb = 0; kb < KB; ++kb)
-#pragma unroll
-                    for (int k16 = 0; k16 < 4; ++k16)
-                        mma_ss(tmem + SL::cWS, desc_kmajor(aS + kb * 16384 + k16 * 32),
-                               desc_mnmajor(st + SL::oW + (kb * 4 + k16) * 2048, 0), id_ws,
-                               (kb | k16) != 0);
+                for (int kk = 0; kk < D / 16; ++kk)
+                    mma_ts(tmem + SL::cWS, tmem + SL::cA + kk * 8,
+                           desc_mnmajor(st + SL::oW + kk * 2048, 0), id_ws, kk != 0);
                 mma_commit(&ms.barWS);
 #pragma unroll
-                for (int kb = 0; kb < KB; ++kb)
-#pragma unroll
-                    for (int k16 = 0; k16 < 4; ++k16)
-                        mma_ss(tmem + SL::cQS + 64 * (c & 1), desc_kmajor(aS + kb * 16384 + k16 * 32),
-                               desc_kmajor(st + SL::oQ + kb * 8192 + k16 * 32), id_qs, (kb | k16) != 0);
+                for (int kk = 0; kk < D / 16; ++kk)
+                    mma_ts(tmem + SL::cQS + 64 * (c & 1), tmem + SL::cA + kk * 8,
+                           desc_kmajor(st + SL::oQ + (kk >> 2) * 8192 + (kk & 3) * 32), id_qs, kk != 0);
                 mma_commit(&ms.barQS[c & 1]);
                 if (!mbar_wait(&ms.barB, c & 1, abort_flag)) break;
                 tc_fence_after_sync();
+                // D3 first: the commit behind the state update then also covers it, so that the
+                // operands in the WS columns are free once barSU has fired.
 #pragma unroll
                 for (int k16 = 0; k16 < 4; ++k16)
-                    mma_ss(tmem + SL::cS, desc_kmajor(aUs + k16 * 32),
-                           desc_mnmajor(st + SL::oK + k16 * 2048, 8192), id_su, k16 != 0);
-                mma_commit(&ms.barSU);
-#pragma unroll
-                for (int k16 = 0; k16 < 4; ++k16)
-                    mma_ss(tmem + SL::cD3 + 64 * (c & 1), desc_kmajor(aU + k16 * 32),
+                    mma_ts(tmem + SL::cD3 + 64 * (c & 1), tmem + SL::cWS + (k16 >> 1) * 32 + (k16 & 1) * 8,
                            desc_kmajor(st + SL::oP + k16 * 32), id_pu, k16 != 0);
                 mma_commit(&ms.barD3[c & 1]);
+#pragma unroll
+                for (int k16 = 0; k16 < 4; ++k16)
+                    mma_ts(tmem + SL::cS, tmem + SL::cWS + (k16 >> 1) * 32 + 16 + (k16 & 1) * 8,
+                           desc_mnmajor(st + SL::oK + k16 * 2048, 8192), id_su, k16 != 0);
+                mma_commit(&ms.barSU);
                 mma_commit(&ms.empty[s]);
             }
         }
@@ -573,17 +569,20 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 }
                 tc_fence_before_sync();
             }
-            // ---- (a) state row -> fp16 operand; decay the register copy to the next chunk entry
+            // ---- (a) state row -> fp16 operand in TMEM; decay the register copy afterwards ----
             {
-                uint8_t *sub = smem + SL::oS + (col0 >> 6) * 16384;
-                const int piece0 = (col0 & 63) >> 3;
+                uint32_t pk[kHalfCols / 2];
 #pragma unroll
-                for (int pc = 0; pc < kHalfCols / 8; ++pc)
-                    *reinterpret_cast<uint4 *>(sub + sw128_offset(r, piece0 + pc)) = make_uint4(
-                        pack_half2(S[8 * pc], S[8 * pc + 1]), pack_half2(S[8 * pc + 2], S[8 * pc + 3]),
-                        pack_half2(S[8 * pc + 4], S[8 * pc + 5]), pack_half2(S[8 * pc + 6], S[8 * pc + 7]));
+                for (int x = 0; x < kHalfCols / 2; ++x) pk[x] = pack_half2(S[2 * x], S[2 * x + 1]);
+                if (kHalfCols == 64)
+                    tmem_st32(tmem + SL::cA + half * (kHalfCols / 2) + lane_base,
+                              reinterpret_cast<const uint32_t (&)[32]>(pk));
+                else
+                    tmem_st16(tmem + SL::cA + half * (kHalfCols / 2) + lane_base,
+                              reinterpret_cast<const uint32_t (&)[16]>(pk));
+                tmem_wait_st();
             }
-            fence_proxy_async_smem();
+            tc_fence_before_sync();
             mbar_arrive(&ms.barA);
             float u[32];                                   // from L2; lands while W S is computed
             if (active) {
@@ -613,19 +612,16 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
 #pragma unroll
                 for (int j = 0; j < 32; ++j) u[j] -= __uint_as_float(ws[j]);
             }
+            {
+                uint32_t pk[32];     // [0,16): U~ of this thread's 32 tokens, [16,32): U~ gamma_C/gamma
 #pragma unroll
-            for (int pc = 0; pc < 4; ++pc) {
-                float xs[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) xs[e] = u[8 * pc + e] * e2[tk0 + 8 * pc + e];
-                *reinterpret_cast<uint4 *>(smem + SL::oU + sw128_offset(r, 4 * half + pc)) =
-                    make_uint4(pack_half2(u[8 * pc], u[8 * pc + 1]), pack_half2(u[8 * pc + 2], u[8 * pc + 3]),
-                               pack_half2(u[8 * pc + 4], u[8 * pc + 5]), pack_half2(u[8 * pc + 6], u[8 * pc + 7]));
-                *reinterpret_cast<uint4 *>(smem + SL::oUs + sw128_offset(r, 4 * half + pc)) =
-                    make_uint4(pack_half2(xs[0], xs[1]), pack_half2(xs[2], xs[3]),
-                               pack_half2(xs[4], xs[5]), pack_half2(xs[6], xs[7]));
+                for (int x = 0; x < 16; ++x) {
+                    pk[x] = pack_half2(u[2 * x], u[2 * x + 1]);
+                    pk[16 + x] = pack_half2(u[2 * x] * e2[tk0 + 2 * x], u[2 * x + 1] * e2[tk0 + 2 * x + 1]);
+                }
+                tmem_st32(tmem + SL::cWS + tk0 + lane_base, pk);   // over this thread's own W S columns
+                tmem_wait_st();
             }
-            fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&ms.barB);
             // ---- behind the MMAs just released: next U row towards L2, previous chunk's output ----
