@@ -174,6 +174,16 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         const float sl2 = scale_sm * 1.4426950408889634f;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
+        if (i_abs < L) {     // the epilogue's rows of o_la and w: on their way to L2 while the tiles run
+            const size_t tok = ((size_t)b * L + i_abs) * H + h;
+#pragma unroll
+            for (int x = 0; x < D * 4 / 128; ++x) prefetch_l2(o_la + tok * D + x * 32);
+            if (w) prefetch_l2(w + tok * 2);
+        }
+        // The compacted keys are in position order, so row i sees exactly the first `cnt` of them:
+        // all n_full earlier ones plus those of the CTA's own chunks at positions <= i.
+        int cnt = n_full;
+        for (int kq = 0; kq < n_end - n_full; ++kq) cnt += ms.pos[kq] <= i_abs ? 1 : 0;
         for (int t = 0; t < T; ++t) {
             ok = mbar_wait(&ms.barS[t & 1], (t >> 1) & 1, abort_flag);
             if (!ok) break;
@@ -186,13 +196,9 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll
             for (int c = 0; c < kBN; ++c) x[c] = __uint_as_float(sv[c >> 5][c & 31]) * sl2;
             const int j0 = t * kBN;
-            if (j0 + kBN > n_full) {                    // tile reaches into the CTA's own chunks
+            if (!__all_sync(0xffffffffu, j0 + kBN <= cnt)) {   // some row of the warp is cut off here
 #pragma unroll
-                for (int c = 0; c < kBN; ++c) {
-                    const int jj = j0 + c;
-                    const bool vis = jj < n_full || (jj < n_end && ms.pos[jj - n_full] <= i_abs);
-                    x[c] = vis ? x[c] : -INFINITY;
-                }
+                for (int c = 0; c < kBN; ++c) x[c] = j0 + c < cnt ? x[c] : -INFINITY;
             }
             float mx = x[0];
 #pragma unroll
@@ -243,66 +249,74 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             ok = mbar_wait(&ms.barO, (T - 1) & 1, abort_flag);
             tc_fence_after_sync();
         }
-        if (ok && i_abs < L) {
-            const size_t tok = ((size_t)b * L + i_abs) * H + h;
+        if (ok) {
+            // (1) each thread normalises its own row of O (TMEM lane r) into shared memory -- the
+            // K/V ring and the P tile are no longer in use -- and records the row's RMS factor;
+            // (2) the warps then walk the rows with the lanes along the head dimension, so that
+            // o_la is read, and out / o_nla are written, as whole contiguous rows.
+            constexpr int kXS = D + 4;                  // padded row stride (floats)
+            float *Xs = reinterpret_cast<float *>(smem + SL::oK);
+            float *row_fn = Xs + kBM * kXS;
+            static_assert((kBM * kXS + kBM) * 4 <= SL::oMisc - SL::oK, "epilogue staging does not fit");
             const float inv = l > 0.f ? 1.f / l : 0.f;
-            const float *ol = o_la + tok * D;
-            float ssn = 0.f, ssl = 0.f;
+            float ssn = 0.f;
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t ov[32];
                 if (T > 0) {
                     tmem_ld32(tO + lane_base + cb * 32, ov);
                     tmem_wait_ld();
-                }
-#pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    const float on = l > 0.f ? __uint_as_float(ov[c]) * inv : 0.f;
-                    ssn = fmaf(on, on, ssn);
                 }
 #pragma unroll
                 for (int c4 = 0; c4 < 8; ++c4) {
-                    const float4 a = __ldg(reinterpret_cast<const float4 *>(ol + cb * 32) + c4);
-                    ssl = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, ssl))));
+                    float4 o;
+                    o.x = l > 0.f ? __uint_as_float(ov[4 * c4]) * inv : 0.f;
+                    o.y = l > 0.f ? __uint_as_float(ov[4 * c4 + 1]) * inv : 0.f;
+                    o.z = l > 0.f ? __uint_as_float(ov[4 * c4 + 2]) * inv : 0.f;
+                    o.w = l > 0.f ? __uint_as_float(ov[4 * c4 + 3]) * inv : 0.f;
+                    ssn = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ssn))));
+                    *reinterpret_cast<float4 *>(Xs + r * kXS + cb * 32 + 4 * c4) = o;
                 }
             }
-            const float fn = rsqrtf(ssn / D + eps), fl = rsqrtf(ssl / D + eps);
-            const float wn = (w ? w[tok * 2] : 0.5f) * fn, wl = (w ? w[tok * 2 + 1] : 0.5f) * fl;
+            row_fn[r] = rsqrtf(ssn / D + eps);
+            if (lse && i_abs < L)
+                lse[(size_t)bh * L + i_abs] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            named_barrier_sync(1, kSoftmaxThreads);
+            constexpr int kLpr = D / 4;                 // lanes per row
+            constexpr int kRpi = 32 / kLpr;             // rows per warp instruction
+            constexpr int kBatch = 8;                   // row steps with their loads in flight together
+            const int sub = lane / kLpr, col = (lane % kLpr) * 4;
+            for (int r0 = warp * 32; r0 < warp * 32 + 32; r0 += kBatch * kRpi) {
+                float4 a[kBatch];
+                float2 wv[kBatch];                      // all loads of the batch are issued before any use
 #pragma unroll
-            for (int cb = 0; cb < D / 32; ++cb) {
-                uint32_t ov[32];
-                if (T > 0) {
-                    tmem_ld32(tO + lane_base + cb * 32, ov);
-                    tmem_wait_ld();
+                for (int u = 0; u < kBatch; ++u) {
+                    const int ia = p * kBM + r0 + u * kRpi + sub;
+                    const size_t tok = ((size_t)b * L + min(ia, L - 1)) * H + h;
+                    a[u] = ia < L ? __ldg(reinterpret_cast<const float4 *>(o_la + tok * D + col))
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+                    wv[u] = w ? __ldg(reinterpret_cast<const float2 *>(w + tok * 2)) : make_float2(0.5f, 0.5f);
                 }
-                float on[32];
 #pragma unroll
-                for (int c = 0; c < 32; ++c) on[c] = l > 0.f ? __uint_as_float(ov[c]) * inv : 0.f;
-                if (o_nla) {
+                for (int u = 0; u < kBatch; ++u) {
+                    const int rr = r0 + u * kRpi + sub, ia = p * kBM + rr;
+                    float ssl = fmaf(a[u].x, a[u].x, fmaf(a[u].y, a[u].y, fmaf(a[u].z, a[u].z, a[u].w * a[u].w)));
 #pragma unroll
-                    for (int c4 = 0; c4 < 8; ++c4)
-                        reinterpret_cast<float4 *>(o_nla + tok * D + cb * 32)[c4] =
-                            make_float4(on[4 * c4], on[4 * c4 + 1], on[4 * c4 + 2], on[4 * c4 + 3]);
-                }
-                if (out) {
-                    float4 a[8];
-#pragma unroll
-                    for (int c4 = 0; c4 < 8; ++c4)
-                        a[c4] = __ldg(reinterpret_cast<const float4 *>(ol + cb * 32) + c4);
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const float4 a0 = a[2 * q4], a1 = a[2 * q4 + 1];
-                        const float *o8 = on + 8 * q4;
-                        uint4 u;
-                        u.x = pack_bf162(fmaf(wn, o8[0], wl * a0.x), fmaf(wn, o8[1], wl * a0.y));
-                        u.y = pack_bf162(fmaf(wn, o8[2], wl * a0.z), fmaf(wn, o8[3], wl * a0.w));
-                        u.z = pack_bf162(fmaf(wn, o8[4], wl * a1.x), fmaf(wn, o8[5], wl * a1.y));
-                        u.w = pack_bf162(fmaf(wn, o8[6], wl * a1.z), fmaf(wn, o8[7], wl * a1.w));
-                        reinterpret_cast<uint4 *>(out + tok * D + cb * 32)[q4] = u;
+                    for (int o = kLpr / 2; o > 0; o >>= 1) ssl += __shfl_xor_sync(0xffffffffu, ssl, o);
+                    if (ia >= L) continue;
+                    const size_t tok = ((size_t)b * L + ia) * H + h;
+                    const float4 on = *reinterpret_cast<const float4 *>(Xs + rr * kXS + col);
+                    if (o_nla) *reinterpret_cast<float4 *>(o_nla + tok * D + col) = on;
+                    if (out) {
+                        const float wn = wv[u].x * row_fn[rr];
+                        const float wl = wv[u].y * rsqrtf(ssl / D + eps);
+                        uint2 pk;
+                        pk.x = pack_bf162(fmaf(wn, on.x, wl * a[u].x), fmaf(wn, on.y, wl * a[u].y));
+                        pk.y = pack_bf162(fmaf(wn, on.z, wl * a[u].z), fmaf(wn, on.w, wl * a[u].w));
+                        *reinterpret_cast<uint2 *>(out + tok * D + col) = pk;
                     }
                 }
             }
-            if (lse) lse[(size_t)bh * L + i_abs] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
         }
     }
     // ------------------------------ teardown ------------------------------
