@@ -297,12 +297,18 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                                   : make_float4(0.f, 0.f, 0.f, 0.f);
                     wv[u] = w ? __ldg(reinterpret_cast<const float2 *>(w + tok * 2)) : make_float2(0.5f, 0.5f);
                 }
+                float ssl_[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u)
+                    ssl_[u] = fmaf(a[u].x, a[u].x, fmaf(a[u].y, a[u].y, fmaf(a[u].z, a[u].z, a[u].w * a[u].w)));
+#pragma unroll
+                for (int o = kLpr / 2; o > 0; o >>= 1)       // the batch's row sums, interleaved
+#pragma unroll
+                    for (int u = 0; u < kBatch; ++u) ssl_[u] += __shfl_xor_sync(0xffffffffu, ssl_[u], o);
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u) {
                     const int rr = r0 + u * kRpi + sub, ia = p * kBM + rr;
-                    float ssl = fmaf(a[u].x, a[u].x, fmaf(a[u].y, a[u].y, fmaf(a[u].z, a[u].z, a[u].w * a[u].w)));
-#pragma unroll
-                    for (int o = kLpr / 2; o > 0; o >>= 1) ssl += __shfl_xor_sync(0xffffffffu, ssl, o);
+                    const float ssl = ssl_[u];
                     if (ia >= L) continue;
                     const size_t tok = ((size_t)b * L + ia) * H + h;
                     const float4 on = *reinterpret_cast<const float4 *>(Xs + rr * kXS + col);
