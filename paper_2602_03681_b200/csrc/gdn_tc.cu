@@ -40,34 +40,38 @@ __device__ __forceinline__ uint4 bf16x8_to_f16x8(uint4 u) {
 }
 
 // ==========================================================================================
-// Prepare: one CTA per pair of chunks of one (batch, head).  Threads 0..127 own one token each
-// (thread r <-> token r of the pair) up to the triangular solve, and one head-dimension row each
-// afterwards; warp 4 issues TMA and MMAs.
+// Prepare: one CTA per chunk of one (batch, head).  One MMA group with M = 128 stacks [Q ; K] on
+// the rows against K: TMEM rows 0-63 then hold Q K^T (-> P) and rows 64-127 K K^T (-> A).  Warps 0-1
+// (rows 0-63) compute the gates, P and the decay factors; warps 2-3 (rows 64-127) build A, solve
+// T = (I + A)^-1 one row per thread, and write the fp16 operands T beta~ and T beta~ gamma; then all
+// 128 threads (one head-dimension row each) store U^T and W^T.  Warp 4 issues TMA and MMAs.
+// 128 TMEM columns and ~50 KB of shared memory per CTA keep four CTAs on an SM, so that the long
+// dependent instruction stream of the solve overlaps with other chunks' loads and stores.
 // ==========================================================================================
 constexpr int kPrepThreads = 160;
 constexpr int kPrepMisc = 2048;
 
 template <int D> struct PrepLayout {
     static constexpr int KB = D / 64;
-    static constexpr int kTile = KB * 128 * 128;           // 128 tokens x D 16-bit values
-    static constexpr int oV = 0;
-    static constexpr int oK = oV + kTile;                  // directly after V (D = 64 stacks them)
-    static constexpr int oX = oK + kTile;                  // Q tile, then A^T (fp32), then T operands
-    static constexpr int kX = kTile > 32768 ? kTile : 32768;
+    static constexpr int oV = 0;                           // V: KB sub-tiles of 64 tokens x 64
+    static constexpr int oQK = KB * 8192;                  // per 64-column block: [Q 8 KB][K 8 KB]
+    static constexpr int oX = oQK + KB * 16384;            // d = 64 only: A^T, then the T operands
+    static constexpr int kX = D == 64 ? 16384 : 0;
     static constexpr int oMisc = oX + kX;
     static constexpr int kTotal = oMisc + kPrepMisc;
+    static constexpr int kLoadBytes = KB * 24576;
 };
 
 struct PrepMisc {
     uint64_t barLoad, barConv, barM, barXfree, barT, barUW;
     uint32_t tmem_base;
     int abort_flag;
-    float G[128], bt[128], wsum[4];
+    float G[64], bt[64], wsum[2];
 };
 static_assert(sizeof(PrepMisc) <= kPrepMisc, "misc page too small");
 
 template <int D>
-__global__ void __launch_bounds__(kPrepThreads)
+__global__ void __launch_bounds__(kPrepThreads, 4)
 gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                       const __grid_constant__ CUtensorMap map_k,
                       const __grid_constant__ CUtensorMap map_v,
@@ -83,9 +87,9 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     PrepMisc &ms = *reinterpret_cast<PrepMisc *>(smem + PL::oMisc);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NC = L / kC;
-    const int pr = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
-    const int tok_first = pr * 128;                    // first token of the pair
-    const bool second_valid = 2 * pr + 1 < NC;
+    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int tok0 = c * kC;
+    const size_t chunk = (size_t)bh * NC + c;
 
     if ((smem_u32(smem) & 1023u) != 0) {
         if (tid == 0) atomicMin(status, (int)NATSL_ERR_CUDA);
@@ -101,242 +105,235 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         ms.abort_flag = 0;
         fence_mbar_init();
     }
-    if (warp == 4) tmem_alloc(&ms.tmem_base, 256);
+    if (warp == 4) tmem_alloc(&ms.tmem_base, 128);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = ms.tmem_base;
     volatile int *abort_flag = &ms.abort_flag;
-    uint8_t *sV = smem + PL::oV, *sK = smem + PL::oK, *sX = smem + PL::oX;
+    uint8_t *sV = smem + PL::oV, *sQK = smem + PL::oQK;
+    // A^T (fp32, two halves of 32 columns j) and later the two fp16 operands: in the two Q blocks
+    // once K K^T / Q K^T and the q copy are done with them (d = 128), or in their own region (d = 64).
+    uint8_t *xLo = D == 128 ? sQK : smem + PL::oX;
+    uint8_t *xHi = D == 128 ? sQK + 16384 : smem + PL::oX + 8192;
 
     if (warp == 4) {
         if (lane == 0) {
-            // ---- loads ----
-            mbar_arrive_expect_tx(&ms.barLoad, 3 * PL::kTile);
+            mbar_arrive_expect_tx(&ms.barLoad, PL::kLoadBytes);
             for (int kb = 0; kb < KB; ++kb) {
-                tma_load_4d(sK + kb * 16384, &map_k, &ms.barLoad, kb * 64, h, tok_first, b);
-                tma_load_4d(sX + kb * 16384, &map_q, &ms.barLoad, kb * 64, h, tok_first, b);
-                tma_load_4d(sV + kb * 16384, &map_v, &ms.barLoad, kb * 64, h, tok_first, b);
+                tma_load_4d(sQK + kb * 16384 + 8192, &map_k, &ms.barLoad, kb * 64, h, tok0, b);
+                tma_load_4d(sQK + kb * 16384, &map_q, &ms.barLoad, kb * 64, h, tok0, b);
+                tma_load_4d(sV + kb * 8192, &map_v, &ms.barLoad, kb * 64, h, tok0, b);
             }
             bool ok = mbar_wait(&ms.barConv, 0, abort_flag);       // tiles converted to fp16
             if (ok) {
-                // ---- fp16 copies of q and k for the scan kernel; K K^T and Q K^T ----
-                const int row0 = bh * L + tok_first;
-                for (int kb = 0; kb < KB; ++kb)
-                    for (int hf = 0; hf < (second_valid ? 2 : 1); ++hf) {
-                        tma_store_2d(&map_qh, sX + kb * 16384 + hf * 8192, kb * 64, row0 + hf * 64);
-                        tma_store_2d(&map_kh, sK + kb * 16384 + hf * 8192, kb * 64, row0 + hf * 64);
-                    }
+                // ---- fp16 copies of q and k for the scan kernel; [Q ; K] K^T ----
+                for (int kb = 0; kb < KB; ++kb) {
+                    tma_store_2d(&map_qh, sQK + kb * 16384, kb * 64, bh * L + tok0);
+                    tma_store_2d(&map_kh, sQK + kb * 16384 + 8192, kb * 64, bh * L + tok0);
+                }
                 tma_store_commit();
                 tc_fence_after_sync();
-                constexpr uint32_t idesc = make_idesc(kFmtF16, 128, 128, false, false);
-                const uint32_t aK = smem_u32(sK), aQ = smem_u32(sX);
+                constexpr uint32_t idesc = make_idesc(kFmtF16, 128, 64, false, false);
+                const uint32_t aQK = smem_u32(sQK);
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
-                    for (int k16 = 0; k16 < 4; ++k16) {
-                        const uint64_t dk = desc_kmajor(aK + kb * 16384 + k16 * 32);
-                        mma_ss(tmem, dk, dk, idesc, (kb | k16) != 0);
-                        mma_ss(tmem + 128, desc_kmajor(aQ + kb * 16384 + k16 * 32), dk, idesc,
-                               (kb | k16) != 0);
-                    }
+                    for (int k16 = 0; k16 < 4; ++k16)
+                        mma_ss(tmem, desc_kmajor(aQK + kb * 16384 + k16 * 32),
+                               desc_kmajor(aQK + kb * 16384 + 8192 + k16 * 32), idesc, (kb | k16) != 0);
                 mma_commit(&ms.barM);
-                tma_store_wait_read();                    // the q copy has left its tile
-                ok = mbar_wait(&ms.barM, 0, abort_flag);  // and Q K^T has read it
+                tma_store_wait_read();                    // the q copy has left its blocks
+                ok = mbar_wait(&ms.barM, 0, abort_flag);  // and the MMAs have read them
                 mbar_arrive(&ms.barXfree);
             }
             if (ok) ok = mbar_wait(&ms.barT, 0, abort_flag);
             if (ok) {
-                // ---- U^T = V^T (T beta~)^T,  W^T = K^T (T beta~ gamma)^T, per chunk ----
+                // ---- U^T = V^T (T beta~)^T,  W^T = K^T (T beta~ gamma)^T ----
                 tc_fence_after_sync();
-                const uint32_t aV = smem_u32(sV), aK = smem_u32(sK), aT = smem_u32(sX);
+                const uint32_t aV = smem_u32(sV), aK = smem_u32(sQK) + 8192, aTb = smem_u32(xLo),
+                               aTg = smem_u32(xHi);
                 if (D == 128) {
                     constexpr uint32_t idesc = make_idesc(kFmtF16, 128, 64, true, false);
 #pragma unroll
-                    for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                        for (int k16 = 0; k16 < 4; ++k16) {
-                            mma_ss(tmem + 64 * hf,
-                                   desc_mnmajor(aV + hf * 8192 + k16 * 2048, 16384),
-                                   desc_kmajor(aT + hf * 16384 + k16 * 32), idesc, k16 != 0);
-                            mma_ss(tmem + 128 + 64 * hf,
-                                   desc_mnmajor(aK + hf * 8192 + k16 * 2048, 16384),
-                                   desc_kmajor(aT + hf * 16384 + 8192 + k16 * 32), idesc, k16 != 0);
-                        }
+                    for (int k16 = 0; k16 < 4; ++k16) {
+                        mma_ss(tmem, desc_mnmajor(aV + k16 * 2048, 8192), desc_kmajor(aTb + k16 * 32),
+                               idesc, k16 != 0);
+                        mma_ss(tmem + 64, desc_mnmajor(aK + k16 * 2048, 16384),
+                               desc_kmajor(aTg + k16 * 32), idesc, k16 != 0);
+                    }
                 } else {
-                    // d = 64: rows 0-63 of M are V^T, rows 64-127 are K^T (the K tile follows the V
-                    // tile in shared memory); N = 128 = [T beta~ ; T beta~ gamma].
+                    // d = 64: rows 0-63 of M are V^T, rows 64-127 are K^T (16 KB further on);
+                    // N = 128 = [T beta~ ; T beta~ gamma] (adjacent).
                     constexpr uint32_t idesc = make_idesc(kFmtF16, 128, 128, true, false);
 #pragma unroll
-                    for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                        for (int k16 = 0; k16 < 4; ++k16)
-                            mma_ss(tmem + 128 * hf,
-                                   desc_mnmajor(aV + hf * 8192 + k16 * 2048, 16384),
-                                   desc_kmajor(aT + hf * 16384 + k16 * 32), idesc, k16 != 0);
+                    for (int k16 = 0; k16 < 4; ++k16)
+                        mma_ss(tmem, desc_mnmajor(aV + k16 * 2048, 16384), desc_kmajor(aTb + k16 * 32),
+                               idesc, k16 != 0);
                 }
                 mma_commit(&ms.barUW);
             }
             tma_store_wait_all();
         }
     } else {
-        const int r = tid, hf = r >> 6, i = r & 63;
-        const int c = 2 * pr + hf;                         // this thread's chunk
-        const bool valid = hf == 0 || second_valid;
+        const int r = tid, i = r & 63;
+        const bool solver = r >= 64;                       // rows 64-127: K K^T
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        // ---- gates: beta~, inclusive cumulative log decay within the chunk ----
-        float gv = 0.f, btv = 0.f;
-        if (valid) {
-            const size_t t = ((size_t)b * L + tok_first + r) * H + h;
-            gv = g[t];
-            btv = route[t] ? 0.f : beta[t];
-        }
-        float G = gv;
+        // ---- gates (warps 0-1): beta~, inclusive cumulative log decay within the chunk ----
+        if (!solver) {
+            const size_t t = ((size_t)b * L + tok0 + i) * H + h;
+            float G = g[t];
+            const float btv = route[t] ? 0.f : beta[t];
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float y = __shfl_up_sync(0xffffffffu, G, o);
-            if (lane >= o) G += y;
+            for (int o = 1; o < 32; o <<= 1) {
+                const float y = __shfl_up_sync(0xffffffffu, G, o);
+                if (lane >= o) G += y;
+            }
+            if (lane == 31) ms.wsum[warp] = G;
+            named_barrier_sync(1, 64);
+            if (warp == 1) G += ms.wsum[0];
+            ms.G[i] = G;
+            ms.bt[i] = btv;
         }
-        if (lane == 31) ms.wsum[warp] = G;
-        named_barrier_sync(1, kRowThreads);
-        if (warp & 1) G += ms.wsum[warp - 1];
-        ms.G[r] = G;
-        ms.bt[r] = btv;
         // ---- tiles to fp16, in place ----
         bool ok = mbar_wait(&ms.barLoad, 0, abort_flag);
         if (ok) {
-            for (int idx = r; idx < 3 * PL::kTile / 16; idx += kRowThreads) {
-                uint4 *pp = reinterpret_cast<uint4 *>(smem) + idx;   // V, K, Q tiles are contiguous
+            for (int idx = r; idx < PL::kLoadBytes / 16; idx += kRowThreads) {
+                uint4 *pp = reinterpret_cast<uint4 *>(smem) + idx;   // V and [Q ; K] are contiguous
                 *pp = bf16x8_to_f16x8(*pp);
             }
             fence_proxy_async_smem();
             mbar_arrive(&ms.barConv);
             ok = mbar_wait(&ms.barXfree, 0, abort_flag);
         }
-        float t[64];
         if (ok) {
-            // ---- A (strictly lower) -> A^T in shared memory; P (lower) -> global ----
             tc_fence_after_sync();
-            float *At = reinterpret_cast<float *>(sX) + hf * 4096;   // At[j][m] = A_mj
-            if (valid) {      // decay factors the scan needs: gamma_i and gamma_C / gamma_i
-                float *gd = Gd + ((size_t)bh * NC + c) * 128;
+            const float G = ms.G[i];
+            uint32_t dd[2][32];
+            tmem_ld32(tmem + lane_base, dd[0]);
+            tmem_ld32(tmem + lane_base + 32, dd[1]);
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            if (!solver) {
+                // ---- decay factors for the scan, P (lower triangle) ----
+                float *gd = Gd + chunk * 128;
                 gd[i] = __expf(G);
-                gd[64 + i] = __expf(ms.G[64 * hf + 63] - G);
-            }
-            {
-                uint32_t d1[2][32];
-                tmem_ld32(tmem + lane_base + 64 * hf, d1[0]);
-                tmem_ld32(tmem + lane_base + 64 * hf + 32, d1[1]);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 64; ++j) {
-                    const float a = j < i ? btv * __expf(G - ms.G[64 * hf + j]) *
-                                                __uint_as_float(d1[j >> 5][j & 31])
-                                          : 0.f;
-                    At[j * 64 + i] = a;
-                }
-            }
-            {
-                uint32_t d2[2][32];
-                tmem_ld32(tmem + 128 + lane_base + 64 * hf, d2[0]);
-                tmem_ld32(tmem + 128 + lane_base + 64 * hf + 32, d2[1]);
-                tmem_wait_ld();
-                uint4 *prow = reinterpret_cast<uint4 *>(Ph + (((size_t)bh * NC + c) * 64 + i) * 64);
+                gd[64 + i] = __expf(ms.G[63] - G);
+                uint4 *prow = reinterpret_cast<uint4 *>(Ph + (chunk * 64 + i) * 64);
 #pragma unroll
                 for (int pc = 0; pc < 8; ++pc) {
                     float x[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const int j = 8 * pc + e;
-                        x[e] = j <= i ? scale_la * __expf(G - ms.G[64 * hf + j]) *
-                                            __uint_as_float(d2[j >> 5][j & 31])
+                        x[e] = j <= i ? scale_la * __expf(G - ms.G[j]) * __uint_as_float(dd[j >> 5][j & 31])
                                       : 0.f;
                     }
-                    if (valid)
-                        prow[pc] = make_uint4(pack_half2(x[0], x[1]), pack_half2(x[2], x[3]),
-                                              pack_half2(x[4], x[5]), pack_half2(x[6], x[7]));
+                    prow[pc] = make_uint4(pack_half2(x[0], x[1]), pack_half2(x[2], x[3]),
+                                          pack_half2(x[4], x[5]), pack_half2(x[6], x[7]));
                 }
-            }
-            tc_fence_before_sync();
-            named_barrier_sync(1, kRowThreads);
-            // ---- row i of T = (I + A)^-1 by back substitution: t_j = [j = i] - sum_{m > j} t_m A_mj
+                mbar_arrive(&ms.barT);
+            } else {
+                // ---- A (strictly lower) -> A^T in shared memory: At[j][m] = A_mj ----
+                const float btv = ms.bt[i];
+                float *AtLo = reinterpret_cast<float *>(xLo), *AtHi = reinterpret_cast<float *>(xHi);
 #pragma unroll
-            for (int j = 0; j < 64; ++j) t[j] = 0.f;
-#pragma unroll
-            for (int j = 63; j >= 0; --j) {
-                const float4 *col = reinterpret_cast<const float4 *>(At + j * 64);
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                for (int m4 = (j + 1) / 4; m4 < 16; ++m4) {
-                    const float4 a = col[m4];
-                    a0 = fmaf(t[4 * m4], a.x, a0);
-                    a1 = fmaf(t[4 * m4 + 1], a.y, a1);
-                    a2 = fmaf(t[4 * m4 + 2], a.z, a2);
-                    a3 = fmaf(t[4 * m4 + 3], a.w, a3);
+                for (int j = 0; j < 64; ++j) {
+                    const float a = j < i ? btv * __expf(G - ms.G[j]) * __uint_as_float(dd[j >> 5][j & 31]) : 0.f;
+                    (j < 32 ? AtLo + j * 64 : AtHi + (j - 32) * 64)[i] = a;
                 }
-                t[j] = (j == i ? 1.f : 0.f) - ((a0 + a1) + (a2 + a3));
-            }
-            named_barrier_sync(1, kRowThreads);          // everyone is done reading A^T
-            // ---- operands T diag(beta~) and T diag(beta~ gamma), fp16 rows ----
-            uint8_t *tb = sX + hf * 16384, *tg = tb + 8192;
+                named_barrier_sync(2, 64);
+                // ---- row i of T = (I + A)^-1 by back substitution, t_j = [j = i] - sum_{m > j} t_m A_mj,
+                // in four blocks of 16 columns from the right.  Real loops keep the code small (a
+                // fully unrolled solve is ~40 KB of instructions executed once: instruction fetch
+                // becomes the bottleneck); the 16 values of the block in flight sit in registers,
+                // finished blocks are parked in this thread's column of the A^T rows they belong to,
+                // which nobody reads any more.
+                auto At_row = [&](int j) { return j < 32 ? AtLo + j * 64 : AtHi + (j - 32) * 64; };
+#pragma unroll 1
+                for (int jb = 3; jb >= 0; --jb) {
+                    float acc[16];
 #pragma unroll
-            for (int pc = 0; pc < 8; ++pc) {
-                float xb[8], xg[8];
+                    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+#pragma unroll 1
+                    for (int m0 = 16 * (jb + 1); m0 < 64; m0 += 4) {      // finished columns m > block
+                        const float t0 = At_row(m0)[i], t1 = At_row(m0 + 1)[i], t2 = At_row(m0 + 2)[i],
+                                    t3 = At_row(m0 + 3)[i];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int j = 8 * pc + e;
-                    xb[e] = t[j] * ms.bt[64 * hf + j];
-                    xg[e] = xb[e] * __expf(ms.G[64 * hf + j]);
+                        for (int j = 0; j < 16; ++j) {
+                            const float4 a = *reinterpret_cast<const float4 *>(At_row(16 * jb + j) + m0);
+                            acc[j] = fmaf(t0, a.x, fmaf(t1, a.y, fmaf(t2, a.z, fmaf(t3, a.w, acc[j]))));
+                        }
+                    }
+                    float tb[16];
+#pragma unroll
+                    for (int j = 15; j >= 0; --j) {                     // inside the block
+                        const float *row = At_row(16 * jb + j) + 16 * jb;
+                        float sacc = acc[j];
+#pragma unroll
+                        for (int m = j + 1; m < 16; ++m) sacc = fmaf(tb[m], row[m], sacc);
+                        tb[j] = (16 * jb + j == i ? 1.f : 0.f) - sacc;
+                    }
+                    named_barrier_sync(2, 64);      // both solver warps are done with the block's rows
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) At_row(16 * jb + j)[i] = tb[j];
                 }
-                *reinterpret_cast<uint4 *>(tb + sw128_offset(i, pc)) =
-                    make_uint4(pack_half2(xb[0], xb[1]), pack_half2(xb[2], xb[3]),
-                               pack_half2(xb[4], xb[5]), pack_half2(xb[6], xb[7]));
-                *reinterpret_cast<uint4 *>(tg + sw128_offset(i, pc)) =
-                    make_uint4(pack_half2(xg[0], xg[1]), pack_half2(xg[2], xg[3]),
-                               pack_half2(xg[4], xg[5]), pack_half2(xg[6], xg[7]));
+                // ---- operands T diag(beta~) and T diag(beta~ gamma), fp16 rows ----
+                float t[64];
+#pragma unroll
+                for (int j = 0; j < 64; ++j) t[j] = At_row(j)[i];
+                named_barrier_sync(2, 64);          // every row is in registers: the region can be reused
+#pragma unroll
+                for (int pc = 0; pc < 8; ++pc) {
+                    float xb[8], xg[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int j = 8 * pc + e;
+                        xb[e] = t[j] * ms.bt[j];
+                        xg[e] = xb[e] * __expf(ms.G[j]);
+                    }
+                    *reinterpret_cast<uint4 *>(xLo + sw128_offset(i, pc)) =
+                        make_uint4(pack_half2(xb[0], xb[1]), pack_half2(xb[2], xb[3]),
+                                   pack_half2(xb[4], xb[5]), pack_half2(xb[6], xb[7]));
+                    *reinterpret_cast<uint4 *>(xHi + sw128_offset(i, pc)) =
+                        make_uint4(pack_half2(xg[0], xg[1]), pack_half2(xg[2], xg[3]),
+                                   pack_half2(xg[4], xg[5]), pack_half2(xg[6], xg[7]));
+                }
+                fence_proxy_async_smem();
+                mbar_arrive(&ms.barT);
             }
-            fence_proxy_async_smem();
-            mbar_arrive(&ms.barT);
             ok = mbar_wait(&ms.barUW, 0, abort_flag);
         }
         if (ok) {
             // ---- U^T (fp32) and W^T (fp16) rows to global; thread r <-> head-dimension row ----
             tc_fence_after_sync();
+            const bool do_u = D == 128 || r < 64, do_w = D == 128 || r >= 64;
+            const int row = D == 128 ? r : i;
+            uint32_t x[2][32];
+            if (do_u) {                                     // warp-uniform
+                tmem_ld32(tmem + lane_base, x[0]);
+                tmem_ld32(tmem + lane_base + 32, x[1]);
+                tmem_wait_ld();
+                // piece-major: 16-byte piece pc (4 tokens) of all D rows is contiguous, so that a
+                // warp's stores here and its loads in the scan are fully coalesced
+                uint4 *dst = reinterpret_cast<uint4 *>(Ut + chunk * D * 64) + row;
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                if (hh == 1 && !second_valid) break;
-                const size_t chunk = (size_t)bh * NC + 2 * pr + hh;
-                const bool do_u = D == 128 || r < 64, do_w = D == 128 || r >= 64;
-                const int row = D == 128 ? r : (r & 63);
-                const int col_u = D == 128 ? 64 * hh : 128 * hh;
-                const int col_w = D == 128 ? 128 + 64 * hh : 128 * hh + 64;
-                uint32_t x[2][32];
-                if (do_u) {                                 // warp-uniform
-                    tmem_ld32(tmem + lane_base + col_u, x[0]);
-                    tmem_ld32(tmem + lane_base + col_u + 32, x[1]);
-                    tmem_wait_ld();
-                    // piece-major: 16-byte piece pc (4 tokens) of all D rows is contiguous, so that a
-                    // warp's stores here and its loads in the scan are fully coalesced
-                    uint4 *dst = reinterpret_cast<uint4 *>(Ut + chunk * D * 64) + row;
-#pragma unroll
-                    for (int pc = 0; pc < 16; ++pc)
-                        dst[pc * D] = make_uint4(x[pc >> 3][(4 * pc) & 31], x[pc >> 3][(4 * pc + 1) & 31],
+                for (int pc = 0; pc < 16; ++pc)
+                    dst[pc * D] = make_uint4(x[pc >> 3][(4 * pc) & 31], x[pc >> 3][(4 * pc + 1) & 31],
                                              x[pc >> 3][(4 * pc + 2) & 31], x[pc >> 3][(4 * pc + 3) & 31]);
-                }
-                if (do_w) {
-                    tmem_ld32(tmem + lane_base + col_w, x[0]);
-                    tmem_ld32(tmem + lane_base + col_w + 32, x[1]);
-                    tmem_wait_ld();
-                    uint4 *dst = reinterpret_cast<uint4 *>(Wt + (chunk * D + row) * 64);
+            }
+            if (do_w) {
+                tmem_ld32(tmem + lane_base + 64, x[0]);
+                tmem_ld32(tmem + lane_base + 96, x[1]);
+                tmem_wait_ld();
+                uint4 *dst = reinterpret_cast<uint4 *>(Wt + (chunk * D + row) * 64);
 #pragma unroll
-                    for (int pc = 0; pc < 8; ++pc) {
-                        const uint32_t *xx = &x[pc >> 2][(8 * pc) & 31];
-                        dst[pc] = make_uint4(
-                            pack_half2(__uint_as_float(xx[0]), __uint_as_float(xx[1])),
-                            pack_half2(__uint_as_float(xx[2]), __uint_as_float(xx[3])),
-                            pack_half2(__uint_as_float(xx[4]), __uint_as_float(xx[5])),
-                            pack_half2(__uint_as_float(xx[6]), __uint_as_float(xx[7])));
-                    }
+                for (int pc = 0; pc < 8; ++pc) {
+                    const uint32_t *xx = &x[pc >> 2][(8 * pc) & 31];
+                    dst[pc] = make_uint4(pack_half2(__uint_as_float(xx[0]), __uint_as_float(xx[1])),
+                                         pack_half2(__uint_as_float(xx[2]), __uint_as_float(xx[3])),
+                                         pack_half2(__uint_as_float(xx[4]), __uint_as_float(xx[5])),
+                                         pack_half2(__uint_as_float(xx[6]), __uint_as_float(xx[7])));
                 }
             }
         }
@@ -345,7 +342,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     __syncthreads();
     if (warp == 4) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem, 256);
+        tmem_dealloc(tmem, 128);
     }
     if (tid == 0 && ms.abort_flag) atomicMin(status, (int)NATSL_ERR_TIMEOUT);
 }
@@ -666,9 +663,9 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
     const int NC = s.L / kC;
     const uint64_t BH = (uint64_t)s.B * s.H;
     CUtensorMap mq, mk, mv, mqh, mkh;
-    if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, 128) ||
-        !tch::make_map_blhd(&mk, k, s.B, s.L, s.H, D, 128) ||
-        !tch::make_map_blhd(&mv, v, s.B, s.L, s.H, D, 128) ||
+    if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, 64) ||
+        !tch::make_map_blhd(&mk, k, s.B, s.L, s.H, D, 64) ||
+        !tch::make_map_blhd(&mv, v, s.B, s.L, s.H, D, 64) ||
         !tch::make_map_2d(&mqh, ws.Qh, BH * s.L, D, 64) ||
         !tch::make_map_2d(&mkh, ws.Kh, BH * s.L, D, 64))
         return cudaErrorInvalidValue;
@@ -676,7 +673,7 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          PrepLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
-    dim3 grid((NC + 1) / 2, s.B * s.H);
+    dim3 grid(NC, s.B * s.H);
     gdn_prepare_tc_kernel<D><<<grid, kPrepThreads, PrepLayout<D>::kTotal, st>>>(
         mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut, (__half *)ws.Ph, ws.Gd,
         status, s.L, s.H);
