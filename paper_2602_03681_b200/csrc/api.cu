@@ -101,6 +101,7 @@ struct BwdWs {
     float *S_c, *dS_c;                                       // [B,H,NC,d,d]
     float *Gcum, *lse, *Dsm, *dGrow, *kappa, *gS;            // [B,H,L] (gS: [B,H,NC,d/32])
     void *k_smb, *k16, *v16, *Qh, *dO16;                     // tensor-core softmax branch: 16-bit [B,H,L,d]
+    GdnTcWs tc;                                              // tensor-core forward recomputation
     size_t bytes;
 };
 
@@ -132,6 +133,15 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.v16 = c.take<char>(h16);
     f.Qh = c.take<char>(h16);
     f.dO16 = c.take<char>(h16);
+    f.tc = GdnTcWs{};
+    if (use_tensor_cores(p)) {
+        f.tc.Qh = f.Qh;                       // the same fp16 copy of q serves both branches
+        f.tc.Kh = c.take<char>(h16);
+        f.tc.Wt = c.take<char>(h16);
+        f.tc.Ut = c.take<float>(TM);
+        f.tc.Ph = c.take<char>(CC * 2);
+        f.tc.Gd = c.take<float>(BHL * 2);
+    }
     f.bytes = c.off;
     return f;
 }
@@ -230,10 +240,11 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(mark());
     float *o_la = p->o_la ? p->o_la : f.o_la;
     if (tensor_cores) {
-        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, f.status, s, st));
+        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, GdnTcExport{}, f.status,
+                                        s, st));
         NATSL_TRY(mark());
-        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, p->state_out, o_la, f.status, s,
-                                     st));
+        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, p->state_out, o_la, GdnTcExport{},
+                                     f.status, s, st));
     } else {
         NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P,
                                           nullptr, nullptr, s, st));
@@ -292,10 +303,16 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     else
         NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
                                    f.status, s32, st));
-    NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
-                                      f.P, f.Abar, f.Gcum, s32, st));
-    NATSL_TRY(launch_gdn_scan_simt(f.q32, f.k32, g, f.W, f.U, f.P, p->scale_la, nullptr, nullptr,
-                                   f.S_c, f.Ut, f.o_la, s32, st));
+    if (tensor_cores) {
+        const GdnTcExport ex{f.W, f.U, f.P, f.Abar, f.Gcum, f.S_c, f.Ut};
+        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, ex, f.status, s, st));
+        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex, f.status, s, st));
+    } else {
+        NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
+                                          f.P, f.Abar, f.Gcum, s32, st));
+        NATSL_TRY(launch_gdn_scan_simt(f.q32, f.k32, g, f.W, f.U, f.P, p->scale_la, nullptr, nullptr,
+                                       f.S_c, f.Ut, f.o_la, s32, st));
+    }
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la,
                                             p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,

@@ -79,8 +79,8 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                       const __grid_constant__ CUtensorMap map_kh, const float *__restrict__ g,
                       const float *__restrict__ beta, const uint8_t *__restrict__ route,
                       float scale_la, __half *__restrict__ Wt, float *__restrict__ Ut,
-                      __half *__restrict__ Ph, float *__restrict__ Gd, int32_t *status, int L,
-                      int H) {
+                      __half *__restrict__ Ph, float *__restrict__ Gd, GdnTcExport ex,
+                      int32_t *status, int L, int H) {
     using PL = PrepLayout<D>;
     constexpr int KB = PL::KB;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -219,6 +219,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 float *gd = Gd + chunk * 128;
                 gd[i] = __expf(G);
                 gd[64 + i] = __expf(ms.G[63] - G);
+                if (ex.Gcum) ex.Gcum[(size_t)bh * L + tok0 + i] = G;
                 uint4 *prow = reinterpret_cast<uint4 *>(Ph + (chunk * 64 + i) * 64);
 #pragma unroll
                 for (int pc = 0; pc < 8; ++pc) {
@@ -231,6 +232,11 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     }
                     prow[pc] = make_uint4(pack_half2(x[0], x[1]), pack_half2(x[2], x[3]),
                                           pack_half2(x[4], x[5]), pack_half2(x[6], x[7]));
+                    if (ex.P) {
+                        float4 *pf = reinterpret_cast<float4 *>(ex.P + (chunk * 64 + i) * 64 + 8 * pc);
+                        pf[0] = make_float4(x[0], x[1], x[2], x[3]);
+                        pf[1] = make_float4(x[4], x[5], x[6], x[7]);
+                    }
                 }
                 mbar_arrive(&ms.barT);
             } else {
@@ -239,8 +245,9 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 float *AtLo = reinterpret_cast<float *>(xLo), *AtHi = reinterpret_cast<float *>(xHi);
 #pragma unroll
                 for (int j = 0; j < 64; ++j) {
-                    const float a = j < i ? btv * __expf(G - ms.G[j]) * __uint_as_float(dd[j >> 5][j & 31]) : 0.f;
-                    (j < 32 ? AtLo + j * 64 : AtHi + (j - 32) * 64)[i] = a;
+                    const float ab = j < i ? __expf(G - ms.G[j]) * __uint_as_float(dd[j >> 5][j & 31]) : 0.f;
+                    (j < 32 ? AtLo + j * 64 : AtHi + (j - 32) * 64)[i] = btv * ab;
+                    if (ex.Abar) ex.Abar[(chunk * 64 + i) * 64 + j] = ab;   // A without the beta~ row factor
                 }
                 named_barrier_sync(2, 64);
                 // ---- row i of T = (I + A)^-1 by back substitution, t_j = [j = i] - sum_{m > j} t_m A_mj,
@@ -321,11 +328,21 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 for (int pc = 0; pc < 16; ++pc)
                     dst[pc * D] = make_uint4(x[pc >> 3][(4 * pc) & 31], x[pc >> 3][(4 * pc + 1) & 31],
                                              x[pc >> 3][(4 * pc + 2) & 31], x[pc >> 3][(4 * pc + 3) & 31]);
+                if (ex.U) {      // token-major fp32 copy
+                    float *uf = ex.U + (((size_t)b * L + tok0) * H + h) * D + row;
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) uf[(size_t)j * H * D] = __uint_as_float(x[j >> 5][j & 31]);
+                }
             }
             if (do_w) {
                 tmem_ld32(tmem + lane_base + 64, x[0]);
                 tmem_ld32(tmem + lane_base + 96, x[1]);
                 tmem_wait_ld();
+                if (ex.W) {
+                    float *wf = ex.W + (((size_t)b * L + tok0) * H + h) * D + row;
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) wf[(size_t)j * H * D] = __uint_as_float(x[j >> 5][j & 31]);
+                }
                 uint4 *dst = reinterpret_cast<uint4 *>(Wt + (chunk * D + row) * 64);
 #pragma unroll
                 for (int pc = 0; pc < 8; ++pc) {
@@ -401,7 +418,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                    const __grid_constant__ CUtensorMap map_ph, const float *__restrict__ Ut,
                    const float *__restrict__ Gd, float scale_la,
                    const float *__restrict__ state_in, float *__restrict__ state_out,
-                   float *__restrict__ o_la, int32_t *status, int L, int H) {
+                   float *__restrict__ o_la, GdnTcExport ex, int32_t *status, int L, int H) {
     using SL = ScanLayout<D>;
     constexpr int KB = SL::KB;
     constexpr int kHalfCols = D / 2;                       // state columns per thread
@@ -566,6 +583,11 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 }
                 tc_fence_before_sync();
             }
+            if (ex.S_c && active) {      // chunk-entry state, [B,H,L/C,dk,dv]
+                float *sc = ex.S_c + (((size_t)bh * NC + c) * D + col0) * D + r;
+#pragma unroll
+                for (int x = 0; x < kHalfCols; ++x) sc[(size_t)x * D] = S[x];
+            }
             // ---- (a) state row -> fp16 operand in TMEM; decay the register copy afterwards ----
             {
                 uint32_t pk[kHalfCols / 2];
@@ -608,6 +630,11 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 32; ++j) u[j] -= __uint_as_float(ws[j]);
+            }
+            if (ex.Ut && active) {       // U~, token-major
+                float *ut = ex.Ut + (((size_t)b * L + (size_t)c * 64 + tk0) * H + h) * D + r;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) ut[(size_t)j * H * D] = u[j];
             }
             {
                 uint32_t pk[32];     // [0,16): U~ of this thread's 32 tokens, [16,32): U~ gamma_C/gamma
@@ -659,7 +686,8 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
 template <int D>
 static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, const float *g,
                                    const float *beta, const uint8_t *route, float scale_la,
-                                   const GdnTcWs &ws, int32_t *status, Shape s, cudaStream_t st) {
+                                   const GdnTcWs &ws, const GdnTcExport &ex, int32_t *status, Shape s,
+                                   cudaStream_t st) {
     const int NC = s.L / kC;
     const uint64_t BH = (uint64_t)s.B * s.H;
     CUtensorMap mq, mk, mv, mqh, mkh;
@@ -676,15 +704,15 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
     dim3 grid(NC, s.B * s.H);
     gdn_prepare_tc_kernel<D><<<grid, kPrepThreads, PrepLayout<D>::kTotal, st>>>(
         mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut, (__half *)ws.Ph, ws.Gd,
-        status, s.L, s.H);
+        ex, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
 
 template <int D>
 static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *state_in,
-                                float *state_out, float *o_la, int32_t *status, Shape s,
-                                cudaStream_t st) {
+                                float *state_out, float *o_la, const GdnTcExport &ex, int32_t *status,
+                                Shape s, cudaStream_t st) {
     const int NC = s.L / kC;
     const uint64_t BH = (uint64_t)s.B * s.H;
     CUtensorMap mwt, mqh, mkh, mph;
@@ -698,23 +726,24 @@ static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *
                                          ScanLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
     gdn_scan_tc_kernel<D><<<s.B * s.H, kScanThreads, ScanLayout<D>::kTotal, st>>>(
-        mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, o_la, status, s.L, s.H);
+        mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, o_la, ex, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, const float *g,
                                   const float *beta, const uint8_t *route, float scale_la,
-                                  const GdnTcWs &ws, int32_t *status, Shape s, cudaStream_t st) {
-    if (s.d == 128) return prepare_tc_impl<128>(q, k, v, g, beta, route, scale_la, ws, status, s, st);
-    return prepare_tc_impl<64>(q, k, v, g, beta, route, scale_la, ws, status, s, st);
+                                  const GdnTcWs &ws, const GdnTcExport &ex, int32_t *status, Shape s,
+                                  cudaStream_t st) {
+    if (s.d == 128) return prepare_tc_impl<128>(q, k, v, g, beta, route, scale_la, ws, ex, status, s, st);
+    return prepare_tc_impl<64>(q, k, v, g, beta, route, scale_la, ws, ex, status, s, st);
 }
 
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
-                               float *state_out, float *o_la, int32_t *status, Shape s,
-                               cudaStream_t st) {
-    if (s.d == 128) return scan_tc_impl<128>(ws, scale_la, state_in, state_out, o_la, status, s, st);
-    return scan_tc_impl<64>(ws, scale_la, state_in, state_out, o_la, status, s, st);
+                               float *state_out, float *o_la, const GdnTcExport &ex, int32_t *status,
+                               Shape s, cudaStream_t st) {
+    if (s.d == 128) return scan_tc_impl<128>(ws, scale_la, state_in, state_out, o_la, ex, status, s, st);
+    return scan_tc_impl<64>(ws, scale_la, state_in, state_out, o_la, ex, status, s, st);
 }
 
 }  // namespace natsl

@@ -72,12 +72,22 @@ struct GdnTcWs {
     void *Ph;        // P per chunk, fp16                [B,H,L/C,64,64]
     float *Gd;       // per chunk: gamma_i (64), gamma_C / gamma_i (64), fp32   [B,H,L/C,128]
 };
+// Optional fp32 copies of the chunkwise quantities the backward needs (all may be null).
+struct GdnTcExport {
+    float *W, *U;    // token-major [B,L,H,d]
+    float *P;        // [B,H,L/C,64,64]
+    float *Abar;     // A without its beta~ row factor, [B,H,L/C,64,64]
+    float *Gcum;     // in-chunk cumulative log decay [B,H,L]
+    float *S_c;      // chunk-entry states [B,H,L/C,d,d]
+    float *Ut;       // U~ = U - W S, token-major [B,L,H,d]
+};
 cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, const float *g,
                                   const float *beta, const uint8_t *route, float scale_la,
-                                  const GdnTcWs &ws, int32_t *status, Shape s, cudaStream_t st);
+                                  const GdnTcWs &ws, const GdnTcExport &ex, int32_t *status, Shape s,
+                                  cudaStream_t st);
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
-                               float *state_out, float *o_la, int32_t *status, Shape s,
-                               cudaStream_t st);
+                               float *state_out, float *o_la, const GdnTcExport &ex, int32_t *status,
+                               Shape s, cudaStream_t st);
 
 // bwd_simt.cu -- fp32 CUDA-core backward
 // A batched matrix operand: element (r, c) of batch (b, h, chunk) is
