@@ -102,6 +102,7 @@ struct BwdWs {
     float *Gcum, *lse, *Dsm, *dGrow, *kappa, *gS;            // [B,H,L] (gS: [B,H,NC,d/32])
     void *k_smb, *k16, *v16, *Qh, *dO16;                     // tensor-core softmax branch: 16-bit [B,H,L,d]
     GdnTcWs tc;                                              // tensor-core forward recomputation
+    float *Tinv;                                             // (I + A)^-1 per chunk [B,H,NC,64,64]
     size_t bytes;
 };
 
@@ -141,6 +142,9 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
         f.tc.Ut = c.take<float>(TM);
         f.tc.Ph = c.take<char>(CC * 2);
         f.tc.Gd = c.take<float>(BHL * 2);
+        f.Tinv = c.take<float>(CC);
+    } else {
+        f.Tinv = nullptr;
     }
     f.bytes = c.off;
     return f;
@@ -304,7 +308,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
                                    f.status, s32, st));
     if (tensor_cores) {
-        const GdnTcExport ex{f.W, f.U, f.P, f.Abar, f.Gcum, f.S_c, f.Ut};
+        const GdnTcExport ex{f.W, f.U, f.P, f.Abar, f.Tinv, f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, ex, f.status, s, st));
         NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex, f.status, s, st));
     } else {
@@ -337,7 +341,12 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 1, TM(f.do_la), TM(f.Ut), CC(f.N), kC, kC, di, 1.f, false, s, st));
-    NATSL_TRY(launch_gdn_tsolve(f.Abar, beta, route, f.dW, f.dUt, f.dKb, f.dVb, s, st));
+    if (tensor_cores) {   // [dKb | dVb] = (I + A)^-T [dW | dU~] with the inverse the forward already formed
+        NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dW), TM(f.dKb), kC, di, kC, 1.f, false, s, st));
+        NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dUt), TM(f.dVb), kC, di, kC, 1.f, false, s, st));
+    } else {
+        NATSL_TRY(launch_gdn_tsolve(f.Abar, beta, route, f.dW, f.dUt, f.dKb, f.dVb, s, st));
+    }
     NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dKb), TM(f.W), CC(f.M), kC, kC, di, -1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dVb), TM(f.U), CC(f.M), kC, kC, di, -1.f, true, s, st));
     NATSL_TRY(launch_mask_scale(f.M, f.N, f.Gcum, beta, route, p->scale_la, f.Mg, f.Ms, f.Ns, s, st));

@@ -289,6 +289,12 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 float t[64];
 #pragma unroll
                 for (int j = 0; j < 64; ++j) t[j] = At_row(j)[i];
+                if (ex.T) {
+                    float4 *tr = reinterpret_cast<float4 *>(ex.T + (chunk * 64 + i) * 64);
+#pragma unroll
+                    for (int j4 = 0; j4 < 16; ++j4)
+                        tr[j4] = make_float4(t[4 * j4], t[4 * j4 + 1], t[4 * j4 + 2], t[4 * j4 + 3]);
+                }
                 named_barrier_sync(2, 64);          // every row is in registers: the region can be reused
 #pragma unroll
                 for (int pc = 0; pc < 8; ++pc) {
