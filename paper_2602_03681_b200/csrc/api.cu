@@ -101,6 +101,7 @@ struct BwdWs {
     float *S_c, *dS_c;                                       // [B,H,NC,d,d]
     float *Gcum, *lse, *Dsm, *dGrow, *kappa, *gS;            // [B,H,L] (gS: [B,H,NC,d/32])
     void *k_smb, *k16, *v16, *Qh, *dO16;                     // tensor-core softmax branch: 16-bit [B,H,L,d]
+    void *dOla16, *dOlag16;                                  // tensor-core reverse scan: fp16 [B,H,L,d]
     GdnTcWs tc;                                              // tensor-core forward recomputation
     float *Tinv;                                             // (I + A)^-1 per chunk [B,H,NC,64,64]
     size_t bytes;
@@ -134,6 +135,8 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.v16 = c.take<char>(h16);
     f.Qh = c.take<char>(h16);
     f.dO16 = c.take<char>(h16);
+    f.dOla16 = c.take<char>(h16);
+    f.dOlag16 = c.take<char>(h16);
     f.tc = GdnTcWs{};
     if (use_tensor_cores(p)) {
         f.tc.Qh = f.Qh;                       // the same fp16 copy of q serves both branches
@@ -327,7 +330,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                               f.lse, s32, st));
     // ---- combination and softmax branch ----
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la, f.do_nla, dw, f.Dsm,
-                                 tensor_cores ? f.dO16 : nullptr, s, st));
+                                 tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
+                                 tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, s, st));
     if (tensor_cores)
         NATSL_TRY(launch_softmax_bwd_tc(q, f.Qh, f.dO16, f.k16, f.v16, p->L, f.sm_idx, f.prefix, f.lse,
                                         f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, f.status, s, st));
@@ -335,8 +339,11 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_softmax_bwd(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix, f.do_nla,
                                      f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
     // ---- linear branch: reverse scan, then chunk-parallel products ----
-    NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
-                               f.dS_c, f.gS, s, st));
+    if (tensor_cores)
+        NATSL_TRY(launch_gdn_rscan_tc(f.dOla16, f.dOlag16, f.tc, f.S_c, f.dUt, f.dS_c, f.gS, f.status, s, st));
+    else
+        NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
+                                   f.dS_c, f.gS, s, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, s, st));

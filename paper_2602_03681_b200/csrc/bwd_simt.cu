@@ -132,7 +132,9 @@ __global__ void __launch_bounds__(kThreads)
 combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_nla,
                    const T *__restrict__ dout, const float *__restrict__ w, float eps,
                    float *__restrict__ do_la, float *__restrict__ do_nla, float *__restrict__ dw,
-                   float *__restrict__ Dsm, __half *__restrict__ do16, int B, int L, int H) {
+                   float *__restrict__ Dsm, __half *__restrict__ do16,
+                   __half *__restrict__ dola16, __half *__restrict__ dolag16,
+                   const float *__restrict__ Gd, float scale_la, int B, int L, int H) {
     constexpr int kCols = D / 32;
     const int lane = threadIdx.x & 31;
     const size_t row = (size_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
@@ -151,6 +153,8 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
     ssl = warp_sum(ssl); ssn = warp_sum(ssn);
     const float fl = rsqrtf(ssl / D + eps), fn = rsqrtf(ssn / D + eps);
     const float wn = w ? w[row * 2] : 0.5f, wl = w ? w[row * 2 + 1] : 0.5f;
+    // scale_la gamma_l of the token (decay from its chunk's entry), for the reverse scan's operand
+    const float sg = dolag16 ? scale_la * Gd[((size_t)(b * H + h) * (L / kC) + l / kC) * 128 + l % kC] : 0.f;
     float dwl = 0.f, dwn = 0.f;
 #pragma unroll
     for (int x = 0; x < kCols; ++x) {
@@ -167,7 +171,12 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
         const float dn = fn * (wn * dy[x] - on[x] * fn * mn);
         do_la[i] = dl;
         do_nla[i] = dn;
-        if (do16) do16[((((size_t)b * H + h) * L + l) * D) + lane + 32 * x] = __float2half_rn(dn);
+        const size_t i16 = ((((size_t)b * H + h) * L + l) * D) + lane + 32 * x;
+        if (do16) do16[i16] = __float2half_rn(dn);
+        if (dolag16) {
+            dola16[i16] = __float2half_rn(dl);
+            dolag16[i16] = __float2half_rn(sg * dl);
+        }
         dsm = fmaf(dn, on[x], dsm);
     }
     dsm = warp_sum(dsm);
@@ -702,23 +711,26 @@ cudaError_t launch_to_f32(const void *a, const void *b, const void *c, float *a3
 template <typename T, int D>
 static cudaError_t combine_bwd_impl(const float *o_la, const float *o_nla, const void *dout,
                                     const float *w, float eps, float *do_la, float *do_nla,
-                                    float *dw, float *Dsm, void *do16, Shape s, cudaStream_t st) {
+                                    float *dw, float *Dsm, void *do16, void *dola16, void *dolag16,
+                                    const float *Gd, float scale_la, Shape s, cudaStream_t st) {
     const size_t rows = (size_t)s.B * s.L * s.H;
     combine_bwd_kernel<T, D><<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
-        o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, (__half *)do16, s.B, s.L, s.H);
+        o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, (__half *)do16, (__half *)dola16,
+        (__half *)dolag16, Gd, scale_la, s.B, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_combine_bwd(const float *o_la, const float *o_nla, const void *dout,
                                const float *w, float eps, float *do_la, float *do_nla, float *dw,
-                               float *Dsm, void *do16, Shape s, cudaStream_t st) {
+                               float *Dsm, void *do16, void *dola16, void *dolag16, const float *Gd,
+                               float scale_la, Shape s, cudaStream_t st) {
     if (s.bf16) {
-        if (s.d == 128) return combine_bwd_impl<__nv_bfloat16, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, s, st);
-        return combine_bwd_impl<__nv_bfloat16, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, s, st);
+        if (s.d == 128) return combine_bwd_impl<__nv_bfloat16, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, s, st);
+        return combine_bwd_impl<__nv_bfloat16, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, s, st);
     }
-    if (s.d == 128) return combine_bwd_impl<float, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, s, st);
-    return combine_bwd_impl<float, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, s, st);
+    if (s.d == 128) return combine_bwd_impl<float, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, s, st);
+    return combine_bwd_impl<float, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, s, st);
 }
 
 template <int D>

@@ -107,7 +107,8 @@ cudaError_t launch_to_f32(const void *a, const void *b, const void *c, float *a3
 // do16: optional fp16 copy of do_nla in [B,H,L,d] layout (tensor-core softmax backward).
 cudaError_t launch_combine_bwd(const float *o_la, const float *o_nla, const void *dout,
                                const float *w, float eps, float *do_la, float *do_nla, float *dw,
-                               float *Dsm, void *do16, Shape s, cudaStream_t st);
+                               float *Dsm, void *do16, void *dola16, void *dolag16, const float *Gd,
+                               float scale_la, Shape s, cudaStream_t st);
 cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const float *v_sm32, int cap,
                                const int32_t *sm_idx, const int32_t *sm_chunk_prefix,
                                const float *do_nla, const float *lse, const float *Dsm,
@@ -117,6 +118,11 @@ cudaError_t launch_gdn_rscan(const float *q32, const float *k32, const float *Gc
                              const float *P, const float *do_la, const float *chunk_states,
                              float scale_la, float *dUt, float *dS_c, float *gS, Shape s,
                              cudaStream_t st);
+// Tensor-core reverse scan (gdn_bwd_tc.cu): dO16 / dOg16 are fp16 [B,H,L,d] copies of the read-out
+// gradient and of scale_la gamma times it; outputs as launch_gdn_rscan (gS: slot 0 of each row).
+cudaError_t launch_gdn_rscan_tc(const void *dO16, const void *dOg16, const GdnTcWs &ws,
+                                const float *S_c, float *dUt, float *dS_c, float *gS,
+                                int32_t *status, Shape s, cudaStream_t st);
 cudaError_t launch_gdn_tsolve(const float *Abar, const float *beta, const uint8_t *route,
                               const float *dW, const float *dUt, float *dKb, float *dVb, Shape s,
                               cudaStream_t st);
