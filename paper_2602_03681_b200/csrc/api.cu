@@ -311,7 +311,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
                                    f.status, s32, st));
     if (tensor_cores) {
-        const GdnTcExport ex{f.W, f.U, f.P, f.Abar, f.Tinv, f.Gcum, f.S_c, f.Ut};
+        const GdnTcExport ex{f.W, f.U, f.P, f.Tinv, f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, ex, f.status, s, st));
         NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex, f.status, s, st));
     } else {

@@ -11,8 +11,10 @@
 // Precision.  q, k, v are exact bf16 inputs, but T, W, U~, P and S are computed quantities: an
 // 8-bit significand on them puts the layer output 1.4-2e-2 x RMS off (the whole error budget), so
 // every tensor-core operand here is fp16 (11-bit significand; the inputs convert exactly, all
-// magnitudes are O(1) and decay factors only shrink them), T is solved in fp32, and U, which is
-// only ever added to an accumulator, stays fp32.
+// magnitudes are O(1) and decay factors only shrink them).  The 16x16 diagonal blocks of T are
+// inverted in fp32, its blocks below the diagonal come from fp16 products with fp32 accumulation
+// (their error stays at the level of the fp16 rounding T gets as an operand anyway), and U, which
+// is only ever added to an accumulator, stays fp32.
 //
 // All products are laid out "transposed", with the head dimension on the MMA's M axis
 // (M = 128 rows = TMEM lanes = one thread each) and the 64 tokens of a chunk on N or K, so that
@@ -42,11 +44,12 @@ __device__ __forceinline__ uint4 bf16x8_to_f16x8(uint4 u) {
 // ==========================================================================================
 // Prepare: one CTA per chunk of one (batch, head).  One MMA group with M = 128 stacks [Q ; K] on
 // the rows against K: TMEM rows 0-63 then hold Q K^T (-> P) and rows 64-127 K K^T (-> A).  Warps 0-1
-// (rows 0-63) compute the gates, P and the decay factors; warps 2-3 (rows 64-127) build A, solve
-// T = (I + A)^-1 one row per thread, and write the fp16 operands T beta~ and T beta~ gamma; then all
+// (rows 0-63) compute the gates, P and the decay factors; warps 2-3 (rows 64-127) build A, form
+// T = (I + A)^-1 blockwise (16x16 diagonal blocks by substitution through warp shuffles, the rest as
+// a handful of warp-level MMAs), and write the fp16 operands T beta~ and T beta~ gamma; then all
 // 128 threads (one head-dimension row each) store U^T and W^T.  Warp 4 issues TMA and MMAs.
-// 128 TMEM columns and ~50 KB of shared memory per CTA keep four CTAs on an SM, so that the long
-// dependent instruction stream of the solve overlaps with other chunks' loads and stores.
+// 128 TMEM columns and ~50 KB of shared memory per CTA keep four CTAs on an SM, so that one chunk's
+// dependent phases overlap with other chunks' loads and stores.
 // ==========================================================================================
 constexpr int kPrepThreads = 160;
 constexpr int kPrepMisc = 2048;
@@ -66,7 +69,7 @@ struct PrepMisc {
     uint64_t barLoad, barConv, barM, barXfree, barT, barUW;
     uint32_t tmem_base;
     int abort_flag;
-    float G[64], bt[64], wsum[2];
+    float G[64], bt[64], btg[64], wsum[2];   // cumulative log decay, beta~, beta~ gamma
 };
 static_assert(sizeof(PrepMisc) <= kPrepMisc, "misc page too small");
 
@@ -112,7 +115,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     const uint32_t tmem = ms.tmem_base;
     volatile int *abort_flag = &ms.abort_flag;
     uint8_t *sV = smem + PL::oV, *sQK = smem + PL::oQK;
-    // A^T (fp32, two halves of 32 columns j) and later the two fp16 operands: in the two Q blocks
+    // The fp16 tiles of A and T during the inversion, and afterwards the two fp16 operands: in the two Q blocks
     // once K K^T / Q K^T and the q copy are done with them (d = 128), or in their own region (d = 64).
     uint8_t *xLo = D == 128 ? sQK : smem + PL::oX;
     uint8_t *xHi = D == 128 ? sQK + 16384 : smem + PL::oX + 8192;
@@ -194,6 +197,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             if (warp == 1) G += ms.wsum[0];
             ms.G[i] = G;
             ms.bt[i] = btv;
+            ms.btg[i] = btv * __expf(G);
         }
         // ---- tiles to fp16, in place ----
         bool ok = mbar_wait(&ms.barLoad, 0, abort_flag);
@@ -240,77 +244,169 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 }
                 mbar_arrive(&ms.barT);
             } else {
-                // ---- A (strictly lower) -> A^T in shared memory: At[j][m] = A_mj ----
+                // ---- T = (I + A)^-1 with 16x16 blocks (T_bb = (I + A_bb)^-1 in fp32 registers; below the
+                // diagonal T_10 = -T_11 A_10 T_00, T_32 likewise, then the 32x32 block
+                // T_[23][01] = -T_[23][23] A_[23][01] T_[01][01], all as warp-level fp16 MMAs) ----
+                const int sw = warp - 2;                   // solver warp: block rows 2 sw and 2 sw + 1
+                const int bk = i >> 4, il = i & 15;        // this thread's block row, its row inside it
+                const int g8 = lane >> 2, t4 = lane & 3;   // fragment coordinates
                 const float btv = ms.bt[i];
-                float *AtLo = reinterpret_cast<float *>(xLo), *AtHi = reinterpret_cast<float *>(xHi);
+                const uint32_t aA = smem_u32(xLo), aT = smem_u32(xHi);
+                // A_ij = beta~_i Gamma_ij (k_i.k_j), j < i: blocks left of the diagonal as fp16 rows of
+                // the A tile (xLo), the row of the diagonal block in registers.
+                float ablk[16];
 #pragma unroll
-                for (int j = 0; j < 64; ++j) {
-                    const float ab = j < i ? __expf(G - ms.G[j]) * __uint_as_float(dd[j >> 5][j & 31]) : 0.f;
-                    (j < 32 ? AtLo + j * 64 : AtHi + (j - 32) * 64)[i] = btv * ab;
-                    if (ex.Abar) ex.Abar[(chunk * 64 + i) * 64 + j] = ab;   // A without the beta~ row factor
-                }
-                named_barrier_sync(2, 64);
-                // ---- row i of T = (I + A)^-1 by back substitution, t_j = [j = i] - sum_{m > j} t_m A_mj,
-                // in four blocks of 16 columns from the right.  Real loops keep the code small (a
-                // fully unrolled solve is ~40 KB of instructions executed once: instruction fetch
-                // becomes the bottleneck); the 16 values of the block in flight sit in registers,
-                // finished blocks are parked in this thread's column of the A^T rows they belong to,
-                // which nobody reads any more.
-                auto At_row = [&](int j) { return j < 32 ? AtLo + j * 64 : AtHi + (j - 32) * 64; };
-#pragma unroll 1
-                for (int jb = 3; jb >= 0; --jb) {
-                    float acc[16];
+                for (int jb = 0; jb < 4; ++jb) {
+                    if (jb <= bk) {
+                        float a[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) acc[j] = 0.f;
-#pragma unroll 1
-                    for (int m0 = 16 * (jb + 1); m0 < 64; m0 += 4) {      // finished columns m > block
-                        const float t0 = At_row(m0)[i], t1 = At_row(m0 + 1)[i], t2 = At_row(m0 + 2)[i],
-                                    t3 = At_row(m0 + 3)[i];
+                        for (int jj = 0; jj < 16; ++jj) {
+                            const int j = 16 * jb + jj;
+                            a[jj] = j < i ? btv * __expf(G - ms.G[j]) * __uint_as_float(dd[j >> 5][j & 31]) : 0.f;
+                        }
+                        if (jb < bk) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float4 a = *reinterpret_cast<const float4 *>(At_row(16 * jb + j) + m0);
-                            acc[j] = fmaf(t0, a.x, fmaf(t1, a.y, fmaf(t2, a.z, fmaf(t3, a.w, acc[j]))));
+                            for (int hp = 0; hp < 2; ++hp)
+                                *reinterpret_cast<uint4 *>(xLo + sw128_offset(i, 2 * jb + hp)) = make_uint4(
+                                    pack_half2(a[8 * hp], a[8 * hp + 1]), pack_half2(a[8 * hp + 2], a[8 * hp + 3]),
+                                    pack_half2(a[8 * hp + 4], a[8 * hp + 5]), pack_half2(a[8 * hp + 6], a[8 * hp + 7]));
+                        } else {
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj) ablk[jj] = a[jj];
                         }
                     }
-                    float tb[16];
+                }
+                // Row il of the diagonal block's inverse: t_j = [j = il] - sum_{m > j} t_m A_mj, from the
+                // right; A_mj sits in the registers of the thread that owns row m of the block.
+                float td[16];
+                {
+                    float sacc[16];
 #pragma unroll
-                    for (int j = 15; j >= 0; --j) {                     // inside the block
-                        const float *row = At_row(16 * jb + j) + 16 * jb;
-                        float sacc = acc[j];
+                    for (int j = 0; j < 16; ++j) sacc[j] = 0.f;
+                    const int grp = lane & 16;
 #pragma unroll
-                        for (int m = j + 1; m < 16; ++m) sacc = fmaf(tb[m], row[m], sacc);
-                        tb[j] = (16 * jb + j == i ? 1.f : 0.f) - sacc;
+                    for (int m = 15; m >= 0; --m) {
+                        td[m] = (m == il ? 1.f : 0.f) - sacc[m];
+#pragma unroll
+                        for (int j = 0; j < m; ++j)
+                            sacc[j] = fmaf(td[m], __shfl_sync(0xffffffffu, ablk[j], grp + m), sacc[j]);
                     }
-                    named_barrier_sync(2, 64);      // both solver warps are done with the block's rows
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) At_row(16 * jb + j)[i] = tb[j];
                 }
-                // ---- operands T diag(beta~) and T diag(beta~ gamma), fp16 rows ----
-                float t[64];
 #pragma unroll
-                for (int j = 0; j < 64; ++j) t[j] = At_row(j)[i];
-                if (ex.T) {
-                    float4 *tr = reinterpret_cast<float4 *>(ex.T + (chunk * 64 + i) * 64);
-#pragma unroll
-                    for (int j4 = 0; j4 < 16; ++j4)
-                        tr[j4] = make_float4(t[4 * j4], t[4 * j4 + 1], t[4 * j4 + 2], t[4 * j4 + 3]);
+                for (int hp = 0; hp < 2; ++hp)              // fp16 copy for the products: T tile (xHi)
+                    *reinterpret_cast<uint4 *>(xHi + sw128_offset(i, 2 * bk + hp)) = make_uint4(
+                        pack_half2(td[8 * hp], td[8 * hp + 1]), pack_half2(td[8 * hp + 2], td[8 * hp + 3]),
+                        pack_half2(td[8 * hp + 4], td[8 * hp + 5]), pack_half2(td[8 * hp + 6], td[8 * hp + 7]));
+                __syncwarp();
+                // Address this lane supplies to a 16x16 ldmatrix.x4 whose corner is (row0, 16-byte piece pc0).
+                const int lrow = (lane & 7) + ((lane >> 3) & 1) * 8, lpc = lane >> 4;
+                auto frag_addr = [&](uint32_t base, int row0, int pc0) {
+                    return base + sw128_offset(row0 + lrow, pc0 + lpc);
+                };
+                auto pack_a = [](const float (&lo)[4], const float (&hi)[4], uint32_t (&o)[4]) {
+                    o[0] = pack_half2(lo[0], lo[1]); o[1] = pack_half2(lo[2], lo[3]);
+                    o[2] = pack_half2(hi[0], hi[1]); o[3] = pack_half2(hi[2], hi[3]);
+                };
+                const int b0 = 2 * sw, b1 = b0 + 1, br = 2 + sw;
+                float t10[2][4] = {};                       // this warp's T_{b1,b0} (sign applied below)
+                {
+                    uint32_t fa[4], fb[4], xa[4];
+                    float x[2][4] = {};
+                    ldmatrix_x4(frag_addr(aT, 16 * b1, 2 * b1), fa);            // T_{b1,b1}
+                    ldmatrix_x4_trans(frag_addr(aA, 16 * b1, 2 * b0), fb);      // A_{b1,b0}
+                    mma_m16n8k16(x[0], fa, fb[0], fb[1]);
+                    mma_m16n8k16(x[1], fa, fb[2], fb[3]);
+                    pack_a(x[0], x[1], xa);
+                    ldmatrix_x4_trans(frag_addr(aT, 16 * b0, 2 * b0), fb);      // T_{b0,b0}
+                    mma_m16n8k16(t10[0], xa, fb[0], fb[1]);
+                    mma_m16n8k16(t10[1], xa, fb[2], fb[3]);
                 }
-                named_barrier_sync(2, 64);          // every row is in registers: the region can be reused
 #pragma unroll
-                for (int pc = 0; pc < 8; ++pc) {
+                for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) t10[nt][e] = -t10[nt][e];
+                    *reinterpret_cast<uint32_t *>(xHi + sw128_offset(16 * b1 + g8, 2 * b0 + nt) + 4 * t4) =
+                        pack_half2(t10[nt][0], t10[nt][1]);
+                    *reinterpret_cast<uint32_t *>(xHi + sw128_offset(16 * b1 + g8 + 8, 2 * b0 + nt) + 4 * t4) =
+                        pack_half2(t10[nt][2], t10[nt][3]);
+                }
+                named_barrier_sync(2, 64);                  // both warps' A rows and T blocks are in place
+                float r2[4][4] = {};                        // block row br of T_[23][01]
+                {
+                    uint32_t fa[4], fb[4], fc[4], ya[2][4];
+                    float y[4][4] = {};                     // T_{br,[23]} A_[23][01]
+#pragma unroll
+                    for (int ks = 0; ks < 2; ++ks) {
+                        if (ks <= sw) {                     // T_23 = 0
+                            ldmatrix_x4(frag_addr(aT, 16 * br, 2 * (2 + ks)), fa);
+                            ldmatrix_x4_trans(frag_addr(aA, 16 * (2 + ks), 0), fb);
+                            ldmatrix_x4_trans(frag_addr(aA, 16 * (2 + ks), 2), fc);
+                            mma_m16n8k16(y[0], fa, fb[0], fb[1]);
+                            mma_m16n8k16(y[1], fa, fb[2], fb[3]);
+                            mma_m16n8k16(y[2], fa, fc[0], fc[1]);
+                            mma_m16n8k16(y[3], fa, fc[2], fc[3]);
+                        }
+                    }
+                    pack_a(y[0], y[1], ya[0]);
+                    pack_a(y[2], y[3], ya[1]);
+                    ldmatrix_x4_trans(frag_addr(aT, 0, 0), fb);                 // T_00
+                    mma_m16n8k16(r2[0], ya[0], fb[0], fb[1]);
+                    mma_m16n8k16(r2[1], ya[0], fb[2], fb[3]);
+                    ldmatrix_x4_trans(frag_addr(aT, 16, 0), fb);                // T_10
+                    mma_m16n8k16(r2[0], ya[1], fb[0], fb[1]);
+                    mma_m16n8k16(r2[1], ya[1], fb[2], fb[3]);
+                    ldmatrix_x4_trans(frag_addr(aT, 16, 2), fb);                // T_11 (T_01 = 0)
+                    mma_m16n8k16(r2[2], ya[1], fb[0], fb[1]);
+                    mma_m16n8k16(r2[3], ya[1], fb[2], fb[3]);
+                }
+                named_barrier_sync(2, 64);                  // both tiles have been read: reuse them
+                // ---- operands T diag(beta~) (xLo) and T diag(beta~ gamma) (xHi), fp16 K-major rows ----
+                float *Trow = ex.T ? ex.T + chunk * 4096 : nullptr;
+                auto put2 = [&](int row, int col, float v0, float v1) {
+                    const float2 fb = *reinterpret_cast<const float2 *>(&ms.bt[col]);
+                    const float2 fg = *reinterpret_cast<const float2 *>(&ms.btg[col]);
+                    const uint32_t off = sw128_offset(row, col >> 3) + (col & 7) * 2;
+                    *reinterpret_cast<uint32_t *>(xLo + off) = pack_half2(v0 * fb.x, v1 * fb.y);
+                    *reinterpret_cast<uint32_t *>(xHi + off) = pack_half2(v0 * fg.x, v1 * fg.y);
+                    if (Trow) *reinterpret_cast<float2 *>(Trow + row * 64 + col) = make_float2(v0, v1);
+                };
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    put2(16 * b1 + g8, 16 * b0 + 8 * nt + 2 * t4, t10[nt][0], t10[nt][1]);
+                    put2(16 * b1 + g8 + 8, 16 * b0 + 8 * nt + 2 * t4, t10[nt][2], t10[nt][3]);
+                }
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+                    put2(16 * br + g8, 8 * nt + 2 * t4, -r2[nt][0], -r2[nt][1]);
+                    put2(16 * br + g8 + 8, 8 * nt + 2 * t4, -r2[nt][2], -r2[nt][3]);
+                }
+#pragma unroll
+                for (int hp = 0; hp < 2; ++hp) {            // own row of the diagonal block
                     float xb[8], xg[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        const int j = 8 * pc + e;
-                        xb[e] = t[j] * ms.bt[j];
-                        xg[e] = xb[e] * __expf(ms.G[j]);
+                        xb[e] = td[8 * hp + e] * ms.bt[16 * bk + 8 * hp + e];
+                        xg[e] = td[8 * hp + e] * ms.btg[16 * bk + 8 * hp + e];
                     }
-                    *reinterpret_cast<uint4 *>(xLo + sw128_offset(i, pc)) =
+                    *reinterpret_cast<uint4 *>(xLo + sw128_offset(i, 2 * bk + hp)) =
                         make_uint4(pack_half2(xb[0], xb[1]), pack_half2(xb[2], xb[3]),
                                    pack_half2(xb[4], xb[5]), pack_half2(xb[6], xb[7]));
-                    *reinterpret_cast<uint4 *>(xHi + sw128_offset(i, pc)) =
+                    *reinterpret_cast<uint4 *>(xHi + sw128_offset(i, 2 * bk + hp)) =
                         make_uint4(pack_half2(xg[0], xg[1]), pack_half2(xg[2], xg[3]),
                                    pack_half2(xg[4], xg[5]), pack_half2(xg[6], xg[7]));
+                    if (Trow) {
+                        float4 *tr = reinterpret_cast<float4 *>(Trow + i * 64 + 16 * bk + 8 * hp);
+                        tr[0] = make_float4(td[8 * hp], td[8 * hp + 1], td[8 * hp + 2], td[8 * hp + 3]);
+                        tr[1] = make_float4(td[8 * hp + 4], td[8 * hp + 5], td[8 * hp + 6], td[8 * hp + 7]);
+                    }
+                }
+                for (int pc = 2 * bk + 2; pc < 8; ++pc) {   // right of the diagonal block: zero
+                    *reinterpret_cast<uint4 *>(xLo + sw128_offset(i, pc)) = make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4 *>(xHi + sw128_offset(i, pc)) = make_uint4(0, 0, 0, 0);
+                    if (Trow) {
+                        float4 *tr = reinterpret_cast<float4 *>(Trow + i * 64 + 8 * pc);
+                        tr[0] = tr[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
                 }
                 fence_proxy_async_smem();
                 mbar_arrive(&ms.barT);

@@ -76,7 +76,6 @@ struct GdnTcWs {
 struct GdnTcExport {
     float *W, *U;    // token-major [B,L,H,d]
     float *P;        // [B,H,L/C,64,64]
-    float *Abar;     // A without its beta~ row factor, [B,H,L/C,64,64]
     float *T;        // (I + A)^-1, [B,H,L/C,64,64]
     float *Gcum;     // in-chunk cumulative log decay [B,H,L]
     float *S_c;      // chunk-entry states [B,H,L/C,d,d]

@@ -271,6 +271,36 @@ __device__ __forceinline__ void tmem_wait_st() {
 }
 
 // ------------------------------------------------------------------------------------------
+// Warp-level MMA (m16n8k16, fp16 operands, fp32 accumulate) for products far below one tcgen05
+// tile (16x16 blocks of a triangular inverse).  Fragments of a lane (g = lane / 4, t = lane % 4):
+// A: a0 (g, 2t..2t+1), a1 (g+8, 2t..), a2 (g, 2t+8..), a3 (g+8, 2t+8..); B: b0 (k 2t..2t+1, n g),
+// b1 (k 2t+8.., n g); C: c0,c1 (g, 2t..2t+1), c2,c3 (g+8, 2t..).
+// ------------------------------------------------------------------------------------------
+// Four 8x8 16-bit matrices; lanes 8m..8m+7 give the row addresses of matrix m, register m of a
+// lane receives elements (g, 2t..2t+1) of matrix m ...
+__device__ __forceinline__ void ldmatrix_x4(uint32_t saddr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(saddr)
+                 : "memory");
+}
+// ... or, transposed, elements (2t..2t+1, g): the B fragment of a matrix stored [k][n], n contiguous.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t saddr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(saddr)
+                 : "memory");
+}
+__device__ __forceinline__ void mma_m16n8k16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0,
+                                             uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+        "{%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// ------------------------------------------------------------------------------------------
 // Swizzled operand rows written by threads
 // ------------------------------------------------------------------------------------------
 // Byte offset, inside a sub-tile, of 16-byte piece `piece` (0..7) of row `row`.
