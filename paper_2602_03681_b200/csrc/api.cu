@@ -302,8 +302,10 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     // ---- forward recomputation, keeping what the backward needs ----
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, p->B,
                                    p->L, p->H, st));
-    NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
-    const bool tensor_cores = use_tensor_cores(p);   // softmax branch on tcgen05; GDN stays fp32
+    const bool tensor_cores = use_tensor_cores(p);
+    const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
+    if (!fused_chunks)
+        NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, f.k_smb, nullptr, f.v16, f.k16, p->L,
                                       p->L, f.status, s, st));
@@ -311,7 +313,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
                                    f.status, s32, st));
     if (tensor_cores) {
-        const GdnTcExport ex{f.W, f.U, f.P, f.Tinv, f.Gcum, f.S_c, f.Ut};
+        const GdnTcExport ex{f.W, f.U, nullptr, f.Tinv, f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, ex, f.status, s, st));
         NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex, f.status, s, st));
     } else {
@@ -344,6 +346,16 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     else
         NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
                                    f.dS_c, f.gS, s, st));
+    AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
+                   f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
+                   p->scale_la, f.dGrow, f.kappa, dbeta, dg};
+    if (fused_chunks) {   // all chunk-level products and the assembly in one kernel per chunk
+        NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.W, f.U,
+                                       f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, f.dGrow,
+                                       f.kappa, dbeta, s, st));
+        NATSL_TRY(launch_gdn_finish(a, dk, dv, s, st));
+        return NATSL_OK;
+    }
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, s, st));
@@ -361,9 +373,6 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ms), TM(f.k32), TM(f.X2), kC, di, kC, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Ns), TM(f.k32), TM(f.X3), kC, di, kC, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ns), TM(f.q32), TM(f.X4), kC, di, kC, 1.f, false, s, st));
-    AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
-                   f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
-                   p->scale_la, f.dGrow, f.kappa, dbeta, dg};
     NATSL_TRY(launch_gdn_assemble(a, dq, dk, dv, s, st));
 #undef NATSL_TRY
     return NATSL_OK;
