@@ -273,22 +273,28 @@ state_dot_kernel(const float *__restrict__ dS_c, const float *__restrict__ S_c, 
 
 // ==========================================================================================
 // Chunk-parallel part of the backward for d = 64: everything that follows the reverse scan, one
-// CTA per chunk, all operands of the chunk staged once in shared memory (fp32, padded rows) and
-// every product a warp-level tf32 MMA (64x64x64; fp32 range, so no operand can under- or overflow):
+// CTA per chunk, all operands of the chunk staged once in shared memory as fp16 tiles and every
+// product (64x64x64) a set of warp-level MMAs fed by ldmatrix:
 //   dQg = dO S0^T        dW = -dU~ S0^T        dK~ = U~ dS1^T        N = dO U~^T
 //   dKb = T^T dW         dVb = T^T dU~         M = -(dKb W^T + dVb U^T)
 //   Ns = scale_la (N . Gamma) [j <= i]    Mg = M . Gamma [j < i]    Ms = diag(beta~) Mg
 //   dq = scale_la gamma dQg + Ns K + dq_softmax
 //   dk = beta~ gamma dKb + (gamma_C/gamma) dK~ + beta~ Mg K + Ms^T K + Ns^T Q      (linear tokens)
 //   dv = beta~ dVb                                                                  (linear tokens)
-// and the per-token sums the gate gradients need (dG, kappa, dbeta).  Each of the 8 warps owns a
-// 16 x 32 block of every 64 x 64 result; dq, dk, dv accumulate in registers across the products.
+// and the per-token sums the gate gradients need (dG, kappa, dbeta).
+// Range.  The forward quantities (U~, S0, T, W, U, q, k) are O(1) like every fp16 operand of the
+// forward kernels; the three gradient tiles are not (their size follows the incoming gradient), so
+// each of dO, dU~, dS1 is scaled by a power of two that brings its largest element of the chunk to
+// (0.5, 1].  Every result is linear in exactly one of the three, and the factor is taken out again
+// where the result is folded into dq, dk, dv and the sums.
+// Each of the 8 warps owns a 16 x 32 block of every 64 x 64 result; dq, dk, dv accumulate in
+// registers across the products.
 // ==========================================================================================
 constexpr int kCkThreads = 256;
-constexpr int kLd = 68;                        // row stride of a staged 64x64 tile, floats
-constexpr int kTileFloats = 64 * kLd;
-constexpr int kCkSlots = 13;
-constexpr int kCkSmem = kCkSlots * kTileFloats * 4 + 5 * 64 * 4;
+constexpr int kLdH = 72;                       // row stride of a staged 64x64 fp16 tile, elements
+constexpr int kTileH = 64 * kLdH;
+constexpr int kCkSlots = 12;
+constexpr int kCkSmem = kCkSlots * kTileH * 2 + 5 * 64 * 4 + 24 * 4;
 
 struct ChunkBwdArgs {
     const __nv_bfloat16 *q, *k, *v;
@@ -300,68 +306,45 @@ struct ChunkBwdArgs {
     int L, H;
 };
 
-__device__ __forceinline__ uint32_t to_tf32(float x) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
-}
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
-        "{%8, %9}, {%0, %1, %2, %3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void cp_async16(void *dst, const void *src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-
-// acc (16 x 32 block at (row0, n0) of a 64 x 64 result) += A B over k = 0..63.
+// acc (16 x 32 block at (row0, n0) of a 64 x 64 result) += A B over k = 0..63, fp16 tiles.
 // AT: A is stored [k][m] (else [m][k]);  BNK: B is stored [n][k] (else [k][n]).
-// Fragment coordinates of a lane: g = lane / 4, t = lane % 4.
 template <bool AT, bool BNK>
-__device__ __forceinline__ void mma64(const float *__restrict__ A, const float *__restrict__ B, int row0,
-                                      int n0, int g, int t, float (&acc)[4][4]) {
+__device__ __forceinline__ void mma64(const __half *A, const __half *B, int row0, int n0, int lane,
+                                      float (&acc)[4][4]) {
+    const int l7 = lane & 7, m1 = (lane >> 3) & 1, m2 = lane >> 4;
+    const uint32_t sa = smem_u32(A), sb = smem_u32(B);
 #pragma unroll
-    for (int k0 = 0; k0 < 64; k0 += 8) {
-        uint32_t a[4];
-        if (!AT) {
-            a[0] = to_tf32(A[(row0 + g) * kLd + k0 + t]);
-            a[1] = to_tf32(A[(row0 + g + 8) * kLd + k0 + t]);
-            a[2] = to_tf32(A[(row0 + g) * kLd + k0 + t + 4]);
-            a[3] = to_tf32(A[(row0 + g + 8) * kLd + k0 + t + 4]);
-        } else {
-            a[0] = to_tf32(A[(k0 + t) * kLd + row0 + g]);
-            a[1] = to_tf32(A[(k0 + t) * kLd + row0 + g + 8]);
-            a[2] = to_tf32(A[(k0 + t + 4) * kLd + row0 + g]);
-            a[3] = to_tf32(A[(k0 + t + 4) * kLd + row0 + g + 8]);
-        }
+    for (int k0 = 0; k0 < 64; k0 += 16) {
+        uint32_t a[4], b[4];
+        if (!AT) ldmatrix_x4(sa + 2 * ((row0 + l7 + 8 * m1) * kLdH + k0 + 8 * m2), a);
+        else ldmatrix_x4_trans(sa + 2 * ((k0 + l7 + 8 * m2) * kLdH + row0 + 8 * m1), a);
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
-            const int n = n0 + 8 * nt + g;
-            const float b0 = BNK ? B[n * kLd + k0 + t] : B[(k0 + t) * kLd + n];
-            const float b1 = BNK ? B[n * kLd + k0 + t + 4] : B[(k0 + t + 4) * kLd + n];
-            mma_tf32(acc[nt], a, to_tf32(b0), to_tf32(b1));
+        for (int np = 0; np < 2; ++np) {       // two 8-column tiles per load
+            const int nb = n0 + 16 * np;
+            if (BNK) ldmatrix_x4(sb + 2 * ((nb + l7 + 8 * m2) * kLdH + k0 + 8 * m1), b);
+            else ldmatrix_x4_trans(sb + 2 * ((k0 + l7 + 8 * m1) * kLdH + nb + 8 * m2), b);
+            mma_m16n8k16(acc[2 * np], a, b[0], b[1]);
+            mma_m16n8k16(acc[2 * np + 1], a, b[2], b[3]);
         }
     }
 }
 
-__device__ __forceinline__ bool sBtLin(const ChunkBwdArgs &p, int b, int c, int i, int h) {
-    return p.route[((size_t)b * p.L + (size_t)c * kC + i) * p.H + h] == 0;
+__device__ __forceinline__ float pow2_scale(float amax) {   // power of two s with s * amax in (0.5, 1]
+    if (!(amax > 0.f) || !isfinite(amax)) return 1.f;
+    int e;
+    frexpf(amax, &e);                                       // amax = m 2^e, m in [0.5, 1)
+    return ldexpf(1.f, -min(max(e, -100), 100));
 }
 
-__global__ void __launch_bounds__(kCkThreads, 1) gdn_bwd_chunk_kernel(ChunkBwdArgs p) {
+__global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdArgs p) {
     constexpr int D = 64;
-    extern __shared__ __align__(16) float sm[];
-    float *sDO = sm, *sDU = sm + kTileFloats, *sUt = sm + 2 * kTileFloats, *sS0 = sm + 3 * kTileFloats,
-          *sDS1 = sm + 4 * kTileFloats, *sT = sm + 5 * kTileFloats, *sW = sm + 6 * kTileFloats,
-          *sU = sm + 7 * kTileFloats, *sK = sm + 8 * kTileFloats, *sQ = sm + 9 * kTileFloats,
-          *sV = sm + 10 * kTileFloats, *sX = sm + 11 * kTileFloats, *sY = sm + 12 * kTileFloats;
-    float *sG = sm + kCkSlots * kTileFloats, *sBt = sG + 64, *rG = sBt + 64, *rK = rG + 64, *rB = rK + 64;
+    extern __shared__ __align__(16) uint8_t smraw[];
+    __half *sm = reinterpret_cast<__half *>(smraw);
+    __half *sDO = sm, *sDU = sm + kTileH, *sUt = sm + 2 * kTileH, *sS0 = sm + 3 * kTileH,
+           *sDS1 = sm + 4 * kTileH, *sT = sm + 5 * kTileH, *sW = sm + 6 * kTileH, *sU = sm + 7 * kTileH,
+           *sK = sm + 8 * kTileH, *sQ = sm + 9 * kTileH, *sX = sm + 10 * kTileH, *sY = sm + 11 * kTileH;
+    float *sG = reinterpret_cast<float *>(sm + kCkSlots * kTileH), *sBt = sG + 64, *rG = sBt + 64,
+          *rK = rG + 64, *rB = rK + 64, *sMax = rB + 64;   // sMax: 3 tiles x 8 warp maxima
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int c = blockIdx.x, bh = blockIdx.y, b = bh / p.H, h = bh % p.H, NC = p.L / kC;
@@ -369,42 +352,85 @@ __global__ void __launch_bounds__(kCkThreads, 1) gdn_bwd_chunk_kernel(ChunkBwdAr
     const size_t tok0 = (((size_t)b * p.L + (size_t)c * kC) * p.H + h) * D;   // element offset of the chunk
     const size_t chunk = (size_t)bh * NC + c;
 
-    // ---- stage the chunk: fp32 tiles asynchronously in the order the products need them ----
-    auto stage = [&](float *dst, const float *src, size_t row_stride) {
+    // ---- stage the chunk.  Thread -> rows r0 + 16 it (it < 4), columns c4..c4+3 of every tile ----
+    const int r0 = tid >> 4, c4 = (tid & 15) * 4;
+    auto ld_tile = [&](float4 (&x)[4], const float *src, size_t row_stride) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it)
+            x[it] = *reinterpret_cast<const float4 *>(src + (size_t)(r0 + 16 * it) * row_stride + c4);
+    };
+    auto st_tile = [&](__half *dst, const float4 (&x)[4], float f) {
+#pragma unroll
+        for (int it = 0; it < 4; ++it)
+            *reinterpret_cast<uint2 *>(dst + (r0 + 16 * it) * kLdH + c4) =
+                make_uint2(pack_half2(f * x[it].x, f * x[it].y), pack_half2(f * x[it].z, f * x[it].w));
+    };
+    auto amax4 = [](const float4 (&x)[4]) {
+        float m = 0.f;
+#pragma unroll
+        for (int it = 0; it < 4; ++it)
+            m = fmaxf(m, fmaxf(fmaxf(fabsf(x[it].x), fabsf(x[it].y)), fmaxf(fabsf(x[it].z), fabsf(x[it].w))));
+        return m;
+    };
+    float scO, scU, scS;
+    {
+        float4 xo[4], xu[4], xs[4];
+        ld_tile(xo, p.dO + tok0, ts);
+        ld_tile(xu, p.dUt + tok0, ts);
+        ld_tile(xs, p.dS_c + chunk * D * D, D);
+        if (tid < 64) {
+            const size_t tk = ((size_t)b * p.L + (size_t)c * kC + tid) * p.H + h;
+            sG[tid] = p.Gcum[(size_t)bh * p.L + c * kC + tid];
+            sBt[tid] = p.route[tk] ? 0.f : p.beta[tk];
+            rG[tid] = 0.f; rK[tid] = 0.f; rB[tid] = 0.f;
+        }
+        const float mo = warp_max(amax4(xo)), mu = warp_max(amax4(xu)), msx = warp_max(amax4(xs));
+        if (lane == 0) { sMax[warp] = mo; sMax[8 + warp] = mu; sMax[16 + warp] = msx; }
+        __syncthreads();
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f;
+#pragma unroll
+        for (int wv = 0; wv < 8; ++wv) {
+            a0 = fmaxf(a0, sMax[wv]); a1 = fmaxf(a1, sMax[8 + wv]); a2 = fmaxf(a2, sMax[16 + wv]);
+        }
+        scO = pow2_scale(a0); scU = pow2_scale(a1); scS = pow2_scale(a2);
+        st_tile(sDO, xo, scO);
+        st_tile(sDU, xu, scU);
+        st_tile(sDS1, xs, scS);
+    }
+    {
+        float4 y0[4], y1[4], y2[4];
+        ld_tile(y0, p.Ut + tok0, ts);
+        ld_tile(y1, p.S_c + chunk * D * D, D);
+        ld_tile(y2, p.Tinv + chunk * 4096, 64);
+        st_tile(sUt, y0, 1.f);
+        st_tile(sS0, y1, 1.f);
+        st_tile(sT, y2, 1.f);
+    }
+    {
+        float4 y1[4], y2[4];
+        ld_tile(y1, p.W + tok0, ts);
+        ld_tile(y2, p.U + tok0, ts);
+        uint2 qk[2][4];
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
-            const int idx = tid + it * kCkThreads, r = idx >> 4, c4 = (idx & 15) * 4;
-            cp_async16(dst + r * kLd + c4, src + (size_t)r * row_stride + c4);
+            const size_t off = tok0 + (size_t)(r0 + 16 * it) * ts + c4;
+            qk[0][it] = *reinterpret_cast<const uint2 *>(p.q + off);
+            qk[1][it] = *reinterpret_cast<const uint2 *>(p.k + off);
         }
-    };
-    stage(sDO, p.dO + tok0, ts);
-    stage(sDU, p.dUt + tok0, ts);
-    stage(sUt, p.Ut + tok0, ts);
-    stage(sS0, p.S_c + chunk * D * D, D);
-    stage(sDS1, p.dS_c + chunk * D * D, D);
-    cp_async_commit();
-    stage(sT, p.Tinv + chunk * 4096, 64);
-    cp_async_commit();
-    stage(sW, p.W + tok0, ts);
-    stage(sU, p.U + tok0, ts);
-    cp_async_commit();
-    if (tid < 64) {
-        const size_t tk = ((size_t)b * p.L + (size_t)c * kC + tid) * p.H + h;
-        sG[tid] = p.Gcum[(size_t)bh * p.L + c * kC + tid];
-        sBt[tid] = p.route[tk] ? 0.f : p.beta[tk];
-        rG[tid] = 0.f; rK[tid] = 0.f; rB[tid] = 0.f;
-    }
+        st_tile(sW, y1, 1.f);
+        st_tile(sU, y2, 1.f);
 #pragma unroll
-    for (int it = 0; it < 4; ++it) {                               // q, k, v: bf16 -> fp32
-        const int idx = tid + it * kCkThreads, r = idx >> 4, c4 = (idx & 15) * 4;
-        const size_t off = tok0 + (size_t)r * ts + c4;
-        store4(sQ + r * kLd + c4, load4(p.q + off));
-        store4(sK + r * kLd + c4, load4(p.k + off));
-        store4(sV + r * kLd + c4, load4(p.v + off));
+        for (int it = 0; it < 4; ++it) {                           // bf16 -> fp16 (exact)
+            auto cv = [](uint32_t w) {
+                return pack_half2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+            };
+            *reinterpret_cast<uint2 *>(sQ + (r0 + 16 * it) * kLdH + c4) = make_uint2(cv(qk[0][it].x), cv(qk[0][it].y));
+            *reinterpret_cast<uint2 *>(sK + (r0 + 16 * it) * kLdH + c4) = make_uint2(cv(qk[1][it].x), cv(qk[1][it].y));
+        }
     }
-    cp_async_wait<2>();
     __syncthreads();
 
+    const float iO = 1.f / scO, iU = 1.f / scU, iS = 1.f / scS;   // powers of two: exact
     const int row0 = 16 * (warp & 3), n0 = 32 * (warp >> 2);
     const int iA = row0 + g, iB = iA + 8;                          // this lane's two rows (tokens)
     const float GA = sG[iA], GB = sG[iB], GC = sG[63];
@@ -419,54 +445,56 @@ __global__ void __launch_bounds__(kCkThreads, 1) gdn_bwd_chunk_kernel(ChunkBwdAr
             for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
     };
     // <row of X, row of acc> over this lane's columns, for its two rows
-    auto rowdot = [&](const float *X, float &sA, float &sB) {
+    auto rowdot = [&](const __half *X, float &sA, float &sB) {
         sA = 0.f; sB = 0.f;
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
-            const float2 xa = *reinterpret_cast<const float2 *>(X + iA * kLd + n0 + 8 * nt + 2 * t);
-            const float2 xb = *reinterpret_cast<const float2 *>(X + iB * kLd + n0 + 8 * nt + 2 * t);
+            const float2 xa = __half22float2(*reinterpret_cast<const __half2 *>(X + iA * kLdH + n0 + 8 * nt + 2 * t));
+            const float2 xb = __half22float2(*reinterpret_cast<const __half2 *>(X + iB * kLdH + n0 + 8 * nt + 2 * t));
             sA = fmaf(xa.x, acc[nt][0], fmaf(xa.y, acc[nt][1], sA));
             sB = fmaf(xb.x, acc[nt][2], fmaf(xb.y, acc[nt][3], sB));
         }
     };
     // acc (scaled per row) -> a staged tile
-    auto put = [&](float *X, float fA, float fB) {
+    auto put = [&](__half *X, float fA, float fB) {
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
-            *reinterpret_cast<float2 *>(X + iA * kLd + n0 + 8 * nt + 2 * t) = make_float2(fA * acc[nt][0], fA * acc[nt][1]);
-            *reinterpret_cast<float2 *>(X + iB * kLd + n0 + 8 * nt + 2 * t) = make_float2(fB * acc[nt][2], fB * acc[nt][3]);
+            *reinterpret_cast<uint32_t *>(X + iA * kLdH + n0 + 8 * nt + 2 * t) = pack_half2(fA * acc[nt][0], fA * acc[nt][1]);
+            *reinterpret_cast<uint32_t *>(X + iB * kLdH + n0 + 8 * nt + 2 * t) = pack_half2(fB * acc[nt][2], fB * acc[nt][3]);
+        }
+    };
+    // dst += (fA | fB) acc
+    auto fold = [&](float (&dst)[4][4], float fA, float fB, bool init) {
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            dst[nt][0] = fmaf(fA, acc[nt][0], init ? 0.f : dst[nt][0]);
+            dst[nt][1] = fmaf(fA, acc[nt][1], init ? 0.f : dst[nt][1]);
+            dst[nt][2] = fmaf(fB, acc[nt][2], init ? 0.f : dst[nt][2]);
+            dst[nt][3] = fmaf(fB, acc[nt][3], init ? 0.f : dst[nt][3]);
         }
     };
     float sA, sB;
 
     // ---- dQg = dO S0^T ----
     zero();
-    mma64<false, true>(sDO, sS0, row0, n0, g, t, acc);
+    mma64<false, true>(sDO, sS0, row0, n0, lane, acc);
     rowdot(sQ, sA, sB);
-    dGA = fmaf(p.scale_la * gamA, sA, dGA); dGB = fmaf(p.scale_la * gamB, sB, dGB);
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-        dq[nt][0] = p.scale_la * gamA * acc[nt][0]; dq[nt][1] = p.scale_la * gamA * acc[nt][1];
-        dq[nt][2] = p.scale_la * gamB * acc[nt][2]; dq[nt][3] = p.scale_la * gamB * acc[nt][3];
-    }
+    dGA = fmaf(iO * p.scale_la * gamA, sA, dGA); dGB = fmaf(iO * p.scale_la * gamB, sB, dGB);
+    fold(dq, iO * p.scale_la * gamA, iO * p.scale_la * gamB, true);
     // ---- dW = -dU~ S0^T  -> X ----
     zero();
-    mma64<false, true>(sDU, sS0, row0, n0, g, t, acc);
+    mma64<false, true>(sDU, sS0, row0, n0, lane, acc);
     put(sX, -1.f, -1.f);
     // ---- dK~ = U~ dS1^T ----
     zero();
-    mma64<false, true>(sUt, sDS1, row0, n0, g, t, acc);
+    mma64<false, true>(sUt, sDS1, row0, n0, lane, acc);
     rowdot(sK, sA, sB);
-    kapA = ktA * sA; kapB = ktB * sB;
+    kapA = iS * ktA * sA; kapB = iS * ktB * sB;
     dGA -= kapA; dGB -= kapB;
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-        dk[nt][0] = ktA * acc[nt][0]; dk[nt][1] = ktA * acc[nt][1];
-        dk[nt][2] = ktB * acc[nt][2]; dk[nt][3] = ktB * acc[nt][3];
-    }
+    fold(dk, iS * ktA, iS * ktB, true);
     // ---- N = dO U~^T;  Ns = scale_la (N . Gamma), j <= i  -> Y ----
     zero();
-    mma64<false, true>(sDO, sUt, row0, n0, g, t, acc);
+    mma64<false, true>(sDO, sUt, row0, n0, lane, acc);
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
@@ -475,39 +503,40 @@ __global__ void __launch_bounds__(kCkThreads, 1) gdn_bwd_chunk_kernel(ChunkBwdAr
             acc[nt][e] = j <= i ? p.scale_la * __expf((e < 2 ? GA : GB) - sG[j]) * acc[nt][e] : 0.f;
         }
     put(sY, 1.f, 1.f);
-    cp_async_wait<1>();
-    __syncthreads();                    // X = dW, Y = Ns, T staged; dO, S0, dS1 are free
+    __syncthreads();                    // X = dW, Y = Ns; dO, S0, dS1 are free
 
     // ---- dKb = T^T dW  -> slot of dO ----
     zero();
-    mma64<true, false>(sT, sX, row0, n0, g, t, acc);
+    mma64<true, false>(sT, sX, row0, n0, lane, acc);
     rowdot(sK, sA, sB);
-    dGA = fmaf(btA * gamA, sA, dGA); dGB = fmaf(btB * gamB, sB, dGB);
-    dbA = fmaf(gamA, sA, dbA); dbB = fmaf(gamB, sB, dbB);
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-        dk[nt][0] = fmaf(btA * gamA, acc[nt][0], dk[nt][0]); dk[nt][1] = fmaf(btA * gamA, acc[nt][1], dk[nt][1]);
-        dk[nt][2] = fmaf(btB * gamB, acc[nt][2], dk[nt][2]); dk[nt][3] = fmaf(btB * gamB, acc[nt][3], dk[nt][3]);
-    }
+    dGA = fmaf(iU * btA * gamA, sA, dGA); dGB = fmaf(iU * btB * gamB, sB, dGB);
+    dbA = fmaf(iU * gamA, sA, dbA); dbB = fmaf(iU * gamB, sB, dbB);
+    fold(dk, iU * btA * gamA, iU * btB * gamB, false);
     put(sDO, 1.f, 1.f);
     // ---- dVb = T^T dU~  -> slot of S0 ----
     zero();
-    mma64<true, false>(sT, sDU, row0, n0, g, t, acc);
-    rowdot(sV, sA, sB);
-    dbA += sA; dbB += sB;
+    mma64<true, false>(sT, sDU, row0, n0, lane, acc);
+    {   // <v, dVb>: v straight from global memory
+        sA = 0.f; sB = 0.f;
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-        dv[nt][0] = btA * acc[nt][0]; dv[nt][1] = btA * acc[nt][1];
-        dv[nt][2] = btB * acc[nt][2]; dv[nt][3] = btB * acc[nt][3];
+        for (int nt = 0; nt < 4; ++nt) {
+            const float2 xa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(
+                p.v + tok0 + (size_t)iA * ts + n0 + 8 * nt + 2 * t));
+            const float2 xb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(
+                p.v + tok0 + (size_t)iB * ts + n0 + 8 * nt + 2 * t));
+            sA = fmaf(xa.x, acc[nt][0], fmaf(xa.y, acc[nt][1], sA));
+            sB = fmaf(xb.x, acc[nt][2], fmaf(xb.y, acc[nt][3], sB));
+        }
     }
+    dbA = fmaf(iU, sA, dbA); dbB = fmaf(iU, sB, dbB);
+    fold(dv, iU * btA, iU * btB, true);
     put(sS0, 1.f, 1.f);
-    cp_async_wait<0>();
-    __syncthreads();                    // dKb, dVb, W, U staged; T, X, dU~ are free
+    __syncthreads();                    // dKb, dVb in place; T, X, dU~ are free
 
     // ---- M = -(dKb W^T + dVb U^T);  Mg = M . Gamma, j < i -> X;  Ms = diag(beta~) Mg -> slot of T ----
     zero();
-    mma64<false, true>(sDO, sW, row0, n0, g, t, acc);
-    mma64<false, true>(sS0, sU, row0, n0, g, t, acc);
+    mma64<false, true>(sDO, sW, row0, n0, lane, acc);
+    mma64<false, true>(sS0, sU, row0, n0, lane, acc);
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
@@ -521,42 +550,29 @@ __global__ void __launch_bounds__(kCkThreads, 1) gdn_bwd_chunk_kernel(ChunkBwdAr
 
     // ---- beta~ Mg K ----
     zero();
-    mma64<false, false>(sX, sK, row0, n0, g, t, acc);
+    mma64<false, false>(sX, sK, row0, n0, lane, acc);
     rowdot(sK, sA, sB);
-    dGA = fmaf(btA, sA, dGA); dGB = fmaf(btB, sB, dGB);
-    dbA += sA; dbB += sB;
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-        dk[nt][0] = fmaf(btA, acc[nt][0], dk[nt][0]); dk[nt][1] = fmaf(btA, acc[nt][1], dk[nt][1]);
-        dk[nt][2] = fmaf(btB, acc[nt][2], dk[nt][2]); dk[nt][3] = fmaf(btB, acc[nt][3], dk[nt][3]);
-    }
+    dGA = fmaf(iU * btA, sA, dGA); dGB = fmaf(iU * btB, sB, dGB);
+    dbA = fmaf(iU, sA, dbA); dbB = fmaf(iU, sB, dbB);
+    fold(dk, iU * btA, iU * btB, false);
     // ---- Ms^T K ----
     zero();
-    mma64<true, false>(sT, sK, row0, n0, g, t, acc);
+    mma64<true, false>(sT, sK, row0, n0, lane, acc);
     rowdot(sK, sA, sB);
-    dGA -= sA; dGB -= sB;
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) dk[nt][e] += acc[nt][e];
+    dGA = fmaf(-iU, sA, dGA); dGB = fmaf(-iU, sB, dGB);
+    fold(dk, iU, iU, false);
     // ---- Ns K ----
     zero();
-    mma64<false, false>(sY, sK, row0, n0, g, t, acc);
+    mma64<false, false>(sY, sK, row0, n0, lane, acc);
     rowdot(sQ, sA, sB);
-    dGA += sA; dGB += sB;
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) dq[nt][e] += acc[nt][e];
+    dGA = fmaf(iO, sA, dGA); dGB = fmaf(iO, sB, dGB);
+    fold(dq, iO, iO, false);
     // ---- Ns^T Q ----
     zero();
-    mma64<true, false>(sY, sQ, row0, n0, g, t, acc);
+    mma64<true, false>(sY, sQ, row0, n0, lane, acc);
     rowdot(sK, sA, sB);
-    dGA -= sA; dGB -= sB;
-#pragma unroll
-    for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) dk[nt][e] += acc[nt][e];
+    dGA = fmaf(-iO, sA, dGA); dGB = fmaf(-iO, sB, dGB);
+    fold(dk, iO, iO, false);
 
     // ---- per-token sums: over the 4 lanes of a row, then over the two column halves ----
     auto quad = [](float x) {
@@ -570,7 +586,8 @@ __global__ void __launch_bounds__(kCkThreads, 1) gdn_bwd_chunk_kernel(ChunkBwdAr
         atomicAdd(rB + iA, dbA); atomicAdd(rB + iB, dbB);
     }
     // ---- dq, dk, dv ----
-    const bool linA = sBtLin(p, b, c, iA, h), linB = sBtLin(p, b, c, iB, h);
+    const bool linA = p.route[((size_t)b * p.L + (size_t)c * kC + iA) * p.H + h] == 0;
+    const bool linB = p.route[((size_t)b * p.L + (size_t)c * kC + iB) * p.H + h] == 0;
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
         const size_t oA = tok0 + (size_t)iA * ts + n0 + 8 * nt + 2 * t, oB = tok0 + (size_t)iB * ts + n0 + 8 * nt + 2 * t;
