@@ -374,10 +374,15 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
     };
     float scO, scU, scS;
     {
-        float4 xo[4], xu[4], xs[4];
+        // Two batches of tiles are in flight at a time: the loads of the next batch are issued
+        // before the previous one is converted and stored.
+        float4 xo[4], xu[4], xs[4], y0[4], y1[4], y2[4];
         ld_tile(xo, p.dO + tok0, ts);
         ld_tile(xu, p.dUt + tok0, ts);
         ld_tile(xs, p.dS_c + chunk * D * D, D);
+        ld_tile(y0, p.Ut + tok0, ts);
+        ld_tile(y1, p.S_c + chunk * D * D, D);
+        ld_tile(y2, p.Tinv + chunk * 4096, 64);
         if (tid < 64) {
             const size_t tk = ((size_t)b * p.L + (size_t)c * kC + tid) * p.H + h;
             sG[tid] = p.Gcum[(size_t)bh * p.L + c * kC + tid];
@@ -396,20 +401,8 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
         st_tile(sDO, xo, scO);
         st_tile(sDU, xu, scU);
         st_tile(sDS1, xs, scS);
-    }
-    {
-        float4 y0[4], y1[4], y2[4];
-        ld_tile(y0, p.Ut + tok0, ts);
-        ld_tile(y1, p.S_c + chunk * D * D, D);
-        ld_tile(y2, p.Tinv + chunk * 4096, 64);
-        st_tile(sUt, y0, 1.f);
-        st_tile(sS0, y1, 1.f);
-        st_tile(sT, y2, 1.f);
-    }
-    {
-        float4 y1[4], y2[4];
-        ld_tile(y1, p.W + tok0, ts);
-        ld_tile(y2, p.U + tok0, ts);
+        ld_tile(xo, p.W + tok0, ts);                              // next batch into the freed registers
+        ld_tile(xu, p.U + tok0, ts);
         uint2 qk[2][4];
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
@@ -417,8 +410,11 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
             qk[0][it] = *reinterpret_cast<const uint2 *>(p.q + off);
             qk[1][it] = *reinterpret_cast<const uint2 *>(p.k + off);
         }
-        st_tile(sW, y1, 1.f);
-        st_tile(sU, y2, 1.f);
+        st_tile(sUt, y0, 1.f);
+        st_tile(sS0, y1, 1.f);
+        st_tile(sT, y2, 1.f);
+        st_tile(sW, xo, 1.f);
+        st_tile(sU, xu, 1.f);
 #pragma unroll
         for (int it = 0; it < 4; ++it) {                           // bf16 -> fp16 (exact)
             auto cv = [](uint32_t w) {
