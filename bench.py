@@ -73,11 +73,16 @@ def load_peaks():
 
 
 def load_traffic():
-    path = os.path.join(ROOT, "profiles", "traffic.json")
+    """DRAM bytes per launch from the committed profiler summaries (profiles/traffic.txt)."""
+    path = os.path.join(ROOT, "profiles", "traffic.txt")
+    out = {}
     if os.path.exists(path):
         with open(path) as f:
-            return json.load(f)
-    return {}
+            for line in f:
+                parts = line.split("#")[0].split()
+                if len(parts) >= 2 and parts[1].isdigit():
+                    out[parts[0]] = int(parts[1])
+    return out
 
 
 # ------------------------------------------------------------------------------------------
