@@ -200,19 +200,24 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll
                 for (int c = 0; c < kBN; ++c) x[c] = j0 + c < cnt ? x[c] : -INFINITY;
             }
-            float mx = x[0];
+            float mx4[4] = {x[0], x[1], x[2], x[3]};      // four independent chains, not one of 63
 #pragma unroll
-            for (int c = 1; c < kBN; ++c) mx = fmaxf(mx, x[c]);
-            const float m_new = fmaxf(m, mx);
+            for (int c = 4; c < kBN; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], x[c]);
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            // The running maximum only has to bound the exponents, not equal the true maximum: it
+            // is raised (and O rescaled) only when a logit exceeds it by more than 8 (base 2), so
+            // probabilities stay below 2^8 and, for inputs whose logits vary little, the accumulator
+            // is never touched between the tiles.  lse = m + log2(l) holds for any such m.
+            const float m_new = (mx > m + 8.f || m == -INFINITY) ? fmaxf(m, mx) : m;
             const float m_use = m_new == -INFINITY ? 0.f : m_new;
-            const float corr = exp2f(m - m_use);        // m = -inf -> 0
-            float psum = 0.f;
+            const float corr = exp2f(m - m_use);        // m = -inf -> 0; unchanged m -> 1
+            float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < kBN; ++c) {
                 x[c] = exp2f(x[c] - m_use);
-                psum += x[c];
+                ps4[c & 3] += x[c];
             }
-            l = l * corr + psum;
+            l = l * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
             m = m_new;
             if (t > 0) {
                 ok = mbar_wait(&ms.barO, (t - 1) & 1, abort_flag);
@@ -259,7 +264,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             float *row_fn = Xs + kBM * kXS;
             static_assert((kBM * kXS + kBM) * 4 <= SL::oMisc - SL::oK, "epilogue staging does not fit");
             const float inv = l > 0.f ? 1.f / l : 0.f;
-            float ssn = 0.f;
+            float ss4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t ov[32];
@@ -274,11 +279,11 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     o.y = l > 0.f ? __uint_as_float(ov[4 * c4 + 1]) * inv : 0.f;
                     o.z = l > 0.f ? __uint_as_float(ov[4 * c4 + 2]) * inv : 0.f;
                     o.w = l > 0.f ? __uint_as_float(ov[4 * c4 + 3]) * inv : 0.f;
-                    ssn = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ssn))));
+                    ss4[c4 & 3] = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ss4[c4 & 3]))));
                     *reinterpret_cast<float4 *>(Xs + r * kXS + cb * 32 + 4 * c4) = o;
                 }
             }
-            row_fn[r] = rsqrtf(ssn / D + eps);
+            row_fn[r] = rsqrtf(((ss4[0] + ss4[1]) + (ss4[2] + ss4[3])) / D + eps);
             if (lse && i_abs < L)
                 lse[(size_t)bh * L + i_abs] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
             named_barrier_sync(1, kSoftmaxThreads);
