@@ -219,6 +219,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     const bool want_cache = p->k_sm || p->v_sm || p->sm_len;
     if (want_cache && !(p->k_sm && p->v_sm && p->sm_len && p->sm_cap > 0)) return NATSL_ERR_NULL;
     if (want_cache && (!aligned16(p->k_sm) || !aligned16(p->v_sm))) return NATSL_ERR_ALIGN;
+    if ((p->o_la && !aligned16(p->o_la)) || (p->o_nla && !aligned16(p->o_nla))) return NATSL_ERR_ALIGN;
     FwdWs f = carve_fwd(p, ws);
     if (!ws || ws_bytes < f.bytes) return NATSL_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -7,7 +7,12 @@
 // are exact bf16 inputs), online softmax in registers (one thread per query row), probabilities
 // written to shared memory as fp16 and P V as an fp16 MMA (V is gathered as fp16: the bf16
 // inputs convert exactly, and an 11-bit probability keeps the branch output within ~2e-3 of
-// its RMS where an 8-bit one would not).  K/V tiles arrive by TMA into a two-stage ring.
+// its RMS where an 8-bit one would not).  K and V tiles arrive by TMA into two-stage rings.
+// Epilogue: the tile's rows of o_la come in by TMA (into the Q tile and the K ring, free once the
+// last Q K^T has run) while the last tile is still being processed; each thread then normalises
+// its own row of both branches, combines them and writes its row of `out` into a swizzled
+// shared-memory tile that one bulk tensor store sends out, so that no global access of the
+// epilogue is issued per thread and row.
 // Warp roles: warps 0-3 softmax/epilogue (thread r <-> query row r <-> TMEM lane r), warp 4 issues
 // the MMAs, warp 5 issues the TMA loads.
 #include "common.cuh"
@@ -42,7 +47,7 @@ template <int D> struct SmLayout {
 };
 
 struct Misc {                    // lives in the last kMiscBytes of the CTA's shared memory
-    uint64_t barQ, full[kStages], empty[kStages], barS[2], barP, barO;
+    uint64_t barQ, fullK[kStages], emptyK[kStages], fullV[kStages], emptyV[kStages], barS[2], barP, barO, barE;
     uint32_t tmem_base;
     int abort_flag;
     int pos[kBM];                // positions of the retained tokens inside the CTA's own chunks
@@ -53,13 +58,15 @@ template <int D>
 __global__ void __launch_bounds__(kThreadsTc)
 softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                           const __grid_constant__ CUtensorMap map_k,
-                          const __grid_constant__ CUtensorMap map_v, int cap, int capv,
-                          const int32_t *__restrict__ sm_idx,
+                          const __grid_constant__ CUtensorMap map_v,
+                          const __grid_constant__ CUtensorMap map_ola,    // o_la  [B,L,H,D] fp32, box 128 x 32
+                          const __grid_constant__ CUtensorMap map_onla,   // o_nla (same geometry), if has_onla
+                          const __grid_constant__ CUtensorMap map_out,    // out [B,L,H,D] bf16, box 128 x 64, if has_out
+                          int cap, int capv, const int32_t *__restrict__ sm_idx,
                           const int32_t *__restrict__ sm_chunk_prefix,
                           const float *__restrict__ o_la, const float *__restrict__ w,
-                          float scale_sm, float eps, __nv_bfloat16 *__restrict__ out,
-                          float *__restrict__ o_nla, float *__restrict__ lse, int32_t *status, int L,
-                          int H) {
+                          float scale_sm, float eps, int has_out, int has_onla,
+                          float *__restrict__ lse, int32_t *status, int L, int H) {
     using SL = SmLayout<D>;
     constexpr int KB = SL::KB;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -81,11 +88,15 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     }
     if (tid == 0) {
         mbar_init(&ms.barQ, 1);
-        for (int s = 0; s < kStages; ++s) { mbar_init(&ms.full[s], 1); mbar_init(&ms.empty[s], 1); }
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&ms.fullK[s], 1); mbar_init(&ms.emptyK[s], 1);
+            mbar_init(&ms.fullV[s], 1); mbar_init(&ms.emptyV[s], 1);
+        }
         mbar_init(&ms.barS[0], 1);
         mbar_init(&ms.barS[1], 1);
         mbar_init(&ms.barP, kSoftmaxThreads);
         mbar_init(&ms.barO, 1);
+        mbar_init(&ms.barE, 1);
         ms.abort_flag = 0;
         fence_mbar_init();
     }
@@ -103,27 +114,56 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 
     if (warp == 5) {
         // ------------------------------ TMA producer ------------------------------
-        if (lane == 0 && T > 0) {      // nothing is loaded for a tile that sees no retained key
-            prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
-            mbar_arrive_expect_tx(&ms.barQ, SL::kQBytes);
-            for (int kb = 0; kb < KB; ++kb)
-                tma_load_4d(smem + SL::oQ + kb * kBM * 128, &map_q, &ms.barQ, kb * 64, h, p * kBM, b);
-            int t = 0;
-            for (; t < T; ++t) {
-                const int s = t % kStages;
-                if (!mbar_wait(&ms.empty[s], ((t / kStages) & 1) ^ 1, abort_flag)) break;
-                mbar_arrive_expect_tx(&ms.full[s], SL::kKStage + SL::kVStage);
-                for (int kb = 0; kb < KB; ++kb) {
-                    tma_load_2d(smem + SL::oK + s * SL::kKStage + kb * kBN * 128, &map_k, &ms.full[s],
-                                kb * 64, bh * cap + t * kBN);
-                    tma_load_2d(smem + SL::oV + s * SL::kVStage + kb * kBN * 128, &map_v, &ms.full[s],
-                                kb * 64, bh * capv + t * kBN);
+        if (lane == 0) {
+            int nk = 0, nv = 0;                 // K / V tiles requested so far
+            bool ok = true;
+            if (T > 0) {                        // nothing is loaded for a tile that sees no retained key
+                prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
+                mbar_arrive_expect_tx(&ms.barQ, SL::kQBytes);
+                for (int kb = 0; kb < KB; ++kb)
+                    tma_load_4d(smem + SL::oQ + kb * kBM * 128, &map_q, &ms.barQ, kb * 64, h, p * kBM, b);
+                // K and V tiles have their own rings: a K tile is free as soon as its Q K^T has run
+                // (early), a V tile only after its P V; K(u) is therefore requested before V(u-1).
+                for (int u = 0; u <= T && ok; ++u) {
+                    if (u < T) {
+                        const int s = u % kStages;
+                        ok = mbar_wait(&ms.emptyK[s], ((u / kStages) & 1) ^ 1, abort_flag);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&ms.fullK[s], SL::kKStage);
+                        for (int kb = 0; kb < KB; ++kb)
+                            tma_load_2d(smem + SL::oK + s * SL::kKStage + kb * kBN * 128, &map_k,
+                                        &ms.fullK[s], kb * 64, bh * cap + u * kBN);
+                        nk = u + 1;
+                    }
+                    if (u >= 1) {
+                        const int t = u - 1, s = t % kStages;
+                        ok = mbar_wait(&ms.emptyV[s], ((t / kStages) & 1) ^ 1, abort_flag);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&ms.fullV[s], SL::kVStage);
+                        for (int kb = 0; kb < KB; ++kb)
+                            tma_load_2d(smem + SL::oV + s * SL::kVStage + kb * kBN * 128, &map_v,
+                                        &ms.fullV[s], kb * 64, bh * capv + t * kBN);
+                        nv = t + 1;
+                    }
                 }
+                // the Q tile and the K ring are free once the last Q K^T has run
+                if (ok) ok = mbar_wait(&ms.emptyK[(T - 1) % kStages], ((T - 1) / kStages) & 1, abort_flag);
+            }
+            bool e_issued = false;
+            if (ok) {                           // the epilogue's rows of o_la, D/32 boxes of 128 x 32
+                mbar_arrive_expect_tx(&ms.barE, kBM * D * 4);
+                for (int cb = 0; cb < D / 32; ++cb)
+                    tma_load_4d(smem + cb * (kBM * 128), &map_ola, &ms.barE, cb * 32, h, p * kBM, b);
+                e_issued = true;
             }
             // on an aborted run: let the copies already issued land before the CTA retires
-            if (*abort_flag)
-                for (int u = max(0, t - kStages); u < t; ++u)
-                    mbar_wait(&ms.full[u % kStages], (u / kStages) & 1, abort_flag);
+            if (*abort_flag) {
+                for (int u = max(0, nk - kStages); u < nk; ++u)
+                    mbar_wait(&ms.fullK[u % kStages], (u / kStages) & 1, abort_flag);
+                for (int u = max(0, nv - kStages); u < nv; ++u)
+                    mbar_wait(&ms.fullV[u % kStages], (u / kStages) & 1, abort_flag);
+                if (e_issued) mbar_wait(&ms.barE, 0, abort_flag);
+            }
         }
     } else if (warp == 4) {
         // ------------------------------ MMA issuer ------------------------------
@@ -140,21 +180,23 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                         mma_ss(tS[t & 1], desc_kmajor(aQ + kb * kBM * 128 + k16 * 32),
                                desc_kmajor(aK + kb * kBN * 128 + k16 * 32), idesc_qk,
                                (kb | k16) != 0);
+                mma_commit(&ms.emptyK[t % kStages]);
                 mma_commit(&ms.barS[t & 1]);
             };
-            bool ok = mbar_wait(&ms.barQ, 0, abort_flag) && mbar_wait(&ms.full[0], 0, abort_flag);
+            bool ok = mbar_wait(&ms.barQ, 0, abort_flag) && mbar_wait(&ms.fullK[0], 0, abort_flag);
             if (ok) {
                 tc_fence_after_sync();
                 issue_qk(0);
             }
             for (int t = 0; ok && t < T; ++t) {
                 if (t + 1 < T) {
-                    ok = mbar_wait(&ms.full[(t + 1) % kStages], ((t + 1) / kStages) & 1, abort_flag);
+                    ok = mbar_wait(&ms.fullK[(t + 1) % kStages], ((t + 1) / kStages) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
                     issue_qk(t + 1);
                 }
-                ok = mbar_wait(&ms.barP, t & 1, abort_flag);
+                ok = mbar_wait(&ms.barP, t & 1, abort_flag) &&
+                     mbar_wait(&ms.fullV[t % kStages], (t / kStages) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t aV = smem_u32(smem + SL::oV + (t % kStages) * SL::kVStage);
@@ -162,7 +204,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 for (int k16 = 0; k16 < 4; ++k16)
                     mma_ss(tO, desc_kmajor(aP + k16 * 32), desc_mnmajor(aV + k16 * 2048, kBN * 128),
                            idesc_pv, (t | k16) != 0);
-                mma_commit(&ms.empty[t % kStages]);
+                mma_commit(&ms.emptyV[t % kStages]);
                 mma_commit(&ms.barO);
             }
         }
@@ -174,11 +216,12 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         const float sl2 = scale_sm * 1.4426950408889634f;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
-        if (i_abs < L) {     // the epilogue's rows of o_la and w: on their way to L2 while the tiles run
+        float2 wv = make_float2(0.5f, 0.5f);             // (w_nla, w_la) of this row
+        if (i_abs < L) {     // the epilogue's rows of o_la: on their way to L2 while the tiles run
             const size_t tok = ((size_t)b * L + i_abs) * H + h;
 #pragma unroll
             for (int x = 0; x < D * 4 / 128; ++x) prefetch_l2(o_la + tok * D + x * 32);
-            if (w) prefetch_l2(w + tok * 2);
+            if (w) wv = __ldg(reinterpret_cast<const float2 *>(w + tok * 2));
         }
         // The compacted keys are in position order, so row i sees exactly the first `cnt` of them:
         // all n_full earlier ones plus those of the CTA's own chunks at positions <= i.
@@ -254,17 +297,12 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             ok = mbar_wait(&ms.barO, (T - 1) & 1, abort_flag);
             tc_fence_after_sync();
         }
+        if (ok) ok = mbar_wait(&ms.barE, 0, abort_flag);        // the tile's rows of o_la have landed
         if (ok) {
-            // (1) each thread normalises its own row of O (TMEM lane r) into shared memory -- the
-            // K/V ring and the P tile are no longer in use -- and records the row's RMS factor;
-            // (2) the warps then walk the rows with the lanes along the head dimension, so that
-            // o_la is read, and out / o_nla are written, as whole contiguous rows.
-            constexpr int kXS = D + 4;                  // padded row stride (floats)
-            float *Xs = reinterpret_cast<float *>(smem + SL::oK);
-            float *row_fn = Xs + kBM * kXS;
-            static_assert((kBM * kXS + kBM) * 4 <= SL::oMisc - SL::oK, "epilogue staging does not fit");
+            // o_la tile: box cb (columns 32 cb ..) at cb * 16 KB, row r = 128 bytes, 16-byte piece j
+            // at j ^ (r & 7).  out tile (bf16): box kb (columns 64 kb ..) at oV + kb * 16 KB.
             const float inv = l > 0.f ? 1.f / l : 0.f;
-            float ss4[4] = {0.f, 0.f, 0.f, 0.f};
+            float ssn4[4] = {0.f, 0.f, 0.f, 0.f}, ssl4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t ov[32];
@@ -273,60 +311,62 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     tmem_wait_ld();
                 }
 #pragma unroll
-                for (int c4 = 0; c4 < 8; ++c4) {
-                    float4 o;
-                    o.x = l > 0.f ? __uint_as_float(ov[4 * c4]) * inv : 0.f;
-                    o.y = l > 0.f ? __uint_as_float(ov[4 * c4 + 1]) * inv : 0.f;
-                    o.z = l > 0.f ? __uint_as_float(ov[4 * c4 + 2]) * inv : 0.f;
-                    o.w = l > 0.f ? __uint_as_float(ov[4 * c4 + 3]) * inv : 0.f;
-                    ss4[c4 & 3] = fmaf(o.x, o.x, fmaf(o.y, o.y, fmaf(o.z, o.z, fmaf(o.w, o.w, ss4[c4 & 3]))));
-                    *reinterpret_cast<float4 *>(Xs + r * kXS + cb * 32 + 4 * c4) = o;
-                }
-            }
-            row_fn[r] = rsqrtf(((ss4[0] + ss4[1]) + (ss4[2] + ss4[3])) / D + eps);
-            if (lse && i_abs < L)
-                lse[(size_t)bh * L + i_abs] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
-            named_barrier_sync(1, kSoftmaxThreads);
-            constexpr int kLpr = D / 4;                 // lanes per row
-            constexpr int kRpi = 32 / kLpr;             // rows per warp instruction
-            constexpr int kBatch = 8;                   // row steps with their loads in flight together
-            const int sub = lane / kLpr, col = (lane % kLpr) * 4;
-            for (int r0 = warp * 32; r0 < warp * 32 + 32; r0 += kBatch * kRpi) {
-                float4 a[kBatch];
-                float2 wv[kBatch];                      // all loads of the batch are issued before any use
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    const int ia = p * kBM + r0 + u * kRpi + sub;
-                    const size_t tok = ((size_t)b * L + min(ia, L - 1)) * H + h;
-                    a[u] = ia < L ? __ldg(reinterpret_cast<const float4 *>(o_la + tok * D + col))
-                                  : make_float4(0.f, 0.f, 0.f, 0.f);
-                    wv[u] = w ? __ldg(reinterpret_cast<const float2 *>(w + tok * 2)) : make_float2(0.5f, 0.5f);
-                }
-                float ssl_[kBatch];
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u)
-                    ssl_[u] = fmaf(a[u].x, a[u].x, fmaf(a[u].y, a[u].y, fmaf(a[u].z, a[u].z, a[u].w * a[u].w)));
-#pragma unroll
-                for (int o = kLpr / 2; o > 0; o >>= 1)       // the batch's row sums, interleaved
-#pragma unroll
-                    for (int u = 0; u < kBatch; ++u) ssl_[u] += __shfl_xor_sync(0xffffffffu, ssl_[u], o);
-#pragma unroll
-                for (int u = 0; u < kBatch; ++u) {
-                    const int rr = r0 + u * kRpi + sub, ia = p * kBM + rr;
-                    const float ssl = ssl_[u];
-                    if (ia >= L) continue;
-                    const size_t tok = ((size_t)b * L + ia) * H + h;
-                    const float4 on = *reinterpret_cast<const float4 *>(Xs + rr * kXS + col);
-                    if (o_nla) *reinterpret_cast<float4 *>(o_nla + tok * D + col) = on;
-                    if (out) {
-                        const float wn = wv[u].x * row_fn[rr];
-                        const float wl = wv[u].y * rsqrtf(ssl / D + eps);
-                        uint2 pk;
-                        pk.x = pack_bf162(fmaf(wn, on.x, wl * a[u].x), fmaf(wn, on.y, wl * a[u].y));
-                        pk.y = pack_bf162(fmaf(wn, on.z, wl * a[u].z), fmaf(wn, on.w, wl * a[u].w));
-                        *reinterpret_cast<uint2 *>(out + tok * D + col) = pk;
+                for (int j = 0; j < 8; ++j) {
+                    const float4 a = *reinterpret_cast<const float4 *>(smem + cb * (kBM * 128) + sw128_offset(r, j));
+                    ssl4[j & 3] = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, ssl4[j & 3]))));
+                    if (l > 0.f) {
+                        const float o0 = __uint_as_float(ov[4 * j]) * inv, o1 = __uint_as_float(ov[4 * j + 1]) * inv,
+                                    o2 = __uint_as_float(ov[4 * j + 2]) * inv, o3 = __uint_as_float(ov[4 * j + 3]) * inv;
+                        ssn4[j & 3] = fmaf(o0, o0, fmaf(o1, o1, fmaf(o2, o2, fmaf(o3, o3, ssn4[j & 3]))));
                     }
                 }
+            }
+            const float wn = wv.x * rsqrtf(((ssn4[0] + ssn4[1]) + (ssn4[2] + ssn4[3])) / D + eps);
+            const float wl = wv.y * rsqrtf(((ssl4[0] + ssl4[1]) + (ssl4[2] + ssl4[3])) / D + eps);
+#pragma unroll
+            for (int cb = 0; cb < D / 32; ++cb) {
+                uint32_t ov[32];
+                if (T > 0) {
+                    tmem_ld32(tO + lane_base + cb * 32, ov);
+                    tmem_wait_ld();
+                }
+#pragma unroll
+                for (int j2 = 0; j2 < 4; ++j2) {            // two 16-byte fp32 pieces -> one bf16 piece
+                    float o[8], y[8];
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int j = 2 * j2 + hh;
+                        float4 *slot = reinterpret_cast<float4 *>(smem + cb * (kBM * 128) + sw128_offset(r, j));
+                        const float4 a = *slot;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) o[4 * hh + e] = l > 0.f ? __uint_as_float(ov[4 * j + e]) * inv : 0.f;
+                        y[4 * hh] = fmaf(wn, o[4 * hh], wl * a.x);
+                        y[4 * hh + 1] = fmaf(wn, o[4 * hh + 1], wl * a.y);
+                        y[4 * hh + 2] = fmaf(wn, o[4 * hh + 2], wl * a.z);
+                        y[4 * hh + 3] = fmaf(wn, o[4 * hh + 3], wl * a.w);
+                        // the raw branch output takes the place of the o_la piece just consumed
+                        if (has_onla) *slot = make_float4(o[4 * hh], o[4 * hh + 1], o[4 * hh + 2], o[4 * hh + 3]);
+                    }
+                    if (has_out)
+                        *reinterpret_cast<uint4 *>(smem + SL::oV + (cb >> 1) * (kBM * 128) +
+                                                   sw128_offset(r, (cb & 1) * 4 + j2)) =
+                            make_uint4(pack_bf162(y[0], y[1]), pack_bf162(y[2], y[3]), pack_bf162(y[4], y[5]),
+                                       pack_bf162(y[6], y[7]));
+                }
+            }
+            if (lse && i_abs < L)
+                lse[(size_t)bh * L + i_abs] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+            fence_proxy_async_smem();
+            named_barrier_sync(1, kSoftmaxThreads);
+            if (tid == 0) {
+                if (has_out)
+                    for (int kb = 0; kb < KB; ++kb)
+                        tma_store_4d(&map_out, smem + SL::oV + kb * (kBM * 128), kb * 64, h, p * kBM, b);
+                if (has_onla)
+                    for (int cb = 0; cb < D / 32; ++cb)
+                        tma_store_4d(&map_onla, smem + cb * (kBM * 128), cb * 32, h, p * kBM, b);
+                tma_store_commit();
+                tma_store_wait_all();
             }
         }
     }
@@ -400,18 +440,23 @@ static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *
                                    void *out, float *o_nla, float *lse, int32_t *status, Shape s,
                                    cudaStream_t st) {
     using SL = SmLayout<D>;
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mola, monla, mout;
     if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, kBM) ||
         !tch::make_map_2d(&mk, k_sm, (uint64_t)s.B * s.H * cap, D, kBN) ||
-        !tch::make_map_2d(&mv, v16, (uint64_t)s.B * s.H * capv, D, kBN))
+        !tch::make_map_2d(&mv, v16, (uint64_t)s.B * s.H * capv, D, kBN) ||
+        !tch::make_map_blhd_f32(&mola, o_la, s.B, s.L, s.H, D, kBM))
         return cudaErrorInvalidValue;
+    monla = mola;                                          // placeholders when an output is not asked for
+    mout = mq;
+    if (o_nla && !tch::make_map_blhd_f32(&monla, o_nla, s.B, s.L, s.H, D, kBM)) return cudaErrorInvalidValue;
+    if (out && !tch::make_map_blhd(&mout, out, s.B, s.L, s.H, D, kBM)) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(softmax_combine_tc_kernel<D>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal);
     if (e != cudaSuccess) return e;
     dim3 grid((s.L + kBM - 1) / kBM, s.B * s.H);
     softmax_combine_tc_kernel<D><<<grid, kThreadsTc, SL::kTotal, st>>>(
-        mq, mk, mv, cap, capv, sm_idx, pre, o_la, w, scale_sm, eps, (__nv_bfloat16 *)out, o_nla, lse,
-        status, s.L, s.H);
+        mq, mk, mv, mola, monla, mout, cap, capv, sm_idx, pre, o_la, w, scale_sm, eps, out ? 1 : 0,
+        o_nla ? 1 : 0, lse, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }

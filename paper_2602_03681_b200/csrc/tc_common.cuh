@@ -114,6 +114,14 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, const void *s
                  "r"(smem_u32(src)), "r"(x), "r"(y)
                  : "memory");
 }
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *m, const void *src, int c0, int c1,
+                                             int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];" ::"l"(
+            reinterpret_cast<uint64_t>(m)),
+        "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() {
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
@@ -319,13 +327,16 @@ __device__ __forceinline__ uint32_t pack_bf162(float lo, float hi) {
 
 }  // namespace tc
 
-// Host side: encoders of the TMA tensor maps (tc_host.cu).  All maps use 16-bit elements, a
-// box whose inner extent is 64 elements (128 bytes) and the 128-byte swizzle.
+// Host side: encoders of the TMA tensor maps (tc_host.cu).  All maps use a box whose inner extent
+// is 128 bytes (64 16-bit or 32 32-bit elements) and the 128-byte swizzle.
 namespace tch {
 // Rows x cols matrix, row-major, `cols` a multiple of 64; box = box_rows x 64.
 bool make_map_2d(CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 // Tensor [B, L, H, d] (d contiguous); box = box_rows tokens x 64 elements of one (batch, head).
 bool make_map_blhd(CUtensorMap *m, const void *base, int B, int L, int H, int d, uint32_t box_rows);
+// The same tensor with fp32 elements: box = box_rows tokens x 32 elements (128 bytes) of one
+// (batch, head), 128-byte swizzle.
+bool make_map_blhd_f32(CUtensorMap *m, const void *base, int B, int L, int H, int d, uint32_t box_rows);
 }  // namespace tch
 
 }  // namespace natsl

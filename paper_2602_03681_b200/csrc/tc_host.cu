@@ -55,5 +55,19 @@ bool make_map_blhd(CUtensorMap *m, const void *base, int B, int L, int H, int d,
                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_map_blhd_f32(CUtensorMap *m, const void *base, int B, int L, int H, int d,
+                       uint32_t box_rows) {
+    EncodeFn enc = encoder();
+    if (!enc || d % 32 != 0 || box_rows == 0 || box_rows > 256) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)d * 4, (cuuint64_t)H * d * 4,
+                                   (cuuint64_t)L * H * d * 4};
+    const cuuint32_t box[4] = {32, 1, box_rows, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void *>(base), dims, strides, box,
+               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace tch
 }  // namespace natsl
