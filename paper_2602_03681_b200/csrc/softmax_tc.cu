@@ -217,12 +217,17 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         float2 wv = make_float2(0.5f, 0.5f);             // (w_nla, w_la) of this row
-        if (i_abs < L) {     // the epilogue's rows of o_la: on their way to L2 while the tiles run
-            const size_t tok = ((size_t)b * L + i_abs) * H + h;
+        if (w && i_abs < L) wv = __ldg(reinterpret_cast<const float2 *>(w + (((size_t)b * L + i_abs) * H + h) * 2));
+        // The epilogue's rows of o_la are pulled towards L2 once the first tile is under way (at the
+        // very start they would compete with the Q / K / V loads everything else waits for).
+        auto prefetch_o_la = [&]() {
+            if (i_abs < L) {
+                const size_t tok = ((size_t)b * L + i_abs) * H + h;
 #pragma unroll
-            for (int x = 0; x < D * 4 / 128; ++x) prefetch_l2(o_la + tok * D + x * 32);
-            if (w) wv = __ldg(reinterpret_cast<const float2 *>(w + tok * 2));
-        }
+                for (int x = 0; x < D * 4 / 128; ++x) prefetch_l2(o_la + tok * D + x * 32);
+            }
+        };
+        if (T <= 1) prefetch_o_la();
         // The compacted keys are in position order, so row i sees exactly the first `cnt` of them:
         // all n_full earlier ones plus those of the CTA's own chunks at positions <= i.
         int cnt = n_full;
@@ -292,6 +297,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&ms.barP);
+            if (t == 0 && T > 1) prefetch_o_la();
         }
         if (ok && T > 0) {
             ok = mbar_wait(&ms.barO, (T - 1) & 1, abort_flag);
@@ -301,7 +307,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         if (ok) {
             // o_la tile: box cb (columns 32 cb ..) at cb * 16 KB, row r = 128 bytes, 16-byte piece j
             // at j ^ (r & 7).  out tile (bf16): box kb (columns 64 kb ..) at oV + kb * 16 KB.
-            const float inv = l > 0.f ? 1.f / l : 0.f;
+            const float inv = l > 0.f ? 1.f / l : 0.f;       // l = 0 (no visible key): o_nla = 0
             float ssn4[4] = {0.f, 0.f, 0.f, 0.f}, ssl4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
@@ -309,19 +315,22 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 if (T > 0) {
                     tmem_ld32(tO + lane_base + cb * 32, ov);
                     tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) ov[e] = 0u;
                 }
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const float4 a = *reinterpret_cast<const float4 *>(smem + cb * (kBM * 128) + sw128_offset(r, j));
                     ssl4[j & 3] = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, ssl4[j & 3]))));
-                    if (l > 0.f) {
-                        const float o0 = __uint_as_float(ov[4 * j]) * inv, o1 = __uint_as_float(ov[4 * j + 1]) * inv,
-                                    o2 = __uint_as_float(ov[4 * j + 2]) * inv, o3 = __uint_as_float(ov[4 * j + 3]) * inv;
-                        ssn4[j & 3] = fmaf(o0, o0, fmaf(o1, o1, fmaf(o2, o2, fmaf(o3, o3, ssn4[j & 3]))));
-                    }
+                    const float o0 = __uint_as_float(ov[4 * j]), o1 = __uint_as_float(ov[4 * j + 1]),
+                                o2 = __uint_as_float(ov[4 * j + 2]), o3 = __uint_as_float(ov[4 * j + 3]);
+                    ssn4[j & 3] = fmaf(o0, o0, fmaf(o1, o1, fmaf(o2, o2, fmaf(o3, o3, ssn4[j & 3]))));
                 }
             }
-            const float wn = wv.x * rsqrtf(((ssn4[0] + ssn4[1]) + (ssn4[2] + ssn4[3])) / D + eps);
+            // mean square of the normalised row = inv^2 * mean square of the accumulator row
+            const float msn = inv * inv * ((ssn4[0] + ssn4[1]) + (ssn4[2] + ssn4[3])) / D;
+            const float wn = wv.x * rsqrtf(msn + eps) * inv;          // applies to the raw accumulator
             const float wl = wv.y * rsqrtf(((ssl4[0] + ssl4[1]) + (ssl4[2] + ssl4[3])) / D + eps);
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
@@ -329,23 +338,26 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 if (T > 0) {
                     tmem_ld32(tO + lane_base + cb * 32, ov);
                     tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) ov[e] = 0u;
                 }
 #pragma unroll
                 for (int j2 = 0; j2 < 4; ++j2) {            // two 16-byte fp32 pieces -> one bf16 piece
-                    float o[8], y[8];
+                    float y[8];
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
                         const int j = 2 * j2 + hh;
                         float4 *slot = reinterpret_cast<float4 *>(smem + cb * (kBM * 128) + sw128_offset(r, j));
                         const float4 a = *slot;
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) o[4 * hh + e] = l > 0.f ? __uint_as_float(ov[4 * j + e]) * inv : 0.f;
-                        y[4 * hh] = fmaf(wn, o[4 * hh], wl * a.x);
-                        y[4 * hh + 1] = fmaf(wn, o[4 * hh + 1], wl * a.y);
-                        y[4 * hh + 2] = fmaf(wn, o[4 * hh + 2], wl * a.z);
-                        y[4 * hh + 3] = fmaf(wn, o[4 * hh + 3], wl * a.w);
+                        const float o0 = __uint_as_float(ov[4 * j]), o1 = __uint_as_float(ov[4 * j + 1]),
+                                    o2 = __uint_as_float(ov[4 * j + 2]), o3 = __uint_as_float(ov[4 * j + 3]);
+                        y[4 * hh] = fmaf(wn, o0, wl * a.x);
+                        y[4 * hh + 1] = fmaf(wn, o1, wl * a.y);
+                        y[4 * hh + 2] = fmaf(wn, o2, wl * a.z);
+                        y[4 * hh + 3] = fmaf(wn, o3, wl * a.w);
                         // the raw branch output takes the place of the o_la piece just consumed
-                        if (has_onla) *slot = make_float4(o[4 * hh], o[4 * hh + 1], o[4 * hh + 2], o[4 * hh + 3]);
+                        if (has_onla) *slot = make_float4(o0 * inv, o1 * inv, o2 * inv, o3 * inv);
                     }
                     if (has_out)
                         *reinterpret_cast<uint4 *>(smem + SL::oV + (cb >> 1) * (kBM * 128) +
@@ -366,7 +378,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     for (int cb = 0; cb < D / 32; ++cb)
                         tma_store_4d(&map_onla, smem + cb * (kBM * 128), cb * 32, h, p * kBM, b);
                 tma_store_commit();
-                tma_store_wait_all();
+                tma_store_wait_read();                      // shared memory may go once it has been read
             }
         }
     }
