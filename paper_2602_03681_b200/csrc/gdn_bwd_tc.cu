@@ -496,7 +496,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int j = n0 + 8 * nt + 2 * t + (e & 1), i = e < 2 ? iA : iB;
-            acc[nt][e] = j <= i ? p.scale_la * __expf((e < 2 ? GA : GB) - sG[j]) * acc[nt][e] : 0.f;
+            acc[nt][e] *= p.scale_la * __expf(j <= i ? (e < 2 ? GA : GB) - sG[j] : -INFINITY);   // branch-free mask
         }
     put(sY, 1.f, 1.f);
     __syncthreads();                    // X = dW, Y = Ns; dO, S0, dS1 are free
@@ -538,7 +538,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int j = n0 + 8 * nt + 2 * t + (e & 1), i = e < 2 ? iA : iB;
-            acc[nt][e] = j < i ? -__expf((e < 2 ? GA : GB) - sG[j]) * acc[nt][e] : 0.f;
+            acc[nt][e] *= -__expf(j < i ? (e < 2 ? GA : GB) - sG[j] : -INFINITY);
         }
     put(sX, 1.f, 1.f);
     put(sT, btA, btB);

@@ -213,26 +213,26 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         if (ok) {
             tc_fence_after_sync();
             const float G = ms.G[i];
-            uint32_t dd[2][32];
-            tmem_ld32(tmem + lane_base, dd[0]);
-            tmem_ld32(tmem + lane_base + 32, dd[1]);
-            tmem_wait_ld();
-            tc_fence_before_sync();
             if (!solver) {
-                // ---- decay factors for the scan, P (lower triangle) ----
+                // ---- decay factors for the scan, P (lower triangle).  A real loop over 8-column
+                // pieces: straight-line code that runs once per CTA is bound by instruction fetch. ----
                 float *gd = Gd + chunk * 128;
                 gd[i] = __expf(G);
                 gd[64 + i] = __expf(ms.G[63] - G);
                 if (ex.Gcum) ex.Gcum[(size_t)bh * L + tok0 + i] = G;
                 uint4 *prow = reinterpret_cast<uint4 *>(Ph + (chunk * 64 + i) * 64);
-#pragma unroll
+#pragma unroll 1
                 for (int pc = 0; pc < 8; ++pc) {
+                    uint32_t d8[8];
+                    tmem_ld8(tmem + lane_base + 8 * pc, d8);
+                    tmem_wait_ld();
                     float x[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
                         const int j = 8 * pc + e;
-                        x[e] = j <= i ? scale_la * __expf(G - ms.G[j]) * __uint_as_float(dd[j >> 5][j & 31])
-                                      : 0.f;
+                        // the mask goes on the exponent (exp(-inf) = 0): a conditional around the whole
+                        // expression compiles to one divergent branch per element
+                        x[e] = scale_la * __expf(j <= i ? G - ms.G[j] : -INFINITY) * __uint_as_float(d8[e]);
                     }
                     prow[pc] = make_uint4(pack_half2(x[0], x[1]), pack_half2(x[2], x[3]),
                                           pack_half2(x[4], x[5]), pack_half2(x[6], x[7]));
@@ -242,11 +242,17 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                         pf[1] = make_float4(x[4], x[5], x[6], x[7]);
                     }
                 }
+                tc_fence_before_sync();
                 mbar_arrive(&ms.barT);
             } else {
                 // ---- T = (I + A)^-1 with 16x16 blocks (T_bb = (I + A_bb)^-1 in fp32 registers; below the
                 // diagonal T_10 = -T_11 A_10 T_00, T_32 likewise, then the 32x32 block
                 // T_[23][01] = -T_[23][23] A_[23][01] T_[01][01], all as warp-level fp16 MMAs) ----
+                uint32_t dd[2][32];
+                tmem_ld32(tmem + lane_base, dd[0]);
+                tmem_ld32(tmem + lane_base + 32, dd[1]);
+                tmem_wait_ld();
+                tc_fence_before_sync();
                 const int sw = warp - 2;                   // solver warp: block rows 2 sw and 2 sw + 1
                 const int bk = i >> 4, il = i & 15;        // this thread's block row, its row inside it
                 const int g8 = lane >> 2, t4 = lane & 3;   // fragment coordinates
@@ -262,7 +268,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) {
                             const int j = 16 * jb + jj;
-                            a[jj] = j < i ? btv * __expf(G - ms.G[j]) * __uint_as_float(dd[j >> 5][j & 31]) : 0.f;
+                            a[jj] = btv * __expf(j < i ? G - ms.G[j] : -INFINITY) * __uint_as_float(dd[j >> 5][j & 31]);
                         }
                         if (jb < bk) {
 #pragma unroll
