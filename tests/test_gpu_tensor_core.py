@@ -162,3 +162,42 @@ def test_bwd_tensor_core_softmax_branch(name, B, H, L, route):
     check_bwd(wl, got, ref, TOL["bf16"])
     lin = x["route"] == 0
     assert np.all(got["dbeta"][~lin] == 0)
+
+
+@pytest.mark.parametrize("scale", [2.0 ** -6, 2.0 ** 6])
+def test_bwd_tensor_core_is_linear_in_the_incoming_gradient(scale):
+    """Every gradient is linear in dout; the chunk kernel rescales its gradient tiles by a power of
+    two per chunk, which must not show in the result."""
+    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+    x = inputs.make_layer_inputs(wl, B=1, H=2, L=256)
+    x["dout"] = (x["dout"] * scale).astype(np.float32)      # power of two: still exact in bf16
+    got = run_bwd(wl, x)
+    ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                            scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+    check_bwd(wl, got, ref, TOL["bf16"])
+
+
+def test_bwd_tensor_core_many_chunks():
+    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+    x = inputs.make_layer_inputs(wl, B=1, H=2, L=1024)
+    got = run_bwd(wl, x)
+    ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                            scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+    check_bwd(wl, got, ref, TOL["bf16"])
+
+
+@pytest.mark.parametrize("name,L", [("cfg1_bf16_prefill", 704), ("cfg4_bf16_train", 448)])
+def test_fwd_tensor_core_out_only(name, L):
+    """The call as the bench makes it: no optional output requested (the raw branch outputs stay in
+    the workspace), last query tile half filled."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS[name]
+    x = inputs.make_layer_inputs(wl, B=2, H=2, L=L)
+    dt = torch.bfloat16
+    res = binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]),
+                             dev(x["beta"]), dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la,
+                             scale_sm=wl.scale_sm)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(res["ws"]) == 0
+    ref = run_oracle(wl, x)
+    check_stored(res["out"].float().cpu().numpy(), ref["out"], TOL["bf16"], "bf16")
