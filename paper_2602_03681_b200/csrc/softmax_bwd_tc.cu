@@ -183,8 +183,9 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
                 for (int c = 0; c < 32; ++c) {
                     const int jj = t * 64 + 32 * half + c;
                     const bool vis = row_ok && (jj < n_full || (jj < n_end && ms.pos[jj - n_full] <= i_abs));
-                    const float pr = exp2f(fmaf(__uint_as_float(sv[c]), sl2, -lse2));
-                    ds[32 * half + c] = vis ? scale_sm * pr * (__uint_as_float(dv[c]) - Di) : 0.f;
+                    // mask on the exponent (exp2(-inf) = 0), not around the expression: no branch
+                    const float pr = exp2f(vis ? fmaf(__uint_as_float(sv[c]), sl2, -lse2) : -INFINITY);
+                    ds[32 * half + c] = scale_sm * pr * (__uint_as_float(dv[c]) - Di);
                 }
             }
             if (t > 0) {
@@ -391,9 +392,9 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                 for (int c = 0; c < 32; ++c) {
                     const int cc = 32 * half + c;
                     const bool vis = pos_j <= i0 + cc;
-                    const float pr = vis ? exp2f(fmaf(__uint_as_float(sv[c]), sl2, -lse2[cc])) : 0.f;
+                    const float pr = exp2f(vis ? fmaf(__uint_as_float(sv[c]), sl2, -lse2[cc]) : -INFINITY);
                     pv[cc] = pr;
-                    ds[cc] = vis ? scale_sm * pr * (__uint_as_float(dv[c]) - dsum[cc]) : 0.f;
+                    ds[cc] = scale_sm * pr * (__uint_as_float(dv[c]) - dsum[cc]);
                 }
             }
             if (t > 0) {
