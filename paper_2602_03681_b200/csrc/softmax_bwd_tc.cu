@@ -26,7 +26,7 @@ constexpr int kMiscB = 2048;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct MiscB {
-    uint64_t barQ, full[2], empty[2], barS, barP, barAcc;
+    uint64_t barQ, full[3], empty[3], barS, barSfree, barP, barAcc;
     uint32_t tmem_base;
     int abort_flag;
     int pos[kRowsB];
@@ -41,7 +41,8 @@ template <int D> struct QLayout {
     static constexpr int KB = D / 64;
     static constexpr int kQ = KB * 128 * 128;             // 128 queries x D fp16
     static constexpr int kKV = KB * 64 * 128;             // 64 keys x D fp16
-    static constexpr int oQ = 0, oDO = kQ, oK = 2 * kQ, oV = oK + 2 * kKV, oDS = oV + 2 * kKV;
+    static constexpr int kStages = 3;
+    static constexpr int oQ = 0, oDO = kQ, oK = 2 * kQ, oV = oK + kStages * kKV, oDS = oV + kStages * kKV;
     static constexpr int oMisc = oDS + 128 * 128;
     static constexpr int kTotal = oMisc + kMiscB;
     static constexpr int kTmem = D == 64 ? 256 : 512;     // S 64 + dP 64 + dQ D
@@ -75,8 +76,9 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
     }
     if (tid == 0) {
         mbar_init(&ms.barQ, 1);
-        for (int s = 0; s < 2; ++s) { mbar_init(&ms.full[s], 1); mbar_init(&ms.empty[s], 1); }
+        for (int s = 0; s < SL::kStages; ++s) { mbar_init(&ms.full[s], 1); mbar_init(&ms.empty[s], 1); }
         mbar_init(&ms.barS, 1);
+        mbar_init(&ms.barSfree, kRowsB);
         mbar_init(&ms.barP, kRowsB);
         mbar_init(&ms.barAcc, 1);
         ms.abort_flag = 0;
@@ -103,8 +105,8 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
             }
             int t = 0;
             for (; t < T; ++t) {
-                const int s = t & 1;
-                if (!mbar_wait(&ms.empty[s], ((t >> 1) & 1) ^ 1, abort_flag)) break;
+                const int s = t % SL::kStages;
+                if (!mbar_wait(&ms.empty[s], ((t / SL::kStages) & 1) ^ 1, abort_flag)) break;
                 mbar_arrive_expect_tx(&ms.full[s], 2 * SL::kKV);
                 for (int kb = 0; kb < KB; ++kb) {
                     tma_load_2d(smem + SL::oK + s * SL::kKV + kb * 8192, &map_k, &ms.full[s], kb * 64,
@@ -114,7 +116,8 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
                 }
             }
             if (*abort_flag)
-                for (int u = max(0, t - 2); u < t; ++u) mbar_wait(&ms.full[u & 1], (u >> 1) & 1, abort_flag);
+                for (int u = max(0, t - SL::kStages); u < t; ++u)
+                    mbar_wait(&ms.full[u % SL::kStages], (u / SL::kStages) & 1, abort_flag);
         }
     } else if (warp == 4) {
         if (lane == 0 && T > 0) {
@@ -123,8 +126,8 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
             const uint32_t aQ = smem_u32(smem + SL::oQ), aDO = smem_u32(smem + SL::oDO),
                            aDS = smem_u32(smem + SL::oDS);
             auto issue_s = [&](int t) {
-                const uint32_t aK = smem_u32(smem + SL::oK + (t & 1) * SL::kKV);
-                const uint32_t aV = smem_u32(smem + SL::oV + (t & 1) * SL::kKV);
+                const uint32_t aK = smem_u32(smem + SL::oK + (t % SL::kStages) * SL::kKV);
+                const uint32_t aV = smem_u32(smem + SL::oV + (t % SL::kStages) * SL::kKV);
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
 #pragma unroll
@@ -142,22 +145,25 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
                 issue_s(0);
             }
             for (int t = 0; ok && t < T; ++t) {
+                // S and dP of the next tile go into the same TMEM columns as soon as the row threads
+                // have read this tile's out of them (barSfree), i.e. while they still compute dS.
+                if (t + 1 < T) {
+                    ok = mbar_wait(&ms.full[(t + 1) % SL::kStages], ((t + 1) / SL::kStages) & 1, abort_flag) &&
+                         mbar_wait(&ms.barSfree, t & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_s(t + 1);
+                }
                 ok = mbar_wait(&ms.barP, t & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
-                const uint32_t aK = smem_u32(smem + SL::oK + (t & 1) * SL::kKV);
+                const uint32_t aK = smem_u32(smem + SL::oK + (t % SL::kStages) * SL::kKV);
 #pragma unroll
                 for (int k16 = 0; k16 < 4; ++k16)
                     mma_ss(tDQ, desc_kmajor(aDS + k16 * 32), desc_mnmajor(aK + k16 * 2048, 8192), id_dq,
                            (t | k16) != 0);
                 mma_commit(&ms.barAcc);
-                if (t + 1 < T) {
-                    ok = mbar_wait(&ms.full[(t + 1) & 1], ((t + 1) >> 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    issue_s(t + 1);     // its commit also covers dQ(t): K/V stage t is free after it
-                }
-                mma_commit(&ms.empty[t & 1]);
+                mma_commit(&ms.empty[t % SL::kStages]);     // K/V stage t is free after dQ(t)
             }
         }
     } else {
@@ -179,6 +185,10 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
                 tmem_ld32(tS + lane_base + 32 * half, sv);
                 tmem_ld32(tDP + lane_base + 32 * half, dv);
                 tmem_wait_ld();
+                if (half == 1) {                            // both halves are in registers
+                    tc_fence_before_sync();
+                    mbar_arrive(&ms.barSfree);
+                }
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
                     const int jj = t * 64 + 32 * half + c;
