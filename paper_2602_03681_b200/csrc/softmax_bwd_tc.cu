@@ -288,6 +288,7 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
         mbar_init(&ms.barQ, 1);
         for (int s = 0; s < 2; ++s) { mbar_init(&ms.full[s], 1); mbar_init(&ms.empty[s], 1 + kRowsB); }
         mbar_init(&ms.barS, 1);
+        mbar_init(&ms.barSfree, kRowsB);
         mbar_init(&ms.barP, kRowsB);
         mbar_init(&ms.barAcc, 1);
         ms.abort_flag = 0;
@@ -349,6 +350,15 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                 issue_s(0);
             }
             for (int t = 0; ok && t < T; ++t) {
+                // S^T and dP^T of the next query tile go into the same TMEM columns as soon as the row
+                // threads have read this tile's out of them, i.e. while they still compute P^T, dS^T.
+                if (t + 1 < T) {
+                    ok = mbar_wait(&ms.full[(t + 1) & 1], ((t + 1) >> 1) & 1, abort_flag) &&
+                         mbar_wait(&ms.barSfree, t & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_s(t + 1);
+                }
                 ok = mbar_wait(&ms.barP, t & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
@@ -362,12 +372,6 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                            (t | k16) != 0);
                 }
                 mma_commit(&ms.barAcc);
-                if (t + 1 < T) {
-                    ok = mbar_wait(&ms.full[(t + 1) & 1], ((t + 1) >> 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    issue_s(t + 1);
-                }
                 mma_commit(&ms.empty[t & 1]);
             }
         }
@@ -398,6 +402,10 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                 tmem_ld32(tS + lane_base + 32 * half, sv);
                 tmem_ld32(tDP + lane_base + 32 * half, dv);
                 tmem_wait_ld();
+                if (half == 1) {                            // both halves are in registers
+                    tc_fence_before_sync();
+                    mbar_arrive(&ms.barSfree);
+                }
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
                     const int cc = 32 * half + c;
