@@ -61,8 +61,14 @@ enum { NATSL_OP_FWD = 0, NATSL_OP_BWD = 1, NATSL_OP_DECODE = 2, NATSL_OP_COMPACT
 
 /* flags */
 enum {
-    NATSL_FORCE_SIMT = 1u << 0   /* use the fp32 CUDA-core kernels even for bf16 tensors (the
+    NATSL_FORCE_SIMT = 1u << 0,  /* use the fp32 CUDA-core kernels even for bf16 tensors (the
                                     default for bf16 is the tcgen05 tensor-core path) */
+    NATSL_SINGLE_PASS_SCAN = 1u << 1   /* forward, tensor-core path: keep the scan over the chunks of a
+                                    (batch, head) in one CTA even when B*H is small.  By default
+                                    such calls split the chunks into segments that run in
+                                    parallel (a second run per segment yields the segment's
+                                    state transition, a small kernel chains the segments); the
+                                    results agree to rounding */
 };
 
 typedef struct natsl_params {

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libnatsl.so")
 NATSL_F32, NATSL_BF16 = 0, 1
 OP_FWD, OP_BWD, OP_DECODE, OP_COMPACT = 0, 1, 2, 3
 FORCE_SIMT = 1
+SINGLE_PASS_SCAN = 2
 ERR_CACHE_FULL = -7
 
 EXPORTS = ["natsl_workspace_size", "natsl_route_compact", "natsl_hybrid_fwd", "natsl_hybrid_bwd",

@@ -50,11 +50,22 @@ struct FwdWs {
     void *k_sm, *v_sm, *v16;
     float *W, *U, *P, *o_la;    // W, U, P: fp32 CUDA-core path only
     GdnTcWs tc;                 // tensor-core path only
+    float *seg_incr, *seg_trans, *seg_start;   // segmented scan: [B*H, nseg, d, d] each
     size_t bytes;
 };
 
 bool use_tensor_cores(const natsl_params *p) {
     return p->dtype == NATSL_BF16 && !(p->flags & NATSL_FORCE_SIMT);
+}
+
+// Segments of the forward scan (tensor-core path): the largest power of two that keeps the two
+// runs per segment within ~one CTA per SM, divides the chunk count and leaves >= 8 chunks each.
+int scan_segments(const natsl_params *p) {
+    if (!use_tensor_cores(p) || (p->flags & NATSL_SINGLE_PASS_SCAN)) return 1;
+    const int NC = p->L / kC, BH = p->B * p->H;
+    int nseg = 1;
+    while (2 * BH * (nseg * 2) <= 128 && NC % (nseg * 2) == 0 && NC / (nseg * 2) >= 8) nseg *= 2;
+    return nseg;
 }
 
 FwdWs carve_fwd(const natsl_params *p, void *ws) {
@@ -79,9 +90,14 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
         f.tc.Ph = c.take<char>(B * H * NC * kC * kC * 2);
         f.tc.Gd = c.take<float>(B * H * L * 2);
         f.W = f.U = f.P = nullptr;
+        const size_t nseg = scan_segments(p), segf = nseg > 1 ? B * H * nseg * d * d : 0;
+        f.seg_incr = c.take<float>(segf);
+        f.seg_trans = c.take<float>(segf);
+        f.seg_start = c.take<float>(segf);
     } else {
         f.v16 = nullptr;
         f.tc = GdnTcWs{};
+        f.seg_incr = f.seg_trans = f.seg_start = nullptr;
         f.W = c.take<float>(B * L * H * d);
         f.U = c.take<float>(B * L * H * d);
         f.P = c.take<float>(B * H * NC * kC * kC);
@@ -251,8 +267,19 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, GdnTcExport{}, f.status,
                                         s, st));
         NATSL_TRY(mark());
-        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, p->state_out, o_la, GdnTcExport{},
-                                     f.status, s, st));
+        const int nseg = scan_segments(p);
+        if (nseg > 1) {   // few (batch, head) pairs: segments in parallel, chained by their transitions
+            ScanSegments sg{1, nseg, (int)(p->L / kC) / nseg, f.seg_incr, f.seg_trans, f.seg_start};
+            NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, o_la, GdnTcExport{}, sg,
+                                         f.status, s, st));
+            NATSL_TRY(launch_scan_combine(p->state_in, sg, s, st));
+            sg.mode = 2;
+            NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, p->state_out, o_la, GdnTcExport{}, sg,
+                                         f.status, s, st));
+        } else {
+            NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, p->state_out, o_la, GdnTcExport{},
+                                         ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, f.status, s, st));
+        }
     } else {
         NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P,
                                           nullptr, nullptr, s, st));
@@ -316,7 +343,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (tensor_cores) {
         const GdnTcExport ex{f.W, f.U, nullptr, f.Tinv, f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, ex, f.status, s, st));
-        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex, f.status, s, st));
+        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex,
+                                     ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, f.status, s, st));
     } else {
         NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
                                           f.P, f.Abar, f.Gcum, s32, st));

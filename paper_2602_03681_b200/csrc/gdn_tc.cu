@@ -526,7 +526,8 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                    const __grid_constant__ CUtensorMap map_ph, const float *__restrict__ Ut,
                    const float *__restrict__ Gd, float scale_la,
                    const float *__restrict__ state_in, float *__restrict__ state_out,
-                   float *__restrict__ o_la, GdnTcExport ex, int32_t *status, int L, int H) {
+                   float *__restrict__ o_la, GdnTcExport ex, ScanSegments sg, int32_t *status, int L,
+                   int H) {
     using SL = ScanLayout<D>;
     constexpr int KB = SL::KB;
     constexpr int kHalfCols = D / 2;                       // state columns per thread
@@ -534,7 +535,14 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
     ScanMisc &ms = *reinterpret_cast<ScanMisc *>(smem + SL::oMisc);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NC = L / kC;
-    const int bh = blockIdx.x, b = bh / H, h = bh % H;
+    // Which (batch, head), which segment of its chunks, and which of the two segment runs (see
+    // ScanSegments): c below counts the chunks of the segment, c0 + c is the chunk's index.
+    const int var = sg.mode == 1 ? (int)(blockIdx.x & 1) : 0;
+    const int slot = sg.mode == 1 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;    // bh * nseg + seg
+    const int seg = sg.mode == 0 ? 0 : slot % sg.nseg;
+    const int bh = sg.mode == 0 ? slot : slot / sg.nseg, b = bh / H, h = bh % H;
+    const int ncs = sg.mode == 0 ? NC : sg.ncs, c0 = seg * ncs;
+    const bool emit_out = sg.mode != 1, zero_u = sg.mode == 1 && var == 1;
 
     if ((smem_u32(smem) & 1023u) != 0) {
         if (tid == 0) atomicMin(status, (int)NATSL_ERR_CUDA);
@@ -560,22 +568,22 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
     if (warp == 9) {
         if (lane == 0) {
             int c = 0;
-            for (; c < NC; ++c) {
+            for (; c < ncs; ++c) {
                 const int s = c % kScanStages;
                 if (!mbar_wait(&ms.empty[s], ((c / kScanStages) & 1) ^ 1, abort_flag)) break;
                 uint8_t *st = smem + s * SL::kStage;
                 mbar_arrive_expect_tx(&ms.full[s], SL::kTx);
-                tma_load_2d(st + SL::oW, &map_wt, &ms.full[s], 0, (bh * NC + c) * D);
+                tma_load_2d(st + SL::oW, &map_wt, &ms.full[s], 0, (bh * NC + c0 + c) * D);
                 for (int kb = 0; kb < KB; ++kb) {
-                    tma_load_2d(st + SL::oQ + kb * 8192, &map_qh, &ms.full[s], kb * 64, bh * L + c * 64);
-                    tma_load_2d(st + SL::oK + kb * 8192, &map_kh, &ms.full[s], kb * 64, bh * L + c * 64);
+                    tma_load_2d(st + SL::oQ + kb * 8192, &map_qh, &ms.full[s], kb * 64, bh * L + (c0 + c) * 64);
+                    tma_load_2d(st + SL::oK + kb * 8192, &map_kh, &ms.full[s], kb * 64, bh * L + (c0 + c) * 64);
                 }
-                tma_load_2d(st + SL::oP, &map_ph, &ms.full[s], 0, (bh * NC + c) * 64);
+                tma_load_2d(st + SL::oP, &map_ph, &ms.full[s], 0, (bh * NC + c0 + c) * 64);
                 // A decay slot is reused kDecaySlots chunks later, i.e. only after the stages of the
                 // chunks up to c + kDecaySlots - kScanStages have been released, which every row
                 // thread's work on chunk c precedes.
                 bulk_load_1d(smem + SL::oG + (c % kDecaySlots) * SL::kG,
-                             Gd + ((size_t)bh * NC + c) * 128, SL::kG, &ms.full[s]);
+                             Gd + ((size_t)bh * NC + c0 + c) * 128, SL::kG, &ms.full[s]);
             }
             if (*abort_flag)
                 for (int u = max(0, c - kScanStages); u < c; ++u)
@@ -587,7 +595,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             constexpr uint32_t id_qs = make_idesc(kFmtF16, 128, 64, false, false);   // B = Q
             constexpr uint32_t id_su = make_idesc(kFmtF16, 128, D, false, true);     // B = K (MN-major)
             constexpr uint32_t id_pu = make_idesc(kFmtF16, 128, 64, false, false);   // B = P
-            for (int c = 0; c < NC; ++c) {
+            for (int c = 0; c < ncs; ++c) {
                 const int s = c % kScanStages;
                 const uint32_t st = smem_u32(smem + s * SL::kStage);
                 if (!mbar_wait(&ms.full[s], (c / kScanStages) & 1, abort_flag)) break;
@@ -598,20 +606,24 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                     mma_ts(tmem + SL::cWS, tmem + SL::cA + kk * 8,
                            desc_mnmajor(st + SL::oW + kk * 2048, 0), id_ws, kk != 0);
                 mma_commit(&ms.barWS);
+                if (emit_out) {
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk)
-                    mma_ts(tmem + SL::cQS + 64 * (c & 1), tmem + SL::cA + kk * 8,
-                           desc_kmajor(st + SL::oQ + (kk >> 2) * 8192 + (kk & 3) * 32), id_qs, kk != 0);
-                mma_commit(&ms.barQS[c & 1]);
+                    for (int kk = 0; kk < D / 16; ++kk)
+                        mma_ts(tmem + SL::cQS + 64 * (c & 1), tmem + SL::cA + kk * 8,
+                               desc_kmajor(st + SL::oQ + (kk >> 2) * 8192 + (kk & 3) * 32), id_qs, kk != 0);
+                    mma_commit(&ms.barQS[c & 1]);
+                }
                 if (!mbar_wait(&ms.barB, c & 1, abort_flag)) break;
                 tc_fence_after_sync();
                 // D3 first: the commit behind the state update then also covers it, so that the
                 // operands in the WS columns are free once barSU has fired.
+                if (emit_out) {
 #pragma unroll
-                for (int k16 = 0; k16 < 4; ++k16)
-                    mma_ts(tmem + SL::cD3 + 64 * (c & 1), tmem + SL::cWS + (k16 >> 1) * 32 + (k16 & 1) * 8,
-                           desc_kmajor(st + SL::oP + k16 * 32), id_pu, k16 != 0);
-                mma_commit(&ms.barD3[c & 1]);
+                    for (int k16 = 0; k16 < 4; ++k16)
+                        mma_ts(tmem + SL::cD3 + 64 * (c & 1), tmem + SL::cWS + (k16 >> 1) * 32 + (k16 & 1) * 8,
+                               desc_kmajor(st + SL::oP + k16 * 32), id_pu, k16 != 0);
+                    mma_commit(&ms.barD3[c & 1]);
+                }
 #pragma unroll
                 for (int k16 = 0; k16 < 4; ++k16)
                     mma_ts(tmem + SL::cS, tmem + SL::cWS + (k16 >> 1) * 32 + 16 + (k16 & 1) * 8,
@@ -630,16 +642,20 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
         float S[kHalfCols];                               // fp32 state, already decayed to chunk entry
 #pragma unroll
         for (int x = 0; x < kHalfCols; ++x)
-            S[x] = (state_in && active) ? state_in[((size_t)bh * D + col0 + x) * D + r] : 0.f;
+            S[x] = !active ? 0.f
+                   : sg.mode == 1 ? (var == 1 && col0 + x == r ? 1.f : 0.f)
+                   : sg.mode == 2 ? sg.start[((size_t)slot * D + col0 + x) * D + r]
+                   : state_in     ? state_in[((size_t)bh * D + col0 + x) * D + r]
+                                  : 0.f;
         // This thread's 8 pieces (4 tokens each) of row r of U^T of chunk c.
         auto u_src = [&](int c) {
-            return reinterpret_cast<const float4 *>(Ut + ((size_t)bh * NC + c) * D * 64) + (tk0 / 4) * D + r;
+            return reinterpret_cast<const float4 *>(Ut + ((size_t)bh * NC + c0 + c) * D * 64) + (tk0 / 4) * D + r;
         };
         // The U row of the next chunk is only pulled into L2 ahead of time and loaded into registers
         // right before it is used: a global load left in flight across TMEM loads makes their
         // consumers wait for it as well.
         auto prefetch_u = [&](int c) {
-            if (active) {
+            if (active && !zero_u) {
                 const float4 *src = u_src(c);
 #pragma unroll
                 for (int x = 0; x < 8; ++x) prefetch_l2(src + x * D);
@@ -651,7 +667,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             if (!mbar_wait(&ms.barQS[c & 1], (c >> 1) & 1, abort_flag)) return false;
             if (!mbar_wait(&ms.barD3[c & 1], (c >> 1) & 1, abort_flag)) return false;
             tc_fence_after_sync();
-            float *dst = o_la + (((size_t)b * L + (size_t)c * 64 + tk0) * H + h) * D + r;
+            float *dst = o_la + (((size_t)b * L + (size_t)(c0 + c) * 64 + tk0) * H + h) * D + r;
 #pragma unroll
             for (int part = 0; part < 2; ++part) {        // 16 tokens at a time keeps registers low
                 uint32_t x[16], y[16];
@@ -671,7 +687,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
         };
         prefetch_u(0);
         bool ok = true;
-        for (int c = 0; c < NC && ok; ++c) {
+        for (int c = 0; c < ncs && ok; ++c) {
             const int s = c % kScanStages;
             const float *e1 = reinterpret_cast<const float *>(smem + SL::oG + (c % kDecaySlots) * SL::kG);
             const float *e2 = e1 + 64;
@@ -692,7 +708,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 tc_fence_before_sync();
             }
             if (ex.S_c && active) {      // chunk-entry state, [B,H,L/C,dk,dv]
-                float *sc = ex.S_c + (((size_t)bh * NC + c) * D + col0) * D + r;
+                float *sc = ex.S_c + (((size_t)bh * NC + c0 + c) * D + col0) * D + r;
 #pragma unroll
                 for (int x = 0; x < kHalfCols; ++x) sc[(size_t)x * D] = S[x];
             }
@@ -712,7 +728,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             tc_fence_before_sync();
             mbar_arrive(&ms.barA);
             float u[32];                                   // from L2; lands while W S is computed
-            if (active) {
+            if (active && !zero_u) {
                 const float4 *src = u_src(c);
 #pragma unroll
                 for (int x = 0; x < 8; ++x) {
@@ -740,7 +756,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 for (int j = 0; j < 32; ++j) u[j] -= __uint_as_float(ws[j]);
             }
             if (ex.Ut && active) {       // U~, token-major
-                float *ut = ex.Ut + (((size_t)b * L + (size_t)c * 64 + tk0) * H + h) * D + r;
+                float *ut = ex.Ut + (((size_t)b * L + (size_t)(c0 + c) * 64 + tk0) * H + h) * D + r;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) ut[(size_t)j * H * D] = u[j];
             }
@@ -757,12 +773,16 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             tc_fence_before_sync();
             mbar_arrive(&ms.barB);
             // ---- behind the MMAs just released: next U row towards L2, previous chunk's output ----
-            if (c + 1 < NC) prefetch_u(c + 1);
-            if (c > 0) ok = emit(c - 1);
+            if (c + 1 < ncs) prefetch_u(c + 1);
+            if (c > 0 && emit_out) ok = emit(c - 1);
         }
-        if (ok) ok = emit(NC - 1);
-        if (ok && state_out) {
-            ok = mbar_wait(&ms.barSU, (NC - 1) & 1, abort_flag);
+        if (ok && emit_out) ok = emit(ncs - 1);
+        // where the state after the segment's last chunk goes
+        float *final_state = sg.mode == 1 ? (var ? sg.trans : sg.incr) + (size_t)slot * D * D
+                             : state_out && (sg.mode == 0 || seg == sg.nseg - 1) ? state_out + (size_t)bh * D * D
+                                                                                   : nullptr;
+        if (ok && final_state) {
+            ok = mbar_wait(&ms.barSU, (ncs - 1) & 1, abort_flag);
             if (ok) {
                 tc_fence_after_sync();
 #pragma unroll
@@ -773,7 +793,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                     if (active) {
 #pragma unroll
                         for (int x = 0; x < 32; ++x)
-                            state_out[((size_t)bh * D + col0 + cb * 32 + x) * D + r] =
+                            final_state[(size_t)(col0 + cb * 32 + x) * D + r] =
                                 S[cb * 32 + x] + __uint_as_float(ds[x]);
                     }
                 }
@@ -789,7 +809,74 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
     if (tid == 0 && ms.abort_flag) atomicMin(status, (int)NATSL_ERR_TIMEOUT);
 }
 
+// start[0] = state_in (or 0); start[s+1] = M_s start[s] + B_s.  The value columns are independent:
+// one CTA per (batch, head) and 8 of them; thread (ag, v) owns key rows ag, ag + 32, ... of column v.
+// M_s is staged through shared memory in tiles of 32 columns (coalesced 128-byte rows).
+template <int D>
+__global__ void __launch_bounds__(256)
+scan_combine_kernel(const float *__restrict__ state_in, const float *__restrict__ incr,
+                    const float *__restrict__ trans, float *__restrict__ start, int nseg) {
+    constexpr int kV = 8, kRows = D / 32;
+    __shared__ float Ss[D][kV + 1];
+    __shared__ float Ms[D][33];
+    const int bh = blockIdx.y, v0 = blockIdx.x * kV, v = threadIdx.x & (kV - 1), ag = threadIdx.x >> 3;
+    for (int i = 0; i < kRows; ++i) {
+        const int a = ag + 32 * i;
+        Ss[a][v] = state_in ? state_in[((size_t)bh * D + a) * D + v0 + v] : 0.f;
+    }
+    __syncthreads();
+    // The tiles of M are fetched one step ahead into registers, so that the chain over the segments
+    // pays one global-memory latency per segment rather than one per tile.
+    constexpr int kTileRegs = D * 32 / 256;
+    float tile[kTileRegs];
+    auto fetch = [&](int sgi, int b0) {
+        const float *src = trans + ((size_t)bh * nseg + sgi) * D * D + b0;
+#pragma unroll
+        for (int i = 0; i < kTileRegs; ++i) {
+            const int idx = threadIdx.x + 256 * i;
+            tile[i] = src[(size_t)(idx >> 5) * D + (idx & 31)];
+        }
+    };
+    if (nseg > 1) fetch(0, 0);
+    for (int sgi = 0; sgi < nseg; ++sgi) {
+        const size_t base = ((size_t)bh * nseg + sgi) * D * D;
+        for (int i = 0; i < kRows; ++i) start[base + (size_t)(ag + 32 * i) * D + v0 + v] = Ss[ag + 32 * i][v];
+        if (sgi + 1 == nseg) break;
+        float acc[kRows];
+#pragma unroll
+        for (int i = 0; i < kRows; ++i) acc[i] = incr[base + (size_t)(ag + 32 * i) * D + v0 + v];
+        for (int b0 = 0; b0 < D; b0 += 32) {
+#pragma unroll
+            for (int i = 0; i < kTileRegs; ++i) {                         // M[a][b0 .. b0+31]
+                const int idx = threadIdx.x + 256 * i;
+                Ms[idx >> 5][idx & 31] = tile[i];
+            }
+            __syncthreads();
+            if (b0 + 32 < D) fetch(sgi, b0 + 32);
+            else if (sgi + 2 < nseg) fetch(sgi + 1, 0);
+#pragma unroll
+            for (int i = 0; i < kRows; ++i) {
+                const float *mr = Ms[ag + 32 * i];
+#pragma unroll 8
+                for (int bb = 0; bb < 32; ++bb) acc[i] = fmaf(mr[bb], Ss[b0 + bb][v], acc[i]);
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int i = 0; i < kRows; ++i) Ss[ag + 32 * i][v] = acc[i];
+        __syncthreads();
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_scan_combine(const float *state_in, const ScanSegments &sg, Shape s, cudaStream_t st) {
+    dim3 grid(s.d / 8, s.B * s.H);
+    if (s.d == 128) scan_combine_kernel<128><<<grid, 256, 0, st>>>(state_in, sg.incr, sg.trans, sg.start, sg.nseg);
+    else scan_combine_kernel<64><<<grid, 256, 0, st>>>(state_in, sg.incr, sg.trans, sg.start, sg.nseg);
+    count_launch();
+    return cudaGetLastError();
+}
 
 template <int D>
 static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, const float *g,
@@ -819,8 +906,8 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
 
 template <int D>
 static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *state_in,
-                                float *state_out, float *o_la, const GdnTcExport &ex, int32_t *status,
-                                Shape s, cudaStream_t st) {
+                                float *state_out, float *o_la, const GdnTcExport &ex,
+                                const ScanSegments &sg, int32_t *status, Shape s, cudaStream_t st) {
     const int NC = s.L / kC;
     const uint64_t BH = (uint64_t)s.B * s.H;
     CUtensorMap mwt, mqh, mkh, mph;
@@ -833,8 +920,9 @@ static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *
                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          ScanLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
-    gdn_scan_tc_kernel<D><<<s.B * s.H, kScanThreads, ScanLayout<D>::kTotal, st>>>(
-        mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, o_la, ex, status, s.L, s.H);
+    const int ctas = s.B * s.H * (sg.mode == 0 ? 1 : sg.nseg) * (sg.mode == 1 ? 2 : 1);
+    gdn_scan_tc_kernel<D><<<ctas, kScanThreads, ScanLayout<D>::kTotal, st>>>(
+        mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, o_la, ex, sg, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -848,10 +936,10 @@ cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, c
 }
 
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
-                               float *state_out, float *o_la, const GdnTcExport &ex, int32_t *status,
-                               Shape s, cudaStream_t st) {
-    if (s.d == 128) return scan_tc_impl<128>(ws, scale_la, state_in, state_out, o_la, ex, status, s, st);
-    return scan_tc_impl<64>(ws, scale_la, state_in, state_out, o_la, ex, status, s, st);
+                               float *state_out, float *o_la, const GdnTcExport &ex,
+                               const ScanSegments &sg, int32_t *status, Shape s, cudaStream_t st) {
+    if (s.d == 128) return scan_tc_impl<128>(ws, scale_la, state_in, state_out, o_la, ex, sg, status, s, st);
+    return scan_tc_impl<64>(ws, scale_la, state_in, state_out, o_la, ex, sg, status, s, st);
 }
 
 }  // namespace natsl

@@ -85,9 +85,25 @@ cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, c
                                   const float *beta, const uint8_t *route, float scale_la,
                                   const GdnTcWs &ws, const GdnTcExport &ex, int32_t *status, Shape s,
                                   cudaStream_t st);
+// Splitting the scan of one (batch, head) over several CTAs when there are few (batch, head)
+// pairs.  The state recurrence S <- (gamma_C I - K~^T W) S + K~^T U is affine in S with a factor
+// that acts on the key dimension only, so a segment of chunks maps its entry state S0 to
+// M_seg S0 + B_seg, and the same scan kernel yields both parts: B_seg as the exit state of a run
+// from S0 = 0, M_seg as the exit state of a run from S0 = I with U = 0.
+//   mode 0: one CTA per (batch, head) over all chunks (state_in / state_out as given);
+//   mode 1: two CTAs per (batch, head, segment), no outputs: B_seg -> incr, M_seg -> trans;
+//   mode 2: one CTA per (batch, head, segment) from the entry state in `start`, with outputs;
+//           the last segment writes state_out.
+// incr, trans, start: [B*H, nseg, d, d] fp32.  Between modes 1 and 2 launch_scan_combine chains the
+// segments: start[0] = state_in (or 0), start[s+1] = M_s start[s] + B_s.
+struct ScanSegments {
+    int mode, nseg, ncs;       // ncs = chunks per segment
+    float *incr, *trans, *start;
+};
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
-                               float *state_out, float *o_la, const GdnTcExport &ex, int32_t *status,
-                               Shape s, cudaStream_t st);
+                               float *state_out, float *o_la, const GdnTcExport &ex,
+                               const ScanSegments &sg, int32_t *status, Shape s, cudaStream_t st);
+cudaError_t launch_scan_combine(const float *state_in, const ScanSegments &sg, Shape s, cudaStream_t st);
 
 // bwd_simt.cu -- fp32 CUDA-core backward
 // A batched matrix operand: element (r, c) of batch (b, h, chunk) is

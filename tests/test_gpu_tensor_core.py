@@ -201,3 +201,23 @@ def test_fwd_tensor_core_out_only(name, L):
     assert binding.natsl_device_status(res["ws"]) == 0
     ref = run_oracle(wl, x)
     check_stored(res["out"].float().cpu().numpy(), ref["out"], TOL["bf16"], "bf16")
+
+
+@pytest.mark.parametrize("name,H,L", [("cfg1_bf16_prefill", 2, 2048), ("cfg4_bf16_train", 3, 1024)])
+def test_fwd_tensor_core_segmented_scan_with_weak_decay(name, H, L):
+    """With few (batch, head) pairs the scan runs as parallel segments chained by their state
+    transitions.  With almost no decay a segment's entry state still matters at its end, so the
+    transition matrices carry real weight here (with the workloads' decay they are ~0)."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS[name]
+    x = inputs.make_layer_inputs(wl, B=1, H=H, L=L)
+    x["g"] = np.full((1, L, H), -1e-3, np.float32)
+    S0 = (0.2 * np.random.default_rng(11).standard_normal((1, H, wl.d, wl.d))).astype(np.float32)
+    seg = run_fwd(wl, x, state_in=S0)
+    one = run_fwd(wl, x, state_in=S0, flags=binding.SINGLE_PASS_SCAN)
+    ref = run_oracle(wl, x, state_in=S0)
+    check_fwd(wl, seg, ref, TOL["bf16"])
+    check_fwd(wl, one, ref, TOL["bf16"])
+    for n in ("o_la", "state_out"):
+        assert rel_err(seg[n], one[n]) <= TOL["bf16"], n
+    assert not np.array_equal(seg["state_out"], one["state_out"])   # the two paths really differ
