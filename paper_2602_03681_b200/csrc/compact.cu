@@ -8,10 +8,12 @@ namespace natsl {
 
 namespace {
 
-constexpr int kCompactThreads = 256;
-constexpr int kCompactTile = 1024;  // chunks scanned per pass (4 per thread)
+constexpr int kCompactThreads = 1024;
+constexpr int kCompactTile = 1024;  // chunks scanned per pass (one per thread)
 
-// One CTA per (batch, head).  A chunk of 64 tokens is one 64-bit ballot word.
+// One CTA per (batch, head).  A chunk of 64 tokens is one 64-bit ballot word.  32 warps, and the
+// route bytes of two chunks per warp in flight at a time: the kernel is a chain of dependent
+// global-memory round trips, so what counts is how few of them each warp makes.
 __global__ void __launch_bounds__(kCompactThreads)
 route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm_idx,
                      int32_t *__restrict__ sm_chunk_prefix, int32_t *__restrict__ lin_idx,
@@ -24,27 +26,34 @@ route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm
     const int bh = blockIdx.x, b = bh / H, h = bh % H;
     const int NC = L / kC;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kWarps = kCompactThreads / 32;
     const uint8_t *rt = route + (size_t)b * L * H + h;
     int base = 0;
 
     for (int tile0 = 0; tile0 < NC; tile0 += kCompactTile) {
         const int nt = min(kCompactTile, NC - tile0);
-        for (int c = warp; c < nt; c += kCompactThreads / 32) {
-            const size_t l0 = (size_t)(tile0 + c) * kC;
-            const unsigned lo = __ballot_sync(0xffffffffu, rt[(l0 + lane) * H] != 0);
-            const unsigned hi = __ballot_sync(0xffffffffu, rt[(l0 + 32 + lane) * H] != 0);
+        for (int c = warp; c < nt; c += 2 * kWarps) {
+            const int c2 = c + kWarps;
+            const size_t l0 = (size_t)(tile0 + c) * kC, l2 = (size_t)(tile0 + c2) * kC;
+            const bool two = c2 < nt;                      // warp-uniform
+            const uint8_t a0 = rt[(l0 + lane) * H], a1 = rt[(l0 + 32 + lane) * H];
+            const uint8_t b0 = two ? rt[(l2 + lane) * H] : (uint8_t)0, b1 = two ? rt[(l2 + 32 + lane) * H] : (uint8_t)0;
+            const unsigned lo = __ballot_sync(0xffffffffu, a0 != 0), hi = __ballot_sync(0xffffffffu, a1 != 0);
+            const unsigned lo2 = __ballot_sync(0xffffffffu, b0 != 0), hi2 = __ballot_sync(0xffffffffu, b1 != 0);
             if (lane == 0) {
                 bits[c] = (unsigned long long)lo | ((unsigned long long)hi << 32);
                 excl[c] = __popc(lo) + __popc(hi);
+                if (two) {
+                    bits[c2] = (unsigned long long)lo2 | ((unsigned long long)hi2 << 32);
+                    excl[c2] = __popc(lo2) + __popc(hi2);
+                }
             }
         }
         for (int c = nt + threadIdx.x; c < kCompactTile; c += kCompactThreads) excl[c] = 0;
         __syncthreads();
-        // exclusive scan of the per-chunk counts: 4 entries per thread, warp scan, warp totals
+        // exclusive scan of the per-chunk counts: one entry per thread, warp scan, scan of the warp totals
         {
-            const int i0 = threadIdx.x * 4;
-            const int c0 = excl[i0], c1 = excl[i0 + 1], c2 = excl[i0 + 2], c3 = excl[i0 + 3];
-            const int mine = c0 + c1 + c2 + c3;
+            const int mine = excl[threadIdx.x];
             int incl = mine;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -53,17 +62,22 @@ route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm
             }
             if (lane == 31) warp_tot[warp] = incl;
             __syncthreads();
-            int woff = 0;
-            for (int wv = 0; wv < warp; ++wv) woff += warp_tot[wv];
-            const int e = woff + incl - mine;
-            excl[i0] = e;
-            excl[i0 + 1] = e + c0;
-            excl[i0 + 2] = e + c0 + c1;
-            excl[i0 + 3] = e + c0 + c1 + c2;
-            if (threadIdx.x == kCompactThreads - 1) tile_total = woff + incl;
+            if (warp == 0) {
+                const int t = warp_tot[lane];
+                int ti = t;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int y = __shfl_up_sync(0xffffffffu, ti, o);
+                    if (lane >= o) ti += y;
+                }
+                warp_tot[lane] = ti - t;                   // exclusive offsets of the warps
+                if (lane == 31) tile_total = ti;
+            }
+            __syncthreads();
+            excl[threadIdx.x] = warp_tot[warp] + incl - mine;
         }
         __syncthreads();
-        for (int c = warp; c < nt; c += kCompactThreads / 32) {
+        for (int c = warp; c < nt; c += kWarps) {
             const int cc = tile0 + c;
             const unsigned long long wbits = bits[c];
             const unsigned lo = (unsigned)wbits, hi = (unsigned)(wbits >> 32);

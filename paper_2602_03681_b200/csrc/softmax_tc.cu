@@ -410,37 +410,38 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
     if (blockIdx.x == 0 && threadIdx.x == 0 && n_sm > cap) atomicMin(status, (int)NATSL_ERR_CACHE_FULL);
     const int n = min(n_sm, cap);
     const int n_pad = min((n + 127) / 128 * 128, capv);
-    const int row = blockIdx.x * kRows + threadIdx.x / kVecPerRow;
     const int piece = threadIdx.x % kVecPerRow;
-    if (row >= n_pad) return;
-    uint4 *dv16 = reinterpret_cast<uint4 *>(v16 + ((size_t)bh * capv + row) * D) + piece;
-    uint4 *dk16 = k16 ? reinterpret_cast<uint4 *>(k16 + ((size_t)bh * capv + row) * D) + piece : nullptr;
-    if (row >= n) {
-        *dv16 = make_uint4(0u, 0u, 0u, 0u);
-        if (dk16) *dk16 = make_uint4(0u, 0u, 0u, 0u);
-        return;
-    }
-    const int tok = sm_idx[(size_t)bh * L + row];
-    const size_t src = (((size_t)b * L + tok) * H + h) * D;
-    const size_t dst = ((size_t)bh * cap + row) * D;
-    const uint4 kk = reinterpret_cast<const uint4 *>(k + src)[piece];
-    reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
-    if (dk16) {
-        const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
-        uint32_t ko[4];
+    // the grid is sized for a typical retention rate; each CTA strides over the rows there are
+    for (int row = blockIdx.x * kRows + threadIdx.x / kVecPerRow; row < n_pad; row += gridDim.x * kRows) {
+        uint4 *dv16 = reinterpret_cast<uint4 *>(v16 + ((size_t)bh * capv + row) * D) + piece;
+        uint4 *dk16 = k16 ? reinterpret_cast<uint4 *>(k16 + ((size_t)bh * capv + row) * D) + piece : nullptr;
+        if (row >= n) {
+            *dv16 = make_uint4(0u, 0u, 0u, 0u);
+            if (dk16) *dk16 = make_uint4(0u, 0u, 0u, 0u);
+            continue;
+        }
+        const int tok = sm_idx[(size_t)bh * L + row];
+        const size_t src = (((size_t)b * L + tok) * H + h) * D;
+        const size_t dst = ((size_t)bh * cap + row) * D;
+        const uint4 kk = reinterpret_cast<const uint4 *>(k + src)[piece];
+        reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
+        if (dk16) {
+            const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
+            uint32_t ko[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                ko[i] = pack_half2(__uint_as_float(kw[i] << 16), __uint_as_float(kw[i] & 0xffff0000u));
+            *dk16 = make_uint4(ko[0], ko[1], ko[2], ko[3]);
+        }
+        const uint4 vv = reinterpret_cast<const uint4 *>(v + src)[piece];
+        if (v_sm) reinterpret_cast<uint4 *>(v_sm + dst)[piece] = vv;
+        const uint32_t wv[4] = {vv.x, vv.y, vv.z, vv.w};
+        uint32_t o[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            ko[i] = pack_half2(__uint_as_float(kw[i] << 16), __uint_as_float(kw[i] & 0xffff0000u));
-        *dk16 = make_uint4(ko[0], ko[1], ko[2], ko[3]);
+            o[i] = pack_half2(__uint_as_float(wv[i] << 16), __uint_as_float(wv[i] & 0xffff0000u));
+        *dv16 = make_uint4(o[0], o[1], o[2], o[3]);
     }
-    const uint4 vv = reinterpret_cast<const uint4 *>(v + src)[piece];
-    if (v_sm) reinterpret_cast<uint4 *>(v_sm + dst)[piece] = vv;
-    const uint32_t wv[4] = {vv.x, vv.y, vv.z, vv.w};
-    uint32_t o[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-        o[i] = pack_half2(__uint_as_float(wv[i] << 16), __uint_as_float(wv[i] & 0xffff0000u));
-    *dv16 = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 }  // namespace
@@ -492,7 +493,8 @@ static cudaError_t gather_tc_impl(const void *k, const void *v, const int32_t *s
                                   int cap, int capv, int32_t *status, Shape s, cudaStream_t st) {
     constexpr int kRows = 256 / (D * 2 / 16);
     const int max_rows = s.L < capv ? s.L : capv;
-    dim3 grid((max_rows + kRows - 1) / kRows, s.B * s.H);
+    const int blocks = (max_rows + kRows - 1) / kRows;
+    dim3 grid(blocks < 48 ? blocks : 48, s.B * s.H);
     gather_kv_tc_kernel<D><<<grid, 256, 0, st>>>(
         (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, sm_idx, pre, (__nv_bfloat16 *)k_sm,
         (__nv_bfloat16 *)v_sm, (__half *)v16, (__half *)k16, cap, capv, status, s.L, s.H);
