@@ -371,7 +371,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                      f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
     // ---- linear branch: reverse scan, then chunk-parallel products ----
     if (tensor_cores)
-        NATSL_TRY(launch_gdn_rscan_tc(f.dOla16, f.dOlag16, f.tc, f.S_c, f.dUt, f.dS_c, f.gS, f.status, s, st));
+        NATSL_TRY(launch_gdn_rscan_tc(f.dOla16, f.dOlag16, f.tc, f.S_c, f.dUt, f.dS_c,
+                                      fused_chunks ? nullptr : f.gS, f.status, s, st));
     else
         NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
                                    f.dS_c, f.gS, s, st));
@@ -380,9 +381,9 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                    p->scale_la, f.dGrow, f.kappa, dbeta, dg};
     if (fused_chunks) {   // all chunk-level products and the assembly in one kernel per chunk
         NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.W, f.U,
-                                       f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, f.dGrow,
-                                       f.kappa, dbeta, s, st));
-        NATSL_TRY(launch_gdn_finish(a, dk, dv, s, st));
+                                       f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
+                                       s, st));
+        NATSL_TRY(launch_gdn_finish(a, dk, dv, s, st, false));   // scatter of the retained tokens' dk, dv
         return NATSL_OK;
     }
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, s, st));

@@ -833,12 +833,15 @@ static cudaError_t assemble_impl(const AssembleArgs &a, void *dq, void *dk, void
 }
 
 template <typename T, int D>
-static cudaError_t finish_impl(const AssembleArgs &a, void *dk, void *dv, Shape s, cudaStream_t st) {
+static cudaError_t finish_impl(const AssembleArgs &a, void *dk, void *dv, Shape s, cudaStream_t st,
+                               bool with_dg) {
     const int NC = s.L / kC;
     const size_t nch = (size_t)s.B * s.H * NC;
-    dg_kernel<<<(unsigned)((nch + 127) / 128), 128, 0, st>>>(a.dGrow, a.kappa, a.gS, a.Gcum,
-                                                            s.d / kDvs, a.dg, s.B, s.L, s.H);
-    count_launch();
+    if (with_dg) {
+        dg_kernel<<<(unsigned)((nch + 127) / 128), 128, 0, st>>>(a.dGrow, a.kappa, a.gS, a.Gcum,
+                                                                s.d / kDvs, a.dg, s.B, s.L, s.H);
+        count_launch();
+    }
     constexpr int kRows = kThreads / (D / 4);
     dim3 grid((a.cap + kRows - 1) / kRows, s.B * s.H);
     scatter_sm_kernel<T, D><<<grid, kThreads, 0, st>>>(a.dk_sm, a.dv_sm, a.cap, a.sm_idx, a.sm_prefix,
@@ -847,13 +850,14 @@ static cudaError_t finish_impl(const AssembleArgs &a, void *dk, void *dv, Shape 
     return cudaGetLastError();
 }
 
-cudaError_t launch_gdn_finish(const AssembleArgs &a, void *dk, void *dv, Shape s, cudaStream_t st) {
+cudaError_t launch_gdn_finish(const AssembleArgs &a, void *dk, void *dv, Shape s, cudaStream_t st,
+                              bool with_dg) {
     if (s.bf16) {
-        if (s.d == 128) return finish_impl<__nv_bfloat16, 128>(a, dk, dv, s, st);
-        return finish_impl<__nv_bfloat16, 64>(a, dk, dv, s, st);
+        if (s.d == 128) return finish_impl<__nv_bfloat16, 128>(a, dk, dv, s, st, with_dg);
+        return finish_impl<__nv_bfloat16, 64>(a, dk, dv, s, st, with_dg);
     }
-    if (s.d == 128) return finish_impl<float, 128>(a, dk, dv, s, st);
-    return finish_impl<float, 64>(a, dk, dv, s, st);
+    if (s.d == 128) return finish_impl<float, 128>(a, dk, dv, s, st, with_dg);
+    return finish_impl<float, 64>(a, dk, dv, s, st, with_dg);
 }
 
 cudaError_t launch_gdn_assemble(const AssembleArgs &a, void *dq, void *dk, void *dv, Shape s,

@@ -294,7 +294,7 @@ constexpr int kCkThreads = 256;
 constexpr int kLdH = 72;                       // row stride of a staged 64x64 fp16 tile, elements
 constexpr int kTileH = 64 * kLdH;
 constexpr int kCkSlots = 12;
-constexpr int kCkSmem = kCkSlots * kTileH * 2 + 5 * 64 * 4 + 24 * 4;
+constexpr int kCkSmem = kCkSlots * kTileH * 2 + 5 * 64 * 4 + 40 * 4;
 
 struct ChunkBwdArgs {
     const __nv_bfloat16 *q, *k, *v;
@@ -302,7 +302,7 @@ struct ChunkBwdArgs {
     const uint8_t *route;
     float scale_la;
     __nv_bfloat16 *dq, *dk, *dv;
-    float *dGrow, *kappa, *dbeta;
+    float *dg, *dbeta;
     int L, H;
 };
 
@@ -344,7 +344,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
            *sDS1 = sm + 4 * kTileH, *sT = sm + 5 * kTileH, *sW = sm + 6 * kTileH, *sU = sm + 7 * kTileH,
            *sK = sm + 8 * kTileH, *sQ = sm + 9 * kTileH, *sX = sm + 10 * kTileH, *sY = sm + 11 * kTileH;
     float *sG = reinterpret_cast<float *>(sm + kCkSlots * kTileH), *sBt = sG + 64, *rG = sBt + 64,
-          *rK = rG + 64, *rB = rK + 64, *sMax = rB + 64;   // sMax: 3 tiles x 8 warp maxima
+          *rK = rG + 64, *rB = rK + 64, *sMax = rB + 64;   // sMax: 3 tiles x 8 warp maxima, 8 partial <dS1, S0>, 4 scan totals
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int c = blockIdx.x, bh = blockIdx.y, b = bh / p.H, h = bh % p.H, NC = p.L / kC;
@@ -390,7 +390,14 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
             rG[tid] = 0.f; rK[tid] = 0.f; rB[tid] = 0.f;
         }
         const float mo = warp_max(amax4(xo)), mu = warp_max(amax4(xu)), msx = warp_max(amax4(xs));
-        if (lane == 0) { sMax[warp] = mo; sMax[8 + warp] = mu; sMax[16 + warp] = msx; }
+        // <dS1, S0> of the chunk (both tiles are in registers, element for element): the decay of the
+        // entry state contributes gamma_C times it to every dg of the chunk
+        float dot = 0.f;
+#pragma unroll
+        for (int it = 0; it < 4; ++it)
+            dot = fmaf(xs[it].x, y1[it].x, fmaf(xs[it].y, y1[it].y, fmaf(xs[it].z, y1[it].z, fmaf(xs[it].w, y1[it].w, dot))));
+        dot = warp_sum(dot);
+        if (lane == 0) { sMax[warp] = mo; sMax[8 + warp] = mu; sMax[16 + warp] = msx; sMax[24 + warp] = dot; }
         __syncthreads();
         float a0 = 0.f, a1 = 0.f, a2 = 0.f;
 #pragma unroll
@@ -602,9 +609,22 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
     }
     __syncthreads();
     if (tid < 64) {
+        // dg_j = sum_{i >= j} dG_i + sum_i kappa_i + gamma_C <dS1, S0>  (i, j: tokens of the chunk)
+        float suf = rG[tid], kap = rK[tid];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float y = __shfl_down_sync(0xffffffffu, suf, o);
+            if (lane + o < 32) suf += y;
+        }
+        kap = warp_sum(kap);
+        if (lane == 0) { sMax[32 + warp] = suf; sMax[34 + warp] = kap; }
+        named_barrier_sync(1, 64);
+        float gs = 0.f;
+#pragma unroll
+        for (int wv = 0; wv < 8; ++wv) gs += sMax[24 + wv];
+        const float extra = sMax[34] + sMax[35] + __expf(sG[63]) * gs + (warp == 0 ? sMax[33] : 0.f);
         const size_t tk = ((size_t)b * p.L + (size_t)c * kC + tid) * p.H + h;
-        p.dGrow[(size_t)bh * p.L + c * kC + tid] = rG[tid];
-        p.kappa[(size_t)bh * p.L + c * kC + tid] = rK[tid];
+        p.dg[tk] = suf + extra;
         p.dbeta[tk] = p.route[tk] ? 0.f : rB[tid];
     }
 }
@@ -629,8 +649,10 @@ static cudaError_t rscan_tc_impl(const void *dO16, const void *dOg16, const GdnT
         mdo, mdog, mqh, mkh, mwt, mph, ws.Gd, dUt, dS_c, status, s.L, s.H);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    state_dot_kernel<<<(unsigned)(BH * NC), 256, 0, st>>>(dS_c, S_c, gS, D / 32, D * D);
-    count_launch();
+    if (gS) {     // (the fused chunk kernel forms <dS1, S0> itself)
+        state_dot_kernel<<<(unsigned)(BH * NC), 256, 0, st>>>(dS_c, S_c, gS, D / 32, D * D);
+        count_launch();
+    }
     return cudaGetLastError();
 }
 
@@ -646,15 +668,15 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
                                  const float *dUt, const float *Ut, const float *S_c, const float *dS_c,
                                  const float *Tinv, const float *W, const float *U, const float *Gcum,
                                  const float *beta, const uint8_t *route, const float *dq_sm,
-                                 float scale_la, void *dq, void *dk, void *dv, float *dGrow,
-                                 float *kappa, float *dbeta, Shape s, cudaStream_t st) {
+                                 float scale_la, void *dq, void *dk, void *dv, float *dg,
+                                 float *dbeta, Shape s, cudaStream_t st) {
     if (s.d != 64 || !s.bf16) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(gdn_bwd_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kCkSmem);
     if (e != cudaSuccess) return e;
     ChunkBwdArgs a{(const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, dO, dUt, Ut,
                    S_c, dS_c, Tinv, W, U, Gcum, beta, dq_sm, route, scale_la, (__nv_bfloat16 *)dq,
-                   (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, dGrow, kappa, dbeta, s.L, s.H};
+                   (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, dg, dbeta, s.L, s.H};
     dim3 grid(s.L / kC, s.B * s.H);
     gdn_bwd_chunk_kernel<<<grid, kCkThreads, kCkSmem, st>>>(a);
     count_launch();

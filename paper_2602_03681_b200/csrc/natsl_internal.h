@@ -159,16 +159,16 @@ cudaError_t launch_gdn_assemble(const AssembleArgs &a, void *dq, void *dk, void 
                                 cudaStream_t st);
 // The last two of those kernels only (dg from the per-token sums, scatter of the retained tokens'
 // dk, dv), for callers that formed dq, dk, dv of the linear tokens and the sums themselves.
-cudaError_t launch_gdn_finish(const AssembleArgs &a, void *dk, void *dv, Shape s, cudaStream_t st);
+cudaError_t launch_gdn_finish(const AssembleArgs &a, void *dk, void *dv, Shape s, cudaStream_t st,
+                              bool with_dg = true);
 // gdn_bwd_tc.cu: everything of the linear branch's backward that follows the reverse scan, fused
-// per chunk (d = 64, bf16 storage): dq (with dq_sm added), dk, dv of the linear tokens, and the
-// per-token sums dGrow, kappa, dbeta.
+// per chunk (d = 64, bf16 storage): dq (with dq_sm added), dk, dv of the linear tokens, dg, dbeta.
 cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, const float *dO,
                                  const float *dUt, const float *Ut, const float *S_c, const float *dS_c,
                                  const float *Tinv, const float *W, const float *U, const float *Gcum,
                                  const float *beta, const uint8_t *route, const float *dq_sm,
-                                 float scale_la, void *dq, void *dk, void *dv, float *dGrow,
-                                 float *kappa, float *dbeta, Shape s, cudaStream_t st);
+                                 float scale_la, void *dq, void *dk, void *dv, float *dg,
+                                 float *dbeta, Shape s, cudaStream_t st);
 
 // decode.cu
 constexpr int kDecodeParts = 4;   // CTAs that share the retained K/V of one (sequence, head)
