@@ -360,7 +360,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                               f.o_la, p->w, p->scale_sm, p->eps, nullptr, f.o_nla,
                                               f.lse, s32, st));
     // ---- combination and softmax branch ----
-    NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la, f.do_nla, dw, f.Dsm,
+    NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la,
+                                 tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,
                                  tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
                                  tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, s, st));
     if (tensor_cores)

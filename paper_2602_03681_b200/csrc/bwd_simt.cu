@@ -170,7 +170,7 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
         const float dl = fl * (wl * dy[x] - ol[x] * fl * ml);
         const float dn = fn * (wn * dy[x] - on[x] * fn * mn);
         do_la[i] = dl;
-        do_nla[i] = dn;
+        if (do_nla) do_nla[i] = dn;   // (the tensor-core softmax backward reads the fp16 copy only)
         const size_t i16 = ((((size_t)b * H + h) * L + l) * D) + lane + 32 * x;
         if (do16) do16[i16] = __float2half_rn(dn);
         if (dolag16) {
