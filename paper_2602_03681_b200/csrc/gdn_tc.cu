@@ -707,11 +707,6 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 }
                 tc_fence_before_sync();
             }
-            if (ex.S_c && active) {      // chunk-entry state, [B,H,L/C,dk,dv]
-                float *sc = ex.S_c + (((size_t)bh * NC + c0 + c) * D + col0) * D + r;
-#pragma unroll
-                for (int x = 0; x < kHalfCols; ++x) sc[(size_t)x * D] = S[x];
-            }
             // ---- (a) state row -> fp16 operand in TMEM; decay the register copy afterwards ----
             {
                 uint32_t pk[kHalfCols / 2];
@@ -727,6 +722,12 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             }
             tc_fence_before_sync();
             mbar_arrive(&ms.barA);
+            // (exports for the backward go behind the arrivals, off the chain between the chunks)
+            if (ex.S_c && active) {      // chunk-entry state, [B,H,L/C,dk,dv]
+                float *sc = ex.S_c + (((size_t)bh * NC + c0 + c) * D + col0) * D + r;
+#pragma unroll
+                for (int x = 0; x < kHalfCols; ++x) sc[(size_t)x * D] = S[x];
+            }
             float u[32];                                   // from L2; lands while W S is computed
             if (active && !zero_u) {
                 const float4 *src = u_src(c);
@@ -755,11 +756,6 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
 #pragma unroll
                 for (int j = 0; j < 32; ++j) u[j] -= __uint_as_float(ws[j]);
             }
-            if (ex.Ut && active) {       // U~, token-major
-                float *ut = ex.Ut + (((size_t)b * L + (size_t)(c0 + c) * 64 + tk0) * H + h) * D + r;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) ut[(size_t)j * H * D] = u[j];
-            }
             {
                 uint32_t pk[32];     // [0,16): U~ of this thread's 32 tokens, [16,32): U~ gamma_C/gamma
 #pragma unroll
@@ -772,6 +768,11 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             }
             tc_fence_before_sync();
             mbar_arrive(&ms.barB);
+            if (ex.Ut && active) {       // U~, token-major
+                float *ut = ex.Ut + (((size_t)b * L + (size_t)(c0 + c) * 64 + tk0) * H + h) * D + r;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) ut[(size_t)j * H * D] = u[j];
+            }
             // ---- behind the MMAs just released: next U row towards L2, previous chunk's output ----
             if (c + 1 < ncs) prefetch_u(c + 1);
             if (c > 0 && emit_out) ok = emit(c - 1);
