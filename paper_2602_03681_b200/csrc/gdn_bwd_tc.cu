@@ -168,12 +168,8 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
             const int c = NC - 1 - n, s = n % kRsStages;
             const float *e1 = reinterpret_cast<const float *>(smem + SL::oG + (n % kRsDecaySlots) * SL::kG);
             const float *e2 = e1 + 64;
-            // ---- dS1 (exit-state gradient of chunk c): store, and fp16 operand into TMEM ----
-            if (active) {
-                float *dst = dS_c + (((size_t)bh * NC + c) * D + col0) * D + r;
-#pragma unroll
-                for (int x = 0; x < kHalfCols; ++x) dst[(size_t)x * D] = G[x];
-            }
+            // ---- dS1 (exit-state gradient of chunk c): fp16 operand into TMEM, then (behind the
+            // arrival, off the chain) the fp32 copy the later products read ----
             {
                 uint32_t pk[kHalfCols / 2];
 #pragma unroll
@@ -188,6 +184,11 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
             }
             tc_fence_before_sync();
             mbar_arrive(&ms.barA);
+            if (active) {
+                float *dst = dS_c + (((size_t)bh * NC + c) * D + col0) * D + r;
+#pragma unroll
+                for (int x = 0; x < kHalfCols; ++x) dst[(size_t)x * D] = G[x];
+            }
             ok = mbar_wait(&ms.full[s], (n / kRsStages) & 1, abort_flag);   // decay factors of the chunk
             if (!ok) break;
             {
@@ -199,20 +200,15 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
             ok = mbar_wait(&ms.barX, n & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
+            float du[32];
             {
                 uint32_t x1[32], x2[32];
                 tmem_ld32(tmem + SL::cX1 + tk0 + lane_base, x1);
                 tmem_ld32(tmem + SL::cX2 + tk0 + lane_base, x2);
                 tmem_wait_ld();
-                float du[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
                     du[j] = fmaf(e2[tk0 + j], __uint_as_float(x2[j]), __uint_as_float(x1[j]));
-                if (active) {
-                    float *dst = dUt + (((size_t)b * L + (size_t)c * 64 + tk0) * H + h) * D + r;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) dst[(size_t)j * H * D] = du[j];
-                }
                 uint32_t pk[16];
 #pragma unroll
                 for (int x = 0; x < 16; ++x) pk[x] = pack_half2(du[2 * x], du[2 * x + 1]);
@@ -222,6 +218,11 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
             }
             tc_fence_before_sync();
             mbar_arrive(&ms.barB);
+            if (active) {                                   // the fp32 copy, behind the arrival
+                float *dst = dUt + (((size_t)b * L + (size_t)c * 64 + tk0) * H + h) * D + r;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) dst[(size_t)j * H * D] = du[j];
+            }
             // ---- dS0 = gamma_C dS1 + Y ----
             ok = mbar_wait(&ms.barY, n & 1, abort_flag);
             if (!ok) break;
