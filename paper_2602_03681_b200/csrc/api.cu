@@ -341,7 +341,9 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
                                    f.status, s32, st));
     if (tensor_cores) {
-        const GdnTcExport ex{f.W, f.U, nullptr, f.Tinv, f.Gcum, f.S_c, f.Ut};
+        // the fused chunk kernel reads W^T, U^T as the forward keeps them: no fp32 copies for it
+        const GdnTcExport ex{fused_chunks ? nullptr : f.W, fused_chunks ? nullptr : f.U, nullptr, f.Tinv,
+                             f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, ex, f.status, s, st));
         NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex,
                                      ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, f.status, s, st));
@@ -381,7 +383,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                    f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
                    p->scale_la, f.dGrow, f.kappa, dbeta, dg};
     if (fused_chunks) {   // all chunk-level products and the assembly in one kernel per chunk
-        NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.W, f.U,
+        NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
                                        s, st));
         NATSL_TRY(launch_gdn_finish(a, dk, dv, s, st, false));   // scatter of the retained tokens' dk, dv

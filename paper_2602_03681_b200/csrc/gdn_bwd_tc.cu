@@ -299,7 +299,8 @@ constexpr int kCkSmem = kCkSlots * kTileH * 2 + 5 * 64 * 4 + 40 * 4;
 
 struct ChunkBwdArgs {
     const __nv_bfloat16 *q, *k, *v;
-    const float *dO, *dUt, *Ut, *S_c, *dS_c, *Tinv, *W, *U, *Gcum, *beta, *dq_sm;
+    const float *dO, *dUt, *Ut, *S_c, *dS_c, *Tinv, *Up, *Gcum, *beta, *dq_sm;   // Up: U^T in 4-token pieces
+    const __half *Wt;                                                            // W^T [chunk][d][64]
     const uint8_t *route;
     float scale_la;
     __nv_bfloat16 *dq, *dk, *dv;
@@ -409,8 +410,15 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
         st_tile(sDO, xo, scO);
         st_tile(sDU, xu, scU);
         st_tile(sDS1, xs, scS);
-        ld_tile(xo, p.W + tok0, ts);                              // next batch into the freed registers
-        ld_tile(xu, p.U + tok0, ts);
+        // next batch into the freed registers: W^T and U^T as the forward kernels keep them (fp16
+        // [d][64] tile; fp32 in 4-token pieces [16][d][4]) -- both are [k][n] operands as they are
+        uint4 wt[2];
+#pragma unroll
+        for (int it = 0; it < 2; ++it)
+            wt[it] = reinterpret_cast<const uint4 *>(p.Wt + chunk * D * 64)[tid + it * kCkThreads];
+#pragma unroll
+        for (int it = 0; it < 4; ++it)
+            xu[it] = reinterpret_cast<const float4 *>(p.Up + chunk * D * 64)[tid + it * kCkThreads];
         uint2 qk[2][4];
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
@@ -421,8 +429,17 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
         st_tile(sUt, y0, 1.f);
         st_tile(sS0, y1, 1.f);
         st_tile(sT, y2, 1.f);
-        st_tile(sW, xo, 1.f);
-        st_tile(sU, xu, 1.f);
+#pragma unroll
+        for (int it = 0; it < 2; ++it) {
+            const int idx = tid + it * kCkThreads;
+            *reinterpret_cast<uint4 *>(sW + (idx >> 3) * kLdH + (idx & 7) * 8) = wt[it];
+        }
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int e = tid + it * kCkThreads, pc = e >> 6, vv = e & 63;
+            *reinterpret_cast<uint2 *>(sU + vv * kLdH + 4 * pc) =
+                make_uint2(pack_half2(xu[it].x, xu[it].y), pack_half2(xu[it].z, xu[it].w));
+        }
 #pragma unroll
         for (int it = 0; it < 4; ++it) {                           // bf16 -> fp16 (exact)
             auto cv = [](uint32_t w) {
@@ -539,8 +556,8 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
 
     // ---- M = -(dKb W^T + dVb U^T);  Mg = M . Gamma, j < i -> X;  Ms = diag(beta~) Mg -> slot of T ----
     zero();
-    mma64<false, true>(sDO, sW, row0, n0, lane, acc);
-    mma64<false, true>(sS0, sU, row0, n0, lane, acc);
+    mma64<false, false>(sDO, sW, row0, n0, lane, acc);      // sW, sU hold W^T, U^T: [k][n] operands
+    mma64<false, false>(sS0, sU, row0, n0, lane, acc);
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
@@ -667,7 +684,7 @@ cudaError_t launch_gdn_rscan_tc(const void *dO16, const void *dOg16, const GdnTc
 
 cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, const float *dO,
                                  const float *dUt, const float *Ut, const float *S_c, const float *dS_c,
-                                 const float *Tinv, const float *W, const float *U, const float *Gcum,
+                                 const float *Tinv, const void *Wt, const float *Up, const float *Gcum,
                                  const float *beta, const uint8_t *route, const float *dq_sm,
                                  float scale_la, void *dq, void *dk, void *dv, float *dg,
                                  float *dbeta, Shape s, cudaStream_t st) {
@@ -676,7 +693,7 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
                                          kCkSmem);
     if (e != cudaSuccess) return e;
     ChunkBwdArgs a{(const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, dO, dUt, Ut,
-                   S_c, dS_c, Tinv, W, U, Gcum, beta, dq_sm, route, scale_la, (__nv_bfloat16 *)dq,
+                   S_c, dS_c, Tinv, Up, Gcum, beta, dq_sm, (const __half *)Wt, route, scale_la, (__nv_bfloat16 *)dq,
                    (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, dg, dbeta, s.L, s.H};
     dim3 grid(s.L / kC, s.B * s.H);
     gdn_bwd_chunk_kernel<<<grid, kCkThreads, kCkSmem, st>>>(a);

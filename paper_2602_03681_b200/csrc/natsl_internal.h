@@ -165,7 +165,7 @@ cudaError_t launch_gdn_finish(const AssembleArgs &a, void *dk, void *dv, Shape s
 // per chunk (d = 64, bf16 storage): dq (with dq_sm added), dk, dv of the linear tokens, dg, dbeta.
 cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, const float *dO,
                                  const float *dUt, const float *Ut, const float *S_c, const float *dS_c,
-                                 const float *Tinv, const float *W, const float *U, const float *Gcum,
+                                 const float *Tinv, const void *Wt, const float *Up, const float *Gcum,
                                  const float *beta, const uint8_t *route, const float *dq_sm,
                                  float scale_la, void *dq, void *dk, void *dv, float *dg,
                                  float *dbeta, Shape s, cudaStream_t st);
