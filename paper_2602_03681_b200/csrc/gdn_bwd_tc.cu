@@ -606,23 +606,47 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
         atomicAdd(rK + iA, kapA); atomicAdd(rK + iB, kapB);
         atomicAdd(rB + iA, dbA); atomicAdd(rB + iB, dbB);
     }
-    // ---- dq, dk, dv ----
-    const bool linA = p.route[((size_t)b * p.L + (size_t)c * kC + iA) * p.H + h] == 0;
-    const bool linB = p.route[((size_t)b * p.L + (size_t)c * kC + iB) * p.H + h] == 0;
+    // ---- dq, dk, dv: through fp32 tiles in the (now free) operand slots, so that every global
+    // access of the epilogue is a contiguous 64-byte piece of a row instead of a scattered pair ----
+    constexpr int kLdF = 68;                                       // row stride of the fp32 tiles
+    float *fDQ = reinterpret_cast<float *>(smraw), *fDK = fDQ + 64 * kLdF, *fDV = fDK + 64 * kLdF;
+    static_assert(3 * 64 * kLdF * 4 <= 6 * kTileH * 2, "the three result tiles must fit in the first six slots");
+    const int er = tid >> 2, ec = (tid & 3) * 16;                  // epilogue: row, first of 16 columns
+    const size_t eoff = tok0 + (size_t)er * ts + ec;
+    float4 dqs[4];                                                 // softmax-branch dq, on its way early
+#pragma unroll
+    for (int x = 0; x < 4; ++x) dqs[x] = *reinterpret_cast<const float4 *>(p.dq_sm + eoff + 4 * x);
+    const bool lin = p.route[((size_t)b * p.L + (size_t)c * kC + er) * p.H + h] == 0;
+    __syncthreads();                                               // all products have read their operands
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
-        const size_t oA = tok0 + (size_t)iA * ts + n0 + 8 * nt + 2 * t, oB = tok0 + (size_t)iB * ts + n0 + 8 * nt + 2 * t;
-        const float2 sa = *reinterpret_cast<const float2 *>(p.dq_sm + oA);
-        const float2 sb = *reinterpret_cast<const float2 *>(p.dq_sm + oB);
-        *reinterpret_cast<__nv_bfloat162 *>(p.dq + oA) = __floats2bfloat162_rn(dq[nt][0] + sa.x, dq[nt][1] + sa.y);
-        *reinterpret_cast<__nv_bfloat162 *>(p.dq + oB) = __floats2bfloat162_rn(dq[nt][2] + sb.x, dq[nt][3] + sb.y);
-        if (linA) {
-            *reinterpret_cast<__nv_bfloat162 *>(p.dk + oA) = __floats2bfloat162_rn(dk[nt][0], dk[nt][1]);
-            *reinterpret_cast<__nv_bfloat162 *>(p.dv + oA) = __floats2bfloat162_rn(dv[nt][0], dv[nt][1]);
-        }
-        if (linB) {
-            *reinterpret_cast<__nv_bfloat162 *>(p.dk + oB) = __floats2bfloat162_rn(dk[nt][2], dk[nt][3]);
-            *reinterpret_cast<__nv_bfloat162 *>(p.dv + oB) = __floats2bfloat162_rn(dv[nt][2], dv[nt][3]);
+        const int cc = n0 + 8 * nt + 2 * t;
+        *reinterpret_cast<float2 *>(fDQ + iA * kLdF + cc) = make_float2(dq[nt][0], dq[nt][1]);
+        *reinterpret_cast<float2 *>(fDQ + iB * kLdF + cc) = make_float2(dq[nt][2], dq[nt][3]);
+        *reinterpret_cast<float2 *>(fDK + iA * kLdF + cc) = make_float2(dk[nt][0], dk[nt][1]);
+        *reinterpret_cast<float2 *>(fDK + iB * kLdF + cc) = make_float2(dk[nt][2], dk[nt][3]);
+        *reinterpret_cast<float2 *>(fDV + iA * kLdF + cc) = make_float2(dv[nt][0], dv[nt][1]);
+        *reinterpret_cast<float2 *>(fDV + iB * kLdF + cc) = make_float2(dv[nt][2], dv[nt][3]);
+    }
+    __syncthreads();
+    {
+        auto row16 = [&](const float *tile, const float4 *add, __nv_bfloat16 *dst) {
+            uint32_t o[8];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                float4 v4 = *reinterpret_cast<const float4 *>(tile + er * kLdF + ec + 4 * x);
+                if (add) { v4.x += add[x].x; v4.y += add[x].y; v4.z += add[x].z; v4.w += add[x].w; }
+                o[2 * x] = pack_bf162(v4.x, v4.y);
+                o[2 * x + 1] = pack_bf162(v4.z, v4.w);
+            }
+            uint4 *d4 = reinterpret_cast<uint4 *>(dst + eoff);
+            d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
+            d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
+        };
+        row16(fDQ, dqs, p.dq);
+        if (lin) {
+            row16(fDK, nullptr, p.dk);
+            row16(fDV, nullptr, p.dv);
         }
     }
     __syncthreads();
