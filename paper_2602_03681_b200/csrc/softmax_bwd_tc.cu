@@ -174,6 +174,13 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
         const float lse2 = row_ok ? lse[(size_t)bh * L + i_abs] * kLog2e : 0.f;
         const float Di = row_ok ? Dsm[(size_t)bh * L + i_abs] : 0.f;
         bool ok = true;
+        // The compacted keys are in position order, so row i sees exactly the first `cnt` of them
+        // (a per-element look-up of the key's position costs a divergent branch per element).
+        int cnt = 0;
+        if (row_ok) {
+            cnt = n_full;
+            for (int kq = 0; kq < n_end - n_full; ++kq) cnt += ms.pos[kq] <= i_abs ? 1 : 0;
+        }
         for (int t = 0; t < T; ++t) {
             ok = mbar_wait(&ms.barS, t & 1, abort_flag);
             if (!ok) break;
@@ -192,7 +199,7 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
                     const int jj = t * 64 + 32 * half + c;
-                    const bool vis = row_ok && (jj < n_full || (jj < n_end && ms.pos[jj - n_full] <= i_abs));
+                    const bool vis = jj < cnt;
                     // mask on the exponent (exp2(-inf) = 0), not around the expression: no branch
                     const float pr = exp2f(vis ? fmaf(__uint_as_float(sv[c]), sl2, -lse2) : -INFINITY);
                     ds[32 * half + c] = scale_sm * pr * (__uint_as_float(dv[c]) - Di);
