@@ -201,7 +201,7 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
                     const int jj = t * 64 + 32 * half + c;
                     const bool vis = jj < cnt;
                     // mask on the exponent (exp2(-inf) = 0), not around the expression: no branch
-                    const float pr = exp2f(vis ? fmaf(__uint_as_float(sv[c]), sl2, -lse2) : -INFINITY);
+                    const float pr = ex2_ftz(vis ? fmaf(__uint_as_float(sv[c]), sl2, -lse2) : -INFINITY);
                     ds[32 * half + c] = scale_sm * pr * (__uint_as_float(dv[c]) - Di);
                 }
             }
@@ -417,7 +417,7 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                 for (int c = 0; c < 32; ++c) {
                     const int cc = 32 * half + c;
                     const bool vis = pos_j <= i0 + cc;
-                    const float pr = exp2f(vis ? fmaf(__uint_as_float(sv[c]), sl2, -lse2[cc]) : -INFINITY);
+                    const float pr = ex2_ftz(vis ? fmaf(__uint_as_float(sv[c]), sl2, -lse2[cc]) : -INFINITY);
                     pv[cc] = pr;
                     ds[cc] = scale_sm * pr * (__uint_as_float(dv[c]) - dsum[cc]);
                 }

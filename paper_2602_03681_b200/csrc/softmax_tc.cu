@@ -262,7 +262,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < kBN; ++c) {
-                x[c] = exp2f(x[c] - m_use);
+                x[c] = ex2_ftz(x[c] - m_use);
                 ps4[c & 3] += x[c];
             }
             l = l * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));

@@ -323,6 +323,13 @@ __device__ __forceinline__ uint32_t sw128_offset(int row, int piece) {
     return (uint32_t)row * 128u + (uint32_t)((piece ^ (row & 7)) << 4);
 }
 
+// 2^x as one special-function instruction (results below 2^-126 flush to zero; exp2f without
+// fast-math adds range fix-ups around the same instruction).
+__device__ __forceinline__ float ex2_ftz(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
     __half2 h = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&h);
