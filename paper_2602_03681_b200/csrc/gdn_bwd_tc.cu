@@ -455,7 +455,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
     const int row0 = 16 * (warp & 3), n0 = 32 * (warp >> 2);
     const int iA = row0 + g, iB = iA + 8;                          // this lane's two rows (tokens)
     const float GA = sG[iA], GB = sG[iB], GC = sG[63];
-    const float gamA = __expf(GA), gamB = __expf(GB), ktA = __expf(GC - GA), ktB = __expf(GC - GB);
+    const float gamA = exp_ftz(GA), gamB = exp_ftz(GB), ktA = exp_ftz(GC - GA), ktB = exp_ftz(GC - GB);
     const float btA = sBt[iA], btB = sBt[iB];
     float dq[4][4], dk[4][4], dv[4][4], acc[4][4];
     float dGA = 0.f, dGB = 0.f, kapA = 0.f, kapB = 0.f, dbA = 0.f, dbB = 0.f;
@@ -521,7 +521,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int j = n0 + 8 * nt + 2 * t + (e & 1), i = e < 2 ? iA : iB;
-            acc[nt][e] *= p.scale_la * __expf(j <= i ? (e < 2 ? GA : GB) - sG[j] : -INFINITY);   // branch-free mask
+            acc[nt][e] *= p.scale_la * exp_ftz(j <= i ? (e < 2 ? GA : GB) - sG[j] : -INFINITY);   // branch-free mask
         }
     put(sY, 1.f, 1.f);
     __syncthreads();                    // X = dW, Y = Ns; dO, S0, dS1 are free
@@ -563,7 +563,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int j = n0 + 8 * nt + 2 * t + (e & 1), i = e < 2 ? iA : iB;
-            acc[nt][e] *= -__expf(j < i ? (e < 2 ? GA : GB) - sG[j] : -INFINITY);
+            acc[nt][e] *= -exp_ftz(j < i ? (e < 2 ? GA : GB) - sG[j] : -INFINITY);
         }
     put(sX, 1.f, 1.f);
     put(sT, btA, btB);
@@ -664,7 +664,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
         float gs = 0.f;
 #pragma unroll
         for (int wv = 0; wv < 8; ++wv) gs += sMax[24 + wv];
-        const float extra = sMax[34] + sMax[35] + __expf(sG[63]) * gs + (warp == 0 ? sMax[33] : 0.f);
+        const float extra = sMax[34] + sMax[35] + exp_ftz(sG[63]) * gs + (warp == 0 ? sMax[33] : 0.f);
         const size_t tk = ((size_t)b * p.L + (size_t)c * kC + tid) * p.H + h;
         p.dg[tk] = suf + extra;
         p.dbeta[tk] = p.route[tk] ? 0.f : rB[tid];

@@ -197,7 +197,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             if (warp == 1) G += ms.wsum[0];
             ms.G[i] = G;
             ms.bt[i] = btv;
-            ms.btg[i] = btv * __expf(G);
+            ms.btg[i] = btv * exp_ftz(G);
         }
         // ---- tiles to fp16, in place ----
         bool ok = mbar_wait(&ms.barLoad, 0, abort_flag);
@@ -217,8 +217,8 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 // ---- decay factors for the scan, P (lower triangle).  A real loop over 8-column
                 // pieces: straight-line code that runs once per CTA is bound by instruction fetch. ----
                 float *gd = Gd + chunk * 128;
-                gd[i] = __expf(G);
-                gd[64 + i] = __expf(ms.G[63] - G);
+                gd[i] = exp_ftz(G);
+                gd[64 + i] = exp_ftz(ms.G[63] - G);
                 if (ex.Gcum) ex.Gcum[(size_t)bh * L + tok0 + i] = G;
                 uint4 *prow = reinterpret_cast<uint4 *>(Ph + (chunk * 64 + i) * 64);
 #pragma unroll 1
@@ -232,7 +232,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                         const int j = 8 * pc + e;
                         // the mask goes on the exponent (exp(-inf) = 0): a conditional around the whole
                         // expression compiles to one divergent branch per element
-                        x[e] = scale_la * __expf(j <= i ? G - ms.G[j] : -INFINITY) * __uint_as_float(d8[e]);
+                        x[e] = scale_la * exp_ftz(j <= i ? G - ms.G[j] : -INFINITY) * __uint_as_float(d8[e]);
                     }
                     prow[pc] = make_uint4(pack_half2(x[0], x[1]), pack_half2(x[2], x[3]),
                                           pack_half2(x[4], x[5]), pack_half2(x[6], x[7]));
@@ -268,7 +268,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll
                         for (int jj = 0; jj < 16; ++jj) {
                             const int j = 16 * jb + jj;
-                            a[jj] = btv * __expf(j < i ? G - ms.G[j] : -INFINITY) * __uint_as_float(dd[j >> 5][j & 31]);
+                            a[jj] = btv * exp_ftz(j < i ? G - ms.G[j] : -INFINITY) * __uint_as_float(dd[j >> 5][j & 31]);
                         }
                         if (jb < bk) {
 #pragma unroll
