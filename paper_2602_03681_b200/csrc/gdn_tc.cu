@@ -473,11 +473,12 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 }
 
 // ==========================================================================================
-// Scan: one CTA per (batch, head), sequential over chunks.  Value column r of the state (row r of
+// Scan: one CTA per (batch, head) -- or per segment of its chunks, see ScanSegments --, sequential
+// over chunks.  Value column r of the state (row r of
 // S^T, TMEM lane r) belongs to the two threads (r, half 0) and (r, half 1) of warps q and q + 4,
 // which split every row between them; warp 8 issues MMAs, warp 9 issues TMA.  The fp32 state
 // lives in the registers of its two threads (half a row each); per chunk c:
-//   (a) S_c (fp16 operand) -> shared memory;                 MMA: WS = S^T W^T, QS = S^T Q^T
+//   (a) S_c (fp16 operand) -> TMEM;                          MMA: WS = S^T W^T, QS = S^T Q^T
 //   (b) U~^T = U^T - WS  -> operands U~ and U~ diag(gamma_C/gamma);
 //                                      MMA: dS = (U~ diag(gamma_C/gamma))^T-rows x K,  D3 = U~^T P^T
 //   (c) [for chunk c-1, behind the MMAs of (b)]  o_la^T = scale_la diag(gamma) QS + D3
