@@ -82,10 +82,13 @@ def route_compact(route: np.ndarray, C: int):
 
 
 def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5, state_in=None,
-               want_cache=False):
+               want_cache=False, block=None):
     """Token-by-token forward (Section 4.1 masks, Section 4.3 GDN + decay-always + Norm).
 
     q,k,v [B,L,H,d]; g,beta [B,L,H]; route [B,L,H]; w [B,L,H,2] or None.
+    block=R: one routing decision per block of R tokens; both operations see the query's own
+    block and the one not chosen is rolled back at the block's end (Section 4.1, the paragraphs
+    on intra-chunk correlations and per-token generation).  route must be constant per block.
     Returns dict(out, o_la, o_nla [B,L,H,d]; lse [B,H,L]; state_out [B,H,d,d];
     and with want_cache: k_sm, v_sm [B,H,L,d], n_sm [B,H]).
     """
@@ -98,11 +101,16 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5,
     kc = np.zeros((B, H, L, d)) if want_cache else None
     vc = np.zeros((B, H, L, d)) if want_cache else None
     n_sm = np.zeros((B, H), np.int32) if want_cache else None
-    rc = _load().natsl_oracle_hybrid_fwd(
-        _p(q), _p(k), _p(v), _p(g), _p(beta), _p(route, _u8p), _p(w), B, L, H, d,
-        ctypes.c_double(scale_la), ctypes.c_double(scale_sm), ctypes.c_double(eps),
-        _p(state_in), _p(out), _p(o_la), _p(o_nla), _p(lse), _p(state_out), _p(kc), _p(vc),
-        _p(n_sm, _i32p))
+    tail = (ctypes.c_double(scale_la), ctypes.c_double(scale_sm), ctypes.c_double(eps),
+            _p(state_in), _p(out), _p(o_la), _p(o_nla), _p(lse), _p(state_out), _p(kc), _p(vc),
+            _p(n_sm, _i32p))
+    head = (_p(q), _p(k), _p(v), _p(g), _p(beta), _p(route, _u8p), _p(w), B, L, H, d)
+    if block is None:
+        rc = _load().natsl_oracle_hybrid_fwd(*head, *tail)
+    else:
+        rc = _load().natsl_oracle_hybrid_fwd_block(*head, int(block), *tail)
+    if rc == -4:
+        raise ValueError("block mode: route must be constant within each block")
     if rc != 0:
         raise RuntimeError(f"natsl_oracle_hybrid_fwd failed ({rc})")
     res = dict(out=out, o_la=o_la, o_nla=o_nla, lse=lse, state_out=state_out)

@@ -27,6 +27,10 @@
  *   state       [B, H, dk, dv] o_la = scale_la * q S  (read after the token's own update)
  *   lse         [B, H, L]      log-sum-exp of the softmax logits, -inf for an empty row
  *
+ * natsl_oracle_hybrid_fwd_block is the same layer with one routing decision per block of
+ * tokens, written the way the paper describes generation: both operations run inside a block
+ * and the one not chosen is rolled back at its end.
+ *
  * Parity pins live in tests/ (closed forms, a library attention routine, brute
  * force on tiny inputs, finite differences); none of them calls back into the
  * formula they check.
@@ -99,10 +103,13 @@ static double rms_factor(const double *o, int d, double eps)
 
 /* One token of the hybrid layer for one (batch, head).
  * S      : dk x dv state, updated in place
- * kc, vc : retained keys / values so far, n_c rows of d; the new token is appended when r = 1
+ * kc, vc : retained keys / values so far, n_c rows of d
+ * delta  : apply the delta update of this token to S;  append: add its K/V to kc, vc.
+ *          Token-level routing sets exactly one of the two (delta for a linear token, append for
+ *          a softmax token); inside an undecided block both are set (see the block-mode forward).
  * Outputs (each may be NULL): o_la, o_nla rows, lse, out row. */
 static void hybrid_token(int d, const double *q, const double *k, const double *v,
-                         double g, double beta, int r, double w_nla, double w_la,
+                         double g, double beta, int delta, int append, double w_nla, double w_la,
                          double scale_la, double scale_sm, double eps,
                          double *S, double *kc, double *vc, int *n_c,
                          double *logit /* scratch, >= n_c+1 */,
@@ -111,7 +118,7 @@ static void hybrid_token(int d, const double *q, const double *k, const double *
     /* decay on every token */
     double alpha = exp(g);
     for (int a = 0; a < d * d; ++a) S[a] *= alpha;
-    if (!r) {
+    if (delta) {
         /* delta rule against the decayed state: S += beta k^T (v - k S) */
         for (int c = 0; c < d; ++c) {
             double ks = 0.0;
@@ -119,7 +126,8 @@ static void hybrid_token(int d, const double *q, const double *k, const double *
             double e = v[c] - ks;
             for (int a = 0; a < d; ++a) S[(size_t)a * d + c] += beta * k[a] * e;
         }
-    } else {
+    }
+    if (append) {
         memcpy(kc + (size_t)(*n_c) * d, k, sizeof(double) * d);
         memcpy(vc + (size_t)(*n_c) * d, v, sizeof(double) * d);
         *n_c += 1;
@@ -131,7 +139,7 @@ static void hybrid_token(int d, const double *q, const double *k, const double *
         for (int a = 0; a < d; ++a) acc += q[a] * S[(size_t)a * d + c];
         o_la[c] = scale_la * acc;
     }
-    /* softmax branch over the retained tokens (this one included when r = 1) */
+    /* softmax branch over the retained tokens (this one included when it was appended) */
     int n = *n_c;
     double lse = -INFINITY;
     for (int c = 0; c < d; ++c) o_nla[c] = 0.0;
@@ -193,7 +201,8 @@ int natsl_oracle_hybrid_fwd(const double *q, const double *k, const double *v,
             for (int i = 0; i < L; ++i) {
                 size_t t = AT3(b, i, h);
                 double wn = w ? w[t * 2 + 0] : 0.5, wl = w ? w[t * 2 + 1] : 0.5;
-                hybrid_token(d, q + t * d, k + t * d, v + t * d, g[t], beta[t], route[t] != 0,
+                hybrid_token(d, q + t * d, k + t * d, v + t * d, g[t], beta[t], route[t] == 0,
+                             route[t] != 0,
                              wn, wl, scale_la, scale_sm, eps, S, kc, vc, &n_c, logit,
                              o_la ? o_la + t * d : NULL, o_nla ? o_nla + t * d : NULL,
                              lse ? lse + (size_t)bh * L + i : NULL, out ? out + t * d : NULL);
@@ -206,6 +215,74 @@ int natsl_oracle_hybrid_fwd(const double *q, const double *k, const double *v,
         free(S); free(kc); free(vc); free(logit);
     }
     return err ? -2 : 0;
+}
+
+/* ---------------------------------------------------------------------------
+ * Block-mode forward (Section 4.1, the paragraphs after the chunk-state case equation and on
+ * per-token generation): one routing decision per block of R tokens, known only when the block
+ * is complete.  Until then both branches treat every token of the block as their own -- the
+ * linear state takes the token's delta update and the token's K/V join the retained set -- so
+ * that each output contains the intra-block correlations of both operations.  At the end of the
+ * block the operation that was not chosen is rolled back: for a linear block the block's K/V are
+ * removed again; for a softmax block the linear state is reset to its value at the start of the
+ * block, with the block's decay applied (Section 4.3, the decay-always equation).
+ *   route [B,L,H] must be constant within each block of R tokens (-4 otherwise); L % R == 0.
+ * Outputs as natsl_oracle_hybrid_fwd.
+ * ------------------------------------------------------------------------- */
+int natsl_oracle_hybrid_fwd_block(const double *q, const double *k, const double *v,
+                                  const double *g, const double *beta, const uint8_t *route,
+                                  const double *w, int B, int L, int H, int d, int R,
+                                  double scale_la, double scale_sm, double eps,
+                                  const double *state_in, double *out, double *o_la,
+                                  double *o_nla, double *lse, double *state_out, double *kc_out,
+                                  double *vc_out, int32_t *n_sm_out)
+{
+    if (d > 512 || d <= 0 || R <= 0 || L % R != 0) return -1;
+    int err = 0, bad_route = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int bh = 0; bh < B * H; ++bh) {
+        int b = bh / H, h = bh % H;
+        double *S = (double *)calloc((size_t)d * d, sizeof(double));
+        double *S_start = (double *)malloc(sizeof(double) * (size_t)d * d);
+        double *kc = (double *)malloc(sizeof(double) * (size_t)L * d);
+        double *vc = (double *)malloc(sizeof(double) * (size_t)L * d);
+        double *logit = (double *)malloc(sizeof(double) * (size_t)(L + 1));
+        if (!S || !S_start || !kc || !vc || !logit) {
+            err = 1;
+        } else {
+            if (state_in) memcpy(S, state_in + (size_t)bh * d * d, sizeof(double) * d * d);
+            int n_c = 0;
+            for (int i0 = 0; i0 < L; i0 += R) {
+                const int r = route[AT3(b, i0, h)] != 0;
+                const int n_start = n_c;
+                double g_block = 0.0;
+                memcpy(S_start, S, sizeof(double) * d * d);
+                for (int i = i0; i < i0 + R; ++i) {
+                    size_t t = AT3(b, i, h);
+                    if ((route[t] != 0) != r) bad_route = 1;
+                    double wn = w ? w[t * 2 + 0] : 0.5, wl = w ? w[t * 2 + 1] : 0.5;
+                    g_block += g[t];
+                    hybrid_token(d, q + t * d, k + t * d, v + t * d, g[t], beta[t], 1, 1,
+                                 wn, wl, scale_la, scale_sm, eps, S, kc, vc, &n_c, logit,
+                                 o_la ? o_la + t * d : NULL, o_nla ? o_nla + t * d : NULL,
+                                 lse ? lse + (size_t)bh * L + i : NULL, out ? out + t * d : NULL);
+                }
+                if (r) {
+                    double decay = exp(g_block);
+                    for (int a = 0; a < d * d; ++a) S[a] = decay * S_start[a];
+                } else {
+                    n_c = n_start;
+                }
+            }
+            if (state_out) memcpy(state_out + (size_t)bh * d * d, S, sizeof(double) * d * d);
+            if (kc_out) memcpy(kc_out + (size_t)bh * L * d, kc, sizeof(double) * (size_t)n_c * d);
+            if (vc_out) memcpy(vc_out + (size_t)bh * L * d, vc, sizeof(double) * (size_t)n_c * d);
+            if (n_sm_out) n_sm_out[bh] = n_c;
+        }
+        free(S); free(S_start); free(kc); free(vc); free(logit);
+    }
+    if (err) return -2;
+    return bad_route ? -4 : 0;
 }
 
 /* ---------------------------------------------------------------------------
@@ -232,7 +309,7 @@ int natsl_oracle_decode_step(const double *q, const double *k, const double *v,
         double *logit = (double *)malloc(sizeof(double) * (size_t)(n_c + 2));
         double wn = w ? w[(size_t)bh * 2] : 0.5, wl = w ? w[(size_t)bh * 2 + 1] : 0.5;
         hybrid_token(d, q + (size_t)bh * d, k + (size_t)bh * d, v + (size_t)bh * d, g[bh], beta[bh],
-                     route[bh] != 0, wn, wl, scale_la, scale_sm, eps,
+                     route[bh] == 0, route[bh] != 0, wn, wl, scale_la, scale_sm, eps,
                      state + (size_t)bh * d * d, k_cache + (size_t)bh * cache_cap * d,
                      v_cache + (size_t)bh * cache_cap * d, &n_c, logit,
                      o_la ? o_la + (size_t)bh * d : NULL, o_nla ? o_nla + (size_t)bh * d : NULL,

@@ -442,3 +442,143 @@ def test_inactive_branch_gradients_vanish():
     assert np.all(gl["dk"][~lin] == 0) and np.all(gl["dv"][~lin] == 0)
     assert np.all(gl["dbeta"][~lin] == 0)
     assert np.abs(gl["dk"][lin]).min() > 0
+
+
+# ------------------------------------------------------------------ block mode (Section 4.1)
+def _block_route(B, L, H, R, p, seed):
+    r = np.random.default_rng(seed)
+    return np.repeat((r.random((B, L // R, H)) < p).astype(np.uint8), R, axis=1)
+
+
+def test_block_mode_fig1c_visibility_pattern():
+    """Fig. 1(c) with its D cells: the query's own chunk is read by both operations, the cells
+    of earlier chunks by exactly one."""
+    rows = [ln.strip() for ln in open(os.path.join(GOLDEN, "fig1c_visibility.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    fig = np.array([list(r) for r in rows])
+    C = 2
+    route = np.zeros(12, np.uint8)
+    route[[0, 1, 6, 7]] = 1
+    x = rand_inputs(1, 12, 1, 4, seed=15)
+    x["route"] = route[None, :, None].copy()
+    x["beta"] = np.full_like(x["beta"], 0.7)
+
+    def influence(field):
+        base = fwd(x, block=C)[field][0, :, 0]
+        vis = np.zeros((12, 12), bool)
+        for j in range(12):
+            y = {n: a.copy() for n, a in x.items()}
+            y["v"][0, j, 0] += 1e-3
+            vis[:, j] = np.abs(fwd(y, block=C)[field][0, :, 0] - base).max(-1) > 0
+        return vis
+
+    sm, la = influence("o_nla"), influence("o_la")
+    chunk = np.arange(12) // C
+    earlier = chunk[:, None] > chunk[None, :]
+    own = (chunk[:, None] == chunk[None, :]) & np.tril(np.ones((12, 12), bool))
+    assert np.array_equal(own, fig == "D")
+    assert np.array_equal(sm & ~earlier, own) and np.array_equal(la & ~earlier, own)
+    assert np.array_equal(sm & earlier, fig == "S")
+    for i in range(12):
+        cols = np.nonzero(la[i] & earlier[i])[0]
+        gcol = np.nonzero(fig[i] == "G")[0]
+        if len(gcol) == 0:
+            assert len(cols) == 0
+        else:
+            assert cols.max() == gcol[0] and np.all(route[cols] == 0)
+    # earlier chunks: every token in exactly one branch
+    assert np.array_equal((sm | la) & earlier, earlier) and not np.any(sm & la & earlier)
+
+
+def test_block_mode_all_softmax_is_causal_attention_and_blockwise_gdn():
+    B, L, H, d, R = 2, 48, 2, 8, 8
+    x = rand_inputs(B, L, H, d, seed=31)
+    x["route"] = np.ones((B, L, H), np.uint8)
+    S0 = RNG.standard_normal((B, H, d, d))
+    r = fwd(x, block=R, state_in=S0)
+    # softmax branch: plain causal attention (library routine)
+    tq, tk, tv = (torch.from_numpy(x[n]).permute(0, 2, 1, 3) for n in ("q", "k", "v"))
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True, scale=1.5)
+    np.testing.assert_allclose(r["o_nla"], ref.permute(0, 2, 1, 3).numpy(), rtol=1e-10, atol=1e-12)
+    # the state only decays
+    G = x["g"].sum(1)                                          # [B,H]
+    np.testing.assert_allclose(r["state_out"], np.exp(G)[..., None, None] * S0, rtol=1e-12)
+    # linear branch: every block is a pure GDN run over the block alone, entered with the
+    # decayed initial state (the token-level oracle with route 0 on that block)
+    for c in range(L // R):
+        sl = slice(c * R, (c + 1) * R)
+        S_c = np.exp(x["g"][:, :c * R].sum(1))[..., None, None] * S0
+        y = {n: x[n][:, sl] for n in ("q", "k", "v", "g", "beta", "w")}
+        y["route"] = np.zeros((B, R, H), np.uint8)
+        blk = fwd(y, state_in=S_c)
+        np.testing.assert_allclose(r["o_la"][:, sl], blk["o_la"], rtol=1e-10, atol=1e-13)
+
+
+def test_block_mode_all_linear_is_gdn_and_block_local_attention():
+    B, L, H, d, R = 1, 40, 2, 8, 8
+    x = rand_inputs(B, L, H, d, seed=32)
+    x["route"] = np.zeros((B, L, H), np.uint8)
+    r = fwd(x, block=R)
+    tok = fwd(x)                                               # token level, all linear: pure GDN
+    np.testing.assert_allclose(r["o_la"], tok["o_la"], rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(r["state_out"], tok["state_out"], rtol=1e-12, atol=1e-15)
+    for c in range(L // R):
+        sl = slice(c * R, (c + 1) * R)
+        tq, tk, tv = (torch.from_numpy(x[n][:, sl]).permute(0, 2, 1, 3) for n in ("q", "k", "v"))
+        ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True, scale=1.5)
+        np.testing.assert_allclose(r["o_nla"][:, sl], ref.permute(0, 2, 1, 3).numpy(), rtol=1e-10,
+                                   atol=1e-12)
+
+
+def test_block_mode_brute_force_mixed_routes():
+    """Mixed routes, tiny: the softmax branch from its dense mask (retained earlier blocks plus
+    the causal part of the own block), the linear branch from the paper's matrix form of the GDN
+    update restarted at each block from the committed state."""
+    B, L, H, d, R = 1, 24, 1, 6, 4
+    x = rand_inputs(B, L, H, d, seed=33)
+    x["route"] = _block_route(B, L, H, R, 0.4, seed=5)
+    assert 0 < x["route"].sum() < L
+    S0 = RNG.standard_normal((B, H, d, d))
+    r = fwd(x, block=R, state_in=S0, want_cache=True)
+    q, k, v = (x[n][0, :, 0] for n in ("q", "k", "v"))
+    g, beta, route = (x[n][0, :, 0] for n in ("g", "beta", "route"))
+    blk = np.arange(L) // R
+    i, j = np.meshgrid(np.arange(L), np.arange(L), indexing="ij")
+    mask = (j <= i) & ((route[j] == 1) | (blk[j] == blk[i]))
+    logits = np.where(mask, 1.5 * q @ k.T, -np.inf)
+    p = np.exp(logits - logits.max(1, keepdims=True))
+    p /= p.sum(1, keepdims=True)
+    np.testing.assert_allclose(r["o_nla"][0, :, 0], p @ v, rtol=1e-10, atol=1e-13)
+    np.testing.assert_allclose(r["lse"][0, 0], np.log(np.exp(logits).sum(1)), rtol=1e-10)
+    # linear branch, in the paper's orientation (its state is the transpose of ours):
+    # S_t = S_{t-1} alpha_t (I - beta_t k_t k_t^T) + beta_t v_t k_t^T,  o_t = S_t q_t
+    Sp = S0[0, 0].T.copy()
+    o_la = np.zeros((L, d))
+    eye = np.eye(d)
+    for c in range(L // R):
+        S_run = Sp.copy()
+        for t in range(c * R, (c + 1) * R):
+            S_run = S_run @ (np.exp(g[t]) * (eye - beta[t] * np.outer(k[t], k[t]))) \
+                + beta[t] * np.outer(v[t], k[t])
+            o_la[t] = 0.5 * S_run @ q[t]
+        Sp = S_run if route[c * R] == 0 else np.exp(g[c * R:(c + 1) * R].sum()) * Sp
+    np.testing.assert_allclose(r["o_la"][0, :, 0], o_la, rtol=1e-10, atol=1e-13)
+    np.testing.assert_allclose(r["state_out"][0, 0], Sp.T, rtol=1e-10, atol=1e-13)
+    # the retained set after the last block: the tokens of the softmax blocks, in order
+    keep = np.nonzero(route)[0]
+    assert r["n_sm"][0, 0] == len(keep)
+    assert np.array_equal(r["k_sm"][0, 0, :len(keep)], k[keep])
+    # combination: same Norm equation as the token-level mode
+    def norm(o):
+        return o / np.sqrt((o * o).mean(-1, keepdims=True) + 1e-5)
+    w = x["w"][0, :, 0]
+    np.testing.assert_allclose(r["out"][0, :, 0], w[:, :1] * norm(p @ v) + w[:, 1:] * norm(o_la),
+                               rtol=1e-10, atol=1e-13)
+
+
+def test_block_mode_rejects_route_that_changes_inside_a_block():
+    x = rand_inputs(1, 16, 1, 4, seed=34)
+    x["route"] = np.zeros((1, 16, 1), np.uint8)
+    x["route"][0, 5, 0] = 1
+    with pytest.raises(ValueError):
+        fwd(x, block=4)
