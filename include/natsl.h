@@ -53,7 +53,8 @@ typedef enum natsl_status {
     NATSL_ERR_CACHE_FULL = -7,  /* decode: a retained-KV cache has no room (device-detected) */
     NATSL_ERR_UNSUPPORTED = -8, /* valid request this build does not implement */
     NATSL_ERR_TOO_LARGE = -9,   /* natsl_hybrid_fwd_static: problem needs more than the built-in scratch */
-    NATSL_ERR_TIMEOUT = -10     /* a bounded device-side wait expired (device-detected); kernel drained */
+    NATSL_ERR_TIMEOUT = -10,    /* a bounded device-side wait expired (device-detected); kernel drained */
+    NATSL_ERR_ROUTE = -11       /* NATSL_BLOCK_ROUTING: route changes inside a block (device-detected) */
 } natsl_status;
 
 enum { NATSL_F32 = 0, NATSL_BF16 = 1 };
@@ -63,12 +64,27 @@ enum { NATSL_OP_FWD = 0, NATSL_OP_BWD = 1, NATSL_OP_DECODE = 2, NATSL_OP_COMPACT
 enum {
     NATSL_FORCE_SIMT = 1u << 0,  /* use the fp32 CUDA-core kernels even for bf16 tensors (the
                                     default for bf16 is the tcgen05 tensor-core path) */
-    NATSL_SINGLE_PASS_SCAN = 1u << 1   /* forward, tensor-core path: keep the scan over the chunks of a
+    NATSL_SINGLE_PASS_SCAN = 1u << 1,  /* forward, tensor-core path: keep the scan over the chunks of a
                                     (batch, head) in one CTA even when B*H is small.  By default
                                     such calls split the chunks into segments that run in
                                     parallel (a second run per segment yields the segment's
                                     state transition, a small kernel chains the segments); the
                                     results agree to rounding */
+    NATSL_BLOCK_ROUTING = 1u << 2      /* forward, tensor-core path: block-level routing, the paper's
+                                    default (Section 4.1, "compute the inner-chunk correlation";
+                                    Section 4.3, chunk size = GDN chunk size).  `route` holds one
+                                    decision per block of C = 64 tokens, repeated over the block's
+                                    tokens.  The decision is known only when the block is complete,
+                                    so both operations treat the tokens of the query's own block as
+                                    theirs: the softmax branch reads the retained tokens of earlier
+                                    blocks plus the causal part of the own block; the linear branch
+                                    reads the state committed by earlier linear blocks and runs the
+                                    delta rule over the own block, whose update is committed to the
+                                    state only if the block is linear (a softmax block leaves the
+                                    decay alone).  state_out, k_sm, v_sm, sm_len hold what is kept
+                                    after the last block.  A route that changes inside a block is
+                                    reported as NATSL_ERR_ROUTE by natsl_device_status.  Backward
+                                    and decode: NATSL_ERR_UNSUPPORTED with this flag */
 };
 
 typedef struct natsl_params {
@@ -115,7 +131,8 @@ int natsl_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk
  *   q,k,v [B,L,H,d] in p->dtype; g,beta [B,L,H] fp32 (g = log decay <= 0);
  *   route [B,L,H] u8; out [B,L,H,d] in p->dtype.
  * The linear branch is computed chunkwise (Section 3, chunkwise equations) with C = 64.
- * Optional outputs are taken from `p`.  Errors: NULL, SHAPE, DTYPE, ALIGN, WORKSPACE, CUDA.
+ * Optional outputs are taken from `p`.  Errors: NULL, SHAPE, DTYPE, ALIGN, WORKSPACE, CUDA;
+ * UNSUPPORTED for NATSL_BLOCK_ROUTING off the tensor-core path (fp32 storage, NATSL_FORCE_SIMT).
  */
 int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g,
                      const float *beta, const uint8_t *route, void *out,

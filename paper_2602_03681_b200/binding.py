@@ -18,7 +18,10 @@ NATSL_F32, NATSL_BF16 = 0, 1
 OP_FWD, OP_BWD, OP_DECODE, OP_COMPACT = 0, 1, 2, 3
 FORCE_SIMT = 1
 SINGLE_PASS_SCAN = 2
+BLOCK_ROUTING = 4
 ERR_CACHE_FULL = -7
+ERR_UNSUPPORTED = -8
+ERR_ROUTE = -11
 
 EXPORTS = ["natsl_workspace_size", "natsl_route_compact", "natsl_hybrid_fwd", "natsl_hybrid_bwd",
            "natsl_decode_step", "natsl_device_status", "natsl_hybrid_fwd_static",

@@ -194,6 +194,7 @@ const char *natsl_strerror(int status) {
         case NATSL_ERR_CUDA: return "CUDA launch or runtime error";
         case NATSL_ERR_CACHE_FULL: return "retained-KV cache full";
         case NATSL_ERR_UNSUPPORTED: return "request not implemented in this build";
+        case NATSL_ERR_ROUTE: return "block-level routing: route changes inside a block";
         case NATSL_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case NATSL_ERR_TOO_LARGE: return "problem needs more scratch than the library's built-in array (NATSL_STATIC_WS_BYTES)";
         default: return "unknown natsl status";
@@ -220,7 +221,7 @@ int natsl_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk
     if (rc != NATSL_OK) return rc;
     if (!route || !sm_idx || !sm_chunk_prefix || !lin_idx || !n_lin) return NATSL_ERR_NULL;
     cudaError_t e = launch_route_compact(route, sm_idx, sm_chunk_prefix, lin_idx, n_lin, nullptr,
-                                         p->B, p->L, p->H, static_cast<cudaStream_t>(stream));
+                                         nullptr, p->B, p->L, p->H, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
 }
 
@@ -236,10 +237,14 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     if (want_cache && !(p->k_sm && p->v_sm && p->sm_len && p->sm_cap > 0)) return NATSL_ERR_NULL;
     if (want_cache && (!aligned16(p->k_sm) || !aligned16(p->v_sm))) return NATSL_ERR_ALIGN;
     if ((p->o_la && !aligned16(p->o_la)) || (p->o_nla && !aligned16(p->o_nla))) return NATSL_ERR_ALIGN;
+    const bool tensor_cores = use_tensor_cores(p);
+    const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
+    if (block && !tensor_cores) return NATSL_ERR_UNSUPPORTED;
     FwdWs f = carve_fwd(p, ws);
     if (!ws || ws_bytes < f.bytes) return NATSL_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Shape s = shape_of(p);
+    const BlockRouting br{block ? route : nullptr, k, v};
 
 #define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
     int stage = 0;
@@ -253,9 +258,8 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     int32_t *sm_len = want_cache ? p->sm_len : f.sm_len;
     void *k_sm = want_cache ? p->k_sm : f.k_sm, *v_sm = want_cache ? p->v_sm : f.v_sm;
     const int32_t cap = want_cache ? p->sm_cap : p->L;
-    NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, sm_len, p->B, p->L,
-                                   p->H, st));
-    const bool tensor_cores = use_tensor_cores(p);
+    NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, sm_len,
+                                   block ? f.status : nullptr, p->B, p->L, p->H, st));
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
                                       f.v16, nullptr, cap, p->L, f.status, s, st));
@@ -264,21 +268,23 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(mark());
     float *o_la = p->o_la ? p->o_la : f.o_la;
     if (tensor_cores) {
-        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, GdnTcExport{}, f.status,
-                                        s, st));
+        // block-level routing: every token takes part in the delta rule of its own block
+        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc,
+                                        GdnTcExport{}, f.status, s, st));
         NATSL_TRY(mark());
         const int nseg = scan_segments(p);
         if (nseg > 1) {   // few (batch, head) pairs: segments in parallel, chained by their transitions
             ScanSegments sg{1, nseg, (int)(p->L / kC) / nseg, f.seg_incr, f.seg_trans, f.seg_start};
             NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, o_la, GdnTcExport{}, sg,
-                                         f.status, s, st));
+                                         br.route, f.status, s, st));
             NATSL_TRY(launch_scan_combine(p->state_in, sg, s, st));
             sg.mode = 2;
             NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, p->state_out, o_la, GdnTcExport{}, sg,
-                                         f.status, s, st));
+                                         br.route, f.status, s, st));
         } else {
             NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, p->state_out, o_la, GdnTcExport{},
-                                         ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, f.status, s, st));
+                                         ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, br.route,
+                                         f.status, s, st));
         }
     } else {
         NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P,
@@ -290,8 +296,8 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(mark());
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, p->L, f.sm_idx, f.prefix, o_la, p->w,
-                                            p->scale_sm, p->eps, out, p->o_nla, p->lse, f.status, s,
-                                            st));
+                                            p->scale_sm, p->eps, out, p->o_nla, p->lse, br, f.status,
+                                            s, st));
     else
         NATSL_TRY(launch_softmax_combine_simt(q, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
                                               p->scale_sm, p->eps, out, p->o_nla, p->lse, s, st));
@@ -308,7 +314,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (rc != NATSL_OK) return rc;
     if (!q || !k || !v || !g || !beta || !route || !dout || !dq || !dk || !dv || !dg || !dbeta)
         return NATSL_ERR_NULL;
-    if (p->state_in) return NATSL_ERR_UNSUPPORTED;
+    if (p->state_in || (p->flags & NATSL_BLOCK_ROUTING)) return NATSL_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
         return NATSL_ERR_ALIGN;
@@ -328,8 +334,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
 #define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
     NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
     // ---- forward recomputation, keeping what the backward needs ----
-    NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, p->B,
-                                   p->L, p->H, st));
+    NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, nullptr,
+                                   p->B, p->L, p->H, st));
     const bool tensor_cores = use_tensor_cores(p);
     const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
     if (!fused_chunks)
@@ -346,7 +352,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                              f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, ex, f.status, s, st));
         NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex,
-                                     ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, f.status, s, st));
+                                     ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, nullptr, f.status,
+                                     s, st));
     } else {
         NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
                                           f.P, f.Abar, f.Gcum, s32, st));
@@ -356,7 +363,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la,
                                             p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
-                                            f.status, s, st));
+                                            BlockRouting{nullptr, nullptr, nullptr}, f.status, s, st));
     else
         NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
                                               f.o_la, p->w, p->scale_sm, p->eps, nullptr, f.o_nla,
@@ -421,6 +428,7 @@ int natsl_decode_step(const void *q, const void *k, const void *v, const float *
         !out)
         return NATSL_ERR_NULL;
     if (cache_cap <= 0) return NATSL_ERR_SHAPE;
+    if (p->flags & NATSL_BLOCK_ROUTING) return NATSL_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(state) ||
         !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
         return NATSL_ERR_ALIGN;

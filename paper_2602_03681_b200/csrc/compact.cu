@@ -17,7 +17,8 @@ constexpr int kCompactTile = 1024;  // chunks scanned per pass (one per thread)
 __global__ void __launch_bounds__(kCompactThreads)
 route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm_idx,
                      int32_t *__restrict__ sm_chunk_prefix, int32_t *__restrict__ lin_idx,
-                     int32_t *__restrict__ n_lin, int32_t *__restrict__ sm_len, int L, int H) {
+                     int32_t *__restrict__ n_lin, int32_t *__restrict__ sm_len,
+                     int32_t *__restrict__ block_status, int L, int H) {
     __shared__ unsigned long long bits[kCompactTile];
     __shared__ int excl[kCompactTile];
     __shared__ int warp_tot[kCompactThreads / 32];
@@ -82,6 +83,9 @@ route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm
             const unsigned long long wbits = bits[c];
             const unsigned lo = (unsigned)wbits, hi = (unsigned)(wbits >> 32);
             const int pre = base + excl[c];
+            // block-level routing: one decision per chunk, so a word is all zeros or all ones
+            if (block_status && lane == 0 && wbits != 0ull && wbits != ~0ull)
+                atomicMin(block_status, (int)NATSL_ERR_ROUTE);
             const unsigned lt = (1u << lane) - 1u;
             const int nlo = __popc(lo), nsm = nlo + __popc(hi);
             int32_t *sm = sm_idx + (size_t)bh * L + pre;
@@ -135,10 +139,10 @@ gather_kv_kernel(const T *__restrict__ k, const T *__restrict__ v, const int32_t
 }  // namespace
 
 cudaError_t launch_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk_prefix,
-                                 int32_t *lin_idx, int32_t *n_lin, int32_t *sm_len, int B, int L,
-                                 int H, cudaStream_t st) {
+                                 int32_t *lin_idx, int32_t *n_lin, int32_t *sm_len,
+                                 int32_t *block_status, int B, int L, int H, cudaStream_t st) {
     route_compact_kernel<<<B * H, kCompactThreads, 0, st>>>(route, sm_idx, sm_chunk_prefix, lin_idx,
-                                                            n_lin, sm_len, L, H);
+                                                            n_lin, sm_len, block_status, L, H);
     count_launch();
     return cudaGetLastError();
 }

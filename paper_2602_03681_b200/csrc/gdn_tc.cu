@@ -186,7 +186,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         if (!solver) {
             const size_t t = ((size_t)b * L + tok0 + i) * H + h;
             float G = g[t];
-            const float btv = route[t] ? 0.f : beta[t];
+            const float btv = route && route[t] ? 0.f : beta[t];   // route == nullptr: beta~ = beta
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const float y = __shfl_up_sync(0xffffffffu, G, o);
@@ -519,7 +519,7 @@ struct ScanMisc {
 };
 static_assert(sizeof(ScanMisc) <= kScanMisc, "misc page too small");
 
-template <int D>
+template <int D, bool kBlock>      // kBlock: block-level routing (softmax blocks are not committed)
 __global__ void __launch_bounds__(kScanThreads, 1)
 gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                    const __grid_constant__ CUtensorMap map_qh,
@@ -527,8 +527,8 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                    const __grid_constant__ CUtensorMap map_ph, const float *__restrict__ Ut,
                    const float *__restrict__ Gd, float scale_la,
                    const float *__restrict__ state_in, float *__restrict__ state_out,
-                   float *__restrict__ o_la, GdnTcExport ex, ScanSegments sg, int32_t *status, int L,
-                   int H) {
+                   float *__restrict__ o_la, GdnTcExport ex, ScanSegments sg,
+                   const uint8_t *__restrict__ block_route, int32_t *status, int L, int H) {
     using SL = ScanLayout<D>;
     constexpr int KB = SL::KB;
     constexpr int kHalfCols = D / 2;                       // state columns per thread
@@ -692,6 +692,11 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             const int s = c % kScanStages;
             const float *e1 = reinterpret_cast<const float *>(smem + SL::oG + (c % kDecaySlots) * SL::kG);
             const float *e2 = e1 + 64;
+            // Block-level routing: the delta rule runs over every block, but a softmax block's
+            // update is not committed -- its state increment is multiplied by zero, so that the
+            // state only decays across it (Section 4.3, the decay-always equation).
+            const float commit =
+                kBlock && block_route[((size_t)b * L + (size_t)(c0 + c) * 64) * H + h] ? 0.f : 1.f;
             ok = mbar_wait(&ms.full[s], (c / kScanStages) & 1, abort_flag);
             if (!ok) break;
             if (c > 0) {                                   // S_c = gamma_C S_{c-1} + dS_{c-1}
@@ -762,7 +767,9 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
 #pragma unroll
                 for (int x = 0; x < 16; ++x) {
                     pk[x] = pack_half2(u[2 * x], u[2 * x + 1]);
-                    pk[16 + x] = pack_half2(u[2 * x] * e2[tk0 + 2 * x], u[2 * x + 1] * e2[tk0 + 2 * x + 1]);
+                    const float f0 = kBlock ? commit * e2[tk0 + 2 * x] : e2[tk0 + 2 * x];
+                    const float f1 = kBlock ? commit * e2[tk0 + 2 * x + 1] : e2[tk0 + 2 * x + 1];
+                    pk[16 + x] = pack_half2(u[2 * x] * f0, u[2 * x + 1] * f1);
                 }
                 tmem_st32(tmem + SL::cWS + tk0 + lane_base, pk);   // over this thread's own W S columns
                 tmem_wait_st();
@@ -909,7 +916,8 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
 template <int D>
 static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *state_in,
                                 float *state_out, float *o_la, const GdnTcExport &ex,
-                                const ScanSegments &sg, int32_t *status, Shape s, cudaStream_t st) {
+                                const ScanSegments &sg, const uint8_t *block_route, int32_t *status,
+                                Shape s, cudaStream_t st) {
     const int NC = s.L / kC;
     const uint64_t BH = (uint64_t)s.B * s.H;
     CUtensorMap mwt, mqh, mkh, mph;
@@ -918,13 +926,14 @@ static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *
         !tch::make_map_2d(&mkh, ws.Kh, BH * s.L, D, 64) ||
         !tch::make_map_2d(&mph, ws.Ph, BH * NC * 64, 64, 64))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(gdn_scan_tc_kernel<D>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+    auto kernel = block_route ? gdn_scan_tc_kernel<D, true> : gdn_scan_tc_kernel<D, false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          ScanLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
     const int ctas = s.B * s.H * (sg.mode == 0 ? 1 : sg.nseg) * (sg.mode == 1 ? 2 : 1);
-    gdn_scan_tc_kernel<D><<<ctas, kScanThreads, ScanLayout<D>::kTotal, st>>>(
-        mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, o_la, ex, sg, status, s.L, s.H);
+    kernel<<<ctas, kScanThreads, ScanLayout<D>::kTotal, st>>>(
+        mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, o_la, ex, sg, block_route, status,
+        s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -939,9 +948,11 @@ cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, c
 
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
                                float *state_out, float *o_la, const GdnTcExport &ex,
-                               const ScanSegments &sg, int32_t *status, Shape s, cudaStream_t st) {
-    if (s.d == 128) return scan_tc_impl<128>(ws, scale_la, state_in, state_out, o_la, ex, sg, status, s, st);
-    return scan_tc_impl<64>(ws, scale_la, state_in, state_out, o_la, ex, sg, status, s, st);
+                               const ScanSegments &sg, const uint8_t *block_route, int32_t *status,
+                               Shape s, cudaStream_t st) {
+    if (s.d == 128)
+        return scan_tc_impl<128>(ws, scale_la, state_in, state_out, o_la, ex, sg, block_route, status, s, st);
+    return scan_tc_impl<64>(ws, scale_la, state_in, state_out, o_la, ex, sg, block_route, status, s, st);
 }
 
 }  // namespace natsl

@@ -18,10 +18,18 @@ struct Shape {
     bool bf16;
 };
 
-// compact.cu
+// Block-level routing (Section 4.1: one decision per block of C tokens, and both operations see
+// the query's own block): the route bytes [B,L,H] and the layer's K and V, from which the softmax
+// kernel reads the own block of a query in a linear block.  route == nullptr: token-level routing.
+struct BlockRouting {
+    const uint8_t *route;
+    const void *k, *v;
+};
+
+// compact.cu  (block_status: where a route that changes inside a chunk is reported, or nullptr)
 cudaError_t launch_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk_prefix,
-                                 int32_t *lin_idx, int32_t *n_lin, int32_t *sm_len, int B, int L,
-                                 int H, cudaStream_t st);
+                                 int32_t *lin_idx, int32_t *n_lin, int32_t *sm_len,
+                                 int32_t *block_status, int B, int L, int H, cudaStream_t st);
 cudaError_t launch_gather_kv(const void *k, const void *v, const int32_t *sm_idx,
                              const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, int32_t cap,
                              int32_t *status, Shape s, cudaStream_t st);
@@ -52,8 +60,8 @@ cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const voi
                                       int32_t capv, const int32_t *sm_idx,
                                       const int32_t *sm_chunk_prefix, const float *o_la,
                                       const float *w, float scale_sm, float eps, void *out,
-                                      float *o_nla, float *lse, int32_t *status, Shape s,
-                                      cudaStream_t st);
+                                      float *o_nla, float *lse, BlockRouting br, int32_t *status,
+                                      Shape s, cudaStream_t st);
 
 // softmax_bwd_tc.cu -- tensor-core backward of the softmax branch (bf16 storage).  Qh is scratch
 // for the fp16 copy of q [B,H,L,d]; dO16 the fp16 branch-output gradient [B,H,L,d]; k16, v16 the
@@ -102,7 +110,8 @@ struct ScanSegments {
 };
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
                                float *state_out, float *o_la, const GdnTcExport &ex,
-                               const ScanSegments &sg, int32_t *status, Shape s, cudaStream_t st);
+                               const ScanSegments &sg, const uint8_t *block_route, int32_t *status,
+                               Shape s, cudaStream_t st);
 cudaError_t launch_scan_combine(const float *state_in, const ScanSegments &sg, Shape s, cudaStream_t st);
 
 // bwd_simt.cu -- fp32 CUDA-core backward

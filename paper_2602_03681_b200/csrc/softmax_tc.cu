@@ -54,7 +54,7 @@ struct Misc {                    // lives in the last kMiscBytes of the CTA's sh
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc page too small");
 
-template <int D>
+template <int D, bool kBlock>      // kBlock: block-level routing (own-block tiles after the retained ones)
 __global__ void __launch_bounds__(kThreadsTc)
 softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                           const __grid_constant__ CUtensorMap map_k,
@@ -62,7 +62,9 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                           const __grid_constant__ CUtensorMap map_ola,    // o_la  [B,L,H,D] fp32, box 128 x 32
                           const __grid_constant__ CUtensorMap map_onla,   // o_nla (same geometry), if has_onla
                           const __grid_constant__ CUtensorMap map_out,    // out [B,L,H,D] bf16, box 128 x 64, if has_out
-                          int cap, int capv, const int32_t *__restrict__ sm_idx,
+                          const __grid_constant__ CUtensorMap map_kd,     // the layer's k, v [B,L,H,D] bf16, box
+                          const __grid_constant__ CUtensorMap map_vd,     //   64 x 64: own-block tiles (block routing)
+                          const uint8_t *__restrict__ block_route, int cap, int capv, const int32_t *__restrict__ sm_idx,
                           const int32_t *__restrict__ sm_chunk_prefix,
                           const float *__restrict__ o_la, const float *__restrict__ w,
                           float scale_sm, float eps, int has_out, int has_onla,
@@ -81,6 +83,20 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     const int n_full = min(pre[c0], cap);             // retained tokens before the CTA's chunks
     const int n_end = min(pre[c1], cap);              // ... up to the end of the CTA's chunks
     const int T = (n_end + kBN - 1) / kBN;
+    // Block-level routing (Section 4.1, intra-chunk correlations of both operations): a query in a
+    // linear block also reads the causal part of its own block, whose tokens are not among the
+    // retained ones.  Each linear block of the CTA's two adds one tile, taken from the layer's
+    // own k and v after the retained tiles (the softmax threads turn its V tile into fp16 in
+    // place, exactly as the gather does for the retained rows).
+    int nx = 0, xc0 = 0;                                // number of own-block tiles; block of the first
+    if (kBlock)
+        for (int e = 0; e < c1 - c0; ++e)
+            if (block_route[((size_t)b * L + (size_t)(c0 + e) * kC) * H + h] == 0) {
+                if (nx == 0) xc0 = e;
+                ++nx;
+            }
+    const int T2 = kBlock ? T + nx : T;
+    auto own_block = [&](int t) { return t == T ? xc0 : 1; };   // block (0 or 1) of own-block tile t >= T
 
     if ((smem_u32(smem) & 1023u) != 0) {              // operand tiles need 1024-byte alignment
         if (tid == 0) atomicMin(status, (int)NATSL_ERR_CUDA);
@@ -117,22 +133,24 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         if (lane == 0) {
             int nk = 0, nv = 0;                 // K / V tiles requested so far
             bool ok = true;
-            if (T > 0) {                        // nothing is loaded for a tile that sees no retained key
+            if (T2 > 0) {                       // nothing is loaded for a tile that sees no key at all
                 prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
                 mbar_arrive_expect_tx(&ms.barQ, SL::kQBytes);
                 for (int kb = 0; kb < KB; ++kb)
                     tma_load_4d(smem + SL::oQ + kb * kBM * 128, &map_q, &ms.barQ, kb * 64, h, p * kBM, b);
                 // K and V tiles have their own rings: a K tile is free as soon as its Q K^T has run
                 // (early), a V tile only after its P V; K(u) is therefore requested before V(u-1).
-                for (int u = 0; u <= T && ok; ++u) {
-                    if (u < T) {
+                for (int u = 0; u <= T2 && ok; ++u) {
+                    if (u < T2) {
                         const int s = u % kStages;
                         ok = mbar_wait(&ms.emptyK[s], ((u / kStages) & 1) ^ 1, abort_flag);
                         if (!ok) break;
                         mbar_arrive_expect_tx(&ms.fullK[s], SL::kKStage);
-                        for (int kb = 0; kb < KB; ++kb)
-                            tma_load_2d(smem + SL::oK + s * SL::kKStage + kb * kBN * 128, &map_k,
-                                        &ms.fullK[s], kb * 64, bh * cap + u * kBN);
+                        for (int kb = 0; kb < KB; ++kb) {
+                            uint8_t *dst = smem + SL::oK + s * SL::kKStage + kb * kBN * 128;
+                            if (!kBlock || u < T) tma_load_2d(dst, &map_k, &ms.fullK[s], kb * 64, bh * cap + u * kBN);
+                            else tma_load_4d(dst, &map_kd, &ms.fullK[s], kb * 64, h, (c0 + own_block(u)) * kC, b);
+                        }
                         nk = u + 1;
                     }
                     if (u >= 1) {
@@ -140,14 +158,16 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                         ok = mbar_wait(&ms.emptyV[s], ((t / kStages) & 1) ^ 1, abort_flag);
                         if (!ok) break;
                         mbar_arrive_expect_tx(&ms.fullV[s], SL::kVStage);
-                        for (int kb = 0; kb < KB; ++kb)
-                            tma_load_2d(smem + SL::oV + s * SL::kVStage + kb * kBN * 128, &map_v,
-                                        &ms.fullV[s], kb * 64, bh * capv + t * kBN);
+                        for (int kb = 0; kb < KB; ++kb) {
+                            uint8_t *dst = smem + SL::oV + s * SL::kVStage + kb * kBN * 128;
+                            if (!kBlock || t < T) tma_load_2d(dst, &map_v, &ms.fullV[s], kb * 64, bh * capv + t * kBN);
+                            else tma_load_4d(dst, &map_vd, &ms.fullV[s], kb * 64, h, (c0 + own_block(t)) * kC, b);
+                        }
                         nv = t + 1;
                     }
                 }
                 // the Q tile and the K ring are free once the last Q K^T has run
-                if (ok) ok = mbar_wait(&ms.emptyK[(T - 1) % kStages], ((T - 1) / kStages) & 1, abort_flag);
+                if (ok) ok = mbar_wait(&ms.emptyK[(T2 - 1) % kStages], ((T2 - 1) / kStages) & 1, abort_flag);
             }
             bool e_issued = false;
             if (ok) {                           // the epilogue's rows of o_la, D/32 boxes of 128 x 32
@@ -167,7 +187,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         }
     } else if (warp == 4) {
         // ------------------------------ MMA issuer ------------------------------
-        if (lane == 0 && T > 0) {
+        if (lane == 0 && T2 > 0) {
             constexpr uint32_t idesc_qk = make_idesc(kFmtBF16, kBM, kBN, false, false);
             constexpr uint32_t idesc_pv = make_idesc(kFmtF16, kBM, D, false, true);
             const uint32_t aQ = smem_u32(smem + SL::oQ), aP = smem_u32(smem + SL::oP);
@@ -188,8 +208,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 tc_fence_after_sync();
                 issue_qk(0);
             }
-            for (int t = 0; ok && t < T; ++t) {
-                if (t + 1 < T) {
+            for (int t = 0; ok && t < T2; ++t) {
+                if (t + 1 < T2) {
                     ok = mbar_wait(&ms.fullK[(t + 1) % kStages], ((t + 1) / kStages) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after_sync();
@@ -227,12 +247,12 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 for (int x = 0; x < D * 4 / 128; ++x) prefetch_l2(o_la + tok * D + x * 32);
             }
         };
-        if (T <= 1) prefetch_o_la();
+        if (T2 <= 1) prefetch_o_la();
         // The compacted keys are in position order, so row i sees exactly the first `cnt` of them:
         // all n_full earlier ones plus those of the CTA's own chunks at positions <= i.
         int cnt = n_full;
         for (int kq = 0; kq < n_end - n_full; ++kq) cnt += ms.pos[kq] <= i_abs ? 1 : 0;
-        for (int t = 0; t < T; ++t) {
+        for (int t = 0; t < T2; ++t) {
             ok = mbar_wait(&ms.barS[t & 1], (t >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
@@ -244,7 +264,12 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll
             for (int c = 0; c < kBN; ++c) x[c] = __uint_as_float(sv[c >> 5][c & 31]) * sl2;
             const int j0 = t * kBN;
-            if (!__all_sync(0xffffffffu, j0 + kBN <= cnt)) {   // some row of the warp is cut off here
+            if (kBlock && t >= T) {
+                // own-block tile: row r sees keys 0 .. r % 64 if it is in that block
+                const int vis = (r >> 6) == own_block(t) ? (r & 63) + 1 : 0;
+#pragma unroll
+                for (int c = 0; c < kBN; ++c) x[c] = c < vis ? x[c] : -INFINITY;
+            } else if (!__all_sync(0xffffffffu, j0 + kBN <= cnt)) {   // some row of the warp is cut off here
 #pragma unroll
                 for (int c = 0; c < kBN; ++c) x[c] = j0 + c < cnt ? x[c] : -INFINITY;
             }
@@ -294,13 +319,25 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 u.w = pack_half2(x[8 * pc + 6], x[8 * pc + 7]);
                 *reinterpret_cast<uint4 *>(prow + sw128_offset(r, pc)) = u;
             }
+            if (kBlock && t >= T) {   // own-block tile: its V rows arrived as bf16; fp16 in place (exact)
+                ok = mbar_wait(&ms.fullV[t % kStages], (t / kStages) & 1, abort_flag);
+                if (!ok) break;
+                uint4 *vt = reinterpret_cast<uint4 *>(smem + SL::oV + (t % kStages) * SL::kVStage);
+                for (int i = r; i < SL::kVStage / 16; i += kSoftmaxThreads) {
+                    const uint4 a = vt[i];
+                    auto cv = [](uint32_t wd) {
+                        return pack_half2(__uint_as_float(wd << 16), __uint_as_float(wd & 0xffff0000u));
+                    };
+                    vt[i] = make_uint4(cv(a.x), cv(a.y), cv(a.z), cv(a.w));
+                }
+            }
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&ms.barP);
-            if (t == 0 && T > 1) prefetch_o_la();
+            if (t == 0 && T2 > 1) prefetch_o_la();
         }
-        if (ok && T > 0) {
-            ok = mbar_wait(&ms.barO, (T - 1) & 1, abort_flag);
+        if (ok && T2 > 0) {
+            ok = mbar_wait(&ms.barO, (T2 - 1) & 1, abort_flag);
             tc_fence_after_sync();
         }
         if (ok) ok = mbar_wait(&ms.barE, 0, abort_flag);        // the tile's rows of o_la have landed
@@ -312,7 +349,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t ov[32];
-                if (T > 0) {
+                if (T2 > 0) {
                     tmem_ld32(tO + lane_base + cb * 32, ov);
                     tmem_wait_ld();
                 } else {
@@ -335,7 +372,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t ov[32];
-                if (T > 0) {
+                if (T2 > 0) {
                     tmem_ld32(tO + lane_base + cb * 32, ov);
                     tmem_wait_ld();
                 } else {
@@ -450,10 +487,10 @@ template <int D>
 static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *v16, int32_t cap,
                                    int32_t capv, const int32_t *sm_idx, const int32_t *pre,
                                    const float *o_la, const float *w, float scale_sm, float eps,
-                                   void *out, float *o_nla, float *lse, int32_t *status, Shape s,
-                                   cudaStream_t st) {
+                                   void *out, float *o_nla, float *lse, BlockRouting br,
+                                   int32_t *status, Shape s, cudaStream_t st) {
     using SL = SmLayout<D>;
-    CUtensorMap mq, mk, mv, mola, monla, mout;
+    CUtensorMap mq, mk, mv, mola, monla, mout, mkd, mvd;
     if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, kBM) ||
         !tch::make_map_2d(&mk, k_sm, (uint64_t)s.B * s.H * cap, D, kBN) ||
         !tch::make_map_2d(&mv, v16, (uint64_t)s.B * s.H * capv, D, kBN) ||
@@ -463,13 +500,18 @@ static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *
     mout = mq;
     if (o_nla && !tch::make_map_blhd_f32(&monla, o_nla, s.B, s.L, s.H, D, kBM)) return cudaErrorInvalidValue;
     if (out && !tch::make_map_blhd(&mout, out, s.B, s.L, s.H, D, kBM)) return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(softmax_combine_tc_kernel<D>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal);
+    mkd = mq;
+    mvd = mq;
+    if (br.route && (!tch::make_map_blhd(&mkd, br.k, s.B, s.L, s.H, D, kBN) ||
+                     !tch::make_map_blhd(&mvd, br.v, s.B, s.L, s.H, D, kBN)))
+        return cudaErrorInvalidValue;
+    auto kernel = br.route ? softmax_combine_tc_kernel<D, true> : softmax_combine_tc_kernel<D, false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal);
     if (e != cudaSuccess) return e;
     dim3 grid((s.L + kBM - 1) / kBM, s.B * s.H);
-    softmax_combine_tc_kernel<D><<<grid, kThreadsTc, SL::kTotal, st>>>(
-        mq, mk, mv, mola, monla, mout, cap, capv, sm_idx, pre, o_la, w, scale_sm, eps, out ? 1 : 0,
-        o_nla ? 1 : 0, lse, status, s.L, s.H);
+    kernel<<<grid, kThreadsTc, SL::kTotal, st>>>(
+        mq, mk, mv, mola, monla, mout, mkd, mvd, br.route, cap, capv, sm_idx, pre, o_la, w, scale_sm, eps,
+        out ? 1 : 0, o_nla ? 1 : 0, lse, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -478,13 +520,13 @@ cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const voi
                                       int32_t capv, const int32_t *sm_idx,
                                       const int32_t *sm_chunk_prefix, const float *o_la,
                                       const float *w, float scale_sm, float eps, void *out,
-                                      float *o_nla, float *lse, int32_t *status, Shape s,
-                                      cudaStream_t st) {
+                                      float *o_nla, float *lse, BlockRouting br, int32_t *status,
+                                      Shape s, cudaStream_t st) {
     if (s.d == 128)
         return softmax_tc_impl<128>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la, w,
-                                    scale_sm, eps, out, o_nla, lse, status, s, st);
+                                    scale_sm, eps, out, o_nla, lse, br, status, s, st);
     return softmax_tc_impl<64>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la, w, scale_sm,
-                               eps, out, o_nla, lse, status, s, st);
+                               eps, out, o_nla, lse, br, status, s, st);
 }
 
 template <int D>

@@ -114,6 +114,17 @@ def route_runs(seed, shape, p, mean_run=8.0):
     return r
 
 
+def route_blocks(seed, shape, p, R=64, force_first=True):
+    """One Bernoulli(p) decision per block of R tokens and head (block-level routing: the paper's
+    chunk size equals the GDN chunk size), repeated over the block's tokens.  shape = (B, L, H)."""
+    B, L, H = shape
+    assert L % R == 0
+    r = (_rng(seed, "route").random((B, L // R, H)) < p).astype(np.uint8)
+    if force_first and L > 0:
+        r[:, 0, :] = 1
+    return np.repeat(r, R, axis=1)
+
+
 def make_layer_inputs(wl: Workload, *, B=None, H=None, L=None, route=None):
     """Inputs of one forward (and backward) call.  B/H/L override the workload's sizes to get
     smaller cases with the same distributions.  Returns a dict of numpy arrays:

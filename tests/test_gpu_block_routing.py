@@ -1,0 +1,105 @@
+"""Parity of the block-routed forward (Section 4.1: one routing decision per block of 64 tokens,
+both operations read the query's own block) with the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_03681_b200 import inputs
+from test_gpu_parity import check_fwd, dev, rel_err, run_fwd, tdtype
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+
+
+def block_inputs(wl, B, H, L, p, seed=0):
+    route = inputs.route_blocks(wl.seed + seed, (B, L, H), p)
+    return inputs.make_layer_inputs(wl, B=B, H=H, L=L, route=route)
+
+
+def oracle_block(wl, x, state_in=None, **kw):
+    return oracle.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"],
+                             scale_la=wl.scale_la, scale_sm=wl.scale_sm, state_in=state_in, block=64,
+                             **kw)
+
+
+@pytest.mark.parametrize("name,B,H,L,p,flags", [
+    ("cfg4_bf16_train", 1, 2, 512, 0.3, 0),        # d = 64
+    ("cfg1_bf16_prefill", 1, 2, 576, 0.3, 0),      # d = 128, ragged last query tile (9 blocks)
+    ("cfg1_bf16_prefill", 2, 3, 1024, 0.15, 0),
+    ("cfg1_bf16_prefill", 1, 1, 2048, 0.2, 0),     # few (batch, head) pairs: segmented scan
+    ("cfg1_bf16_prefill", 1, 1, 2048, 0.2, 2),     # ... and the same in one pass
+    ("cfg4_bf16_train", 1, 2, 64, 0.0, 0),         # a single block
+])
+def test_block_routed_forward_matches_oracle(name, B, H, L, p, flags):
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS[name]
+    x = block_inputs(wl, B, H, L, p)
+    rng = np.random.default_rng(7)
+    S0 = (0.1 * rng.standard_normal((B, H, wl.d, wl.d))).astype(np.float32)
+    ref = oracle_block(wl, x, state_in=S0.astype(np.float64))
+    got = run_fwd(wl, x, state_in=S0, flags=binding.BLOCK_ROUTING | flags)
+    check_fwd(wl, got, ref, TOL_BF16)
+    # the mode is not the token-level one: with the same inputs the two differ visibly
+    tok = run_fwd(wl, x, state_in=S0, flags=flags)
+    assert rel_err(tok["out"], ref["out"]) > 10 * TOL_BF16 or x["route"].all()
+
+
+@pytest.mark.parametrize("p", [0.0, 1.0])
+def test_block_routing_all_linear_and_all_softmax(p):
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    x = block_inputs(wl, 1, 2, 384, 0.5)
+    x["route"][:] = int(p)
+    ref = oracle_block(wl, x)
+    got = run_fwd(wl, x, flags=binding.BLOCK_ROUTING)
+    check_fwd(wl, got, ref, TOL_BF16)
+
+
+def test_block_routing_prefill_hands_over_the_kept_cache_and_state():
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    B, H, L = 1, 2, 512
+    x = block_inputs(wl, B, H, L, 0.4)
+    ref = oracle_block(wl, x, want_cache=True)
+    dt = tdtype(wl)
+    res = binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]),
+                             dev(x["beta"]), dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la,
+                             scale_sm=wl.scale_sm, want=("state_out", "cache"),
+                             flags=binding.BLOCK_ROUTING)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(res["ws"]) == 0
+    k_sm, v_sm, sm_len = res["k_sm"], res["v_sm"], res["sm_len"]
+    n = sm_len.cpu().numpy()
+    assert np.array_equal(n, ref["n_sm"])                  # integer work: exact
+    for b in range(B):
+        for h in range(H):
+            assert np.array_equal(k_sm[b, h, :n[b, h]].float().cpu().numpy(), ref["k_sm"][b, h, :n[b, h]])
+            assert np.array_equal(v_sm[b, h, :n[b, h]].float().cpu().numpy(), ref["v_sm"][b, h, :n[b, h]])
+    assert rel_err(res["state_out"].cpu().numpy(), ref["state_out"]) <= TOL_BF16
+
+
+def test_block_routing_reports_a_route_that_changes_inside_a_block():
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    x = block_inputs(wl, 1, 2, 256, 0.5)
+    x["route"][0, 70, 1] ^= 1
+    dt = tdtype(wl)
+    res = binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]),
+                             dev(x["beta"]), dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la,
+                             scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(res["ws"]) == binding.ERR_ROUTE
+
+
+def test_block_routing_off_the_tensor_core_path_is_refused():
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    x = block_inputs(wl, 1, 1, 128, 0.5)
+    dt = tdtype(wl)
+    with pytest.raises(binding.NatslError) as ei:
+        binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]),
+                           dev(x["beta"]), dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la,
+                           scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING | binding.FORCE_SIMT)
+    assert ei.value.status == binding.ERR_UNSUPPORTED
