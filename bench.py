@@ -52,6 +52,19 @@ def useful_flops(route: np.ndarray, d: int, C: int = 64):
     return {"gdn_prepare": prepare, "gdn_scan": scan, "softmax_combine": softmax}
 
 
+def useful_flops_block(route: np.ndarray, d: int, C: int = 64):
+    """The same count under block-level routing: every block runs the delta rule with all C of its
+    tokens, and a query in a linear block also reads the causal part of its own block."""
+    B, L, H = route.shape
+    r = route.astype(np.int64)
+    nblk = B * (L // C) * H
+    prepare = float(nblk * (6 * C * C * d + 2 * C * C * d))
+    scan = float(nblk * (2 * d * d * 3 * C + 2 * C * C * d))
+    own = (np.arange(L) % C + 1)[None, :, None] * (1 - r)
+    softmax = float(4 * d * (np.cumsum(r, axis=1) + own).sum())
+    return {"gdn_prepare": prepare, "gdn_scan": scan, "softmax_combine": softmax}
+
+
 def min_hbm_bytes_fwd(wl, B):
     """q, k, v read once + out written once + the small per-token tensors."""
     e = 2 if wl.dtype == "bf16" else 4
@@ -404,9 +417,12 @@ def bench_other_workloads(peaks):
     from paper_2602_03681_b200 import binding
     res = {}
     dt = torch.bfloat16
-    for name, ops in (("cfg2_bf16_long_prefill", ("fwd",)), ("cfg4_bf16_train", ("fwd", "bwd"))):
-        wl = inputs.WORKLOADS[name]
-        x = inputs.make_layer_inputs(wl)
+    for name, ops in (("cfg2_bf16_long_prefill", ("fwd",)), ("cfg4_bf16_train", ("fwd", "bwd")),
+                      ("cfg1_bf16_prefill/block_routing", ("fwd",))):
+        block = name.endswith("/block_routing")          # the same shapes, one route per 64 tokens
+        wl = inputs.WORKLOADS[name.split("/")[0]]
+        x = inputs.make_layer_inputs(
+            wl, route=inputs.route_blocks(wl.seed, (wl.B, wl.L, wl.H), wl.p_softmax) if block else None)
         d = {m: torch.from_numpy(x[m]).cuda() for m in ("g", "beta", "route", "w")}
         for m in ("q", "k", "v", "dout"):
             d[m] = torch.from_numpy(x[m]).cuda().to(dt)
@@ -416,6 +432,7 @@ def bench_other_workloads(peaks):
             if op == "fwd":
                 ws["fwd"] = binding.hybrid_fwd(d["q"], d["k"], d["v"], d["g"], d["beta"], d["route"],
                                                d["w"], scale_la=wl.scale_la, scale_sm=wl.scale_sm,
+                                               flags=binding.BLOCK_ROUTING if block else 0,
                                                ws=ws["fwd"])["ws"]
             else:
                 ws["bwd"] = binding.hybrid_bwd(d["q"], d["k"], d["v"], d["g"], d["beta"], d["route"],
@@ -435,7 +452,7 @@ def bench_other_workloads(peaks):
                 torch.cuda.synchronize()
                 best = min(best, e0.elapsed_time(e1))
             ms[op] = best
-        fl = sum(useful_flops(x["route"], wl.d, wl.C).values())
+        fl = sum((useful_flops_block if block else useful_flops)(x["route"], wl.d, wl.C).values())
         total_ms = sum(ms.values())
         entry = {"ms": ms, "tokens_per_s": wl.B * wl.L / (total_ms * 1e-3),
                  "useful_fwd_gflop": fl / 1e9,

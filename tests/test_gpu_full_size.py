@@ -21,6 +21,18 @@ def test_fwd_full_size(name):
     check_fwd(wl, got, ref, TOL[wl.dtype])
 
 
+def test_fwd_full_size_block_routing():
+    """The prefill workload's shapes with one routing decision per block of 64 tokens
+    (Section 4.1), every element against the block-mode oracle."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    route = inputs.route_blocks(wl.seed, (wl.B, wl.L, wl.H), wl.p_softmax)
+    x = inputs.make_layer_inputs(wl, route=route)
+    got = run_fwd(wl, x, flags=binding.BLOCK_ROUTING)
+    ref = run_oracle(wl, x, block=64)
+    check_fwd(wl, got, ref, TOL[wl.dtype])
+
+
 def test_fwd_bwd_full_size_training_workload():
     wl = inputs.WORKLOADS["cfg4_bf16_train"]
     x = inputs.make_layer_inputs(wl)
