@@ -146,6 +146,8 @@ def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5
 def decode_step(q, k, v, g, beta, route, w, state, k_cache, v_cache, cache_len, *, scale_la,
                 scale_sm, eps=1e-5):
     """One generation step; `state`, `k_cache`, `v_cache`, `cache_len` are updated IN PLACE.
+    route 0 / 1: linear / softmax token; 2: token of a block whose decision is still open (folded
+    into the state and appended to the cache; see block_end).
 
     q,k,v [B,H,d]; g,beta,route [B,H]; w [B,H,2] or None; state [B,H,d,d] float64;
     k_cache,v_cache [B,H,cap,d] float64; cache_len [B,H] int32.
@@ -169,3 +171,18 @@ def decode_step(q, k, v, g, beta, route, w, state, k_cache, v_cache, cache_len, 
     if rc != 0:
         raise RuntimeError(f"natsl_oracle_decode_step failed ({rc})")
     return dict(out=out, o_la=o_la, o_nla=o_nla)
+
+
+def block_end(route_block, g_block, state, state_start, cache_len, R):
+    """End of a block of R tokens decoded with route 2 (Section 4.1, roll-back of the operation
+    that was not chosen).  `state`, `state_start`, `cache_len` are updated IN PLACE."""
+    for a in (state, state_start):
+        assert a.dtype == np.float64 and a.flags.c_contiguous
+    assert cache_len.dtype == np.int32 and cache_len.flags.c_contiguous
+    route_block = np.ascontiguousarray(route_block, dtype=np.uint8)
+    g_block = _d(g_block)
+    B, H, d, _ = state.shape
+    rc = _load().natsl_oracle_block_end(_p(route_block, _u8p), _p(g_block), B, H, d, int(R),
+                                        _p(state), _p(state_start), _p(cache_len, _i32p))
+    if rc != 0:
+        raise RuntimeError(f"natsl_oracle_block_end failed ({rc})")

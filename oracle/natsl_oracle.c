@@ -286,8 +286,11 @@ int natsl_oracle_hybrid_fwd_block(const double *q, const double *k, const double
 }
 
 /* ---------------------------------------------------------------------------
- * One decode step (Section 4.1, per-token generation, with the route of the new
- * token known, so nothing has to be rolled back).
+ * One decode step (Section 4.1, per-token generation).  route 0 / 1: the route of the new
+ * token is known (token-level routing), so nothing has to be rolled back.  route 2: the token
+ * belongs to a block whose decision is still open -- it is folded into the state AND appended
+ * to the retained K/V (the pseudo-update of both hidden states); natsl_oracle_block_end undoes
+ * one of the two when the block is complete.
  *   q,k,v [B,H,d]; g,beta [B,H]; route [B,H]; w [B,H,2] or NULL
  *   state [B,H,d,d] in place; k_cache,v_cache [B,H,cap,d]; cache_len [B,H] in place
  * Returns -3 if a sequence would overflow its cache (nothing is modified for it).
@@ -305,11 +308,11 @@ int natsl_oracle_decode_step(const double *q, const double *k, const double *v,
 #pragma omp parallel for schedule(dynamic, 1)
     for (int bh = 0; bh < B * H; ++bh) {
         int n_c = cache_len[bh];
-        if (route[bh] && n_c >= cache_cap) { err = 3; continue; }
+        if (route[bh] != 0 && n_c >= cache_cap) { err = 3; continue; }
         double *logit = (double *)malloc(sizeof(double) * (size_t)(n_c + 2));
         double wn = w ? w[(size_t)bh * 2] : 0.5, wl = w ? w[(size_t)bh * 2 + 1] : 0.5;
         hybrid_token(d, q + (size_t)bh * d, k + (size_t)bh * d, v + (size_t)bh * d, g[bh], beta[bh],
-                     route[bh] == 0, route[bh] != 0, wn, wl, scale_la, scale_sm, eps,
+                     route[bh] != 1, route[bh] != 0, wn, wl, scale_la, scale_sm, eps,
                      state + (size_t)bh * d * d, k_cache + (size_t)bh * cache_cap * d,
                      v_cache + (size_t)bh * cache_cap * d, &n_c, logit,
                      o_la ? o_la + (size_t)bh * d : NULL, o_nla ? o_nla + (size_t)bh * d : NULL,
@@ -318,6 +321,32 @@ int natsl_oracle_decode_step(const double *q, const double *k, const double *v,
         free(logit);
     }
     return err ? -3 : 0;
+}
+
+/* ---------------------------------------------------------------------------
+ * End of a block during generation (Section 4.1: "reroll the hidden states of the operations
+ * that are not selected"): R tokens were decoded with route 2 since the last call.
+ *   route_block [B,H]: the block's decision.  1 (softmax): the linear state is reset to its value
+ *       at the start of the block, state_start, times the block's decay exp(g_block) (Section 4.3,
+ *       decay-always equation); the appended K/V stay.  0 (linear): the state stays, the block's
+ *       R cache entries are removed.
+ *   state_start [B,H,d,d] is then set to the new state: the start of the next block.
+ * ------------------------------------------------------------------------- */
+int natsl_oracle_block_end(const uint8_t *route_block, const double *g_block, int B, int H, int d,
+                           int R, double *state, double *state_start, int32_t *cache_len)
+{
+    for (int bh = 0; bh < B * H; ++bh) {
+        double *S = state + (size_t)bh * d * d, *S0 = state_start + (size_t)bh * d * d;
+        if (route_block[bh]) {
+            double decay = exp(g_block[bh]);
+            for (int a = 0; a < d * d; ++a) S[a] = decay * S0[a];
+        } else {
+            if (cache_len[bh] < R) return -1;
+            cache_len[bh] -= R;
+        }
+        memcpy(S0, S, sizeof(double) * (size_t)d * d);
+    }
+    return 0;
 }
 
 /* ---------------------------------------------------------------------------

@@ -582,3 +582,32 @@ def test_block_mode_rejects_route_that_changes_inside_a_block():
     x["route"][0, 5, 0] = 1
     with pytest.raises(ValueError):
         fwd(x, block=4)
+
+
+def test_block_mode_generation_protocol_equals_the_forward():
+    """Decoding token by token with the decision open (route 2) and rolling back at each block's
+    end gives what the block-mode forward gives: outputs, final state, kept K/V."""
+    B, L, H, d, R = 2, 20, 2, 6, 4
+    x = rand_inputs(B, L, H, d, seed=35)
+    x["route"] = _block_route(B, L, H, R, 0.5, seed=6)
+    S0 = RNG.standard_normal((B, H, d, d))
+    ref = fwd(x, block=R, state_in=S0, want_cache=True)
+    state, start = S0.copy(), S0.copy()
+    kc, vc = np.zeros((B, H, L, d)), np.zeros((B, H, L, d))
+    n = np.zeros((B, H), np.int32)
+    undecided = np.full((B, H), 2, np.uint8)
+    for t in range(L):
+        r = oracle.decode_step(x["q"][:, t], x["k"][:, t], x["v"][:, t], x["g"][:, t], x["beta"][:, t],
+                               undecided, x["w"][:, t], state, kc, vc, n, scale_la=0.5, scale_sm=1.5)
+        np.testing.assert_allclose(r["out"], ref["out"][:, t], rtol=1e-11, atol=1e-14)
+        if (t + 1) % R == 0:
+            blk = slice(t + 1 - R, t + 1)
+            oracle.block_end(x["route"][:, t], x["g"][:, blk].sum(1), state, start, n, R)
+            assert np.array_equal(state, start)
+    np.testing.assert_allclose(state, ref["state_out"], rtol=1e-11, atol=1e-14)
+    assert np.array_equal(n, ref["n_sm"])
+    # a linear block leaves its entries behind the length; the next block overwrites them
+    for b in range(B):
+        for h in range(H):
+            assert np.array_equal(kc[b, h, :n[b, h]], ref["k_sm"][b, h, :n[b, h]])
+            assert np.array_equal(vc[b, h, :n[b, h]], ref["v_sm"][b, h, :n[b, h]])
