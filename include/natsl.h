@@ -54,7 +54,8 @@ typedef enum natsl_status {
     NATSL_ERR_UNSUPPORTED = -8, /* valid request this build does not implement */
     NATSL_ERR_TOO_LARGE = -9,   /* natsl_hybrid_fwd_static: problem needs more than the built-in scratch */
     NATSL_ERR_TIMEOUT = -10,    /* a bounded device-side wait expired (device-detected); kernel drained */
-    NATSL_ERR_ROUTE = -11       /* NATSL_BLOCK_ROUTING: route changes inside a block (device-detected) */
+    NATSL_ERR_ROUTE = -11       /* block-level routing: route changes inside a block, or a block end
+                                   without the block's cache entries (device-detected) */
 } natsl_status;
 
 enum { NATSL_F32 = 0, NATSL_BF16 = 1 };
@@ -83,8 +84,9 @@ enum {
                                     state only if the block is linear (a softmax block leaves the
                                     decay alone).  state_out, k_sm, v_sm, sm_len hold what is kept
                                     after the last block.  A route that changes inside a block is
-                                    reported as NATSL_ERR_ROUTE by natsl_device_status.  Backward
-                                    and decode: NATSL_ERR_UNSUPPORTED with this flag */
+                                    reported as NATSL_ERR_ROUTE by natsl_device_status.  Backward:
+                                    NATSL_ERR_UNSUPPORTED with this flag.  Generation: route 2 in
+                                    natsl_decode_step and natsl_decode_block_end (no flag needed) */
 };
 
 typedef struct natsl_params {
@@ -174,14 +176,18 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                      const natsl_params *p, void *ws, size_t ws_bytes, void *stream);
 
 /*
- * One generation step (Section 4.1, per-token generation; the new token's route is known, so
- * no roll-back is needed): decay the state, apply the delta rule (route 0) or append the
- * token's K/V to the retained cache (route 1), then read both branches and combine.
+ * One generation step (Section 4.1, per-token generation): decay the state, apply the delta
+ * rule (route 0) or append the token's K/V to the retained cache (route 1), then read both
+ * branches and combine.  With routes 0 / 1 the new token's route is known (token-level routing)
+ * and no roll-back is needed.  route 2 is a token of a block whose decision is still open
+ * (block-level routing): it is folded into the state and appended to the cache, so that both
+ * operations see it (the paper's pseudo-update of both hidden states); natsl_decode_block_end
+ * undoes one of the two when the block is complete.
  *   q,k,v [B,H,d] in p->dtype; g,beta [B,H] fp32; route [B,H] u8; p->w [B,H,2] or NULL;
  *   state [B,H,d,d] fp32, updated in place;
  *   k_cache,v_cache [B,H,cache_cap,d] in p->dtype; cache_len [B,H] i32, updated in place;
  *   out [B,H,d] in p->dtype.
- * A sequence whose cache is full and whose token is routed to softmax is left untouched,
+ * A sequence whose cache is full and whose token is to be appended is left untouched,
  * its out row is zero-filled and NATSL_ERR_CACHE_FULL is recorded in the status word at the
  * start of the workspace.  ws must hold natsl_workspace_size(p, NATSL_OP_DECODE) bytes and be
  * zero-filled once before its first use; besides the status word it holds per-head tickets and
@@ -192,6 +198,26 @@ int natsl_decode_step(const void *q, const void *k, const void *v, const float *
                       const float *beta, const uint8_t *route, float *state,
                       void *k_cache, void *v_cache, int32_t *cache_len, int32_t cache_cap,
                       void *out, const natsl_params *p, void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * End of a block during generation under block-level routing (Section 4.1: after observing the
+ * entire chunk, the hidden state of the operation that was not selected is rolled back).
+ * block_len tokens were decoded with route 2 since the previous call (or since the prefill).
+ *   route_block [B,H] u8: the block's decision.  1 (softmax): the linear state is reset to its
+ *       value at the start of the block, state_start, times the block's decay exp(g_block)
+ *       (Section 4.3: the decay is applied on softmax blocks too); the block's K/V stay in the
+ *       cache.  0 (linear): the state stays; the block's block_len cache entries are dropped
+ *       (cache_len -= block_len).
+ *   g_block [B,H] fp32: sum of the g values of the block's tokens.
+ *   state, state_start [B,H,d,d] fp32, device; state_start is then set to the new state, the
+ *       start of the next block.  Before the first block the caller makes it a copy of `state`.
+ *   cache_len [B,H] i32, in place.  A linear block with fewer than block_len entries in its cache
+ *       records NATSL_ERR_ROUTE in the status word (ws: the decode workspace).
+ * Errors: NULL, SHAPE, ALIGN, WORKSPACE, CUDA.
+ */
+int natsl_decode_block_end(const uint8_t *route_block, const float *g_block, float *state,
+                           float *state_start, int32_t *cache_len, int32_t block_len,
+                           const natsl_params *p, void *ws, size_t ws_bytes, void *stream);
 
 /* Synchronises `stream`, returns (and clears) the status word kernels wrote at ws[0]. */
 int natsl_device_status(void *ws, void *stream);

@@ -24,7 +24,7 @@ ERR_UNSUPPORTED = -8
 ERR_ROUTE = -11
 
 EXPORTS = ["natsl_workspace_size", "natsl_route_compact", "natsl_hybrid_fwd", "natsl_hybrid_bwd",
-           "natsl_decode_step", "natsl_device_status", "natsl_hybrid_fwd_static",
+           "natsl_decode_step", "natsl_decode_block_end", "natsl_device_status", "natsl_hybrid_fwd_static",
            "natsl_stage_name", "natsl_launch_count", "natsl_strerror"]
 ERR_TOO_LARGE = -9
 STATIC_WS_BYTES = 32 << 20
@@ -183,6 +183,14 @@ def natsl_decode_step(q, k, v, g, beta, route, state, k_cache, v_cache, cache_le
                                    _ptr(state), _ptr(k_cache), _ptr(v_cache), _ptr(cache_len),
                                    ctypes.c_int32(cap), _ptr(out), ctypes.byref(p), _ptr(ws),
                                    ctypes.c_size_t(ws.numel()), _stream()))
+
+
+def natsl_decode_block_end(route_block, g_block, state, state_start, cache_len, block_len,
+                           p: natsl_params, ws):
+    _check(lib().natsl_decode_block_end(_ptr(route_block), _ptr(g_block), _ptr(state),
+                                        _ptr(state_start), _ptr(cache_len), ctypes.c_int32(block_len),
+                                        ctypes.byref(p), _ptr(ws), ctypes.c_size_t(ws.numel()),
+                                        _stream()))
 
 
 def natsl_device_status(ws) -> int:

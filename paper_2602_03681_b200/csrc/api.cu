@@ -428,7 +428,6 @@ int natsl_decode_step(const void *q, const void *k, const void *v, const float *
         !out)
         return NATSL_ERR_NULL;
     if (cache_cap <= 0) return NATSL_ERR_SHAPE;
-    if (p->flags & NATSL_BLOCK_ROUTING) return NATSL_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(state) ||
         !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
         return NATSL_ERR_ALIGN;
@@ -437,6 +436,21 @@ int natsl_decode_step(const void *q, const void *k, const void *v, const float *
                                        cache_len, cache_cap, out, p->scale_la, p->scale_sm, p->eps,
                                        ws, shape_of(p),
                                        static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
+}
+
+int natsl_decode_block_end(const uint8_t *route_block, const float *g_block, float *state,
+                           float *state_start, int32_t *cache_len, int32_t block_len,
+                           const natsl_params *p, void *ws, size_t ws_bytes, void *stream) {
+    int rc = check_params(p, false);
+    if (rc != NATSL_OK) return rc;
+    if (!route_block || !g_block || !state || !state_start || !cache_len) return NATSL_ERR_NULL;
+    if (block_len <= 0) return NATSL_ERR_SHAPE;
+    if (!aligned16(state) || !aligned16(state_start) || !aligned16(ws)) return NATSL_ERR_ALIGN;
+    if (!ws || ws_bytes < decode_workspace_bytes(p->B, p->H, p->d)) return NATSL_ERR_WORKSPACE;
+    cudaError_t e = launch_decode_block_end(route_block, g_block, state, state_start, cache_len,
+                                            block_len, ws, shape_of(p),
+                                            static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
 }
 

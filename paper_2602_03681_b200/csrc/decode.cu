@@ -1,6 +1,8 @@
 // Decode step (Section 4.1, per-token generation): decay the fp32 d x d state, apply the gated
-// delta rule (linear token) or retain the token's K/V (softmax token), read both branches and
-// combine their RMS-normalised outputs (Section 4.3, Norm equation).
+// delta rule (linear token) or retain the token's K/V (softmax token) -- or both, while the
+// decision of the token's block is still open -- read both branches and combine their
+// RMS-normalised outputs (Section 4.3, Norm equation).  decode_block_end_kernel rolls back the
+// operation that was not chosen once a block is complete.
 //
 // HBM-bound: per (sequence, head) the state is read and written once (2 d^2 4 bytes) and the
 // retained K/V are read once.  To keep enough bytes in flight and the SMs evenly loaded, each
@@ -90,7 +92,11 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
         reinterpret_cast<float *>(ws + dec_off_partials(BH)) + (size_t)bh * kDecodeParts * (D + 2);
     float *ola_ws = reinterpret_cast<float *>(ws + dec_off_ola(BH, D)) + (size_t)bh * D;
 
-    const int r = route[bh] != 0;
+    // route 0: linear token (delta rule); 1: softmax token (appended to the cache); 2: token of a
+    // block whose decision is still open -- both (Section 4.1, pseudo-update of both hidden states)
+    const int rv = route[bh];
+    const bool r = rv != 0;                        // append, and attend to itself
+    const bool fold = rv != 1;                     // delta rule
     const int n_old = cache_len[bh];
     const bool cache_full = r && n_old >= cap;     // no room: the sequence is left untouched
     if (tid < D) {
@@ -200,7 +206,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
         float (*redv)[kCols] = reinterpret_cast<float (*)[kCols]>(smem);   // [kSlots][kCols]
         const int c0 = (part - kDecodeParts) * kCols;
         const float alpha = __expf(g[bh]);
-        const float bt = r ? 0.f : beta[bh];
+        const float bt = fold ? beta[bh] : 0.f;
         const int slot = warp * kRpl + lane / kLpr;
         const int col = (lane % kLpr) * 4;
         float *sp = state + (size_t)bh * D * D + c0;
@@ -212,7 +218,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
         for (int rr = 0; rr < kR; ++rr) {
             s[rr].x *= alpha; s[rr].y *= alpha; s[rr].z *= alpha; s[rr].w *= alpha;
         }
-        if (!r) {   // block-uniform
+        if (fold) {   // block-uniform
             float4 p = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int rr = 0; rr < kR; ++rr) {
@@ -318,7 +324,46 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
     if (r && tid == 0) cache_len[bh] = n_old + 1;
 }
 
+// End of a block of R tokens decoded with the decision open: a softmax block resets the state to
+// its value at the block's start times the block's decay (the block's K/V stay in the cache); a
+// linear block keeps the state and drops its R cache entries.  state_start then holds the new
+// state: the start of the next block.  One CTA per (sequence, head).
+__global__ void __launch_bounds__(256)
+decode_block_end_kernel(const uint8_t *__restrict__ route_block, const float *__restrict__ g_block,
+                        float *__restrict__ state, float *__restrict__ state_start,
+                        int32_t *__restrict__ cache_len, int R, int n4, int32_t *status) {
+    const int bh = blockIdx.x;
+    float4 *S = reinterpret_cast<float4 *>(state) + (size_t)bh * n4;
+    float4 *S0 = reinterpret_cast<float4 *>(state_start) + (size_t)bh * n4;
+    if (route_block[bh]) {
+        const float decay = expf(g_block[bh]);
+        for (int i = threadIdx.x; i < n4; i += blockDim.x) {
+            float4 a = S0[i];
+            a.x *= decay; a.y *= decay; a.z *= decay; a.w *= decay;
+            S[i] = a;
+            S0[i] = a;
+        }
+    } else {
+        for (int i = threadIdx.x; i < n4; i += blockDim.x) S0[i] = S[i];
+        if (threadIdx.x == 0) {
+            const int n = cache_len[bh];
+            if (n < R) atomicMin(status, (int)NATSL_ERR_ROUTE);   // the block's entries are not there
+            else cache_len[bh] = n - R;
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_decode_block_end(const uint8_t *route_block, const float *g_block, float *state,
+                                    float *state_start, int32_t *cache_len, int32_t block_len,
+                                    void *ws, Shape s, cudaStream_t st) {
+    decode_block_end_kernel<<<s.B * s.H, 256, 0, st>>>(route_block, g_block, state, state_start,
+                                                       cache_len, block_len, s.d * s.d / 4,
+                                                       reinterpret_cast<int32_t *>(ws));
+    count_launch();
+    return cudaGetLastError();
+}
 
 size_t decode_workspace_bytes(int B, int H, int d) {
     return dec_off_ola((size_t)B * H, d) + ((size_t)B * H * d * 4 + 255) / 256 * 256;

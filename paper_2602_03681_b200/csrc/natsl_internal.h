@@ -189,5 +189,8 @@ cudaError_t launch_decode_step(const void *q, const void *k, const void *v, cons
                                float *state, void *k_cache, void *v_cache, int32_t *cache_len,
                                int32_t cache_cap, void *out, float scale_la, float scale_sm,
                                float eps, void *ws, Shape s, cudaStream_t st);
+cudaError_t launch_decode_block_end(const uint8_t *route_block, const float *g_block, float *state,
+                                    float *state_start, int32_t *cache_len, int32_t block_len,
+                                    void *ws, Shape s, cudaStream_t st);
 
 }  // namespace natsl

@@ -6,7 +6,7 @@ import torch
 
 import oracle
 from paper_2602_03681_b200 import inputs
-from test_gpu_parity import check_fwd, dev, rel_err, run_fwd, tdtype
+from test_gpu_parity import check_fwd, check_stored, dev, rel_err, run_fwd, tdtype
 
 pytestmark = pytest.mark.gpu
 
@@ -103,3 +103,86 @@ def test_block_routing_off_the_tensor_core_path_is_refused():
                            dev(x["beta"]), dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la,
                            scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING | binding.FORCE_SIMT)
     assert ei.value.status == binding.ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------ generation
+def decode_blocks(wl, x, t0, t1, state, kc, vc, n, ref, tol):
+    """Decode tokens t0..t1 of x with the block decision open, rolling back at each block's end;
+    every step's output is checked against row t of the block-mode forward `ref`."""
+    from paper_2602_03681_b200 import binding
+    dt = tdtype(wl)
+    B, _, H, d = x["q"].shape
+    p = binding.make_params(B, H, 0, d, binding._dtype_code(kc), wl.scale_la, wl.scale_sm)
+    ws = binding.alloc_workspace(p, binding.OP_DECODE)
+    start = state.clone()
+    undecided = torch.full((B, H), 2, dtype=torch.uint8, device="cuda")
+    for t in range(t0, t1):
+        w = dev(x["w"][:, t])
+        p.w = w.data_ptr()
+        out = torch.empty((B, H, d), dtype=dt, device="cuda")
+        binding.natsl_decode_step(dev(x["q"][:, t], dt), dev(x["k"][:, t], dt), dev(x["v"][:, t], dt),
+                                  dev(x["g"][:, t]), dev(x["beta"][:, t]), undecided, state, kc, vc, n,
+                                  out, p, ws)
+        check_stored(out.float().cpu().numpy(), ref["out"][:, t], tol, wl.dtype, f"step{t}")
+        if (t + 1) % 64 == 0:
+            g_block = x["g"][:, t - 63:t + 1].astype(np.float64).sum(1).astype(np.float32)
+            binding.natsl_decode_block_end(dev(x["route"][:, t]), dev(g_block), state, start, n, 64, p, ws)
+            assert torch.equal(state, start)
+    assert binding.natsl_device_status(ws) == 0
+
+
+@pytest.mark.parametrize("name,B,H,L0,L", [("cfg3_bf16_decode", 2, 2, 256, 448),
+                                           ("cfg4_bf16_train", 1, 3, 128, 256)])
+def test_block_routed_prefill_then_generation(name, B, H, L0, L):
+    """Prefill L0 tokens, then generate up to L with route 2 and block ends: every step equals the
+    block-mode forward over the whole sequence; so do the final state and the kept K/V."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS[name]
+    x = block_inputs(wl, B, H, L, 0.4)
+    ref = oracle_block(wl, x, want_cache=True)
+    dt = tdtype(wl)
+    pre = binding.hybrid_fwd(*(dev(x[n][:, :L0], dt) for n in ("q", "k", "v")), dev(x["g"][:, :L0]),
+                             dev(x["beta"][:, :L0]), dev(x["route"][:, :L0]), dev(x["w"][:, :L0]),
+                             scale_la=wl.scale_la, scale_sm=wl.scale_sm, want=("state_out", "cache"),
+                             sm_cap=L, flags=binding.BLOCK_ROUTING)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(pre["ws"]) == 0
+    state, kc, vc, n = pre["state_out"], pre["k_sm"], pre["v_sm"], pre["sm_len"]
+    decode_blocks(wl, x, L0, L, state, kc, vc, n, ref, TOL_BF16)
+    assert np.array_equal(n.cpu().numpy(), ref["n_sm"])
+    assert rel_err(state.cpu().numpy(), ref["state_out"]) <= TOL_BF16
+    for b in range(B):
+        for h in range(H):
+            m = ref["n_sm"][b, h]
+            assert np.array_equal(kc[b, h, :m].float().cpu().numpy(), ref["k_sm"][b, h, :m])
+            assert np.array_equal(vc[b, h, :m].float().cpu().numpy(), ref["v_sm"][b, h, :m])
+
+
+def test_block_routed_generation_from_scratch_fp32():
+    """fp32 storage, no prefill: two blocks generated from an empty state and cache, 1e-4."""
+    wl = inputs.WORKLOADS["cfg0_f32_tiny_fwd"]
+    B, H, L = 2, 2, 128
+    x = block_inputs(wl, B, H, L, 0.5)
+    x["route"][:, :64] = 0                 # a linear block first: its entries are dropped again
+    x["route"][:, 64:] = 1
+    ref = oracle_block(wl, x, want_cache=True)
+    state = torch.zeros((B, H, wl.d, wl.d), device="cuda")
+    kc = torch.zeros((B, H, L, wl.d), device="cuda")
+    vc = torch.zeros_like(kc)
+    n = torch.zeros((B, H), dtype=torch.int32, device="cuda")
+    decode_blocks(wl, x, 0, L, state, kc, vc, n, ref, 1e-4)
+    assert np.array_equal(n.cpu().numpy(), ref["n_sm"]) and np.all(ref["n_sm"] == 64)
+    assert rel_err(state.cpu().numpy(), ref["state_out"]) <= 1e-4
+    assert np.array_equal(kc[:, :, :64].cpu().numpy(), ref["k_sm"][:, :, :64].astype(np.float32))
+
+
+def test_block_end_without_the_blocks_entries_is_reported():
+    from paper_2602_03681_b200 import binding
+    p = binding.make_params(1, 1, 0, 64, binding.NATSL_F32, 1.0, 1.0)
+    ws = binding.alloc_workspace(p, binding.OP_DECODE)
+    state = torch.zeros((1, 1, 64, 64), device="cuda")
+    n = torch.full((1, 1), 10, dtype=torch.int32, device="cuda")
+    binding.natsl_decode_block_end(torch.zeros((1, 1), dtype=torch.uint8, device="cuda"),
+                                   torch.zeros((1, 1), device="cuda"), state, state.clone(), n, 64, p, ws)
+    assert binding.natsl_device_status(ws) == binding.ERR_ROUTE
+    assert n.item() == 10
