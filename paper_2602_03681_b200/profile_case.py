@@ -6,6 +6,7 @@ calls of `--op` on the current device and exits.  Nothing is timed or checked he
     python -m paper_2602_03681_b200.profile_case --op fwd --workload cfg1_bf16_prefill --B 1
     python -m paper_2602_03681_b200.profile_case --op decode --workload cfg3_bf16_decode --B 8 --iters 4
     python -m paper_2602_03681_b200.profile_case --op bwd --workload cfg4_bf16_train --B 1
+    python -m paper_2602_03681_b200.profile_case --op fwd --flags 4        (block-level routing)
 """
 from __future__ import annotations
 
@@ -81,6 +82,9 @@ def main():
         kw["B"] = args.B
     if args.L:
         kw["L"] = args.L
+    if args.op == "fwd" and args.flags & binding.BLOCK_ROUTING:   # one route per block of 64 tokens
+        kw["route"] = inputs.route_blocks(wl.seed, (kw.get("B", wl.B), kw.get("L", wl.L), wl.H),
+                                          wl.p_softmax)
     x = inputs.make_layer_inputs(wl, **kw)
     q, k, v = (dev(x[m], dt) for m in ("q", "k", "v"))
     g, beta, route, w = (dev(x[m]) for m in ("g", "beta", "route", "w"))
