@@ -611,3 +611,39 @@ def test_block_mode_generation_protocol_equals_the_forward():
         for h in range(H):
             assert np.array_equal(kc[b, h, :n[b, h]], ref["k_sm"][b, h, :n[b, h]])
             assert np.array_equal(vc[b, h, :n[b, h]], ref["v_sm"][b, h, :n[b, h]])
+
+
+# ------------------------------------------------------------------ score layer (Section 4.1)
+def test_score_layer_closed_forms_and_brute_force():
+    from oracle import router
+    r = np.random.default_rng(41)
+    B, L, Dm, H, C = 2, 24, 10, 3, 4
+    x = r.standard_normal((B, L, Dm))
+    w = r.standard_normal((H, 2, Dm))
+    res = router.score_layer(x, w, C)
+    # brute force, loop by loop
+    for b in range(B):
+        for c in range(L // C):
+            for h in range(H):
+                for o in range(2):
+                    s = 0.0
+                    for dd in range(Dm):
+                        m = sum(x[b, c * C + i, dd] for i in range(C)) / C
+                        s += w[h, o, dd] * m
+                    assert abs(res["scores"][b, c, h, o] - s) < 1e-12
+                sm = np.exp(res["scores"][b, c, h]) / np.exp(res["scores"][b, c, h]).sum()
+                assert np.all(res["route"][b, c * C:(c + 1) * C, h] == np.argmax(sm))
+    # a chunk of identical tokens: the mean is the token, the score is W x
+    xc = np.repeat(r.standard_normal((1, 3, Dm)), C, axis=1)
+    rc = router.score_layer(xc, w, C)
+    np.testing.assert_allclose(rc["scores"][0], np.einsum("cd,hod->cho", xc[0, ::C], w), rtol=1e-12)
+    # one-hot rows pick out the mean of one feature; equal rows tie, and the tie goes to linear
+    w1 = np.zeros((1, 2, Dm))
+    w1[0, :, 7] = 1.0
+    r1 = router.score_layer(x, w1, C)
+    np.testing.assert_allclose(r1["scores"][..., 0, 1], x[..., 7].reshape(B, L // C, C).mean(-1), rtol=1e-12)
+    assert not r1["route"].any()
+    # scaling the softmax row up flips every chunk whose pooled feature is positive
+    w1[0, 1, 7] = 2.0
+    r2 = router.score_layer(x, w1, C)
+    assert np.array_equal(r2["route"][:, ::C, 0] == 1, x[..., 7].reshape(B, L // C, C).mean(-1) > 0)
