@@ -461,7 +461,38 @@ def bench_other_workloads(peaks):
         res[name] = entry
         del d, ws
         torch.cuda.empty_cache()
+    res["score_layer"] = bench_score_layer(peaks)
     return res
+
+
+def bench_score_layer(peaks):
+    """The attention score layer on the prefill shapes (d_model = H d): HBM-bound, X is read once."""
+    import torch
+
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    Dm = wl.H * wl.d
+    gen = torch.Generator(device="cuda").manual_seed(wl.seed)
+    reps = 6                               # distinct inputs in turn: 6 x 67 MB > L2
+    xs = [torch.randn((wl.B, wl.L, Dm), device="cuda", generator=gen).to(torch.bfloat16) for _ in range(reps)]
+    w = torch.randn((wl.H, 2, Dm), device="cuda", generator=gen) / Dm ** 0.5
+    route = torch.empty((wl.B, wl.L, wl.H), dtype=torch.uint8, device="cuda")
+    p = binding.make_params(wl.B, wl.H, wl.L, wl.d, binding.NATSL_BF16, 1.0, 1.0)
+    for x in xs[:3]:
+        binding.natsl_score_layer(x, w, None, route, p)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n = 4 * reps
+    e0.record()
+    for i in range(n):
+        binding.natsl_score_layer(xs[i % reps], w, None, route, p)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / n
+    nbytes = wl.B * wl.L * Dm * 2 + wl.B * wl.L * wl.H
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"ms": ms, "d_model": Dm, "algorithmic_bytes": nbytes, "achieved_gbs": gbs,
+            "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
 
 
 def bench_decode(args, peaks, peak_kind, traffic):

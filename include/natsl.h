@@ -129,6 +129,25 @@ int natsl_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk
                         void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * Attention score layer (Section 4.1, the score equation and the arg max after it): per chunk of
+ * C = 64 tokens, score = W^score Mean(X_chunk), one score per operation and head, and the
+ * operation with the higher score becomes the chunk's route.  Its output is a `route` for
+ * NATSL_BLOCK_ROUTING.
+ *   x       [B,L,d_model] in p->dtype (the layer's input features), d_model a multiple of 8
+ *           (bf16) or 4 (fp32), 16-byte aligned;
+ *   w_score [H,2,d_model] fp32, 16-byte aligned: row (h, 0) scores linear attention, row (h, 1)
+ *           softmax attention (every head has its own mask, Section 4.3);
+ *   scores  [B,L/C,H,2] fp32, or NULL;
+ *   route   [B,L,H] u8: 1 where the softmax score is strictly higher (a tie keeps linear, the first
+ *           operation), repeated over the chunk's tokens.
+ * The softmax over the two scores is monotone and is not formed.  fp32 accumulation throughout.
+ * Only B, L, H, C, dtype of `p` are used (d must still be valid).  No workspace.
+ * Errors: NULL, SHAPE, DTYPE, ALIGN, CUDA.
+ */
+int natsl_score_layer(const void *x, const float *w_score, float *scores, uint8_t *route,
+                      int32_t d_model, const natsl_params *p, void *stream);
+
+/*
  * Forward of the whole layer (header comment; Sections 4.1 and 4.3).
  *   q,k,v [B,L,H,d] in p->dtype; g,beta [B,L,H] fp32 (g = log decay <= 0);
  *   route [B,L,H] u8; out [B,L,H,d] in p->dtype.

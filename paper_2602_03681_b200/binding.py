@@ -25,6 +25,7 @@ ERR_ROUTE = -11
 
 EXPORTS = ["natsl_workspace_size", "natsl_route_compact", "natsl_hybrid_fwd", "natsl_hybrid_bwd",
            "natsl_decode_step", "natsl_decode_block_end", "natsl_device_status", "natsl_hybrid_fwd_static",
+           "natsl_score_layer",
            "natsl_stage_name", "natsl_launch_count", "natsl_strerror"]
 ERR_TOO_LARGE = -9
 STATIC_WS_BYTES = 32 << 20
@@ -191,6 +192,11 @@ def natsl_decode_block_end(route_block, g_block, state, state_start, cache_len, 
                                         _ptr(state_start), _ptr(cache_len), ctypes.c_int32(block_len),
                                         ctypes.byref(p), _ptr(ws), ctypes.c_size_t(ws.numel()),
                                         _stream()))
+
+
+def natsl_score_layer(x, w_score, scores, route, p: natsl_params):
+    _check(lib().natsl_score_layer(_ptr(x), _ptr(w_score), _ptr(scores), _ptr(route),
+                                   ctypes.c_int32(x.shape[-1]), ctypes.byref(p), _stream()))
 
 
 def natsl_device_status(ws) -> int:

@@ -225,6 +225,22 @@ int natsl_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk
     return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
 }
 
+int natsl_score_layer(const void *x, const float *w_score, float *scores, uint8_t *route,
+                      int32_t d_model, const natsl_params *p, void *stream) {
+    int rc = check_params(p, true);
+    if (rc != NATSL_OK) return rc;
+    if (!x || !w_score || !route) return NATSL_ERR_NULL;
+    // a row of X is read in 16-byte pieces
+    const int per16 = p->dtype == NATSL_BF16 ? 8 : 4;
+    // (the pooled rows of a CTA's two chunks and their scores live in shared memory)
+    if (d_model <= 0 || d_model % per16 != 0 || ((size_t)d_model + 2 * (size_t)p->H) * 8 > 200 * 1024)
+        return NATSL_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(w_score)) return NATSL_ERR_ALIGN;
+    cudaError_t e = launch_score_layer(x, w_score, scores, route, d_model, shape_of(p),
+                                       static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
+}
+
 int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g,
                      const float *beta, const uint8_t *route, void *out, const natsl_params *p,
                      void *ws, size_t ws_bytes, void *stream) {

@@ -26,6 +26,10 @@ struct BlockRouting {
     const void *k, *v;
 };
 
+// router.cu -- attention score layer: scores [B,L/C,H,2] (may be nullptr) and route [B,L,H]
+cudaError_t launch_score_layer(const void *x, const float *w_score, float *scores, uint8_t *route,
+                               int d_model, Shape s, cudaStream_t st);
+
 // compact.cu  (block_status: where a route that changes inside a chunk is reported, or nullptr)
 cudaError_t launch_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk_prefix,
                                  int32_t *lin_idx, int32_t *n_lin, int32_t *sm_len,
