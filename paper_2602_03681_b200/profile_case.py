@@ -7,6 +7,7 @@ calls of `--op` on the current device and exits.  Nothing is timed or checked he
     python -m paper_2602_03681_b200.profile_case --op decode --workload cfg3_bf16_decode --B 8 --iters 4
     python -m paper_2602_03681_b200.profile_case --op bwd --workload cfg4_bf16_train --B 1
     python -m paper_2602_03681_b200.profile_case --op fwd --flags 4        (block-level routing)
+    python -m paper_2602_03681_b200.profile_case --op score --iters 6      (attention score layer)
 """
 from __future__ import annotations
 
@@ -19,7 +20,7 @@ from . import binding, inputs
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", choices=["fwd", "bwd", "decode"], default="fwd")
+    ap.add_argument("--op", choices=["fwd", "bwd", "decode", "score"], default="fwd")
     ap.add_argument("--workload", default=None, choices=sorted(inputs.WORKLOADS),
                     help="default: the workload that belongs to --op")
     ap.add_argument("--B", type=int, default=None, help="batch override (smaller case)")
@@ -30,7 +31,7 @@ def main():
     args = ap.parse_args()
     if args.workload is None:
         args.workload = {"fwd": "cfg1_bf16_prefill", "bwd": "cfg4_bf16_train",
-                         "decode": "cfg3_bf16_decode"}[args.op]
+                         "decode": "cfg3_bf16_decode", "score": "cfg1_bf16_prefill"}[args.op]
     if (inputs.WORKLOADS[args.workload].call == "decode") != (args.op == "decode"):
         ap.error(f"workload {args.workload} does not belong to --op {args.op}")
 
@@ -58,6 +59,18 @@ def main():
         if args.report:
             print(f"{args.op} {args.workload}: ms per call",
                   [round(a.elapsed_time(b), 4) for a, b in events], note)
+
+    if args.op == "score":      # the attention score layer on the workload's shapes, d_model = H d
+        B, L, Dm = args.B or wl.B, args.L or wl.L, wl.H * wl.d
+        gen = torch.Generator(device="cuda").manual_seed(wl.seed)
+        xs = [torch.randn((B, L, Dm), device="cuda", generator=gen).to(dt) for _ in range(3)]
+        w = torch.randn((wl.H, 2, Dm), device="cuda", generator=gen) / Dm ** 0.5
+        route = torch.empty((B, L, wl.H), dtype=torch.uint8, device="cuda")
+        p = binding.make_params(B, wl.H, L, wl.d, code, 1.0, 1.0)
+        for i in range(args.iters):
+            timed(lambda: binding.natsl_score_layer(xs[i % 3], w, None, route, p))
+        finish()
+        return
 
     if args.op == "decode":
         B = args.B or wl.B
