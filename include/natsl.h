@@ -71,7 +71,7 @@ enum {
                                     parallel (a second run per segment yields the segment's
                                     state transition, a small kernel chains the segments); the
                                     results agree to rounding */
-    NATSL_BLOCK_ROUTING = 1u << 2      /* forward, tensor-core path: block-level routing, the paper's
+    NATSL_BLOCK_ROUTING = 1u << 2,     /* forward, tensor-core path: block-level routing, the paper's
                                     default (Section 4.1, "compute the inner-chunk correlation";
                                     Section 4.3, chunk size = GDN chunk size).  `route` holds one
                                     decision per block of C = 64 tokens, repeated over the block's
@@ -87,6 +87,18 @@ enum {
                                     reported as NATSL_ERR_ROUTE by natsl_device_status.  Backward:
                                     NATSL_ERR_UNSUPPORTED with this flag.  Generation: route 2 in
                                     natsl_decode_step and natsl_decode_block_end (no flag needed) */
+    NATSL_APPEND_CACHE = 1u << 3       /* forward, tensor-core path: prefill in pieces.  p->k_sm, p->v_sm,
+                                    p->sm_len (required) are read AND written: the cache already
+                                    holds sm_len[b,h] retained tokens of earlier pieces of the same
+                                    sequences; the softmax branch of this piece reads them as
+                                    earlier tokens, and the piece's own retained tokens are
+                                    appended behind them (sm_len grows; NATSL_ERR_CACHE_FULL in the
+                                    status word if sm_cap would be exceeded).  Together with
+                                    p->state_in = the previous piece's state_out this continues a
+                                    sequence exactly where the last call stopped (Section 4.1: the
+                                    two hidden states kept during generation are the linear state
+                                    and the KV cache).  natsl_workspace_size depends on the flag
+                                    and on p->sm_cap.  Backward: NATSL_ERR_UNSUPPORTED */
 };
 
 typedef struct natsl_params {

@@ -19,6 +19,7 @@ OP_FWD, OP_BWD, OP_DECODE, OP_COMPACT = 0, 1, 2, 3
 FORCE_SIMT = 1
 SINGLE_PASS_SCAN = 2
 BLOCK_ROUTING = 4
+APPEND_CACHE = 8
 ERR_CACHE_FULL = -7
 ERR_UNSUPPORTED = -8
 ERR_ROUTE = -11
@@ -207,9 +208,10 @@ def natsl_device_status(ws) -> int:
 # Convenience wrappers (allocation + marshalling; no arithmetic).
 # ---------------------------------------------------------------------------------------------
 def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5, state_in=None,
-               want=(), flags=0, sm_cap=0, ws=None):
+               want=(), flags=0, sm_cap=0, ws=None, cache=None):
     """Allocate outputs and run natsl_hybrid_fwd.  `want` may name optional outputs:
-    "o_la", "o_nla", "lse", "state_out", "cache" (compacted K/V with capacity sm_cap or L)."""
+    "o_la", "o_nla", "lse", "state_out", "cache" (compacted K/V with capacity sm_cap or L).
+    cache=(k_sm, v_sm, sm_len): use these existing cache tensors (with APPEND_CACHE: in and out)."""
     B, L, H, d = q.shape
     dev = q.device
     out = torch.empty_like(q)
@@ -223,7 +225,10 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5,
     if "state_out" in want:
         opt["state_out"] = torch.empty((B, H, d, d), dtype=torch.float32, device=dev)
     cap = 0
-    if "cache" in want:
+    if cache is not None:
+        opt["k_sm"], opt["v_sm"], opt["sm_len"] = cache
+        cap = cache[0].shape[2]
+    elif "cache" in want:
         cap = sm_cap or L
         opt["k_sm"] = torch.zeros((B, H, cap, d), dtype=q.dtype, device=dev)
         opt["v_sm"] = torch.zeros((B, H, cap, d), dtype=q.dtype, device=dev)

@@ -82,7 +82,9 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
     f.k_sm = c.take<char>(B * H * L * d * esz);
     f.v_sm = c.take<char>(B * H * L * d * esz);
     if (use_tensor_cores(p)) {
-        f.v16 = c.take<char>(B * H * L * d * 2);          // fp16 V of the retained tokens
+        // fp16 V of the retained tokens; when the call appends to a cache, of the whole cache
+        const size_t capv = (p->flags & NATSL_APPEND_CACHE) && p->sm_cap > 0 ? (size_t)p->sm_cap : L;
+        f.v16 = c.take<char>(B * H * capv * d * 2);
         f.tc.Qh = c.take<char>(B * H * L * d * 2);
         f.tc.Kh = c.take<char>(B * H * L * d * 2);
         f.tc.Wt = c.take<char>(B * H * L * d * 2);
@@ -221,7 +223,8 @@ int natsl_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk
     if (rc != NATSL_OK) return rc;
     if (!route || !sm_idx || !sm_chunk_prefix || !lin_idx || !n_lin) return NATSL_ERR_NULL;
     cudaError_t e = launch_route_compact(route, sm_idx, sm_chunk_prefix, lin_idx, n_lin, nullptr,
-                                         nullptr, p->B, p->L, p->H, static_cast<cudaStream_t>(stream));
+                                         nullptr, nullptr, p->B, p->L, p->H,
+                                         static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
 }
 
@@ -256,6 +259,9 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     const bool tensor_cores = use_tensor_cores(p);
     const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
     if (block && !tensor_cores) return NATSL_ERR_UNSUPPORTED;
+    const bool append = (p->flags & NATSL_APPEND_CACHE) != 0;
+    if (append && !tensor_cores) return NATSL_ERR_UNSUPPORTED;
+    if (append && !want_cache) return NATSL_ERR_NULL;
     FwdWs f = carve_fwd(p, ws);
     if (!ws || ws_bytes < f.bytes) return NATSL_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -274,11 +280,13 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     int32_t *sm_len = want_cache ? p->sm_len : f.sm_len;
     void *k_sm = want_cache ? p->k_sm : f.k_sm, *v_sm = want_cache ? p->v_sm : f.v_sm;
     const int32_t cap = want_cache ? p->sm_cap : p->L;
+    const int32_t capv = append ? p->sm_cap : p->L;          // rows per head of the fp16 V copy
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, sm_len,
-                                   block ? f.status : nullptr, p->B, p->L, p->H, st));
+                                   append ? sm_len : nullptr, block ? f.status : nullptr, p->B, p->L,
+                                   p->H, st));
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
-                                      f.v16, nullptr, cap, p->L, f.status, s, st));
+                                      f.v16, nullptr, cap, capv, f.status, s, st));
     else
         NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
     NATSL_TRY(mark());
@@ -311,7 +319,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     }
     NATSL_TRY(mark());
     if (tensor_cores)
-        NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, p->L, f.sm_idx, f.prefix, o_la, p->w,
+        NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, capv, f.sm_idx, f.prefix, o_la, p->w,
                                             p->scale_sm, p->eps, out, p->o_nla, p->lse, br, f.status,
                                             s, st));
     else
@@ -330,7 +338,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (rc != NATSL_OK) return rc;
     if (!q || !k || !v || !g || !beta || !route || !dout || !dq || !dk || !dv || !dg || !dbeta)
         return NATSL_ERR_NULL;
-    if (p->state_in || (p->flags & NATSL_BLOCK_ROUTING)) return NATSL_ERR_UNSUPPORTED;
+    if (p->state_in || (p->flags & (NATSL_BLOCK_ROUTING | NATSL_APPEND_CACHE))) return NATSL_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
         return NATSL_ERR_ALIGN;
@@ -351,7 +359,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
     // ---- forward recomputation, keeping what the backward needs ----
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, nullptr,
-                                   p->B, p->L, p->H, st));
+                                   nullptr, p->B, p->L, p->H, st));
     const bool tensor_cores = use_tensor_cores(p);
     const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
     if (!fused_chunks)

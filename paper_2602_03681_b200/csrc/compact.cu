@@ -17,7 +17,7 @@ constexpr int kCompactTile = 1024;  // chunks scanned per pass (one per thread)
 __global__ void __launch_bounds__(kCompactThreads)
 route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm_idx,
                      int32_t *__restrict__ sm_chunk_prefix, int32_t *__restrict__ lin_idx,
-                     int32_t *__restrict__ n_lin, int32_t *__restrict__ sm_len,
+                     int32_t *__restrict__ n_lin, int32_t *sm_len, const int32_t *base_in,
                      int32_t *__restrict__ block_status, int L, int H) {
     __shared__ unsigned long long bits[kCompactTile];
     __shared__ int excl[kCompactTile];
@@ -29,7 +29,12 @@ route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kWarps = kCompactThreads / 32;
     const uint8_t *rt = route + (size_t)b * L * H + h;
-    int base = 0;
+    // Appending to a cache that already holds base0 retained tokens of earlier calls: the prefix
+    // sums start there, the positions listed in sm_idx are still this call's own (index - base0).
+    // (base_in may be the same array as sm_len: it is read here, written at the very end.)
+    const int base0 = base_in ? base_in[bh] : 0;
+    int base = base0;
+    __syncthreads();
 
     for (int tile0 = 0; tile0 < NC; tile0 += kCompactTile) {
         const int nt = min(kCompactTile, NC - tile0);
@@ -88,7 +93,7 @@ route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm
                 atomicMin(block_status, (int)NATSL_ERR_ROUTE);
             const unsigned lt = (1u << lane) - 1u;
             const int nlo = __popc(lo), nsm = nlo + __popc(hi);
-            int32_t *sm = sm_idx + (size_t)bh * L + pre;
+            int32_t *sm = sm_idx + (size_t)bh * L + (pre - base0);
             int32_t *li = lin_idx + ((size_t)bh * NC + cc) * kC;
             if (lane == 0) {
                 sm_chunk_prefix[(size_t)bh * (NC + 1) + cc] = pre;
@@ -140,9 +145,10 @@ gather_kv_kernel(const T *__restrict__ k, const T *__restrict__ v, const int32_t
 
 cudaError_t launch_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk_prefix,
                                  int32_t *lin_idx, int32_t *n_lin, int32_t *sm_len,
-                                 int32_t *block_status, int B, int L, int H, cudaStream_t st) {
+                                 const int32_t *base_in, int32_t *block_status, int B, int L, int H,
+                                 cudaStream_t st) {
     route_compact_kernel<<<B * H, kCompactThreads, 0, st>>>(route, sm_idx, sm_chunk_prefix, lin_idx,
-                                                            n_lin, sm_len, block_status, L, H);
+                                                            n_lin, sm_len, base_in, block_status, L, H);
     count_launch();
     return cudaGetLastError();
 }

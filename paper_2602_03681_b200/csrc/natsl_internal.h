@@ -30,10 +30,12 @@ struct BlockRouting {
 cudaError_t launch_score_layer(const void *x, const float *w_score, float *scores, uint8_t *route,
                                int d_model, Shape s, cudaStream_t st);
 
-// compact.cu  (block_status: where a route that changes inside a chunk is reported, or nullptr)
+// compact.cu  (block_status: where a route that changes inside a chunk is reported, or nullptr;
+// base_in [B,H]: retained tokens already in the cache the call appends to, or nullptr for none)
 cudaError_t launch_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk_prefix,
                                  int32_t *lin_idx, int32_t *n_lin, int32_t *sm_len,
-                                 int32_t *block_status, int B, int L, int H, cudaStream_t st);
+                                 const int32_t *base_in, int32_t *block_status, int B, int L, int H,
+                                 cudaStream_t st);
 cudaError_t launch_gather_kv(const void *k, const void *v, const int32_t *sm_idx,
                              const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, int32_t cap,
                              int32_t *status, Shape s, cudaStream_t st);

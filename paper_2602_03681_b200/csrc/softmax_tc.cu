@@ -116,9 +116,9 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         ms.abort_flag = 0;
         fence_mbar_init();
     }
-    if (tid < kBM) {
+    if (tid < kBM) {    // sm_idx lists this call's retained tokens; pre[0] of them were there before
         const int jj = n_full + tid;
-        ms.pos[tid] = jj < n_end ? sm_idx[(size_t)bh * L + jj] : 0x7fffffff;
+        ms.pos[tid] = jj < n_end ? sm_idx[(size_t)bh * L + jj - pre[0]] : 0x7fffffff;
     }
     if (warp == 4) tmem_alloc(&ms.tmem_base, 256);
     tc_fence_before_sync();
@@ -447,6 +447,7 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
     if (blockIdx.x == 0 && threadIdx.x == 0 && n_sm > cap) atomicMin(status, (int)NATSL_ERR_CACHE_FULL);
     const int n = min(n_sm, cap);
     const int n_pad = min((n + 127) / 128 * 128, capv);
+    const int n_prev = sm_chunk_prefix[(size_t)bh * (NC + 1)];   // rows of earlier calls (appending)
     const int piece = threadIdx.x % kVecPerRow;
     // the grid is sized for a typical retention rate; each CTA strides over the rows there are
     for (int row = blockIdx.x * kRows + threadIdx.x / kVecPerRow; row < n_pad; row += gridDim.x * kRows) {
@@ -457,9 +458,19 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
             if (dk16) *dk16 = make_uint4(0u, 0u, 0u, 0u);
             continue;
         }
-        const int tok = sm_idx[(size_t)bh * L + row];
-        const size_t src = (((size_t)b * L + tok) * H + h) * D;
         const size_t dst = ((size_t)bh * cap + row) * D;
+        if (row < n_prev) {     // already in the cache: only the fp16 copy of its V row is made
+            const uint4 vv = reinterpret_cast<const uint4 *>(v_sm + dst)[piece];
+            const uint32_t wv[4] = {vv.x, vv.y, vv.z, vv.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                o[i] = pack_half2(__uint_as_float(wv[i] << 16), __uint_as_float(wv[i] & 0xffff0000u));
+            *dv16 = make_uint4(o[0], o[1], o[2], o[3]);
+            continue;
+        }
+        const int tok = sm_idx[(size_t)bh * L + row - n_prev];
+        const size_t src = (((size_t)b * L + tok) * H + h) * D;
         const uint4 kk = reinterpret_cast<const uint4 *>(k + src)[piece];
         reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
         if (dk16) {
