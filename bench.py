@@ -462,7 +462,51 @@ def bench_other_workloads(peaks):
         del d, ws
         torch.cuda.empty_cache()
     res["score_layer"] = bench_score_layer(peaks)
+    res["cfg2_bf16_long_prefill/in_4_pieces"] = bench_prefill_in_pieces()
     return res
+
+
+def bench_prefill_in_pieces(n_pieces=4):
+    """The long-context workload prefilled piece by piece: state chained through state_in /
+    state_out, retained K/V appended to one cache (device-resident inputs, best of 3)."""
+    import torch
+
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg2_bf16_long_prefill"]
+    x = inputs.make_layer_inputs(wl)
+    n = wl.L // n_pieces
+    dt = torch.bfloat16
+    pieces = []
+    for i in range(n_pieces):
+        sl = slice(i * n, (i + 1) * n)
+        pieces.append([torch.from_numpy(np.ascontiguousarray(x[m][:, sl])).cuda().to(dt) for m in ("q", "k", "v")] +
+                      [torch.from_numpy(np.ascontiguousarray(x[m][:, sl])).cuda() for m in ("g", "beta", "route", "w")])
+    cap = int(x["route"].sum(1).max()) + 128
+    cache = (torch.zeros((wl.B, wl.H, cap, wl.d), dtype=dt, device="cuda"),
+             torch.zeros((wl.B, wl.H, cap, wl.d), dtype=dt, device="cuda"),
+             torch.zeros((wl.B, wl.H), dtype=torch.int32, device="cuda"))
+    ws = [None]
+
+    def run():
+        cache[2].zero_()
+        state = None
+        for a in pieces:
+            r = binding.hybrid_fwd(*a, scale_la=wl.scale_la, scale_sm=wl.scale_sm, state_in=state,
+                                   want=("state_out",), cache=cache, flags=binding.APPEND_CACHE, ws=ws[0])
+            state, ws[0] = r["state_out"], r["ws"]
+
+    run()
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        run()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    assert binding.natsl_device_status(ws[0]) == 0
+    return {"ms": best, "pieces": n_pieces, "tokens_per_s": wl.B * wl.L / (best * 1e-3), "cache_rows": cap}
 
 
 def bench_score_layer(peaks):

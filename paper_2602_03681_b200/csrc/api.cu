@@ -286,7 +286,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
                                    p->H, st));
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
-                                      f.v16, nullptr, cap, capv, f.status, s, st));
+                                      f.v16, nullptr, cap, capv, append, f.status, s, st));
     else
         NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
     NATSL_TRY(mark());
@@ -320,8 +320,8 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(mark());
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, capv, f.sm_idx, f.prefix, o_la, p->w,
-                                            p->scale_sm, p->eps, out, p->o_nla, p->lse, br, f.status,
-                                            s, st));
+                                            p->scale_sm, p->eps, out, p->o_nla, p->lse, br, append,
+                                            f.status, s, st));
     else
         NATSL_TRY(launch_softmax_combine_simt(q, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
                                               p->scale_sm, p->eps, out, p->o_nla, p->lse, s, st));
@@ -366,7 +366,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, f.k_smb, nullptr, f.v16, f.k16, p->L,
-                                      p->L, f.status, s, st));
+                                      p->L, false, f.status, s, st));
     else
         NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
                                    f.status, s32, st));
@@ -387,7 +387,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la,
                                             p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
-                                            BlockRouting{nullptr, nullptr, nullptr}, f.status, s, st));
+                                            BlockRouting{nullptr, nullptr, nullptr}, false, f.status, s,
+                                            st));
     else
         NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
                                               f.o_la, p->w, p->scale_sm, p->eps, nullptr, f.o_nla,

@@ -34,7 +34,6 @@ route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm
     // (base_in may be the same array as sm_len: it is read here, written at the very end.)
     const int base0 = base_in ? base_in[bh] : 0;
     int base = base0;
-    __syncthreads();
 
     for (int tile0 = 0; tile0 < NC; tile0 += kCompactTile) {
         const int nt = min(kCompactTile, NC - tile0);

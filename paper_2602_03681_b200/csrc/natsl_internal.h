@@ -60,14 +60,14 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
 // softmax_tc.cu -- tensor-core softmax branch + combination (bf16 storage)
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
                                 const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
-                                void *k16, int32_t cap, int32_t capv, int32_t *status, Shape s,
-                                cudaStream_t st);
+                                void *k16, int32_t cap, int32_t capv, bool appending, int32_t *status,
+                                Shape s, cudaStream_t st);
 cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const void *v16, int32_t cap,
                                       int32_t capv, const int32_t *sm_idx,
                                       const int32_t *sm_chunk_prefix, const float *o_la,
                                       const float *w, float scale_sm, float eps, void *out,
-                                      float *o_nla, float *lse, BlockRouting br, int32_t *status,
-                                      Shape s, cudaStream_t st);
+                                      float *o_nla, float *lse, BlockRouting br, bool appending,
+                                      int32_t *status, Shape s, cudaStream_t st);
 
 // softmax_bwd_tc.cu -- tensor-core backward of the softmax branch (bf16 storage).  Qh is scratch
 // for the fp16 copy of q [B,H,L,d]; dO16 the fp16 branch-output gradient [B,H,L,d]; k16, v16 the

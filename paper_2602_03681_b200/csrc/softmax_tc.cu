@@ -64,7 +64,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                           const __grid_constant__ CUtensorMap map_out,    // out [B,L,H,D] bf16, box 128 x 64, if has_out
                           const __grid_constant__ CUtensorMap map_kd,     // the layer's k, v [B,L,H,D] bf16, box
                           const __grid_constant__ CUtensorMap map_vd,     //   64 x 64: own-block tiles (block routing)
-                          const uint8_t *__restrict__ block_route, int cap, int capv, const int32_t *__restrict__ sm_idx,
+                          const uint8_t *__restrict__ block_route, int appending, int cap, int capv, const int32_t *__restrict__ sm_idx,
                           const int32_t *__restrict__ sm_chunk_prefix,
                           const float *__restrict__ o_la, const float *__restrict__ w,
                           float scale_sm, float eps, int has_out, int has_onla,
@@ -116,9 +116,9 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         ms.abort_flag = 0;
         fence_mbar_init();
     }
-    if (tid < kBM) {    // sm_idx lists this call's retained tokens; pre[0] of them were there before
-        const int jj = n_full + tid;
-        ms.pos[tid] = jj < n_end ? sm_idx[(size_t)bh * L + jj - pre[0]] : 0x7fffffff;
+    if (tid < kBM) {    // sm_idx lists this call's retained tokens; when the call appends to a
+        const int jj = n_full + tid - (appending ? pre[0] : 0);   // cache, pre[0] were there before
+        ms.pos[tid] = n_full + tid < n_end ? sm_idx[(size_t)bh * L + jj] : 0x7fffffff;
     }
     if (warp == 4) tmem_alloc(&ms.tmem_base, 256);
     tc_fence_before_sync();
@@ -438,7 +438,8 @@ __global__ void __launch_bounds__(256)
 gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__restrict__ v,
                     const int32_t *__restrict__ sm_idx, const int32_t *__restrict__ sm_chunk_prefix,
                     __nv_bfloat16 *__restrict__ k_sm, __nv_bfloat16 *__restrict__ v_sm,
-                    __half *__restrict__ v16, __half *__restrict__ k16, int cap, int capv, int32_t *status, int L, int H) {
+                    __half *__restrict__ v16, __half *__restrict__ k16, int cap, int capv, int appending,
+                    int32_t *status, int L, int H) {
     constexpr int kVecPerRow = D * 2 / 16;
     constexpr int kRows = 256 / kVecPerRow;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
@@ -447,7 +448,7 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
     if (blockIdx.x == 0 && threadIdx.x == 0 && n_sm > cap) atomicMin(status, (int)NATSL_ERR_CACHE_FULL);
     const int n = min(n_sm, cap);
     const int n_pad = min((n + 127) / 128 * 128, capv);
-    const int n_prev = sm_chunk_prefix[(size_t)bh * (NC + 1)];   // rows of earlier calls (appending)
+    const int n_prev = appending ? sm_chunk_prefix[(size_t)bh * (NC + 1)] : 0;   // rows of earlier calls
     const int piece = threadIdx.x % kVecPerRow;
     // the grid is sized for a typical retention rate; each CTA strides over the rows there are
     for (int row = blockIdx.x * kRows + threadIdx.x / kVecPerRow; row < n_pad; row += gridDim.x * kRows) {
@@ -499,7 +500,7 @@ static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *
                                    int32_t capv, const int32_t *sm_idx, const int32_t *pre,
                                    const float *o_la, const float *w, float scale_sm, float eps,
                                    void *out, float *o_nla, float *lse, BlockRouting br,
-                                   int32_t *status, Shape s, cudaStream_t st) {
+                                   bool appending, int32_t *status, Shape s, cudaStream_t st) {
     using SL = SmLayout<D>;
     CUtensorMap mq, mk, mv, mola, monla, mout, mkd, mvd;
     if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, kBM) ||
@@ -521,7 +522,7 @@ static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *
     if (e != cudaSuccess) return e;
     dim3 grid((s.L + kBM - 1) / kBM, s.B * s.H);
     kernel<<<grid, kThreadsTc, SL::kTotal, st>>>(
-        mq, mk, mv, mola, monla, mout, mkd, mvd, br.route, cap, capv, sm_idx, pre, o_la, w, scale_sm, eps,
+        mq, mk, mv, mola, monla, mout, mkd, mvd, br.route, appending ? 1 : 0, cap, capv, sm_idx, pre, o_la, w, scale_sm, eps,
         out ? 1 : 0, o_nla ? 1 : 0, lse, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
@@ -531,37 +532,38 @@ cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const voi
                                       int32_t capv, const int32_t *sm_idx,
                                       const int32_t *sm_chunk_prefix, const float *o_la,
                                       const float *w, float scale_sm, float eps, void *out,
-                                      float *o_nla, float *lse, BlockRouting br, int32_t *status,
-                                      Shape s, cudaStream_t st) {
+                                      float *o_nla, float *lse, BlockRouting br, bool appending,
+                                      int32_t *status, Shape s, cudaStream_t st) {
     if (s.d == 128)
         return softmax_tc_impl<128>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la, w,
-                                    scale_sm, eps, out, o_nla, lse, br, status, s, st);
+                                    scale_sm, eps, out, o_nla, lse, br, appending, status, s, st);
     return softmax_tc_impl<64>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la, w, scale_sm,
-                               eps, out, o_nla, lse, br, status, s, st);
+                               eps, out, o_nla, lse, br, appending, status, s, st);
 }
 
 template <int D>
 static cudaError_t gather_tc_impl(const void *k, const void *v, const int32_t *sm_idx,
                                   const int32_t *pre, void *k_sm, void *v_sm, void *v16, void *k16,
-                                  int cap, int capv, int32_t *status, Shape s, cudaStream_t st) {
+                                  int cap, int capv, bool appending, int32_t *status, Shape s,
+                                  cudaStream_t st) {
     constexpr int kRows = 256 / (D * 2 / 16);
     const int max_rows = s.L < capv ? s.L : capv;
     const int blocks = (max_rows + kRows - 1) / kRows;
     dim3 grid(blocks < 48 ? blocks : 48, s.B * s.H);
     gather_kv_tc_kernel<D><<<grid, 256, 0, st>>>(
         (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, sm_idx, pre, (__nv_bfloat16 *)k_sm,
-        (__nv_bfloat16 *)v_sm, (__half *)v16, (__half *)k16, cap, capv, status, s.L, s.H);
+        (__nv_bfloat16 *)v_sm, (__half *)v16, (__half *)k16, cap, capv, appending ? 1 : 0, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
                                 const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
-                                void *k16, int32_t cap, int32_t capv, int32_t *status, Shape s,
-                                cudaStream_t st) {
+                                void *k16, int32_t cap, int32_t capv, bool appending, int32_t *status,
+                                Shape s, cudaStream_t st) {
     if (s.d == 128)
-        return gather_tc_impl<128>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, status, s, st);
-    return gather_tc_impl<64>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, status, s, st);
+        return gather_tc_impl<128>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st);
+    return gather_tc_impl<64>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st);
 }
 
 }  // namespace natsl

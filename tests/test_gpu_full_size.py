@@ -33,6 +33,21 @@ def test_fwd_full_size_block_routing():
     check_fwd(wl, got, ref, TOL[wl.dtype])
 
 
+def test_fwd_full_size_long_context_in_pieces():
+    """The long-context workload prefilled in four pieces of 8192 tokens (state chained, retained
+    K/V appended to one cache), every element against the oracle's forward over all 32768 tokens."""
+    from test_gpu_chunked_prefill import prefill_in_pieces
+    from test_gpu_parity import rel_err
+    wl = inputs.WORKLOADS["cfg2_bf16_long_prefill"]
+    x = inputs.make_layer_inputs(wl)
+    ref = run_oracle(wl, x, want_cache=True)
+    cap = int(ref["n_sm"].max()) + 128
+    got = prefill_in_pieces(wl, x, (8192,) * 4, cap=cap, flags=0)
+    check_stored(got["out"], ref["out"], TOL[wl.dtype], wl.dtype)
+    assert rel_err(got["state"], ref["state_out"]) <= TOL[wl.dtype]
+    assert np.array_equal(got["sm_len"], ref["n_sm"])
+
+
 def test_fwd_bwd_full_size_training_workload():
     wl = inputs.WORKLOADS["cfg4_bf16_train"]
     x = inputs.make_layer_inputs(wl)
