@@ -71,7 +71,7 @@ enum {
                                     parallel (a second run per segment yields the segment's
                                     state transition, a small kernel chains the segments); the
                                     results agree to rounding */
-    NATSL_BLOCK_ROUTING = 1u << 2,     /* forward, tensor-core path: block-level routing, the paper's
+    NATSL_BLOCK_ROUTING = 1u << 2,     /* forward (both paths): block-level routing, the paper's
                                     default (Section 4.1, "compute the inner-chunk correlation";
                                     Section 4.3, chunk size = GDN chunk size).  `route` holds one
                                     decision per block of C = 64 tokens, repeated over the block's
@@ -165,7 +165,7 @@ int natsl_score_layer(const void *x, const float *w_score, float *scores, uint8_
  *   route [B,L,H] u8; out [B,L,H,d] in p->dtype.
  * The linear branch is computed chunkwise (Section 3, chunkwise equations) with C = 64.
  * Optional outputs are taken from `p`.  Errors: NULL, SHAPE, DTYPE, ALIGN, WORKSPACE, CUDA;
- * UNSUPPORTED for NATSL_BLOCK_ROUTING off the tensor-core path (fp32 storage, NATSL_FORCE_SIMT).
+ * UNSUPPORTED for NATSL_APPEND_CACHE off the tensor-core path (fp32 storage, NATSL_FORCE_SIMT).
  */
 int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g,
                      const float *beta, const uint8_t *route, void *out,

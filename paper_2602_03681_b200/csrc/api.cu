@@ -258,7 +258,6 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     if ((p->o_la && !aligned16(p->o_la)) || (p->o_nla && !aligned16(p->o_nla))) return NATSL_ERR_ALIGN;
     const bool tensor_cores = use_tensor_cores(p);
     const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
-    if (block && !tensor_cores) return NATSL_ERR_UNSUPPORTED;
     const bool append = (p->flags & NATSL_APPEND_CACHE) != 0;
     if (append && !tensor_cores) return NATSL_ERR_UNSUPPORTED;
     if (append && !want_cache) return NATSL_ERR_NULL;
@@ -311,11 +310,11 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
                                          f.status, s, st));
         }
     } else {
-        NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, route, p->scale_la, f.W, f.U, f.P,
-                                          nullptr, nullptr, s, st));
+        NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.W,
+                                          f.U, f.P, nullptr, nullptr, s, st));
         NATSL_TRY(mark());
         NATSL_TRY(launch_gdn_scan_simt(q, k, g, f.W, f.U, f.P, p->scale_la, p->state_in,
-                                       p->state_out, nullptr, nullptr, o_la, s, st));
+                                       p->state_out, nullptr, nullptr, o_la, br.route, s, st));
     }
     NATSL_TRY(mark());
     if (tensor_cores)
@@ -324,7 +323,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
                                             f.status, s, st));
     else
         NATSL_TRY(launch_softmax_combine_simt(q, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
-                                              p->scale_sm, p->eps, out, p->o_nla, p->lse, s, st));
+                                              p->scale_sm, p->eps, out, p->o_nla, p->lse, br, s, st));
     NATSL_TRY(mark());
 #undef NATSL_TRY
     return NATSL_OK;
@@ -382,7 +381,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
                                           f.P, f.Abar, f.Gcum, s32, st));
         NATSL_TRY(launch_gdn_scan_simt(f.q32, f.k32, g, f.W, f.U, f.P, p->scale_la, nullptr, nullptr,
-                                       f.S_c, f.Ut, f.o_la, s32, st));
+                                       f.S_c, f.Ut, f.o_la, nullptr, s32, st));
     }
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la,
@@ -392,7 +391,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     else
         NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
                                               f.o_la, p->w, p->scale_sm, p->eps, nullptr, f.o_nla,
-                                              f.lse, s32, st));
+                                              f.lse, BlockRouting{nullptr, nullptr, nullptr}, s32, st));
     // ---- combination and softmax branch ----
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la,
                                  tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,

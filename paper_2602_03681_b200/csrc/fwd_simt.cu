@@ -55,7 +55,7 @@ gdn_prepare_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const 
     load_tile<T, D>(v + tok0 * D, ts, Vs);
     if (threadIdx.x < kC) {
         const size_t t = tok0 + (size_t)threadIdx.x * H;
-        bts[threadIdx.x] = route[t] ? 0.f : beta[t];
+        bts[threadIdx.x] = route && route[t] ? 0.f : beta[t];   // route == nullptr: beta~ = beta
         Gs[threadIdx.x] = g[t];
     }
     __syncthreads();
@@ -135,7 +135,8 @@ gdn_scan_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const flo
                      const float *__restrict__ W, const float *__restrict__ U,
                      const float *__restrict__ P, float scale_la, const float *__restrict__ state_in,
                      float *__restrict__ state_out, float *__restrict__ chunk_states,
-                     float *__restrict__ Ut, float *__restrict__ o_la, int L, int H) {
+                     float *__restrict__ Ut, float *__restrict__ o_la,
+                     const uint8_t *__restrict__ block_route, int L, int H) {
     extern __shared__ float smem[];
     float *Ss = smem;                        // [D][32]
     float *Ws = Ss + D * kDvs;               // [64][D+1]
@@ -243,7 +244,9 @@ gdn_scan_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const flo
             float acc[kPer];
 #pragma unroll
             for (int x = 0; x < kPer; ++x) acc[x] = gC * Ss[a * kDvs + cs + x];
-            for (int j = 0; j < kC; ++j) {
+            // block-level routing: a softmax block's update is not committed, the state only decays
+            const bool commit = !(block_route && block_route[tok0]);
+            for (int j = 0; commit && j < kC; ++j) {
                 const float kv = Ks[j * (D + 1) + a] * __expf(gl - Gs[j]);
                 const float *ur = Us + j * (kDvs + 1) + cs;
 #pragma unroll
@@ -274,7 +277,9 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
                             const int32_t *__restrict__ sm_chunk_prefix,
                             const float *__restrict__ o_la, const float *__restrict__ w,
                             float scale_sm, float eps, T *__restrict__ out,
-                            float *__restrict__ o_nla, float *__restrict__ lse, int L, int H) {
+                            float *__restrict__ o_nla, float *__restrict__ lse,
+                            const uint8_t *__restrict__ block_route, const T *__restrict__ k_tok,
+                            const T *__restrict__ v_tok, int L, int H) {
     extern __shared__ float smem[];
     float *Qs = smem;                      // [64][D]
     float *Kt = Qs + kC * D;               // [32][D+1]
@@ -302,12 +307,21 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
     }
     const T *kb = k_sm + (size_t)bh * cap * D, *vb = v_sm + (size_t)bh * cap * D;
 
-    for (int j0 = 0; j0 < n_end; j0 += 32) {
+    // Block-level routing: a query in a linear block also reads the causal part of its own block
+    // (two more tiles of 32 keys, taken from the layer's own k and v).
+    const int n_ret = (n_end + 31) / 32 * 32;
+    const int n_all = n_ret + (block_route && block_route[tok0] == 0 ? kC : 0);
+    for (int j0 = 0; j0 < n_all; j0 += 32) {
+        const bool own = j0 >= n_ret;
         __syncthreads();
         for (int idx = threadIdx.x; idx < 32 * D / 4; idx += kThreads) {
             const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
             float4 kx = make_float4(0.f, 0.f, 0.f, 0.f), vx = kx;
-            if (j0 + r < n_end) {
+            if (own) {
+                const size_t src = (tok0 + (size_t)(j0 - n_ret + r) * H) * D + c4;
+                kx = load4(k_tok + src);
+                vx = load4(v_tok + src);
+            } else if (j0 + r < n_end) {
                 kx = load4(kb + (size_t)(j0 + r) * D + c4);
                 vx = load4(vb + (size_t)(j0 + r) * D + c4);
             }
@@ -316,8 +330,9 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
             store4(Vt + r * D + c4, vx);
         }
         if (threadIdx.x < 32)
-            pos[threadIdx.x] = (j0 + threadIdx.x < n_end) ? sm_idx[(size_t)bh * L + j0 + threadIdx.x]
-                                                          : 0x7fffffff;
+            pos[threadIdx.x] = own ? c * kC + (j0 - n_ret) + (int)threadIdx.x
+                               : (j0 + threadIdx.x < n_end) ? sm_idx[(size_t)bh * L + j0 + threadIdx.x]
+                                                            : 0x7fffffff;
         __syncthreads();
         const int my_pos = pos[lane];
         const float *kr = Kt + lane * (D + 1);
@@ -421,15 +436,15 @@ cudaError_t launch_gdn_prepare_simt(const void *q, const void *k, const void *v,
 template <typename T, int D>
 static cudaError_t scan_impl(const void *q, const void *k, const float *g, const float *W,
                              const float *U, const float *P, float scale_la, const float *state_in,
-                             float *state_out, float *chunk_states, float *Ut, float *o_la, Shape s,
-                             cudaStream_t st) {
+                             float *state_out, float *chunk_states, float *Ut, float *o_la,
+                             const uint8_t *block_route, Shape s, cudaStream_t st) {
     const size_t smem = simt_scan_smem(D);
     cudaError_t e = set_smem(gdn_scan_simt_kernel<T, D>, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(D / kDvs, s.B * s.H);
     gdn_scan_simt_kernel<T, D><<<grid, kThreads, smem, st>>>(
         (const T *)q, (const T *)k, g, W, U, P, scale_la, state_in, state_out, chunk_states, Ut,
-        o_la, s.L, s.H);
+        o_la, block_route, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -437,23 +452,24 @@ static cudaError_t scan_impl(const void *q, const void *k, const float *g, const
 cudaError_t launch_gdn_scan_simt(const void *q, const void *k, const float *g, const float *W,
                                  const float *U, const float *P, float scale_la,
                                  const float *state_in, float *state_out, float *chunk_states,
-                                 float *Ut, float *o_la, Shape s, cudaStream_t st) {
+                                 float *Ut, float *o_la, const uint8_t *block_route, Shape s,
+                                 cudaStream_t st) {
     NATSL_DISPATCH(scan_impl, q, k, g, W, U, P, scale_la, state_in, state_out, chunk_states, Ut, o_la,
-                   s, st);
+                   block_route, s, st);
 }
 
 template <typename T, int D>
 static cudaError_t softmax_impl(const void *q, const void *k_sm, const void *v_sm, int32_t cap,
                                 const int32_t *sm_idx, const int32_t *pre, const float *o_la,
                                 const float *w, float scale_sm, float eps, void *out, float *o_nla,
-                                float *lse, Shape s, cudaStream_t st) {
+                                float *lse, BlockRouting br, Shape s, cudaStream_t st) {
     const size_t smem = simt_softmax_smem(D);
     cudaError_t e = set_smem(softmax_combine_simt_kernel<T, D>, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(s.L / kC, s.B * s.H);
     softmax_combine_simt_kernel<T, D><<<grid, kThreads, smem, st>>>(
         (const T *)q, (const T *)k_sm, (const T *)v_sm, cap, sm_idx, pre, o_la, w, scale_sm, eps,
-        (T *)out, o_nla, lse, s.L, s.H);
+        (T *)out, o_nla, lse, br.route, (const T *)br.k, (const T *)br.v, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -462,9 +478,10 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
                                         int32_t cap, const int32_t *sm_idx,
                                         const int32_t *sm_chunk_prefix, const float *o_la,
                                         const float *w, float scale_sm, float eps, void *out,
-                                        float *o_nla, float *lse, Shape s, cudaStream_t st) {
+                                        float *o_nla, float *lse, BlockRouting br, Shape s,
+                                        cudaStream_t st) {
     NATSL_DISPATCH(softmax_impl, q, k_sm, v_sm, cap, sm_idx, sm_chunk_prefix, o_la, w, scale_sm, eps,
-                   out, o_nla, lse, s, st);
+                   out, o_nla, lse, br, s, st);
 }
 
 }  // namespace natsl

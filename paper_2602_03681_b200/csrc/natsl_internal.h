@@ -50,12 +50,14 @@ cudaError_t launch_gdn_prepare_simt(const void *q, const void *k, const void *v,
 cudaError_t launch_gdn_scan_simt(const void *q, const void *k, const float *g, const float *W,
                                  const float *U, const float *P, float scale_la,
                                  const float *state_in, float *state_out, float *chunk_states,
-                                 float *Ut, float *o_la, Shape s, cudaStream_t st);
+                                 float *Ut, float *o_la, const uint8_t *block_route, Shape s,
+                                 cudaStream_t st);
 cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const void *v_sm,
                                         int32_t cap, const int32_t *sm_idx,
                                         const int32_t *sm_chunk_prefix, const float *o_la,
                                         const float *w, float scale_sm, float eps, void *out,
-                                        float *o_nla, float *lse, Shape s, cudaStream_t st);
+                                        float *o_nla, float *lse, BlockRouting br, Shape s,
+                                        cudaStream_t st);
 
 // softmax_tc.cu -- tensor-core softmax branch + combination (bf16 storage)
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,

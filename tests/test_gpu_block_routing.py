@@ -93,16 +93,20 @@ def test_block_routing_reports_a_route_that_changes_inside_a_block():
     assert binding.natsl_device_status(res["ws"]) == binding.ERR_ROUTE
 
 
-def test_block_routing_off_the_tensor_core_path_is_refused():
+@pytest.mark.parametrize("name,B,H,L,p,flags,tol", [
+    ("cfg0_f32_tiny_fwd", 1, 2, 256, 0.3, 0, 1e-4),       # fp32 storage: CUDA-core path, fp32 bar
+    ("cfg0_f32_tiny_fwd", 2, 1, 448, 0.5, 0, 1e-4),
+    ("cfg1_bf16_prefill", 1, 2, 320, 0.3, 1, 2e-2),       # bf16 storage forced onto the CUDA-core path
+])
+def test_block_routed_forward_on_the_cuda_core_path(name, B, H, L, p, flags, tol):
     from paper_2602_03681_b200 import binding
-    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
-    x = block_inputs(wl, 1, 1, 128, 0.5)
-    dt = tdtype(wl)
-    with pytest.raises(binding.NatslError) as ei:
-        binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]),
-                           dev(x["beta"]), dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la,
-                           scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING | binding.FORCE_SIMT)
-    assert ei.value.status == binding.ERR_UNSUPPORTED
+    wl = inputs.WORKLOADS[name]
+    x = block_inputs(wl, B, H, L, p)
+    rng = np.random.default_rng(8)
+    S0 = (0.1 * rng.standard_normal((B, H, wl.d, wl.d))).astype(np.float32)
+    ref = oracle_block(wl, x, state_in=S0.astype(np.float64))
+    got = run_fwd(wl, x, state_in=S0, flags=binding.BLOCK_ROUTING | flags)
+    check_fwd(wl, got, ref, tol)
 
 
 # ------------------------------------------------------------------ generation
