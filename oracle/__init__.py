@@ -120,8 +120,9 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5,
 
 
 def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5, state_in=None,
-               dstate_out=None):
+               dstate_out=None, block=None):
     """Analytic reverse-mode gradients of hybrid_fwd's `out` (and state_out) contraction.
+    block=R: of the block-mode forward (hybrid_fwd with the same `block`).
 
     Returns dict(dq, dk, dv [B,L,H,d]; dg, dbeta [B,L,H]; dw [B,L,H,2]; dstate_in [B,H,d,d]).
     """
@@ -133,11 +134,16 @@ def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5
     dg, dbeta = np.zeros((B, L, H)), np.zeros((B, L, H))
     dw = np.zeros((B, L, H, 2))
     dstate_in = np.zeros((B, H, d, d))
-    rc = _load().natsl_oracle_hybrid_bwd(
-        _p(q), _p(k), _p(v), _p(g), _p(beta), _p(route, _u8p), _p(w), _p(dout), B, L, H, d,
-        ctypes.c_double(scale_la), ctypes.c_double(scale_sm), ctypes.c_double(eps),
-        _p(state_in), _p(dstate_out), _p(dq), _p(dk), _p(dv), _p(dg), _p(dbeta), _p(dw),
-        _p(dstate_in))
+    head = (_p(q), _p(k), _p(v), _p(g), _p(beta), _p(route, _u8p), _p(w), _p(dout), B, L, H, d)
+    tail = (ctypes.c_double(scale_la), ctypes.c_double(scale_sm), ctypes.c_double(eps),
+            _p(state_in), _p(dstate_out), _p(dq), _p(dk), _p(dv), _p(dg), _p(dbeta), _p(dw),
+            _p(dstate_in))
+    if block is None:
+        rc = _load().natsl_oracle_hybrid_bwd(*head, *tail)
+    else:
+        rc = _load().natsl_oracle_hybrid_bwd_block(*head, int(block), *tail)
+    if rc == -4:
+        raise ValueError("block mode: route must be constant within each block")
     if rc != 0:
         raise RuntimeError(f"natsl_oracle_hybrid_bwd failed ({rc})")
     return dict(dq=dq, dk=dk, dv=dv, dg=dg, dbeta=dbeta, dw=dw, dstate_in=dstate_in)

@@ -538,3 +538,216 @@ int natsl_oracle_hybrid_bwd(const double *q, const double *k, const double *v,
     }
     return err ? -2 : 0;
 }
+
+/* ---------------------------------------------------------------------------
+ * Analytic backward of natsl_oracle_hybrid_fwd_block (reverse mode, token by token): the chain
+ * rule applied to that forward, statement by statement, in reverse order.
+ *   - softmax branch: query i reads key j <= i when j's block is a softmax block or j is in i's
+ *     own block; ds = p (dp - <do, o>) as in the token-level backward (Section 4.2).
+ *   - linear branch: inside a block the delta rule runs over every token from the block's start
+ *     state.  A linear block hands its last state on, so the state gradient flows back through
+ *     the block's tokens.  A softmax block hands on exp(sum g) * (start state): the incoming
+ *     gradient goes straight to the start state (times the decay) and to every g of the block;
+ *     the block's own token chain receives gradient from its outputs only.
+ * Arguments as natsl_oracle_hybrid_bwd, plus the block length R.
+ * ------------------------------------------------------------------------- */
+int natsl_oracle_hybrid_bwd_block(const double *q, const double *k, const double *v,
+                                  const double *g, const double *beta, const uint8_t *route,
+                                  const double *w, const double *dout, int B, int L, int H, int d,
+                                  int R, double scale_la, double scale_sm, double eps,
+                                  const double *state_in, const double *dstate_out,
+                                  double *dq, double *dk, double *dv, double *dg, double *dbeta,
+                                  double *dw, double *dstate_in)
+{
+    if (d > 512 || d <= 0 || R <= 0 || L % R != 0) return -1;
+    int err = 0, bad_route = 0;
+    size_t dd = (size_t)d * d;
+    int NB = L / R;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int bh = 0; bh < B * H; ++bh) {
+        int b = bh / H, h = bh % H;
+        double *after = (double *)malloc(sizeof(double) * dd * (size_t)L);        /* state after token i */
+        double *start = (double *)malloc(sizeof(double) * dd * (size_t)(NB + 1)); /* state at block starts */
+        double *o_la = (double *)malloc(sizeof(double) * (size_t)L * d);
+        double *o_nla = (double *)malloc(sizeof(double) * (size_t)L * d);
+        double *do_la = (double *)malloc(sizeof(double) * (size_t)L * d);
+        double *do_nla = (double *)malloc(sizeof(double) * (size_t)L * d);
+        double *lse = (double *)malloc(sizeof(double) * (size_t)L);
+        double *dS = (double *)calloc(dd, sizeof(double));
+        double *dC = (double *)malloc(sizeof(double) * dd);
+        double *Sbar = (double *)malloc(sizeof(double) * dd);
+        double *p = (double *)malloc(sizeof(double) * (size_t)(L + 1));
+        if (!after || !start || !o_la || !o_nla || !do_la || !do_nla || !lse || !dS || !dC || !Sbar || !p) {
+            err = 1;
+            goto done;
+        }
+        /* ---- forward recomputation, keeping every state ---- */
+        if (state_in) memcpy(start, state_in + (size_t)bh * dd, sizeof(double) * dd);
+        else memset(start, 0, sizeof(double) * dd);
+        for (int c = 0; c < NB; ++c) {
+            int i0 = c * R, r = route[AT3(b, i0, h)] != 0;
+            double g_block = 0.0;
+            for (int i = i0; i < i0 + R; ++i) {
+                size_t t = AT3(b, i, h);
+                if ((route[t] != 0) != r) bad_route = 1;
+                const double *qi = q + t * d, *ki = k + t * d, *vi = v + t * d;
+                const double *Sp = i == i0 ? start + dd * c : after + dd * (i - 1);
+                double *Sn = after + dd * i;
+                double alpha = exp(g[t]);
+                g_block += g[t];
+                for (size_t a = 0; a < dd; ++a) Sn[a] = alpha * Sp[a];
+                for (int cc = 0; cc < d; ++cc) {
+                    double ks = 0.0;
+                    for (int a = 0; a < d; ++a) ks += ki[a] * Sn[(size_t)a * d + cc];
+                    double e = vi[cc] - ks;
+                    for (int a = 0; a < d; ++a) Sn[(size_t)a * d + cc] += beta[t] * ki[a] * e;
+                }
+                for (int cc = 0; cc < d; ++cc) {
+                    double acc = 0.0;
+                    for (int a = 0; a < d; ++a) acc += qi[a] * Sn[(size_t)a * d + cc];
+                    o_la[(size_t)i * d + cc] = scale_la * acc;
+                    o_nla[(size_t)i * d + cc] = 0.0;
+                }
+                /* softmax branch: keys of softmax blocks and of the own block, j <= i */
+                double m = -INFINITY;
+                for (int j = 0; j <= i; ++j) {
+                    size_t tj = AT3(b, j, h);
+                    p[j] = -INFINITY;
+                    if (!(route[tj] || j >= i0)) continue;
+                    const double *kj = k + tj * d;
+                    double sc = 0.0;
+                    for (int a = 0; a < d; ++a) sc += qi[a] * kj[a];
+                    p[j] = scale_sm * sc;
+                    if (p[j] > m) m = p[j];
+                }
+                double z = 0.0;
+                for (int j = 0; j <= i; ++j) if (p[j] > -INFINITY) { p[j] = exp(p[j] - m); z += p[j]; } else p[j] = 0.0;
+                for (int j = 0; j <= i; ++j) {
+                    if (p[j] == 0.0) continue;
+                    const double *vj = v + AT3(b, j, h) * d;
+                    for (int cc = 0; cc < d; ++cc) o_nla[(size_t)i * d + cc] += p[j] / z * vj[cc];
+                }
+                lse[i] = m + log(z);               /* the own token is always visible: z > 0 */
+            }
+            double *Snext = start + dd * (c + 1);
+            if (r) {
+                double decay = exp(g_block);
+                for (size_t a = 0; a < dd; ++a) Snext[a] = decay * start[dd * c + a];
+            } else {
+                memcpy(Snext, after + dd * (i0 + R - 1), sizeof(double) * dd);
+            }
+        }
+        /* ---- combination backward, row by row (as in the token-level backward) ---- */
+        for (int i = 0; i < L; ++i) {
+            size_t t = AT3(b, i, h);
+            double wn = w ? w[t * 2] : 0.5, wl = w ? w[t * 2 + 1] : 0.5;
+            const double *ol = o_la + (size_t)i * d, *on = o_nla + (size_t)i * d;
+            const double *dy = dout + t * d;
+            double fl = rms_factor(ol, d, eps), fn = rms_factor(on, d, eps);
+            double dwn = 0.0, dwl = 0.0, ml = 0.0, mn = 0.0;
+            for (int c = 0; c < d; ++c) {
+                dwn += dy[c] * on[c] * fn;
+                dwl += dy[c] * ol[c] * fl;
+                mn += wn * dy[c] * on[c] * fn;
+                ml += wl * dy[c] * ol[c] * fl;
+            }
+            mn /= d; ml /= d;
+            for (int c = 0; c < d; ++c) {
+                do_nla[(size_t)i * d + c] = fn * (wn * dy[c] - on[c] * fn * mn);
+                do_la[(size_t)i * d + c] = fl * (wl * dy[c] - ol[c] * fl * ml);
+            }
+            if (dw) { dw[t * 2] = dwn; dw[t * 2 + 1] = dwl; }
+        }
+        for (int i = 0; i < L; ++i) {
+            size_t t = AT3(b, i, h);
+            for (int a = 0; a < d; ++a) { dq[t * d + a] = 0.0; dk[t * d + a] = 0.0; dv[t * d + a] = 0.0; }
+            dg[t] = 0.0;
+        }
+        /* ---- softmax branch backward ---- */
+        for (int i = 0; i < L; ++i) {
+            size_t t = AT3(b, i, h);
+            int i0 = i / R * R;
+            const double *qi = q + t * d;
+            const double *doi = do_nla + (size_t)i * d, *oi = o_nla + (size_t)i * d;
+            double D = 0.0;
+            for (int c = 0; c < d; ++c) D += doi[c] * oi[c];
+            for (int j = 0; j <= i; ++j) {
+                size_t tj = AT3(b, j, h);
+                if (!(route[tj] || j >= i0)) continue;
+                const double *kj = k + tj * d, *vj = v + tj * d;
+                double sc = 0.0, dp = 0.0;
+                for (int a = 0; a < d; ++a) sc += qi[a] * kj[a];
+                double pij = exp(scale_sm * sc - lse[i]);
+                for (int c = 0; c < d; ++c) dp += doi[c] * vj[c];
+                double ds = pij * (dp - D);
+                for (int c = 0; c < d; ++c) dv[tj * d + c] += pij * doi[c];
+                for (int a = 0; a < d; ++a) {
+                    dq[t * d + a] += scale_sm * ds * kj[a];
+                    dk[tj * d + a] += scale_sm * ds * qi[a];
+                }
+            }
+        }
+        /* ---- linear branch backward: blocks in reverse order ---- */
+        if (dstate_out) memcpy(dS, dstate_out + (size_t)bh * dd, sizeof(double) * dd);
+        for (int c = NB - 1; c >= 0; --c) {
+            int i0 = c * R, r = route[AT3(b, i0, h)] != 0;
+            double dg_block = 0.0;
+            if (r) {
+                /* next start = exp(sum g) * start_c: straight to the start state and to every g */
+                double g_block = 0.0, acc = 0.0;
+                for (int i = i0; i < i0 + R; ++i) g_block += g[AT3(b, i, h)];
+                double decay = exp(g_block);
+                for (size_t a = 0; a < dd; ++a) {
+                    acc += dS[a] * start[dd * c + a];
+                    dC[a] = decay * dS[a];
+                    dS[a] = 0.0;                   /* the block's own chain feeds nothing later */
+                }
+                dg_block = decay * acc;
+            } else {
+                memset(dC, 0, sizeof(double) * dd);
+            }
+            for (int i = i0 + R - 1; i >= i0; --i) {
+                size_t t = AT3(b, i, h);
+                const double *qi = q + t * d, *ki = k + t * d, *vi = v + t * d;
+                const double *Sp = i == i0 ? start + dd * c : after + dd * (i - 1);
+                const double *Sn = after + dd * i;
+                const double *doi = do_la + (size_t)i * d;
+                double alpha = exp(g[t]), bt = beta[t];
+                for (int a = 0; a < d; ++a) {
+                    double acc = 0.0;
+                    for (int cc = 0; cc < d; ++cc) acc += doi[cc] * Sn[(size_t)a * d + cc];
+                    dq[t * d + a] += scale_la * acc;
+                    for (int cc = 0; cc < d; ++cc) dS[(size_t)a * d + cc] += scale_la * qi[a] * doi[cc];
+                }
+                for (size_t a = 0; a < dd; ++a) Sbar[a] = alpha * Sp[a];
+                double dbt = 0.0;
+                for (int cc = 0; cc < d; ++cc) {
+                    double ks = 0.0, kds = 0.0;
+                    for (int a = 0; a < d; ++a) {
+                        ks += ki[a] * Sbar[(size_t)a * d + cc];
+                        kds += ki[a] * dS[(size_t)a * d + cc];
+                    }
+                    double e = vi[cc] - ks;
+                    double de = bt * kds;
+                    dbt += kds * e;
+                    dv[t * d + cc] += de;
+                    for (int a = 0; a < d; ++a)
+                        dk[t * d + a] += bt * e * dS[(size_t)a * d + cc] - de * Sbar[(size_t)a * d + cc];
+                    for (int a = 0; a < d; ++a) dS[(size_t)a * d + cc] -= ki[a] * de;
+                }
+                double da = 0.0;
+                for (size_t a = 0; a < dd; ++a) da += dS[a] * Sp[a];
+                dg[t] = alpha * da + dg_block;
+                dbeta[t] = dbt;
+                for (size_t a = 0; a < dd; ++a) dS[a] *= alpha;
+            }
+            for (size_t a = 0; a < dd; ++a) dS[a] += dC[a];
+        }
+        if (dstate_in) memcpy(dstate_in + (size_t)bh * dd, dS, sizeof(double) * dd);
+    done:
+        free(after); free(start); free(o_la); free(o_nla); free(do_la); free(do_nla); free(lse);
+        free(dS); free(dC); free(Sbar); free(p);
+    }
+    if (err) return -2;
+    return bad_route ? -4 : 0;
+}

@@ -647,3 +647,62 @@ def test_score_layer_closed_forms_and_brute_force():
     w1[0, 1, 7] = 2.0
     r2 = router.score_layer(x, w1, C)
     assert np.array_equal(r2["route"][:, ::C, 0] == 1, x[..., 7].reshape(B, L // C, C).mean(-1) > 0)
+
+
+def test_block_mode_backward_finite_differences():
+    B, L, H, d, R = 1, 20, 2, 5, 4
+    x = rand_inputs(B, L, H, d, seed=36, unit=False)
+    x["q"] *= 0.5
+    x["k"] *= 0.4
+    x["route"] = _block_route(B, L, H, R, 0.5, seed=7)
+    assert 0 < x["route"].sum() < x["route"].size
+    dout = RNG.standard_normal((B, L, H, d))
+    S0 = RNG.standard_normal((B, H, d, d)) * 0.3
+    dS = RNG.standard_normal((B, H, d, d))
+
+    def loss():
+        r = fwd(x, state_in=S0, block=R)
+        return (r["out"] * dout).sum() + (r["state_out"] * dS).sum()
+
+    gr = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], dout,
+                           scale_la=0.5, scale_sm=1.5, state_in=S0, dstate_out=dS, block=R)
+    h = 1e-6
+    pick = np.random.default_rng(9)
+    arrays = [(x[n], gr[gn], n) for n, gn in [("q", "dq"), ("k", "dk"), ("v", "dv"), ("g", "dg"),
+                                              ("beta", "dbeta"), ("w", "dw")]]
+    arrays.append((S0, gr["dstate_in"], "state_in"))
+    for arr, grad, name in arrays:
+        flat = arr.reshape(-1)
+        for idx in pick.choice(flat.size, size=min(40, flat.size), replace=False):
+            old = flat[idx]
+            flat[idx] = old + h
+            lp = loss()
+            flat[idx] = old - h
+            lm = loss()
+            flat[idx] = old
+            fd, an = (lp - lm) / (2 * h), grad.reshape(-1)[idx]
+            assert abs(fd - an) <= 2e-6 * max(1.0, abs(an)) + 1e-7, (name, idx, fd, an)
+
+
+def test_block_mode_backward_special_cases():
+    B, L, H, d, R = 1, 24, 2, 6, 8
+    x = rand_inputs(B, L, H, d, seed=37)
+    dout = RNG.standard_normal((B, L, H, d))
+    kw = dict(scale_la=0.5, scale_sm=1.5)
+    args = lambda y: (y["q"], y["k"], y["v"], y["g"], y["beta"], y["route"], y["w"], dout)
+    # all blocks linear, only the linear branch weighted: the token-level backward of pure GDN
+    x["route"] = np.zeros((B, L, H), np.uint8)
+    x["w"] = np.stack([np.zeros_like(x["g"]), np.ones_like(x["g"])], -1)
+    gb = oracle.hybrid_bwd(*args(x), block=R, **kw)
+    gt = oracle.hybrid_bwd(*args(x), **kw)
+    for n in ("dq", "dk", "dv", "dg", "dbeta"):
+        np.testing.assert_allclose(gb[n], gt[n], rtol=1e-10, atol=1e-13, err_msg=n)
+    # all blocks softmax, only the softmax branch weighted: the token-level backward of causal
+    # attention (every token retained); nothing reaches g or beta
+    x["route"] = np.ones((B, L, H), np.uint8)
+    x["w"] = np.stack([np.ones_like(x["g"]), np.zeros_like(x["g"])], -1)
+    gb = oracle.hybrid_bwd(*args(x), block=R, **kw)
+    gt = oracle.hybrid_bwd(*args(x), **kw)
+    for n in ("dq", "dk", "dv"):
+        np.testing.assert_allclose(gb[n], gt[n], rtol=1e-10, atol=1e-13, err_msg=n)
+    assert np.all(gb["dg"] == 0) and np.all(gb["dbeta"] == 0)
