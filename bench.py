@@ -418,7 +418,8 @@ def bench_other_workloads(peaks):
     res = {}
     dt = torch.bfloat16
     for name, ops in (("cfg2_bf16_long_prefill", ("fwd",)), ("cfg4_bf16_train", ("fwd", "bwd")),
-                      ("cfg1_bf16_prefill/block_routing", ("fwd",))):
+                      ("cfg1_bf16_prefill/block_routing", ("fwd",)),
+                      ("cfg4_bf16_train/block_routing", ("fwd", "bwd"))):
         block = name.endswith("/block_routing")          # the same shapes, one route per 64 tokens
         wl = inputs.WORKLOADS[name.split("/")[0]]
         x = inputs.make_layer_inputs(
@@ -437,7 +438,9 @@ def bench_other_workloads(peaks):
             else:
                 ws["bwd"] = binding.hybrid_bwd(d["q"], d["k"], d["v"], d["g"], d["beta"], d["route"],
                                                d["w"], d["dout"], scale_la=wl.scale_la,
-                                               scale_sm=wl.scale_sm, ws=ws["bwd"])["ws"]
+                                               scale_sm=wl.scale_sm,
+                                               flags=binding.BLOCK_ROUTING if block else 0,
+                                               ws=ws["bwd"])["ws"]
 
         ms = {}
         for op in ops:

@@ -337,7 +337,10 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (rc != NATSL_OK) return rc;
     if (!q || !k || !v || !g || !beta || !route || !dout || !dq || !dk || !dv || !dg || !dbeta)
         return NATSL_ERR_NULL;
-    if (p->state_in || (p->flags & (NATSL_BLOCK_ROUTING | NATSL_APPEND_CACHE))) return NATSL_ERR_UNSUPPORTED;
+    if (p->state_in || (p->flags & NATSL_APPEND_CACHE)) return NATSL_ERR_UNSUPPORTED;
+    // block-level routing: on the path with the fused chunk kernel only (bf16 storage, d = 64)
+    const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
+    if (block && !(use_tensor_cores(p) && p->d == 64)) return NATSL_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
         return NATSL_ERR_ALIGN;
@@ -358,7 +361,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
     // ---- forward recomputation, keeping what the backward needs ----
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, nullptr,
-                                   nullptr, p->B, p->L, p->H, st));
+                                   block ? f.status : nullptr, p->B, p->L, p->H, st));
+    const uint8_t *block_route = block ? route : nullptr;
     const bool tensor_cores = use_tensor_cores(p);
     const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
     if (!fused_chunks)
@@ -373,10 +377,11 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         // the fused chunk kernel reads W^T, U^T as the forward keeps them: no fp32 copies for it
         const GdnTcExport ex{fused_chunks ? nullptr : f.W, fused_chunks ? nullptr : f.U, nullptr, f.Tinv,
                              f.Gcum, f.S_c, f.Ut};
-        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, route, p->scale_la, f.tc, ex, f.status, s, st));
+        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc, ex,
+                                        f.status, s, st));
         NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex,
-                                     ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, nullptr, f.status,
-                                     s, st));
+                                     ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, block_route,
+                                     f.status, s, st));
     } else {
         NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
                                           f.P, f.Abar, f.Gcum, s32, st));
@@ -386,15 +391,14 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la,
                                             p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
-                                            BlockRouting{nullptr, nullptr, nullptr}, false, f.status, s,
-                                            st));
+                                            BlockRouting{block_route, k, v}, false, f.status, s, st));
     else
         NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
                                               f.o_la, p->w, p->scale_sm, p->eps, nullptr, f.o_nla,
                                               f.lse, BlockRouting{nullptr, nullptr, nullptr}, s32, st));
     // ---- combination and softmax branch ----
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la,
-                                 tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,
+                                 tensor_cores && !block ? nullptr : f.do_nla, dw, f.Dsm,
                                  tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
                                  tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, s, st));
     if (tensor_cores)
@@ -406,17 +410,31 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     // ---- linear branch: reverse scan, then chunk-parallel products ----
     if (tensor_cores)
         NATSL_TRY(launch_gdn_rscan_tc(f.dOla16, f.dOlag16, f.tc, f.S_c, f.dUt, f.dS_c,
-                                      fused_chunks ? nullptr : f.gS, f.status, s, st));
+                                      fused_chunks ? nullptr : f.gS, block_route, f.status, s, st));
     else
         NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
                                    f.dS_c, f.gS, s, st));
     AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
                    f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
                    p->scale_la, f.dGrow, f.kappa, dbeta, dg};
+    if (fused_chunks && block) {
+        // Every token has a softmax-branch dk, dv here: the retained tokens' from the compacted
+        // gradients, the tokens of linear blocks' from their own block.  Both go to fp32
+        // token-major buffers (each token is written by exactly one of the two), which the chunk
+        // kernel adds to its own dk, dv.
+        float *dk_x = f.X3, *dv_x = f.X4;
+        NATSL_TRY(launch_gdn_finish(a, dk_x, dv_x, s32, st, false));
+        NATSL_TRY(launch_softmax_bwd_own_block(q, k, v, f.do_nla, f.lse, f.Dsm, route, p->scale_sm,
+                                               f.dq_sm, dk_x, dv_x, s, st));
+        NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
+                                       f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
+                                       true, dk_x, dv_x, s, st));
+        return NATSL_OK;
+    }
     if (fused_chunks) {   // all chunk-level products and the assembly in one kernel per chunk
         NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
-                                       s, st));
+                                       false, nullptr, nullptr, s, st));
         NATSL_TRY(launch_gdn_finish(a, dk, dv, s, st, false));   // scatter of the retained tokens' dk, dv
         return NATSL_OK;
     }

@@ -54,7 +54,7 @@ struct RsMisc {
 };
 static_assert(sizeof(RsMisc) <= kRsMisc, "misc page too small");
 
-template <int D>
+template <int D, bool kBlock>      // kBlock: block-level routing (softmax blocks were not committed)
 __global__ void __launch_bounds__(kRsThreads, 1)
 gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) [B*H*L][D], box 64
                     const __grid_constant__ CUtensorMap map_dog,   // scale_la gamma dO (fp16), box 64
@@ -62,7 +62,7 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
                     const __grid_constant__ CUtensorMap map_wt,    // W^T [B*H*NC*D][64], box D
                     const __grid_constant__ CUtensorMap map_ph,    // P [B*H*NC*64][64], box 64
                     const float *__restrict__ Gd, float *__restrict__ dUt, float *__restrict__ dS_c,
-                    int32_t *status, int L, int H) {
+                    const uint8_t *__restrict__ block_route, int32_t *status, int L, int H) {
     using SL = RsLayout<D>;
     constexpr int KB = SL::KB;
     constexpr int kHalfCols = D / 2;
@@ -168,6 +168,9 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
             const int c = NC - 1 - n, s = n % kRsStages;
             const float *e1 = reinterpret_cast<const float *>(smem + SL::oG + (n % kRsDecaySlots) * SL::kG);
             const float *e2 = e1 + 64;
+            // block-level routing: the update K~^T U~ of a softmax block never reached the state,
+            // so the exit-state gradient does not flow into its dU~ (it still decays into dS0)
+            const float commit = kBlock && block_route[((size_t)b * L + (size_t)c * 64) * H + h] ? 0.f : 1.f;
             // ---- dS1 (exit-state gradient of chunk c): fp16 operand into TMEM, then (behind the
             // arrival, off the chain) the fp32 copy the later products read ----
             {
@@ -208,7 +211,8 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
-                    du[j] = fmaf(e2[tk0 + j], __uint_as_float(x2[j]), __uint_as_float(x1[j]));
+                    du[j] = fmaf(kBlock ? commit * e2[tk0 + j] : e2[tk0 + j], __uint_as_float(x2[j]),
+                                 __uint_as_float(x1[j]));
                 uint32_t pk[16];
 #pragma unroll
                 for (int x = 0; x < 16; ++x) pk[x] = pack_half2(du[2 * x], du[2 * x + 1]);
@@ -306,6 +310,11 @@ struct ChunkBwdArgs {
     __nv_bfloat16 *dq, *dk, *dv;
     float *dg, *dbeta;
     int L, H;
+    // Block-level routing (kernel instantiated with kBlock): every token takes part in the delta rule (beta~ = beta), a
+    // softmax block's update was not committed (its exit-state gradient reaches nothing but the
+    // decay), and every token's dk, dv also has a softmax-branch part, given in dk_x, dv_x
+    // (fp32, token-major).
+    const float *dk_x, *dv_x;
 };
 
 // acc (16 x 32 block at (row0, n0) of a 64 x 64 result) += A B over k = 0..63, fp16 tiles.
@@ -338,6 +347,7 @@ __device__ __forceinline__ float pow2_scale(float amax) {   // power of two s wi
     return ldexpf(1.f, -min(max(e, -100), 100));
 }
 
+template <bool kBlock>   // kBlock: block-level routing (see ChunkBwdArgs)
 __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdArgs p) {
     constexpr int D = 64;
     extern __shared__ __align__(16) uint8_t smraw[];
@@ -388,7 +398,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
         if (tid < 64) {
             const size_t tk = ((size_t)b * p.L + (size_t)c * kC + tid) * p.H + h;
             sG[tid] = p.Gcum[(size_t)bh * p.L + c * kC + tid];
-            sBt[tid] = p.route[tk] ? 0.f : p.beta[tk];
+            sBt[tid] = !kBlock && p.route[tk] ? 0.f : p.beta[tk];
             rG[tid] = 0.f; rK[tid] = 0.f; rB[tid] = 0.f;
         }
         const float mo = warp_max(amax4(xo)), mu = warp_max(amax4(xu)), msx = warp_max(amax4(xs));
@@ -409,7 +419,8 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
         scO = pow2_scale(a0); scU = pow2_scale(a1); scS = pow2_scale(a2);
         st_tile(sDO, xo, scO);
         st_tile(sDU, xu, scU);
-        st_tile(sDS1, xs, scS);
+        // (an uncommitted block: the tile is zero, so dK~ and kappa vanish; <dS1, S0> above does not)
+        st_tile(sDS1, xs, kBlock && p.route[((size_t)b * p.L + (size_t)c * kC) * p.H + h] ? 0.f : scS);
         // next batch into the freed registers: W^T and U^T as the forward kernels keep them (fp16
         // [d][64] tile; fp32 in 4-token pieces [16][d][4]) -- both are [k][n] operands as they are
         uint4 wt[2];
@@ -616,7 +627,8 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
     float4 dqs[4];                                                 // softmax-branch dq, on its way early
 #pragma unroll
     for (int x = 0; x < 4; ++x) dqs[x] = *reinterpret_cast<const float4 *>(p.dq_sm + eoff + 4 * x);
-    const bool lin = p.route[((size_t)b * p.L + (size_t)c * kC + er) * p.H + h] == 0;
+    const bool lin = kBlock || p.route[((size_t)b * p.L + (size_t)c * kC + er) * p.H + h] == 0;
+
     __syncthreads();                                               // all products have read their operands
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
@@ -630,12 +642,17 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
     }
     __syncthreads();
     {
-        auto row16 = [&](const float *tile, const float4 *add, __nv_bfloat16 *dst) {
+        // add: values already in registers; gadd: fp32 token-major tensor read here (block routing)
+        auto row16 = [&](const float *tile, const float4 *add, const float *gadd, __nv_bfloat16 *dst) {
             uint32_t o[8];
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
                 float4 v4 = *reinterpret_cast<const float4 *>(tile + er * kLdF + ec + 4 * x);
                 if (add) { v4.x += add[x].x; v4.y += add[x].y; v4.z += add[x].z; v4.w += add[x].w; }
+                if (gadd) {
+                    const float4 y = *reinterpret_cast<const float4 *>(gadd + eoff + 4 * x);
+                    v4.x += y.x; v4.y += y.y; v4.z += y.z; v4.w += y.w;
+                }
                 o[2 * x] = pack_bf162(v4.x, v4.y);
                 o[2 * x + 1] = pack_bf162(v4.z, v4.w);
             }
@@ -643,10 +660,10 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
             d4[0] = make_uint4(o[0], o[1], o[2], o[3]);
             d4[1] = make_uint4(o[4], o[5], o[6], o[7]);
         };
-        row16(fDQ, dqs, p.dq);
+        row16(fDQ, dqs, nullptr, p.dq);
         if (lin) {
-            row16(fDK, nullptr, p.dk);
-            row16(fDV, nullptr, p.dv);
+            row16(fDK, nullptr, kBlock ? p.dk_x : nullptr, p.dk);
+            row16(fDV, nullptr, kBlock ? p.dv_x : nullptr, p.dv);
         }
     }
     __syncthreads();
@@ -667,7 +684,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
         const float extra = sMax[34] + sMax[35] + exp_ftz(sG[63]) * gs + (warp == 0 ? sMax[33] : 0.f);
         const size_t tk = ((size_t)b * p.L + (size_t)c * kC + tid) * p.H + h;
         p.dg[tk] = suf + extra;
-        p.dbeta[tk] = p.route[tk] ? 0.f : rB[tid];
+        p.dbeta[tk] = !kBlock && p.route[tk] ? 0.f : rB[tid];
     }
 }
 
@@ -676,7 +693,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
 template <int D>
 static cudaError_t rscan_tc_impl(const void *dO16, const void *dOg16, const GdnTcWs &ws,
                                  const float *S_c, float *dUt, float *dS_c, float *gS,
-                                 int32_t *status, Shape s, cudaStream_t st) {
+                                 const uint8_t *block_route, int32_t *status, Shape s, cudaStream_t st) {
     const int NC = s.L / kC;
     const uint64_t BH = (uint64_t)s.B * s.H;
     CUtensorMap mdo, mdog, mqh, mkh, mwt, mph;
@@ -684,11 +701,12 @@ static cudaError_t rscan_tc_impl(const void *dO16, const void *dOg16, const GdnT
         !tch::make_map_2d(&mqh, ws.Qh, BH * s.L, D, 64) || !tch::make_map_2d(&mkh, ws.Kh, BH * s.L, D, 64) ||
         !tch::make_map_2d(&mwt, ws.Wt, BH * NC * D, 64, D) || !tch::make_map_2d(&mph, ws.Ph, BH * NC * 64, 64, 64))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(gdn_rscan_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    auto kernel = block_route ? gdn_rscan_tc_kernel<D, true> : gdn_rscan_tc_kernel<D, false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          RsLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
-    gdn_rscan_tc_kernel<D><<<s.B * s.H, kRsThreads, RsLayout<D>::kTotal, st>>>(
-        mdo, mdog, mqh, mkh, mwt, mph, ws.Gd, dUt, dS_c, status, s.L, s.H);
+    kernel<<<s.B * s.H, kRsThreads, RsLayout<D>::kTotal, st>>>(
+        mdo, mdog, mqh, mkh, mwt, mph, ws.Gd, dUt, dS_c, block_route, status, s.L, s.H);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (gS) {     // (the fused chunk kernel forms <dS1, S0> itself)
@@ -700,9 +718,9 @@ static cudaError_t rscan_tc_impl(const void *dO16, const void *dOg16, const GdnT
 
 cudaError_t launch_gdn_rscan_tc(const void *dO16, const void *dOg16, const GdnTcWs &ws,
                                 const float *S_c, float *dUt, float *dS_c, float *gS,
-                                int32_t *status, Shape s, cudaStream_t st) {
-    if (s.d == 128) return rscan_tc_impl<128>(dO16, dOg16, ws, S_c, dUt, dS_c, gS, status, s, st);
-    return rscan_tc_impl<64>(dO16, dOg16, ws, S_c, dUt, dS_c, gS, status, s, st);
+                                const uint8_t *block_route, int32_t *status, Shape s, cudaStream_t st) {
+    if (s.d == 128) return rscan_tc_impl<128>(dO16, dOg16, ws, S_c, dUt, dS_c, gS, block_route, status, s, st);
+    return rscan_tc_impl<64>(dO16, dOg16, ws, S_c, dUt, dS_c, gS, block_route, status, s, st);
 }
 
 
@@ -711,16 +729,18 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
                                  const float *Tinv, const void *Wt, const float *Up, const float *Gcum,
                                  const float *beta, const uint8_t *route, const float *dq_sm,
                                  float scale_la, void *dq, void *dk, void *dv, float *dg,
-                                 float *dbeta, Shape s, cudaStream_t st) {
+                                 float *dbeta, bool block, const float *dk_x, const float *dv_x, Shape s,
+                                 cudaStream_t st) {
     if (s.d != 64 || !s.bf16) return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(gdn_bwd_chunk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    auto kernel = block ? gdn_bwd_chunk_kernel<true> : gdn_bwd_chunk_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kCkSmem);
     if (e != cudaSuccess) return e;
     ChunkBwdArgs a{(const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, dO, dUt, Ut,
                    S_c, dS_c, Tinv, Up, Gcum, beta, dq_sm, (const __half *)Wt, route, scale_la, (__nv_bfloat16 *)dq,
-                   (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, dg, dbeta, s.L, s.H};
+                   (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, dg, dbeta, s.L, s.H, dk_x, dv_x};
     dim3 grid(s.L / kC, s.B * s.H);
-    gdn_bwd_chunk_kernel<<<grid, kCkThreads, kCkSmem, st>>>(a);
+    kernel<<<grid, kCkThreads, kCkSmem, st>>>(a);
     count_launch();
     return cudaGetLastError();
 }

@@ -154,7 +154,7 @@ cudaError_t launch_gdn_rscan(const float *q32, const float *k32, const float *Gc
 // gradient and of scale_la gamma times it; outputs as launch_gdn_rscan (gS: slot 0 of each row).
 cudaError_t launch_gdn_rscan_tc(const void *dO16, const void *dOg16, const GdnTcWs &ws,
                                 const float *S_c, float *dUt, float *dS_c, float *gS,
-                                int32_t *status, Shape s, cudaStream_t st);
+                                const uint8_t *block_route, int32_t *status, Shape s, cudaStream_t st);
 cudaError_t launch_gdn_tsolve(const float *Abar, const float *beta, const uint8_t *route,
                               const float *dW, const float *dUt, float *dKb, float *dVb, Shape s,
                               cudaStream_t st);
@@ -185,7 +185,15 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
                                  const float *Tinv, const void *Wt, const float *Up, const float *Gcum,
                                  const float *beta, const uint8_t *route, const float *dq_sm,
                                  float scale_la, void *dq, void *dk, void *dv, float *dg,
-                                 float *dbeta, Shape s, cudaStream_t st);
+                                 float *dbeta, bool block, const float *dk_x, const float *dv_x, Shape s,
+                                 cudaStream_t st);
+
+// softmax_bwd_own.cu -- block-level routing: softmax-branch backward through the own block of the
+// queries of a linear block (adds to dq_sm, writes dk_x / dv_x rows of the linear blocks)
+cudaError_t launch_softmax_bwd_own_block(const void *q, const void *k, const void *v,
+                                         const float *do_nla, const float *lse, const float *Dsm,
+                                         const uint8_t *route, float scale_sm, float *dq_sm,
+                                         float *dk_x, float *dv_x, Shape s, cudaStream_t st);
 
 // decode.cu
 constexpr int kDecodeParts = 4;   // CTAs that share the retained K/V of one (sequence, head)

@@ -190,3 +190,36 @@ def test_block_end_without_the_blocks_entries_is_reported():
                                    torch.zeros((1, 1), device="cuda"), state, state.clone(), n, 64, p, ws)
     assert binding.natsl_device_status(ws) == binding.ERR_ROUTE
     assert n.item() == 10
+
+
+# ------------------------------------------------------------------ backward
+@pytest.mark.parametrize("B,H,L,p", [(1, 2, 256, 0.4), (2, 3, 512, 0.25), (1, 1, 64, 0.0), (1, 2, 192, 1.0)])
+def test_block_routed_backward_matches_oracle(B, H, L, p):
+    """Backward under block-level routing (bf16 storage, d = 64: the path with the fused chunk
+    kernel) against the oracle's block-mode backward."""
+    from paper_2602_03681_b200 import binding
+    from test_gpu_parity import check_bwd, run_bwd
+    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+    x = block_inputs(wl, B, H, L, p)
+    if p in (0.0, 1.0):
+        x["route"][:] = int(p)
+    ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                            scale_la=wl.scale_la, scale_sm=wl.scale_sm, block=64)
+    got = run_bwd(wl, x, flags=binding.BLOCK_ROUTING)
+    check_bwd(wl, got, ref, TOL_BF16)
+    tok = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                            scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+    if 0 < p < 1:       # the mode differs visibly from token-level routing on the same inputs
+        assert rel_err(tok["dk"], ref["dk"]) > 10 * TOL_BF16
+
+
+def test_block_routed_backward_other_shapes_are_refused():
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]           # d = 128
+    x = block_inputs(wl, 1, 1, 128, 0.5)
+    dt = tdtype(wl)
+    with pytest.raises(binding.NatslError) as e:
+        binding.hybrid_bwd(*(dev(x[m], dt) for m in ("q", "k", "v")), dev(x["g"]), dev(x["beta"]),
+                           dev(x["route"]), dev(x["w"]), dev(x["dout"], dt), scale_la=wl.scale_la,
+                           scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING)
+    assert e.value.status == binding.ERR_UNSUPPORTED
