@@ -398,7 +398,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                               f.lse, BlockRouting{nullptr, nullptr, nullptr}, s32, st));
     // ---- combination and softmax branch ----
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la,
-                                 tensor_cores && !block ? nullptr : f.do_nla, dw, f.Dsm,
+                                 tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,
                                  tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
                                  tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, s, st));
     if (tensor_cores)
@@ -424,7 +424,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         // kernel adds to its own dk, dv.
         float *dk_x = f.X3, *dv_x = f.X4;
         NATSL_TRY(launch_gdn_finish(a, dk_x, dv_x, s32, st, false));
-        NATSL_TRY(launch_softmax_bwd_own_block(q, k, v, f.do_nla, f.lse, f.Dsm, route, p->scale_sm,
+        NATSL_TRY(launch_softmax_bwd_own_block(q, k, v, f.dO16, f.lse, f.Dsm, route, p->scale_sm,
                                                f.dq_sm, dk_x, dv_x, s, st));
         NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,

@@ -688,6 +688,119 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// Backward of the softmax branch through a query's own block under block-level routing
+// (Section 4.1: both operations compute the inner-chunk correlations; Section 4.2: ds = p (dp -
+// <do, o>)).  A query in a linear block reads, besides the retained tokens of earlier softmax
+// blocks (the kernels over the compacted K/V handle those), the causal part of its own block of
+// 64 tokens.  One CTA per linear block adds that part, five 64 x 64 x 64 products on the
+// warp-level tensor-core path of the chunk kernel above (fp16 tiles, fp32 accumulation):
+//   S = Q K^T, dP = dO V^T;  p_ij = exp(scale s_ij - lse_i), ds_ij = scale p_ij (dp_ij - D_i), j <= i
+//   dq += dS K  (added to the query-side result of the compacted kernels)
+//   dk  = dS^T Q,  dv = P^T dO  (written: the tokens of a linear block have no other
+//                                 softmax-branch gradient)
+// with lse_i and D_i = <do_i, o_i> of the whole softmax row.  d = 64.
+constexpr int kOwnSmem = 6 * kTileH * 2;
+
+__global__ void __launch_bounds__(kCkThreads, 3)
+softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
+                             const __nv_bfloat16 *__restrict__ v, const __half *__restrict__ do16,
+                             const float *__restrict__ lse, const float *__restrict__ Dsm,
+                             const uint8_t *__restrict__ route, float scale_sm,
+                             float *__restrict__ dq_sm, float *__restrict__ dk_x,
+                             float *__restrict__ dv_x, int L, int H) {
+    constexpr int D = 64;
+    extern __shared__ __align__(16) uint8_t smraw[];
+    __half *sQ = reinterpret_cast<__half *>(smraw), *sK = sQ + kTileH, *sV = sK + kTileH, *sDO = sV + kTileH,
+           *sP = sDO + kTileH, *sDS = sP + kTileH;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    const size_t ts = (size_t)H * D;
+    const size_t tok0 = (((size_t)b * L + (size_t)c * kC) * H + h) * D;
+    if (route[((size_t)b * L + (size_t)c * kC) * H + h]) return;   // a softmax block: its tokens are retained ones
+    {
+        const int r0 = tid >> 4, c4 = (tid & 15) * 4;
+        auto cv = [](uint32_t w) {                                  // bf16 pair -> fp16 pair (exact)
+            return pack_half2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+        };
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int r = r0 + 16 * it;
+            const size_t off = tok0 + (size_t)r * ts + c4;
+            const uint2 xq = *reinterpret_cast<const uint2 *>(q + off), xk = *reinterpret_cast<const uint2 *>(k + off),
+                        xv = *reinterpret_cast<const uint2 *>(v + off);
+            const uint2 xo = *reinterpret_cast<const uint2 *>(do16 + ((size_t)bh * L + (size_t)c * kC + r) * D + c4);
+            *reinterpret_cast<uint2 *>(sQ + r * kLdH + c4) = make_uint2(cv(xq.x), cv(xq.y));
+            *reinterpret_cast<uint2 *>(sK + r * kLdH + c4) = make_uint2(cv(xk.x), cv(xk.y));
+            *reinterpret_cast<uint2 *>(sV + r * kLdH + c4) = make_uint2(cv(xv.x), cv(xv.y));
+            *reinterpret_cast<uint2 *>(sDO + r * kLdH + c4) = xo;
+        }
+    }
+    __syncthreads();
+    const int row0 = 16 * (warp & 3), n0 = 32 * (warp >> 2);
+    const int iA = row0 + g, iB = iA + 8;
+    const size_t rowA = (size_t)bh * L + (size_t)c * kC + iA;
+    const float l2e = 1.4426950408889634f;
+    const float lseA = lse[rowA] * l2e, lseB = lse[rowA + 8] * l2e, DA = Dsm[rowA], DB = Dsm[rowA + 8];
+    float pr[4][4], acc[4][4];
+    auto zero = [](float (&a)[4][4]) {
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) a[nt][e] = 0.f;
+    };
+    auto put = [&](__half *X, const float (&a)[4][4]) {
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            *reinterpret_cast<uint32_t *>(X + iA * kLdH + n0 + 8 * nt + 2 * t) = pack_half2(a[nt][0], a[nt][1]);
+            *reinterpret_cast<uint32_t *>(X + iB * kLdH + n0 + 8 * nt + 2 * t) = pack_half2(a[nt][2], a[nt][3]);
+        }
+    };
+    // p = exp(scale s - lse), causal inside the block (mask on the exponent: no branch per element)
+    zero(pr);
+    mma64<false, true>(sQ, sK, row0, n0, lane, pr);
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int j = n0 + 8 * nt + 2 * t + (e & 1), i = e < 2 ? iA : iB;
+            pr[nt][e] = ex2_ftz(j <= i ? fmaf(pr[nt][e], scale_sm * l2e, -(e < 2 ? lseA : lseB)) : -INFINITY);
+        }
+    put(sP, pr);
+    // ds = scale p (dp - D)
+    zero(acc);
+    mma64<false, true>(sDO, sV, row0, n0, lane, acc);
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[nt][e] = scale_sm * pr[nt][e] * (acc[nt][e] - (e < 2 ? DA : DB));
+    put(sDS, acc);
+    __syncthreads();
+    auto out2 = [&](float *dst, const float (&a)[4][4], bool add) {
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            float2 *pa = reinterpret_cast<float2 *>(dst + tok0 + (size_t)iA * ts + n0 + 8 * nt + 2 * t);
+            float2 *pb = reinterpret_cast<float2 *>(dst + tok0 + (size_t)iB * ts + n0 + 8 * nt + 2 * t);
+            float2 va = make_float2(a[nt][0], a[nt][1]), vb = make_float2(a[nt][2], a[nt][3]);
+            if (add) {
+                const float2 ca = *pa, cb = *pb;
+                va.x += ca.x; va.y += ca.y; vb.x += cb.x; vb.y += cb.y;
+            }
+            *pa = va;
+            *pb = vb;
+        }
+    };
+    zero(acc);
+    mma64<false, false>(sDS, sK, row0, n0, lane, acc);          // dq += dS K
+    out2(dq_sm, acc, true);
+    zero(acc);
+    mma64<true, false>(sDS, sQ, row0, n0, lane, acc);           // dk = dS^T Q
+    out2(dk_x, acc, false);
+    zero(acc);
+    mma64<true, false>(sP, sDO, row0, n0, lane, acc);           // dv = P^T dO
+    out2(dv_x, acc, false);
+}
+
 }  // namespace
 
 template <int D>
@@ -741,6 +854,22 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
                    (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, dg, dbeta, s.L, s.H, dk_x, dv_x};
     dim3 grid(s.L / kC, s.B * s.H);
     kernel<<<grid, kCkThreads, kCkSmem, st>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_bwd_own_block(const void *q, const void *k, const void *v,
+                                         const void *do16, const float *lse, const float *Dsm,
+                                         const uint8_t *route, float scale_sm, float *dq_sm,
+                                         float *dk_x, float *dv_x, Shape s, cudaStream_t st) {
+    if (s.d != 64 || !s.bf16) return cudaErrorInvalidValue;
+    cudaError_t e = cudaFuncSetAttribute(softmax_bwd_own_block_kernel,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kOwnSmem);
+    if (e != cudaSuccess) return e;
+    dim3 grid(s.L / kC, s.B * s.H);
+    softmax_bwd_own_block_kernel<<<grid, kCkThreads, kOwnSmem, st>>>(
+        (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, (const __half *)do16,
+        lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }

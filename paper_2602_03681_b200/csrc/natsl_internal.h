@@ -188,10 +188,10 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
                                  float *dbeta, bool block, const float *dk_x, const float *dv_x, Shape s,
                                  cudaStream_t st);
 
-// softmax_bwd_own.cu -- block-level routing: softmax-branch backward through the own block of the
-// queries of a linear block (adds to dq_sm, writes dk_x / dv_x rows of the linear blocks)
+// block-level routing: softmax-branch backward through the own block of the queries of a linear
+// block (adds to dq_sm, writes the dk_x / dv_x rows of the linear blocks); do16: fp16 [B,H,L,d]
 cudaError_t launch_softmax_bwd_own_block(const void *q, const void *k, const void *v,
-                                         const float *do_nla, const float *lse, const float *Dsm,
+                                         const void *do16, const float *lse, const float *Dsm,
                                          const uint8_t *route, float scale_sm, float *dq_sm,
                                          float *dk_x, float *dv_x, Shape s, cudaStream_t st);
 

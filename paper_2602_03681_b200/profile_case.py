@@ -95,7 +95,7 @@ def main():
         kw["B"] = args.B
     if args.L:
         kw["L"] = args.L
-    if args.op == "fwd" and args.flags & binding.BLOCK_ROUTING:   # one route per block of 64 tokens
+    if args.op in ("fwd", "bwd") and args.flags & binding.BLOCK_ROUTING:   # one route per block of 64 tokens
         kw["route"] = inputs.route_blocks(wl.seed, (kw.get("B", wl.B), kw.get("L", wl.L), wl.H),
                                           wl.p_softmax)
     x = inputs.make_layer_inputs(wl, **kw)
@@ -116,7 +116,7 @@ def main():
             def call():
                 nonlocal ws
                 ws = binding.hybrid_bwd(q, k, v, g, beta, route, w, dout, scale_la=wl.scale_la,
-                                        scale_sm=wl.scale_sm, ws=ws)["ws"]
+                                        scale_sm=wl.scale_sm, flags=args.flags, ws=ws)["ws"]
             timed(call)
     finish()
 
