@@ -71,7 +71,7 @@ enum {
                                     parallel (a second run per segment yields the segment's
                                     state transition, a small kernel chains the segments); the
                                     results agree to rounding */
-    NATSL_BLOCK_ROUTING = 1u << 2,     /* forward (both paths): block-level routing, the paper's
+    NATSL_BLOCK_ROUTING = 1u << 2,     /* forward (both paths), backward: block-level routing, the paper's
                                     default (Section 4.1, "compute the inner-chunk correlation";
                                     Section 4.3, chunk size = GDN chunk size).  `route` holds one
                                     decision per block of C = 64 tokens, repeated over the block's
@@ -85,7 +85,8 @@ enum {
                                     decay alone).  state_out, k_sm, v_sm, sm_len hold what is kept
                                     after the last block.  A route that changes inside a block is
                                     reported as NATSL_ERR_ROUTE by natsl_device_status.  Backward:
-                                    NATSL_ERR_UNSUPPORTED with this flag.  Generation: route 2 in
+                                    built for bf16 storage with d = 64, NATSL_ERR_UNSUPPORTED
+                                    otherwise.  Generation: route 2 in
                                     natsl_decode_step and natsl_decode_block_end (no flag needed) */
     NATSL_APPEND_CACHE = 1u << 3       /* forward, tensor-core path: prefill in pieces.  p->k_sm, p->v_sm,
                                     p->sm_len (required) are read AND written: the cache already

@@ -62,6 +62,22 @@ def test_fwd_bwd_full_size_training_workload():
     assert np.all(gb["dbeta"][~lin] == 0)
 
 
+def test_fwd_bwd_full_size_training_workload_block_routing():
+    """The training workload with one routing decision per block of 64 tokens: forward and
+    backward, every element against the block-mode oracle."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+    route = inputs.route_blocks(wl.seed, (wl.B, wl.L, wl.H), wl.p_softmax)
+    x = inputs.make_layer_inputs(wl, route=route)
+    got = run_fwd(wl, x, flags=binding.BLOCK_ROUTING)
+    ref = run_oracle(wl, x, block=64)
+    check_fwd(wl, got, ref, TOL[wl.dtype])
+    gb = run_bwd(wl, x, flags=binding.BLOCK_ROUTING)
+    rb = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                           scale_la=wl.scale_la, scale_sm=wl.scale_sm, block=64)
+    check_bwd(wl, gb, rb, TOL[wl.dtype])
+
+
 def test_decode_full_size_sampled_sequences():
     from paper_2602_03681_b200 import binding
     wl = inputs.WORKLOADS["cfg3_bf16_decode"]
