@@ -138,15 +138,20 @@ def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5
     tail = (ctypes.c_double(scale_la), ctypes.c_double(scale_sm), ctypes.c_double(eps),
             _p(state_in), _p(dstate_out), _p(dq), _p(dk), _p(dv), _p(dg), _p(dbeta), _p(dw),
             _p(dstate_in))
+    dscore = None
     if block is None:
         rc = _load().natsl_oracle_hybrid_bwd(*head, *tail)
     else:
-        rc = _load().natsl_oracle_hybrid_bwd_block(*head, int(block), *tail)
+        dscore = np.zeros((B, L // int(block), H, 2))
+        rc = _load().natsl_oracle_hybrid_bwd_block(*head, int(block), *tail, _p(dscore))
     if rc == -4:
         raise ValueError("block mode: route must be constant within each block")
     if rc != 0:
         raise RuntimeError(f"natsl_oracle_hybrid_bwd failed ({rc})")
-    return dict(dq=dq, dk=dk, dv=dv, dg=dg, dbeta=dbeta, dw=dw, dstate_in=dstate_in)
+    res = dict(dq=dq, dk=dk, dv=dv, dg=dg, dbeta=dbeta, dw=dw, dstate_in=dstate_in)
+    if dscore is not None:
+        res["dscore"] = dscore      # [B, L/R, H, 2]: (linear, softmax) mask gradients per block
+    return res
 
 
 def decode_step(q, k, v, g, beta, route, w, state, k_cache, v_cache, cache_len, *, scale_la,

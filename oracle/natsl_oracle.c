@@ -549,7 +549,15 @@ int natsl_oracle_hybrid_bwd(const double *q, const double *k, const double *v,
  *     the block's tokens.  A softmax block hands on exp(sum g) * (start state): the incoming
  *     gradient goes straight to the start state (times the decay) and to every g of the block;
  *     the block's own token chain receives gradient from its outputs only.
- * Arguments as natsl_oracle_hybrid_bwd, plus the block length R.
+ * Arguments as natsl_oracle_hybrid_bwd, plus the block length R and
+ *   dscore [B, L/R, H, 2] (may be NULL): gradients of the two operation scores' masks per block
+ *   (Section 4.2), index 0 = linear, 1 = softmax, computed for the active operation only and
+ *   zero for the other ("set d score = 0 if the mask is 0"):
+ *     softmax block t: sum over its keys j and all queries i >= j of dM_ij = p_ij (dp_ij - <do_i, o_i>)
+ *                      (the dM^nla and d score^nla equations);
+ *     linear block t : <dS_next, U_t>, U_t = the update the block commits to the state, i.e. the
+ *                      gradient of a mask m_t in S_next = decay S_start + m_t U_t (the paper's
+ *                      d score^la equation names the two factors dS and S without indices).
  * ------------------------------------------------------------------------- */
 int natsl_oracle_hybrid_bwd_block(const double *q, const double *k, const double *v,
                                   const double *g, const double *beta, const uint8_t *route,
@@ -557,10 +565,11 @@ int natsl_oracle_hybrid_bwd_block(const double *q, const double *k, const double
                                   int R, double scale_la, double scale_sm, double eps,
                                   const double *state_in, const double *dstate_out,
                                   double *dq, double *dk, double *dv, double *dg, double *dbeta,
-                                  double *dw, double *dstate_in)
+                                  double *dw, double *dstate_in, double *dscore)
 {
     if (d > 512 || d <= 0 || R <= 0 || L % R != 0) return -1;
     int err = 0, bad_route = 0;
+    if (dscore) memset(dscore, 0, sizeof(double) * (size_t)B * (L / R) * H * 2);
     size_t dd = (size_t)d * d;
     int NB = L / R;
 #pragma omp parallel for schedule(dynamic, 1)
@@ -680,6 +689,7 @@ int natsl_oracle_hybrid_bwd_block(const double *q, const double *k, const double
                 double pij = exp(scale_sm * sc - lse[i]);
                 for (int c = 0; c < d; ++c) dp += doi[c] * vj[c];
                 double ds = pij * (dp - D);
+                if (dscore && route[tj]) dscore[(((size_t)b * NB + j / R) * H + h) * 2 + 1] += ds;
                 for (int c = 0; c < d; ++c) dv[tj * d + c] += pij * doi[c];
                 for (int a = 0; a < d; ++a) {
                     dq[t * d + a] += scale_sm * ds * kj[a];
@@ -705,6 +715,14 @@ int natsl_oracle_hybrid_bwd_block(const double *q, const double *k, const double
                 dg_block = decay * acc;
             } else {
                 memset(dC, 0, sizeof(double) * dd);
+                if (dscore) {   /* <dS_next, committed update>, update = last state - decayed start */
+                    double g_block = 0.0, acc = 0.0;
+                    for (int i = i0; i < i0 + R; ++i) g_block += g[AT3(b, i, h)];
+                    double decay = exp(g_block);
+                    const double *Se = after + dd * (i0 + R - 1);
+                    for (size_t a = 0; a < dd; ++a) acc += dS[a] * (Se[a] - decay * start[dd * c + a]);
+                    dscore[(((size_t)b * NB + c) * H + h) * 2] = acc;
+                }
             }
             for (int i = i0 + R - 1; i >= i0; --i) {
                 size_t t = AT3(b, i, h);

@@ -706,3 +706,55 @@ def test_block_mode_backward_special_cases():
     for n in ("dq", "dk", "dv"):
         np.testing.assert_allclose(gb[n], gt[n], rtol=1e-10, atol=1e-13, err_msg=n)
     assert np.all(gb["dg"] == 0) and np.all(gb["dbeta"] == 0)
+
+
+def test_block_mode_score_gradients_against_a_relaxed_mask_forward():
+    """d score per block (Section 4.2): finite differences of a forward in which the masks are
+    real numbers -- mu_t multiplies e^A of the keys of softmax block t for every query, m_t scales
+    the update a linear block commits to the state."""
+    B, L, H, d, R = 1, 16, 1, 4, 4
+    x = rand_inputs(B, L, H, d, seed=38)
+    x["route"] = np.repeat(np.array([1, 0, 1, 0], np.uint8), R)[None, :, None]
+    dout = RNG.standard_normal((B, L, H, d))
+    q, k, v = (x[n][0, :, 0] for n in ("q", "k", "v"))
+    g, beta, route, w = (x[n][0, :, 0] for n in ("g", "beta", "route", "w"))
+    blk = np.arange(L) // R
+    NB = L // R
+
+    def loss(mu, m):
+        i, j = np.meshgrid(np.arange(L), np.arange(L), indexing="ij")
+        vis = (j <= i) & ((route[j] == 1) | (blk[j] == blk[i]))
+        weight = np.where(route[j] == 1, mu[blk[j]], 1.0)              # mask value of the key's block
+        e = np.where(vis, weight * np.exp(1.5 * q @ k.T), 0.0)
+        o_nla = (e / e.sum(1, keepdims=True)) @ v
+        S = np.zeros((d, d))                                          # ours: o = q S
+        o_la = np.zeros((L, d))
+        for c in range(NB):
+            run = S.copy()
+            for t in range(c * R, (c + 1) * R):
+                run = np.exp(g[t]) * run
+                run = run + beta[t] * np.outer(k[t], v[t] - k[t] @ run)
+                o_la[t] = 0.5 * q[t] @ run
+            decayed = np.exp(g[c * R:(c + 1) * R].sum()) * S
+            S = decayed + (m[c] if route[c * R] == 0 else 0.0) * (run - decayed)
+        norm = lambda o: o / np.sqrt((o * o).mean(-1, keepdims=True) + 1e-5)
+        out = w[:, :1] * norm(o_nla) + w[:, 1:] * norm(o_la)
+        return (out * dout[0, :, 0]).sum()
+
+    ones = np.ones(NB)
+    np.testing.assert_allclose(loss(ones, ones), (fwd(x, block=R)["out"] * dout).sum(), rtol=1e-10)
+    gr = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], dout,
+                           scale_la=0.5, scale_sm=1.5, block=R)["dscore"][0, :, 0]
+    h = 1e-6
+    for c in range(NB):
+        for op in (0, 1):
+            e = np.zeros(NB)
+            e[c] = h
+            fd = ((loss(ones, ones + e) - loss(ones, ones - e)) if op == 0
+                  else (loss(ones + e, ones) - loss(ones - e, ones))) / (2 * h)
+            active = (route[c * R] == 1) == (op == 1)
+            if active:
+                assert abs(fd - gr[c, op]) <= 1e-6 * max(1.0, abs(fd)), (c, op, fd, gr[c, op])
+                assert abs(fd) > 1e-6 or c == NB - 1       # (the last linear block feeds nothing)
+            else:
+                assert gr[c, op] == 0.0                    # not computed for the inactive operation
