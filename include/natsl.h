@@ -122,6 +122,13 @@ typedef struct natsl_params {
     void *const *stage_events; /* host array of cudaEvent_t owned by the caller, or NULL: the    */
     int32_t n_stage_events;    /*   library records event[i] on `stream` before stage i and one  */
                                /*   after the last stage (see natsl_stage_name); for profiling.  */
+    float *dscore;          /* backward with NATSL_BLOCK_ROUTING, optional: gradients of the score    */
+                            /*   layer's two masks per block [B,L/C,H,2] fp32 = (linear, softmax), */
+                            /*   Section 4.2: for a softmax block the sum over its keys j and all  */
+                            /*   queries i >= j of dM_ij = p_ij (dp_ij - <do_i, o_i>); for a linear */
+                            /*   block <dS_next, U> with U the update the block commits to the     */
+                            /*   state; zero for the operation the block did not choose.  NULL:    */
+                            /*   not computed.  Without the flag: NATSL_ERR_UNSUPPORTED.           */
 } natsl_params;
 
 /* Bytes of workspace `op` needs for these shapes (host call, launches nothing). */

@@ -48,7 +48,7 @@ class natsl_params(ctypes.Structure):
                 ("o_nla", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("k_sm", ctypes.c_void_p),
                 ("v_sm", ctypes.c_void_p), ("sm_len", ctypes.c_void_p),
                 ("sm_cap", ctypes.c_int32), ("stage_events", ctypes.c_void_p),
-                ("n_stage_events", ctypes.c_int32)]
+                ("n_stage_events", ctypes.c_int32), ("dscore", ctypes.c_void_p)]
 
 
 _lib = None
@@ -242,7 +242,8 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5,
     return res
 
 
-def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5, ws=None, flags=0):
+def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5, ws=None, flags=0,
+               want_dscore=False):
     """Allocate gradients and run natsl_hybrid_bwd.  Returns dict(dq, dk, dv, dg, dbeta, dw, ws)."""
     B, L, H, d = q.shape
     dev = q.device
@@ -251,7 +252,14 @@ def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5
     dbeta = torch.empty((B, L, H), dtype=torch.float32, device=dev)
     dw = torch.empty((B, L, H, 2), dtype=torch.float32, device=dev)
     p = make_params(B, H, L, d, _dtype_code(q), scale_la, scale_sm, eps, w=w, flags=flags)
+    dscore = None
+    if want_dscore:
+        dscore = torch.empty((B, L // 64, H, 2), dtype=torch.float32, device=dev)
+        p.dscore = dscore.data_ptr()
     if ws is None:
         ws = alloc_workspace(p, OP_BWD, dev)
     natsl_hybrid_bwd(q, k, v, g, beta, route, dout, dq, dk, dv, dg, dbeta, dw, p, ws)
-    return dict(dq=dq, dk=dk, dv=dv, dg=dg, dbeta=dbeta, dw=dw, ws=ws)
+    res = dict(dq=dq, dk=dk, dv=dv, dg=dg, dbeta=dbeta, dw=dw, ws=ws)
+    if dscore is not None:
+        res["dscore"] = dscore
+    return res

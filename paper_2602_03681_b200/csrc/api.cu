@@ -341,6 +341,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     // block-level routing: on the path with the fused chunk kernel only (bf16 storage, d = 64)
     const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
     if (block && !(use_tensor_cores(p) && p->d == 64)) return NATSL_ERR_UNSUPPORTED;
+    if (p->dscore && !block) return NATSL_ERR_UNSUPPORTED;   // score gradients: one decision per block
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
         return NATSL_ERR_ALIGN;
@@ -403,7 +404,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                  tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, s, st));
     if (tensor_cores)
         NATSL_TRY(launch_softmax_bwd_tc(q, f.Qh, f.dO16, f.k16, f.v16, p->L, f.sm_idx, f.prefix, f.lse,
-                                        f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, f.status, s, st));
+                                        f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm,
+                                        p->dscore ? f.dGrow : nullptr, f.status, s, st));
     else
         NATSL_TRY(launch_softmax_bwd(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix, f.do_nla,
                                      f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
@@ -428,13 +430,15 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                                f.dq_sm, dk_x, dv_x, s, st));
         NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
-                                       true, dk_x, dv_x, s, st));
+                                       true, dk_x, dv_x, p->dscore ? f.kappa : nullptr, s, st));
+        if (p->dscore)   // (dGrow, kappa: [B,H,L] scratch the fused path does not otherwise use)
+            NATSL_TRY(launch_dscore(route, f.prefix, f.dGrow, f.kappa, p->L, p->dscore, s, st));
         return NATSL_OK;
     }
     if (fused_chunks) {   // all chunk-level products and the assembly in one kernel per chunk
         NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
-                                       false, nullptr, nullptr, s, st));
+                                       false, nullptr, nullptr, nullptr, s, st));
         NATSL_TRY(launch_gdn_finish(a, dk, dv, s, st, false));   // scatter of the retained tokens' dk, dv
         return NATSL_OK;
     }

@@ -315,6 +315,8 @@ struct ChunkBwdArgs {
     // decay), and every token's dk, dv also has a softmax-branch part, given in dk_x, dv_x
     // (fp32, token-major).
     const float *dk_x, *dv_x;
+    float *kap_c;    // [B,H,L/C] or nullptr: sum over the chunk of kappa = <dS1, K~^T U~>, the gradient
+                     // of a mask on the update this chunk commits to the state (Section 4.2, d score^la)
 };
 
 // acc (16 x 32 block at (row0, n0) of a 64 x 64 result) += A B over k = 0..63, fp16 tiles.
@@ -682,6 +684,7 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
 #pragma unroll
         for (int wv = 0; wv < 8; ++wv) gs += sMax[24 + wv];
         const float extra = sMax[34] + sMax[35] + exp_ftz(sG[63]) * gs + (warp == 0 ? sMax[33] : 0.f);
+        if (kBlock && p.kap_c && tid == 0) p.kap_c[chunk] = sMax[34] + sMax[35];
         const size_t tk = ((size_t)b * p.L + (size_t)c * kC + tid) * p.H + h;
         p.dg[tk] = suf + extra;
         p.dbeta[tk] = !kBlock && p.route[tk] ? 0.f : rB[tid];
@@ -842,8 +845,8 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
                                  const float *Tinv, const void *Wt, const float *Up, const float *Gcum,
                                  const float *beta, const uint8_t *route, const float *dq_sm,
                                  float scale_la, void *dq, void *dk, void *dv, float *dg,
-                                 float *dbeta, bool block, const float *dk_x, const float *dv_x, Shape s,
-                                 cudaStream_t st) {
+                                 float *dbeta, bool block, const float *dk_x, const float *dv_x,
+                                 float *kap_c, Shape s, cudaStream_t st) {
     if (s.d != 64 || !s.bf16) return cudaErrorInvalidValue;
     auto kernel = block ? gdn_bwd_chunk_kernel<true> : gdn_bwd_chunk_kernel<false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -851,9 +854,42 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
     if (e != cudaSuccess) return e;
     ChunkBwdArgs a{(const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, dO, dUt, Ut,
                    S_c, dS_c, Tinv, Up, Gcum, beta, dq_sm, (const __half *)Wt, route, scale_la, (__nv_bfloat16 *)dq,
-                   (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, dg, dbeta, s.L, s.H, dk_x, dv_x};
+                   (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, dg, dbeta, s.L, s.H, dk_x, dv_x, kap_c};
     dim3 grid(s.L / kC, s.B * s.H);
     kernel<<<grid, kCkThreads, kCkSmem, st>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// d score per block and head (Section 4.2), for the active operation only: a softmax block sums the
+// mask gradients of its 64 keys (contiguous in the compacted order), a linear block takes the kappa
+// sum of its chunk; the other entry is zero.  dscore [B, L/C, H, 2] = (linear, softmax).
+namespace {
+__global__ void __launch_bounds__(64)
+dscore_kernel(const uint8_t *__restrict__ route, const int32_t *__restrict__ sm_chunk_prefix,
+              const float *__restrict__ dmask, const float *__restrict__ kap_c, int cap,
+              float *__restrict__ dscore, int L, int H) {
+    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H, NC = L / kC;
+    float *dst = dscore + (((size_t)b * NC + c) * H + h) * 2;
+    if (route[((size_t)b * L + (size_t)c * kC) * H + h]) {
+        const int row = sm_chunk_prefix[(size_t)bh * (NC + 1) + c] + (int)threadIdx.x;
+        float x = row < cap ? dmask[(size_t)bh * cap + row] : 0.f;
+        x = warp_sum(x);
+        __shared__ float part[2];
+        if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = x;
+        __syncthreads();
+        if (threadIdx.x == 0) { dst[0] = 0.f; dst[1] = part[0] + part[1]; }
+    } else if (threadIdx.x == 0) {
+        dst[0] = kap_c[(size_t)bh * NC + c];
+        dst[1] = 0.f;
+    }
+}
+}  // namespace
+
+cudaError_t launch_dscore(const uint8_t *route, const int32_t *sm_chunk_prefix, const float *dmask,
+                          const float *kap_c, int cap, float *dscore, Shape s, cudaStream_t st) {
+    dim3 grid(s.L / kC, s.B * s.H);
+    dscore_kernel<<<grid, 64, 0, st>>>(route, sm_chunk_prefix, dmask, kap_c, cap, dscore, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }

@@ -78,7 +78,7 @@ cudaError_t launch_softmax_bwd_tc(const void *q, void *Qh, const void *dO16, con
                                   const void *v16, int cap, const int32_t *sm_idx,
                                   const int32_t *sm_chunk_prefix, const float *lse, const float *Dsm,
                                   float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
-                                  int32_t *status, Shape s, cudaStream_t st);
+                                  float *dmask, int32_t *status, Shape s, cudaStream_t st);
 
 // gdn_tc.cu -- tensor-core chunkwise Gated DeltaNet (bf16 storage): intermediates in workspace
 struct GdnTcWs {
@@ -185,8 +185,10 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
                                  const float *Tinv, const void *Wt, const float *Up, const float *Gcum,
                                  const float *beta, const uint8_t *route, const float *dq_sm,
                                  float scale_la, void *dq, void *dk, void *dv, float *dg,
-                                 float *dbeta, bool block, const float *dk_x, const float *dv_x, Shape s,
-                                 cudaStream_t st);
+                                 float *dbeta, bool block, const float *dk_x, const float *dv_x,
+                                 float *kap_c, Shape s, cudaStream_t st);
+cudaError_t launch_dscore(const uint8_t *route, const int32_t *sm_chunk_prefix, const float *dmask,
+                          const float *kap_c, int cap, float *dscore, Shape s, cudaStream_t st);
 
 // block-level routing: softmax-branch backward through the own block of the queries of a linear
 // block (adds to dq_sm, writes the dk_x / dv_x rows of the linear blocks); do16: fp16 [B,H,L,d]

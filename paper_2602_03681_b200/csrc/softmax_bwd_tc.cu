@@ -263,7 +263,7 @@ template <int D> struct KLayout {
     static constexpr int kTmem = D == 64 ? 256 : 512;     // S^T 64 + dP^T 64 + dV D + dK D
 };
 
-template <int D>
+template <int D, bool kMask>       // kMask: also the per-key sums of the mask gradient (dmask)
 __global__ void __launch_bounds__(kThreadsB)
 softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B*H*L][D], box 64
                           const __grid_constant__ CUtensorMap map_do,   // dO16, box 64
@@ -273,6 +273,7 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                           const int32_t *__restrict__ sm_chunk_prefix,
                           const float *__restrict__ lse, const float *__restrict__ Dsm,
                           float scale_sm, float *__restrict__ dk_sm, float *__restrict__ dv_sm,
+                          float *__restrict__ dmask,     // [B*H*cap]: sum_i p_ij (dp_ij - D_i) per key j
                           int32_t *status, int L, int H) {
     using SL = KLayout<D>;
     constexpr int KB = SL::KB;
@@ -388,6 +389,7 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
         const int pos_j = key_ok ? sm_idx[(size_t)bh * L + j] : 0x7fffffff;
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         const float sl2 = scale_sm * kLog2e;
+        float msum = 0.f;                                   // mask gradient of this key, over all queries
         bool ok = true;
         for (int t = 0; t < T; ++t) {
             const int i0 = (qt0 + t) * 64;
@@ -419,7 +421,9 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                     const bool vis = pos_j <= i0 + cc;
                     const float pr = ex2_ftz(vis ? fmaf(__uint_as_float(sv[c]), sl2, -lse2[cc]) : -INFINITY);
                     pv[cc] = pr;
-                    ds[cc] = scale_sm * pr * (__uint_as_float(dv[c]) - dsum[cc]);
+                    const float dm = pr * (__uint_as_float(dv[c]) - dsum[cc]);   // dM_ij (Section 4.2)
+                    if (kMask) msum += dm;
+                    ds[cc] = scale_sm * dm;
                 }
             }
             if (t > 0) {
@@ -447,6 +451,7 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
         if (ok) {      // the TMEM loads are warp-wide: only the stores depend on the key being real
             float4 *dv_dst = reinterpret_cast<float4 *>(dv_sm + ((size_t)bh * cap + j) * D);
             float4 *dk_dst = reinterpret_cast<float4 *>(dk_sm + ((size_t)bh * cap + j) * D);
+            if (kMask && key_ok) dmask[(size_t)bh * cap + j] = msum;
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t x[32], y[32];
@@ -503,7 +508,7 @@ static cudaError_t softmax_bwd_tc_impl(const void *q, void *Qh, const void *dO16
                                        const void *v16, int cap, const int32_t *sm_idx,
                                        const int32_t *pre, const float *lse, const float *Dsm,
                                        float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
-                                       int32_t *status, Shape s, cudaStream_t st) {
+                                       float *dmask, int32_t *status, Shape s, cudaStream_t st) {
     const uint64_t BH = (uint64_t)s.B * s.H;
     const size_t pieces = (size_t)s.B * s.L * s.H * (D / 8);
     to_f16_bhld_kernel<D><<<(unsigned)((pieces + 255) / 256), 256, 0, st>>>(
@@ -518,8 +523,8 @@ static cudaError_t softmax_bwd_tc_impl(const void *q, void *Qh, const void *dO16
     cudaError_t e = cudaFuncSetAttribute(softmax_bwd_dq_tc_kernel<D>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, QLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(softmax_bwd_dkv_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             KLayout<D>::kTotal);
+    auto dkv = dmask ? softmax_bwd_dkv_tc_kernel<D, true> : softmax_bwd_dkv_tc_kernel<D, false>;
+    e = cudaFuncSetAttribute(dkv, cudaFuncAttributeMaxDynamicSharedMemorySize, KLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
     dim3 gq((s.L + 127) / 128, s.B * s.H);
     softmax_bwd_dq_tc_kernel<D><<<gq, kThreadsB, QLayout<D>::kTotal, st>>>(
@@ -527,8 +532,8 @@ static cudaError_t softmax_bwd_tc_impl(const void *q, void *Qh, const void *dO16
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     dim3 gk((s.L + 127) / 128, s.B * s.H);
-    softmax_bwd_dkv_tc_kernel<D><<<gk, kThreadsB, KLayout<D>::kTotal, st>>>(
-        mq64, mdo64, mk128, mv128, cap, sm_idx, pre, lse, Dsm, scale_sm, dk_sm, dv_sm, status, s.L, s.H);
+    dkv<<<gk, kThreadsB, KLayout<D>::kTotal, st>>>(
+        mq64, mdo64, mk128, mv128, cap, sm_idx, pre, lse, Dsm, scale_sm, dk_sm, dv_sm, dmask, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -537,12 +542,12 @@ cudaError_t launch_softmax_bwd_tc(const void *q, void *Qh, const void *dO16, con
                                   const void *v16, int cap, const int32_t *sm_idx,
                                   const int32_t *sm_chunk_prefix, const float *lse, const float *Dsm,
                                   float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
-                                  int32_t *status, Shape s, cudaStream_t st) {
+                                  float *dmask, int32_t *status, Shape s, cudaStream_t st) {
     if (s.d == 128)
         return softmax_bwd_tc_impl<128>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm,
-                                        scale_sm, dq_sm, dk_sm, dv_sm, status, s, st);
+                                        scale_sm, dq_sm, dk_sm, dv_sm, dmask, status, s, st);
     return softmax_bwd_tc_impl<64>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm,
-                                   scale_sm, dq_sm, dk_sm, dv_sm, status, s, st);
+                                   scale_sm, dq_sm, dk_sm, dv_sm, dmask, status, s, st);
 }
 
 }  // namespace natsl

@@ -223,3 +223,38 @@ def test_block_routed_backward_other_shapes_are_refused():
                            dev(x["route"]), dev(x["w"]), dev(x["dout"], dt), scale_la=wl.scale_la,
                            scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING)
     assert e.value.status == binding.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("B,H,L,p", [(1, 2, 256, 0.4), (2, 3, 512, 0.25)])
+def test_block_routed_backward_score_gradients(B, H, L, p):
+    """d score per block and head (Section 4.2) against the oracle: nonzero only for the operation
+    the block chose."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+    x = block_inputs(wl, B, H, L, p)
+    ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                            scale_la=wl.scale_la, scale_sm=wl.scale_sm, block=64)["dscore"]
+    dt = tdtype(wl)
+    res = binding.hybrid_bwd(*(dev(x[m], dt) for m in ("q", "k", "v")), dev(x["g"]), dev(x["beta"]),
+                             dev(x["route"]), dev(x["w"]), dev(x["dout"], dt), scale_la=wl.scale_la,
+                             scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING, want_dscore=True)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(res["ws"]) == 0
+    got = res["dscore"].cpu().numpy()
+    blocks = x["route"][:, ::64]                                   # [B, L/64, H]
+    assert np.all(got[..., 0][blocks == 1] == 0) and np.all(got[..., 1][blocks == 0] == 0)
+    for op in (0, 1):
+        assert rel_err(got[..., op], ref[..., op]) <= TOL_BF16, (op, rel_err(got[..., op], ref[..., op]))
+    assert np.abs(ref[..., 1]).max() > 0 and np.abs(ref[..., 0]).max() > 0
+
+
+def test_score_gradients_need_block_routing():
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+    x = inputs.make_layer_inputs(wl, B=1, H=1, L=128)
+    dt = tdtype(wl)
+    with pytest.raises(binding.NatslError) as e:
+        binding.hybrid_bwd(*(dev(x[m], dt) for m in ("q", "k", "v")), dev(x["g"]), dev(x["beta"]),
+                           dev(x["route"]), dev(x["w"]), dev(x["dout"], dt), scale_la=wl.scale_la,
+                           scale_sm=wl.scale_sm, want_dscore=True)
+    assert e.value.status == binding.ERR_UNSUPPORTED
