@@ -466,7 +466,99 @@ def bench_other_workloads(peaks):
         torch.cuda.empty_cache()
     res["score_layer"] = bench_score_layer(peaks)
     res["cfg2_bf16_long_prefill/in_4_pieces"] = bench_prefill_in_pieces()
+    res["serving_131072_tokens"] = bench_long_context_serving()
     return res
+
+
+def bench_long_context_serving(L=131072, piece=16384, decode_steps=64):
+    """A long-context serving loop on the long-context workload's head shapes (B=1, H=16, d=128,
+    5 % clustered softmax tokens): the prompt is prefilled in pieces (state chained, retained K/V
+    appended to one cache), then tokens are generated with one decode step captured in a CUDA graph
+    and replayed.  Inputs are drawn on the device (seeded); the code path is the one the parity
+    tests cover at 32768 tokens."""
+    import torch
+
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg2_bf16_long_prefill"]
+    B, H, d, dt = 1, wl.H, wl.d, torch.bfloat16
+    gen = torch.Generator(device="cuda").manual_seed(wl.seed)
+    route_all = inputs.route_runs(wl.seed, (B, L + decode_steps, H), wl.p_softmax)
+    cap = int(route_all.sum(1).max()) + 128
+
+    def draw(n):
+        q = torch.nn.functional.normalize(torch.randn((B, n, H, d), device="cuda", generator=gen), dim=-1)
+        k = torch.nn.functional.normalize(torch.randn((B, n, H, d), device="cuda", generator=gen), dim=-1)
+        v = torch.randn((B, n, H, d), device="cuda", generator=gen)
+        g = -torch.nn.functional.softplus(torch.randn((B, n, H), device="cuda", generator=gen) + wl.g_shift)
+        beta = torch.sigmoid(torch.randn((B, n, H), device="cuda", generator=gen))
+        w = torch.softmax(torch.randn((B, n, H, 2), device="cuda", generator=gen), dim=-1)
+        return [q.to(dt), k.to(dt), v.to(dt), g, beta, w]
+
+    pieces = []
+    for i in range(L // piece):
+        q, k, v, g, beta, w = draw(piece)
+        r = torch.from_numpy(np.ascontiguousarray(route_all[:, i * piece:(i + 1) * piece])).cuda()
+        pieces.append([q, k, v, g, beta, r, w])
+    cache = (torch.zeros((B, H, cap, d), dtype=dt, device="cuda"),
+             torch.zeros((B, H, cap, d), dtype=dt, device="cuda"),
+             torch.zeros((B, H), dtype=torch.int32, device="cuda"))
+    ws = [None]
+    state = [None]
+
+    def prefill():
+        cache[2].zero_()
+        st = None
+        for a in pieces:
+            r = binding.hybrid_fwd(*a, scale_la=wl.scale_la, scale_sm=wl.scale_sm, state_in=st,
+                                   want=("state_out",), cache=cache, flags=binding.APPEND_CACHE, ws=ws[0])
+            st, ws[0] = r["state_out"], r["ws"]
+        state[0] = st
+
+    prefill()
+    torch.cuda.synchronize()
+    best = float("inf")
+    for _ in range(2):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        prefill()
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    assert binding.natsl_device_status(ws[0]) == 0
+    # generation: one captured step, replayed; per-step inputs are copied into its static buffers
+    tq, tk, tv, tg, tb, tw = draw(decode_steps)
+    troute = torch.from_numpy(np.ascontiguousarray(route_all[:, L:])).cuda()
+    sq, sk, sv = (torch.zeros((B, H, d), dtype=dt, device="cuda") for _ in range(3))
+    sg, sb = torch.zeros((B, H), device="cuda"), torch.zeros((B, H), device="cuda")
+    sr = torch.zeros((B, H), dtype=torch.uint8, device="cuda")
+    sw = torch.zeros((B, H, 2), device="cuda")
+    out = torch.zeros((B, H, d), dtype=dt, device="cuda")
+    p = binding.make_params(B, H, 0, d, binding.NATSL_BF16, wl.scale_la, wl.scale_sm, w=sw)
+    dws = binding.alloc_workspace(p, binding.OP_DECODE)
+    st, n = state[0], cache[2]
+
+    def load(t):
+        sq.copy_(tq[:, t]); sk.copy_(tk[:, t]); sv.copy_(tv[:, t])
+        sg.copy_(tg[:, t]); sb.copy_(tb[:, t]); sr.copy_(troute[:, t]); sw.copy_(tw[:, t])
+
+    load(0)
+    binding.natsl_decode_step(sq, sk, sv, sg, sb, sr, st, cache[0], cache[1], n, out, p, dws)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        binding.natsl_decode_step(sq, sk, sv, sg, sb, sr, st, cache[0], cache[1], n, out, p, dws)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(1, decode_steps):
+        load(t)
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(dws) == 0
+    return {"prompt_tokens": L, "pieces": L // piece, "prefill_ms": best,
+            "prefill_tokens_per_s": L / (best * 1e-3), "retained_per_head_max": cap - 128,
+            "decode_ms_per_token": e0.elapsed_time(e1) / (decode_steps - 1),
+            "decode": "one step captured in a CUDA graph, replayed; includes the copies of the step's inputs"}
 
 
 def bench_prefill_in_pieces(n_pieces=4):
