@@ -1,6 +1,8 @@
 // Route compaction: the per-token routing mask becomes per-chunk index lists (Section 4.1,
 // column masks M^nla / M^la), with warp ballots and a block prefix sum; and a gather of the
-// retained tokens' K/V rows into the compacted cache layout [B,H,cap,d].
+// retained tokens' K/V rows into the compacted cache layout [B,H,cap,d].  Two options: the
+// prefix sums may start behind the entries a cache already holds (prefill in pieces), and the
+// route may be checked to be one decision per chunk (block-level routing).
 #include "common.cuh"
 #include "natsl_internal.h"
 

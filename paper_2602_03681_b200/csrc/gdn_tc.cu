@@ -7,6 +7,9 @@
 //   A_ij = beta~_i Gamma_ij (k_i.k_j) (j < i),  T = (I + A)^-1,
 //   U = T diag(beta~) V,  W = T diag(beta~ gamma) K,  P_ij = scale_la Gamma_ij (q_i.k_j) (j <= i)
 //   U~ = U - W S;  O = scale_la diag(gamma) Q S + P U~;  S <- gamma_C S + (diag(gamma_C/gamma) K)^T U~
+// Block-level routing (Section 4.1: both operations compute the inner-chunk correlations) uses the
+// same kernels with beta~ = beta for every token and the state update of a softmax block left
+// out (S <- gamma_C S), so that its chunk sees the delta rule but the later ones do not.
 //
 // Precision.  q, k, v are exact bf16 inputs, but T, W, U~, P and S are computed quantities: an
 // 8-bit significand on them puts the layer output 1.4-2e-2 x RMS off (the whole error budget), so

@@ -15,6 +15,8 @@
 // epilogue is issued per thread and row.
 // Warp roles: warps 0-3 softmax/epilogue (thread r <-> query row r <-> TMEM lane r), warp 4 issues
 // the MMAs, warp 5 issues the TMA loads.
+// Block-level routing (template flag): after the retained tiles, one more tile per linear block of
+// the CTA's two, holding that block's own 64 tokens (Section 4.1, inner-chunk correlations).
 #include "common.cuh"
 #include "natsl_internal.h"
 #include "tc_common.cuh"
