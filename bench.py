@@ -389,6 +389,10 @@ def run_ours(args):
         "clocks": clocks,
         "roofline": roofline,
         "stages_ms": stage_ms,
+        "stages_note": ("stage times are taken in a separate pass with the library's per-stage events, "
+                        "which makes it run the stages in sequence; in the timed steps the compaction "
+                        "and the gather run on a side stream beside the prepare kernel, so a step is "
+                        "shorter than the sum of the stages"),
         "step": {"useful_tflops": step_tf, "frac_of_bf16_peak": step_tf / peak_tf,
                  "useful_gflop": total_flops / 1e9, "min_hbm_bytes": min_hbm_bytes_fwd(wl, B),
                  "hbm_floor_ms": min_hbm_bytes_fwd(wl, B) / (peaks["hbm_gbs"] * 1e9) * 1e3},

@@ -88,7 +88,7 @@ enum {
                                     built for bf16 storage with d = 64, NATSL_ERR_UNSUPPORTED
                                     otherwise.  Generation: route 2 in
                                     natsl_decode_step and natsl_decode_block_end (no flag needed) */
-    NATSL_APPEND_CACHE = 1u << 3       /* forward, tensor-core path: prefill in pieces.  p->k_sm, p->v_sm,
+    NATSL_APPEND_CACHE = 1u << 3,      /* forward, tensor-core path: prefill in pieces.  p->k_sm, p->v_sm,
                                     p->sm_len (required) are read AND written: the cache already
                                     holds sm_len[b,h] retained tokens of earlier pieces of the same
                                     sequences; the softmax branch of this piece reads them as
@@ -100,6 +100,13 @@ enum {
                                     two hidden states kept during generation are the linear state
                                     and the KV cache).  natsl_workspace_size depends on the flag
                                     and on p->sm_cap.  Backward: NATSL_ERR_UNSUPPORTED */
+    NATSL_SINGLE_STREAM = 1u << 4      /* forward, tensor-core path: launch everything on the caller's
+                                    stream.  By default the route compaction and the gather of the
+                                    retained K/V run beside the linear branch's prepare kernel on a
+                                    stream the library creates once per device (forked from and
+                                    joined to the caller's stream with events, so the call is still
+                                    ordered like any other work on that stream).  Also implied by
+                                    p->stage_events.  natsl_hybrid_fwd_static always sets it */
 };
 
 typedef struct natsl_params {

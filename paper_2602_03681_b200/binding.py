@@ -20,6 +20,7 @@ FORCE_SIMT = 1
 SINGLE_PASS_SCAN = 2
 BLOCK_ROUTING = 4
 APPEND_CACHE = 8
+SINGLE_STREAM = 16
 ERR_CACHE_FULL = -7
 ERR_UNSUPPORTED = -8
 ERR_ROUTE = -11

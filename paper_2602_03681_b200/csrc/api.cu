@@ -5,6 +5,7 @@
 #include "natsl_internal.h"
 
 #include <atomic>
+#include <mutex>
 
 using namespace natsl;
 
@@ -173,6 +174,39 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
 
 }  // namespace
 
+namespace {
+
+// The compaction and the gather of the retained K/V do not depend on the linear branch's prepare
+// kernel (and that kernel does not depend on them), so the forward runs them beside it: on a
+// library-owned stream per device, forked from the caller's stream with one event and joined back
+// with another before the softmax kernel.  Stream and events are created on first use and kept;
+// a mutex covers the enqueue of a call, since the two event objects are shared by all calls.
+struct SideStream {
+    cudaStream_t st = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+    bool tried = false;
+};
+SideStream g_side[64];
+std::mutex g_side_mu;
+
+SideStream *side_stream_locked() {   // g_side_mu held; nullptr: run everything on the caller's stream
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    SideStream &s = g_side[dev];
+    if (!s.tried) {
+        s.tried = true;
+        if (cudaStreamCreateWithFlags(&s.st, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) {
+            s.st = nullptr;
+            (void)cudaGetLastError();
+        }
+    }
+    return s.st ? &s : nullptr;
+}
+
+}  // namespace
+
 extern "C" {
 
 uint64_t natsl_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
@@ -276,18 +310,33 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     };
     NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
     NATSL_TRY(mark());
+    // Stage 0 (compaction, gather) beside stage 1 (prepare) on the side stream -- unless the caller
+    // asks for one stream or for per-stage events, whose differences are only meaningful in sequence.
+    std::unique_lock<std::mutex> side_lock;
+    SideStream *side = nullptr;
+    if (tensor_cores && !(p->flags & NATSL_SINGLE_STREAM) && !p->stage_events) {
+        side_lock = std::unique_lock<std::mutex>(g_side_mu);
+        side = side_stream_locked();
+        if (!side) side_lock.unlock();
+    }
+    cudaStream_t st0 = side ? side->st : st;
+    if (side) {
+        NATSL_TRY(cudaEventRecord(side->fork, st));
+        NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
+    }
     int32_t *sm_len = want_cache ? p->sm_len : f.sm_len;
     void *k_sm = want_cache ? p->k_sm : f.k_sm, *v_sm = want_cache ? p->v_sm : f.v_sm;
     const int32_t cap = want_cache ? p->sm_cap : p->L;
     const int32_t capv = append ? p->sm_cap : p->L;          // rows per head of the fp16 V copy
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, sm_len,
                                    append ? sm_len : nullptr, block ? f.status : nullptr, p->B, p->L,
-                                   p->H, st));
+                                   p->H, st0));
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
-                                      f.v16, nullptr, cap, capv, append, f.status, s, st));
+                                      f.v16, nullptr, cap, capv, append, f.status, s, st0));
     else
         NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
+    if (side) NATSL_TRY(cudaEventRecord(side->join, st0));
     NATSL_TRY(mark());
     float *o_la = p->o_la ? p->o_la : f.o_la;
     if (tensor_cores) {
@@ -317,6 +366,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
                                        p->state_out, nullptr, nullptr, o_la, br.route, s, st));
     }
     NATSL_TRY(mark());
+    if (side) NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, capv, f.sm_idx, f.prefix, o_la, p->w,
                                             p->scale_sm, p->eps, out, p->o_nla, p->lse, br, append,

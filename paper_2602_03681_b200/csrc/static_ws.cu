@@ -49,5 +49,7 @@ extern "C" int natsl_hybrid_fwd_static(const void *q, const void *k, const void 
     if (rc != NATSL_OK) return rc;
     // natsl_hybrid_fwd clears the status word at the head of the workspace and overwrites every
     // other scratch region before reading it, so stale contents of an earlier call are harmless.
-    return natsl_hybrid_fwd(q, k, v, g, beta, route, out, p, ws, (size_t)NATSL_STATIC_WS_BYTES, stream);
+    natsl_params ps = *p;
+    ps.flags |= NATSL_SINGLE_STREAM;     // no library-owned stream: nothing is created by this call
+    return natsl_hybrid_fwd(q, k, v, g, beta, route, out, &ps, ws, (size_t)NATSL_STATIC_WS_BYTES, stream);
 }
