@@ -100,12 +100,14 @@ enum {
                                     two hidden states kept during generation are the linear state
                                     and the KV cache).  natsl_workspace_size depends on the flag
                                     and on p->sm_cap.  Backward: NATSL_ERR_UNSUPPORTED */
-    NATSL_SINGLE_STREAM = 1u << 4      /* forward, tensor-core path: launch everything on the caller's
-                                    stream.  By default the route compaction and the gather of the
-                                    retained K/V run beside the linear branch's prepare kernel on a
-                                    stream the library creates once per device (forked from and
+    NATSL_SINGLE_STREAM = 1u << 4      /* forward and backward, tensor-core path: launch everything on
+                                    the caller's stream.  By default stages that do not depend on
+                                    each other (route compaction + gather beside the linear branch's
+                                    prepare kernel; in the backward also the reverse scan beside the
+                                    softmax branch's backward) run side by side, one of them on a
+                                    stream the library creates once per device, forked from and
                                     joined to the caller's stream with events, so the call is still
-                                    ordered like any other work on that stream).  Also implied by
+                                    ordered like any other work on that stream.  Also implied by
                                     p->stage_events.  natsl_hybrid_fwd_static always sets it */
 };
 

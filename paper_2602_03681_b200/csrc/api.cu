@@ -410,17 +410,32 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
 
 #define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
     NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
-    // ---- forward recomputation, keeping what the backward needs ----
-    NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, nullptr,
-                                   block ? f.status : nullptr, p->B, p->L, p->H, st));
     const uint8_t *block_route = block ? route : nullptr;
     const bool tensor_cores = use_tensor_cores(p);
     const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
+    // Two pairs of independent stages run side by side on the library's side stream (as in the
+    // forward): compaction + gather beside the prepare kernel, and the reverse scan of the linear
+    // branch beside the softmax branch's backward.
+    std::unique_lock<std::mutex> side_lock;
+    SideStream *side = nullptr;
+    if (fused_chunks && !(p->flags & NATSL_SINGLE_STREAM)) {
+        side_lock = std::unique_lock<std::mutex>(g_side_mu);
+        side = side_stream_locked();
+        if (!side) side_lock.unlock();
+    }
+    cudaStream_t st0 = side ? side->st : st;
+    if (side) {
+        NATSL_TRY(cudaEventRecord(side->fork, st));
+        NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
+    }
+    // ---- forward recomputation, keeping what the backward needs ----
+    NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, nullptr,
+                                   block ? f.status : nullptr, p->B, p->L, p->H, st0));
     if (!fused_chunks)
         NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, f.k_smb, nullptr, f.v16, f.k16, p->L,
-                                      p->L, false, f.status, s, st));
+                                      p->L, false, f.status, s, st0));
     else
         NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
                                    f.status, s32, st));
@@ -439,6 +454,10 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gdn_scan_simt(f.q32, f.k32, g, f.W, f.U, f.P, p->scale_la, nullptr, nullptr,
                                        f.S_c, f.Ut, f.o_la, nullptr, s32, st));
     }
+    if (side) {
+        NATSL_TRY(cudaEventRecord(side->join, st0));
+        NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
+    }
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la,
                                             p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
@@ -452,20 +471,29 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                  tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,
                                  tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
                                  tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, s, st));
-    if (tensor_cores)
+    if (side) {     // the reverse scan below goes to the side stream
+        NATSL_TRY(cudaEventRecord(side->fork, st));
+        NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
+    }
+    if (tensor_cores)   // (d = 64: the prepare kernel has left the fp16 copy of q in f.Qh, and the reverse
+                        //  scan on the side stream reads it, so it is not written again)
         NATSL_TRY(launch_softmax_bwd_tc(q, f.Qh, f.dO16, f.k16, f.v16, p->L, f.sm_idx, f.prefix, f.lse,
                                         f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm,
-                                        p->dscore ? f.dGrow : nullptr, f.status, s, st));
+                                        p->dscore ? f.dGrow : nullptr, fused_chunks, f.status, s, st));
     else
         NATSL_TRY(launch_softmax_bwd(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix, f.do_nla,
                                      f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
     // ---- linear branch: reverse scan, then chunk-parallel products ----
     if (tensor_cores)
         NATSL_TRY(launch_gdn_rscan_tc(f.dOla16, f.dOlag16, f.tc, f.S_c, f.dUt, f.dS_c,
-                                      fused_chunks ? nullptr : f.gS, block_route, f.status, s, st));
+                                      fused_chunks ? nullptr : f.gS, block_route, f.status, s, st0));
     else
         NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
                                    f.dS_c, f.gS, s, st));
+    if (side) {
+        NATSL_TRY(cudaEventRecord(side->join, st0));
+        NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
+    }
     AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
                    f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
                    p->scale_la, f.dGrow, f.kappa, dbeta, dg};

@@ -508,12 +508,15 @@ static cudaError_t softmax_bwd_tc_impl(const void *q, void *Qh, const void *dO16
                                        const void *v16, int cap, const int32_t *sm_idx,
                                        const int32_t *pre, const float *lse, const float *Dsm,
                                        float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
-                                       float *dmask, int32_t *status, Shape s, cudaStream_t st) {
+                                       float *dmask, bool qh_ready, int32_t *status, Shape s,
+                                       cudaStream_t st) {
     const uint64_t BH = (uint64_t)s.B * s.H;
-    const size_t pieces = (size_t)s.B * s.L * s.H * (D / 8);
-    to_f16_bhld_kernel<D><<<(unsigned)((pieces + 255) / 256), 256, 0, st>>>(
-        (const __nv_bfloat16 *)q, (__half *)Qh, s.B, s.L, s.H);
-    count_launch();
+    if (!qh_ready) {      // (the linear branch's prepare kernel leaves the same fp16 copy of q behind)
+        const size_t pieces = (size_t)s.B * s.L * s.H * (D / 8);
+        to_f16_bhld_kernel<D><<<(unsigned)((pieces + 255) / 256), 256, 0, st>>>(
+            (const __nv_bfloat16 *)q, (__half *)Qh, s.B, s.L, s.H);
+        count_launch();
+    }
     CUtensorMap mq128, mdo128, mk64, mv64, mq64, mdo64, mk128, mv128;
     if (!tch::make_map_2d(&mq128, Qh, BH * s.L, D, 128) || !tch::make_map_2d(&mdo128, dO16, BH * s.L, D, 128) ||
         !tch::make_map_2d(&mk64, k16, BH * cap, D, 64) || !tch::make_map_2d(&mv64, v16, BH * cap, D, 64) ||
@@ -542,12 +545,13 @@ cudaError_t launch_softmax_bwd_tc(const void *q, void *Qh, const void *dO16, con
                                   const void *v16, int cap, const int32_t *sm_idx,
                                   const int32_t *sm_chunk_prefix, const float *lse, const float *Dsm,
                                   float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
-                                  float *dmask, int32_t *status, Shape s, cudaStream_t st) {
+                                  float *dmask, bool qh_ready, int32_t *status, Shape s,
+                                  cudaStream_t st) {
     if (s.d == 128)
         return softmax_bwd_tc_impl<128>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm,
-                                        scale_sm, dq_sm, dk_sm, dv_sm, dmask, status, s, st);
+                                        scale_sm, dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st);
     return softmax_bwd_tc_impl<64>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm,
-                                   scale_sm, dq_sm, dk_sm, dv_sm, dmask, status, s, st);
+                                   scale_sm, dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st);
 }
 
 }  // namespace natsl
