@@ -471,29 +471,35 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                  tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,
                                  tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
                                  tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, s, st));
-    if (side) {     // the reverse scan below goes to the side stream
+    // Dependencies from here on: the query-side softmax kernel, the key-side one and the reverse
+    // scan need only what is already there; the chunk kernel needs the first and the third; the
+    // scatter of the retained tokens' dk, dv needs the second.  With token-level routing the chunk
+    // kernel therefore does not wait for the key-side kernel: side stream = reverse scan, key-side
+    // kernel, scatter; caller's stream = query-side kernel, chunk kernel.  (Block-level routing:
+    // the chunk kernel adds the scattered gradients, so only the reverse scan goes aside.)
+    const bool kv_aside = side && !block;
+    if (side) {
         NATSL_TRY(cudaEventRecord(side->fork, st));
         NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
     }
+    // ---- linear branch: reverse scan (then chunk-parallel products) ----
+    if (tensor_cores)
+        NATSL_TRY(launch_gdn_rscan_tc(f.dOla16, f.dOlag16, f.tc, f.S_c, f.dUt, f.dS_c,
+                                      fused_chunks ? nullptr : f.gS, block_route, f.status, s, st0));
+    if (side) NATSL_TRY(cudaEventRecord(side->join, st0));
     if (tensor_cores)   // (d = 64: the prepare kernel has left the fp16 copy of q in f.Qh, and the reverse
                         //  scan on the side stream reads it, so it is not written again)
         NATSL_TRY(launch_softmax_bwd_tc(q, f.Qh, f.dO16, f.k16, f.v16, p->L, f.sm_idx, f.prefix, f.lse,
                                         f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm,
-                                        p->dscore ? f.dGrow : nullptr, fused_chunks, f.status, s, st));
+                                        p->dscore ? f.dGrow : nullptr, fused_chunks, f.status, s, st,
+                                        kv_aside ? st0 : st));
     else
         NATSL_TRY(launch_softmax_bwd(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix, f.do_nla,
                                      f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
-    // ---- linear branch: reverse scan, then chunk-parallel products ----
-    if (tensor_cores)
-        NATSL_TRY(launch_gdn_rscan_tc(f.dOla16, f.dOlag16, f.tc, f.S_c, f.dUt, f.dS_c,
-                                      fused_chunks ? nullptr : f.gS, block_route, f.status, s, st0));
-    else
+    if (!tensor_cores)
         NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
                                    f.dS_c, f.gS, s, st));
-    if (side) {
-        NATSL_TRY(cudaEventRecord(side->join, st0));
-        NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
-    }
+    if (side) NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));     // the reverse scan has finished
     AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
                    f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
                    p->scale_la, f.dGrow, f.kappa, dbeta, dg};
@@ -517,7 +523,12 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
                                        false, nullptr, nullptr, nullptr, s, st));
-        NATSL_TRY(launch_gdn_finish(a, dk, dv, s, st, false));   // scatter of the retained tokens' dk, dv
+        // scatter of the retained tokens' dk, dv (rows the chunk kernel does not write)
+        NATSL_TRY(launch_gdn_finish(a, dk, dv, s, kv_aside ? st0 : st, false));
+        if (kv_aside) {
+            NATSL_TRY(cudaEventRecord(side->join, st0));
+            NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
+        }
         return NATSL_OK;
     }
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, s, st));

@@ -78,7 +78,8 @@ cudaError_t launch_softmax_bwd_tc(const void *q, void *Qh, const void *dO16, con
                                   const void *v16, int cap, const int32_t *sm_idx,
                                   const int32_t *sm_chunk_prefix, const float *lse, const float *Dsm,
                                   float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
-                                  float *dmask, bool qh_ready, int32_t *status, Shape s, cudaStream_t st);
+                                  float *dmask, bool qh_ready, int32_t *status, Shape s, cudaStream_t st,
+                                  cudaStream_t st_kv);   // st: query-side kernel, st_kv: key-side kernel
 
 // gdn_tc.cu -- tensor-core chunkwise Gated DeltaNet (bf16 storage): intermediates in workspace
 struct GdnTcWs {

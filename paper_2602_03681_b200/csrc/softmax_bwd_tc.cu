@@ -509,7 +509,7 @@ static cudaError_t softmax_bwd_tc_impl(const void *q, void *Qh, const void *dO16
                                        const int32_t *pre, const float *lse, const float *Dsm,
                                        float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
                                        float *dmask, bool qh_ready, int32_t *status, Shape s,
-                                       cudaStream_t st) {
+                                       cudaStream_t st, cudaStream_t st_kv) {
     const uint64_t BH = (uint64_t)s.B * s.H;
     if (!qh_ready) {      // (the linear branch's prepare kernel leaves the same fp16 copy of q behind)
         const size_t pieces = (size_t)s.B * s.L * s.H * (D / 8);
@@ -535,7 +535,7 @@ static cudaError_t softmax_bwd_tc_impl(const void *q, void *Qh, const void *dO16
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     dim3 gk((s.L + 127) / 128, s.B * s.H);
-    dkv<<<gk, kThreadsB, KLayout<D>::kTotal, st>>>(
+    dkv<<<gk, kThreadsB, KLayout<D>::kTotal, st_kv>>>(
         mq64, mdo64, mk128, mv128, cap, sm_idx, pre, lse, Dsm, scale_sm, dk_sm, dv_sm, dmask, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
@@ -546,12 +546,12 @@ cudaError_t launch_softmax_bwd_tc(const void *q, void *Qh, const void *dO16, con
                                   const int32_t *sm_chunk_prefix, const float *lse, const float *Dsm,
                                   float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
                                   float *dmask, bool qh_ready, int32_t *status, Shape s,
-                                  cudaStream_t st) {
+                                  cudaStream_t st, cudaStream_t st_kv) {
     if (s.d == 128)
         return softmax_bwd_tc_impl<128>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm,
-                                        scale_sm, dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st);
+                                        scale_sm, dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st, st_kv);
     return softmax_bwd_tc_impl<64>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm,
-                                   scale_sm, dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st);
+                                   scale_sm, dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st, st_kv);
 }
 
 }  // namespace natsl
