@@ -476,8 +476,9 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     // scatter of the retained tokens' dk, dv needs the second.  With token-level routing the chunk
     // kernel therefore does not wait for the key-side kernel: side stream = reverse scan, key-side
     // kernel, scatter; caller's stream = query-side kernel, chunk kernel.  (Block-level routing:
-    // the chunk kernel adds the scattered gradients, so only the reverse scan goes aside.)
-    const bool kv_aside = side && !block;
+    // the chunk kernel adds the scattered gradients and so waits for the side stream, but the
+    // own-block kernel, which needs the query-side kernel only, still runs beside the key-side one.)
+    const bool kv_aside = side != nullptr;
     if (side) {
         NATSL_TRY(cudaEventRecord(side->fork, st));
         NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
@@ -509,9 +510,13 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         // token-major buffers (each token is written by exactly one of the two), which the chunk
         // kernel adds to its own dk, dv.
         float *dk_x = f.X3, *dv_x = f.X4;
-        NATSL_TRY(launch_gdn_finish(a, dk_x, dv_x, s32, st, false));
+        NATSL_TRY(launch_gdn_finish(a, dk_x, dv_x, s32, kv_aside ? st0 : st, false));
         NATSL_TRY(launch_softmax_bwd_own_block(q, k, v, f.dO16, f.lse, f.Dsm, route, p->scale_sm,
                                                f.dq_sm, dk_x, dv_x, s, st));
+        if (kv_aside) {
+            NATSL_TRY(cudaEventRecord(side->join, st0));
+            NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
+        }
         NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
                                        true, dk_x, dv_x, p->dscore ? f.kappa : nullptr, s, st));
