@@ -52,6 +52,32 @@ def useful_flops(route: np.ndarray, d: int, C: int = 64):
     return {"gdn_prepare": prepare, "gdn_scan": scan, "softmax_combine": softmax}
 
 
+BWD_FORMULA = ("per chunk with n linear tokens, C = 64: gradient products 8 C n d [P^T dO, dO U~^T, dP K, dP^T Q] "
+               "+ 8 n d^2 [K~ dS, W^T dU~, U~ dS^T, dU~ S0^T] + 4 C d^2 [(s gamma Q)^T dO, dO S0^T] "
+               "+ 12 n^2 d [T^T dU, T^T dW, dU (beta V)^T, dW (beta gamma K)^T, dA K, dA^T K] + 4 n^3 [T^T dT T^T]; "
+               "plus the chunkwise quantities the backward needs again: 6 n^2 d + 2 C n d [K K^T, T beta V, "
+               "T beta gamma K, Q K^T] + 2 n d^2 [W S0]  (all linear: 28 C^2 d + 14 C d^2 + 4 C^3); "
+               "softmax branch: 2.5 x its forward = 10 d sum_i |{j <= i : route_j = 1}| [S, dP, dV, dQ, dK]")
+
+
+def useful_flops_bwd(route: np.ndarray, d: int, C: int = 64):
+    """Useful FLOPs of one backward from the realised routing mask (BWD_FORMULA)."""
+    B, L, H = route.shape
+    r = route.astype(np.int64)
+    n = (C - r.reshape(B, L // C, C, H).sum(2)).astype(np.float64)
+    grad = 8 * C * n * d + 8 * n * d * d + 4 * C * d * d + 12 * n * n * d + 4 * n ** 3
+    again = 6 * n * n * d + 2 * C * n * d + 2 * n * d * d
+    nvis = np.cumsum(r, axis=1)
+    return {"gdn_bwd": float((grad + again).sum()), "softmax_bwd": float(10 * d * nvis.sum())}
+
+
+def tensor_roofline(flops, ms, peaks, peak_kind, traffic=None):
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+            "frac": tf / peaks["bf16_tflops"], "frac_of_nominal_2250": tf / 2250.0,
+            "peak_source": peak_kind, "traffic": traffic, "useful_gflop": flops / 1e9, "ms": ms}
+
+
 def useful_flops_block(route: np.ndarray, d: int, C: int = 64):
     """The same count under block-level routing: every block runs the delta rule with all C of its
     tokens, and a query in a linear block also reads the causal part of its own block."""
@@ -400,7 +426,7 @@ def run_ours(args):
 
     if world == 1 and not args.no_extras:
         line["decode"] = bench_decode(args, peaks, peak_kind, traffic)
-        line["other_workloads"] = bench_other_workloads(peaks)
+        line["other_workloads"] = bench_other_workloads(peaks, peak_kind, traffic)
     if world == 1 and not args.no_cpu:
         xs = x if args.cpu_sample_B >= B else inputs.make_layer_inputs(wl_rank, B=args.cpu_sample_B)
         sb = min(args.cpu_sample_B, B)
@@ -413,7 +439,7 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def bench_other_workloads(peaks):
+def bench_other_workloads(peaks, peak_kind="measured", traffic=None):
     """Forward of the long-context workload and forward + backward of the training workload
     (device-resident inputs, CUDA events, best of 3 after a warm-up), with useful FLOPs."""
     import torch
@@ -461,10 +487,20 @@ def bench_other_workloads(peaks):
             ms[op] = best
         fl = sum((useful_flops_block if block else useful_flops)(x["route"], wl.d, wl.C).values())
         total_ms = sum(ms.values())
+        traffic = traffic or {}
+        base = name.split("/")[0]
         entry = {"ms": ms, "tokens_per_s": wl.B * wl.L / (total_ms * 1e-3),
                  "useful_fwd_gflop": fl / 1e9,
                  "fwd_useful_tflops": fl / (ms["fwd"] * 1e-3) / 1e12,
-                 "fwd_frac_of_bf16_peak": fl / (ms["fwd"] * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+                 "fwd_frac_of_bf16_peak": fl / (ms["fwd"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                 "roofline": {"fwd": tensor_roofline(fl, ms["fwd"], peaks, peak_kind,
+                                                     None if block else traffic.get(f"fwd:{base}"))}}
+        if "bwd" in ops and not block:
+            fb = sum(useful_flops_bwd(x["route"], wl.d, wl.C).values())
+            entry["useful_bwd_gflop"] = fb / 1e9
+            entry["bwd_flop_formula"] = BWD_FORMULA
+            entry["roofline"]["bwd"] = tensor_roofline(fb, ms["bwd"], peaks, peak_kind, traffic.get(f"bwd:{base}"))
+            entry["roofline"]["fwd+bwd"] = tensor_roofline(fl + fb, total_ms, peaks, peak_kind)
         res[name] = entry
         del d, ws
         torch.cuda.empty_cache()

@@ -5,7 +5,7 @@
  * (1 = softmax token, K/V retained; 0 = linear token, folded into the state):
  *
  *   linear branch  (Section 4.3, Gated DeltaNet equation; decay on every token, the
- *                   "always apply the decay" equation; update only for linear tokens,
+ *                   decay-update equation of the same section; update only for linear tokens,
  *                   Section 4.1 case equation for the chunk state):
  *       Sbar = exp(g_i) S ;  S = r_i ? Sbar : Sbar + beta_i k_i^T (v_i - k_i Sbar)
  *       o_la_i = scale_la * q_i S
@@ -16,11 +16,18 @@
  *       RMSnorm(x) = x / sqrt(mean_d(x^2) + eps)
  *
  * Every pointer below is a DEVICE pointer unless it says "host".  The caller owns all
- * buffers and the stream; the library allocates nothing, keeps no per-call state, and only
- * enqueues kernels on `stream` (a cudaStream_t passed as void*; NULL = default stream).
- * Calls are asynchronous.  All tensors are dense, row-major, innermost dimension
- * contiguous, in the shapes given.  Base pointers of q,k,v,out,dout,dq,dk,dv, the caches
- * and the workspace must be 16-byte aligned.
+ * buffers and the stream; the library allocates no device memory and keeps no per-call state.
+ * Calls are asynchronous and ordered on `stream` (a cudaStream_t passed as void*; NULL = default
+ * stream) like any other work of that stream.  What the library does own, per device and created
+ * on the first forward or backward call there that may use it: one non-blocking stream and two
+ * events, on which stages that do not depend on each other run beside the caller's stream (forked
+ * from it and joined back into it within the call), and one process-wide mutex that covers the
+ * enqueue of such a call, because the two events are shared.  NATSL_SINGLE_STREAM and
+ * natsl_hybrid_fwd_static use none of this.  The device of `stream` and of all tensors must be
+ * the current device of the calling thread.
+ * All tensors are dense, row-major, innermost dimension contiguous, in the shapes given (no
+ * strides are taken: a caller with another layout makes a contiguous copy).  Base pointers of
+ * q,k,v,out,dout,dq,dk,dv, the caches and the workspace must be 16-byte aligned.
  *
  * Precision of the default path for NATSL_BF16 (tcgen05 tensor cores): q, k, v are used as
  * given; every computed tensor-core operand is held in fp16 with fp32 accumulation, and q, k, v
@@ -72,7 +79,7 @@ enum {
                                     state transition, a small kernel chains the segments); the
                                     results agree to rounding */
     NATSL_BLOCK_ROUTING = 1u << 2,     /* forward (both paths), backward: block-level routing, the paper's
-                                    default (Section 4.1, "compute the inner-chunk correlation";
+                                    default (Section 4.1, paragraph on intra-chunk correlations;
                                     Section 4.3, chunk size = GDN chunk size).  `route` holds one
                                     decision per block of C = 64 tokens, repeated over the block's
                                     tokens.  The decision is known only when the block is complete,
@@ -203,12 +210,20 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
  *   - All calls on a device share the one array, which keeps the previous call's contents; the
  *     library re-initialises what it needs.  Two calls that overlap on the GPU (different
  *     streams, no ordering between them) race on it: keep them on one stream or order them.
+ *   - The array is the one of the calling thread's current device: `stream` and all tensors must
+ *     belong to that device.
+ *   - Conditions only the device can see (NATSL_ERR_ROUTE, NATSL_ERR_CACHE_FULL, NATSL_ERR_TIMEOUT)
+ *     go to the status word at the head of the array; natsl_static_status reads it.
  * Errors otherwise as natsl_hybrid_fwd.
  */
 #define NATSL_STATIC_WS_BYTES (32u << 20)
 int natsl_hybrid_fwd_static(const void *q, const void *k, const void *v, const float *g,
                             const float *beta, const uint8_t *route, void *out,
                             const natsl_params *p, void *stream);
+
+/* natsl_device_status for the built-in scratch of the current device (no counterpart in the
+ * paper): synchronises `stream`, returns and clears the status word.  Allocates nothing. */
+int natsl_static_status(void *stream);
 
 /*
  * Backward of natsl_hybrid_fwd's `out` (Section 4.2 states the properties: the softmax-branch
@@ -278,6 +293,18 @@ const char *natsl_stage_name(int op, int i);
 
 /* Number of kernels this library has launched in this process so far (host counter). */
 uint64_t natsl_launch_count(void);
+
+/*
+ * Test hook for the time-out path (no counterpart in the paper).  Every device-side wait of the
+ * tensor-core kernels is bounded (about two seconds by default); when a wait runs out the kernel
+ * records NATSL_ERR_TIMEOUT in the status word, waits for its own copies in flight, frees its
+ * tensor memory and returns.  This call sets, for all following forward calls of the process,
+ *   kcycles              the bound in units of 1024 clock cycles (0: back to the default), and
+ *   withhold_scan_flags  non-zero: the scan does not raise the per-chunk counters the softmax
+ *                        kernel's epilogue waits for, so that exactly this wait runs out.
+ * Nothing faults and nothing hangs: the call returns after the bound and reports the time-out.
+ */
+void natsl_debug_set_wait_limit(uint32_t kcycles, int withhold_scan_flags);
 
 #ifdef __cplusplus
 }

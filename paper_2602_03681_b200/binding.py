@@ -27,8 +27,9 @@ ERR_ROUTE = -11
 
 EXPORTS = ["natsl_workspace_size", "natsl_route_compact", "natsl_hybrid_fwd", "natsl_hybrid_bwd",
            "natsl_decode_step", "natsl_decode_block_end", "natsl_device_status", "natsl_hybrid_fwd_static",
-           "natsl_score_layer",
+           "natsl_score_layer", "natsl_static_status", "natsl_debug_set_wait_limit",
            "natsl_stage_name", "natsl_launch_count", "natsl_strerror"]
+ERR_TIMEOUT = -10
 ERR_TOO_LARGE = -9
 STATIC_WS_BYTES = 32 << 20
 
@@ -69,8 +70,10 @@ def lib() -> ctypes.CDLL:
         _lib.natsl_stage_name.restype = ctypes.c_char_p
         _lib.natsl_stage_name.argtypes = [ctypes.c_int, ctypes.c_int]
         _lib.natsl_launch_count.restype = ctypes.c_uint64
-        for name in EXPORTS[:7]:
+        for name in EXPORTS[:7] + ["natsl_score_layer", "natsl_static_status"]:
             getattr(_lib, name).restype = ctypes.c_int
+        _lib.natsl_debug_set_wait_limit.restype = None
+        _lib.natsl_debug_set_wait_limit.argtypes = [ctypes.c_uint32, ctypes.c_int]
     return _lib
 
 
@@ -203,6 +206,17 @@ def natsl_score_layer(x, w_score, scores, route, p: natsl_params):
 
 def natsl_device_status(ws) -> int:
     return int(lib().natsl_device_status(_ptr(ws), _stream()))
+
+
+def natsl_static_status() -> int:
+    """Status word of the library's built-in scratch on the current device (synchronises)."""
+    return int(lib().natsl_static_status(_stream()))
+
+
+def natsl_debug_set_wait_limit(kcycles: int, withhold_scan_flags: bool = False):
+    """Test hook: bound of the device-side waits in units of 1024 cycles (0 = default) and whether
+    the scan withholds the per-chunk flags the softmax kernel waits for."""
+    lib().natsl_debug_set_wait_limit(int(kcycles), 1 if withhold_scan_flags else 0)
 
 
 # ---------------------------------------------------------------------------------------------

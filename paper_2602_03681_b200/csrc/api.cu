@@ -10,6 +10,11 @@
 using namespace natsl;
 
 namespace natsl {
+// Test hooks (natsl_debug_set_wait_limit): a bound for the device-side waits of the following
+// launches, and whether the scan withholds the per-chunk flags the softmax kernel waits for.
+static std::atomic<uint32_t> g_debug_wait_kcycles{0};
+static std::atomic<int> g_debug_withhold_flags{0};
+int debug_wait_kcycles() { return (int)g_debug_wait_kcycles.load(std::memory_order_relaxed); }
 static std::atomic<uint64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 }  // namespace natsl
@@ -47,9 +52,11 @@ int check_params(const natsl_params *p, bool needs_L) {
 Shape shape_of(const natsl_params *p) { return Shape{p->B, p->H, p->L, p->d, p->dtype == NATSL_BF16}; }
 
 struct FwdWs {
-    int32_t *status, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
+    int32_t *status, *emit_flags, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
+    size_t head_bytes;          // status page + emit_flags: cleared at the start of every call
     void *k_sm, *v_sm, *v16;
-    float *W, *U, *P, *o_la;    // W, U, P: fp32 CUDA-core path only
+    void *o_la16;               // tensor-core path: the linear read-out as fp16 [B,L,H,d]
+    float *W, *U, *P, *o_la;    // fp32 CUDA-core path only
     GdnTcWs tc;                 // tensor-core path only
     float *seg_incr, *seg_trans, *seg_start;   // segmented scan: [B*H, nseg, d, d] each
     size_t bytes;
@@ -75,6 +82,9 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
     const size_t B = p->B, H = p->H, L = p->L, d = p->d, NC = L / kC;
     const size_t esz = p->dtype == NATSL_BF16 ? 2 : 4;
     f.status = c.take<int32_t>(kStatusBytes / 4);
+    // one counter per chunk, raised by the scan as the chunk's read-out is complete (tensor-core path)
+    f.emit_flags = c.take<int32_t>(use_tensor_cores(p) ? B * H * NC : 0);
+    f.head_bytes = c.off;
     f.sm_idx = c.take<int32_t>(B * H * L);
     f.prefix = c.take<int32_t>(B * H * (NC + 1));
     f.lin_idx = c.take<int32_t>(B * H * L);
@@ -97,15 +107,18 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
         f.seg_incr = c.take<float>(segf);
         f.seg_trans = c.take<float>(segf);
         f.seg_start = c.take<float>(segf);
+        f.o_la16 = c.take<char>(B * L * H * d * 2);
+        f.o_la = nullptr;
     } else {
         f.v16 = nullptr;
+        f.o_la16 = nullptr;
         f.tc = GdnTcWs{};
         f.seg_incr = f.seg_trans = f.seg_start = nullptr;
         f.W = c.take<float>(B * L * H * d);
         f.U = c.take<float>(B * L * H * d);
         f.P = c.take<float>(B * H * NC * kC * kC);
+        f.o_la = c.take<float>(B * L * H * d);
     }
-    f.o_la = c.take<float>(B * L * H * d);
     f.bytes = c.off;
     return f;
 }
@@ -121,34 +134,58 @@ struct BwdWs {
     float *Gcum, *lse, *Dsm, *dGrow, *kappa, *gS;            // [B,H,L] (gS: [B,H,NC,d/32])
     void *k_smb, *k16, *v16, *Qh, *dO16;                     // tensor-core softmax branch: 16-bit [B,H,L,d]
     void *dOla16, *dOlag16;                                  // tensor-core reverse scan: fp16 [B,H,L,d]
+    void *o_la16;                                            // linear read-out as fp16 [B,L,H,d]
     GdnTcWs tc;                                              // tensor-core forward recomputation
     float *Tinv;                                             // (I + A)^-1 per chunk [B,H,NC,64,64]
     size_t bytes;
 };
 
+// Only what the selected path uses is carved (a buffer the path does not touch gets no bytes and a
+// pointer nobody dereferences).  Paths: `fused` = tensor cores with d = 64 (reverse scan + one
+// fused kernel per chunk), tensor cores with d = 128 (chunk-level products as batched tile GEMMs),
+// fp32 CUDA cores.  Three pairs with disjoint lifetimes share their bytes on the tensor-core paths:
+// o_la (dead once the combination's backward has run) / dUt (written by the reverse scan after it),
+// o_nla / dq_sm likewise, and the fp16 o_la / the fp16 gradient copy dO16.
 BwdWs carve_bwd(const natsl_params *p, void *ws) {
     Carver c(ws);
     BwdWs f;
     const size_t B = p->B, H = p->H, L = p->L, d = p->d, NC = L / kC;
     const size_t TM = B * L * H * d, CC = B * H * NC * kC * kC, ST = B * H * NC * d * d, BHL = B * H * L;
+    const bool tcs = use_tensor_cores(p), fused = tcs && p->d == 64, general = !fused;
+    const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
+    auto tm = [&](bool need) { return c.take<float>(need ? TM : 0); };
+    auto cc = [&](bool need) { return c.take<float>(need ? CC : 0); };
     f.status = c.take<int32_t>(kStatusBytes / 4);
     f.sm_idx = c.take<int32_t>(BHL);
     f.prefix = c.take<int32_t>(B * H * (NC + 1));
     f.lin_idx = c.take<int32_t>(BHL);
     f.n_lin = c.take<int32_t>(B * H * NC);
     f.sm_len = c.take<int32_t>(B * H);
-    float **tm[] = {&f.k_sm32, &f.v_sm32, &f.q32, &f.k32, &f.v32, &f.W, &f.U, &f.Ut, &f.o_la,
-                    &f.o_nla, &f.do_la, &f.do_nla, &f.dUt, &f.dQg, &f.dW, &f.dKt, &f.dKb, &f.dVb,
-                    &f.X1p, &f.X2, &f.X3, &f.X4, &f.dq_sm, &f.dk_sm, &f.dv_sm};
-    for (float **t : tm) *t = c.take<float>(TM);
-    float **cc[] = {&f.P, &f.Abar, &f.M, &f.N, &f.Mg, &f.Ms, &f.Ns};
-    for (float **t : cc) *t = c.take<float>(CC);
+    f.k_sm32 = tm(!tcs); f.v_sm32 = tm(!tcs);
+    f.q32 = tm(general); f.k32 = tm(general); f.v32 = tm(general);
+    f.W = tm(general); f.U = tm(general);
+    f.Ut = tm(true);
+    f.o_la = tm(true);
+    f.o_nla = tm(true);
+    f.do_la = tm(true);
+    f.do_nla = tm(!tcs);
+    f.dUt = tcs ? f.o_la : tm(true);
+    f.dQg = tm(general); f.dW = tm(general); f.dKt = tm(general); f.dKb = tm(general); f.dVb = tm(general);
+    f.X1p = tm(general); f.X2 = tm(general);
+    f.X3 = tm(general || block); f.X4 = tm(general || block);
+    f.dq_sm = tcs ? f.o_nla : tm(true);
+    f.dk_sm = tm(true); f.dv_sm = tm(true);
+    f.P = cc(!tcs); f.Abar = cc(!tcs);
+    f.M = cc(general); f.N = cc(general); f.Mg = cc(general); f.Ms = cc(general); f.Ns = cc(general);
     f.S_c = c.take<float>(ST);
     f.dS_c = c.take<float>(ST);
-    float **sm[] = {&f.Gcum, &f.lse, &f.Dsm, &f.dGrow, &f.kappa};
-    for (float **t : sm) *t = c.take<float>(BHL);
-    f.gS = c.take<float>(B * H * NC * (d / 32));
-    const size_t h16 = use_tensor_cores(p) ? TM * 2 : 0;
+    f.Gcum = c.take<float>(BHL);
+    f.lse = c.take<float>(BHL);
+    f.Dsm = c.take<float>(BHL);
+    f.dGrow = c.take<float>(BHL);
+    f.kappa = c.take<float>(BHL);
+    f.gS = c.take<float>(general ? B * H * NC * (d / 32) : 0);
+    const size_t h16 = tcs ? TM * 2 : 0;
     f.k_smb = c.take<char>(h16);
     f.k16 = c.take<char>(h16);
     f.v16 = c.take<char>(h16);
@@ -156,8 +193,9 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.dO16 = c.take<char>(h16);
     f.dOla16 = c.take<char>(h16);
     f.dOlag16 = c.take<char>(h16);
+    f.o_la16 = f.dO16;
     f.tc = GdnTcWs{};
-    if (use_tensor_cores(p)) {
+    if (tcs) {
         f.tc.Qh = f.Qh;                       // the same fp16 copy of q serves both branches
         f.tc.Kh = c.take<char>(h16);
         f.tc.Wt = c.take<char>(h16);
@@ -188,6 +226,24 @@ struct SideStream {
 };
 SideStream g_side[64];
 std::mutex g_side_mu;
+
+// Joins the side stream back into the caller's stream when a call leaves early after the fork,
+// so that no library-owned stream is left with work the caller's stream does not wait for.
+struct SideJoin {
+    SideStream *side = nullptr;
+    cudaStream_t st = nullptr;
+    bool pending = false;
+    void forked(SideStream *s, cudaStream_t caller) { side = s; st = caller; pending = true; }
+    cudaError_t join() {
+        if (!pending) return cudaSuccess;
+        pending = false;
+        cudaError_t e = cudaEventRecord(side->join, side->st);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, side->join, 0);
+        return e;
+    }
+    ~SideJoin() { (void)join(); }
+};
+
 
 SideStream *side_stream_locked() {   // g_side_mu held; nullptr: run everything on the caller's stream
     int dev = 0;
@@ -257,7 +313,7 @@ int natsl_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk
     if (rc != NATSL_OK) return rc;
     if (!route || !sm_idx || !sm_chunk_prefix || !lin_idx || !n_lin) return NATSL_ERR_NULL;
     cudaError_t e = launch_route_compact(route, sm_idx, sm_chunk_prefix, lin_idx, n_lin, nullptr,
-                                         nullptr, nullptr, p->B, p->L, p->H,
+                                         nullptr, nullptr, 0, p->B, p->L, p->H,
                                          static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
 }
@@ -308,12 +364,13 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
             return cudaEventRecord(static_cast<cudaEvent_t>(p->stage_events[stage++]), st);
         return cudaSuccess;
     };
-    NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
+    NATSL_TRY(cudaMemsetAsync(f.status, 0, f.head_bytes, st));
     NATSL_TRY(mark());
     // Stage 0 (compaction, gather) beside stage 1 (prepare) on the side stream -- unless the caller
     // asks for one stream or for per-stage events, whose differences are only meaningful in sequence.
     std::unique_lock<std::mutex> side_lock;
     SideStream *side = nullptr;
+    SideJoin side_join;
     if (tensor_cores && !(p->flags & NATSL_SINGLE_STREAM) && !p->stage_events) {
         side_lock = std::unique_lock<std::mutex>(g_side_mu);
         side = side_stream_locked();
@@ -323,57 +380,66 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     if (side) {
         NATSL_TRY(cudaEventRecord(side->fork, st));
         NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
+        side_join.forked(side, st);
     }
     int32_t *sm_len = want_cache ? p->sm_len : f.sm_len;
     void *k_sm = want_cache ? p->k_sm : f.k_sm, *v_sm = want_cache ? p->v_sm : f.v_sm;
     const int32_t cap = want_cache ? p->sm_cap : p->L;
     const int32_t capv = append ? p->sm_cap : p->L;          // rows per head of the fp16 V copy
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, sm_len,
-                                   append ? sm_len : nullptr, block ? f.status : nullptr, p->B, p->L,
-                                   p->H, st0));
+                                   append ? sm_len : nullptr, block ? f.status : nullptr, cap, p->B,
+                                   p->L, p->H, st0));
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
                                       f.v16, nullptr, cap, capv, append, f.status, s, st0));
     else
         NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
-    if (side) NATSL_TRY(cudaEventRecord(side->join, st0));
     NATSL_TRY(mark());
-    float *o_la = p->o_la ? p->o_la : f.o_la;
     if (tensor_cores) {
         // block-level routing: every token takes part in the delta rule of its own block
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc,
                                         GdnTcExport{}, f.status, s, st));
         NATSL_TRY(mark());
+        // The side stream joins here, before the scan, so that nothing stands between the scan and
+        // the softmax kernel in the stream: the softmax kernel is launched as a programmatic dependent
+        // of the scan, starts once the scan's CTAs are all resident, runs its Q K^T / P V loop beside
+        // it on the multiprocessors the scan leaves free, and picks up o_la chunk by chunk behind the
+        // counters the scan raises.  Per-stage events and NATSL_SINGLE_STREAM switch this off
+        // (stages in sequence).
+        NATSL_TRY(side_join.join());
+        const bool beside = !p->stage_events && !(p->flags & NATSL_SINGLE_STREAM);
+        int32_t *flags_scan = beside && !g_debug_withhold_flags.load(std::memory_order_relaxed) ? f.emit_flags : nullptr;
+        const int32_t *flags_softmax = beside ? f.emit_flags : nullptr;
+        const ScanOut so{f.o_la16, p->o_la, flags_scan};
         const int nseg = scan_segments(p);
         if (nseg > 1) {   // few (batch, head) pairs: segments in parallel, chained by their transitions
             ScanSegments sg{1, nseg, (int)(p->L / kC) / nseg, f.seg_incr, f.seg_trans, f.seg_start};
-            NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, o_la, GdnTcExport{}, sg,
+            NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, so, GdnTcExport{}, sg,
                                          br.route, f.status, s, st));
             NATSL_TRY(launch_scan_combine(p->state_in, sg, s, st));
             sg.mode = 2;
-            NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, p->state_out, o_la, GdnTcExport{}, sg,
+            NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, p->state_out, so, GdnTcExport{}, sg,
                                          br.route, f.status, s, st));
         } else {
-            NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, p->state_out, o_la, GdnTcExport{},
+            NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, p->state_out, so, GdnTcExport{},
                                          ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, br.route,
                                          f.status, s, st));
         }
+        NATSL_TRY(mark());
+        NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, capv, f.sm_idx, f.prefix, f.o_la16,
+                                            flags_softmax, p->w, p->scale_sm, p->eps, out, p->o_nla,
+                                            p->lse, br, append, f.status, s, st));
     } else {
+        float *o_la = p->o_la ? p->o_la : f.o_la;
         NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.W,
                                           f.U, f.P, nullptr, nullptr, s, st));
         NATSL_TRY(mark());
         NATSL_TRY(launch_gdn_scan_simt(q, k, g, f.W, f.U, f.P, p->scale_la, p->state_in,
                                        p->state_out, nullptr, nullptr, o_la, br.route, s, st));
-    }
-    NATSL_TRY(mark());
-    if (side) NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
-    if (tensor_cores)
-        NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, capv, f.sm_idx, f.prefix, o_la, p->w,
-                                            p->scale_sm, p->eps, out, p->o_nla, p->lse, br, append,
-                                            f.status, s, st));
-    else
+        NATSL_TRY(mark());
         NATSL_TRY(launch_softmax_combine_simt(q, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
                                               p->scale_sm, p->eps, out, p->o_nla, p->lse, br, s, st));
+    }
     NATSL_TRY(mark());
 #undef NATSL_TRY
     return NATSL_OK;
@@ -430,7 +496,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     }
     // ---- forward recomputation, keeping what the backward needs ----
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, nullptr,
-                                   block ? f.status : nullptr, p->B, p->L, p->H, st0));
+                                   block ? f.status : nullptr, p->L, p->B, p->L, p->H, st0));
     if (!fused_chunks)
         NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
     if (tensor_cores)
@@ -445,8 +511,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                              f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc, ex,
                                         f.status, s, st));
-        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, f.o_la, ex,
-                                     ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, block_route,
+        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, ScanOut{f.o_la16, f.o_la, nullptr},
+                                     ex, ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, block_route,
                                      f.status, s, st));
     } else {
         NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
@@ -459,8 +525,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
     }
     if (tensor_cores)
-        NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la,
-                                            p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
+        NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la16,
+                                            nullptr, p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
                                             BlockRouting{block_route, k, v}, false, f.status, s, st));
     else
         NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
@@ -592,6 +658,11 @@ int natsl_decode_block_end(const uint8_t *route_block, const float *g_block, flo
                                             block_len, ws, shape_of(p),
                                             static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
+}
+
+void natsl_debug_set_wait_limit(uint32_t kcycles, int withhold_scan_flags) {
+    g_debug_wait_kcycles.store(kcycles > 0x7fffffffu ? 0x7fffffffu : kcycles, std::memory_order_relaxed);
+    g_debug_withhold_flags.store(withhold_scan_flags ? 1 : 0, std::memory_order_relaxed);
 }
 
 int natsl_device_status(void *ws, void *stream) {

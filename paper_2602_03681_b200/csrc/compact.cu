@@ -20,7 +20,7 @@ __global__ void __launch_bounds__(kCompactThreads)
 route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm_idx,
                      int32_t *__restrict__ sm_chunk_prefix, int32_t *__restrict__ lin_idx,
                      int32_t *__restrict__ n_lin, int32_t *sm_len, const int32_t *base_in,
-                     int32_t *__restrict__ block_status, int L, int H) {
+                     int32_t *__restrict__ block_status, int cap, int L, int H) {
     __shared__ unsigned long long bits[kCompactTile];
     __shared__ int excl[kCompactTile];
     __shared__ int warp_tot[kCompactThreads / 32];
@@ -115,7 +115,9 @@ route_compact_kernel(const uint8_t *__restrict__ route, int32_t *__restrict__ sm
     }
     if (threadIdx.x == 0) {
         sm_chunk_prefix[(size_t)bh * (NC + 1) + NC] = base;
-        if (sm_len) sm_len[bh] = base;
+        // The stored length never exceeds the rows the cache has (the gather stops there and
+        // reports the overflow), so a later decode step cannot be led past the head's rows.
+        if (sm_len) sm_len[bh] = cap > 0 ? min(base, cap) : base;
     }
 }
 
@@ -146,10 +148,10 @@ gather_kv_kernel(const T *__restrict__ k, const T *__restrict__ v, const int32_t
 
 cudaError_t launch_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk_prefix,
                                  int32_t *lin_idx, int32_t *n_lin, int32_t *sm_len,
-                                 const int32_t *base_in, int32_t *block_status, int B, int L, int H,
-                                 cudaStream_t st) {
-    route_compact_kernel<<<B * H, kCompactThreads, 0, st>>>(route, sm_idx, sm_chunk_prefix, lin_idx,
-                                                            n_lin, sm_len, base_in, block_status, L, H);
+                                 const int32_t *base_in, int32_t *block_status, int cap, int B, int L,
+                                 int H, cudaStream_t st) {
+    route_compact_kernel<<<B * H, kCompactThreads, 0, st>>>(route, sm_idx, sm_chunk_prefix, lin_idx, n_lin,
+                                                            sm_len, base_in, block_status, cap, L, H);
     count_launch();
     return cudaGetLastError();
 }

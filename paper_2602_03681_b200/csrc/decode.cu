@@ -82,7 +82,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
     __shared__ __align__(16) float qs[D], ks[D], vs[D];
     __shared__ float sm_m[kTileKeys], sm_z[kTileKeys];
     __shared__ float norm_red[2][kWarps];
-    __shared__ int s_last, s_abort;
+    __shared__ int s_last, s_abort[2];   // s_abort[1]: wait limit (see mbar_wait)
 
     const int part = blockIdx.x, bh = blockIdx.y;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -97,7 +97,11 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
     const int rv = route[bh];
     const bool r = rv != 0;                        // append, and attend to itself
     const bool fold = rv != 1;                     // delta rule
-    const int n_old = cache_len[bh];
+    // A stored length outside [0, cap] (a prefill whose cache overflowed, a caller's mistake) is
+    // clamped, so that no copy below can leave the head's rows, and reported.
+    const int n_raw = cache_len[bh];
+    const int n_old = min(max(n_raw, 0), cap);
+    if (n_raw != n_old && tid == 0 && part == 0) atomicMin(status, (int)NATSL_ERR_CACHE_FULL);
     const bool cache_full = r && n_old >= cap;     // no room: the sequence is left untouched
     if (tid < D) {
         qs[tid] = to_f32(q[(size_t)bh * D + tid]);
@@ -106,11 +110,12 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
     }
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], kWorkThreads); }
-        s_abort = 0;
+        s_abort[0] = 0;
+        s_abort[1] = 0;
         fence_mbar_init();
     }
     __syncthreads();
-    volatile int *abort_flag = &s_abort;
+    volatile int *abort_flag = s_abort;
 
     if (part < kDecodeParts) {
         // ---------------- cache CTA: one slice of the retained K/V ----------------
@@ -134,8 +139,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
                 }
                 if (*abort_flag)           // let the copies already issued land before the CTA retires
                     for (int u = max(t_begin, t - kStages); u < t; ++u)
-                        mbar_wait(&full[(u - t_begin) % kStages], ((u - t_begin) / kStages) & 1,
-                                  abort_flag);
+                        mbar_wait_drain(&full[(u - t_begin) % kStages], ((u - t_begin) / kStages) & 1);
             }
         } else {
             const int stream = tid / kLpk, piece = tid % kLpk;
@@ -267,7 +271,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
         const int old = atomicAdd(ticket, 1);
         s_last = old == kCtasPerHead - 1;
         if (s_last) *ticket = 0;                      // ready for the next step
-        if (s_abort) atomicMin(status, (int)NATSL_ERR_TIMEOUT);
+        if (s_abort[0]) atomicMin(status, (int)NATSL_ERR_TIMEOUT);
     }
     __syncthreads();
     if (!s_last) return;

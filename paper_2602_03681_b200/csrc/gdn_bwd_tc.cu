@@ -50,7 +50,7 @@ template <int D> struct RsLayout {
 struct RsMisc {
     uint64_t full[kRsStages], empty[kRsStages], barA, barX, barB, barY;
     uint32_t tmem_base;
-    int abort_flag;
+    int abort_flag, wait_kcycles;   // in this order: the waits read the limit as abort_flag[1]
 };
 static_assert(sizeof(RsMisc) <= kRsMisc, "misc page too small");
 
@@ -62,7 +62,7 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
                     const __grid_constant__ CUtensorMap map_wt,    // W^T [B*H*NC*D][64], box D
                     const __grid_constant__ CUtensorMap map_ph,    // P [B*H*NC*64][64], box 64
                     const float *__restrict__ Gd, float *__restrict__ dUt, float *__restrict__ dS_c,
-                    const uint8_t *__restrict__ block_route, int32_t *status, int L, int H) {
+                    const uint8_t *__restrict__ block_route, int32_t *status, int L, int H, int wait_kcycles) {
     using SL = RsLayout<D>;
     constexpr int KB = SL::KB;
     constexpr int kHalfCols = D / 2;
@@ -83,6 +83,7 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
         mbar_init(&ms.barX, 1);
         mbar_init(&ms.barY, 1);
         ms.abort_flag = 0;
+        ms.wait_kcycles = wait_kcycles;
         fence_mbar_init();
     }
     if (warp == 8) tmem_alloc(&ms.tmem_base, SL::kTmemCols);
@@ -111,9 +112,8 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
                 bulk_load_1d(smem + SL::oG + (n % kRsDecaySlots) * SL::kG, Gd + ((size_t)bh * NC + c) * 128,
                              SL::kG, &ms.full[s]);
             }
-            if (*abort_flag)
-                for (int u = max(0, n - kRsStages); u < n; ++u)
-                    mbar_wait(&ms.full[u % kRsStages], (u / kRsStages) & 1, abort_flag);
+            for (int u = max(0, n - kRsStages); u < n; ++u)      // no copy in flight at retirement
+                mbar_wait_drain(&ms.full[u % kRsStages], (u / kRsStages) & 1);
         }
     } else if (warp == 8) {
         if (lane == 0) {
@@ -822,7 +822,7 @@ static cudaError_t rscan_tc_impl(const void *dO16, const void *dOg16, const GdnT
                                          RsLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
     kernel<<<s.B * s.H, kRsThreads, RsLayout<D>::kTotal, st>>>(
-        mdo, mdog, mqh, mkh, mwt, mph, ws.Gd, dUt, dS_c, block_route, status, s.L, s.H);
+        mdo, mdog, mqh, mkh, mwt, mph, ws.Gd, dUt, dS_c, block_route, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (gS) {     // (the fused chunk kernel forms <dS1, S0> itself)

@@ -71,8 +71,8 @@ template <int D> struct PrepLayout {
 struct PrepMisc {
     uint64_t barLoad, barConv, barM, barXfree, barT, barUW;
     uint32_t tmem_base;
-    int abort_flag;
-    float G[64], bt[64], btg[64], wsum[2];   // cumulative log decay, beta~, beta~ gamma
+    int abort_flag, wait_kcycles;   // in this order: the waits read the limit as abort_flag[1]
+    alignas(16) float G[64], bt[64], btg[64], wsum[2];   // cumulative log decay, beta~, beta~ gamma (read in pairs)
 };
 static_assert(sizeof(PrepMisc) <= kPrepMisc, "misc page too small");
 
@@ -86,7 +86,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                       const float *__restrict__ beta, const uint8_t *__restrict__ route,
                       float scale_la, __half *__restrict__ Wt, float *__restrict__ Ut,
                       __half *__restrict__ Ph, float *__restrict__ Gd, GdnTcExport ex,
-                      int32_t *status, int L, int H) {
+                      int32_t *status, int L, int H, int prefetch_ahead, int wait_kcycles) {
     using PL = PrepLayout<D>;
     constexpr int KB = PL::KB;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -109,6 +109,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         mbar_init(&ms.barT, kRowThreads);
         mbar_init(&ms.barUW, 1);
         ms.abort_flag = 0;
+        ms.wait_kcycles = wait_kcycles;
         fence_mbar_init();
     }
     if (warp == 4) tmem_alloc(&ms.tmem_base, 128);
@@ -130,6 +131,17 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 tma_load_4d(sQK + kb * 16384 + 8192, &map_k, &ms.barLoad, kb * 64, h, tok0, b);
                 tma_load_4d(sQK + kb * 16384, &map_q, &ms.barLoad, kb * 64, h, tok0, b);
                 tma_load_4d(sV + kb * 8192, &map_v, &ms.barLoad, kb * 64, h, tok0, b);
+            }
+            {   // the tiles of the CTA that will follow this one on its SM: towards L2 now, so that its
+                // wait for the first bytes is an L2 round trip, not a DRAM one behind a full wave's loads
+                const int lin = bh * NC + c + prefetch_ahead;
+                const int bh2 = lin / NC, c2 = lin % NC;
+                if (prefetch_ahead > 0 && bh2 < (int)gridDim.y)
+                    for (int kb = 0; kb < KB; ++kb) {
+                        tma_prefetch_4d(&map_k, kb * 64, bh2 % H, c2 * kC, bh2 / H);
+                        tma_prefetch_4d(&map_q, kb * 64, bh2 % H, c2 * kC, bh2 / H);
+                        tma_prefetch_4d(&map_v, kb * 64, bh2 % H, c2 * kC, bh2 / H);
+                    }
             }
             bool ok = mbar_wait(&ms.barConv, 0, abort_flag);       // tiles converted to fp16
             if (ok) {
@@ -487,9 +499,18 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 //   (c) [for chunk c-1, behind the MMAs of (b)]  o_la^T = scale_la diag(gamma) QS + D3
 //   next chunk: S_{c+1} = gamma_C S_c + dS
 // QS and D3 are double-buffered in TMEM so that (c) of chunk c-1 runs behind the MMAs of chunk c.
+// The read-out leaves the kernel as fp16 in the orientation the row threads hold it in, one tile
+// per chunk in 16-byte pieces of 8 tokens: o_laT [B,H,L/C,8 pieces,d,8 tokens], row r of piece p at
+// slot r ^ p.  A thread then stores four 16-byte pieces per chunk and a warp's store is 512
+// contiguous bytes, where token-major rows took one narrow store per token (the load/store unit's
+// instruction rate, not its bytes, bounded that version).  The softmax kernel's epilogue copies the
+// 16 KB tile into shared memory as it is and reads it transposed; the slot permutation keeps
+// those reads free of bank conflicts.  Warp 10 publishes the per-chunk completion counters for a kernel that
+// consumes o_laT beside this one: the release fence costs a few thousand cycles and must not sit
+// on the row threads' chain.
 // ==========================================================================================
 constexpr int kScanRowThreads = 256;
-constexpr int kScanThreads = 320;
+constexpr int kScanThreads = 352;
 constexpr int kScanStages = 3;
 constexpr int kScanMisc = 1024;
 constexpr int kDecaySlots = 8;                             // ring of per-chunk decay factors
@@ -518,7 +539,8 @@ template <int D> struct ScanLayout {
 struct ScanMisc {
     uint64_t full[kScanStages], empty[kScanStages], barA, barWS, barQS[2], barB, barSU, barD3[2];
     uint32_t tmem_base;
-    int abort_flag;
+    int abort_flag, wait_kcycles;   // in this order: the waits read the limit as abort_flag[1]
+    int emit_count;                 // row warps x chunks whose read-out rows have been stored
 };
 static_assert(sizeof(ScanMisc) <= kScanMisc, "misc page too small");
 
@@ -530,9 +552,13 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                    const __grid_constant__ CUtensorMap map_ph, const float *__restrict__ Ut,
                    const float *__restrict__ Gd, float scale_la,
                    const float *__restrict__ state_in, float *__restrict__ state_out,
-                   float *__restrict__ o_la, GdnTcExport ex, ScanSegments sg,
-                   const uint8_t *__restrict__ block_route, int32_t *status, int L, int H) {
+                   __half *__restrict__ o_la16, float *__restrict__ o_la32, int32_t *emit_flags,
+                   GdnTcExport ex, ScanSegments sg,
+                   const uint8_t *__restrict__ block_route, int32_t *status, int L, int H, int wait_kcycles) {
     using SL = ScanLayout<D>;
+    // A kernel launched behind this one as a programmatic dependent (the softmax branch) may start
+    // as soon as every CTA of this grid is resident; it reads o_la chunk by chunk behind emit_flags.
+    launch_dependents();
     constexpr int KB = SL::KB;
     constexpr int kHalfCols = D / 2;                       // state columns per thread
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -560,6 +586,8 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
         mbar_init(&ms.barSU, 1);
         for (int s = 0; s < 2; ++s) { mbar_init(&ms.barQS[s], 1); mbar_init(&ms.barD3[s], 1); }
         ms.abort_flag = 0;
+        ms.wait_kcycles = wait_kcycles;
+        ms.emit_count = 0;
         fence_mbar_init();
     }
     if (warp == 8) tmem_alloc(&ms.tmem_base, SL::kTmemCols);
@@ -589,9 +617,10 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 bulk_load_1d(smem + SL::oG + (c % kDecaySlots) * SL::kG,
                              Gd + ((size_t)bh * NC + c0 + c) * 128, SL::kG, &ms.full[s]);
             }
-            if (*abort_flag)
-                for (int u = max(0, c - kScanStages); u < c; ++u)
-                    mbar_wait(&ms.full[u % kScanStages], (u / kScanStages) & 1, abort_flag);
+            // No copy may be in flight when the CTA retires: the copies issued last are waited for
+            // here, with a bound of their own and whatever the abort flag says.
+            for (int u = max(0, c - kScanStages); u < c; ++u)
+                mbar_wait_drain(&ms.full[u % kScanStages], (u / kScanStages) & 1);
         }
     } else if (warp == 8) {
         if (lane == 0) {
@@ -619,8 +648,15 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 }
                 if (!mbar_wait(&ms.barB, c & 1, abort_flag)) break;
                 tc_fence_after_sync();
-                // D3 first: the commit behind the state update then also covers it, so that the
-                // operands in the WS columns are free once barSU has fired.
+                // The state update first: it is on the chain between the chunks.  The output product
+                // behind it still reads its operand from the WS columns after barSU has fired; the
+                // next writer of those columns is the next chunk's W S product, issued behind it by
+                // this thread, and MMAs of one thread execute in issue order.
+#pragma unroll
+                for (int k16 = 0; k16 < 4; ++k16)
+                    mma_ts(tmem + SL::cS, tmem + SL::cWS + (k16 >> 1) * 32 + 16 + (k16 & 1) * 8,
+                           desc_mnmajor(st + SL::oK + k16 * 2048, 8192), id_su, k16 != 0);
+                mma_commit(&ms.barSU);
                 if (emit_out) {
 #pragma unroll
                     for (int k16 = 0; k16 < 4; ++k16)
@@ -628,12 +664,32 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                                desc_kmajor(st + SL::oP + k16 * 32), id_pu, k16 != 0);
                     mma_commit(&ms.barD3[c & 1]);
                 }
-#pragma unroll
-                for (int k16 = 0; k16 < 4; ++k16)
-                    mma_ts(tmem + SL::cS, tmem + SL::cWS + (k16 >> 1) * 32 + 16 + (k16 & 1) * 8,
-                           desc_mnmajor(st + SL::oK + k16 * 2048, 8192), id_su, k16 != 0);
-                mma_commit(&ms.barSU);
                 mma_commit(&ms.empty[s]);
+            }
+        }
+    } else if (warp == 10) {
+        // Publisher: raises the per-chunk counters once all eight row warps have stored a chunk's
+        // rows.  The row warps count in shared memory (after a block-scope fence); the gpu-scope
+        // fence here then covers their stores, as in the usual "barrier, one thread fences and
+        // sets the flag" hand-over.  Several chunks are published behind one fence when it lags.
+        if (lane == 0 && emit_flags && emit_out) {
+            volatile int *cnt = &ms.emit_count;
+            const long long limit = wait_limit(abort_flag);
+            long long t0 = clock64();
+            int published = 0;
+            while (published < ncs) {
+                const int done = *cnt / kScanRowWarps;
+                if (done > published) {
+                    __threadfence();
+                    for (int c = published; c < done; ++c)
+                        red_release_add(emit_flags + (size_t)bh * NC + c0 + c, kScanRowWarps);
+                    published = done;
+                    t0 = clock64();
+                } else {
+                    if (*abort_flag) break;
+                    if (clock64() - t0 > limit) { *abort_flag = 1; break; }
+                    __nanosleep(128);
+                }
             }
         }
     } else {
@@ -643,7 +699,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const int col0 = half * kHalfCols;                // this thread's state columns (key dim)
         const int tk0 = half * 32;                        // ... and its tokens of every chunk
-        float S[kHalfCols];                               // fp32 state, already decayed to chunk entry
+        float S[kHalfCols];                               // fp32 state at the entry of the current chunk
 #pragma unroll
         for (int x = 0; x < kHalfCols; ++x)
             S[x] = !active ? 0.f
@@ -671,22 +727,42 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             if (!mbar_wait(&ms.barQS[c & 1], (c >> 1) & 1, abort_flag)) return false;
             if (!mbar_wait(&ms.barD3[c & 1], (c >> 1) & 1, abort_flag)) return false;
             tc_fence_after_sync();
-            float *dst = o_la + (((size_t)b * L + (size_t)(c0 + c) * 64 + tk0) * H + h) * D + r;
+            const size_t off = (((size_t)b * L + (size_t)(c0 + c) * 64 + tk0) * H + h) * D + r;
+            uint32_t pk[16];                               // this thread's 32 tokens of row r, fp16 pairs
 #pragma unroll
             for (int part = 0; part < 2; ++part) {        // 16 tokens at a time keeps registers low
                 uint32_t x[16], y[16];
                 tmem_ld16(tmem + SL::cQS + 64 * (c & 1) + tk0 + 16 * part + lane_base, x);
                 tmem_ld16(tmem + SL::cD3 + 64 * (c & 1) + tk0 + 16 * part + lane_base, y);
                 tmem_wait_ld();
-                if (active) {
+                float o[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        dst[(size_t)(16 * part + i) * H * D] =
-                            fmaf(scale_la * e1[tk0 + 16 * part + i], __uint_as_float(x[i]),
-                                 __uint_as_float(y[i]));
+                for (int i = 0; i < 16; ++i)
+                    o[i] = fmaf(scale_la * e1[tk0 + 16 * part + i], __uint_as_float(x[i]), __uint_as_float(y[i]));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) pk[8 * part + i] = pack_half2(o[2 * i], o[2 * i + 1]);
+                if (o_la32 && active) {                    // fp32 token-major copy (tests, backward)
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) o_la32[off + (size_t)(16 * part + i) * H * D] = o[i];
+                }
+            }
+            if (active) {
+                uint4 *dst = reinterpret_cast<uint4 *>(o_la16 + ((size_t)bh * NC + c0 + c) * D * 64);
+#pragma unroll
+                for (int x4 = 0; x4 < 4; ++x4) {
+                    const int pc = tk0 / 8 + x4;
+                    dst[pc * D + (r ^ pc)] = make_uint4(pk[4 * x4], pk[4 * x4 + 1], pk[4 * x4 + 2], pk[4 * x4 + 3]);
                 }
             }
             tc_fence_before_sync();
+            // this warp's rows of the chunk are stored: count it for the publisher
+            if (emit_flags) {
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence_block();
+                    atomicAdd(&ms.emit_count, 1);
+                }
+            }
             return true;
         };
         prefetch_u(0);
@@ -706,13 +782,15 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                 ok = mbar_wait(&ms.barSU, (c - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
+                // decay across the previous chunk and its increment in one pass over the row
+                const float gC = reinterpret_cast<const float *>(smem + SL::oG + ((c - 1) % kDecaySlots) * SL::kG)[63];
 #pragma unroll
                 for (int cb = 0; cb < kHalfCols / 32; ++cb) {
                     uint32_t ds[32];
                     tmem_ld32(tmem + SL::cS + col0 + cb * 32 + lane_base, ds);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) S[cb * 32 + x] += __uint_as_float(ds[x]);
+                    for (int x = 0; x < 32; ++x) S[cb * 32 + x] = fmaf(S[cb * 32 + x], gC, __uint_as_float(ds[x]));
                 }
                 tc_fence_before_sync();
             }
@@ -748,11 +826,6 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             } else {
 #pragma unroll
                 for (int x = 0; x < 32; ++x) u[x] = 0.f;
-            }
-            {
-                const float gC = e1[63];
-#pragma unroll
-                for (int x = 0; x < kHalfCols; ++x) S[x] *= gC;
             }
             // ---- (b) U~ = U - W S for this thread's 32 tokens ----
             ok = mbar_wait(&ms.barWS, c & 1, abort_flag);
@@ -797,6 +870,8 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             ok = mbar_wait(&ms.barSU, (ncs - 1) & 1, abort_flag);
             if (ok) {
                 tc_fence_after_sync();
+                const float gC_last =
+                    reinterpret_cast<const float *>(smem + SL::oG + ((ncs - 1) % kDecaySlots) * SL::kG)[63];
 #pragma unroll
                 for (int cb = 0; cb < kHalfCols / 32; ++cb) {
                     uint32_t ds[32];
@@ -806,7 +881,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
 #pragma unroll
                         for (int x = 0; x < 32; ++x)
                             final_state[(size_t)(col0 + cb * 32 + x) * D + r] =
-                                S[cb * 32 + x] + __uint_as_float(ds[x]);
+                                fmaf(S[cb * 32 + x], gC_last, __uint_as_float(ds[x]));
                     }
                 }
             }
@@ -911,14 +986,14 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
     dim3 grid(NC, s.B * s.H);
     gdn_prepare_tc_kernel<D><<<grid, kPrepThreads, PrepLayout<D>::kTotal, st>>>(
         mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut, (__half *)ws.Ph, ws.Gd,
-        ex, status, s.L, s.H);
+        ex, status, s.L, s.H, 4 * sm_count(), debug_wait_kcycles());
     count_launch();
     return cudaGetLastError();
 }
 
 template <int D>
 static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *state_in,
-                                float *state_out, float *o_la, const GdnTcExport &ex,
+                                float *state_out, const ScanOut &out, const GdnTcExport &ex,
                                 const ScanSegments &sg, const uint8_t *block_route, int32_t *status,
                                 Shape s, cudaStream_t st) {
     const int NC = s.L / kC;
@@ -935,8 +1010,8 @@ static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *
     if (e != cudaSuccess) return e;
     const int ctas = s.B * s.H * (sg.mode == 0 ? 1 : sg.nseg) * (sg.mode == 1 ? 2 : 1);
     kernel<<<ctas, kScanThreads, ScanLayout<D>::kTotal, st>>>(
-        mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, o_la, ex, sg, block_route, status,
-        s.L, s.H);
+        mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, (__half *)out.o_la16, out.o_la32,
+        out.emit_flags, ex, sg, block_route, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
     return cudaGetLastError();
 }
@@ -950,12 +1025,12 @@ cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, c
 }
 
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
-                               float *state_out, float *o_la, const GdnTcExport &ex,
+                               float *state_out, const ScanOut &out, const GdnTcExport &ex,
                                const ScanSegments &sg, const uint8_t *block_route, int32_t *status,
                                Shape s, cudaStream_t st) {
     if (s.d == 128)
-        return scan_tc_impl<128>(ws, scale_la, state_in, state_out, o_la, ex, sg, block_route, status, s, st);
-    return scan_tc_impl<64>(ws, scale_la, state_in, state_out, o_la, ex, sg, block_route, status, s, st);
+        return scan_tc_impl<128>(ws, scale_la, state_in, state_out, out, ex, sg, block_route, status, s, st);
+    return scan_tc_impl<64>(ws, scale_la, state_in, state_out, out, ex, sg, block_route, status, s, st);
 }
 
 }  // namespace natsl

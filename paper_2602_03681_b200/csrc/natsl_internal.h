@@ -31,11 +31,12 @@ cudaError_t launch_score_layer(const void *x, const float *w_score, float *score
                                int d_model, Shape s, cudaStream_t st);
 
 // compact.cu  (block_status: where a route that changes inside a chunk is reported, or nullptr;
-// base_in [B,H]: retained tokens already in the cache the call appends to, or nullptr for none)
+// base_in [B,H]: retained tokens already in the cache the call appends to, or nullptr for none;
+// cap: rows per head of the cache sm_len describes -- the stored length is clamped to it; 0: none)
 cudaError_t launch_route_compact(const uint8_t *route, int32_t *sm_idx, int32_t *sm_chunk_prefix,
                                  int32_t *lin_idx, int32_t *n_lin, int32_t *sm_len,
-                                 const int32_t *base_in, int32_t *block_status, int B, int L, int H,
-                                 cudaStream_t st);
+                                 const int32_t *base_in, int32_t *block_status, int cap, int B, int L,
+                                 int H, cudaStream_t st);
 cudaError_t launch_gather_kv(const void *k, const void *v, const int32_t *sm_idx,
                              const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, int32_t cap,
                              int32_t *status, Shape s, cudaStream_t st);
@@ -66,10 +67,16 @@ cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_
                                 Shape s, cudaStream_t st);
 cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const void *v16, int32_t cap,
                                       int32_t capv, const int32_t *sm_idx,
-                                      const int32_t *sm_chunk_prefix, const float *o_la,
-                                      const float *w, float scale_sm, float eps, void *out,
-                                      float *o_nla, float *lse, BlockRouting br, bool appending,
-                                      int32_t *status, Shape s, cudaStream_t st);
+                                      const int32_t *sm_chunk_prefix, const void *o_la16,
+                                      const int32_t *emit_flags, const float *w, float scale_sm,
+                                      float eps, void *out, float *o_nla, float *lse, BlockRouting br,
+                                      bool appending, int32_t *status, Shape s, cudaStream_t st);
+// (o_la16: the linear branch's read-out, o_laT [B,H,L/C,8,d,8] fp16; emit_flags: see ScanOut -- when given, the
+// kernel is launched as a programmatic dependent of the kernel before it in the stream, the scan)
+int sm_count();   // multiprocessors of the current device (cached per device)
+// Bound of the device-side waits in units of 1024 cycles, 0 = the default (about two seconds);
+// non-zero only after natsl_debug_set_wait_limit.  Every tensor-core kernel launch passes it on.
+int debug_wait_kcycles();
 
 // softmax_bwd_tc.cu -- tensor-core backward of the softmax branch (bf16 storage).  Qh is scratch
 // for the fp16 copy of q [B,H,L,d]; dO16 the fp16 branch-output gradient [B,H,L,d]; k16, v16 the
@@ -117,8 +124,19 @@ struct ScanSegments {
     int mode, nseg, ncs;       // ncs = chunks per segment
     float *incr, *trans, *start;
 };
+// Where the scan's read-out goes: o_la16 = o_laT [B,H,L/C,8,d,8] fp16 always (one transposed tile per
+// chunk: what the softmax kernel's epilogue reads), o_la32 the same in fp32 or nullptr, and emit_flags [B*H, L/C] (or nullptr): one counter
+// per chunk, zeroed by the caller, that each of the eight row warps of the scan CTA raises by one
+// (release) once its rows of the chunk are written, so that a kernel running beside the scan can
+// consume o_la chunk by chunk.
+struct ScanOut {
+    void *o_la16;
+    float *o_la32;
+    int32_t *emit_flags;
+};
+constexpr int kScanRowWarps = 8;
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,
-                               float *state_out, float *o_la, const GdnTcExport &ex,
+                               float *state_out, const ScanOut &out, const GdnTcExport &ex,
                                const ScanSegments &sg, const uint8_t *block_route, int32_t *status,
                                Shape s, cudaStream_t st);
 cudaError_t launch_scan_combine(const float *state_in, const ScanSegments &sg, Shape s, cudaStream_t st);

@@ -28,9 +28,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct MiscB {
     uint64_t barQ, full[3], empty[3], barS, barSfree, barP, barAcc;
     uint32_t tmem_base;
-    int abort_flag;
-    int pos[kRowsB];
-    float lse2[2][64], dsum[2][64];   // key side: per query of the tile in flight (double-buffered)
+    int abort_flag, wait_kcycles;   // in this order: the waits read the limit as abort_flag[1]
+    alignas(16) int pos[kRowsB];
+    alignas(16) float lse2[2][64], dsum[2][64];   // key side: per query of the tile in flight (double-buffered)
 };
 static_assert(sizeof(MiscB) <= kMiscB, "misc page too small");
 
@@ -57,7 +57,7 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
                          int cap, const int32_t *__restrict__ sm_idx,
                          const int32_t *__restrict__ sm_chunk_prefix, const float *__restrict__ lse,
                          const float *__restrict__ Dsm, float scale_sm, float *__restrict__ dq_sm,
-                         int32_t *status, int L, int H) {
+                         int32_t *status, int L, int H, int wait_kcycles) {
     using SL = QLayout<D>;
     constexpr int KB = SL::KB;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -82,6 +82,7 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
         mbar_init(&ms.barP, kRowsB);
         mbar_init(&ms.barAcc, 1);
         ms.abort_flag = 0;
+        ms.wait_kcycles = wait_kcycles;
         fence_mbar_init();
     }
     if (tid < kRowsB) {
@@ -115,9 +116,9 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
                                 bh * cap + t * 64);
                 }
             }
-            if (*abort_flag)
-                for (int u = max(0, t - SL::kStages); u < t; ++u)
-                    mbar_wait(&ms.full[u % SL::kStages], (u / SL::kStages) & 1, abort_flag);
+            for (int u = max(0, t - SL::kStages); u < t; ++u)    // no copy in flight at retirement
+                mbar_wait_drain(&ms.full[u % SL::kStages], (u / SL::kStages) & 1);
+            mbar_wait_drain(&ms.barQ, 0);
         }
     } else if (warp == 4) {
         if (lane == 0 && T > 0) {
@@ -274,7 +275,7 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                           const float *__restrict__ lse, const float *__restrict__ Dsm,
                           float scale_sm, float *__restrict__ dk_sm, float *__restrict__ dv_sm,
                           float *__restrict__ dmask,     // [B*H*cap]: sum_i p_ij (dp_ij - D_i) per key j
-                          int32_t *status, int L, int H) {
+                          int32_t *status, int L, int H, int wait_kcycles) {
     using SL = KLayout<D>;
     constexpr int KB = SL::KB;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -300,6 +301,7 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
         mbar_init(&ms.barP, kRowsB);
         mbar_init(&ms.barAcc, 1);
         ms.abort_flag = 0;
+        ms.wait_kcycles = wait_kcycles;
         fence_mbar_init();
     }
     if (warp == 4) tmem_alloc(&ms.tmem_base, SL::kTmem);
@@ -329,8 +331,8 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                                 bh * L + (qt0 + t) * 64);
                 }
             }
-            if (*abort_flag)
-                for (int u = max(0, t - 2); u < t; ++u) mbar_wait(&ms.full[u & 1], (u >> 1) & 1, abort_flag);
+            for (int u = max(0, t - 2); u < t; ++u) mbar_wait_drain(&ms.full[u & 1], (u >> 1) & 1);
+            mbar_wait_drain(&ms.barQ, 0);
         }
     } else if (warp == 4) {
         if (lane == 0) {
@@ -531,12 +533,12 @@ static cudaError_t softmax_bwd_tc_impl(const void *q, void *Qh, const void *dO16
     if (e != cudaSuccess) return e;
     dim3 gq((s.L + 127) / 128, s.B * s.H);
     softmax_bwd_dq_tc_kernel<D><<<gq, kThreadsB, QLayout<D>::kTotal, st>>>(
-        mq128, mdo128, mk64, mv64, cap, sm_idx, pre, lse, Dsm, scale_sm, dq_sm, status, s.L, s.H);
+        mq128, mdo128, mk64, mv64, cap, sm_idx, pre, lse, Dsm, scale_sm, dq_sm, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     dim3 gk((s.L + 127) / 128, s.B * s.H);
     dkv<<<gk, kThreadsB, KLayout<D>::kTotal, st_kv>>>(
-        mq64, mdo64, mk128, mv128, cap, sm_idx, pre, lse, Dsm, scale_sm, dk_sm, dv_sm, dmask, status, s.L, s.H);
+        mq64, mdo64, mk128, mv128, cap, sm_idx, pre, lse, Dsm, scale_sm, dk_sm, dv_sm, dmask, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
     return cudaGetLastError();
 }

@@ -8,11 +8,18 @@
 // written to shared memory as fp16 and P V as an fp16 MMA (V is gathered as fp16: the bf16
 // inputs convert exactly, and an 11-bit probability keeps the branch output within ~2e-3 of
 // its RMS where an 8-bit one would not).  K and V tiles arrive by TMA into two-stage rings.
-// Epilogue: the tile's rows of o_la come in by TMA (into the Q tile and the K ring, free once the
-// last Q K^T has run) while the last tile is still being processed; each thread then normalises
+// Epilogue: o_la arrives as the scan leaves it, fp16 and transposed per chunk (o_laT, one 16 KB tile
+// per chunk: [8 pieces][d][8 tokens], row r of piece p at slot r ^ p); the CTA's two tiles come in
+// by bulk copies (into the Q tile, free once the last Q K^T has run) while the last K/V tile is still
+// being processed, and each thread reads its query's column out of them (the slot permutation
+// spreads a warp's four pieces over the banks), normalises
 // its own row of both branches, combines them and writes its row of `out` into a swizzled
 // shared-memory tile that one bulk tensor store sends out, so that no global access of the
 // epilogue is issued per thread and row.
+// The kernel may run beside the scan that produces o_la (launched behind it as a programmatic
+// dependent): nothing before the epilogue needs o_la, and the epilogue's load waits, bounded, for
+// the per-chunk counters the scan raises (emit_flags); CTAs are then ordered by query tile first,
+// so that the tiles whose chunks the scan finishes first are also scheduled first.
 // Warp roles: warps 0-3 softmax/epilogue (thread r <-> query row r <-> TMEM lane r), warp 4 issues
 // the MMAs, warp 5 issues the TMA loads.
 // Block-level routing (template flag): after the retained tiles, one more tile per linear block of
@@ -51,8 +58,8 @@ template <int D> struct SmLayout {
 struct Misc {                    // lives in the last kMiscBytes of the CTA's shared memory
     uint64_t barQ, fullK[kStages], emptyK[kStages], fullV[kStages], emptyV[kStages], barS[2], barP, barO, barE;
     uint32_t tmem_base;
-    int abort_flag;
-    int pos[kBM];                // positions of the retained tokens inside the CTA's own chunks
+    int abort_flag, wait_kcycles;   // in this order: the waits read the limit as abort_flag[1]
+    alignas(16) int pos[kBM];    // positions of the retained tokens inside the CTA's own chunks
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc page too small");
 
@@ -61,16 +68,15 @@ __global__ void __launch_bounds__(kThreadsTc)
 softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                           const __grid_constant__ CUtensorMap map_k,
                           const __grid_constant__ CUtensorMap map_v,
-                          const __grid_constant__ CUtensorMap map_ola,    // o_la  [B,L,H,D] fp32, box 128 x 32
-                          const __grid_constant__ CUtensorMap map_onla,   // o_nla (same geometry), if has_onla
                           const __grid_constant__ CUtensorMap map_out,    // out [B,L,H,D] bf16, box 128 x 64, if has_out
                           const __grid_constant__ CUtensorMap map_kd,     // the layer's k, v [B,L,H,D] bf16, box
                           const __grid_constant__ CUtensorMap map_vd,     //   64 x 64: own-block tiles (block routing)
                           const uint8_t *__restrict__ block_route, int appending, int cap, int capv, const int32_t *__restrict__ sm_idx,
                           const int32_t *__restrict__ sm_chunk_prefix,
-                          const float *__restrict__ o_la, const float *__restrict__ w,
-                          float scale_sm, float eps, int has_out, int has_onla,
-                          float *__restrict__ lse, int32_t *status, int L, int H) {
+                          const __half *__restrict__ o_laT, const int32_t *emit_flags, int prefetch_ahead,
+                          const float *__restrict__ w,
+                          float scale_sm, float eps, int has_out, float *__restrict__ o_nla,
+                          float *__restrict__ lse, int32_t *status, int L, int H, int wait_kcycles) {
     using SL = SmLayout<D>;
     constexpr int KB = SL::KB;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -78,8 +84,10 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NP = (L + kBM - 1) / kBM, NC = L / kC;
-    const int p = NP - 1 - (int)blockIdx.x;           // long rows first
-    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    // grid = (B*H, NP).  Beside the scan: tiles in ascending order, all (batch, head) pairs of a tile
+    // before the next tile.  Otherwise: long rows first.
+    const int p = emit_flags ? (int)blockIdx.y : NP - 1 - (int)blockIdx.y;
+    const int bh = blockIdx.x, b = bh / H, h = bh % H;
     const int c0 = 2 * p, c1 = min(2 * p + 2, NC);
     const int32_t *pre = sm_chunk_prefix + (size_t)bh * (NC + 1);
     const int n_full = min(pre[c0], cap);             // retained tokens before the CTA's chunks
@@ -116,6 +124,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         mbar_init(&ms.barO, 1);
         mbar_init(&ms.barE, 1);
         ms.abort_flag = 0;
+        ms.wait_kcycles = wait_kcycles;
         fence_mbar_init();
     }
     if (tid < kBM) {    // sm_idx lists this call's retained tokens; when the call appends to a
@@ -135,6 +144,14 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         if (lane == 0) {
             int nk = 0, nv = 0;                 // K / V tiles requested so far
             bool ok = true;
+            {   // the Q tile of the CTA that will follow this one on its SM: towards L2 now
+                const int lin = (int)(blockIdx.y * gridDim.x + blockIdx.x) + prefetch_ahead;
+                const int by2 = lin / (int)gridDim.x, bh2 = lin % (int)gridDim.x;
+                if (prefetch_ahead > 0 && by2 < NP) {
+                    const int p2 = emit_flags ? by2 : NP - 1 - by2;
+                    for (int kb = 0; kb < KB; ++kb) tma_prefetch_4d(&map_q, kb * 64, bh2 % H, p2 * kBM, bh2 / H);
+                }
+            }
             if (T2 > 0) {                       // nothing is loaded for a tile that sees no key at all
                 prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
                 mbar_arrive_expect_tx(&ms.barQ, SL::kQBytes);
@@ -171,21 +188,29 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 // the Q tile and the K ring are free once the last Q K^T has run
                 if (ok) ok = mbar_wait(&ms.emptyK[(T2 - 1) % kStages], ((T2 - 1) / kStages) & 1, abort_flag);
             }
+            // beside the scan: the tile's chunks of o_la are complete once all row warps of the scan
+            // CTA have raised the chunk's counter
+            if (emit_flags) {
+                for (int c = c0; c < c1 && ok; ++c)
+                    ok = wait_counter_ge(emit_flags + (size_t)bh * NC + c, kScanRowWarps, abort_flag);
+                fence_proxy_async_all();
+            }
             bool e_issued = false;
-            if (ok) {                           // the epilogue's rows of o_la, D/32 boxes of 128 x 32
-                mbar_arrive_expect_tx(&ms.barE, kBM * D * 4);
-                for (int cb = 0; cb < D / 32; ++cb)
-                    tma_load_4d(smem + cb * (kBM * 128), &map_ola, &ms.barE, cb * 32, h, p * kBM, b);
+            if (ok) {                           // the o_laT tiles of the CTA's one or two chunks
+                mbar_arrive_expect_tx(&ms.barE, (c1 - c0) * D * 128);
+                for (int e = 0; e < c1 - c0; ++e)
+                    bulk_load_1d(smem + SL::oQ + e * (D * 128), o_laT + ((size_t)bh * NC + c0 + e) * D * 64,
+                                 D * 128, &ms.barE);
                 e_issued = true;
             }
-            // on an aborted run: let the copies already issued land before the CTA retires
-            if (*abort_flag) {
-                for (int u = max(0, nk - kStages); u < nk; ++u)
-                    mbar_wait(&ms.fullK[u % kStages], (u / kStages) & 1, abort_flag);
-                for (int u = max(0, nv - kStages); u < nv; ++u)
-                    mbar_wait(&ms.fullV[u % kStages], (u / kStages) & 1, abort_flag);
-                if (e_issued) mbar_wait(&ms.barE, 0, abort_flag);
-            }
+            // No copy may be in flight when the CTA retires, aborted or not: wait (with a bound of
+            // their own) for the copies issued last.
+            if (T2 > 0) mbar_wait_drain(&ms.barQ, 0);
+            for (int u = max(0, nk - kStages); u < nk; ++u)
+                mbar_wait_drain(&ms.fullK[u % kStages], (u / kStages) & 1);
+            for (int u = max(0, nv - kStages); u < nv; ++u)
+                mbar_wait_drain(&ms.fullV[u % kStages], (u / kStages) & 1);
+            if (e_issued) mbar_wait_drain(&ms.barE, 0);
         }
     } else if (warp == 4) {
         // ------------------------------ MMA issuer ------------------------------
@@ -240,16 +265,6 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         bool ok = true;
         float2 wv = make_float2(0.5f, 0.5f);             // (w_nla, w_la) of this row
         if (w && i_abs < L) wv = __ldg(reinterpret_cast<const float2 *>(w + (((size_t)b * L + i_abs) * H + h) * 2));
-        // The epilogue's rows of o_la are pulled towards L2 once the first tile is under way (at the
-        // very start they would compete with the Q / K / V loads everything else waits for).
-        auto prefetch_o_la = [&]() {
-            if (i_abs < L) {
-                const size_t tok = ((size_t)b * L + i_abs) * H + h;
-#pragma unroll
-                for (int x = 0; x < D * 4 / 128; ++x) prefetch_l2(o_la + tok * D + x * 32);
-            }
-        };
-        if (T2 <= 1) prefetch_o_la();
         // The compacted keys are in position order, so row i sees exactly the first `cnt` of them:
         // all n_full earlier ones plus those of the CTA's own chunks at positions <= i.
         int cnt = n_full;
@@ -336,7 +351,6 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&ms.barP);
-            if (t == 0 && T2 > 1) prefetch_o_la();
         }
         if (ok && T2 > 0) {
             ok = mbar_wait(&ms.barO, (T2 - 1) & 1, abort_flag);
@@ -344,10 +358,20 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         }
         if (ok) ok = mbar_wait(&ms.barE, 0, abort_flag);        // the tile's rows of o_la have landed
         if (ok) {
-            // o_la tile: box cb (columns 32 cb ..) at cb * 16 KB, row r = 128 bytes, 16-byte piece j
-            // at j ^ (r & 7).  out tile (bf16): box kb (columns 64 kb ..) at oV + kb * 16 KB.
+            // o_laT tiles (fp16): chunk e of the CTA at oQ + e * D * 128; piece p (tokens 8 p ..) of
+            // head-dimension row `row` at 16-byte slot p * D + (row ^ p).
+            // out tile (bf16): box kb (columns 64 kb ..) at oV + kb * 16 KB, row r, piece j at j ^ (r & 7).
             const float inv = l > 0.f ? 1.f / l : 0.f;       // l = 0 (no visible key): o_nla = 0
             float ssn4[4] = {0.f, 0.f, 0.f, 0.f}, ssl4[4] = {0.f, 0.f, 0.f, 0.f};
+            const int tok = r & 63, tp = tok >> 3;
+            const uint8_t *la_col = smem + SL::oQ + (r >> 6) * (D * 128) + tp * (D * 16) + (tok & 7) * 2;
+            auto la_piece = [&](int cb, int j2, float (&a)[8]) {     // o_la of this query, columns 32 cb + 8 j2 ..
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int row = 32 * cb + 8 * j2 + e;
+                    a[e] = __half2float(*reinterpret_cast<const __half *>(la_col + ((row ^ tp) << 4)));
+                }
+            };
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t ov[32];
@@ -359,18 +383,22 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     for (int e = 0; e < 32; ++e) ov[e] = 0u;
                 }
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float4 a = *reinterpret_cast<const float4 *>(smem + cb * (kBM * 128) + sw128_offset(r, j));
-                    ssl4[j & 3] = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, ssl4[j & 3]))));
-                    const float o0 = __uint_as_float(ov[4 * j]), o1 = __uint_as_float(ov[4 * j + 1]),
-                                o2 = __uint_as_float(ov[4 * j + 2]), o3 = __uint_as_float(ov[4 * j + 3]);
-                    ssn4[j & 3] = fmaf(o0, o0, fmaf(o1, o1, fmaf(o2, o2, fmaf(o3, o3, ssn4[j & 3]))));
+                for (int j2 = 0; j2 < 4; ++j2) {
+                    float a[8];
+                    la_piece(cb, j2, a);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float o = __uint_as_float(ov[8 * j2 + e]);
+                        ssl4[e & 3] = fmaf(a[e], a[e], ssl4[e & 3]);
+                        ssn4[e & 3] = fmaf(o, o, ssn4[e & 3]);
+                    }
                 }
             }
             // mean square of the normalised row = inv^2 * mean square of the accumulator row
             const float msn = inv * inv * ((ssn4[0] + ssn4[1]) + (ssn4[2] + ssn4[3])) / D;
             const float wn = wv.x * rsqrtf(msn + eps) * inv;          // applies to the raw accumulator
             const float wl = wv.y * rsqrtf(((ssl4[0] + ssl4[1]) + (ssl4[2] + ssl4[3])) / D + eps);
+            float *onla_row = o_nla && i_abs < L ? o_nla + (((size_t)b * L + i_abs) * H + h) * D : nullptr;
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t ov[32];
@@ -382,27 +410,23 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     for (int e = 0; e < 32; ++e) ov[e] = 0u;
                 }
 #pragma unroll
-                for (int j2 = 0; j2 < 4; ++j2) {            // two 16-byte fp32 pieces -> one bf16 piece
-                    float y[8];
+                for (int j2 = 0; j2 < 4; ++j2) {
+                    float a[8], y[8];
+                    la_piece(cb, j2, a);
 #pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
-                        const int j = 2 * j2 + hh;
-                        float4 *slot = reinterpret_cast<float4 *>(smem + cb * (kBM * 128) + sw128_offset(r, j));
-                        const float4 a = *slot;
-                        const float o0 = __uint_as_float(ov[4 * j]), o1 = __uint_as_float(ov[4 * j + 1]),
-                                    o2 = __uint_as_float(ov[4 * j + 2]), o3 = __uint_as_float(ov[4 * j + 3]);
-                        y[4 * hh] = fmaf(wn, o0, wl * a.x);
-                        y[4 * hh + 1] = fmaf(wn, o1, wl * a.y);
-                        y[4 * hh + 2] = fmaf(wn, o2, wl * a.z);
-                        y[4 * hh + 3] = fmaf(wn, o3, wl * a.w);
-                        // the raw branch output takes the place of the o_la piece just consumed
-                        if (has_onla) *slot = make_float4(o0 * inv, o1 * inv, o2 * inv, o3 * inv);
-                    }
+                    for (int e = 0; e < 8; ++e) y[e] = fmaf(wn, __uint_as_float(ov[8 * j2 + e]), wl * a[e]);
                     if (has_out)
                         *reinterpret_cast<uint4 *>(smem + SL::oV + (cb >> 1) * (kBM * 128) +
                                                    sw128_offset(r, (cb & 1) * 4 + j2)) =
                             make_uint4(pack_bf162(y[0], y[1]), pack_bf162(y[2], y[3]), pack_bf162(y[4], y[5]),
                                        pack_bf162(y[6], y[7]));
+                    if (onla_row) {         // the raw branch output (fp32), straight from the registers
+                        float4 *dst = reinterpret_cast<float4 *>(onla_row + cb * 32 + j2 * 8);
+                        dst[0] = make_float4(__uint_as_float(ov[8 * j2]) * inv, __uint_as_float(ov[8 * j2 + 1]) * inv,
+                                             __uint_as_float(ov[8 * j2 + 2]) * inv, __uint_as_float(ov[8 * j2 + 3]) * inv);
+                        dst[1] = make_float4(__uint_as_float(ov[8 * j2 + 4]) * inv, __uint_as_float(ov[8 * j2 + 5]) * inv,
+                                             __uint_as_float(ov[8 * j2 + 6]) * inv, __uint_as_float(ov[8 * j2 + 7]) * inv);
+                    }
                 }
             }
             if (lse && i_abs < L)
@@ -413,9 +437,6 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 if (has_out)
                     for (int kb = 0; kb < KB; ++kb)
                         tma_store_4d(&map_out, smem + SL::oV + kb * (kBM * 128), kb * 64, h, p * kBM, b);
-                if (has_onla)
-                    for (int cb = 0; cb < D / 32; ++cb)
-                        tma_store_4d(&map_onla, smem + cb * (kBM * 128), cb * 32, h, p * kBM, b);
                 tma_store_commit();
                 tma_store_wait_read();                      // shared memory may go once it has been read
             }
@@ -500,19 +521,17 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
 template <int D>
 static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *v16, int32_t cap,
                                    int32_t capv, const int32_t *sm_idx, const int32_t *pre,
-                                   const float *o_la, const float *w, float scale_sm, float eps,
-                                   void *out, float *o_nla, float *lse, BlockRouting br,
-                                   bool appending, int32_t *status, Shape s, cudaStream_t st) {
+                                   const void *o_la16, const int32_t *emit_flags, const float *w,
+                                   float scale_sm, float eps, void *out, float *o_nla, float *lse,
+                                   BlockRouting br, bool appending, int32_t *status, Shape s,
+                                   cudaStream_t st) {
     using SL = SmLayout<D>;
-    CUtensorMap mq, mk, mv, mola, monla, mout, mkd, mvd;
+    CUtensorMap mq, mk, mv, mout, mkd, mvd;
     if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, kBM) ||
         !tch::make_map_2d(&mk, k_sm, (uint64_t)s.B * s.H * cap, D, kBN) ||
-        !tch::make_map_2d(&mv, v16, (uint64_t)s.B * s.H * capv, D, kBN) ||
-        !tch::make_map_blhd_f32(&mola, o_la, s.B, s.L, s.H, D, kBM))
+        !tch::make_map_2d(&mv, v16, (uint64_t)s.B * s.H * capv, D, kBN))
         return cudaErrorInvalidValue;
-    monla = mola;                                          // placeholders when an output is not asked for
-    mout = mq;
-    if (o_nla && !tch::make_map_blhd_f32(&monla, o_nla, s.B, s.L, s.H, D, kBM)) return cudaErrorInvalidValue;
+    mout = mq;                                             // placeholder when `out` is not asked for
     if (out && !tch::make_map_blhd(&mout, out, s.B, s.L, s.H, D, kBM)) return cudaErrorInvalidValue;
     mkd = mq;
     mvd = mq;
@@ -522,25 +541,37 @@ static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *
     auto kernel = br.route ? softmax_combine_tc_kernel<D, true> : softmax_combine_tc_kernel<D, false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal);
     if (e != cudaSuccess) return e;
-    dim3 grid((s.L + kBM - 1) / kBM, s.B * s.H);
-    kernel<<<grid, kThreadsTc, SL::kTotal, st>>>(
-        mq, mk, mv, mola, monla, mout, mkd, mvd, br.route, appending ? 1 : 0, cap, capv, sm_idx, pre, o_la, w, scale_sm, eps,
-        out ? 1 : 0, o_nla ? 1 : 0, lse, status, s.L, s.H);
+    // With emit_flags the kernel is launched as a programmatic dependent of the kernel before it in
+    // the stream (the scan): it may start once all of the scan's CTAs are resident, and finds o_la
+    // through the flags.  A launch the runtime serialises instead finds every flag already raised.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(s.B * s.H, (s.L + kBM - 1) / kBM);
+    cfg.blockDim = dim3(kThreadsTc);
+    cfg.dynamicSmemBytes = SL::kTotal;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = emit_flags ? 1 : 0;
+    e = cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mout, mkd, mvd, br.route, appending ? 1 : 0,
+                           (int)cap, (int)capv, sm_idx, pre, (const __half *)o_la16, emit_flags, 2 * sm_count(), w, scale_sm, eps,
+                           out ? 1 : 0, o_nla, lse, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const void *v16, int32_t cap,
                                       int32_t capv, const int32_t *sm_idx,
-                                      const int32_t *sm_chunk_prefix, const float *o_la,
-                                      const float *w, float scale_sm, float eps, void *out,
-                                      float *o_nla, float *lse, BlockRouting br, bool appending,
-                                      int32_t *status, Shape s, cudaStream_t st) {
+                                      const int32_t *sm_chunk_prefix, const void *o_la16,
+                                      const int32_t *emit_flags, const float *w, float scale_sm,
+                                      float eps, void *out, float *o_nla, float *lse, BlockRouting br,
+                                      bool appending, int32_t *status, Shape s, cudaStream_t st) {
     if (s.d == 128)
-        return softmax_tc_impl<128>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la, w,
-                                    scale_sm, eps, out, o_nla, lse, br, appending, status, s, st);
-    return softmax_tc_impl<64>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la, w, scale_sm,
-                               eps, out, o_nla, lse, br, appending, status, s, st);
+        return softmax_tc_impl<128>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la16, emit_flags,
+                                    w, scale_sm, eps, out, o_nla, lse, br, appending, status, s, st);
+    return softmax_tc_impl<64>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la16, emit_flags, w,
+                               scale_sm, eps, out, o_nla, lse, br, appending, status, s, st);
 }
 
 template <int D>

@@ -22,6 +22,7 @@ std::mutex g_static_ws_mu;
 
 // In host code `g_static_ws` is only a handle for the runtime, not an address a kernel may use:
 // the device address has to be asked for, once per device, with that device current.
+// (The array of the CURRENT device: the caller's stream and tensors must belong to it.)
 int static_ws_address(void **ptr) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return NATSL_ERR_CUDA;
@@ -52,4 +53,13 @@ extern "C" int natsl_hybrid_fwd_static(const void *q, const void *k, const void 
     natsl_params ps = *p;
     ps.flags |= NATSL_SINGLE_STREAM;     // no library-owned stream: nothing is created by this call
     return natsl_hybrid_fwd(q, k, v, g, beta, route, out, &ps, ws, (size_t)NATSL_STATIC_WS_BYTES, stream);
+}
+
+// The status word of the built-in scratch of the current device: what natsl_device_status reads
+// from a caller's workspace.  Allocates nothing.
+extern "C" int natsl_static_status(void *stream) {
+    void *ws = nullptr;
+    const int rc = static_ws_address(&ws);
+    if (rc != NATSL_OK) return rc;
+    return natsl_device_status(ws, stream);
 }

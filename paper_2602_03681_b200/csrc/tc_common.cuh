@@ -48,19 +48,75 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity, ui
     return ok != 0;
 }
 
-// Every wait in the tensor-core kernels is bounded: after kWaitLimitCycles without the phase
-// completing, the waiter raises `*abort_flag` (a shared-memory word all later waits of the CTA
-// see) and returns false; the kernel then records NATSL_ERR_TIMEOUT, drains and returns.
+// Every wait in the tensor-core kernels is bounded: after the limit without the phase completing,
+// the waiter raises `*abort_flag` (a shared-memory word all later waits of the CTA see) and returns
+// false; the kernel then records NATSL_ERR_TIMEOUT, drains and returns.  The word after the flag
+// (abort_flag[1]) holds the limit in units of 1024 cycles, 0 meaning the default of about two
+// seconds; kernels get it as a launch parameter, which only natsl_debug_set_wait_limit makes
+// non-zero.
 constexpr long long kWaitLimitCycles = 4000000000LL;   // ~2 s at 1.9 GHz
+constexpr long long kDrainLimitCycles = 200000000LL;   // ~0.1 s: copies in flight land in microseconds
+
+__device__ __forceinline__ long long wait_limit(volatile int *abort_flag) {
+    const int k = abort_flag[1];
+    return k > 0 ? (long long)k << 10 : kWaitLimitCycles;
+}
 
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity,
                                           volatile int *abort_flag) {
     if (mbar_try_wait(bar, parity, 20000u)) return true;
-    const long long t0 = clock64();
+    const long long t0 = clock64(), limit = wait_limit(abort_flag);
     while (true) {
         if (mbar_try_wait(bar, parity, 20000u)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > limit) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+// After an abort: wait for a copy that has already been issued to land, whatever the abort flag
+// says, with a bound of its own, so that no copy is in flight when the CTA retires.
+__device__ __forceinline__ bool mbar_wait_drain(uint64_t *bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity, 20000u))
+        if (clock64() - t0 > kDrainLimitCycles) return false;
+    return true;
+}
+
+// ------------------------------------------------------------------------------------------
+// Hand-over of global data between kernels that run side by side
+// ------------------------------------------------------------------------------------------
+// Programmatic dependent launch: a kernel launched behind this one with the programmatic
+// stream-serialisation attribute may be scheduled once every CTA of this grid has executed this
+// (or exited).  Without such a dependent it does nothing.
+__device__ __forceinline__ void launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+// Producer: the calling thread's earlier global writes (and those of threads it has synchronised
+// with) become visible to whoever reads the counter with acquire semantics.
+__device__ __forceinline__ void red_release_add(int32_t *p, int32_t v) {
+    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int32_t ld_acquire(const int32_t *p) {
+    int32_t v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Global data made visible through an acquire is about to be read by the async proxy (TMA).
+__device__ __forceinline__ void fence_proxy_async_all() {
+    asm volatile("fence.proxy.async;" ::: "memory");
+}
+// Consumer: bounded like mbar_wait (same abort flag, same limit); polls with a short sleep.
+__device__ __forceinline__ bool wait_counter_ge(const int32_t *p, int32_t target,
+                                                volatile int *abort_flag) {
+    if (ld_acquire(p) >= target) return true;
+    const long long t0 = clock64(), limit = wait_limit(abort_flag);
+    while (true) {
+        __nanosleep(256);
+        if (ld_acquire(p) >= target) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
@@ -96,6 +152,13 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *m, uin
 }
 // Pull the line holding `p` into L2.  Unlike a load it has no destination register, so nothing
 // later in the thread can end up waiting on it.
+// The same for a whole tile of a tensor map: no destination, no barrier, nothing to wait for.
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *m, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(
+                     reinterpret_cast<uint64_t>(m)),
+                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+}
 __device__ __forceinline__ void prefetch_l2(const void *p) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<uint64_t>(p)) : "memory");
 }

@@ -2,6 +2,7 @@
 // encoder is looked up through the runtime (no link-time dependency on libcuda).
 #include <mutex>
 
+#include "natsl_internal.h"
 #include "tc_common.cuh"
 
 namespace natsl {
@@ -70,4 +71,17 @@ bool make_map_blhd_f32(CUtensorMap *m, const void *base, int B, int L, int H, in
 }
 
 }  // namespace tch
+
+int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 }  // namespace natsl

@@ -28,6 +28,7 @@ def main():
     ap.add_argument("--iters", type=int, default=2)
     ap.add_argument("--flags", type=int, default=0)
     ap.add_argument("--report", action="store_true", help="print CUDA-event time of each call")
+    ap.add_argument("--stream", action="store_true", help="run on a stream of its own, not the default stream")
     args = ap.parse_args()
     if args.workload is None:
         args.workload = {"fwd": "cfg1_bf16_prefill", "bwd": "cfg4_bf16_train",
@@ -40,6 +41,8 @@ def main():
     code = binding.NATSL_F32 if wl.dtype == "f32" else binding.NATSL_BF16
     torch.cuda.set_device(0)
     binding.lib()
+    if args.stream:
+        torch.cuda.set_stream(torch.cuda.Stream())
 
     def dev(a, t=None):
         x = torch.from_numpy(a).cuda()

@@ -81,7 +81,7 @@ def test_fwd_bwd_full_size_training_workload_block_routing():
 def test_decode_full_size_sampled_sequences():
     from paper_2602_03681_b200 import binding
     wl = inputs.WORKLOADS["cfg3_bf16_decode"]
-    steps = 12
+    steps = wl.L                       # all 256 steps of the workload; 4 of its 64 sequences checked
     x = inputs.make_decode_inputs(wl, steps=steps)
     B, H, d = wl.B, wl.H, wl.d
     dt = torch.bfloat16

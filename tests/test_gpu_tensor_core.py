@@ -102,6 +102,51 @@ def test_fwd_tensor_core_cache_too_small_is_reported():
     torch.cuda.synchronize()
     assert binding.natsl_device_status(res["ws"]) == binding.ERR_CACHE_FULL
     assert torch.isfinite(res["out"].float()).all()
+    assert int(res["sm_len"].max()) <= 64         # the stored length never exceeds the cache's rows
+
+
+def test_decode_after_an_overflowed_prefill_stays_inside_the_cache():
+    """A prefill whose cache was too small reports it and leaves sm_len = sm_cap; a decode step that
+    follows (queued before the host could look at the status) reads only the cache's own rows, and
+    a stored length beyond the capacity is clamped and reported, not followed."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    B, H, L, cap = 1, 2, 256, 64
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L, route=np.ones((B, L, H), np.uint8))
+    dt = torch.bfloat16
+    res = binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]),
+                             dev(x["beta"]), dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la,
+                             scale_sm=wl.scale_sm, want=("cache", "state_out"), sm_cap=cap)
+    p = binding.make_params(B, H, 0, wl.d, binding.NATSL_BF16, wl.scale_la, wl.scale_sm)
+    dws = binding.alloc_workspace(p, binding.OP_DECODE)
+    tok = inputs.make_layer_inputs(wl, B=B, H=H, L=64)
+    q1, k1, v1 = (dev(tok[m][:, 0], dt) for m in ("q", "k", "v"))
+    g1, b1 = dev(tok["g"][:, 0]), dev(tok["beta"][:, 0])
+    r0 = torch.zeros((B, H), dtype=torch.uint8, device="cuda")          # linear token: no append
+    out = torch.empty((B, H, wl.d), dtype=dt, device="cuda")
+    state = res["state_out"].clone()
+    binding.natsl_decode_step(q1, k1, v1, g1, b1, r0, state, res["k_sm"], res["v_sm"], res["sm_len"],
+                              out, p, dws)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(res["ws"]) == binding.ERR_CACHE_FULL   # the prefill's report
+    assert binding.natsl_device_status(dws) == 0                              # the step itself is clean
+    assert res["sm_len"].cpu().tolist() == [[cap, cap]]
+    assert torch.isfinite(out.float()).all()
+    # the same step checked against the oracle's decode on the cache the prefill left
+    import oracle
+    ref = oracle.decode_step(tok["q"][:, 0], tok["k"][:, 0], tok["v"][:, 0], tok["g"][:, 0],
+                             tok["beta"][:, 0], np.zeros((B, H), np.uint8), None,
+                             res["state_out"].cpu().numpy().astype(np.float64),
+                             res["k_sm"].float().cpu().numpy().astype(np.float64),
+                             res["v_sm"].float().cpu().numpy().astype(np.float64),
+                             np.full((B, H), cap, np.int32), scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+    check_stored(out.float().cpu().numpy(), ref["out"], TOL["bf16"], "bf16")
+    # a length the caller corrupted: clamped to the capacity and reported
+    bad = torch.full((B, H), cap + 1000, dtype=torch.int32, device="cuda")
+    binding.natsl_decode_step(q1, k1, v1, g1, b1, r0, state, res["k_sm"], res["v_sm"], bad, out, p, dws)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(dws) == binding.ERR_CACHE_FULL
+    assert torch.isfinite(out.float()).all()
 
 
 @pytest.mark.parametrize("g_value", [0.0, -3.0])
