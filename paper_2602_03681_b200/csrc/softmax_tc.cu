@@ -365,13 +365,9 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             float ssn4[4] = {0.f, 0.f, 0.f, 0.f}, ssl4[4] = {0.f, 0.f, 0.f, 0.f};
             const int tok = r & 63, tp = tok >> 3;
             const uint8_t *la_col = smem + SL::oQ + (r >> 6) * (D * 128) + tp * (D * 16) + (tok & 7) * 2;
-            auto la_piece = [&](int cb, int j2, float (&a)[8]) {     // o_la of this query, columns 32 cb + 8 j2 ..
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int row = 32 * cb + 8 * j2 + e;
-                    a[e] = __half2float(*reinterpret_cast<const __half *>(la_col + ((row ^ tp) << 4)));
-                }
-            };
+            // This query's column of o_la is read once, kept as fp16 pairs (D / 2 registers: the logits of
+            // the main loop are dead by now) and used twice: for its mean square and for the output.
+            uint32_t la2[D / 2];
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t ov[32];
@@ -383,15 +379,16 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     for (int e = 0; e < 32; ++e) ov[e] = 0u;
                 }
 #pragma unroll
-                for (int j2 = 0; j2 < 4; ++j2) {
-                    float a[8];
-                    la_piece(cb, j2, a);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float o = __uint_as_float(ov[8 * j2 + e]);
-                        ssl4[e & 3] = fmaf(a[e], a[e], ssl4[e & 3]);
-                        ssn4[e & 3] = fmaf(o, o, ssn4[e & 3]);
-                    }
+                for (int e = 0; e < 32; e += 2) {
+                    const int row = 32 * cb + e;
+                    const __half a0 = *reinterpret_cast<const __half *>(la_col + ((row ^ tp) << 4));
+                    const __half a1 = *reinterpret_cast<const __half *>(la_col + (((row + 1) ^ tp) << 4));
+                    const __half2 ap = __halves2half2(a0, a1);
+                    la2[(32 * cb + e) / 2] = *reinterpret_cast<const uint32_t *>(&ap);
+                    const float2 af = __half22float2(ap);
+                    ssl4[(e >> 1) & 3] = fmaf(af.x, af.x, fmaf(af.y, af.y, ssl4[(e >> 1) & 3]));
+                    const float o0 = __uint_as_float(ov[e]), o1 = __uint_as_float(ov[e + 1]);
+                    ssn4[(e >> 1) & 3] = fmaf(o0, o0, fmaf(o1, o1, ssn4[(e >> 1) & 3]));
                 }
             }
             // mean square of the normalised row = inv^2 * mean square of the accumulator row
@@ -411,10 +408,13 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 }
 #pragma unroll
                 for (int j2 = 0; j2 < 4; ++j2) {
-                    float a[8], y[8];
-                    la_piece(cb, j2, a);
+                    float y[8];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) y[e] = fmaf(wn, __uint_as_float(ov[8 * j2 + e]), wl * a[e]);
+                    for (int e = 0; e < 8; e += 2) {
+                        const float2 af = __half22float2(*reinterpret_cast<const __half2 *>(&la2[(32 * cb + 8 * j2 + e) / 2]));
+                        y[e] = fmaf(wn, __uint_as_float(ov[8 * j2 + e]), wl * af.x);
+                        y[e + 1] = fmaf(wn, __uint_as_float(ov[8 * j2 + e + 1]), wl * af.y);
+                    }
                     if (has_out)
                         *reinterpret_cast<uint4 *>(smem + SL::oV + (cb >> 1) * (kBM * 128) +
                                                    sw128_offset(r, (cb & 1) * 4 + j2)) =
