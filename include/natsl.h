@@ -107,7 +107,7 @@ enum {
                                     two hidden states kept during generation are the linear state
                                     and the KV cache).  natsl_workspace_size depends on the flag
                                     and on p->sm_cap.  Backward: NATSL_ERR_UNSUPPORTED */
-    NATSL_SINGLE_STREAM = 1u << 4      /* forward and backward, tensor-core path: launch everything on
+    NATSL_SINGLE_STREAM = 1u << 4,     /* forward and backward, tensor-core path: launch everything on
                                     the caller's stream.  By default stages that do not depend on
                                     each other (route compaction + gather beside the linear branch's
                                     prepare kernel; in the backward also the reverse scan beside the
@@ -115,7 +115,21 @@ enum {
                                     stream the library creates once per device, forked from and
                                     joined to the caller's stream with events, so the call is still
                                     ordered like any other work on that stream.  Also implied by
-                                    p->stage_events.  natsl_hybrid_fwd_static always sets it */
+                                    p->stage_events.  natsl_hybrid_fwd_static always sets it.  The
+                                    forward then also runs its kernels strictly one after the other
+                                    (by default the softmax branch starts while the scan of the linear
+                                    branch is still running and picks its read-out up chunk by chunk) */
+    NATSL_SAVE_FOR_BWD = 1u << 5,      /* forward of a training step: `ws` is a BACKWARD workspace
+                                    (natsl_workspace_size(p, NATSL_OP_BWD) bytes).  The forward runs in
+                                    it and leaves there what the backward needs (chunk-entry states,
+                                    the chunkwise operands, log-sum-exp, the raw branch outputs), so
+                                    that natsl_hybrid_bwd with NATSL_SAVED_FWD on the same inputs, the
+                                    same p and the same ws starts at the gradients.  Produces `out`
+                                    and p->state_out; the other optional outputs, NATSL_APPEND_CACHE
+                                    and p->stage_events are NATSL_ERR_UNSUPPORTED with it */
+    NATSL_SAVED_FWD = 1u << 6          /* backward: `ws` holds such a forward (same inputs, same p apart
+                                    from this flag).  One backward per saved forward: the backward
+                                    reuses some of the saved buffers for its own results */
 };
 
 typedef struct natsl_params {
@@ -138,6 +152,8 @@ typedef struct natsl_params {
     void *const *stage_events; /* host array of cudaEvent_t owned by the caller, or NULL: the    */
     int32_t n_stage_events;    /*   library records event[i] on `stream` before stage i and one  */
                                /*   after the last stage (see natsl_stage_name); for profiling.  */
+    const float *dstate_out; /* backward, optional: gradient w.r.t. state_out [B,H,d,d] fp32; NULL => 0 */
+    float *dstate_in;       /* backward, optional: receives the gradient w.r.t. state_in [B,H,d,d]    */
     float *dscore;          /* backward with NATSL_BLOCK_ROUTING, optional: gradients of the score    */
                             /*   layer's two masks per block [B,L/C,H,2] fp32 = (linear, softmax), */
                             /*   Section 4.2: for a softmax block the sum over its keys j and all  */
@@ -228,10 +244,15 @@ int natsl_static_status(void *stream);
 /*
  * Backward of natsl_hybrid_fwd's `out` (Section 4.2 states the properties: the softmax-branch
  * logit gradient is p (dp - <do,o>), and k, v gradients of an operation vanish for tokens
- * inactive for it).  Self-contained: recomputes what it needs from the inputs.
+ * inactive for it).  Self-contained: recomputes what it needs from the inputs, unless the forward
+ * was run with NATSL_SAVE_FOR_BWD in the same workspace (then pass NATSL_SAVED_FWD).
  *   dout [B,L,H,d] in p->dtype; dq,dk,dv [B,L,H,d] in p->dtype;
  *   dg,dbeta [B,L,H] fp32; dw [B,L,H,2] fp32 or NULL.
- * p->state_in must be NULL (zero initial state).  Errors as forward.
+ * The linear state is carried across calls (Section 3, chunkwise recurrence): with p->state_in the
+ * sequence continues an earlier piece; p->dstate_out is the gradient arriving at this piece's
+ * final state from the pieces after it, p->dstate_in receives the gradient for the piece before
+ * (both optional).  The retained K/V of earlier pieces are not part of this call: their gradients
+ * belong to the calls that produced them.  Errors as forward.
  */
 int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g,
                      const float *beta, const uint8_t *route, const void *dout,

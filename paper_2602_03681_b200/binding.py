@@ -21,6 +21,8 @@ SINGLE_PASS_SCAN = 2
 BLOCK_ROUTING = 4
 APPEND_CACHE = 8
 SINGLE_STREAM = 16
+SAVE_FOR_BWD = 32
+SAVED_FWD = 64
 ERR_CACHE_FULL = -7
 ERR_UNSUPPORTED = -8
 ERR_ROUTE = -11
@@ -50,7 +52,8 @@ class natsl_params(ctypes.Structure):
                 ("o_nla", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("k_sm", ctypes.c_void_p),
                 ("v_sm", ctypes.c_void_p), ("sm_len", ctypes.c_void_p),
                 ("sm_cap", ctypes.c_int32), ("stage_events", ctypes.c_void_p),
-                ("n_stage_events", ctypes.c_int32), ("dscore", ctypes.c_void_p)]
+                ("n_stage_events", ctypes.c_int32), ("dstate_out", ctypes.c_void_p),
+                ("dstate_in", ctypes.c_void_p), ("dscore", ctypes.c_void_p)]
 
 
 _lib = None
@@ -258,15 +261,23 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5,
 
 
 def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5, ws=None, flags=0,
-               want_dscore=False):
-    """Allocate gradients and run natsl_hybrid_bwd.  Returns dict(dq, dk, dv, dg, dbeta, dw, ws)."""
+               want_dscore=False, state_in=None, dstate_out=None, want_dstate_in=False):
+    """Allocate gradients and run natsl_hybrid_bwd.  Returns dict(dq, dk, dv, dg, dbeta, dw, ws)
+    (+ dscore, dstate_in when asked for)."""
     B, L, H, d = q.shape
     dev = q.device
     dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
     dg = torch.empty((B, L, H), dtype=torch.float32, device=dev)
     dbeta = torch.empty((B, L, H), dtype=torch.float32, device=dev)
     dw = torch.empty((B, L, H, 2), dtype=torch.float32, device=dev)
-    p = make_params(B, H, L, d, _dtype_code(q), scale_la, scale_sm, eps, w=w, flags=flags)
+    p = make_params(B, H, L, d, _dtype_code(q), scale_la, scale_sm, eps, w=w, flags=flags,
+                    state_in=state_in)
+    dstate_in = None
+    if dstate_out is not None:
+        p.dstate_out = dstate_out.data_ptr()
+    if want_dstate_in:
+        dstate_in = torch.empty((B, H, d, d), dtype=torch.float32, device=dev)
+        p.dstate_in = dstate_in.data_ptr()
     dscore = None
     if want_dscore:
         dscore = torch.empty((B, L // 64, H, 2), dtype=torch.float32, device=dev)
@@ -277,4 +288,6 @@ def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, scale_la, scale_sm, eps=1e-5
     res = dict(dq=dq, dk=dk, dv=dv, dg=dg, dbeta=dbeta, dw=dw, ws=ws)
     if dscore is not None:
         res["dscore"] = dscore
+    if dstate_in is not None:
+        res["dstate_in"] = dstate_in
     return res

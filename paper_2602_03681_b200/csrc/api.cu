@@ -263,6 +263,77 @@ SideStream *side_stream_locked() {   // g_side_mu held; nullptr: run everything 
 
 }  // namespace
 
+// The forward as the backward needs it: the same kernels as natsl_hybrid_fwd's, which here also leave
+// the chunkwise quantities the gradient kernels read (chunk-entry states, U~, (I + A)^-1, cumulative
+// decays, log-sum-exp, raw branch outputs) in the backward workspace `f`.  natsl_hybrid_bwd runs it
+// itself unless the caller did, through natsl_hybrid_fwd with NATSL_SAVE_FOR_BWD (then `out` and
+// `state_out` are produced as well).
+static int bwd_forward_part(const void *q, const void *k, const void *v, const float *g,
+                            const float *beta, const uint8_t *route, void *out, float *state_out,
+                            const natsl_params *p, const BwdWs &f, cudaStream_t st) {
+    const Shape s = shape_of(p);
+    Shape s32 = s;              // the same shapes with fp32 storage (the fp32 copies)
+    s32.bf16 = false;
+    const long long B = p->B, H = p->H, L = p->L, d = p->d;
+    const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
+    const uint8_t *block_route = block ? route : nullptr;
+    const bool tensor_cores = use_tensor_cores(p);
+    const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
+#define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
+    NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
+    // compaction + gather beside the prepare kernel, on the library's side stream (as in the forward)
+    std::unique_lock<std::mutex> side_lock;
+    SideStream *side = nullptr;
+    SideJoin side_join;
+    if (fused_chunks && !(p->flags & NATSL_SINGLE_STREAM)) {
+        side_lock = std::unique_lock<std::mutex>(g_side_mu);
+        side = side_stream_locked();
+        if (!side) side_lock.unlock();
+    }
+    cudaStream_t st0 = side ? side->st : st;
+    if (side) {
+        NATSL_TRY(cudaEventRecord(side->fork, st));
+        NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
+        side_join.forked(side, st);
+    }
+    NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, nullptr,
+                                   block ? f.status : nullptr, p->L, p->B, p->L, p->H, st0));
+    if (!fused_chunks)
+        NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
+    if (tensor_cores)
+        NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, f.k_smb, nullptr, f.v16, f.k16, p->L,
+                                      p->L, false, f.status, s, st0));
+    else
+        NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
+                                   f.status, s32, st));
+    if (tensor_cores) {
+        // the fused chunk kernel reads W^T, U^T as the forward keeps them: no fp32 copies for it
+        const GdnTcExport ex{fused_chunks ? nullptr : f.W, fused_chunks ? nullptr : f.U, nullptr, f.Tinv,
+                             f.Gcum, f.S_c, f.Ut};
+        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc, ex,
+                                        f.status, s, st));
+        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, state_out, ScanOut{f.o_la16, f.o_la, nullptr},
+                                     ex, ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, block_route,
+                                     f.status, s, st));
+    } else {
+        NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
+                                          f.P, f.Abar, f.Gcum, s32, st));
+        NATSL_TRY(launch_gdn_scan_simt(f.q32, f.k32, g, f.W, f.U, f.P, p->scale_la, p->state_in, state_out,
+                                       f.S_c, f.Ut, f.o_la, nullptr, s32, st));
+    }
+    NATSL_TRY(side_join.join());
+    if (tensor_cores)
+        NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la16,
+                                            nullptr, p->w, p->scale_sm, p->eps, out, f.o_nla, f.lse,
+                                            BlockRouting{block_route, k, v}, false, f.status, s, st));
+    else
+        NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
+                                              f.o_la, p->w, p->scale_sm, p->eps, out, f.o_nla,
+                                              f.lse, BlockRouting{nullptr, nullptr, nullptr}, s32, st));
+#undef NATSL_TRY
+    return NATSL_OK;
+}
+
 extern "C" {
 
 uint64_t natsl_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
@@ -351,9 +422,18 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     const bool append = (p->flags & NATSL_APPEND_CACHE) != 0;
     if (append && !tensor_cores) return NATSL_ERR_UNSUPPORTED;
     if (append && !want_cache) return NATSL_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (p->flags & NATSL_SAVE_FOR_BWD) {
+        // The forward of a training step: run in the backward's workspace, where it leaves what
+        // natsl_hybrid_bwd (with NATSL_SAVED_FWD) would otherwise compute again.
+        if (append || want_cache || p->o_la || p->o_nla || p->lse || p->stage_events) return NATSL_ERR_UNSUPPORTED;
+        if (block && !(tensor_cores && p->d == 64)) return NATSL_ERR_UNSUPPORTED;
+        const BwdWs fb = carve_bwd(p, ws);
+        if (!ws || ws_bytes < fb.bytes) return NATSL_ERR_WORKSPACE;
+        return bwd_forward_part(q, k, v, g, beta, route, out, p->state_out, p, fb, st);
+    }
     FwdWs f = carve_fwd(p, ws);
     if (!ws || ws_bytes < f.bytes) return NATSL_ERR_WORKSPACE;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     const Shape s = shape_of(p);
     const BlockRouting br{block ? route : nullptr, k, v};
 
@@ -453,7 +533,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (rc != NATSL_OK) return rc;
     if (!q || !k || !v || !g || !beta || !route || !dout || !dq || !dk || !dv || !dg || !dbeta)
         return NATSL_ERR_NULL;
-    if (p->state_in || (p->flags & NATSL_APPEND_CACHE)) return NATSL_ERR_UNSUPPORTED;
+    if (p->flags & NATSL_APPEND_CACHE) return NATSL_ERR_UNSUPPORTED;
     // block-level routing: on the path with the fused chunk kernel only (bf16 storage, d = 64)
     const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
     if (block && !(use_tensor_cores(p) && p->d == 64)) return NATSL_ERR_UNSUPPORTED;
@@ -473,65 +553,27 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     auto CC = [&](const float *x) { return BMat{x, H * NC * kC * kC, NC * kC * kC, (long long)kC * kC, kC}; };
     auto ST = [&](const float *x) { return BMat{x, H * NC * d * d, NC * d * d, d * d, (int)d}; };
     const int di = p->d;
-
-#define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
-    NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
     const uint8_t *block_route = block ? route : nullptr;
     const bool tensor_cores = use_tensor_cores(p);
     const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
-    // Two pairs of independent stages run side by side on the library's side stream (as in the
-    // forward): compaction + gather beside the prepare kernel, and the reverse scan of the linear
-    // branch beside the softmax branch's backward.
+
+    // ---- forward, keeping what the backward needs (unless the caller's forward already did) ----
+    if (!(p->flags & NATSL_SAVED_FWD)) {
+        rc = bwd_forward_part(q, k, v, g, beta, route, nullptr, nullptr, p, f, st);
+        if (rc != NATSL_OK) return rc;
+    }
+#define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
+    // From here on two more pairs of independent stages run side by side on the library's side
+    // stream: the reverse scan of the linear branch beside the softmax branch's backward.
     std::unique_lock<std::mutex> side_lock;
     SideStream *side = nullptr;
+    SideJoin side_join;
     if (fused_chunks && !(p->flags & NATSL_SINGLE_STREAM)) {
         side_lock = std::unique_lock<std::mutex>(g_side_mu);
         side = side_stream_locked();
         if (!side) side_lock.unlock();
     }
     cudaStream_t st0 = side ? side->st : st;
-    if (side) {
-        NATSL_TRY(cudaEventRecord(side->fork, st));
-        NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
-    }
-    // ---- forward recomputation, keeping what the backward needs ----
-    NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, nullptr,
-                                   block ? f.status : nullptr, p->L, p->B, p->L, p->H, st0));
-    if (!fused_chunks)
-        NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
-    if (tensor_cores)
-        NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, f.k_smb, nullptr, f.v16, f.k16, p->L,
-                                      p->L, false, f.status, s, st0));
-    else
-        NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
-                                   f.status, s32, st));
-    if (tensor_cores) {
-        // the fused chunk kernel reads W^T, U^T as the forward keeps them: no fp32 copies for it
-        const GdnTcExport ex{fused_chunks ? nullptr : f.W, fused_chunks ? nullptr : f.U, nullptr, f.Tinv,
-                             f.Gcum, f.S_c, f.Ut};
-        NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc, ex,
-                                        f.status, s, st));
-        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, ScanOut{f.o_la16, f.o_la, nullptr},
-                                     ex, ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, block_route,
-                                     f.status, s, st));
-    } else {
-        NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
-                                          f.P, f.Abar, f.Gcum, s32, st));
-        NATSL_TRY(launch_gdn_scan_simt(f.q32, f.k32, g, f.W, f.U, f.P, p->scale_la, nullptr, nullptr,
-                                       f.S_c, f.Ut, f.o_la, nullptr, s32, st));
-    }
-    if (side) {
-        NATSL_TRY(cudaEventRecord(side->join, st0));
-        NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
-    }
-    if (tensor_cores)
-        NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la16,
-                                            nullptr, p->w, p->scale_sm, p->eps, nullptr, f.o_nla, f.lse,
-                                            BlockRouting{block_route, k, v}, false, f.status, s, st));
-    else
-        NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
-                                              f.o_la, p->w, p->scale_sm, p->eps, nullptr, f.o_nla,
-                                              f.lse, BlockRouting{nullptr, nullptr, nullptr}, s32, st));
     // ---- combination and softmax branch ----
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la,
                                  tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,
@@ -548,11 +590,13 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (side) {
         NATSL_TRY(cudaEventRecord(side->fork, st));
         NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
+        side_join.forked(side, st);
     }
     // ---- linear branch: reverse scan (then chunk-parallel products) ----
     if (tensor_cores)
         NATSL_TRY(launch_gdn_rscan_tc(f.dOla16, f.dOlag16, f.tc, f.S_c, f.dUt, f.dS_c,
-                                      fused_chunks ? nullptr : f.gS, block_route, f.status, s, st0));
+                                      fused_chunks ? nullptr : f.gS, p->dstate_out, p->dstate_in,
+                                      block_route, f.status, s, st0));
     if (side) NATSL_TRY(cudaEventRecord(side->join, st0));
     if (tensor_cores)   // (d = 64: the prepare kernel has left the fp16 copy of q in f.Qh, and the reverse
                         //  scan on the side stream reads it, so it is not written again)
@@ -565,7 +609,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                      f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
     if (!tensor_cores)
         NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
-                                   f.dS_c, f.gS, s, st));
+                                   f.dS_c, f.gS, p->dstate_out, p->dstate_in, s, st));
     if (side) NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));     // the reverse scan has finished
     AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
                    f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
@@ -579,10 +623,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gdn_finish(a, dk_x, dv_x, s32, kv_aside ? st0 : st, false));
         NATSL_TRY(launch_softmax_bwd_own_block(q, k, v, f.dO16, f.lse, f.Dsm, route, p->scale_sm,
                                                f.dq_sm, dk_x, dv_x, s, st));
-        if (kv_aside) {
-            NATSL_TRY(cudaEventRecord(side->join, st0));
-            NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
-        }
+        NATSL_TRY(side_join.join());      // the side stream's last kernels
         NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
                                        true, dk_x, dv_x, p->dscore ? f.kappa : nullptr, s, st));
@@ -596,10 +637,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                        false, nullptr, nullptr, nullptr, s, st));
         // scatter of the retained tokens' dk, dv (rows the chunk kernel does not write)
         NATSL_TRY(launch_gdn_finish(a, dk, dv, s, kv_aside ? st0 : st, false));
-        if (kv_aside) {
-            NATSL_TRY(cudaEventRecord(side->join, st0));
-            NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));
-        }
+        NATSL_TRY(side_join.join());      // the side stream's last kernels
         return NATSL_OK;
     }
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, s, st));

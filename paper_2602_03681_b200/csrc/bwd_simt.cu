@@ -387,7 +387,8 @@ gdn_rscan_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
                  const float *__restrict__ Gcum, const float *__restrict__ W,
                  const float *__restrict__ P, const float *__restrict__ do_la,
                  const float *__restrict__ chunk_states, float scale_la, float *__restrict__ dUt,
-                 float *__restrict__ dS_c, float *__restrict__ gS, int L, int H) {
+                 float *__restrict__ dS_c, float *__restrict__ gS, const float *__restrict__ dstate_out,
+                 float *__restrict__ dstate_in, int L, int H) {
     extern __shared__ float smem[];
     float *dSs = smem;                       // [D][32]
     float *Ws = dSs + D * kDvs;              // [64][D+1]
@@ -405,7 +406,8 @@ gdn_rscan_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
     const int c0 = slice * kDvs;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    for (int idx = threadIdx.x; idx < D * kDvs; idx += kThreads) dSs[idx] = 0.f;
+    for (int idx = threadIdx.x; idx < D * kDvs; idx += kThreads)     // gradient arriving at the final state
+        dSs[idx] = dstate_out ? dstate_out[((size_t)bh * D + idx / kDvs) * D + c0 + idx % kDvs] : 0.f;
 
     for (int c = NC - 1; c >= 0; --c) {
         const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
@@ -497,6 +499,10 @@ gdn_rscan_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
             __syncthreads();
 #pragma unroll
             for (int x = 0; x < kPer; ++x) dSs[a * kDvs + cs + x] = acc[x];
+            if (c == 0 && dstate_in) {      // what is left after the first chunk: the initial state's gradient
+#pragma unroll
+                for (int x = 0; x < kPer; ++x) dstate_in[((size_t)bh * D + a) * D + c0 + cs + x] = acc[x];
+            }
         }
     }
 }
@@ -769,25 +775,26 @@ cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const floa
 template <int D>
 static cudaError_t rscan_impl(const float *q32, const float *k32, const float *Gcum, const float *W,
                               const float *P, const float *do_la, const float *chunk_states,
-                              float scale_la, float *dUt, float *dS_c, float *gS, Shape s,
-                              cudaStream_t st) {
+                              float scale_la, float *dUt, float *dS_c, float *gS,
+                              const float *dstate_out, float *dstate_in, Shape s, cudaStream_t st) {
     const size_t smem = sizeof(float) * (D * kDvs + 3 * kC * (D + 1) + kC * (kC + 1) +
                                          2 * kC * (kDvs + 1) + kC + 8);
     cudaError_t e = set_smem(gdn_rscan_kernel<D>, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(D / kDvs, s.B * s.H);
     gdn_rscan_kernel<D><<<grid, kThreads, smem, st>>>(q32, k32, Gcum, W, P, do_la, chunk_states,
-                                                      scale_la, dUt, dS_c, gS, s.L, s.H);
+                                                      scale_la, dUt, dS_c, gS, dstate_out, dstate_in, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_gdn_rscan(const float *q32, const float *k32, const float *Gcum, const float *W,
                              const float *P, const float *do_la, const float *chunk_states,
-                             float scale_la, float *dUt, float *dS_c, float *gS, Shape s,
-                             cudaStream_t st) {
-    if (s.d == 128) return rscan_impl<128>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, s, st);
-    return rscan_impl<64>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, s, st);
+                             float scale_la, float *dUt, float *dS_c, float *gS,
+                             const float *dstate_out, float *dstate_in, Shape s, cudaStream_t st) {
+    if (s.d == 128)
+        return rscan_impl<128>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, dstate_out, dstate_in, s, st);
+    return rscan_impl<64>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, dstate_out, dstate_in, s, st);
 }
 
 cudaError_t launch_gdn_tsolve(const float *Abar, const float *beta, const uint8_t *route,

@@ -62,6 +62,7 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
                     const __grid_constant__ CUtensorMap map_wt,    // W^T [B*H*NC*D][64], box D
                     const __grid_constant__ CUtensorMap map_ph,    // P [B*H*NC*64][64], box 64
                     const float *__restrict__ Gd, float *__restrict__ dUt, float *__restrict__ dS_c,
+                    const float *__restrict__ dstate_out, float *__restrict__ dstate_in,
                     const uint8_t *__restrict__ block_route, int32_t *status, int L, int H, int wait_kcycles) {
     using SL = RsLayout<D>;
     constexpr int KB = SL::KB;
@@ -162,7 +163,8 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
         const int col0 = half * kHalfCols, tk0 = half * 32;
         float G[kHalfCols];                                 // dS^T row r, key columns col0..
 #pragma unroll
-        for (int x = 0; x < kHalfCols; ++x) G[x] = 0.f;
+        for (int x = 0; x < kHalfCols; ++x)     // gradient arriving at the final state, if any
+            G[x] = active && dstate_out ? dstate_out[((size_t)bh * D + col0 + x) * D + r] : 0.f;
         bool ok = true;
         for (int n = 0; n < NC && ok; ++n) {
             const int c = NC - 1 - n, s = n % kRsStages;
@@ -240,6 +242,10 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
                 for (int x = 0; x < 32; ++x) G[cb * 32 + x] += __uint_as_float(y[x]);
             }
             tc_fence_before_sync();
+        }
+        if (ok && active && dstate_in) {                    // what is left is the gradient of the initial state
+#pragma unroll
+            for (int x = 0; x < kHalfCols; ++x) dstate_in[((size_t)bh * D + col0 + x) * D + r] = G[x];
         }
     }
     tc_fence_before_sync();
@@ -809,6 +815,7 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
 template <int D>
 static cudaError_t rscan_tc_impl(const void *dO16, const void *dOg16, const GdnTcWs &ws,
                                  const float *S_c, float *dUt, float *dS_c, float *gS,
+                                 const float *dstate_out, float *dstate_in,
                                  const uint8_t *block_route, int32_t *status, Shape s, cudaStream_t st) {
     const int NC = s.L / kC;
     const uint64_t BH = (uint64_t)s.B * s.H;
@@ -822,7 +829,8 @@ static cudaError_t rscan_tc_impl(const void *dO16, const void *dOg16, const GdnT
                                          RsLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
     kernel<<<s.B * s.H, kRsThreads, RsLayout<D>::kTotal, st>>>(
-        mdo, mdog, mqh, mkh, mwt, mph, ws.Gd, dUt, dS_c, block_route, status, s.L, s.H, debug_wait_kcycles());
+        mdo, mdog, mqh, mkh, mwt, mph, ws.Gd, dUt, dS_c, dstate_out, dstate_in, block_route, status, s.L, s.H,
+        debug_wait_kcycles());
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (gS) {     // (the fused chunk kernel forms <dS1, S0> itself)
@@ -834,9 +842,11 @@ static cudaError_t rscan_tc_impl(const void *dO16, const void *dOg16, const GdnT
 
 cudaError_t launch_gdn_rscan_tc(const void *dO16, const void *dOg16, const GdnTcWs &ws,
                                 const float *S_c, float *dUt, float *dS_c, float *gS,
+                                const float *dstate_out, float *dstate_in,
                                 const uint8_t *block_route, int32_t *status, Shape s, cudaStream_t st) {
-    if (s.d == 128) return rscan_tc_impl<128>(dO16, dOg16, ws, S_c, dUt, dS_c, gS, block_route, status, s, st);
-    return rscan_tc_impl<64>(dO16, dOg16, ws, S_c, dUt, dS_c, gS, block_route, status, s, st);
+    if (s.d == 128)
+        return rscan_tc_impl<128>(dO16, dOg16, ws, S_c, dUt, dS_c, gS, dstate_out, dstate_in, block_route, status, s, st);
+    return rscan_tc_impl<64>(dO16, dOg16, ws, S_c, dUt, dS_c, gS, dstate_out, dstate_in, block_route, status, s, st);
 }
 
 

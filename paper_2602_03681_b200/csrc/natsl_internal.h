@@ -165,14 +165,17 @@ cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const floa
                                const float *do_nla, const float *lse, const float *Dsm,
                                float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm, Shape s,
                                cudaStream_t st);
+// dstate_out [B,H,d,d] (or nullptr: zero): the gradient the scan starts from, at the final state;
+// dstate_in (or nullptr): receives what is left after the first chunk, the initial state's gradient.
 cudaError_t launch_gdn_rscan(const float *q32, const float *k32, const float *Gcum, const float *W,
                              const float *P, const float *do_la, const float *chunk_states,
-                             float scale_la, float *dUt, float *dS_c, float *gS, Shape s,
-                             cudaStream_t st);
+                             float scale_la, float *dUt, float *dS_c, float *gS,
+                             const float *dstate_out, float *dstate_in, Shape s, cudaStream_t st);
 // Tensor-core reverse scan (gdn_bwd_tc.cu): dO16 / dOg16 are fp16 [B,H,L,d] copies of the read-out
 // gradient and of scale_la gamma times it; outputs as launch_gdn_rscan (gS: slot 0 of each row).
 cudaError_t launch_gdn_rscan_tc(const void *dO16, const void *dOg16, const GdnTcWs &ws,
                                 const float *S_c, float *dUt, float *dS_c, float *gS,
+                                const float *dstate_out, float *dstate_in,
                                 const uint8_t *block_route, int32_t *status, Shape s, cudaStream_t st);
 cudaError_t launch_gdn_tsolve(const float *Abar, const float *beta, const uint8_t *route,
                               const float *dW, const float *dUt, float *dKb, float *dVb, Shape s,
