@@ -495,12 +495,43 @@ def bench_other_workloads(peaks, peak_kind="measured", traffic=None):
                  "fwd_frac_of_bf16_peak": fl / (ms["fwd"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
                  "roofline": {"fwd": tensor_roofline(fl, ms["fwd"], peaks, peak_kind,
                                                      None if block else traffic.get(f"fwd:{base}"))}}
+        if "bwd" in ops:
+            # the training step as a user runs it: forward in the backward's workspace
+            # (NATSL_SAVE_FOR_BWD), then the backward from what the forward left there
+            bflags = binding.BLOCK_ROUTING if block else 0
+            pt = binding.make_params(wl.B, wl.H, wl.L, wl.d, binding.NATSL_BF16, wl.scale_la, wl.scale_sm,
+                                     w=d["w"], flags=bflags | binding.SAVE_FOR_BWD)
+            wst = binding.alloc_workspace(pt, binding.OP_BWD)
+            outt = torch.empty_like(d["q"])
+
+            def train_step():
+                binding.natsl_hybrid_fwd(d["q"], d["k"], d["v"], d["g"], d["beta"], d["route"], outt, pt, wst)
+                binding.hybrid_bwd(d["q"], d["k"], d["v"], d["g"], d["beta"], d["route"], d["w"], d["dout"],
+                                   scale_la=wl.scale_la, scale_sm=wl.scale_sm,
+                                   flags=bflags | binding.SAVED_FWD, ws=wst)
+
+            train_step()
+            torch.cuda.synchronize()
+            best = float("inf")
+            for _ in range(3):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                train_step()
+                e1.record()
+                torch.cuda.synchronize()
+                best = min(best, e0.elapsed_time(e1))
+            assert binding.natsl_device_status(wst) == 0
+            entry["ms"]["fwd_saved+bwd"] = best
+            entry["train_tokens_per_s"] = wl.B * wl.L / (best * 1e-3)
+            entry["bwd_workspace_bytes"] = int(wst.numel())
+            del wst, outt
         if "bwd" in ops and not block:
             fb = sum(useful_flops_bwd(x["route"], wl.d, wl.C).values())
             entry["useful_bwd_gflop"] = fb / 1e9
             entry["bwd_flop_formula"] = BWD_FORMULA
             entry["roofline"]["bwd"] = tensor_roofline(fb, ms["bwd"], peaks, peak_kind, traffic.get(f"bwd:{base}"))
             entry["roofline"]["fwd+bwd"] = tensor_roofline(fl + fb, total_ms, peaks, peak_kind)
+            entry["roofline"]["fwd_saved+bwd"] = tensor_roofline(fl + fb, entry["ms"]["fwd_saved+bwd"], peaks, peak_kind)
         res[name] = entry
         del d, ws
         torch.cuda.empty_cache()

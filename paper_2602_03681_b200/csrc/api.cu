@@ -548,7 +548,6 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     Shape s32 = s;              // the same shapes with fp32 storage (the fp32 copies)
     s32.bf16 = false;
     const long long B = p->B, H = p->H, L = p->L, d = p->d, NC = L / kC;
-    (void)B;
     auto TM = [&](const float *x) { return BMat{x, L * H * d, d, (long long)kC * H * d, (int)(H * d)}; };
     auto CC = [&](const float *x) { return BMat{x, H * NC * kC * kC, NC * kC * kC, (long long)kC * kC, kC}; };
     auto ST = [&](const float *x) { return BMat{x, H * NC * d * d, NC * d * d, d * d, (int)d}; };
@@ -575,10 +574,14 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     }
     cudaStream_t st0 = side ? side->st : st;
     // ---- combination and softmax branch ----
+    // Tensor cores: the fp16 gradient operands are scaled by a power of two taken from max |dout|,
+    // so that a loss-scaled or a tiny dout stays inside fp16's range (grad_scale, common.cuh).
+    if (tensor_cores) NATSL_TRY(launch_dout_amax(dout, (size_t)(B * L * H * d), s.bf16, f.status, st));
+    const int32_t *gsc = tensor_cores ? f.status : nullptr;
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la,
                                  tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,
                                  tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
-                                 tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, s, st));
+                                 tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, gsc, s, st));
     // Dependencies from here on: the query-side softmax kernel, the key-side one and the reverse
     // scan need only what is already there; the chunk kernel needs the first and the third; the
     // scatter of the retained tokens' dk, dv needs the second.  With token-level routing the chunk
@@ -622,7 +625,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         float *dk_x = f.X3, *dv_x = f.X4;
         NATSL_TRY(launch_gdn_finish(a, dk_x, dv_x, s32, kv_aside ? st0 : st, false));
         NATSL_TRY(launch_softmax_bwd_own_block(q, k, v, f.dO16, f.lse, f.Dsm, route, p->scale_sm,
-                                               f.dq_sm, dk_x, dv_x, s, st));
+                                               f.dq_sm, dk_x, dv_x, gsc, s, st));
         NATSL_TRY(side_join.join());      // the side stream's last kernels
         NATSL_TRY(launch_gdn_bwd_chunk(q, k, v, f.do_la, f.dUt, f.Ut, f.S_c, f.dS_c, f.Tinv, f.tc.Wt, f.tc.Ut,
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,

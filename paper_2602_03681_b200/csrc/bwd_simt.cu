@@ -127,6 +127,20 @@ __global__ void to_f32_kernel(const T *__restrict__ a, const T *__restrict__ b, 
 // combination backward (row-local): do_la, do_nla, dw, Dsm = <do_nla, o_nla>
 // one warp per (token, head) row
 // ------------------------------------------------------------------------------------------
+// max |dout| over the whole tensor, as the bit pattern of a non-negative float (ordered like an
+// integer), into the status page; the word is zeroed by the caller beforehand.
+template <typename T>
+__global__ void __launch_bounds__(256)
+dout_amax_kernel(const T *__restrict__ dout, size_t n4, int32_t *status) {
+    float m = 0.f;
+    for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < n4; i += (size_t)gridDim.x * 256) {
+        const float4 x = load4(dout + 4 * i);
+        m = fmaxf(fmaxf(m, fmaxf(fabsf(x.x), fabsf(x.y))), fmaxf(fabsf(x.z), fabsf(x.w)));
+    }
+    m = warp_max(m);
+    if ((threadIdx.x & 31) == 0 && m > 0.f) atomicMax(status + kGradAmaxWord, __float_as_int(m));
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_nla,
@@ -134,8 +148,9 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
                    float *__restrict__ do_la, float *__restrict__ do_nla, float *__restrict__ dw,
                    float *__restrict__ Dsm, __half *__restrict__ do16,
                    __half *__restrict__ dola16, __half *__restrict__ dolag16,
-                   const float *__restrict__ Gd, float scale_la, int B, int L, int H) {
+                   const float *__restrict__ Gd, float scale_la, const int32_t *gsc, int B, int L, int H) {
     constexpr int kCols = D / 32;
+    const float gs = grad_scale(gsc).x;      // scale of the fp16 operand copies (and of Dsm with them)
     const int lane = threadIdx.x & 31;
     const size_t row = (size_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
     if (row >= (size_t)B * L * H) return;
@@ -172,17 +187,17 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
         do_la[i] = dl;
         if (do_nla) do_nla[i] = dn;   // (the tensor-core softmax backward reads the fp16 copy only)
         const size_t i16 = ((((size_t)b * H + h) * L + l) * D) + lane + 32 * x;
-        if (do16) do16[i16] = __float2half_rn(dn);
+        if (do16) do16[i16] = __float2half_rn(gs * dn);
         if (dolag16) {
-            dola16[i16] = __float2half_rn(dl);
-            dolag16[i16] = __float2half_rn(sg * dl);
+            dola16[i16] = __float2half_rn(gs * dl);
+            dolag16[i16] = __float2half_rn(gs * sg * dl);
         }
         dsm = fmaf(dn, on[x], dsm);
     }
     dsm = warp_sum(dsm);
     if (lane == 0) {
         if (dw) { dw[row * 2] = dwn; dw[row * 2 + 1] = dwl; }
-        Dsm[((size_t)b * H + h) * L + l] = dsm;
+        Dsm[((size_t)b * H + h) * L + l] = gs * dsm;
     }
 }
 
@@ -718,11 +733,23 @@ template <typename T, int D>
 static cudaError_t combine_bwd_impl(const float *o_la, const float *o_nla, const void *dout,
                                     const float *w, float eps, float *do_la, float *do_nla,
                                     float *dw, float *Dsm, void *do16, void *dola16, void *dolag16,
-                                    const float *Gd, float scale_la, Shape s, cudaStream_t st) {
+                                    const float *Gd, float scale_la, const int32_t *gsc, Shape s,
+                                    cudaStream_t st) {
     const size_t rows = (size_t)s.B * s.L * s.H;
     combine_bwd_kernel<T, D><<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
         o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, (__half *)do16, (__half *)dola16,
-        (__half *)dolag16, Gd, scale_la, s.B, s.L, s.H);
+        (__half *)dolag16, Gd, scale_la, gsc, s.B, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dout_amax(const void *dout, size_t n, bool bf16, int32_t *status, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(status + kGradAmaxWord, 0, sizeof(int32_t), st);
+    if (e != cudaSuccess) return e;
+    const size_t n4 = n / 4;
+    const unsigned blocks = (unsigned)((n4 + 255) / 256 < 1184 ? (n4 + 255) / 256 : 1184);
+    if (bf16) dout_amax_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16 *)dout, n4, status);
+    else dout_amax_kernel<float><<<blocks, 256, 0, st>>>((const float *)dout, n4, status);
     count_launch();
     return cudaGetLastError();
 }
@@ -730,13 +757,13 @@ static cudaError_t combine_bwd_impl(const float *o_la, const float *o_nla, const
 cudaError_t launch_combine_bwd(const float *o_la, const float *o_nla, const void *dout,
                                const float *w, float eps, float *do_la, float *do_nla, float *dw,
                                float *Dsm, void *do16, void *dola16, void *dolag16, const float *Gd,
-                               float scale_la, Shape s, cudaStream_t st) {
+                               float scale_la, const int32_t *gsc, Shape s, cudaStream_t st) {
     if (s.bf16) {
-        if (s.d == 128) return combine_bwd_impl<__nv_bfloat16, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, s, st);
-        return combine_bwd_impl<__nv_bfloat16, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, s, st);
+        if (s.d == 128) return combine_bwd_impl<__nv_bfloat16, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st);
+        return combine_bwd_impl<__nv_bfloat16, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st);
     }
-    if (s.d == 128) return combine_bwd_impl<float, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, s, st);
-    return combine_bwd_impl<float, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, s, st);
+    if (s.d == 128) return combine_bwd_impl<float, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st);
+    return combine_bwd_impl<float, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st);
 }
 
 template <int D>

@@ -40,6 +40,22 @@ __device__ __forceinline__ float warp_sum(float x) {
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
     return x;
 }
+// Scale of the incoming gradient in the tensor-core backward.  The reverse scan and the softmax
+// branch's backward take the read-out gradients as fp16 operands; so that a loss-scaled or a very
+// small dout stays inside fp16's range, those operands are multiplied by a power of two s chosen
+// from max |dout| (word kGradAmaxWord of the status page holds its bit pattern) such that the
+// largest scaled |dout| lies in [4, 8) -- s = 1 for gradients of order one -- and every result
+// formed from them is multiplied by 1 / s, exactly, where it is written.  Returns (s, 1 / s).
+constexpr int kGradAmaxWord = 4;
+__device__ __forceinline__ float2 grad_scale(const int32_t *status) {
+    const int bits = status ? status[kGradAmaxWord] : 0;
+    const int e = ((bits >> 23) & 0xff) - 127;            // floor(log2 amax) of a normal number
+    if (bits <= 0 || e >= 128 || e <= -127) return make_float2(1.f, 1.f);   // zero, inf, nan, subnormal
+    int k = 2 - e;
+    k = k > 100 ? 100 : (k < -100 ? -100 : k);
+    return make_float2(__int_as_float((k + 127) << 23), __int_as_float((127 - k) << 23));
+}
+
 __device__ __forceinline__ float warp_max(float x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));

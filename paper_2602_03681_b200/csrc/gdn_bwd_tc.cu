@@ -161,10 +161,13 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
         const bool active = r < D;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const int col0 = half * kHalfCols, tk0 = half * 32;
+        // The read-out gradients arrive times the power of two gsc.x (grad_scale): the gradient
+        // state is carried in those units, and what leaves the kernel is multiplied by gsc.y = 1 / gsc.x.
+        const float2 gsc = grad_scale(status);
         float G[kHalfCols];                                 // dS^T row r, key columns col0..
 #pragma unroll
         for (int x = 0; x < kHalfCols; ++x)     // gradient arriving at the final state, if any
-            G[x] = active && dstate_out ? dstate_out[((size_t)bh * D + col0 + x) * D + r] : 0.f;
+            G[x] = active && dstate_out ? gsc.x * dstate_out[((size_t)bh * D + col0 + x) * D + r] : 0.f;
         bool ok = true;
         for (int n = 0; n < NC && ok; ++n) {
             const int c = NC - 1 - n, s = n % kRsStages;
@@ -192,7 +195,7 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
             if (active) {
                 float *dst = dS_c + (((size_t)bh * NC + c) * D + col0) * D + r;
 #pragma unroll
-                for (int x = 0; x < kHalfCols; ++x) dst[(size_t)x * D] = G[x];
+                for (int x = 0; x < kHalfCols; ++x) dst[(size_t)x * D] = gsc.y * G[x];
             }
             ok = mbar_wait(&ms.full[s], (n / kRsStages) & 1, abort_flag);   // decay factors of the chunk
             if (!ok) break;
@@ -227,7 +230,7 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
             if (active) {                                   // the fp32 copy, behind the arrival
                 float *dst = dUt + (((size_t)b * L + (size_t)c * 64 + tk0) * H + h) * D + r;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) dst[(size_t)j * H * D] = du[j];
+                for (int j = 0; j < 32; ++j) dst[(size_t)j * H * D] = gsc.y * du[j];
             }
             // ---- dS0 = gamma_C dS1 + Y ----
             ok = mbar_wait(&ms.barY, n & 1, abort_flag);
@@ -245,7 +248,7 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
         }
         if (ok && active && dstate_in) {                    // what is left is the gradient of the initial state
 #pragma unroll
-            for (int x = 0; x < kHalfCols; ++x) dstate_in[((size_t)bh * D + col0 + x) * D + r] = G[x];
+            for (int x = 0; x < kHalfCols; ++x) dstate_in[((size_t)bh * D + col0 + x) * D + r] = gsc.y * G[x];
         }
     }
     tc_fence_before_sync();
@@ -717,8 +720,9 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
                              const float *__restrict__ lse, const float *__restrict__ Dsm,
                              const uint8_t *__restrict__ route, float scale_sm,
                              float *__restrict__ dq_sm, float *__restrict__ dk_x,
-                             float *__restrict__ dv_x, int L, int H) {
+                             float *__restrict__ dv_x, const int32_t *gsc_status, int L, int H) {
     constexpr int D = 64;
+    const float ginv = grad_scale(gsc_status).y;   // do16 and Dsm arrive times the gradient scale
     extern __shared__ __align__(16) uint8_t smraw[];
     __half *sQ = reinterpret_cast<__half *>(smraw), *sK = sQ + kTileH, *sV = sK + kTileH, *sDO = sV + kTileH,
            *sP = sDO + kTileH, *sDS = sP + kTileH;
@@ -790,7 +794,7 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
         for (int nt = 0; nt < 4; ++nt) {
             float2 *pa = reinterpret_cast<float2 *>(dst + tok0 + (size_t)iA * ts + n0 + 8 * nt + 2 * t);
             float2 *pb = reinterpret_cast<float2 *>(dst + tok0 + (size_t)iB * ts + n0 + 8 * nt + 2 * t);
-            float2 va = make_float2(a[nt][0], a[nt][1]), vb = make_float2(a[nt][2], a[nt][3]);
+            float2 va = make_float2(ginv * a[nt][0], ginv * a[nt][1]), vb = make_float2(ginv * a[nt][2], ginv * a[nt][3]);
             if (add) {
                 const float2 ca = *pa, cb = *pb;
                 va.x += ca.x; va.y += ca.y; vb.x += cb.x; vb.y += cb.y;
@@ -907,7 +911,8 @@ cudaError_t launch_dscore(const uint8_t *route, const int32_t *sm_chunk_prefix, 
 cudaError_t launch_softmax_bwd_own_block(const void *q, const void *k, const void *v,
                                          const void *do16, const float *lse, const float *Dsm,
                                          const uint8_t *route, float scale_sm, float *dq_sm,
-                                         float *dk_x, float *dv_x, Shape s, cudaStream_t st) {
+                                         float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
+                                         cudaStream_t st) {
     if (s.d != 64 || !s.bf16) return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(softmax_bwd_own_block_kernel,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kOwnSmem);
@@ -915,7 +920,7 @@ cudaError_t launch_softmax_bwd_own_block(const void *q, const void *k, const voi
     dim3 grid(s.L / kC, s.B * s.H);
     softmax_bwd_own_block_kernel<<<grid, kCkThreads, kOwnSmem, st>>>(
         (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, (const __half *)do16,
-        lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, s.L, s.H);
+        lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, gsc, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }

@@ -156,10 +156,14 @@ cudaError_t launch_bgemm(bool ta, bool tb, int mask, BMat A, BMat B, BMat C, int
 cudaError_t launch_to_f32(const void *a, const void *b, const void *c, float *a32, float *b32,
                           float *c32, size_t n, bool bf16, cudaStream_t st);
 // do16: optional fp16 copy of do_nla in [B,H,L,d] layout (tensor-core softmax backward).
+// gsc: the status page holding max |dout| (see grad_scale in common.cuh), or nullptr for no scaling.
+// With it the fp16 copies and Dsm are written times the scale.
 cudaError_t launch_combine_bwd(const float *o_la, const float *o_nla, const void *dout,
                                const float *w, float eps, float *do_la, float *do_nla, float *dw,
                                float *Dsm, void *do16, void *dola16, void *dolag16, const float *Gd,
-                               float scale_la, Shape s, cudaStream_t st);
+                               float scale_la, const int32_t *gsc, Shape s, cudaStream_t st);
+// max |dout| (n elements) into word kGradAmaxWord of the status page (zeroed first)
+cudaError_t launch_dout_amax(const void *dout, size_t n, bool bf16, int32_t *status, cudaStream_t st);
 cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const float *v_sm32, int cap,
                                const int32_t *sm_idx, const int32_t *sm_chunk_prefix,
                                const float *do_nla, const float *lse, const float *Dsm,
@@ -217,7 +221,8 @@ cudaError_t launch_dscore(const uint8_t *route, const int32_t *sm_chunk_prefix, 
 cudaError_t launch_softmax_bwd_own_block(const void *q, const void *k, const void *v,
                                          const void *do16, const float *lse, const float *Dsm,
                                          const uint8_t *route, float scale_sm, float *dq_sm,
-                                         float *dk_x, float *dv_x, Shape s, cudaStream_t st);
+                                         float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
+                                         cudaStream_t st);
 
 // decode.cu
 constexpr int kDecodeParts = 4;   // CTAs that share the retained K/V of one (sequence, head)

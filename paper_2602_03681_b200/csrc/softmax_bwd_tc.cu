@@ -224,6 +224,7 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
             tc_fence_after_sync();
         }
         if (ok) {
+            const float gi = grad_scale(status).y;          // dO and Dsm arrive times the gradient scale
             float4 *dst = reinterpret_cast<float4 *>(dq_sm + (((size_t)b * L + i_abs) * H + h) * D);
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
@@ -235,8 +236,8 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
                 if (!row_ok) continue;
 #pragma unroll
                 for (int c4 = 0; c4 < 8; ++c4)
-                    dst[cb * 8 + c4] = T > 0 ? make_float4(__uint_as_float(x[4 * c4]), __uint_as_float(x[4 * c4 + 1]),
-                                                           __uint_as_float(x[4 * c4 + 2]), __uint_as_float(x[4 * c4 + 3]))
+                    dst[cb * 8 + c4] = T > 0 ? make_float4(gi * __uint_as_float(x[4 * c4]), gi * __uint_as_float(x[4 * c4 + 1]),
+                                                           gi * __uint_as_float(x[4 * c4 + 2]), gi * __uint_as_float(x[4 * c4 + 3]))
                                              : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
@@ -453,7 +454,8 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
         if (ok) {      // the TMEM loads are warp-wide: only the stores depend on the key being real
             float4 *dv_dst = reinterpret_cast<float4 *>(dv_sm + ((size_t)bh * cap + j) * D);
             float4 *dk_dst = reinterpret_cast<float4 *>(dk_sm + ((size_t)bh * cap + j) * D);
-            if (kMask && key_ok) dmask[(size_t)bh * cap + j] = msum;
+            const float gi = grad_scale(status).y;          // dO and Dsm arrive times the gradient scale
+            if (kMask && key_ok) dmask[(size_t)bh * cap + j] = gi * msum;
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t x[32], y[32];
@@ -463,10 +465,10 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                 if (!key_ok) continue;
 #pragma unroll
                 for (int c4 = 0; c4 < 8; ++c4) {
-                    dv_dst[cb * 8 + c4] = make_float4(__uint_as_float(x[4 * c4]), __uint_as_float(x[4 * c4 + 1]),
-                                                      __uint_as_float(x[4 * c4 + 2]), __uint_as_float(x[4 * c4 + 3]));
-                    dk_dst[cb * 8 + c4] = make_float4(__uint_as_float(y[4 * c4]), __uint_as_float(y[4 * c4 + 1]),
-                                                      __uint_as_float(y[4 * c4 + 2]), __uint_as_float(y[4 * c4 + 3]));
+                    dv_dst[cb * 8 + c4] = make_float4(gi * __uint_as_float(x[4 * c4]), gi * __uint_as_float(x[4 * c4 + 1]),
+                                                      gi * __uint_as_float(x[4 * c4 + 2]), gi * __uint_as_float(x[4 * c4 + 3]));
+                    dk_dst[cb * 8 + c4] = make_float4(gi * __uint_as_float(y[4 * c4]), gi * __uint_as_float(y[4 * c4 + 1]),
+                                                      gi * __uint_as_float(y[4 * c4 + 2]), gi * __uint_as_float(y[4 * c4 + 3]));
                 }
             }
         }

@@ -209,16 +209,23 @@ def test_bwd_tensor_core_softmax_branch(name, B, H, L, route):
     assert np.all(got["dbeta"][~lin] == 0)
 
 
-@pytest.mark.parametrize("scale", [2.0 ** -6, 2.0 ** 6])
-def test_bwd_tensor_core_is_linear_in_the_incoming_gradient(scale):
-    """Every gradient is linear in dout; the chunk kernel rescales its gradient tiles by a power of
-    two per chunk, which must not show in the result."""
-    wl = inputs.WORKLOADS["cfg4_bf16_train"]
-    x = inputs.make_layer_inputs(wl, B=1, H=2, L=256)
+@pytest.mark.parametrize("scale", [2.0 ** -20, 2.0 ** -6, 2.0 ** 6, 2.0 ** 20])
+@pytest.mark.parametrize("name,block", [("cfg4_bf16_train", False), ("cfg4_bf16_train", True),
+                                        ("cfg1_bf16_prefill", False)])
+def test_bwd_tensor_core_is_linear_in_the_incoming_gradient(scale, name, block):
+    """Every gradient is linear in dout.  A loss-scaled or a tiny dout must not leave the range of
+    the fp16 operands: the read-out gradients are scaled by a power of two taken from max |dout|
+    (reverse scan, softmax backward), the chunk kernel rescales its gradient tiles per chunk, and
+    neither may show in the result."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS[name]
+    B, H, L = 1, 2, 256
+    route = inputs.route_blocks(wl.seed, (B, L, H), wl.p_softmax) if block else None
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L, route=route)
     x["dout"] = (x["dout"] * scale).astype(np.float32)      # power of two: still exact in bf16
-    got = run_bwd(wl, x)
+    got = run_bwd(wl, x, flags=binding.BLOCK_ROUTING if block else 0)
     ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
-                            scale_la=wl.scale_la, scale_sm=wl.scale_sm)
+                            scale_la=wl.scale_la, scale_sm=wl.scale_sm, block=64 if block else None)
     check_bwd(wl, got, ref, TOL["bf16"])
 
 
