@@ -124,7 +124,8 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
 }
 
 struct BwdWs {
-    int32_t *status, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
+    int32_t *status, *emit_flags, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
+    size_t head_bytes;                                       // status page + emit_flags: cleared per forward
     float *k_sm32, *v_sm32;                                  // [B,H,L,d] compacted, fp32
     float *q32, *k32, *v32;                                  // token-major fp32 copies
     float *W, *U, *Ut, *o_la, *o_nla, *do_la, *do_nla;       // token-major
@@ -156,6 +157,8 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     auto tm = [&](bool need) { return c.take<float>(need ? TM : 0); };
     auto cc = [&](bool need) { return c.take<float>(need ? CC : 0); };
     f.status = c.take<int32_t>(kStatusBytes / 4);
+    f.emit_flags = c.take<int32_t>(tcs ? B * H * NC : 0);    // per-chunk counters of the scan (forward part)
+    f.head_bytes = c.off;
     f.sm_idx = c.take<int32_t>(BHL);
     f.prefix = c.take<int32_t>(B * H * (NC + 1));
     f.lin_idx = c.take<int32_t>(BHL);
@@ -279,8 +282,9 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
     const uint8_t *block_route = block ? route : nullptr;
     const bool tensor_cores = use_tensor_cores(p);
     const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
+    int32_t *flags = tensor_cores && !(p->flags & NATSL_SINGLE_STREAM) ? f.emit_flags : nullptr;
 #define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
-    NATSL_TRY(cudaMemsetAsync(f.status, 0, kStatusBytes, st));
+    NATSL_TRY(cudaMemsetAsync(f.status, 0, f.head_bytes, st));
     // compaction + gather beside the prepare kernel, on the library's side stream (as in the forward)
     std::unique_lock<std::mutex> side_lock;
     SideStream *side = nullptr;
@@ -312,7 +316,10 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
                              f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc, ex,
                                         f.status, s, st));
-        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, state_out, ScanOut{f.o_la16, f.o_la, nullptr},
+        // (the side stream joins before the scan, so that the softmax kernel follows the scan directly
+        // and can run beside it as its programmatic dependent, as in natsl_hybrid_fwd)
+        NATSL_TRY(side_join.join());
+        NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, state_out, ScanOut{f.o_la16, f.o_la, flags},
                                      ex, ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, block_route,
                                      f.status, s, st));
     } else {
@@ -324,7 +331,7 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
     NATSL_TRY(side_join.join());
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la16,
-                                            nullptr, p->w, p->scale_sm, p->eps, out, f.o_nla, f.lse,
+                                            flags, p->w, p->scale_sm, p->eps, out, f.o_nla, f.lse,
                                             BlockRouting{block_route, k, v}, false, f.status, s, st));
     else
         NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,

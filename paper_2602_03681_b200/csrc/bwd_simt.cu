@@ -133,7 +133,17 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 dout_amax_kernel(const T *__restrict__ dout, size_t n4, int32_t *status) {
     float m = 0.f;
-    for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < n4; i += (size_t)gridDim.x * 256) {
+    const size_t stride = (size_t)gridDim.x * 256;
+    size_t i = (size_t)blockIdx.x * 256 + threadIdx.x;
+    for (; i + 3 * stride < n4; i += 4 * stride) {          // four loads in flight per thread
+        float4 x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) x[u] = load4(dout + 4 * (i + u * stride));
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            m = fmaxf(fmaxf(m, fmaxf(fabsf(x[u].x), fabsf(x[u].y))), fmaxf(fabsf(x[u].z), fabsf(x[u].w)));
+    }
+    for (; i < n4; i += stride) {
         const float4 x = load4(dout + 4 * i);
         m = fmaxf(fmaxf(m, fmaxf(fabsf(x.x), fabsf(x.y))), fmaxf(fabsf(x.z), fabsf(x.w)));
     }

@@ -20,7 +20,8 @@ from . import binding, inputs
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", choices=["fwd", "bwd", "decode", "score"], default="fwd")
+    ap.add_argument("--op", choices=["fwd", "bwd", "train", "decode", "score"], default="fwd",
+                    help="train: forward with NATSL_SAVE_FOR_BWD, then the backward from what it saved")
     ap.add_argument("--workload", default=None, choices=sorted(inputs.WORKLOADS),
                     help="default: the workload that belongs to --op")
     ap.add_argument("--B", type=int, default=None, help="batch override (smaller case)")
@@ -31,7 +32,7 @@ def main():
     ap.add_argument("--stream", action="store_true", help="run on a stream of its own, not the default stream")
     args = ap.parse_args()
     if args.workload is None:
-        args.workload = {"fwd": "cfg1_bf16_prefill", "bwd": "cfg4_bf16_train",
+        args.workload = {"fwd": "cfg1_bf16_prefill", "bwd": "cfg4_bf16_train", "train": "cfg4_bf16_train",
                          "decode": "cfg3_bf16_decode", "score": "cfg1_bf16_prefill"}[args.op]
     if (inputs.WORKLOADS[args.workload].call == "decode") != (args.op == "decode"):
         ap.error(f"workload {args.workload} does not belong to --op {args.op}")
@@ -98,7 +99,7 @@ def main():
         kw["B"] = args.B
     if args.L:
         kw["L"] = args.L
-    if args.op in ("fwd", "bwd") and args.flags & binding.BLOCK_ROUTING:   # one route per block of 64 tokens
+    if args.op in ("fwd", "bwd", "train") and args.flags & binding.BLOCK_ROUTING:   # one route per block of 64 tokens
         kw["route"] = inputs.route_blocks(wl.seed, (kw.get("B", wl.B), kw.get("L", wl.L), wl.H),
                                           wl.p_softmax)
     x = inputs.make_layer_inputs(wl, **kw)
@@ -111,6 +112,19 @@ def main():
                 nonlocal ws
                 ws = binding.hybrid_fwd(q, k, v, g, beta, route, w, scale_la=wl.scale_la,
                                         scale_sm=wl.scale_sm, flags=args.flags, ws=ws)["ws"]
+            timed(call)
+    elif args.op == "train":
+        dout = dev(x["dout"], dt)
+        B, L, H, d = q.shape
+        p = binding.make_params(B, H, L, d, code, wl.scale_la, wl.scale_sm, w=w,
+                                flags=args.flags | binding.SAVE_FOR_BWD)
+        ws = binding.alloc_workspace(p, binding.OP_BWD)
+        out = torch.empty_like(q)
+        for _ in range(args.iters):
+            def call():
+                binding.natsl_hybrid_fwd(q, k, v, g, beta, route, out, p, ws)
+                binding.hybrid_bwd(q, k, v, g, beta, route, w, dout, scale_la=wl.scale_la,
+                                   scale_sm=wl.scale_sm, flags=args.flags | binding.SAVED_FWD, ws=ws)
             timed(call)
     else:
         dout = dev(x["dout"], dt)
