@@ -86,18 +86,16 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                       const float *__restrict__ beta, const uint8_t *__restrict__ route,
                       float scale_la, __half *__restrict__ Wt, float *__restrict__ Ut,
                       __half *__restrict__ Ph, float *__restrict__ Gd, GdnTcExport ex,
-                      int32_t *status, int L, int H, int prefetch_ahead, int wait_kcycles) {
+                      int32_t *status, int L, int H, int wait_kcycles) {
     using PL = PrepLayout<D>;
     constexpr int KB = PL::KB;
     extern __shared__ __align__(1024) uint8_t smem[];
     PrepMisc &ms = *reinterpret_cast<PrepMisc *>(smem + PL::oMisc);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NC = L / kC;
-    // CTA order: head fastest, then chunk, then batch.  The H CTAs that run side by side then read
-    // the H heads of the same 64 tokens, i.e. whole contiguous rows of [B,L,H,d] (and of g, beta,
-    // route), instead of 128-byte pieces 64 tokens apart.
-    const int h = (int)(blockIdx.x % H), c = (int)((blockIdx.x / H) % NC), b = (int)(blockIdx.x / (H * NC));
-    const int bh = b * H + h;
+    // (chunk fastest: a head-fastest order, whole rows of [B,L,H,d] read by neighbouring CTAs, and L2
+    // prefetches of the next wave's tiles were both measured slower)
+    const int c = (int)(blockIdx.x % NC), bh = (int)(blockIdx.x / NC), b = bh / H, h = bh % H;
     const int tok0 = c * kC;
     const size_t chunk = (size_t)bh * NC + c;
 
@@ -135,17 +133,6 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 tma_load_4d(sQK + kb * 16384 + 8192, &map_k, &ms.barLoad, kb * 64, h, tok0, b);
                 tma_load_4d(sQK + kb * 16384, &map_q, &ms.barLoad, kb * 64, h, tok0, b);
                 tma_load_4d(sV + kb * 8192, &map_v, &ms.barLoad, kb * 64, h, tok0, b);
-            }
-            {   // the tiles of the CTA that will follow this one on its SM: towards L2 now, so that its
-                // wait for the first bytes is an L2 round trip, not a DRAM one behind a full wave's loads
-                const unsigned lin = blockIdx.x + prefetch_ahead;
-                const int h2 = (int)(lin % H), c2 = (int)((lin / H) % NC), b2 = (int)(lin / (H * NC));
-                if (prefetch_ahead > 0 && lin < gridDim.x)
-                    for (int kb = 0; kb < KB; ++kb) {
-                        tma_prefetch_4d(&map_k, kb * 64, h2, c2 * kC, b2);
-                        tma_prefetch_4d(&map_q, kb * 64, h2, c2 * kC, b2);
-                        tma_prefetch_4d(&map_v, kb * 64, h2, c2 * kC, b2);
-                    }
             }
             bool ok = mbar_wait(&ms.barConv, 0, abort_flag);       // tiles converted to fp16
             if (ok) {
@@ -206,17 +193,6 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             const size_t t = ((size_t)b * L + tok0 + i) * H + h;
             float G = g[t];
             const float btv = route && route[t] ? 0.f : beta[t];   // route == nullptr: beta~ = beta
-            {   // the same three values of the CTA that will follow this one on its SM: towards L2 now
-                // (under load these scattered 4-byte loads are the longest wait of a chunk)
-                const unsigned lin = blockIdx.x + prefetch_ahead;
-                const int h2 = (int)(lin % H), c2 = (int)((lin / H) % NC), b2 = (int)(lin / (H * NC));
-                if (prefetch_ahead > 0 && lin < gridDim.x) {
-                    const size_t t2 = ((size_t)b2 * L + c2 * kC + i) * H + h2;
-                    prefetch_l2(g + t2);
-                    prefetch_l2(beta + t2);
-                    if (route) prefetch_l2(route + t2);
-                }
-            }
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const float y = __shfl_up_sync(0xffffffffu, G, o);
@@ -1001,7 +977,7 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
     const unsigned grid = (unsigned)NC * s.B * s.H;
     gdn_prepare_tc_kernel<D><<<grid, kPrepThreads, PrepLayout<D>::kTotal, st>>>(
         mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut, (__half *)ws.Ph, ws.Gd,
-        ex, status, s.L, s.H, 4 * sm_count(), debug_wait_kcycles());
+        ex, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
     return cudaGetLastError();
 }

@@ -73,7 +73,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                           const __grid_constant__ CUtensorMap map_vd,     //   64 x 64: own-block tiles (block routing)
                           const uint8_t *__restrict__ block_route, int appending, int cap, int capv, const int32_t *__restrict__ sm_idx,
                           const int32_t *__restrict__ sm_chunk_prefix,
-                          const __half *__restrict__ o_laT, const int32_t *emit_flags, int prefetch_ahead,
+                          const __half *__restrict__ o_laT, const int32_t *emit_flags,
                           const float *__restrict__ w,
                           float scale_sm, float eps, int has_out, float *__restrict__ o_nla,
                           float *__restrict__ lse, int32_t *status, int L, int H, int wait_kcycles) {
@@ -144,14 +144,6 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         if (lane == 0) {
             int nk = 0, nv = 0;                 // K / V tiles requested so far
             bool ok = true;
-            {   // the Q tile of the CTA that will follow this one on its SM: towards L2 now
-                const int lin = (int)(blockIdx.y * gridDim.x + blockIdx.x) + prefetch_ahead;
-                const int by2 = lin / (int)gridDim.x, bh2 = lin % (int)gridDim.x;
-                if (prefetch_ahead > 0 && by2 < NP) {
-                    const int p2 = emit_flags ? by2 : NP - 1 - by2;
-                    for (int kb = 0; kb < KB; ++kb) tma_prefetch_4d(&map_q, kb * 64, bh2 % H, p2 * kBM, bh2 / H);
-                }
-            }
             if (T2 > 0) {                       // nothing is loaded for a tile that sees no key at all
                 prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
                 mbar_arrive_expect_tx(&ms.barQ, SL::kQBytes);
@@ -555,7 +547,7 @@ static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *
     cfg.attrs = attr;
     cfg.numAttrs = emit_flags ? 1 : 0;
     e = cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mout, mkd, mvd, br.route, appending ? 1 : 0,
-                           (int)cap, (int)capv, sm_idx, pre, (const __half *)o_la16, emit_flags, 2 * sm_count(), w, scale_sm, eps,
+                           (int)cap, (int)capv, sm_idx, pre, (const __half *)o_la16, emit_flags, w, scale_sm, eps,
                            out ? 1 : 0, o_nla, lse, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
     return e;

@@ -152,13 +152,6 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *m, uin
 }
 // Pull the line holding `p` into L2.  Unlike a load it has no destination register, so nothing
 // later in the thread can end up waiting on it.
-// The same for a whole tile of a tensor map: no destination, no barrier, nothing to wait for.
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *m, int c0, int c1, int c2, int c3) {
-    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(
-                     reinterpret_cast<uint64_t>(m)),
-                 "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-                 : "memory");
-}
 __device__ __forceinline__ void prefetch_l2(const void *p) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<uint64_t>(p)) : "memory");
 }
