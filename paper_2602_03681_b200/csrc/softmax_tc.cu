@@ -5,9 +5,12 @@
 // One CTA owns 128 consecutive queries of one (batch, head) and walks the compacted K/V of that
 // head in tiles of 64 retained tokens: logits = Q K^T as a bf16 tcgen05 MMA into TMEM (q and k
 // are exact bf16 inputs), online softmax in registers (one thread per query row), probabilities
-// written to shared memory as fp16 and P V as an fp16 MMA (V is gathered as fp16: the bf16
-// inputs convert exactly, and an 11-bit probability keeps the branch output within ~2e-3 of
-// its RMS where an 8-bit one would not).  K and V tiles arrive by TMA into two-stage rings.
+// written as fp16 into the TMEM columns their logits came from and P V as an fp16 MMA with A in
+// TMEM (V is gathered as fp16: the bf16 inputs convert exactly, and an 11-bit probability keeps the
+// branch output within ~2e-3 of its RMS where an 8-bit one would not).  The logits are
+// double-buffered in TMEM, so the probabilities of tile t + 1 never wait for the product of tile
+// t; with P in a single shared-memory tile every tile paid that product's latency.  K and V
+// tiles arrive by TMA into two-stage rings.
 // Epilogue: o_la arrives as the scan leaves it, fp16 and transposed per chunk (o_laT, one 16 KB tile
 // per chunk: [8 pieces][d][8 tokens], row r of piece p at slot r ^ p); the CTA's two tiles come in
 // by bulk copies (into the Q tile, free once the last Q K^T has run) while the last K/V tile is still
@@ -46,12 +49,10 @@ template <int D> struct SmLayout {
     static constexpr int kQBytes = KB * kBM * 128;
     static constexpr int kKStage = KB * kBN * 128;
     static constexpr int kVStage = KB * kBN * 128;
-    static constexpr int kPBytes = kBM * 128;
     static constexpr int oQ = 0;
     static constexpr int oK = oQ + kQBytes;
     static constexpr int oV = oK + kStages * kKStage;
-    static constexpr int oP = oV + kStages * kVStage;
-    static constexpr int oMisc = oP + kPBytes;
+    static constexpr int oMisc = oV + kStages * kVStage;
     static constexpr int kTotal = oMisc + kMiscBytes;
 };
 
@@ -209,7 +210,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         if (lane == 0 && T2 > 0) {
             constexpr uint32_t idesc_qk = make_idesc(kFmtBF16, kBM, kBN, false, false);
             constexpr uint32_t idesc_pv = make_idesc(kFmtF16, kBM, D, false, true);
-            const uint32_t aQ = smem_u32(smem + SL::oQ), aP = smem_u32(smem + SL::oP);
+            const uint32_t aQ = smem_u32(smem + SL::oQ);
             auto issue_qk = [&](int t) {
                 const uint32_t aK = smem_u32(smem + SL::oK + (t % kStages) * SL::kKStage);
 #pragma unroll
@@ -240,8 +241,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 tc_fence_after_sync();
                 const uint32_t aV = smem_u32(smem + SL::oV + (t % kStages) * SL::kVStage);
 #pragma unroll
-                for (int k16 = 0; k16 < 4; ++k16)
-                    mma_ss(tO, desc_kmajor(aP + k16 * 32), desc_mnmajor(aV + k16 * 2048, kBN * 128),
+                for (int k16 = 0; k16 < 4; ++k16)      // A = P(t): fp16 pairs in the first 32 columns of S(t)
+                    mma_ts(tO, tS[t & 1] + k16 * 8, desc_mnmajor(aV + k16 * 2048, kBN * 128),
                            idesc_pv, (t | k16) != 0);
                 mma_commit(&ms.emptyV[t % kStages]);
                 mma_commit(&ms.barO);
@@ -301,11 +302,16 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             }
             l = l * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
             m = m_new;
-            if (t > 0) {
+            // barO's phases are consumed strictly in order, one per tile (a parity wait cannot skip a
+            // phase): before the accumulator is touched when it has to be rescaled, otherwise at the
+            // end of the tile, when the previous tile's product has had the whole tile to finish.
+            bool waited_o = false;
+            if (t > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+                waited_o = true;
                 ok = mbar_wait(&ms.barO, (t - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after_sync();
-                if (__any_sync(0xffffffffu, corr != 1.f)) {
+                {
 #pragma unroll
                     for (int cb = 0; cb < D / 32; ++cb) {
                         uint32_t ov[32];
@@ -318,15 +324,12 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     tmem_wait_st();
                 }
             }
-            uint8_t *prow = smem + SL::oP;
+            {
+                uint32_t pk[32];                        // P(t), over the logits this thread has consumed
 #pragma unroll
-            for (int pc = 0; pc < 8; ++pc) {
-                uint4 u;
-                u.x = pack_half2(x[8 * pc + 0], x[8 * pc + 1]);
-                u.y = pack_half2(x[8 * pc + 2], x[8 * pc + 3]);
-                u.z = pack_half2(x[8 * pc + 4], x[8 * pc + 5]);
-                u.w = pack_half2(x[8 * pc + 6], x[8 * pc + 7]);
-                *reinterpret_cast<uint4 *>(prow + sw128_offset(r, pc)) = u;
+                for (int c = 0; c < 32; ++c) pk[c] = pack_half2(x[2 * c], x[2 * c + 1]);
+                tmem_st32(tS[t & 1] + lane_base, pk);
+                tmem_wait_st();
             }
             if (kBlock && t >= T) {   // own-block tile: its V rows arrived as bf16; fp16 in place (exact)
                 ok = mbar_wait(&ms.fullV[t % kStages], (t / kStages) & 1, abort_flag);
@@ -339,6 +342,12 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                     };
                     vt[i] = make_uint4(cv(a.x), cv(a.y), cv(a.z), cv(a.w));
                 }
+            }
+            // (before the arrival below, not after it: once this thread has arrived, the MMA warp may
+            // complete the next phase of barO too, and a parity wait two phases behind never returns)
+            if (t > 0 && !waited_o) {
+                ok = mbar_wait(&ms.barO, (t - 1) & 1, abort_flag);
+                if (!ok) break;
             }
             fence_proxy_async_smem();
             tc_fence_before_sync();
