@@ -137,7 +137,7 @@ typedef struct natsl_params {
     int32_t C;              /* chunk size; must be 64 (Section 5: NAtS chunk = GDN chunk = 64) */
     int32_t dtype;          /* storage type of q,k,v,out,dout,dq,dk,dv and the KV caches */
     float scale_la;         /* logit scale of the linear read-out */
-    float scale_sm;         /* logit scale of the softmax branch */
+    float scale_sm;         /* logit scale of the softmax branch; > 0 on the tensor-core path */
     float eps;              /* RMS-norm epsilon, > 0 */
     uint32_t flags;
     const float *w;         /* [B,L,H,2] (decode: [B,H,2]) = (w_nla, w_la); NULL => (0.5, 0.5) */

@@ -272,7 +272,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             tmem_wait_ld();
             float x[kBN];
 #pragma unroll
-            for (int c = 0; c < kBN; ++c) x[c] = __uint_as_float(sv[c >> 5][c & 31]) * sl2;
+            for (int c = 0; c < kBN; ++c) x[c] = __uint_as_float(sv[c >> 5][c & 31]);   // raw logits: the scale
+                                                                                        // goes into the exponent's FMA
             const int j0 = t * kBN;
             if (kBlock && t >= T) {
                 // own-block tile: row r sees keys 0 .. r % 64 if it is in that block
@@ -286,7 +287,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             float mx4[4] = {x[0], x[1], x[2], x[3]};      // four independent chains, not one of 63
 #pragma unroll
             for (int c = 4; c < kBN; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], x[c]);
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            // (scale_sm > 0, checked on the host: the maximum of the raw logits is the maximum logit)
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
             // The running maximum only has to bound the exponents, not equal the true maximum: it
             // is raised (and O rescaled) only when a logit exceeds it by more than 8 (base 2), so
             // probabilities stay below 2^8 and, for inputs whose logits vary little, the accumulator
@@ -297,7 +299,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             float ps4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < kBN; ++c) {
-                x[c] = ex2_ftz(x[c] - m_use);
+                x[c] = ex2_ftz(fmaf(x[c], sl2, -m_use));
                 ps4[c & 3] += x[c];
             }
             l = l * corr + ((ps4[0] + ps4[1]) + (ps4[2] + ps4[3]));
