@@ -127,9 +127,16 @@ enum {
                                     same p and the same ws starts at the gradients.  Produces `out`
                                     and p->state_out; the other optional outputs, NATSL_APPEND_CACHE
                                     and p->stage_events are NATSL_ERR_UNSUPPORTED with it */
-    NATSL_SAVED_FWD = 1u << 6          /* backward: `ws` holds such a forward (same inputs, same p apart
+    NATSL_SAVED_FWD = 1u << 6,         /* backward: `ws` holds such a forward (same inputs, same p apart
                                     from this flag).  One backward per saved forward: the backward
                                     reuses some of the saved buffers for its own results */
+    NATSL_QK_NORM = 1u << 7            /* forward: q and k are normalised inside the kernels, differently
+                                    for the two operations that share them (Section 4.3): L2 over the
+                                    d columns of the head for the linear operation,
+                                    x / sqrt(sum x^2 + norm_eps), and RMS per softmax head for the
+                                    softmax operation, x / sqrt(mean x^2 + norm_eps), no gain.
+                                    Without the flag q and k are used as given.  See p->G for what
+                                    is built */
 };
 
 typedef struct natsl_params {
@@ -161,6 +168,23 @@ typedef struct natsl_params {
                             /*   block <dS_next, U> with U the update the block commits to the     */
                             /*   state; zero for the operation the block did not choose.  NULL:    */
                             /*   not computed.  Without the flag: NATSL_ERR_UNSUPPORTED.           */
+    int32_t G;              /* softmax heads per linear head (Section 4.3: several softmax heads are   */
+                            /*   grouped under one linear head and share its route); 0 or 1: none.     */
+                            /*   The paper does not say how one q, k, v serves two head counts; here   */
+                            /*   the G softmax heads of head h are the G slices of d / G columns of    */
+                            /*   q, k, v [B,L,H,d]: softmax head (h, s) attends with columns           */
+                            /*   [s d/G, (s+1) d/G) over the retained tokens of route[:,:,h] and fills */
+                            /*   those columns of the softmax output, which is RMS-normalised per      */
+                            /*   slice; the linear operation, its state and the two weights stay per   */
+                            /*   head h over all d columns.  p->lse becomes [B,H,G,L].                 */
+                            /*   Built: natsl_hybrid_fwd with token-level routing, for fp32 storage    */
+                            /*   (d / G in {32, 64, 128}) and on the tensor-core path for d = 128,     */
+                            /*   G = 2 (the appendix's two softmax heads per linear head; three would  */
+                            /*   need d = 192).  G > 1 or NATSL_QK_NORM with anything else (backward,  */
+                            /*   decode, NATSL_BLOCK_ROUTING, NATSL_APPEND_CACHE, NATSL_SAVE_FOR_BWD,  */
+                            /*   NATSL_FORCE_SIMT on bf16, NATSL_QK_NORM with p->k_sm):                */
+                            /*   NATSL_ERR_UNSUPPORTED.                                                */
+    float norm_eps;         /* NATSL_QK_NORM: epsilon under the square roots, >= 0                     */
 } natsl_params;
 
 /* Bytes of workspace `op` needs for these shapes (host call, launches nothing). */

@@ -23,6 +23,7 @@ APPEND_CACHE = 8
 SINGLE_STREAM = 16
 SAVE_FOR_BWD = 32
 SAVED_FWD = 64
+QK_NORM = 128
 ERR_CACHE_FULL = -7
 ERR_UNSUPPORTED = -8
 ERR_ROUTE = -11
@@ -53,7 +54,8 @@ class natsl_params(ctypes.Structure):
                 ("v_sm", ctypes.c_void_p), ("sm_len", ctypes.c_void_p),
                 ("sm_cap", ctypes.c_int32), ("stage_events", ctypes.c_void_p),
                 ("n_stage_events", ctypes.c_int32), ("dstate_out", ctypes.c_void_p),
-                ("dstate_in", ctypes.c_void_p), ("dscore", ctypes.c_void_p)]
+                ("dstate_in", ctypes.c_void_p), ("dscore", ctypes.c_void_p),
+                ("G", ctypes.c_int32), ("norm_eps", ctypes.c_float)]
 
 
 _lib = None
@@ -136,8 +138,9 @@ def _dtype_code(t) -> int:
 
 def make_params(B, H, L, d, dtype_code, scale_la, scale_sm, eps=1e-5, C=64, flags=0, w=None,
                 state_in=None, state_out=None, o_la=None, o_nla=None, lse=None, k_sm=None,
-                v_sm=None, sm_len=None, sm_cap=0) -> natsl_params:
+                v_sm=None, sm_len=None, sm_cap=0, G=0, norm_eps=0.0) -> natsl_params:
     p = natsl_params()
+    p.G, p.norm_eps = G, norm_eps
     p.B, p.H, p.L, p.d, p.C, p.dtype = B, H, L, d, C, dtype_code
     p.scale_la, p.scale_sm, p.eps, p.flags = scale_la, scale_sm, eps, flags
     for name, t in dict(w=w, state_in=state_in, state_out=state_out, o_la=o_la, o_nla=o_nla,
@@ -226,10 +229,11 @@ def natsl_debug_set_wait_limit(kcycles: int, withhold_scan_flags: bool = False):
 # Convenience wrappers (allocation + marshalling; no arithmetic).
 # ---------------------------------------------------------------------------------------------
 def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5, state_in=None,
-               want=(), flags=0, sm_cap=0, ws=None, cache=None):
+               want=(), flags=0, sm_cap=0, ws=None, cache=None, G=0, norm_eps=0.0):
     """Allocate outputs and run natsl_hybrid_fwd.  `want` may name optional outputs:
     "o_la", "o_nla", "lse", "state_out", "cache" (compacted K/V with capacity sm_cap or L).
-    cache=(k_sm, v_sm, sm_len): use these existing cache tensors (with APPEND_CACHE: in and out)."""
+    cache=(k_sm, v_sm, sm_len): use these existing cache tensors (with APPEND_CACHE: in and out).
+    G: softmax heads per linear head (lse is then [B,H,G,L]); norm_eps goes with the QK_NORM flag."""
     B, L, H, d = q.shape
     dev = q.device
     out = torch.empty_like(q)
@@ -239,7 +243,7 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5,
     if "o_nla" in want:
         opt["o_nla"] = torch.empty((B, L, H, d), dtype=torch.float32, device=dev)
     if "lse" in want:
-        opt["lse"] = torch.empty((B, H, L), dtype=torch.float32, device=dev)
+        opt["lse"] = torch.empty((B, H, G, L) if G > 1 else (B, H, L), dtype=torch.float32, device=dev)
     if "state_out" in want:
         opt["state_out"] = torch.empty((B, H, d, d), dtype=torch.float32, device=dev)
     cap = 0
@@ -252,7 +256,7 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, scale_la, scale_sm, eps=1e-5,
         opt["v_sm"] = torch.zeros((B, H, cap, d), dtype=q.dtype, device=dev)
         opt["sm_len"] = torch.zeros((B, H), dtype=torch.int32, device=dev)
     p = make_params(B, H, L, d, _dtype_code(q), scale_la, scale_sm, eps, flags=flags, w=w,
-                    state_in=state_in, sm_cap=cap, **opt)
+                    state_in=state_in, sm_cap=cap, G=G, norm_eps=norm_eps, **opt)
     if ws is None:
         ws = alloc_workspace(p, OP_FWD, dev)
     natsl_hybrid_fwd(q, k, v, g, beta, route, out, p, ws)

@@ -46,7 +46,18 @@ int check_params(const natsl_params *p, bool needs_L) {
     if (p->C != kC) return NATSL_ERR_SHAPE;
     if (needs_L && (p->L <= 0 || p->L % p->C != 0)) return NATSL_ERR_SHAPE;
     if (!(p->eps > 0.f)) return NATSL_ERR_SHAPE;
+    if (p->G < 0 || (p->G > 1 && p->d % p->G != 0)) return NATSL_ERR_SHAPE;
+    if ((p->flags & NATSL_QK_NORM) && !(p->norm_eps >= 0.f)) return NATSL_ERR_SHAPE;
     return NATSL_OK;
+}
+
+// Grouped softmax heads / per-operation q, k normalisation (Section 4.3): what the forward supports.
+bool grouped_or_normed(const natsl_params *p) { return p->G > 1 || (p->flags & NATSL_QK_NORM); }
+HeadGroups head_groups(const natsl_params *p) {
+    HeadGroups hg;
+    hg.G = p->G > 1 ? p->G : 1;
+    hg.norm_eps = (p->flags & NATSL_QK_NORM) ? p->norm_eps : -1.f;
+    return hg;
 }
 
 Shape shape_of(const natsl_params *p) { return Shape{p->B, p->H, p->L, p->d, p->dtype == NATSL_BF16}; }
@@ -57,6 +68,7 @@ struct FwdWs {
     void *k_sm, *v_sm, *v16;
     void *o_la16;               // tensor-core path: the linear read-out as fp16 [B,L,H,d]
     float *W, *U, *P, *o_la;    // fp32 CUDA-core path only
+    float *q_la, *k_la, *q_sm, *k_nsm;   // fp32 storage with NATSL_QK_NORM: normalised copies of q and k
     GdnTcWs tc;                 // tensor-core path only
     float *seg_incr, *seg_trans, *seg_start;   // segmented scan: [B*H, nseg, d, d] each
     size_t bytes;
@@ -121,6 +133,11 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
         f.P = c.take<float>(B * H * NC * kC * kC);
         f.o_la = c.take<float>(B * L * H * d);
     }
+    const size_t nrm = !use_tensor_cores(p) && (p->flags & NATSL_QK_NORM) ? B * L * H * d : 0;
+    f.q_la = c.take<float>(nrm);
+    f.k_la = c.take<float>(nrm);
+    f.q_sm = c.take<float>(nrm);
+    f.k_nsm = c.take<float>(nrm);
     f.bytes = c.off;
     return f;
 }
@@ -432,6 +449,17 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     const bool append = (p->flags & NATSL_APPEND_CACHE) != 0;
     if (append && !tensor_cores) return NATSL_ERR_UNSUPPORTED;
     if (append && !want_cache) return NATSL_ERR_NULL;
+    const HeadGroups hg = head_groups(p);
+    if (grouped_or_normed(p)) {
+        if (block || append || (p->flags & NATSL_SAVE_FOR_BWD)) return NATSL_ERR_UNSUPPORTED;
+        if ((p->flags & NATSL_QK_NORM) && want_cache) return NATSL_ERR_UNSUPPORTED;   // (the cache would hold normalised keys)
+        if (tensor_cores) {
+            if (hg.G > 1 && !(hg.G == 2 && p->d == 128)) return NATSL_ERR_UNSUPPORTED;
+        } else {
+            if (p->dtype != NATSL_F32) return NATSL_ERR_UNSUPPORTED;
+            if (hg.G > 1 && (hg.G > 4 || p->d / hg.G < 32)) return NATSL_ERR_UNSUPPORTED;
+        }
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (p->flags & NATSL_SAVE_FOR_BWD) {
         // The forward of a training step: run in the backward's workspace, where it leaves what
@@ -479,11 +507,18 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, sm_len,
                                    append ? sm_len : nullptr, block ? f.status : nullptr, cap, p->B,
                                    p->L, p->H, st0));
+    // fp32 storage with NATSL_QK_NORM: normalised copies first (the tensor-core kernels normalise inside)
+    const void *q_la = q, *k_la = k, *q_sm = q, *k_nsm = k;
+    if (!tensor_cores && hg.norm_eps >= 0.f) {
+        NATSL_TRY(launch_qk_norm_f32((const float *)q, (const float *)k, f.q_la, f.k_la, f.q_sm, f.k_nsm,
+                                     (size_t)p->B * p->L * p->H, p->d, hg.G, hg.norm_eps, st));
+        q_la = f.q_la; k_la = f.k_la; q_sm = f.q_sm; k_nsm = f.k_nsm;
+    }
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
-                                      f.v16, nullptr, cap, capv, append, f.status, s, st0));
+                                      f.v16, nullptr, cap, capv, append, f.status, s, st0, hg));
     else
-        NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
+        NATSL_TRY(launch_gather_kv(k_nsm, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
     NATSL_TRY(mark());
     if (tensor_cores) {
         // block-level routing: every token takes part in the delta rule of its own block
@@ -503,8 +538,8 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
             if (n_late < 4 || NCi - n_late < 4) n_late = 0;
         }
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc,
-                                        GdnTcExport{}, f.status, PrepRange{0, NCi - n_late, nullptr, false},
-                                        s, st));
+                                        GdnTcExport{}, f.status,
+                                        PrepRange{0, NCi - n_late, nullptr, false, hg.norm_eps}, s, st));
         NATSL_TRY(mark());
         // The side stream joins here, before the scan, so that nothing stands between the scan and
         // the softmax kernel in the stream: the softmax kernel is launched as a programmatic dependent
@@ -532,22 +567,23 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
             if (n_late)
                 NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc,
                                                 GdnTcExport{}, f.status,
-                                                PrepRange{NCi - n_late, n_late, f.ready_flags, true}, s, st));
+                                                PrepRange{NCi - n_late, n_late, f.ready_flags, true, hg.norm_eps},
+                                                s, st));
         }
         NATSL_TRY(mark());
         NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, capv, f.sm_idx, f.prefix, f.o_la16,
                                             flags_softmax, p->w, p->scale_sm, p->eps, out, p->o_nla,
-                                            p->lse, br, append, f.status, s, st));
+                                            p->lse, br, append, f.status, s, st, hg));
     } else {
         float *o_la = p->o_la ? p->o_la : f.o_la;
-        NATSL_TRY(launch_gdn_prepare_simt(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.W,
+        NATSL_TRY(launch_gdn_prepare_simt(q_la, k_la, v, g, beta, block ? nullptr : route, p->scale_la, f.W,
                                           f.U, f.P, nullptr, nullptr, s, st));
         NATSL_TRY(mark());
-        NATSL_TRY(launch_gdn_scan_simt(q, k, g, f.W, f.U, f.P, p->scale_la, p->state_in,
+        NATSL_TRY(launch_gdn_scan_simt(q_la, k_la, g, f.W, f.U, f.P, p->scale_la, p->state_in,
                                        p->state_out, nullptr, nullptr, o_la, br.route, s, st));
         NATSL_TRY(mark());
-        NATSL_TRY(launch_softmax_combine_simt(q, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
-                                              p->scale_sm, p->eps, out, p->o_nla, p->lse, br, s, st));
+        NATSL_TRY(launch_softmax_combine_simt(q_sm, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
+                                              p->scale_sm, p->eps, out, p->o_nla, p->lse, br, s, st, hg.G));
     }
     NATSL_TRY(mark());
 #undef NATSL_TRY
@@ -563,6 +599,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (!q || !k || !v || !g || !beta || !route || !dout || !dq || !dk || !dv || !dg || !dbeta)
         return NATSL_ERR_NULL;
     if (p->flags & NATSL_APPEND_CACHE) return NATSL_ERR_UNSUPPORTED;
+    if (grouped_or_normed(p)) return NATSL_ERR_UNSUPPORTED;   // grouped heads, q/k normalisation: forward only
     if (use_tensor_cores(p) && !(p->scale_sm > 0.f)) return NATSL_ERR_SHAPE;
     // block-level routing: on the path with the fused chunk kernel only (bf16 storage, d = 64)
     const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
@@ -705,6 +742,7 @@ int natsl_decode_step(const void *q, const void *k, const void *v, const float *
         !out)
         return NATSL_ERR_NULL;
     if (cache_cap <= 0) return NATSL_ERR_SHAPE;
+    if (grouped_or_normed(p)) return NATSL_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(state) ||
         !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
         return NATSL_ERR_ALIGN;

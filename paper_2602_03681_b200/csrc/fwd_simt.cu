@@ -267,10 +267,14 @@ gdn_scan_simt_kernel(const T *__restrict__ q, const T *__restrict__ k, const flo
 
 // ------------------------------------------------------------------------------------------
 // Softmax branch over the retained tokens (Section 4.1, O_nla with mask M^nla) with the
-// combination (Section 4.3, Norm equation) as epilogue.  grid = (L/64, B*H); each warp owns
+// combination (Section 4.3, Norm equation) as epilogue.  grid = (L/64, B*H*G); each warp owns
 // 8 query rows, each lane one key of the current 32-key tile.
+// G softmax heads per linear head (Section 4.3, grouped heads): softmax head (h, sg) works on the
+// columns [sg D, (sg+1) D) of q, k, v rows of DL = G D columns; lists, weights and the linear read-out
+// are those of linear head h; the softmax output is normalised over its D columns, the linear
+// read-out over all DL, and the CTA writes its D columns of `out`.  lse is [B,H,G,L].
 // ------------------------------------------------------------------------------------------
-template <typename T, int D>
+template <typename T, int D, int G>
 __global__ void __launch_bounds__(kThreads)
 softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
                             const T *__restrict__ v_sm, int cap, const int32_t *__restrict__ sm_idx,
@@ -286,16 +290,18 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
     float *Vt = Kt + 32 * (D + 1);         // [32][D]
     int *pos = reinterpret_cast<int *>(Vt + 32 * D);  // [32]
 
-    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    constexpr int DL = D * G;
+    const int c = blockIdx.x, bhg = blockIdx.y, bh = bhg / G, sg = bhg % G, b = bh / H, h = bh % H;
     const int NC = L / kC;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const size_t ts = (size_t)H * D;
+    const size_t ts = (size_t)H * DL;
     const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
     const int n_end = min(sm_chunk_prefix[(size_t)bh * (NC + 1) + c + 1], cap);
+    const int col0 = sg * D;                             // first column of this softmax head
 
     for (int idx = threadIdx.x; idx < kC * D / 4; idx += kThreads) {
         const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
-        store4(Qs + r * D + c4, load4(q + tok0 * D + (size_t)r * ts + c4));
+        store4(Qs + r * D + c4, load4(q + tok0 * DL + (size_t)r * ts + col0 + c4));
     }
     constexpr int kQ = 8, kCols = D / 32;
     float m[kQ], z[kQ], acc[kQ][kCols];
@@ -305,7 +311,7 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
 #pragma unroll
         for (int x = 0; x < kCols; ++x) acc[r][x] = 0.f;
     }
-    const T *kb = k_sm + (size_t)bh * cap * D, *vb = v_sm + (size_t)bh * cap * D;
+    const T *kb = k_sm + (size_t)bh * cap * DL + col0, *vb = v_sm + (size_t)bh * cap * DL + col0;
 
     // Block-level routing: a query in a linear block also reads the causal part of its own block
     // (two more tiles of 32 keys, taken from the layer's own k and v).
@@ -318,12 +324,12 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
             const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
             float4 kx = make_float4(0.f, 0.f, 0.f, 0.f), vx = kx;
             if (own) {
-                const size_t src = (tok0 + (size_t)(j0 - n_ret + r) * H) * D + c4;
+                const size_t src = (tok0 + (size_t)(j0 - n_ret + r) * H) * DL + col0 + c4;
                 kx = load4(k_tok + src);
                 vx = load4(v_tok + src);
             } else if (j0 + r < n_end) {
-                kx = load4(kb + (size_t)(j0 + r) * D + c4);
-                vx = load4(vb + (size_t)(j0 + r) * D + c4);
+                kx = load4(kb + (size_t)(j0 + r) * DL + c4);
+                vx = load4(vb + (size_t)(j0 + r) * DL + c4);
             }
             float *kp = Kt + r * (D + 1) + c4;
             kp[0] = kx.x; kp[1] = kx.y; kp[2] = kx.z; kp[3] = kx.w;
@@ -370,20 +376,58 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
 #pragma unroll
         for (int x = 0; x < kCols; ++x) {
             on[x] = acc[r][x] * inv;
-            ol[x] = o_la[t * D + lane + 32 * x];
+            ol[x] = o_la[t * DL + col0 + lane + 32 * x];
             ssn = fmaf(on[x], on[x], ssn);
             ssl = fmaf(ol[x], ol[x], ssl);
         }
+        if (G > 1)        // the linear read-out is normalised over its whole row
+            for (int x = 0; x < DL / 32; ++x) {
+                if ((32 * x) / D == sg) continue;
+                const float y = o_la[t * DL + lane + 32 * x];
+                ssl = fmaf(y, y, ssl);
+            }
         ssn = warp_sum(ssn);
         ssl = warp_sum(ssl);
-        const float fn = rsqrtf(ssn / D + eps), fl = rsqrtf(ssl / D + eps);
+        const float fn = rsqrtf(ssn / D + eps), fl = rsqrtf(ssl / DL + eps);
         const float wn = w ? w[t * 2] : 0.5f, wl = w ? w[t * 2 + 1] : 0.5f;
 #pragma unroll
         for (int x = 0; x < kCols; ++x) {
-            if (out) out[t * D + lane + 32 * x] = from_f32<T>(wn * on[x] * fn + wl * ol[x] * fl);
-            if (o_nla) o_nla[t * D + lane + 32 * x] = on[x];
+            if (out) out[t * DL + col0 + lane + 32 * x] = from_f32<T>(wn * on[x] * fn + wl * ol[x] * fl);
+            if (o_nla) o_nla[t * DL + col0 + lane + 32 * x] = on[x];
         }
-        if (lse && lane == 0) lse[(size_t)bh * L + i] = z[r] > 0.f ? m[r] + __logf(z[r]) : -INFINITY;
+        if (lse && lane == 0) lse[(size_t)bhg * L + i] = z[r] > 0.f ? m[r] + __logf(z[r]) : -INFINITY;
+    }
+}
+
+// Per-operation normalisation of q and k for fp32 storage (Section 4.3): one warp per row of d
+// columns writes the L2-normalised row (linear operation) and the row with each of its G slices
+// RMS-normalised (softmax operation).  The tensor-core path does both inside its kernels instead.
+__global__ void __launch_bounds__(256)
+qk_norm_f32_kernel(const float *__restrict__ q, const float *__restrict__ k, float *__restrict__ q_la,
+                   float *__restrict__ k_la, float *__restrict__ q_sm, float *__restrict__ k_sm,
+                   size_t rows, int d, int G, float norm_eps) {
+    const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const int ds = d / G;                                // 32, 64 or 128: a multiple of the warp size
+    for (int which = 0; which < 2; ++which) {
+        const float *src = (which ? k : q) + row * d;
+        float *la = (which ? k_la : q_la) + row * d, *sm = (which ? k_sm : q_sm) + row * d;
+        float x[4], ss_all = 0.f;
+        for (int j = 0; j < d / 32; ++j) {
+            x[j] = src[lane + 32 * j];
+            ss_all = fmaf(x[j], x[j], ss_all);
+        }
+        ss_all = warp_sum(ss_all);
+        const float rl = rsqrtf(ss_all + norm_eps);
+        for (int sg = 0; sg < G; ++sg) {
+            float ss = 0.f;
+            for (int j = sg * ds / 32; j < (sg + 1) * ds / 32; ++j) ss = fmaf(x[j], x[j], ss);
+            ss = warp_sum(ss);
+            const float rs = rsqrtf(ss / ds + norm_eps);
+            for (int j = sg * ds / 32; j < (sg + 1) * ds / 32; ++j) sm[lane + 32 * j] = x[j] * rs;
+        }
+        for (int j = 0; j < d / 32; ++j) la[lane + 32 * j] = x[j] * rl;
     }
 }
 
@@ -458,16 +502,16 @@ cudaError_t launch_gdn_scan_simt(const void *q, const void *k, const float *g, c
                    block_route, s, st);
 }
 
-template <typename T, int D>
+template <typename T, int D, int G = 1>
 static cudaError_t softmax_impl(const void *q, const void *k_sm, const void *v_sm, int32_t cap,
                                 const int32_t *sm_idx, const int32_t *pre, const float *o_la,
                                 const float *w, float scale_sm, float eps, void *out, float *o_nla,
                                 float *lse, BlockRouting br, Shape s, cudaStream_t st) {
     const size_t smem = simt_softmax_smem(D);
-    cudaError_t e = set_smem(softmax_combine_simt_kernel<T, D>, smem);
+    cudaError_t e = set_smem(softmax_combine_simt_kernel<T, D, G>, smem);
     if (e != cudaSuccess) return e;
-    dim3 grid(s.L / kC, s.B * s.H);
-    softmax_combine_simt_kernel<T, D><<<grid, kThreads, smem, st>>>(
+    dim3 grid(s.L / kC, s.B * s.H * G);
+    softmax_combine_simt_kernel<T, D, G><<<grid, kThreads, smem, st>>>(
         (const T *)q, (const T *)k_sm, (const T *)v_sm, cap, sm_idx, pre, o_la, w, scale_sm, eps,
         (T *)out, o_nla, lse, br.route, (const T *)br.k, (const T *)br.v, s.L, s.H);
     count_launch();
@@ -479,9 +523,29 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
                                         const int32_t *sm_chunk_prefix, const float *o_la,
                                         const float *w, float scale_sm, float eps, void *out,
                                         float *o_nla, float *lse, BlockRouting br, Shape s,
-                                        cudaStream_t st) {
+                                        cudaStream_t st, int G) {
+    if (G > 1) {      // grouped softmax heads: fp32 storage, d / G in {32, 64}
+        if (s.bf16) return cudaErrorInvalidValue;
+#define NATSL_GROUPED(DS, GG)                                                                           \
+        if (s.d == DS * GG && G == GG)                                                                  \
+            return softmax_impl<float, DS, GG>(q, k_sm, v_sm, cap, sm_idx, sm_chunk_prefix, o_la, w,    \
+                                               scale_sm, eps, out, o_nla, lse, br, s, st)
+        NATSL_GROUPED(32, 2);
+        NATSL_GROUPED(64, 2);
+        NATSL_GROUPED(32, 4);
+#undef NATSL_GROUPED
+        return cudaErrorInvalidValue;
+    }
     NATSL_DISPATCH(softmax_impl, q, k_sm, v_sm, cap, sm_idx, sm_chunk_prefix, o_la, w, scale_sm, eps,
                    out, o_nla, lse, br, s, st);
+}
+
+cudaError_t launch_qk_norm_f32(const float *q, const float *k, float *q_la, float *k_la, float *q_sm,
+                               float *k_sm, size_t rows, int d, int G, float norm_eps, cudaStream_t st) {
+    qk_norm_f32_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(q, k, q_la, k_la, q_sm, k_sm, rows, d, G,
+                                                                  norm_eps);
+    count_launch();
+    return cudaGetLastError();
 }
 
 }  // namespace natsl

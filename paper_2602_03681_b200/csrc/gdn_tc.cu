@@ -87,7 +87,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                       float scale_la, __half *__restrict__ Wt, float *__restrict__ Ut,
                       __half *__restrict__ Ph, float *__restrict__ Gd, GdnTcExport ex,
                       int32_t *status, int L, int H, int c_begin, int n_range, int32_t *ready_flags,
-                      int wait_kcycles) {
+                      float norm_eps, int wait_kcycles) {
     using PL = PrepLayout<D>;
     // (a kernel launched behind this one as a programmatic dependent may start once every CTA of
     // this grid is resident; see the launch of the second part)
@@ -216,11 +216,50 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         }
         // ---- tiles to fp16, in place ----
         bool ok = mbar_wait(&ms.barLoad, 0, abort_flag);
-        if (ok) {
+        if (ok && norm_eps >= 0.f) {
+            // L2-normalised q and k for the linear operation (Section 4.3): thread r owns row r of
+            // [Q ; K] (all KB blocks of it), takes its 16-byte pieces in an order that spreads the warp
+            // over the banks, and scales while it converts.  V is converted as below.
+            static_assert(PL::oV == 0 && PL::oQK == KB * 8192, "V tile first, [Q ; K] blocks behind it");
+            for (int idx = r; idx < KB * 8192 / 16; idx += kRowThreads) {
+                uint4 *pp = reinterpret_cast<uint4 *>(smem) + idx;
+                *pp = bf16x8_to_f16x8(*pp);
+            }
+            uint8_t *rowp = sQK + (solver ? 8192 : 0) + i * 128;
+            float ss = 0.f;
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint4 a = *reinterpret_cast<const uint4 *>(rowp + kb * 16384 + ((c ^ (i & 7)) << 4));
+                    const uint32_t wd[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float lo = __uint_as_float(wd[e] << 16), hi = __uint_as_float(wd[e] & 0xffff0000u);
+                        ss = fmaf(lo, lo, fmaf(hi, hi, ss));
+                    }
+                }
+            const float rn = rsqrtf(ss + norm_eps);
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint4 *pp = reinterpret_cast<uint4 *>(rowp + kb * 16384 + ((c ^ (i & 7)) << 4));
+                    const uint4 a = *pp;
+                    const uint32_t wd[4] = {a.x, a.y, a.z, a.w};
+                    uint32_t o[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        o[e] = pack_half2(__uint_as_float(wd[e] << 16) * rn, __uint_as_float(wd[e] & 0xffff0000u) * rn);
+                    *pp = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+        } else if (ok) {
             for (int idx = r; idx < PL::kLoadBytes / 16; idx += kRowThreads) {
                 uint4 *pp = reinterpret_cast<uint4 *>(smem) + idx;   // V and [Q ; K] are contiguous
                 *pp = bf16x8_to_f16x8(*pp);
             }
+        }
+        if (ok) {
             fence_proxy_async_smem();
             mbar_arrive(&ms.barConv);
             ok = mbar_wait(&ms.barXfree, 0, abort_flag);
@@ -1010,7 +1049,7 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
     cfg.numAttrs = pr.beside_previous ? 1 : 0;    // a part that runs beside the kernel launched before it
     e = cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut,
                            (__half *)ws.Ph, ws.Gd, ex, status, s.L, s.H, c_begin, n_range, pr.ready_flags,
-                           debug_wait_kcycles());
+                           pr.norm_eps, debug_wait_kcycles());
     count_launch();
     return e;
 }

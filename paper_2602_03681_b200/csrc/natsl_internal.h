@@ -26,6 +26,15 @@ struct BlockRouting {
     const void *k, *v;
 };
 
+// Grouped softmax heads and per-operation q/k normalisation (Section 4.3): G softmax heads per
+// linear head, each a slice of d / G columns of the linear head's q, k, v; norm_eps >= 0: q and k are
+// L2-normalised for the linear operation and RMS-normalised (per softmax head) for the softmax one,
+// inside the kernels; norm_eps < 0: used as given.
+struct HeadGroups {
+    int G = 1;
+    float norm_eps = -1.f;
+};
+
 // router.cu -- attention score layer: scores [B,L/C,H,2] (may be nullptr) and route [B,L,H]
 cudaError_t launch_score_layer(const void *x, const float *w_score, float *scores, uint8_t *route,
                                int d_model, Shape s, cudaStream_t st);
@@ -58,19 +67,25 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
                                         const int32_t *sm_chunk_prefix, const float *o_la,
                                         const float *w, float scale_sm, float eps, void *out,
                                         float *o_nla, float *lse, BlockRouting br, Shape s,
-                                        cudaStream_t st);
+                                        cudaStream_t st, int G = 1);
+// (G > 1: grouped softmax heads, fp32 storage only; see HeadGroups)
+// fp32 storage: q, k [rows, d] -> L2-normalised rows (q_la, k_la) and rows with each of the G slices
+// RMS-normalised (q_sm, k_sm)
+cudaError_t launch_qk_norm_f32(const float *q, const float *k, float *q_la, float *k_la, float *q_sm,
+                               float *k_sm, size_t rows, int d, int G, float norm_eps, cudaStream_t st);
 
 // softmax_tc.cu -- tensor-core softmax branch + combination (bf16 storage)
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
                                 const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
                                 void *k16, int32_t cap, int32_t capv, bool appending, int32_t *status,
-                                Shape s, cudaStream_t st);
+                                Shape s, cudaStream_t st, HeadGroups hg = HeadGroups{});
 cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const void *v16, int32_t cap,
                                       int32_t capv, const int32_t *sm_idx,
                                       const int32_t *sm_chunk_prefix, const void *o_la16,
                                       const int32_t *emit_flags, const float *w, float scale_sm,
                                       float eps, void *out, float *o_nla, float *lse, BlockRouting br,
-                                      bool appending, int32_t *status, Shape s, cudaStream_t st);
+                                      bool appending, int32_t *status, Shape s, cudaStream_t st,
+                                      HeadGroups hg = HeadGroups{});
 // (o_la16: the linear branch's read-out, o_laT [B,H,L/C,8,d,8] fp16; emit_flags: see ScanOut -- when given, the
 // kernel is launched as a programmatic dependent of the kernel before it in the stream, the scan)
 int sm_count();   // multiprocessors of the current device (cached per device)
@@ -113,6 +128,7 @@ struct PrepRange {
     int c_begin, n_chunks;
     int32_t *ready_flags;
     bool beside_previous;
+    float norm_eps = -1.f;     // >= 0: q and k rows are L2-normalised as the tiles are converted (Section 4.3)
 };
 cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, const float *g,
                                   const float *beta, const uint8_t *route, float scale_la,

@@ -27,6 +27,14 @@
 // the MMAs, warp 5 issues the TMA loads.
 // Block-level routing (template flag): after the retained tiles, one more tile per linear block of
 // the CTA's two, holding that block's own 64 tokens (Section 4.1, inner-chunk correlations).
+// Grouped softmax heads (template count kG; Section 4.3, several softmax heads under one linear head's
+// mask): the kG softmax heads of linear head h are the kG column slices of D columns of its q, k, v.
+// A CTA then serves one softmax head: its Q, K, V tiles are the slice's columns of the same tensors
+// ([B,L,H,kG D] read as [B,L,H kG,D]), the retained-token lists, the counters and the weights are the
+// linear head's, the softmax output is normalised over the slice and the linear read-out over its
+// whole row of kG D columns, of which the CTA writes its slice.  With norm_eps >= 0 the logits are
+// those of RMS-normalised q and k rows (Section 4.3), both as fp16: the K rows were normalised when
+// they were gathered, the softmax threads normalise the Q tile in place before the first product.
 #include "common.cuh"
 #include "natsl_internal.h"
 #include "tc_common.cuh"
@@ -57,14 +65,16 @@ template <int D> struct SmLayout {
 };
 
 struct Misc {                    // lives in the last kMiscBytes of the CTA's shared memory
-    uint64_t barQ, fullK[kStages], emptyK[kStages], fullV[kStages], emptyV[kStages], barS[2], barP, barO, barE;
+    uint64_t barQ, barQn, fullK[kStages], emptyK[kStages], fullV[kStages], emptyV[kStages], barS[2], barP, barO, barE;
     uint32_t tmem_base;
     int abort_flag, wait_kcycles;   // in this order: the waits read the limit as abort_flag[1]
     alignas(16) int pos[kBM];    // positions of the retained tokens inside the CTA's own chunks
 };
 static_assert(sizeof(Misc) <= kMiscBytes, "misc page too small");
 
-template <int D, bool kBlock>      // kBlock: block-level routing (own-block tiles after the retained ones)
+// kBlock: block-level routing (own-block tiles after the retained ones); kG: softmax heads per linear
+// head; kNorm: RMS-normalised q and k (norm_eps is read only then)
+template <int D, bool kBlock, int kG, bool kNorm>
 __global__ void __launch_bounds__(kThreadsTc)
 softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                           const __grid_constant__ CUtensorMap map_k,
@@ -76,10 +86,14 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                           const int32_t *__restrict__ sm_chunk_prefix,
                           const __half *__restrict__ o_laT, const int32_t *emit_flags,
                           const float *__restrict__ w,
-                          float scale_sm, float eps, int has_out, float *__restrict__ o_nla,
+                          float scale_sm, float eps, float norm_eps, int has_out, float *__restrict__ o_nla,
                           float *__restrict__ lse, int32_t *status, int L, int H, int wait_kcycles) {
     using SL = SmLayout<D>;
     constexpr int KB = SL::KB;
+    constexpr int DL = D * kG;                            // columns of the linear head
+    // the two o_laT tiles of the epilogue land in the Q tile and, for grouped heads, the K ring behind it
+    static_assert(2 * DL * 128 <= SL::kQBytes + (kG > 1 ? kStages * SL::kKStage : 0), "o_laT tiles do not fit");
+    static_assert(kG == 1 || SL::oK == SL::oQ + SL::kQBytes, "K ring must follow the Q tile");
     extern __shared__ __align__(1024) uint8_t smem[];
     Misc &ms = *reinterpret_cast<Misc *>(smem + SL::oMisc);
 
@@ -88,7 +102,9 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     // grid = (B*H, NP).  Beside the scan: tiles in ascending order, all (batch, head) pairs of a tile
     // before the next tile.  Otherwise: long rows first.
     const int p = emit_flags ? (int)blockIdx.y : NP - 1 - (int)blockIdx.y;
-    const int bh = blockIdx.x, b = bh / H, h = bh % H;
+    // blockIdx.x = (batch, linear head, softmax head of the group); H counts linear heads
+    const int bhg = blockIdx.x, bh = bhg / kG, sg = bhg % kG, b = bh / H, h = bh % H;
+    const int hq = h * kG + sg;                           // head index in the [B,L,H kG,D] view
     const int c0 = 2 * p, c1 = min(2 * p + 2, NC);
     const int32_t *pre = sm_chunk_prefix + (size_t)bh * (NC + 1);
     const int n_full = min(pre[c0], cap);             // retained tokens before the CTA's chunks
@@ -115,6 +131,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     }
     if (tid == 0) {
         mbar_init(&ms.barQ, 1);
+        mbar_init(&ms.barQn, kSoftmaxThreads);       // normalised queries written (NATSL_QK_NORM)
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ms.fullK[s], 1); mbar_init(&ms.emptyK[s], 1);
             mbar_init(&ms.fullV[s], 1); mbar_init(&ms.emptyV[s], 1);
@@ -149,7 +166,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 prefetch_tmap(&map_q); prefetch_tmap(&map_k); prefetch_tmap(&map_v);
                 mbar_arrive_expect_tx(&ms.barQ, SL::kQBytes);
                 for (int kb = 0; kb < KB; ++kb)
-                    tma_load_4d(smem + SL::oQ + kb * kBM * 128, &map_q, &ms.barQ, kb * 64, h, p * kBM, b);
+                    tma_load_4d(smem + SL::oQ + kb * kBM * 128, &map_q, &ms.barQ, kb * 64, hq, p * kBM, b);
                 // K and V tiles have their own rings: a K tile is free as soon as its Q K^T has run
                 // (early), a V tile only after its P V; K(u) is therefore requested before V(u-1).
                 for (int u = 0; u <= T2 && ok; ++u) {
@@ -160,8 +177,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                         mbar_arrive_expect_tx(&ms.fullK[s], SL::kKStage);
                         for (int kb = 0; kb < KB; ++kb) {
                             uint8_t *dst = smem + SL::oK + s * SL::kKStage + kb * kBN * 128;
-                            if (!kBlock || u < T) tma_load_2d(dst, &map_k, &ms.fullK[s], kb * 64, bh * cap + u * kBN);
-                            else tma_load_4d(dst, &map_kd, &ms.fullK[s], kb * 64, h, (c0 + own_block(u)) * kC, b);
+                            if (!kBlock || u < T) tma_load_2d(dst, &map_k, &ms.fullK[s], sg * D + kb * 64, bh * cap + u * kBN);
+                            else tma_load_4d(dst, &map_kd, &ms.fullK[s], kb * 64, hq, (c0 + own_block(u)) * kC, b);
                         }
                         nk = u + 1;
                     }
@@ -172,8 +189,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                         mbar_arrive_expect_tx(&ms.fullV[s], SL::kVStage);
                         for (int kb = 0; kb < KB; ++kb) {
                             uint8_t *dst = smem + SL::oV + s * SL::kVStage + kb * kBN * 128;
-                            if (!kBlock || t < T) tma_load_2d(dst, &map_v, &ms.fullV[s], kb * 64, bh * capv + t * kBN);
-                            else tma_load_4d(dst, &map_vd, &ms.fullV[s], kb * 64, h, (c0 + own_block(t)) * kC, b);
+                            if (!kBlock || t < T) tma_load_2d(dst, &map_v, &ms.fullV[s], sg * D + kb * 64, bh * capv + t * kBN);
+                            else tma_load_4d(dst, &map_vd, &ms.fullV[s], kb * 64, hq, (c0 + own_block(t)) * kC, b);
                         }
                         nv = t + 1;
                     }
@@ -190,10 +207,10 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             }
             bool e_issued = false;
             if (ok) {                           // the o_laT tiles of the CTA's one or two chunks
-                mbar_arrive_expect_tx(&ms.barE, (c1 - c0) * D * 128);
+                mbar_arrive_expect_tx(&ms.barE, (c1 - c0) * DL * 128);
                 for (int e = 0; e < c1 - c0; ++e)
-                    bulk_load_1d(smem + SL::oQ + e * (D * 128), o_laT + ((size_t)bh * NC + c0 + e) * D * 64,
-                                 D * 128, &ms.barE);
+                    bulk_load_1d(smem + SL::oQ + e * (DL * 128), o_laT + ((size_t)bh * NC + c0 + e) * DL * 64,
+                                 DL * 128, &ms.barE);
                 e_issued = true;
             }
             // No copy may be in flight when the CTA retires, aborted or not: wait (with a bound of
@@ -208,7 +225,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     } else if (warp == 4) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0 && T2 > 0) {
-            constexpr uint32_t idesc_qk = make_idesc(kFmtBF16, kBM, kBN, false, false);
+            // logits: q and k as given are bf16; normalised ones are fp16 (see the softmax threads)
+            constexpr uint32_t idesc_qk = make_idesc(kNorm ? kFmtF16 : kFmtBF16, kBM, kBN, false, false);
             constexpr uint32_t idesc_pv = make_idesc(kFmtF16, kBM, D, false, true);
             const uint32_t aQ = smem_u32(smem + SL::oQ);
             auto issue_qk = [&](int t) {
@@ -223,7 +241,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 mma_commit(&ms.emptyK[t % kStages]);
                 mma_commit(&ms.barS[t & 1]);
             };
-            bool ok = mbar_wait(&ms.barQ, 0, abort_flag) && mbar_wait(&ms.fullK[0], 0, abort_flag);
+            bool ok = mbar_wait(&ms.barQ, 0, abort_flag) && (!kNorm || mbar_wait(&ms.barQn, 0, abort_flag)) &&
+                      mbar_wait(&ms.fullK[0], 0, abort_flag);
             if (ok) {
                 tc_fence_after_sync();
                 issue_qk(0);
@@ -256,13 +275,54 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         const float sl2 = scale_sm * 1.4426950408889634f;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
+        if (kNorm && T2 > 0) {
+            // RMS-normalised queries (Section 4.3): thread r rewrites row r of the Q tile (bf16, as loaded)
+            // as fp16 of the normalised row, over the D columns of its softmax head; the keys were
+            // normalised and stored as fp16 when they were gathered, so the logit product is an fp16
+            // MMA (bf16 keeps 8 bits: rounding the normalised keys to it alone costs 2.8e-2 of the
+            // branch output's RMS).  Eight 16-byte pieces per row and block, taken in an order that
+            // spreads the warp over the banks.
+            ok = mbar_wait(&ms.barQ, 0, abort_flag);
+            if (ok) {
+                uint8_t *rowp = smem + SL::oQ + tid * 128;
+                float ss = 0.f;
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint4 a = *reinterpret_cast<const uint4 *>(rowp + kb * kBM * 128 + ((c ^ (tid & 7)) << 4));
+                        const uint32_t wd[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float lo = __uint_as_float(wd[e] << 16), hi = __uint_as_float(wd[e] & 0xffff0000u);
+                            ss = fmaf(lo, lo, fmaf(hi, hi, ss));
+                        }
+                    }
+                const float rq = rsqrtf(ss / D + norm_eps);
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        uint4 *pp = reinterpret_cast<uint4 *>(rowp + kb * kBM * 128 + ((c ^ (tid & 7)) << 4));
+                        const uint4 a = *pp;
+                        const uint32_t wd[4] = {a.x, a.y, a.z, a.w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            o[e] = pack_half2(__uint_as_float(wd[e] << 16) * rq, __uint_as_float(wd[e] & 0xffff0000u) * rq);
+                        *pp = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                fence_proxy_async_smem();
+                mbar_arrive(&ms.barQn);
+            }
+        }
         float2 wv = make_float2(0.5f, 0.5f);             // (w_nla, w_la) of this row
         if (w && i_abs < L) wv = __ldg(reinterpret_cast<const float2 *>(w + (((size_t)b * L + i_abs) * H + h) * 2));
         // The compacted keys are in position order, so row i sees exactly the first `cnt` of them:
         // all n_full earlier ones plus those of the CTA's own chunks at positions <= i.
         int cnt = n_full;
         for (int kq = 0; kq < n_end - n_full; ++kq) cnt += ms.pos[kq] <= i_abs ? 1 : 0;
-        for (int t = 0; t < T2; ++t) {
+        for (int t = 0; ok && t < T2; ++t) {
             ok = mbar_wait(&ms.barS[t & 1], (t >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
@@ -367,7 +427,16 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             const float inv = l > 0.f ? 1.f / l : 0.f;       // l = 0 (no visible key): o_nla = 0
             float ssn4[4] = {0.f, 0.f, 0.f, 0.f}, ssl4[4] = {0.f, 0.f, 0.f, 0.f};
             const int tok = r & 63, tp = tok >> 3;
-            const uint8_t *la_col = smem + SL::oQ + (r >> 6) * (D * 128) + tp * (D * 16) + (tok & 7) * 2;
+            const uint8_t *la_col = smem + SL::oQ + (r >> 6) * (DL * 128) + tp * (DL * 16) + (tok & 7) * 2;
+            if (kG > 1) {        // the other softmax heads' columns of the linear row: mean square only
+#pragma unroll 4
+                for (int row = 0; row < DL; row += 2) {
+                    if (row / D == sg) continue;
+                    const float a0 = __half2float(*reinterpret_cast<const __half *>(la_col + ((row ^ tp) << 4)));
+                    const float a1 = __half2float(*reinterpret_cast<const __half *>(la_col + (((row + 1) ^ tp) << 4)));
+                    ssl4[(row >> 1) & 3] = fmaf(a0, a0, fmaf(a1, a1, ssl4[(row >> 1) & 3]));
+                }
+            }
             // This query's column of o_la is read once, kept as fp16 pairs (D / 2 registers: the logits of
             // the main loop are dead by now) and used twice: for its mean square and for the output.
             uint32_t la2[D / 2];
@@ -383,7 +452,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 }
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
-                    const int row = 32 * cb + e;
+                    const int row = sg * D + 32 * cb + e;
                     const __half a0 = *reinterpret_cast<const __half *>(la_col + ((row ^ tp) << 4));
                     const __half a1 = *reinterpret_cast<const __half *>(la_col + (((row + 1) ^ tp) << 4));
                     const __half2 ap = __halves2half2(a0, a1);
@@ -397,8 +466,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             // mean square of the normalised row = inv^2 * mean square of the accumulator row
             const float msn = inv * inv * ((ssn4[0] + ssn4[1]) + (ssn4[2] + ssn4[3])) / D;
             const float wn = wv.x * rsqrtf(msn + eps) * inv;          // applies to the raw accumulator
-            const float wl = wv.y * rsqrtf(((ssl4[0] + ssl4[1]) + (ssl4[2] + ssl4[3])) / D + eps);
-            float *onla_row = o_nla && i_abs < L ? o_nla + (((size_t)b * L + i_abs) * H + h) * D : nullptr;
+            const float wl = wv.y * rsqrtf(((ssl4[0] + ssl4[1]) + (ssl4[2] + ssl4[3])) / DL + eps);
+            float *onla_row = o_nla && i_abs < L ? o_nla + (((size_t)b * L + i_abs) * H + h) * DL + sg * D : nullptr;
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t ov[32];
@@ -433,13 +502,13 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 }
             }
             if (lse && i_abs < L)
-                lse[(size_t)bh * L + i_abs] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                lse[(size_t)bhg * L + i_abs] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
             fence_proxy_async_smem();
             named_barrier_sync(1, kSoftmaxThreads);
             if (tid == 0) {
                 if (has_out)
                     for (int kb = 0; kb < KB; ++kb)
-                        tma_store_4d(&map_out, smem + SL::oV + kb * (kBM * 128), kb * 64, h, p * kBM, b);
+                        tma_store_4d(&map_out, smem + SL::oV + kb * (kBM * 128), kb * 64, hq, p * kBM, b);
                 tma_store_commit();
                 tma_store_wait_read();                      // shared memory may go once it has been read
             }
@@ -465,7 +534,7 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
                     const int32_t *__restrict__ sm_idx, const int32_t *__restrict__ sm_chunk_prefix,
                     __nv_bfloat16 *__restrict__ k_sm, __nv_bfloat16 *__restrict__ v_sm,
                     __half *__restrict__ v16, __half *__restrict__ k16, int cap, int capv, int appending,
-                    int32_t *status, int L, int H) {
+                    int groups, float norm_eps, int32_t *status, int L, int H) {
     constexpr int kVecPerRow = D * 2 / 16;
     constexpr int kRows = 256 / kVecPerRow;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
@@ -498,7 +567,27 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
         }
         const int tok = sm_idx[(size_t)bh * L + row - n_prev];
         const size_t src = (((size_t)b * L + tok) * H + h) * D;
-        const uint4 kk = reinterpret_cast<const uint4 *>(k + src)[piece];
+        uint4 kk = reinterpret_cast<const uint4 *>(k + src)[piece];
+        if (norm_eps >= 0.f) {
+            // RMS-normalised keys of the softmax operation (Section 4.3), per softmax head = per slice of
+            // D / groups columns: the slice's pieces sit in neighbouring lanes of the row's lanes
+            const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
+            float f[8], ss = 0.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                f[2 * i] = __uint_as_float(kw[i] << 16);
+                f[2 * i + 1] = __uint_as_float(kw[i] & 0xffff0000u);
+                ss = fmaf(f[2 * i], f[2 * i], fmaf(f[2 * i + 1], f[2 * i + 1], ss));
+            }
+            const int lanes = kVecPerRow / groups;            // lanes per slice (a power of two)
+            const unsigned row_mask = (kVecPerRow == 32 ? 0xffffffffu : ((1u << kVecPerRow) - 1u))
+                                      << ((threadIdx.x & 31) & ~(kVecPerRow - 1));
+            for (int o = 1; o < lanes; o <<= 1) ss += __shfl_xor_sync(row_mask, ss, o);
+            const float rk = rsqrtf(ss * groups / D + norm_eps);
+            // stored as fp16 (the softmax kernel's logit product is an fp16 MMA in this mode)
+            kk = make_uint4(pack_half2(f[0] * rk, f[1] * rk), pack_half2(f[2] * rk, f[3] * rk),
+                            pack_half2(f[4] * rk, f[5] * rk), pack_half2(f[6] * rk, f[7] * rk));
+        }
         reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
         if (dk16) {
             const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
@@ -521,34 +610,41 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
 
 }  // namespace
 
-template <int D>
+template <int D, int G>      // D: columns of a softmax head; G of them per linear head (s.d = D G)
 static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *v16, int32_t cap,
                                    int32_t capv, const int32_t *sm_idx, const int32_t *pre,
                                    const void *o_la16, const int32_t *emit_flags, const float *w,
-                                   float scale_sm, float eps, void *out, float *o_nla, float *lse,
+                                   float scale_sm, float eps, float norm_eps, void *out, float *o_nla, float *lse,
                                    BlockRouting br, bool appending, int32_t *status, Shape s,
                                    cudaStream_t st) {
     using SL = SmLayout<D>;
     CUtensorMap mq, mk, mv, mout, mkd, mvd;
-    if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, kBM) ||
-        !tch::make_map_2d(&mk, k_sm, (uint64_t)s.B * s.H * cap, D, kBN) ||
-        !tch::make_map_2d(&mv, v16, (uint64_t)s.B * s.H * capv, D, kBN))
+    // q, out, k, v [B,L,H,G D] are read as [B,L,H G,D]; the compacted K/V rows keep all G D columns
+    if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H * G, D, kBM) ||
+        !tch::make_map_2d(&mk, k_sm, (uint64_t)s.B * s.H * cap, D * G, kBN) ||
+        !tch::make_map_2d(&mv, v16, (uint64_t)s.B * s.H * capv, D * G, kBN))
         return cudaErrorInvalidValue;
     mout = mq;                                             // placeholder when `out` is not asked for
-    if (out && !tch::make_map_blhd(&mout, out, s.B, s.L, s.H, D, kBM)) return cudaErrorInvalidValue;
+    if (out && !tch::make_map_blhd(&mout, out, s.B, s.L, s.H * G, D, kBM)) return cudaErrorInvalidValue;
     mkd = mq;
     mvd = mq;
-    if (br.route && (!tch::make_map_blhd(&mkd, br.k, s.B, s.L, s.H, D, kBN) ||
-                     !tch::make_map_blhd(&mvd, br.v, s.B, s.L, s.H, D, kBN)))
+    if (br.route && (!tch::make_map_blhd(&mkd, br.k, s.B, s.L, s.H * G, D, kBN) ||
+                     !tch::make_map_blhd(&mvd, br.v, s.B, s.L, s.H * G, D, kBN)))
         return cudaErrorInvalidValue;
-    auto kernel = br.route ? softmax_combine_tc_kernel<D, true> : softmax_combine_tc_kernel<D, false>;
+    // (block-level routing is built without grouping and without normalisation only)
+    auto kernel = softmax_combine_tc_kernel<D, false, G, false>;
+    if (norm_eps >= 0.f) kernel = softmax_combine_tc_kernel<D, false, G, true>;
+    if (br.route) {
+        if (G > 1 || norm_eps >= 0.f) return cudaErrorInvalidValue;
+        kernel = softmax_combine_tc_kernel<D, true, 1, false>;
+    }
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal);
     if (e != cudaSuccess) return e;
     // With emit_flags the kernel is launched as a programmatic dependent of the kernel before it in
     // the stream (the scan): it may start once all of the scan's CTAs are resident, and finds o_la
     // through the flags.  A launch the runtime serialises instead finds every flag already raised.
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(s.B * s.H, (s.L + kBM - 1) / kBM);
+    cfg.gridDim = dim3(s.B * s.H * G, (s.L + kBM - 1) / kBM);
     cfg.blockDim = dim3(kThreadsTc);
     cfg.dynamicSmemBytes = SL::kTotal;
     cfg.stream = st;
@@ -559,7 +655,7 @@ static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *
     cfg.numAttrs = emit_flags ? 1 : 0;
     e = cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mout, mkd, mvd, br.route, appending ? 1 : 0,
                            (int)cap, (int)capv, sm_idx, pre, (const __half *)o_la16, emit_flags, w, scale_sm, eps,
-                           out ? 1 : 0, o_nla, lse, status, s.L, s.H, debug_wait_kcycles());
+                           norm_eps, out ? 1 : 0, o_nla, lse, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
     return e;
 }
@@ -569,26 +665,32 @@ cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const voi
                                       const int32_t *sm_chunk_prefix, const void *o_la16,
                                       const int32_t *emit_flags, const float *w, float scale_sm,
                                       float eps, void *out, float *o_nla, float *lse, BlockRouting br,
-                                      bool appending, int32_t *status, Shape s, cudaStream_t st) {
+                                      bool appending, int32_t *status, Shape s, cudaStream_t st,
+                                      HeadGroups hg) {
+    if (hg.G == 2 && s.d == 128)
+        return softmax_tc_impl<64, 2>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la16, emit_flags,
+                                      w, scale_sm, eps, hg.norm_eps, out, o_nla, lse, br, appending, status, s, st);
+    if (hg.G > 1) return cudaErrorInvalidValue;
     if (s.d == 128)
-        return softmax_tc_impl<128>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la16, emit_flags,
-                                    w, scale_sm, eps, out, o_nla, lse, br, appending, status, s, st);
-    return softmax_tc_impl<64>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la16, emit_flags, w,
-                               scale_sm, eps, out, o_nla, lse, br, appending, status, s, st);
+        return softmax_tc_impl<128, 1>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la16, emit_flags,
+                                       w, scale_sm, eps, hg.norm_eps, out, o_nla, lse, br, appending, status, s, st);
+    return softmax_tc_impl<64, 1>(q, k_sm, v16, cap, capv, sm_idx, sm_chunk_prefix, o_la16, emit_flags, w,
+                                  scale_sm, eps, hg.norm_eps, out, o_nla, lse, br, appending, status, s, st);
 }
 
 template <int D>
 static cudaError_t gather_tc_impl(const void *k, const void *v, const int32_t *sm_idx,
                                   const int32_t *pre, void *k_sm, void *v_sm, void *v16, void *k16,
                                   int cap, int capv, bool appending, int32_t *status, Shape s,
-                                  cudaStream_t st) {
+                                  cudaStream_t st, HeadGroups hg) {
     constexpr int kRows = 256 / (D * 2 / 16);
     const int max_rows = s.L < capv ? s.L : capv;
     const int blocks = (max_rows + kRows - 1) / kRows;
     dim3 grid(blocks < 48 ? blocks : 48, s.B * s.H);
     gather_kv_tc_kernel<D><<<grid, 256, 0, st>>>(
         (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, sm_idx, pre, (__nv_bfloat16 *)k_sm,
-        (__nv_bfloat16 *)v_sm, (__half *)v16, (__half *)k16, cap, capv, appending ? 1 : 0, status, s.L, s.H);
+        (__nv_bfloat16 *)v_sm, (__half *)v16, (__half *)k16, cap, capv, appending ? 1 : 0, hg.G, hg.norm_eps,
+        status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -596,10 +698,10 @@ static cudaError_t gather_tc_impl(const void *k, const void *v, const int32_t *s
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
                                 const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
                                 void *k16, int32_t cap, int32_t capv, bool appending, int32_t *status,
-                                Shape s, cudaStream_t st) {
+                                Shape s, cudaStream_t st, HeadGroups hg) {
     if (s.d == 128)
-        return gather_tc_impl<128>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st);
-    return gather_tc_impl<64>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st);
+        return gather_tc_impl<128>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st, hg);
+    return gather_tc_impl<64>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st, hg);
 }
 
 }  // namespace natsl
