@@ -535,10 +535,50 @@ def bench_other_workloads(peaks, peak_kind="measured", traffic=None):
         res[name] = entry
         del d, ws
         torch.cuda.empty_cache()
+    res["grouped_heads_6x2_qk_norm"] = bench_grouped_heads(peaks, peak_kind)
     res["score_layer"] = bench_score_layer(peaks)
     res["cfg2_bf16_long_prefill/in_4_pieces"] = bench_prefill_in_pieces()
     res["serving_131072_tokens"] = bench_long_context_serving()
     return res
+
+
+def bench_grouped_heads(peaks, peak_kind, B=10, H=6, G=2):
+    """Forward with grouped softmax heads and in-kernel q/k normalisation (Section 4.3) on the
+    smaller model's head counts (appendix: six linear heads, twelve softmax heads) at the prefill
+    workload's length and head size: H = 6 linear heads of d = 128, G = 2 softmax heads of 64 each,
+    L = 4096, B = 10 (60 (batch, head) pairs, close to the prefill workload's 64).  The useful FLOPs
+    are those of the ungrouped layer: G heads of d / G columns do the same logit and value products."""
+    import dataclasses
+
+    import torch
+
+    from paper_2602_03681_b200 import binding
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg1_bf16_prefill"], B=B, H=H, seed=5)
+    x = inputs.make_layer_inputs(wl)
+    d = {m: torch.from_numpy(x[m]).cuda() for m in ("g", "beta", "route", "w")}
+    for m in ("q", "k", "v"):
+        d[m] = torch.from_numpy(x[m]).cuda().to(torch.bfloat16)
+    ms = {}
+    for label, kw in (("grouped_qk_norm", dict(G=G, flags=binding.QK_NORM, norm_eps=1e-6,
+                                               scale_sm=float(wl.d // G) ** -0.5)),
+                      ("plain_same_shapes", dict(scale_sm=wl.scale_sm))):
+        ws = None
+        best = float("inf")
+        for it in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ws = binding.hybrid_fwd(d["q"], d["k"], d["v"], d["g"], d["beta"], d["route"], d["w"],
+                                    scale_la=wl.scale_la, ws=ws, **kw)["ws"]
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                best = min(best, e0.elapsed_time(e1))
+        assert binding.natsl_device_status(ws) == 0
+        ms[label] = best
+    fl = sum(useful_flops(x["route"], wl.d, wl.C).values())
+    return {"B": B, "H_linear": H, "G": G, "L": wl.L, "d": wl.d, "ms": ms,
+            "tokens_per_s": B * wl.L / (ms["grouped_qk_norm"] * 1e-3), "useful_fwd_gflop": fl / 1e9,
+            "roofline": {"fwd": tensor_roofline(fl, ms["grouped_qk_norm"], peaks, peak_kind)}}
 
 
 def bench_long_context_serving(L=131072, piece=16384, decode_steps=64):

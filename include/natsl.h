@@ -92,8 +92,9 @@ enum {
                                     decay alone).  state_out, k_sm, v_sm, sm_len hold what is kept
                                     after the last block.  A route that changes inside a block is
                                     reported as NATSL_ERR_ROUTE by natsl_device_status.  Backward:
-                                    built for bf16 storage with d = 64, NATSL_ERR_UNSUPPORTED
-                                    otherwise.  Generation: route 2 in
+                                    built on every path (bf16 storage with d = 64: fused per
+                                    chunk; d = 128 and fp32 storage: the chunk-level products as
+                                    separate kernels).  Generation: route 2 in
                                     natsl_decode_step and natsl_decode_block_end (no flag needed) */
     NATSL_APPEND_CACHE = 1u << 3,      /* forward, tensor-core path: prefill in pieces.  p->k_sm, p->v_sm,
                                     p->sm_len (required) are read AND written: the cache already

@@ -152,6 +152,9 @@ struct BwdWs {
     float *P, *Abar, *M, *N, *Mg, *Ms, *Ns;                  // [B,H,NC,64,64]
     float *S_c, *dS_c;                                       // [B,H,NC,d,d]
     float *Gcum, *lse, *Dsm, *dGrow, *kappa, *gS;            // [B,H,L] (gS: [B,H,NC,d/32])
+    float *dk_x, *dv_x, *dmask;                              // block-level routing off the fused path: the
+                                                             // softmax branch's dk, dv of every token
+                                                             // (token-major), mask gradients per retained key [B,H,L]
     void *k_smb, *k16, *v16, *Qh, *dO16;                     // tensor-core softmax branch: 16-bit [B,H,L,d]
     void *dOla16, *dOlag16;                                  // tensor-core reverse scan: fp16 [B,H,L,d]
     void *o_la16;                                            // linear read-out as fp16 [B,L,H,d]
@@ -190,7 +193,7 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.o_la = tm(true);
     f.o_nla = tm(true);
     f.do_la = tm(true);
-    f.do_nla = tm(!tcs);
+    f.do_nla = tm(!tcs || (general && block));     // (fp32 own-block kernel of block-level routing)
     f.dUt = tcs ? f.o_la : tm(true);
     f.dQg = tm(general); f.dW = tm(general); f.dKt = tm(general); f.dKb = tm(general); f.dVb = tm(general);
     f.X1p = tm(general); f.X2 = tm(general);
@@ -207,6 +210,8 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.dGrow = c.take<float>(BHL);
     f.kappa = c.take<float>(BHL);
     f.gS = c.take<float>(general ? B * H * NC * (d / 32) : 0);
+    f.dk_x = tm(general && block); f.dv_x = tm(general && block);
+    f.dmask = c.take<float>(general && block ? BHL : 0);
     const size_t h16 = tcs ? TM * 2 : 0;
     f.k_smb = c.take<char>(h16);
     f.k16 = c.take<char>(h16);
@@ -342,10 +347,10 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
                                      ex, ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, block_route,
                                      f.status, s, st));
     } else {
-        NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, route, p->scale_la, f.W, f.U,
-                                          f.P, f.Abar, f.Gcum, s32, st));
+        NATSL_TRY(launch_gdn_prepare_simt(f.q32, f.k32, f.v32, g, beta, block ? nullptr : route, p->scale_la,
+                                          f.W, f.U, f.P, f.Abar, f.Gcum, s32, st));
         NATSL_TRY(launch_gdn_scan_simt(f.q32, f.k32, g, f.W, f.U, f.P, p->scale_la, p->state_in, state_out,
-                                       f.S_c, f.Ut, f.o_la, nullptr, s32, st));
+                                       f.S_c, f.Ut, f.o_la, block_route, s32, st));
     }
     NATSL_TRY(side_join.join());
     if (tensor_cores)
@@ -355,7 +360,7 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
     else
         NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
                                               f.o_la, p->w, p->scale_sm, p->eps, out, f.o_nla,
-                                              f.lse, BlockRouting{nullptr, nullptr, nullptr}, s32, st));
+                                              f.lse, BlockRouting{block_route, f.k32, f.v32}, s32, st));
 #undef NATSL_TRY
     return NATSL_OK;
 }
@@ -465,7 +470,6 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
         // The forward of a training step: run in the backward's workspace, where it leaves what
         // natsl_hybrid_bwd (with NATSL_SAVED_FWD) would otherwise compute again.
         if (append || want_cache || p->o_la || p->o_nla || p->lse || p->stage_events) return NATSL_ERR_UNSUPPORTED;
-        if (block && !(tensor_cores && p->d == 64)) return NATSL_ERR_UNSUPPORTED;
         const BwdWs fb = carve_bwd(p, ws);
         if (!ws || ws_bytes < fb.bytes) return NATSL_ERR_WORKSPACE;
         return bwd_forward_part(q, k, v, g, beta, route, out, p->state_out, p, fb, st);
@@ -601,9 +605,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (p->flags & NATSL_APPEND_CACHE) return NATSL_ERR_UNSUPPORTED;
     if (grouped_or_normed(p)) return NATSL_ERR_UNSUPPORTED;   // grouped heads, q/k normalisation: forward only
     if (use_tensor_cores(p) && !(p->scale_sm > 0.f)) return NATSL_ERR_SHAPE;
-    // block-level routing: on the path with the fused chunk kernel only (bf16 storage, d = 64)
     const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
-    if (block && !(use_tensor_cores(p) && p->d == 64)) return NATSL_ERR_UNSUPPORTED;
     if (p->dscore && !block) return NATSL_ERR_UNSUPPORTED;   // score gradients: one decision per block
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(dout) || !aligned16(dq) ||
         !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
@@ -645,8 +647,9 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     // so that a loss-scaled or a tiny dout stays inside fp16's range (grad_scale, common.cuh).
     if (tensor_cores) NATSL_TRY(launch_dout_amax(dout, (size_t)(B * L * H * d), s.bf16, f.status, st));
     const int32_t *gsc = tensor_cores ? f.status : nullptr;
+    const bool general_block = block && !fused_chunks;   // block-level routing with separate chunk-level products
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la,
-                                 tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,
+                                 tensor_cores && !general_block ? nullptr : f.do_nla, dw, f.Dsm,
                                  tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
                                  tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, gsc, s, st));
     // Dependencies from here on: the query-side softmax kernel, the key-side one and the reverse
@@ -672,16 +675,17 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                         //  scan on the side stream reads it, so it is not written again)
         NATSL_TRY(launch_softmax_bwd_tc(q, f.Qh, f.dO16, f.k16, f.v16, p->L, f.sm_idx, f.prefix, f.lse,
                                         f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm,
-                                        p->dscore ? f.dGrow : nullptr, fused_chunks, f.status, s, st,
-                                        kv_aside ? st0 : st));
+                                        p->dscore ? (general_block ? f.dmask : f.dGrow) : nullptr, fused_chunks,
+                                        f.status, s, st, kv_aside ? st0 : st));
     else
         NATSL_TRY(launch_softmax_bwd(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix, f.do_nla,
-                                     f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st));
+                                     f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st,
+                                     p->dscore ? f.dmask : nullptr));
     if (!tensor_cores)
         NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
-                                   f.dS_c, f.gS, p->dstate_out, p->dstate_in, s, st));
+                                   f.dS_c, f.gS, p->dstate_out, p->dstate_in, s, st, block_route));
     if (side) NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));     // the reverse scan has finished
-    AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
+    AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, general_block ? nullptr : route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
                    f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
                    p->scale_la, f.dGrow, f.kappa, dbeta, dg};
     if (fused_chunks && block) {
@@ -698,7 +702,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                        f.Gcum, beta, route, f.dq_sm, p->scale_la, dq, dk, dv, dg, dbeta,
                                        true, dk_x, dv_x, p->dscore ? f.kappa : nullptr, s, st));
         if (p->dscore)   // (dGrow, kappa: [B,H,L] scratch the fused path does not otherwise use)
-            NATSL_TRY(launch_dscore(route, f.prefix, f.dGrow, f.kappa, p->L, p->dscore, s, st));
+            NATSL_TRY(launch_dscore(route, f.prefix, f.dGrow, f.kappa, nullptr, p->L, p->dscore, s, st));
         return NATSL_OK;
     }
     if (fused_chunks) {   // all chunk-level products and the assembly in one kernel per chunk
@@ -710,6 +714,18 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(side_join.join());      // the side stream's last kernels
         return NATSL_OK;
     }
+    // (block-level routing: beta~ = beta for every token, so the kernels below get no route)
+    const uint8_t *route_bt = general_block ? nullptr : route;
+    if (general_block) {
+        // Every token has a softmax-branch dk, dv: the retained tokens' from the compacted gradients, the
+        // tokens of linear blocks' from their own block (each token is written by exactly one of the
+        // two); the assembly adds them to the linear branch's.
+        NATSL_TRY(launch_gdn_finish(a, f.dk_x, f.dv_x, s32, st, false));
+        NATSL_TRY(launch_softmax_bwd_own_block_simt(f.q32, f.k32, f.v32, f.do_nla, f.lse, f.Dsm, route,
+                                                    p->scale_sm, f.dq_sm, f.dk_x, f.dv_x, gsc, s32, st));
+        a.dk_x = f.dk_x;
+        a.dv_x = f.dv_x;
+    }
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, s, st));
@@ -718,16 +734,18 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dW), TM(f.dKb), kC, di, kC, 1.f, false, s, st));
         NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dUt), TM(f.dVb), kC, di, kC, 1.f, false, s, st));
     } else {
-        NATSL_TRY(launch_gdn_tsolve(f.Abar, beta, route, f.dW, f.dUt, f.dKb, f.dVb, s, st));
+        NATSL_TRY(launch_gdn_tsolve(f.Abar, beta, route_bt, f.dW, f.dUt, f.dKb, f.dVb, s, st));
     }
     NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dKb), TM(f.W), CC(f.M), kC, kC, di, -1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dVb), TM(f.U), CC(f.M), kC, kC, di, -1.f, true, s, st));
-    NATSL_TRY(launch_mask_scale(f.M, f.N, f.Gcum, beta, route, p->scale_la, f.Mg, f.Ms, f.Ns, s, st));
+    NATSL_TRY(launch_mask_scale(f.M, f.N, f.Gcum, beta, route_bt, p->scale_la, f.Mg, f.Ms, f.Ns, s, st));
     NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Mg), TM(f.k32), TM(f.X1p), kC, di, kC, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ms), TM(f.k32), TM(f.X2), kC, di, kC, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Ns), TM(f.k32), TM(f.X3), kC, di, kC, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ns), TM(f.q32), TM(f.X4), kC, di, kC, 1.f, false, s, st));
     NATSL_TRY(launch_gdn_assemble(a, dq, dk, dv, s, st));
+    if (p->dscore)   // softmax blocks: the mask gradients of their keys; linear blocks: the kappa of their tokens
+        NATSL_TRY(launch_dscore(route, f.prefix, f.dmask, nullptr, f.kappa, p->L, p->dscore, s, st));
 #undef NATSL_TRY
     return NATSL_OK;
 }

@@ -309,7 +309,9 @@ softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ 
                        const int32_t *__restrict__ sm_chunk_prefix,
                        const float *__restrict__ do_nla, const float *__restrict__ lse,
                        const float *__restrict__ Dsm, float scale_sm, float *__restrict__ dk_sm,
-                       float *__restrict__ dv_sm, int L, int H) {
+                       float *__restrict__ dv_sm, float *__restrict__ dmask, int L, int H) {
+    // dmask [B,H,cap] (or nullptr): per retained key j the sum over its queries of
+    // dM_ij = p_ij (dp_ij - <do_i, o_i>), the mask gradient of Section 4.2
     extern __shared__ float smem[];
     float *Kt = smem;                       // [32][D+1]
     float *Vt = Kt + 32 * (D + 1);          // [32][D+1]
@@ -349,7 +351,7 @@ softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ 
     const int c_first = pos[0] / kC;
     constexpr int kPer = D / 8;
     const int kj = threadIdx.x >> 3, cs = threadIdx.x & 7;
-    float adk[kPer], adv[kPer];
+    float adk[kPer], adv[kPer], adm = 0.f;
 #pragma unroll
     for (int x = 0; x < kPer; ++x) { adk[x] = 0.f; adv[x] = 0.f; }
 
@@ -384,6 +386,7 @@ softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ 
         __syncthreads();
         for (int il = 0; il < kC; ++il) {
             const float pj = Ps[il * 33 + kj], ds = Dss[il * 33 + kj];
+            adm += ds;
             const float *dor = dOs + il * D + cs, *qr = Qs + il * D + cs;
 #pragma unroll
             for (int x = 0; x < kPer; ++x) {
@@ -397,6 +400,84 @@ softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ 
         float *dvr = dv_sm + ((size_t)bh * cap + j0 + kj) * D + cs;
 #pragma unroll
         for (int x = 0; x < kPer; ++x) { dkr[8 * x] = scale_sm * adk[x]; dvr[8 * x] = adv[x]; }
+        if (dmask && cs == 0) dmask[(size_t)bh * cap + j0 + kj] = adm;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Block-level routing (Section 4.1, inner-chunk correlations): a query in a linear block also reads
+// the causal part of its own block, whose tokens are not among the retained ones.  One CTA per
+// linear block adds that part of the softmax branch's backward in fp32:
+//   p_ij = exp(scale s_ij - lse_i), ds_ij = p_ij (dp_ij - D_i), j <= i, with lse_i and
+//   D_i = <do_i, o_i> of the whole softmax row;
+//   dq_sm += scale dS K;  dk_x = scale dS^T Q,  dv_x = P^T dO  (written: the tokens of a linear
+//   block have no other softmax-branch gradient).  grid = (L/64, B*H); softmax blocks return.
+// Dsm arrives times the gradient scale of the tensor-core kernels (gsc; 1 without them).
+// ------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(kThreads)
+softmax_bwd_own_block_simt_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
+                                  const float *__restrict__ v32, const float *__restrict__ do_nla,
+                                  const float *__restrict__ lse, const float *__restrict__ Dsm,
+                                  const uint8_t *__restrict__ route, float scale_sm,
+                                  float *__restrict__ dq_sm, float *__restrict__ dk_x,
+                                  float *__restrict__ dv_x, const int32_t *gsc, int L, int H) {
+    extern __shared__ float smem[];
+    float *Qs = smem;                        // [64][D+1]
+    float *Ks = Qs + kC * (D + 1);
+    float *Vs = Ks + kC * (D + 1);
+    float *dOs = Vs + kC * (D + 1);
+    float *Ps = dOs + kC * (D + 1);          // [64][65]
+    float *dSs = Ps + kC * (kC + 1);         // [64][65]
+    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    const size_t ts = (size_t)H * D;
+    const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
+    if (route[tok0]) return;                 // a softmax block: its tokens are retained ones
+    const float ginv = grad_scale(gsc).y;
+    for (int idx = threadIdx.x; idx < kC * D / 4; idx += kThreads) {
+        const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
+        const size_t src = tok0 * D + (size_t)r * ts + c4;
+        const float4 a = load4(q32 + src), bb = load4(k32 + src), cc = load4(v32 + src), dd = load4(do_nla + src);
+        float *p0 = Qs + r * (D + 1) + c4, *p1 = Ks + r * (D + 1) + c4, *p2 = Vs + r * (D + 1) + c4,
+              *p3 = dOs + r * (D + 1) + c4;
+        p0[0] = a.x; p0[1] = a.y; p0[2] = a.z; p0[3] = a.w;
+        p1[0] = bb.x; p1[1] = bb.y; p1[2] = bb.z; p1[3] = bb.w;
+        p2[0] = cc.x; p2[1] = cc.y; p2[2] = cc.z; p2[3] = cc.w;
+        p3[0] = dd.x; p3[1] = dd.y; p3[2] = dd.z; p3[3] = dd.w;
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < kC * kC; idx += kThreads) {
+        const int i = idx >> 6, j = idx & 63;
+        float pj = 0.f, ds = 0.f;
+        if (j <= i) {
+            const float *qr = Qs + i * (D + 1), *kr = Ks + j * (D + 1), *dor = dOs + i * (D + 1), *vr = Vs + j * (D + 1);
+            float s = 0.f, dp = 0.f;
+#pragma unroll 8
+            for (int x = 0; x < D; ++x) {
+                s = fmaf(qr[x], kr[x], s);
+                dp = fmaf(dor[x], vr[x], dp);
+            }
+            const size_t row = (size_t)bh * L + (size_t)c * kC + i;
+            pj = __expf(s * scale_sm - lse[row]);
+            ds = pj * (dp - ginv * Dsm[row]);
+        }
+        Ps[i * (kC + 1) + j] = pj;
+        dSs[i * (kC + 1) + j] = ds;
+    }
+    __syncthreads();
+    // thread (row r, column group cg): D / 4 columns cg, cg + 4, ... of dq_r, dk_r, dv_r
+    const int r = threadIdx.x >> 2, cg = threadIdx.x & 3;
+    for (int x = cg; x < D; x += 4) {
+        float aq = 0.f, ak = 0.f, av = 0.f;
+        for (int j = 0; j <= r; ++j) aq = fmaf(dSs[r * (kC + 1) + j], Ks[j * (D + 1) + x], aq);
+        for (int i = r; i < kC; ++i) {
+            ak = fmaf(dSs[i * (kC + 1) + r], Qs[i * (D + 1) + x], ak);
+            av = fmaf(Ps[i * (kC + 1) + r], dOs[i * (D + 1) + x], av);
+        }
+        const size_t dst = tok0 * D + (size_t)r * ts + x;
+        dq_sm[dst] += scale_sm * aq;
+        dk_x[dst] = scale_sm * ak;
+        dv_x[dst] = av;
     }
 }
 
@@ -413,7 +494,10 @@ gdn_rscan_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
                  const float *__restrict__ P, const float *__restrict__ do_la,
                  const float *__restrict__ chunk_states, float scale_la, float *__restrict__ dUt,
                  float *__restrict__ dS_c, float *__restrict__ gS, const float *__restrict__ dstate_out,
-                 float *__restrict__ dstate_in, int L, int H) {
+                 float *__restrict__ dstate_in, const uint8_t *__restrict__ block_route, int L, int H) {
+    // block_route (block-level routing): a softmax block's update was not committed to the state, so
+    // its exit-state gradient reaches the entry state through the decay only: no K~ dS term in dU~, and
+    // the stored chunk-exit gradient (which the dK~ product reads) is zero; <dS1, S0> is not.
     extern __shared__ float smem[];
     float *dSs = smem;                       // [D][32]
     float *Ws = dSs + D * kDvs;              // [64][D+1]
@@ -436,6 +520,7 @@ gdn_rscan_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
 
     for (int c = NC - 1; c >= 0; --c) {
         const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
+        const float commit = block_route && block_route[tok0] ? 0.f : 1.f;
         __syncthreads();
         // store the chunk-exit gradient and the partial <dS1, S0>
         {
@@ -443,7 +528,7 @@ gdn_rscan_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
             for (int idx = threadIdx.x; idx < D * kDvs; idx += kThreads) {
                 const int a = idx / kDvs, cc = idx % kDvs;
                 const size_t gi = (((size_t)bh * NC + c) * D + a) * D + c0 + cc;
-                dS_c[gi] = dSs[idx];
+                dS_c[gi] = commit * dSs[idx];
                 part = fmaf(dSs[idx], chunk_states[gi], part);
             }
             part = warp_sum(part);
@@ -495,7 +580,7 @@ gdn_rscan_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
 #pragma unroll
                 for (int x = 0; x < 8; ++x) acc2[x] = fmaf(kv, sr[x], acc2[x]);
             }
-            const float kt = __expf(gl - Gs[r]);
+            const float kt = commit * __expf(gl - Gs[r]);
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
                 acc[x] = fmaf(kt, acc2[x], acc[x]);
@@ -549,7 +634,7 @@ gdn_tsolve_kernel(const float *__restrict__ Abar, const float *__restrict__ beta
     const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
     if (threadIdx.x < kC) {
         const size_t t = tok0 + (size_t)threadIdx.x * H;
-        bts[threadIdx.x] = route[t] ? 0.f : beta[t];
+        bts[threadIdx.x] = route && route[t] ? 0.f : beta[t];   // route == nullptr: beta~ = beta
     }
     __syncthreads();
     const float *Ab = Abar + ((size_t)bh * (L / kC) + c) * kC * kC;
@@ -586,7 +671,7 @@ mask_scale_kernel(const float *__restrict__ M, const float *__restrict__ N,
     const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
     if (threadIdx.x < kC) {
         const size_t t = ((size_t)b * L + (size_t)c * kC + threadIdx.x) * H + h;
-        bts[threadIdx.x] = route[t] ? 0.f : beta[t];
+        bts[threadIdx.x] = route && route[t] ? 0.f : beta[t];
         Gs[threadIdx.x] = Gcum[(size_t)bh * L + c * kC + threadIdx.x];
     }
     __syncthreads();
@@ -614,7 +699,8 @@ gdn_assemble_kernel(const float *__restrict__ q32, const float *__restrict__ k32
                     const float *__restrict__ dVb, const float *__restrict__ dKt,
                     const float *__restrict__ X1p, const float *__restrict__ X2,
                     const float *__restrict__ X3, const float *__restrict__ X4,
-                    const float *__restrict__ dq_sm, float scale_la, T *__restrict__ dq,
+                    const float *__restrict__ dq_sm, const float *__restrict__ dk_x,
+                    const float *__restrict__ dv_x, float scale_la, T *__restrict__ dq,
                     T *__restrict__ dk, T *__restrict__ dv, float *__restrict__ dGrow,
                     float *__restrict__ kappa, float *__restrict__ dbeta, int B, int L, int H) {
     constexpr int kCols = D / 32;
@@ -626,7 +712,9 @@ gdn_assemble_kernel(const float *__restrict__ q32, const float *__restrict__ k32
     const int l = bl % L, b = bl / L;
     const size_t bhl = ((size_t)b * H + h) * L;
     const float Gi = Gcum[bhl + l], GC = Gcum[bhl + (l | (kC - 1))];
-    const bool lin = route[row] == 0;
+    // route == nullptr (block-level routing): every token takes part in the delta rule, and every
+    // token's dk, dv also has a softmax-branch part, given in dk_x, dv_x (fp32, token-major)
+    const bool lin = !route || route[row] == 0;
     const float bt = lin ? beta[row] : 0.f;
     const float gam = __expf(Gi), kt = __expf(GC - Gi);
     float kdKb = 0.f, qdQg = 0.f, kdKt = 0.f, kX1 = 0.f, kX2 = 0.f, qX3 = 0.f, kX4 = 0.f, vdVb = 0.f;
@@ -641,8 +729,8 @@ gdn_assemble_kernel(const float *__restrict__ q32, const float *__restrict__ k32
         kX4 = fmaf(kv, x4, kX4); vdVb = fmaf(vv, a_dVb, vdVb);
         dq[i] = from_f32<T>(scale_la * gam * a_dQg + x3 + dq_sm[i]);
         if (lin) {
-            dk[i] = from_f32<T>(bt * gam * a_dKb + kt * a_dKt + bt * x1 + x2 + x4);
-            dv[i] = from_f32<T>(bt * a_dVb);
+            dk[i] = from_f32<T>(bt * gam * a_dKb + kt * a_dKt + bt * x1 + x2 + x4 + (dk_x ? dk_x[i] : 0.f));
+            dv[i] = from_f32<T>(bt * a_dVb + (dv_x ? dv_x[i] : 0.f));
         }
     }
     kdKb = warp_sum(kdKb); qdQg = warp_sum(qdQg); kdKt = warp_sum(kdKt); kX1 = warp_sum(kX1);
@@ -781,7 +869,7 @@ static cudaError_t softmax_bwd_impl(const float *q32, const float *k_sm32, const
                                     int cap, const int32_t *sm_idx, const int32_t *pre,
                                     const float *do_nla, const float *lse, const float *Dsm,
                                     float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
-                                    Shape s, cudaStream_t st) {
+                                    float *dmask, Shape s, cudaStream_t st) {
     const size_t smem_q = sizeof(float) * (2 * kC * D + 2 * 32 * (D + 1) + 32);
     const size_t smem_k = sizeof(float) * (2 * 32 * (D + 1) + 2 * kC * D + 2 * kC * 33 + 2 * kC + 32);
     cudaError_t e = set_smem(softmax_bwd_dq_kernel<D>, smem_q);
@@ -795,7 +883,7 @@ static cudaError_t softmax_bwd_impl(const float *q32, const float *k_sm32, const
     dim3 gk((cap + 31) / 32, s.B * s.H);
     softmax_bwd_dkv_kernel<D><<<gk, kThreads, smem_k, st>>>(q32, k_sm32, v_sm32, cap, sm_idx, pre,
                                                             do_nla, lse, Dsm, scale_sm, dk_sm, dv_sm,
-                                                            s.L, s.H);
+                                                            dmask, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -804,23 +892,49 @@ cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const floa
                                const int32_t *sm_idx, const int32_t *sm_chunk_prefix,
                                const float *do_nla, const float *lse, const float *Dsm,
                                float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm, Shape s,
-                               cudaStream_t st) {
-    if (s.d == 128) return softmax_bwd_impl<128>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, scale_sm, dq_sm, dk_sm, dv_sm, s, st);
-    return softmax_bwd_impl<64>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, scale_sm, dq_sm, dk_sm, dv_sm, s, st);
+                               cudaStream_t st, float *dmask) {
+    if (s.d == 128) return softmax_bwd_impl<128>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, scale_sm, dq_sm, dk_sm, dv_sm, dmask, s, st);
+    return softmax_bwd_impl<64>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, scale_sm, dq_sm, dk_sm, dv_sm, dmask, s, st);
+}
+
+template <int D>
+static cudaError_t own_block_impl(const float *q32, const float *k32, const float *v32, const float *do_nla,
+                                  const float *lse, const float *Dsm, const uint8_t *route, float scale_sm,
+                                  float *dq_sm, float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
+                                  cudaStream_t st) {
+    const size_t smem = sizeof(float) * (4 * kC * (D + 1) + 2 * kC * (kC + 1));
+    cudaError_t e = set_smem(softmax_bwd_own_block_simt_kernel<D>, smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid(s.L / kC, s.B * s.H);
+    softmax_bwd_own_block_simt_kernel<D><<<grid, kThreads, smem, st>>>(q32, k32, v32, do_nla, lse, Dsm, route,
+                                                                      scale_sm, dq_sm, dk_x, dv_x, gsc, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_bwd_own_block_simt(const float *q32, const float *k32, const float *v32,
+                                              const float *do_nla, const float *lse, const float *Dsm,
+                                              const uint8_t *route, float scale_sm, float *dq_sm,
+                                              float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
+                                              cudaStream_t st) {
+    if (s.d == 128) return own_block_impl<128>(q32, k32, v32, do_nla, lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, gsc, s, st);
+    return own_block_impl<64>(q32, k32, v32, do_nla, lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, gsc, s, st);
 }
 
 template <int D>
 static cudaError_t rscan_impl(const float *q32, const float *k32, const float *Gcum, const float *W,
                               const float *P, const float *do_la, const float *chunk_states,
                               float scale_la, float *dUt, float *dS_c, float *gS,
-                              const float *dstate_out, float *dstate_in, Shape s, cudaStream_t st) {
+                              const float *dstate_out, float *dstate_in, const uint8_t *block_route, Shape s,
+                              cudaStream_t st) {
     const size_t smem = sizeof(float) * (D * kDvs + 3 * kC * (D + 1) + kC * (kC + 1) +
                                          2 * kC * (kDvs + 1) + kC + 8);
     cudaError_t e = set_smem(gdn_rscan_kernel<D>, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(D / kDvs, s.B * s.H);
     gdn_rscan_kernel<D><<<grid, kThreads, smem, st>>>(q32, k32, Gcum, W, P, do_la, chunk_states,
-                                                      scale_la, dUt, dS_c, gS, dstate_out, dstate_in, s.L, s.H);
+                                                      scale_la, dUt, dS_c, gS, dstate_out, dstate_in, block_route,
+                                                      s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -828,10 +942,11 @@ static cudaError_t rscan_impl(const float *q32, const float *k32, const float *G
 cudaError_t launch_gdn_rscan(const float *q32, const float *k32, const float *Gcum, const float *W,
                              const float *P, const float *do_la, const float *chunk_states,
                              float scale_la, float *dUt, float *dS_c, float *gS,
-                             const float *dstate_out, float *dstate_in, Shape s, cudaStream_t st) {
+                             const float *dstate_out, float *dstate_in, Shape s, cudaStream_t st,
+                             const uint8_t *block_route) {
     if (s.d == 128)
-        return rscan_impl<128>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, dstate_out, dstate_in, s, st);
-    return rscan_impl<64>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, dstate_out, dstate_in, s, st);
+        return rscan_impl<128>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, dstate_out, dstate_in, block_route, s, st);
+    return rscan_impl<64>(q32, k32, Gcum, W, P, do_la, chunk_states, scale_la, dUt, dS_c, gS, dstate_out, dstate_in, block_route, s, st);
 }
 
 cudaError_t launch_gdn_tsolve(const float *Abar, const float *beta, const uint8_t *route,
@@ -861,13 +976,15 @@ static cudaError_t assemble_impl(const AssembleArgs &a, void *dq, void *dk, void
     const size_t rows = (size_t)s.B * s.L * s.H;
     gdn_assemble_kernel<T, D><<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
         a.q32, a.k32, a.v32, a.Gcum, a.beta, a.route, a.dQg, a.dKb, a.dVb, a.dKt, a.X1p, a.X2, a.X3,
-        a.X4, a.dq_sm, a.scale_la, (T *)dq, (T *)dk, (T *)dv, a.dGrow, a.kappa, a.dbeta, s.B, s.L, s.H);
+        a.X4, a.dq_sm, a.dk_x, a.dv_x, a.scale_la, (T *)dq, (T *)dk, (T *)dv, a.dGrow, a.kappa, a.dbeta, s.B,
+        s.L, s.H);
     count_launch();
     const int NC = s.L / kC;
     const size_t nch = (size_t)s.B * s.H * NC;
     dg_kernel<<<(unsigned)((nch + 127) / 128), 128, 0, st>>>(a.dGrow, a.kappa, a.gS, a.Gcum,
                                                             s.d / kDvs, a.dg, s.B, s.L, s.H);
     count_launch();
+    if (a.dk_x) return cudaGetLastError();   // (the retained tokens' gradients came in through dk_x, dv_x)
     constexpr int kRows = kThreads / (D / 4);
     dim3 grid((a.cap + kRows - 1) / kRows, s.B * s.H);
     scatter_sm_kernel<T, D><<<grid, kThreads, 0, st>>>(a.dk_sm, a.dv_sm, a.cap, a.sm_idx, a.sm_prefix,

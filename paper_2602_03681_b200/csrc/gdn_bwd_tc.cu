@@ -261,12 +261,14 @@ gdn_rscan_tc_kernel(const __grid_constant__ CUtensorMap map_do,    // dO (fp16) 
 }
 
 // gS[chunk] = <dS1[chunk], S0[chunk]> (first slot of the row; the other slots are zeroed).
+// Block-level routing (block_route given): the exit-state gradient of a softmax block, whose update
+// was not committed, is then cleared, so that the dK~ product that reads it next yields zero.
 __global__ void __launch_bounds__(256)
-state_dot_kernel(const float *__restrict__ dS_c, const float *__restrict__ S_c, float *__restrict__ gS,
-                 int n_slices, int dd) {
+state_dot_kernel(float *__restrict__ dS_c, const float *__restrict__ S_c, float *__restrict__ gS,
+                 int n_slices, int dd, const uint8_t *__restrict__ block_route, int L, int H) {
     __shared__ float red[8];
     const size_t chunk = blockIdx.x;
-    const float4 *a = reinterpret_cast<const float4 *>(dS_c + chunk * dd);
+    float4 *a = reinterpret_cast<float4 *>(dS_c + chunk * dd);
     const float4 *bq = reinterpret_cast<const float4 *>(S_c + chunk * dd);
     float acc = 0.f;
     for (int i = threadIdx.x; i < dd / 4; i += 256) {
@@ -281,6 +283,13 @@ state_dot_kernel(const float *__restrict__ dS_c, const float *__restrict__ S_c, 
         for (int wv = 0; wv < 8; ++wv) t += red[wv];
         gS[chunk * n_slices] = t;
         for (int sl = 1; sl < n_slices; ++sl) gS[chunk * n_slices + sl] = 0.f;
+    }
+    if (block_route) {
+        const int NC = L / kC;
+        const size_t bh = chunk / NC;
+        const int c = (int)(chunk % NC), b = (int)(bh / H), h = (int)(bh % H);
+        if (block_route[((size_t)b * L + (size_t)c * kC) * H + h])       // (every thread has read its part above)
+            for (int i = threadIdx.x; i < dd / 4; i += 256) a[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
 }
 
@@ -838,7 +847,7 @@ static cudaError_t rscan_tc_impl(const void *dO16, const void *dOg16, const GdnT
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if (gS) {     // (the fused chunk kernel forms <dS1, S0> itself)
-        state_dot_kernel<<<(unsigned)(BH * NC), 256, 0, st>>>(dS_c, S_c, gS, D / 32, D * D);
+        state_dot_kernel<<<(unsigned)(BH * NC), 256, 0, st>>>(dS_c, S_c, gS, D / 32, D * D, block_route, s.L, s.H);
         count_launch();
     }
     return cudaGetLastError();
@@ -881,8 +890,8 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
 namespace {
 __global__ void __launch_bounds__(64)
 dscore_kernel(const uint8_t *__restrict__ route, const int32_t *__restrict__ sm_chunk_prefix,
-              const float *__restrict__ dmask, const float *__restrict__ kap_c, int cap,
-              float *__restrict__ dscore, int L, int H) {
+              const float *__restrict__ dmask, const float *__restrict__ kap_c,
+              const float *__restrict__ kappa_tok, int cap, float *__restrict__ dscore, int L, int H) {
     const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H, NC = L / kC;
     float *dst = dscore + (((size_t)b * NC + c) * H + h) * 2;
     if (route[((size_t)b * L + (size_t)c * kC) * H + h]) {
@@ -893,6 +902,12 @@ dscore_kernel(const uint8_t *__restrict__ route, const int32_t *__restrict__ sm_
         if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = x;
         __syncthreads();
         if (threadIdx.x == 0) { dst[0] = 0.f; dst[1] = part[0] + part[1]; }
+    } else if (kappa_tok) {
+        float x = warp_sum(kappa_tok[(size_t)bh * L + (size_t)c * kC + threadIdx.x]);
+        __shared__ float part2[2];
+        if ((threadIdx.x & 31) == 0) part2[threadIdx.x >> 5] = x;
+        __syncthreads();
+        if (threadIdx.x == 0) { dst[0] = part2[0] + part2[1]; dst[1] = 0.f; }
     } else if (threadIdx.x == 0) {
         dst[0] = kap_c[(size_t)bh * NC + c];
         dst[1] = 0.f;
@@ -901,9 +916,10 @@ dscore_kernel(const uint8_t *__restrict__ route, const int32_t *__restrict__ sm_
 }  // namespace
 
 cudaError_t launch_dscore(const uint8_t *route, const int32_t *sm_chunk_prefix, const float *dmask,
-                          const float *kap_c, int cap, float *dscore, Shape s, cudaStream_t st) {
+                          const float *kap_c, const float *kappa_tok, int cap, float *dscore, Shape s,
+                          cudaStream_t st) {
     dim3 grid(s.L / kC, s.B * s.H);
-    dscore_kernel<<<grid, 64, 0, st>>>(route, sm_chunk_prefix, dmask, kap_c, cap, dscore, s.L, s.H);
+    dscore_kernel<<<grid, 64, 0, st>>>(route, sm_chunk_prefix, dmask, kap_c, kappa_tok, cap, dscore, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }

@@ -195,13 +195,23 @@ cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const floa
                                const int32_t *sm_idx, const int32_t *sm_chunk_prefix,
                                const float *do_nla, const float *lse, const float *Dsm,
                                float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm, Shape s,
-                               cudaStream_t st);
+                               cudaStream_t st, float *dmask = nullptr);
+// (dmask [B,H,cap] or nullptr: per retained key the sum of the mask gradients of Section 4.2)
+// Block-level routing, fp32: the softmax branch's backward through the own block of the queries of a
+// linear block (adds to dq_sm, writes the dk_x / dv_x rows of the linear blocks).  gsc: gradient
+// scale of the tensor-core kernels that Dsm carries (nullptr: none).
+cudaError_t launch_softmax_bwd_own_block_simt(const float *q32, const float *k32, const float *v32,
+                                              const float *do_nla, const float *lse, const float *Dsm,
+                                              const uint8_t *route, float scale_sm, float *dq_sm,
+                                              float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
+                                              cudaStream_t st);
 // dstate_out [B,H,d,d] (or nullptr: zero): the gradient the scan starts from, at the final state;
 // dstate_in (or nullptr): receives what is left after the first chunk, the initial state's gradient.
 cudaError_t launch_gdn_rscan(const float *q32, const float *k32, const float *Gcum, const float *W,
                              const float *P, const float *do_la, const float *chunk_states,
                              float scale_la, float *dUt, float *dS_c, float *gS,
-                             const float *dstate_out, float *dstate_in, Shape s, cudaStream_t st);
+                             const float *dstate_out, float *dstate_in, Shape s, cudaStream_t st,
+                             const uint8_t *block_route = nullptr);
 // Tensor-core reverse scan (gdn_bwd_tc.cu): dO16 / dOg16 are fp16 [B,H,L,d] copies of the read-out
 // gradient and of scale_la gamma times it; outputs as launch_gdn_rscan (gS: slot 0 of each row).
 cudaError_t launch_gdn_rscan_tc(const void *dO16, const void *dOg16, const GdnTcWs &ws,
@@ -222,6 +232,9 @@ struct AssembleArgs {
     int cap;
     float scale_la;
     float *dGrow, *kappa, *dbeta, *dg;
+    // block-level routing on the path with separate chunk-level products: route == nullptr (every token
+    // takes part in the delta rule) and the softmax-branch dk, dv of every token, fp32 token-major
+    const float *dk_x = nullptr, *dv_x = nullptr;
 };
 // dq (all tokens), dk/dv (linear tokens from the GDN branch, retained tokens scattered from the
 // compacted softmax-branch gradients), dbeta, dg.  Three kernels.
@@ -240,8 +253,10 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
                                  float scale_la, void *dq, void *dk, void *dv, float *dg,
                                  float *dbeta, bool block, const float *dk_x, const float *dv_x,
                                  float *kap_c, Shape s, cudaStream_t st);
+// (kap_c [B,H,L/C]: the chunk sums of kappa, or kappa_tok [B,H,L]: kappa per token, summed here)
 cudaError_t launch_dscore(const uint8_t *route, const int32_t *sm_chunk_prefix, const float *dmask,
-                          const float *kap_c, int cap, float *dscore, Shape s, cudaStream_t st);
+                          const float *kap_c, const float *kappa_tok, int cap, float *dscore, Shape s,
+                          cudaStream_t st);
 
 // block-level routing: softmax-branch backward through the own block of the queries of a linear
 // block (adds to dq_sm, writes the dk_x / dv_x rows of the linear blocks); do16: fp16 [B,H,L,d]

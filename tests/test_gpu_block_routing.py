@@ -193,58 +193,88 @@ def test_block_end_without_the_blocks_entries_is_reported():
 
 
 # ------------------------------------------------------------------ backward
-@pytest.mark.parametrize("B,H,L,p", [(1, 2, 256, 0.4), (2, 3, 512, 0.25), (1, 1, 64, 0.0), (1, 2, 192, 1.0)])
-def test_block_routed_backward_matches_oracle(B, H, L, p):
-    """Backward under block-level routing (bf16 storage, d = 64: the path with the fused chunk
-    kernel) against the oracle's block-mode backward."""
+BWD_PATHS = {     # workload, flags, tolerance
+    "fused_d64": ("cfg4_bf16_train", 0, TOL_BF16),          # tensor cores, one fused kernel per chunk
+    "tc_d128": ("cfg1_bf16_prefill", 0, TOL_BF16),          # tensor cores, chunk-level products as tile GEMMs
+    "f32_d64": ("cfg0_f32_tiny_fwd", 0, 1e-4),              # fp32 storage, CUDA cores
+    "bf16_simt": ("cfg4_bf16_train", 1, 2e-4),              # fp32 arithmetic on bf16 storage (FORCE_SIMT)
+}
+
+
+@pytest.mark.parametrize("path,B,H,L,p", [
+    ("fused_d64", 1, 2, 256, 0.4), ("fused_d64", 2, 3, 512, 0.25), ("fused_d64", 1, 1, 64, 0.0),
+    ("fused_d64", 1, 2, 192, 1.0),
+    ("tc_d128", 1, 2, 256, 0.4), ("tc_d128", 2, 2, 320, 0.25), ("tc_d128", 1, 1, 128, 0.0), ("tc_d128", 1, 1, 128, 1.0),
+    ("f32_d64", 1, 2, 256, 0.4), ("f32_d64", 2, 1, 192, 0.6), ("f32_d64", 1, 1, 128, 0.0), ("f32_d64", 1, 1, 128, 1.0),
+    ("bf16_simt", 1, 2, 192, 0.4),
+])
+def test_block_routed_backward_matches_oracle(path, B, H, L, p):
+    """Backward under block-level routing against the oracle's block-mode backward, on every path."""
     from paper_2602_03681_b200 import binding
     from test_gpu_parity import check_bwd, run_bwd
-    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+    name, flags, tol = BWD_PATHS[path]
+    wl = inputs.WORKLOADS[name]
     x = block_inputs(wl, B, H, L, p)
     if p in (0.0, 1.0):
         x["route"][:] = int(p)
     ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
                             scale_la=wl.scale_la, scale_sm=wl.scale_sm, block=64)
-    got = run_bwd(wl, x, flags=binding.BLOCK_ROUTING)
-    check_bwd(wl, got, ref, TOL_BF16)
+    got = run_bwd(wl, x, flags=binding.BLOCK_ROUTING | flags)
+    check_bwd(wl, got, ref, tol)
     tok = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
                             scale_la=wl.scale_la, scale_sm=wl.scale_sm)
     if 0 < p < 1:       # the mode differs visibly from token-level routing on the same inputs
         assert rel_err(tok["dk"], ref["dk"]) > 10 * TOL_BF16
 
 
-def test_block_routed_backward_other_shapes_are_refused():
+def test_block_routed_backward_fp32_d128_with_states():
+    """fp32 storage at d = 128, with an initial state, a gradient at the final state and the gradient of
+    the initial state."""
+    import dataclasses
     from paper_2602_03681_b200 import binding
-    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]           # d = 128
-    x = block_inputs(wl, 1, 1, 128, 0.5)
-    dt = tdtype(wl)
-    with pytest.raises(binding.NatslError) as e:
-        binding.hybrid_bwd(*(dev(x[m], dt) for m in ("q", "k", "v")), dev(x["g"]), dev(x["beta"]),
-                           dev(x["route"]), dev(x["w"]), dev(x["dout"], dt), scale_la=wl.scale_la,
-                           scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING)
-    assert e.value.status == binding.ERR_UNSUPPORTED
+    from test_gpu_parity import check_bwd
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg0_f32_tiny_fwd"], d=128, seed=17)
+    B, H, L = 1, 2, 192
+    x = block_inputs(wl, B, H, L, 0.4)
+    r = np.random.default_rng(4)
+    s0 = (0.1 * r.standard_normal((B, H, 128, 128))).astype(np.float32)
+    ds = (0.05 * r.standard_normal((B, H, 128, 128))).astype(np.float32)
+    ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                            scale_la=wl.scale_la, scale_sm=wl.scale_sm, block=64, state_in=s0, dstate_out=ds)
+    res = binding.hybrid_bwd(*(dev(x[m]) for m in ("q", "k", "v")), dev(x["g"]), dev(x["beta"]),
+                             dev(x["route"]), dev(x["w"]), dev(x["dout"]), scale_la=wl.scale_la,
+                             scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING, state_in=dev(s0),
+                             dstate_out=dev(ds), want_dstate_in=True)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(res["ws"]) == 0
+    got = {n: t.float().cpu().numpy() for n, t in res.items() if n != "ws"}
+    check_bwd(wl, got, ref, 1e-4)
+    assert rel_err(got["dstate_in"], ref["dstate_in"]) <= 1e-4
 
 
-@pytest.mark.parametrize("B,H,L,p", [(1, 2, 256, 0.4), (2, 3, 512, 0.25)])
-def test_block_routed_backward_score_gradients(B, H, L, p):
+@pytest.mark.parametrize("path,B,H,L,p", [("fused_d64", 1, 2, 256, 0.4), ("fused_d64", 2, 3, 512, 0.25),
+                                          ("tc_d128", 1, 2, 320, 0.4), ("f32_d64", 2, 2, 256, 0.4),
+                                          ("bf16_simt", 1, 2, 192, 0.4)])
+def test_block_routed_backward_score_gradients(path, B, H, L, p):
     """d score per block and head (Section 4.2) against the oracle: nonzero only for the operation
     the block chose."""
     from paper_2602_03681_b200 import binding
-    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+    name, flags, tol = BWD_PATHS[path]
+    wl = inputs.WORKLOADS[name]
     x = block_inputs(wl, B, H, L, p)
     ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
                             scale_la=wl.scale_la, scale_sm=wl.scale_sm, block=64)["dscore"]
     dt = tdtype(wl)
     res = binding.hybrid_bwd(*(dev(x[m], dt) for m in ("q", "k", "v")), dev(x["g"]), dev(x["beta"]),
                              dev(x["route"]), dev(x["w"]), dev(x["dout"], dt), scale_la=wl.scale_la,
-                             scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING, want_dscore=True)
+                             scale_sm=wl.scale_sm, flags=binding.BLOCK_ROUTING | flags, want_dscore=True)
     torch.cuda.synchronize()
     assert binding.natsl_device_status(res["ws"]) == 0
     got = res["dscore"].cpu().numpy()
     blocks = x["route"][:, ::64]                                   # [B, L/64, H]
     assert np.all(got[..., 0][blocks == 1] == 0) and np.all(got[..., 1][blocks == 0] == 0)
     for op in (0, 1):
-        assert rel_err(got[..., op], ref[..., op]) <= TOL_BF16, (op, rel_err(got[..., op], ref[..., op]))
+        assert rel_err(got[..., op], ref[..., op]) <= tol, (op, rel_err(got[..., op], ref[..., op]))
     assert np.abs(ref[..., 1]).max() > 0 and np.abs(ref[..., 0]).max() > 0
 
 

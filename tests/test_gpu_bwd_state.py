@@ -57,6 +57,8 @@ def test_bwd_through_initial_and_final_state(name, B, H, L, flags, tol):
 
 @pytest.mark.parametrize("name,B,H,L,block", [("cfg4_bf16_train", 2, 3, 448, False),
                                               ("cfg4_bf16_train", 1, 2, 256, True),
+                                              ("cfg1_bf16_prefill", 1, 2, 256, True),
+                                              ("cfg0_f32_tiny_fwd", 1, 2, 192, True),
                                               ("cfg1_bf16_prefill", 1, 2, 256, False),
                                               ("cfg0_f32_tiny_fwd", 1, 2, 128, False)])
 def test_saved_forward_then_backward(name, B, H, L, block):
