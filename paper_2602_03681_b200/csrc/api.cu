@@ -63,8 +63,8 @@ HeadGroups head_groups(const natsl_params *p) {
 Shape shape_of(const natsl_params *p) { return Shape{p->B, p->H, p->L, p->d, p->dtype == NATSL_BF16}; }
 
 struct FwdWs {
-    int32_t *status, *emit_flags, *ready_flags, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
-    size_t head_bytes;          // status page + the two sets of counters: cleared at the start of every call
+    int32_t *status, *emit_flags, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
+    size_t head_bytes;          // status page + emit_flags: cleared at the start of every call
     void *k_sm, *v_sm, *v16;
     void *o_la16;               // tensor-core path: the linear read-out as fp16 [B,L,H,d]
     float *W, *U, *P, *o_la;    // fp32 CUDA-core path only
@@ -96,8 +96,6 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
     f.status = c.take<int32_t>(kStatusBytes / 4);
     // one counter per chunk, raised by the scan as the chunk's read-out is complete (tensor-core path)
     f.emit_flags = c.take<int32_t>(use_tensor_cores(p) ? B * H * NC : 0);
-    // one counter per chunk, raised by the part of the prepare kernel that runs beside the scan
-    f.ready_flags = c.take<int32_t>(use_tensor_cores(p) ? B * H * NC : 0);
     f.head_bytes = c.off;
     f.sm_idx = c.take<int32_t>(B * H * L);
     f.prefix = c.take<int32_t>(B * H * (NC + 1));
@@ -339,7 +337,7 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
         const GdnTcExport ex{fused_chunks ? nullptr : f.W, fused_chunks ? nullptr : f.U, nullptr, f.Tinv,
                              f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc, ex,
-                                        f.status, PrepRange{0, 0, nullptr, false}, s, st));
+                                        f.status, s, st));
         // (the side stream joins before the scan, so that the softmax kernel follows the scan directly
         // and can run beside it as its programmatic dependent, as in natsl_hybrid_fwd)
         NATSL_TRY(side_join.join());
@@ -526,24 +524,10 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(mark());
     if (tensor_cores) {
         // block-level routing: every token takes part in the delta rule of its own block
-        // With fewer (batch, head) pairs than multiprocessors the scan, one CTA per pair, leaves the
-        // rest of the device idle.  The prepare kernel then runs in two parts: the first chunks of
-        // every sequence before the scan, the others beside it, launched behind the scan as its
-        // programmatic dependent (all CTAs of the scan are resident by then, and this part waits for
-        // nothing, so neither can starve the other) and published per chunk through counters the
-        // scan's loader waits for.  The share that runs late is what the free multiprocessors finish
-        // in step with the scan, less a tenth.
         const bool beside = !p->stage_events && !(p->flags & NATSL_SINGLE_STREAM);
         const int nseg = scan_segments(p);
-        const int NCi = (int)(p->L / kC), BHi = p->B * p->H, sms = sm_count();
-        int n_late = 0;
-        if (beside && nseg == 1 && BHi < sms && !g_debug_withhold_flags.load(std::memory_order_relaxed)) {
-            n_late = (int)((long long)NCi * (sms - BHi) * 9 / ((long long)sms * 10));
-            if (n_late < 4 || NCi - n_late < 4) n_late = 0;
-        }
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc,
-                                        GdnTcExport{}, f.status,
-                                        PrepRange{0, NCi - n_late, nullptr, false, hg.norm_eps}, s, st));
+                                        GdnTcExport{}, f.status, s, st, hg.norm_eps));
         NATSL_TRY(mark());
         // The side stream joins here, before the scan, so that nothing stands between the scan and
         // the softmax kernel in the stream: the softmax kernel is launched as a programmatic dependent
@@ -554,8 +538,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(side_join.join());
         int32_t *flags_scan = beside && !g_debug_withhold_flags.load(std::memory_order_relaxed) ? f.emit_flags : nullptr;
         const int32_t *flags_softmax = beside ? f.emit_flags : nullptr;
-        ScanOut so{f.o_la16, p->o_la, flags_scan};
-        if (n_late) { so.ready_flags = f.ready_flags; so.ready_from = NCi - n_late; }
+        const ScanOut so{f.o_la16, p->o_la, flags_scan};
         if (nseg > 1) {   // few (batch, head) pairs: segments in parallel, chained by their transitions
             ScanSegments sg{1, nseg, (int)(p->L / kC) / nseg, f.seg_incr, f.seg_trans, f.seg_start};
             NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, nullptr, nullptr, so, GdnTcExport{}, sg,
@@ -568,11 +551,6 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
             NATSL_TRY(launch_gdn_scan_tc(f.tc, p->scale_la, p->state_in, p->state_out, so, GdnTcExport{},
                                          ScanSegments{0, 1, 0, nullptr, nullptr, nullptr}, br.route,
                                          f.status, s, st));
-            if (n_late)
-                NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc,
-                                                GdnTcExport{}, f.status,
-                                                PrepRange{NCi - n_late, n_late, f.ready_flags, true, hg.norm_eps},
-                                                s, st));
         }
         NATSL_TRY(mark());
         NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, capv, f.sm_idx, f.prefix, f.o_la16,

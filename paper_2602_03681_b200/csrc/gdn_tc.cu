@@ -86,12 +86,8 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                       const float *__restrict__ beta, const uint8_t *__restrict__ route,
                       float scale_la, __half *__restrict__ Wt, float *__restrict__ Ut,
                       __half *__restrict__ Ph, float *__restrict__ Gd, GdnTcExport ex,
-                      int32_t *status, int L, int H, int c_begin, int n_range, int32_t *ready_flags,
-                      float norm_eps, int wait_kcycles) {
+                      int32_t *status, int L, int H, float norm_eps, int wait_kcycles) {
     using PL = PrepLayout<D>;
-    // (a kernel launched behind this one as a programmatic dependent may start once every CTA of
-    // this grid is resident; see the launch of the second part)
-    launch_dependents();
     constexpr int KB = PL::KB;
     extern __shared__ __align__(1024) uint8_t smem[];
     PrepMisc &ms = *reinterpret_cast<PrepMisc *>(smem + PL::oMisc);
@@ -99,12 +95,7 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     const int NC = L / kC;
     // (chunk fastest: a head-fastest order, whole rows of [B,L,H,d] read by neighbouring CTAs, and L2
     // prefetches of the next wave's tiles were both measured slower)
-    // The grid covers the chunks [c_begin, c_begin + n_range) of every (batch, head).  A part that
-    // runs beside the scan (ready_flags given) goes chunk by chunk, all (batch, head) pairs of a chunk
-    // before the next chunk, which is the order the scan consumes them in.
-    const int BHn = (int)(gridDim.x / n_range);
-    const int c = c_begin + (ready_flags ? (int)(blockIdx.x / BHn) : (int)(blockIdx.x % n_range));
-    const int bh = ready_flags ? (int)(blockIdx.x % BHn) : (int)(blockIdx.x / n_range), b = bh / H, h = bh % H;
+    const int c = (int)(blockIdx.x % NC), bh = (int)(blockIdx.x / NC), b = bh / H, h = bh % H;
     const int tok0 = c * kC;
     const size_t chunk = (size_t)bh * NC + c;
 
@@ -519,14 +510,6 @@ gdn_prepare_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     }
     tc_fence_before_sync();
     __syncthreads();
-    // The chunk's operands are complete: every thread's stores precede the barrier, and the thread
-    // that issued the bulk stores of the q, k copies has waited for them.  That thread publishes the
-    // chunk for a scan running beside this kernel.
-    if (ready_flags && tid == 4 * 32 && !ms.abort_flag) {
-        fence_proxy_async_all();
-        __threadfence();
-        red_release_add(ready_flags + chunk, 1);
-    }
     if (warp == 4) {
         tc_fence_after_sync();
         tmem_dealloc(tmem, 128);
@@ -600,7 +583,7 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
                    const float *__restrict__ Gd, float scale_la,
                    const float *__restrict__ state_in, float *__restrict__ state_out,
                    __half *__restrict__ o_la16, float *__restrict__ o_la32, int32_t *emit_flags,
-                   const int32_t *ready_flags, int ready_from, GdnTcExport ex, ScanSegments sg,
+                   GdnTcExport ex, ScanSegments sg,
                    const uint8_t *__restrict__ block_route, int32_t *status, int L, int H, int wait_kcycles) {
     using SL = ScanLayout<D>;
     // A kernel launched behind this one as a programmatic dependent (the softmax branch) may start
@@ -650,12 +633,6 @@ gdn_scan_tc_kernel(const __grid_constant__ CUtensorMap map_wt,
             for (; c < ncs; ++c) {
                 const int s = c % kScanStages;
                 if (!mbar_wait(&ms.empty[s], ((c / kScanStages) & 1) ^ 1, abort_flag)) break;
-                // chunks the prepare kernel's second part produces while this kernel runs: wait
-                // (bounded) for the chunk's counter, then let the async proxy see what it covers
-                if (ready_flags && c0 + c >= ready_from) {
-                    if (!wait_counter_ge(ready_flags + (size_t)bh * NC + c0 + c, 1, abort_flag)) break;
-                    fence_proxy_async_all();
-                }
                 uint8_t *st = smem + s * SL::kStage;
                 mbar_arrive_expect_tx(&ms.full[s], SL::kTx);
                 tma_load_2d(st + SL::oW, &map_wt, &ms.full[s], 0, (bh * NC + c0 + c) * D);
@@ -1022,10 +999,9 @@ template <int D>
 static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, const float *g,
                                    const float *beta, const uint8_t *route, float scale_la,
                                    const GdnTcWs &ws, const GdnTcExport &ex, int32_t *status,
-                                   const PrepRange &pr, Shape s, cudaStream_t st) {
+                                   float norm_eps, Shape s, cudaStream_t st) {
     const int NC = s.L / kC;
     const uint64_t BH = (uint64_t)s.B * s.H;
-    const int c_begin = pr.n_chunks > 0 ? pr.c_begin : 0, n_range = pr.n_chunks > 0 ? pr.n_chunks : NC;
     CUtensorMap mq, mk, mv, mqh, mkh;
     if (!tch::make_map_blhd(&mq, q, s.B, s.L, s.H, D, 64) ||
         !tch::make_map_blhd(&mk, k, s.B, s.L, s.H, D, 64) ||
@@ -1033,25 +1009,16 @@ static cudaError_t prepare_tc_impl(const void *q, const void *k, const void *v, 
         !tch::make_map_2d(&mqh, ws.Qh, BH * s.L, D, 64) ||
         !tch::make_map_2d(&mkh, ws.Kh, BH * s.L, D, 64))
         return cudaErrorInvalidValue;
-    auto kernel = gdn_prepare_tc_kernel<D>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gdn_prepare_tc_kernel<D>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          PrepLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)n_range * (unsigned)BH);
-    cfg.blockDim = dim3(kPrepThreads);
-    cfg.dynamicSmemBytes = PrepLayout<D>::kTotal;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = pr.beside_previous ? 1 : 0;    // a part that runs beside the kernel launched before it
-    e = cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut,
-                           (__half *)ws.Ph, ws.Gd, ex, status, s.L, s.H, c_begin, n_range, pr.ready_flags,
-                           pr.norm_eps, debug_wait_kcycles());
+    dim3 grid((unsigned)NC * (unsigned)BH);
+    gdn_prepare_tc_kernel<D><<<grid, kPrepThreads, PrepLayout<D>::kTotal, st>>>(
+        mq, mk, mv, mqh, mkh, g, beta, route, scale_la, (__half *)ws.Wt, ws.Ut, (__half *)ws.Ph, ws.Gd, ex,
+        status, s.L, s.H, norm_eps, debug_wait_kcycles());
     count_launch();
-    return e;
+    return cudaGetLastError();
 }
 
 template <int D>
@@ -1074,17 +1041,17 @@ static cudaError_t scan_tc_impl(const GdnTcWs &ws, float scale_la, const float *
     const int ctas = s.B * s.H * (sg.mode == 0 ? 1 : sg.nseg) * (sg.mode == 1 ? 2 : 1);
     kernel<<<ctas, kScanThreads, ScanLayout<D>::kTotal, st>>>(
         mwt, mqh, mkh, mph, ws.Ut, ws.Gd, scale_la, state_in, state_out, (__half *)out.o_la16, out.o_la32,
-        out.emit_flags, out.ready_flags, out.ready_from, ex, sg, block_route, status, s.L, s.H, debug_wait_kcycles());
+        out.emit_flags, ex, sg, block_route, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, const float *g,
                                   const float *beta, const uint8_t *route, float scale_la,
-                                  const GdnTcWs &ws, const GdnTcExport &ex, int32_t *status,
-                                  const PrepRange &pr, Shape s, cudaStream_t st) {
-    if (s.d == 128) return prepare_tc_impl<128>(q, k, v, g, beta, route, scale_la, ws, ex, status, pr, s, st);
-    return prepare_tc_impl<64>(q, k, v, g, beta, route, scale_la, ws, ex, status, pr, s, st);
+                                  const GdnTcWs &ws, const GdnTcExport &ex, int32_t *status, Shape s,
+                                  cudaStream_t st, float norm_eps) {
+    if (s.d == 128) return prepare_tc_impl<128>(q, k, v, g, beta, route, scale_la, ws, ex, status, norm_eps, s, st);
+    return prepare_tc_impl<64>(q, k, v, g, beta, route, scale_la, ws, ex, status, norm_eps, s, st);
 }
 
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,

@@ -120,20 +120,11 @@ struct GdnTcExport {
     float *S_c;      // chunk-entry states [B,H,L/C,d,d]
     float *Ut;       // U~ = U - W S, token-major [B,L,H,d]
 };
-// Which chunks a launch of the prepare kernel covers.  n_chunks == 0: all of them.  A second part
-// that runs beside the scan (beside_previous: launched as a programmatic dependent of the kernel
-// before it in the stream) raises ready_flags [B*H, L/C] per chunk, which the scan's producer waits
-// for from chunk ScanOut::ready_from on.
-struct PrepRange {
-    int c_begin, n_chunks;
-    int32_t *ready_flags;
-    bool beside_previous;
-    float norm_eps = -1.f;     // >= 0: q and k rows are L2-normalised as the tiles are converted (Section 4.3)
-};
+// norm_eps >= 0: q and k rows are L2-normalised as the tiles are converted (Section 4.3, HeadGroups)
 cudaError_t launch_gdn_prepare_tc(const void *q, const void *k, const void *v, const float *g,
                                   const float *beta, const uint8_t *route, float scale_la,
-                                  const GdnTcWs &ws, const GdnTcExport &ex, int32_t *status,
-                                  const PrepRange &pr, Shape s, cudaStream_t st);
+                                  const GdnTcWs &ws, const GdnTcExport &ex, int32_t *status, Shape s,
+                                  cudaStream_t st, float norm_eps = -1.f);
 // Splitting the scan of one (batch, head) over several CTAs when there are few (batch, head)
 // pairs.  The state recurrence S <- (gamma_C I - K~^T W) S + K~^T U is affine in S with a factor
 // that acts on the key dimension only, so a segment of chunks maps its entry state S0 to
@@ -158,8 +149,6 @@ struct ScanOut {
     void *o_la16;
     float *o_la32;
     int32_t *emit_flags;
-    const int32_t *ready_flags = nullptr;   // see PrepRange: chunks >= ready_from are waited for
-    int ready_from = 0;
 };
 constexpr int kScanRowWarps = 8;
 cudaError_t launch_gdn_scan_tc(const GdnTcWs &ws, float scale_la, const float *state_in,

@@ -6,7 +6,7 @@ on the same seeded inputs:
 * fp32 storage (CUDA-core kernels): d = 64 and 128, G = 1, 2, 4, with and without normalisation;
 * bf16 storage (tensor-core kernels): d = 128 with G = 2 -- six linear heads with twelve softmax heads,
   the appendix's smaller model -- and G = 1 with normalisation, on shapes that take the one-pass scan,
-  the segmented scan and the prepare kernel split around the scan;
+  and the segmented scan;
 * requests that are not built come back as NATSL_ERR_UNSUPPORTED, before any launch.
 """
 import dataclasses
@@ -85,7 +85,7 @@ def test_fp32_storage(d, G, norm, B, H, L):
 @pytest.mark.parametrize("G,norm,B,H,L,flags", [
     (2, True, 1, 6, 1024, 0),        # six linear heads x two softmax heads; segmented scan (few heads)
     (2, False, 1, 6, 512, 0),
-    (2, True, 8, 6, 512, 0),         # 48 (batch, head) pairs: one-pass scan, prepare kernel split around it
+    (2, True, 8, 6, 512, 0),         # 48 (batch, head) pairs: one-pass scan
     (2, True, 2, 3, 320, 16),        # stages in sequence on the caller's stream; ragged last query tile
     (1, True, 2, 4, 384, 0),         # normalisation alone
     (2, True, 1, 2, 192, 2),         # one-pass scan with few heads
