@@ -131,7 +131,7 @@ enum {
     NATSL_SAVED_FWD = 1u << 6,         /* backward: `ws` holds such a forward (same inputs, same p apart
                                     from this flag).  One backward per saved forward: the backward
                                     reuses some of the saved buffers for its own results */
-    NATSL_QK_NORM = 1u << 7            /* forward: q and k are normalised inside the kernels, differently
+    NATSL_QK_NORM = 1u << 7            /* forward and backward: q and k are normalised inside the kernels, differently
                                     for the two operations that share them (Section 4.3): L2 over the
                                     d columns of the head for the linear operation,
                                     x / sqrt(sum x^2 + norm_eps), and RMS per softmax head for the
@@ -181,10 +181,12 @@ typedef struct natsl_params {
                             /*   Built: natsl_hybrid_fwd with token-level routing, for fp32 storage    */
                             /*   (d / G in {32, 64, 128}) and on the tensor-core path for d = 128,     */
                             /*   G = 2 (the appendix's two softmax heads per linear head; three would  */
-                            /*   need d = 192).  G > 1 or NATSL_QK_NORM with anything else (backward,  */
-                            /*   decode, NATSL_BLOCK_ROUTING, NATSL_APPEND_CACHE, NATSL_SAVE_FOR_BWD,  */
-                            /*   NATSL_FORCE_SIMT on bf16, NATSL_QK_NORM with p->k_sm):                */
-                            /*   NATSL_ERR_UNSUPPORTED.                                                */
+                            /*   need d = 192); natsl_hybrid_bwd for the same shapes except bf16       */
+                            /*   storage with d = 64 (self-contained call, token-level routing).       */
+                            /*   G > 1 or NATSL_QK_NORM with anything else (decode,                    */
+                            /*   NATSL_BLOCK_ROUTING, NATSL_APPEND_CACHE, NATSL_SAVE_FOR_BWD /         */
+                            /*   NATSL_SAVED_FWD, NATSL_FORCE_SIMT on bf16, NATSL_QK_NORM with         */
+                            /*   p->k_sm): NATSL_ERR_UNSUPPORTED.                                      */
     float norm_eps;         /* NATSL_QK_NORM: epsilon under the square roots, >= 0                     */
 } natsl_params;
 

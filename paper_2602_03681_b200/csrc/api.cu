@@ -145,6 +145,8 @@ struct BwdWs {
     size_t head_bytes;                                       // status page + emit_flags: cleared per forward
     float *k_sm32, *v_sm32;                                  // [B,H,L,d] compacted, fp32
     float *q32, *k32, *v32;                                  // token-major fp32 copies
+    float *qs32, *ks32;                                      // NATSL_QK_NORM, fp32 storage: RMS-normalised q, k
+                                                             // (q32, k32 then hold the L2-normalised ones)
     float *W, *U, *Ut, *o_la, *o_nla, *do_la, *do_nla;       // token-major
     float *dUt, *dQg, *dW, *dKt, *dKb, *dVb, *X1p, *X2, *X3, *X4, *dq_sm, *dk_sm, *dv_sm;
     float *P, *Abar, *M, *N, *Mg, *Ms, *Ns;                  // [B,H,NC,64,64]
@@ -186,6 +188,9 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.sm_len = c.take<int32_t>(B * H);
     f.k_sm32 = tm(!tcs); f.v_sm32 = tm(!tcs);
     f.q32 = tm(general); f.k32 = tm(general); f.v32 = tm(general);
+    const bool normed = !tcs && (p->flags & NATSL_QK_NORM);
+    f.qs32 = tm(normed); f.ks32 = tm(normed);
+    const size_t Gg = p->G > 1 ? (size_t)p->G : 1;           // softmax heads per linear head: lse, Dsm per softmax head
     f.W = tm(general); f.U = tm(general);
     f.Ut = tm(true);
     f.o_la = tm(true);
@@ -203,8 +208,8 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.S_c = c.take<float>(ST);
     f.dS_c = c.take<float>(ST);
     f.Gcum = c.take<float>(BHL);
-    f.lse = c.take<float>(BHL);
-    f.Dsm = c.take<float>(BHL);
+    f.lse = c.take<float>(BHL * Gg);
+    f.Dsm = c.take<float>(BHL * Gg);
     f.dGrow = c.take<float>(BHL);
     f.kappa = c.take<float>(BHL);
     f.gS = c.take<float>(general ? B * H * NC * (d / 32) : 0);
@@ -326,18 +331,30 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
                                    block ? f.status : nullptr, p->L, p->B, p->L, p->H, st0));
     if (!fused_chunks)
         NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
+    // fp32 storage with NATSL_QK_NORM: q32, k32 become the L2-normalised rows (everything of the linear
+    // branch reads those), qs32, ks32 the slice-wise RMS-normalised ones (softmax branch)
+    // (tensor cores: the kernels normalise inside; only the fp32 copies the separate chunk-level products
+    // of the backward read are made here)
+    const HeadGroups hg = head_groups(p);
+    const float *qs = f.q32, *ks = f.k32;
+    if (hg.norm_eps >= 0.f) {
+        NATSL_TRY(launch_qk_norm_f32(q, k, s.bf16, f.q32, f.k32, tensor_cores ? nullptr : f.qs32,
+                                     tensor_cores ? nullptr : f.ks32, (size_t)(B * L * H), p->d, hg.G,
+                                     hg.norm_eps, st));
+        if (!tensor_cores) { qs = f.qs32; ks = f.ks32; }
+    }
     if (tensor_cores)
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, f.k_smb, nullptr, f.v16, f.k16, p->L,
-                                      p->L, false, f.status, s, st0));
+                                      p->L, false, f.status, s, st0, hg));
     else
-        NATSL_TRY(launch_gather_kv(f.k32, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
+        NATSL_TRY(launch_gather_kv(ks, f.v32, f.sm_idx, f.prefix, f.k_sm32, f.v_sm32, p->L,
                                    f.status, s32, st));
     if (tensor_cores) {
         // the fused chunk kernel reads W^T, U^T as the forward keeps them: no fp32 copies for it
         const GdnTcExport ex{fused_chunks ? nullptr : f.W, fused_chunks ? nullptr : f.U, nullptr, f.Tinv,
                              f.Gcum, f.S_c, f.Ut};
         NATSL_TRY(launch_gdn_prepare_tc(q, k, v, g, beta, block ? nullptr : route, p->scale_la, f.tc, ex,
-                                        f.status, s, st));
+                                        f.status, s, st, hg.norm_eps));
         // (the side stream joins before the scan, so that the softmax kernel follows the scan directly
         // and can run beside it as its programmatic dependent, as in natsl_hybrid_fwd)
         NATSL_TRY(side_join.join());
@@ -354,11 +371,11 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
     if (tensor_cores)
         NATSL_TRY(launch_softmax_combine_tc(q, f.k_smb, f.v16, p->L, p->L, f.sm_idx, f.prefix, f.o_la16,
                                             flags, p->w, p->scale_sm, p->eps, out, f.o_nla, f.lse,
-                                            BlockRouting{block_route, k, v}, false, f.status, s, st));
+                                            BlockRouting{block_route, k, v}, false, f.status, s, st, hg));
     else
-        NATSL_TRY(launch_softmax_combine_simt(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
+        NATSL_TRY(launch_softmax_combine_simt(qs, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
                                               f.o_la, p->w, p->scale_sm, p->eps, out, f.o_nla,
-                                              f.lse, BlockRouting{block_route, f.k32, f.v32}, s32, st));
+                                              f.lse, BlockRouting{block_route, f.k32, f.v32}, s32, st, hg.G));
 #undef NATSL_TRY
     return NATSL_OK;
 }
@@ -512,7 +529,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     // fp32 storage with NATSL_QK_NORM: normalised copies first (the tensor-core kernels normalise inside)
     const void *q_la = q, *k_la = k, *q_sm = q, *k_nsm = k;
     if (!tensor_cores && hg.norm_eps >= 0.f) {
-        NATSL_TRY(launch_qk_norm_f32((const float *)q, (const float *)k, f.q_la, f.k_la, f.q_sm, f.k_nsm,
+        NATSL_TRY(launch_qk_norm_f32(q, k, false, f.q_la, f.k_la, f.q_sm, f.k_nsm,
                                      (size_t)p->B * p->L * p->H, p->d, hg.G, hg.norm_eps, st));
         q_la = f.q_la; k_la = f.k_la; q_sm = f.q_sm; k_nsm = f.k_nsm;
     }
@@ -581,7 +598,16 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (!q || !k || !v || !g || !beta || !route || !dout || !dq || !dk || !dv || !dg || !dbeta)
         return NATSL_ERR_NULL;
     if (p->flags & NATSL_APPEND_CACHE) return NATSL_ERR_UNSUPPORTED;
-    if (grouped_or_normed(p)) return NATSL_ERR_UNSUPPORTED;   // grouped heads, q/k normalisation: forward only
+    const HeadGroups hg = head_groups(p);
+    if (grouped_or_normed(p)) {      // grouped heads, q/k normalisation: the paths with separate chunk-level products
+        if (p->flags & (NATSL_BLOCK_ROUTING | NATSL_SAVED_FWD)) return NATSL_ERR_UNSUPPORTED;
+        if (use_tensor_cores(p)) {
+            if (p->d != 128 || hg.G > 2) return NATSL_ERR_UNSUPPORTED;
+        } else {
+            if (p->dtype != NATSL_F32) return NATSL_ERR_UNSUPPORTED;
+            if (hg.G > 1 && (hg.G > 4 || p->d / hg.G < 32)) return NATSL_ERR_UNSUPPORTED;
+        }
+    }
     if (use_tensor_cores(p) && !(p->scale_sm > 0.f)) return NATSL_ERR_SHAPE;
     const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
     if (p->dscore && !block) return NATSL_ERR_UNSUPPORTED;   // score gradients: one decision per block
@@ -629,7 +655,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la,
                                  tensor_cores && !general_block ? nullptr : f.do_nla, dw, f.Dsm,
                                  tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
-                                 tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, gsc, s, st));
+                                 tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, gsc, s, st, hg.G));
     // Dependencies from here on: the query-side softmax kernel, the key-side one and the reverse
     // scan need only what is already there; the chunk kernel needs the first and the third; the
     // scatter of the retained tokens' dk, dv needs the second.  With token-level routing the chunk
@@ -654,17 +680,19 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_softmax_bwd_tc(q, f.Qh, f.dO16, f.k16, f.v16, p->L, f.sm_idx, f.prefix, f.lse,
                                         f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm,
                                         p->dscore ? (general_block ? f.dmask : f.dGrow) : nullptr, fused_chunks,
-                                        f.status, s, st, kv_aside ? st0 : st));
+                                        f.status, s, st, kv_aside ? st0 : st, hg));
     else
-        NATSL_TRY(launch_softmax_bwd(f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix, f.do_nla,
-                                     f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm, s, st,
-                                     p->dscore ? f.dmask : nullptr));
+        NATSL_TRY(launch_softmax_bwd(hg.norm_eps >= 0.f ? f.qs32 : f.q32, f.k_sm32, f.v_sm32, p->L, f.sm_idx,
+                                     f.prefix, f.do_nla, f.lse, f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm,
+                                     s, st, p->dscore ? f.dmask : nullptr, hg.G));
     if (!tensor_cores)
         NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
                                    f.dS_c, f.gS, p->dstate_out, p->dstate_in, s, st, block_route));
     if (side) NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));     // the reverse scan has finished
+    // (with the normalisation the two operations' dq stay apart until its backward at the very end)
+    const bool normed = hg.norm_eps >= 0.f;
     AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, general_block ? nullptr : route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
-                   f.X3, f.X4, f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
+                   f.X3, f.X4, normed ? nullptr : f.dq_sm, f.dk_sm, f.dv_sm, f.gS, f.sm_idx, f.prefix, p->L,
                    p->scale_la, f.dGrow, f.kappa, dbeta, dg};
     if (fused_chunks && block) {
         // Every token has a softmax-branch dk, dv here: the retained tokens' from the compacted
@@ -721,7 +749,22 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ms), TM(f.k32), TM(f.X2), kC, di, kC, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Ns), TM(f.k32), TM(f.X3), kC, di, kC, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ns), TM(f.q32), TM(f.X4), kC, di, kC, 1.f, false, s, st));
-    NATSL_TRY(launch_gdn_assemble(a, dq, dk, dv, s, st));
+    // With the normalisation the assembly's dq, dk are gradients with respect to the normalised rows; a
+    // last kernel applies the two row-local Jacobians.  fp32 storage: in place.  bf16 storage: the
+    // assembly writes fp32 (into buffers the chunk-level products are done with) and the last kernel
+    // rounds once.
+    if (!normed) {
+        NATSL_TRY(launch_gdn_assemble(a, dq, dk, dv, s, st));
+    } else if (!s.bf16) {
+        NATSL_TRY(launch_gdn_assemble(a, dq, dk, dv, s, st));
+        NATSL_TRY(launch_qk_norm_bwd_f32(q, k, false, route, (const float *)dq, f.dq_sm, (const float *)dk, nullptr,
+                                         dq, dk, nullptr, (size_t)(B * L * H), p->d, hg.G, hg.norm_eps, st));
+    } else {
+        float *dq32 = f.dW, *dk32 = f.W, *dv32 = f.U;
+        NATSL_TRY(launch_gdn_assemble(a, dq32, dk32, dv32, s32, st));
+        NATSL_TRY(launch_qk_norm_bwd_f32(q, k, true, route, dq32, f.dq_sm, dk32, dv32, dq, dk, dv,
+                                         (size_t)(B * L * H), p->d, hg.G, hg.norm_eps, st));
+    }
     if (p->dscore)   // softmax blocks: the mask gradients of their keys; linear blocks: the kappa of their tokens
         NATSL_TRY(launch_dscore(route, f.prefix, f.dmask, nullptr, f.kappa, p->L, p->dscore, s, st));
 #undef NATSL_TRY

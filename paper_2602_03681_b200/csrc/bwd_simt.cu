@@ -151,6 +151,9 @@ dout_amax_kernel(const T *__restrict__ dout, size_t n4, int32_t *status) {
     if ((threadIdx.x & 31) == 0 && m > 0.f) atomicMax(status + kGradAmaxWord, __float_as_int(m));
 }
 
+// G > 1 (grouped softmax heads, Section 4.3): the softmax branch's output is normalised per slice of
+// D / G columns, so its part of the backward (do_nla, dw_nla, D_i = <do_i, o_i>) is formed per slice;
+// Dsm is then [B,H,G,L].
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_nla,
@@ -158,7 +161,7 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
                    float *__restrict__ do_la, float *__restrict__ do_nla, float *__restrict__ dw,
                    float *__restrict__ Dsm, __half *__restrict__ do16,
                    __half *__restrict__ dola16, __half *__restrict__ dolag16,
-                   const float *__restrict__ Gd, float scale_la, const int32_t *gsc, int B, int L, int H) {
+                   const float *__restrict__ Gd, float scale_la, const int32_t *gsc, int G, int B, int L, int H) {
     constexpr int kCols = D / 32;
     const float gs = grad_scale(gsc).x;      // scale of the fp16 operand copies (and of Dsm with them)
     const int lane = threadIdx.x & 31;
@@ -167,33 +170,51 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
     const int h = row % H;
     const size_t bl = row / H;
     const int l = bl % L, b = bl / L;
-    float ol[kCols], on[kCols], dy[kCols], ssl = 0.f, ssn = 0.f;
+    const int ds = D / G;                    // columns per softmax head (a multiple of 32)
+    float ol[kCols], on[kCols], dy[kCols], ssl = 0.f, ssn[kCols];
 #pragma unroll
     for (int x = 0; x < kCols; ++x) {
         const size_t i = row * D + lane + 32 * x;
         ol[x] = o_la[i]; on[x] = o_nla[i]; dy[x] = to_f32(dout[i]);
         ssl = fmaf(ol[x], ol[x], ssl);
-        ssn = fmaf(on[x], on[x], ssn);
+        ssn[x] = warp_sum(on[x] * on[x]);     // sum of squares of this 32-column group
     }
-    ssl = warp_sum(ssl); ssn = warp_sum(ssn);
-    const float fl = rsqrtf(ssl / D + eps), fn = rsqrtf(ssn / D + eps);
+    ssl = warp_sum(ssl);
+    const float fl = rsqrtf(ssl / D + eps);
+    float fn[kCols];                          // RMS factor of the slice a 32-column group belongs to
+#pragma unroll
+    for (int x = 0; x < kCols; ++x) {
+        float t = 0.f;
+#pragma unroll
+        for (int y = 0; y < kCols; ++y) t += (32 * y) / ds == (32 * x) / ds ? ssn[y] : 0.f;
+        fn[x] = rsqrtf(t / ds + eps);
+    }
     const float wn = w ? w[row * 2] : 0.5f, wl = w ? w[row * 2 + 1] : 0.5f;
     // scale_la gamma_l of the token (decay from its chunk's entry), for the reverse scan's operand
     const float sg = dolag16 ? scale_la * Gd[((size_t)(b * H + h) * (L / kC) + l / kC) * 128 + l % kC] : 0.f;
-    float dwl = 0.f, dwn = 0.f;
+    float dwl = 0.f, dwn_g[kCols];
 #pragma unroll
     for (int x = 0; x < kCols; ++x) {
         dwl = fmaf(dy[x], ol[x] * fl, dwl);
-        dwn = fmaf(dy[x], on[x] * fn, dwn);
+        dwn_g[x] = warp_sum(dy[x] * on[x] * fn[x]);
     }
-    dwl = warp_sum(dwl); dwn = warp_sum(dwn);
-    const float ml = wl * dwl / D, mn = wn * dwn / D;
-    float dsm = 0.f;
+    dwl = warp_sum(dwl);
+    float dwn = 0.f, mn[kCols];               // mn: w_nla <dy, y_nla> / ds over the group's slice
+#pragma unroll
+    for (int x = 0; x < kCols; ++x) {
+        dwn += dwn_g[x];
+        float t = 0.f;
+#pragma unroll
+        for (int y = 0; y < kCols; ++y) t += (32 * y) / ds == (32 * x) / ds ? dwn_g[y] : 0.f;
+        mn[x] = wn * t / ds;
+    }
+    const float ml = wl * dwl / D;
+    float dsm_g[kCols];
 #pragma unroll
     for (int x = 0; x < kCols; ++x) {
         const size_t i = row * D + lane + 32 * x;
         const float dl = fl * (wl * dy[x] - ol[x] * fl * ml);
-        const float dn = fn * (wn * dy[x] - on[x] * fn * mn);
+        const float dn = fn[x] * (wn * dy[x] - on[x] * fn[x] * mn[x]);
         do_la[i] = dl;
         if (do_nla) do_nla[i] = dn;   // (the tensor-core softmax backward reads the fp16 copy only)
         const size_t i16 = ((((size_t)b * H + h) * L + l) * D) + lane + 32 * x;
@@ -202,19 +223,25 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
             dola16[i16] = __float2half_rn(gs * dl);
             dolag16[i16] = __float2half_rn(gs * sg * dl);
         }
-        dsm = fmaf(dn, on[x], dsm);
+        dsm_g[x] = warp_sum(dn * on[x]);
     }
-    dsm = warp_sum(dsm);
     if (lane == 0) {
         if (dw) { dw[row * 2] = dwn; dw[row * 2 + 1] = dwl; }
-        Dsm[((size_t)b * H + h) * L + l] = gs * dsm;
+        for (int g = 0; g < G; ++g) {
+            float t = 0.f;
+#pragma unroll
+            for (int x = 0; x < kCols; ++x) t += (32 * x) / ds == g ? dsm_g[x] : 0.f;
+            Dsm[(((size_t)b * H + h) * G + g) * L + l] = gs * t;
+        }
     }
 }
 
 // ------------------------------------------------------------------------------------------
 // softmax backward, query side: dq_sm.  grid = (L/64, B*H), same tiling as the forward.
 // ------------------------------------------------------------------------------------------
-template <int D>
+// G softmax heads per linear head (Section 4.3): the kernel's head is a slice of D columns of rows of
+// DL = G D columns; lse and Dsm are [B,H,G,L].
+template <int D, int G>
 __global__ void __launch_bounds__(kThreads)
 softmax_bwd_dq_kernel(const float *__restrict__ q32, const float *__restrict__ k_sm32,
                       const float *__restrict__ v_sm32, int cap, const int32_t *__restrict__ sm_idx,
@@ -229,37 +256,38 @@ softmax_bwd_dq_kernel(const float *__restrict__ q32, const float *__restrict__ k
     float *Vt = Kt + 32 * (D + 1);         // [32][D+1]
     int *pos = reinterpret_cast<int *>(Vt + 32 * (D + 1));
 
-    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
+    constexpr int DL = D * G;
+    const int c = blockIdx.x, bhg = blockIdx.y, bh = bhg / G, col0 = (bhg % G) * D, b = bh / H, h = bh % H;
     const int NC = L / kC;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const size_t ts = (size_t)H * D;
+    const size_t ts = (size_t)H * DL;
     const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
     const int n_end = min(sm_chunk_prefix[(size_t)bh * (NC + 1) + c + 1], cap);
 
     for (int idx = threadIdx.x; idx < kC * D / 4; idx += kThreads) {
         const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
-        store4(Qs + r * D + c4, load4(q32 + tok0 * D + (size_t)r * ts + c4));
-        store4(dOs + r * D + c4, load4(do_nla + tok0 * D + (size_t)r * ts + c4));
+        store4(Qs + r * D + c4, load4(q32 + tok0 * DL + (size_t)r * ts + col0 + c4));
+        store4(dOs + r * D + c4, load4(do_nla + tok0 * DL + (size_t)r * ts + col0 + c4));
     }
     constexpr int kQ = 8, kCols = D / 32;
     float acc[kQ][kCols], lse_r[kQ], dsm_r[kQ];
 #pragma unroll
     for (int r = 0; r < kQ; ++r) {
         const int i = c * kC + warp * kQ + r;
-        lse_r[r] = lse[(size_t)bh * L + i];
-        dsm_r[r] = Dsm[(size_t)bh * L + i];
+        lse_r[r] = lse[(size_t)bhg * L + i];
+        dsm_r[r] = Dsm[(size_t)bhg * L + i];
 #pragma unroll
         for (int x = 0; x < kCols; ++x) acc[r][x] = 0.f;
     }
-    const float *kb = k_sm32 + (size_t)bh * cap * D, *vb = v_sm32 + (size_t)bh * cap * D;
+    const float *kb = k_sm32 + (size_t)bh * cap * DL + col0, *vb = v_sm32 + (size_t)bh * cap * DL + col0;
     for (int j0 = 0; j0 < n_end; j0 += 32) {
         __syncthreads();
         for (int idx = threadIdx.x; idx < 32 * D / 4; idx += kThreads) {
             const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
             float4 kx = make_float4(0.f, 0.f, 0.f, 0.f), vx = kx;
             if (j0 + r < n_end) {
-                kx = load4(kb + (size_t)(j0 + r) * D + c4);
-                vx = load4(vb + (size_t)(j0 + r) * D + c4);
+                kx = load4(kb + (size_t)(j0 + r) * DL + c4);
+                vx = load4(vb + (size_t)(j0 + r) * DL + c4);
             }
             float *kp = Kt + r * (D + 1) + c4, *vp = Vt + r * (D + 1) + c4;
             kp[0] = kx.x; kp[1] = kx.y; kp[2] = kx.z; kp[3] = kx.w;
@@ -295,14 +323,14 @@ softmax_bwd_dq_kernel(const float *__restrict__ q32, const float *__restrict__ k
     for (int r = 0; r < kQ; ++r) {
         const size_t t = tok0 + (size_t)(warp * kQ + r) * H;
 #pragma unroll
-        for (int x = 0; x < kCols; ++x) dq_sm[t * D + lane + 32 * x] = scale_sm * acc[r][x];
+        for (int x = 0; x < kCols; ++x) dq_sm[t * DL + col0 + lane + 32 * x] = scale_sm * acc[r][x];
     }
 }
 
 // ------------------------------------------------------------------------------------------
 // softmax backward, key side: dk_sm, dv_sm per compacted key.  grid = (ceil(cap/32), B*H).
 // ------------------------------------------------------------------------------------------
-template <int D>
+template <int D, int G>
 __global__ void __launch_bounds__(kThreads)
 softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ k_sm32,
                        const float *__restrict__ v_sm32, int cap, const int32_t *__restrict__ sm_idx,
@@ -323,21 +351,22 @@ softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ 
     float *dsm_s = lse_s + kC;              // [64]
     int *pos = reinterpret_cast<int *>(dsm_s + kC);
 
-    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    constexpr int DL = D * G;
+    const int bhg = blockIdx.y, bh = bhg / G, col0 = (bhg % G) * D, b = bh / H, h = bh % H;
     const int NC = L / kC;
     const int n_sm = min(sm_chunk_prefix[(size_t)bh * (NC + 1) + NC], cap);
     const int j0 = blockIdx.x * 32;
     if (j0 >= n_sm) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const size_t ts = (size_t)H * D;
-    const float *kb = k_sm32 + (size_t)bh * cap * D, *vb = v_sm32 + (size_t)bh * cap * D;
+    const size_t ts = (size_t)H * DL;
+    const float *kb = k_sm32 + (size_t)bh * cap * DL + col0, *vb = v_sm32 + (size_t)bh * cap * DL + col0;
 
     for (int idx = threadIdx.x; idx < 32 * D / 4; idx += kThreads) {
         const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
         float4 kx = make_float4(0.f, 0.f, 0.f, 0.f), vx = kx;
         if (j0 + r < n_sm) {
-            kx = load4(kb + (size_t)(j0 + r) * D + c4);
-            vx = load4(vb + (size_t)(j0 + r) * D + c4);
+            kx = load4(kb + (size_t)(j0 + r) * DL + c4);
+            vx = load4(vb + (size_t)(j0 + r) * DL + c4);
         }
         float *kp = Kt + r * (D + 1) + c4, *vp = Vt + r * (D + 1) + c4;
         kp[0] = kx.x; kp[1] = kx.y; kp[2] = kx.z; kp[3] = kx.w;
@@ -360,12 +389,12 @@ softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ 
         __syncthreads();
         for (int idx = threadIdx.x; idx < kC * D / 4; idx += kThreads) {
             const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
-            store4(Qs + r * D + c4, load4(q32 + tok0 * D + (size_t)r * ts + c4));
-            store4(dOs + r * D + c4, load4(do_nla + tok0 * D + (size_t)r * ts + c4));
+            store4(Qs + r * D + c4, load4(q32 + tok0 * DL + (size_t)r * ts + col0 + c4));
+            store4(dOs + r * D + c4, load4(do_nla + tok0 * DL + (size_t)r * ts + col0 + c4));
         }
         if (threadIdx.x < kC) {
-            lse_s[threadIdx.x] = lse[(size_t)bh * L + c * kC + threadIdx.x];
-            dsm_s[threadIdx.x] = Dsm[(size_t)bh * L + c * kC + threadIdx.x];
+            lse_s[threadIdx.x] = lse[(size_t)bhg * L + c * kC + threadIdx.x];
+            dsm_s[threadIdx.x] = Dsm[(size_t)bhg * L + c * kC + threadIdx.x];
         }
         __syncthreads();
         const float *kr = Kt + lane * (D + 1), *vr = Vt + lane * (D + 1);
@@ -396,11 +425,11 @@ softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ 
         }
     }
     if (j0 + kj < n_sm) {
-        float *dkr = dk_sm + ((size_t)bh * cap + j0 + kj) * D + cs;
-        float *dvr = dv_sm + ((size_t)bh * cap + j0 + kj) * D + cs;
+        float *dkr = dk_sm + ((size_t)bh * cap + j0 + kj) * DL + col0 + cs;
+        float *dvr = dv_sm + ((size_t)bh * cap + j0 + kj) * DL + col0 + cs;
 #pragma unroll
         for (int x = 0; x < kPer; ++x) { dkr[8 * x] = scale_sm * adk[x]; dvr[8 * x] = adv[x]; }
-        if (dmask && cs == 0) dmask[(size_t)bh * cap + j0 + kj] = adm;
+        if (dmask && cs == 0) dmask[(size_t)bhg * cap + j0 + kj] = adm;
     }
 }
 
@@ -727,7 +756,7 @@ gdn_assemble_kernel(const float *__restrict__ q32, const float *__restrict__ k32
         kdKb = fmaf(kv, a_dKb, kdKb); qdQg = fmaf(qv, a_dQg, qdQg); kdKt = fmaf(kv, a_dKt, kdKt);
         kX1 = fmaf(kv, x1, kX1); kX2 = fmaf(kv, x2, kX2); qX3 = fmaf(qv, x3, qX3);
         kX4 = fmaf(kv, x4, kX4); vdVb = fmaf(vv, a_dVb, vdVb);
-        dq[i] = from_f32<T>(scale_la * gam * a_dQg + x3 + dq_sm[i]);
+        dq[i] = from_f32<T>(scale_la * gam * a_dQg + x3 + (dq_sm ? dq_sm[i] : 0.f));
         if (lin) {
             dk[i] = from_f32<T>(bt * gam * a_dKb + kt * a_dKt + bt * x1 + x2 + x4 + (dk_x ? dk_x[i] : 0.f));
             dv[i] = from_f32<T>(bt * a_dVb + (dv_x ? dv_x[i] : 0.f));
@@ -832,11 +861,11 @@ static cudaError_t combine_bwd_impl(const float *o_la, const float *o_nla, const
                                     const float *w, float eps, float *do_la, float *do_nla,
                                     float *dw, float *Dsm, void *do16, void *dola16, void *dolag16,
                                     const float *Gd, float scale_la, const int32_t *gsc, Shape s,
-                                    cudaStream_t st) {
+                                    cudaStream_t st, int G) {
     const size_t rows = (size_t)s.B * s.L * s.H;
     combine_bwd_kernel<T, D><<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
         o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, (__half *)do16, (__half *)dola16,
-        (__half *)dolag16, Gd, scale_la, gsc, s.B, s.L, s.H);
+        (__half *)dolag16, Gd, scale_la, gsc, G, s.B, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -855,16 +884,17 @@ cudaError_t launch_dout_amax(const void *dout, size_t n, bool bf16, int32_t *sta
 cudaError_t launch_combine_bwd(const float *o_la, const float *o_nla, const void *dout,
                                const float *w, float eps, float *do_la, float *do_nla, float *dw,
                                float *Dsm, void *do16, void *dola16, void *dolag16, const float *Gd,
-                               float scale_la, const int32_t *gsc, Shape s, cudaStream_t st) {
+                               float scale_la, const int32_t *gsc, Shape s, cudaStream_t st, int G) {
+    if (G < 1 || s.d % (32 * G) != 0) return cudaErrorInvalidValue;
     if (s.bf16) {
-        if (s.d == 128) return combine_bwd_impl<__nv_bfloat16, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st);
-        return combine_bwd_impl<__nv_bfloat16, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st);
+        if (s.d == 128) return combine_bwd_impl<__nv_bfloat16, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st, G);
+        return combine_bwd_impl<__nv_bfloat16, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st, G);
     }
-    if (s.d == 128) return combine_bwd_impl<float, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st);
-    return combine_bwd_impl<float, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st);
+    if (s.d == 128) return combine_bwd_impl<float, 128>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st, G);
+    return combine_bwd_impl<float, 64>(o_la, o_nla, dout, w, eps, do_la, do_nla, dw, Dsm, do16, dola16, dolag16, Gd, scale_la, gsc, s, st, G);
 }
 
-template <int D>
+template <int D, int G = 1>
 static cudaError_t softmax_bwd_impl(const float *q32, const float *k_sm32, const float *v_sm32,
                                     int cap, const int32_t *sm_idx, const int32_t *pre,
                                     const float *do_nla, const float *lse, const float *Dsm,
@@ -872,16 +902,16 @@ static cudaError_t softmax_bwd_impl(const float *q32, const float *k_sm32, const
                                     float *dmask, Shape s, cudaStream_t st) {
     const size_t smem_q = sizeof(float) * (2 * kC * D + 2 * 32 * (D + 1) + 32);
     const size_t smem_k = sizeof(float) * (2 * 32 * (D + 1) + 2 * kC * D + 2 * kC * 33 + 2 * kC + 32);
-    cudaError_t e = set_smem(softmax_bwd_dq_kernel<D>, smem_q);
+    cudaError_t e = set_smem(softmax_bwd_dq_kernel<D, G>, smem_q);
     if (e != cudaSuccess) return e;
-    e = set_smem(softmax_bwd_dkv_kernel<D>, smem_k);
+    e = set_smem(softmax_bwd_dkv_kernel<D, G>, smem_k);
     if (e != cudaSuccess) return e;
-    dim3 gq(s.L / kC, s.B * s.H);
-    softmax_bwd_dq_kernel<D><<<gq, kThreads, smem_q, st>>>(q32, k_sm32, v_sm32, cap, sm_idx, pre,
+    dim3 gq(s.L / kC, s.B * s.H * G);
+    softmax_bwd_dq_kernel<D, G><<<gq, kThreads, smem_q, st>>>(q32, k_sm32, v_sm32, cap, sm_idx, pre,
                                                            do_nla, lse, Dsm, scale_sm, dq_sm, s.L, s.H);
     count_launch();
-    dim3 gk((cap + 31) / 32, s.B * s.H);
-    softmax_bwd_dkv_kernel<D><<<gk, kThreads, smem_k, st>>>(q32, k_sm32, v_sm32, cap, sm_idx, pre,
+    dim3 gk((cap + 31) / 32, s.B * s.H * G);
+    softmax_bwd_dkv_kernel<D, G><<<gk, kThreads, smem_k, st>>>(q32, k_sm32, v_sm32, cap, sm_idx, pre,
                                                             do_nla, lse, Dsm, scale_sm, dk_sm, dv_sm,
                                                             dmask, s.L, s.H);
     count_launch();
@@ -892,7 +922,18 @@ cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const floa
                                const int32_t *sm_idx, const int32_t *sm_chunk_prefix,
                                const float *do_nla, const float *lse, const float *Dsm,
                                float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm, Shape s,
-                               cudaStream_t st, float *dmask) {
+                               cudaStream_t st, float *dmask, int G) {
+    if (G > 1) {      // grouped softmax heads: slices of 32 or 64 columns
+#define NATSL_GROUPED(DS, GG)                                                                                 \
+        if (s.d == DS * GG && G == GG)                                                                        \
+            return softmax_bwd_impl<DS, GG>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, \
+                                            scale_sm, dq_sm, dk_sm, dv_sm, dmask, s, st)
+        NATSL_GROUPED(32, 2);
+        NATSL_GROUPED(64, 2);
+        NATSL_GROUPED(32, 4);
+#undef NATSL_GROUPED
+        return cudaErrorInvalidValue;
+    }
     if (s.d == 128) return softmax_bwd_impl<128>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, scale_sm, dq_sm, dk_sm, dv_sm, dmask, s, st);
     return softmax_bwd_impl<64>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, scale_sm, dq_sm, dk_sm, dv_sm, dmask, s, st);
 }

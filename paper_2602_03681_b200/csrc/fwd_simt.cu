@@ -402,8 +402,9 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
 // Per-operation normalisation of q and k for fp32 storage (Section 4.3): one warp per row of d
 // columns writes the L2-normalised row (linear operation) and the row with each of its G slices
 // RMS-normalised (softmax operation).  The tensor-core path does both inside its kernels instead.
+template <typename T>
 __global__ void __launch_bounds__(256)
-qk_norm_f32_kernel(const float *__restrict__ q, const float *__restrict__ k, float *__restrict__ q_la,
+qk_norm_f32_kernel(const T *__restrict__ q, const T *__restrict__ k, float *__restrict__ q_la,
                    float *__restrict__ k_la, float *__restrict__ q_sm, float *__restrict__ k_sm,
                    size_t rows, int d, int G, float norm_eps) {
     const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -411,23 +412,83 @@ qk_norm_f32_kernel(const float *__restrict__ q, const float *__restrict__ k, flo
     if (row >= rows) return;
     const int ds = d / G;                                // 32, 64 or 128: a multiple of the warp size
     for (int which = 0; which < 2; ++which) {
-        const float *src = (which ? k : q) + row * d;
-        float *la = (which ? k_la : q_la) + row * d, *sm = (which ? k_sm : q_sm) + row * d;
+        const T *src = (which ? k : q) + row * d;
+        float *la = (which ? k_la : q_la) + row * d, *sm = (which ? k_sm : q_sm);
         float x[4], ss_all = 0.f;
         for (int j = 0; j < d / 32; ++j) {
-            x[j] = src[lane + 32 * j];
+            x[j] = to_f32(src[lane + 32 * j]);
             ss_all = fmaf(x[j], x[j], ss_all);
         }
         ss_all = warp_sum(ss_all);
         const float rl = rsqrtf(ss_all + norm_eps);
-        for (int sg = 0; sg < G; ++sg) {
+        for (int sg = 0; sm && sg < G; ++sg) {
             float ss = 0.f;
             for (int j = sg * ds / 32; j < (sg + 1) * ds / 32; ++j) ss = fmaf(x[j], x[j], ss);
             ss = warp_sum(ss);
             const float rs = rsqrtf(ss / ds + norm_eps);
-            for (int j = sg * ds / 32; j < (sg + 1) * ds / 32; ++j) sm[lane + 32 * j] = x[j] * rs;
+            for (int j = sg * ds / 32; j < (sg + 1) * ds / 32; ++j) sm[row * d + lane + 32 * j] = x[j] * rs;
         }
         for (int j = 0; j < d / 32; ++j) la[lane + 32 * j] = x[j] * rl;
+    }
+}
+
+// Backward of that normalisation, in place on fp32 gradients, one warp per row.  On entry dq holds the
+// gradient with respect to the L2-normalised q (linear operation) and dq_sm the one with respect to the
+// slice-wise RMS-normalised q (softmax operation); dk holds, for a linear token, the gradient with
+// respect to the L2-normalised k and, for a retained token, the one with respect to the RMS-normalised k
+// (a token's k reaches only the operation the token was routed to).  x^ = x r, r = (sum x^2 + e)^-1/2:
+// dx = r (g - x^ <x^, g>);  x~ = x r, r = (mean x^2 + e)^-1/2 over a slice of ds columns:
+// dx = r (g - x~ <x~, g> / ds).
+template <typename T>
+__global__ void __launch_bounds__(256)
+qk_norm_bwd_f32_kernel(const T *__restrict__ q, const T *__restrict__ k,
+                       const uint8_t *__restrict__ route, const float *dq_la,
+                       const float *__restrict__ dq_sm, const float *dk_in, const float *dv_in,
+                       T *dq, T *dk, T *dv, size_t rows, int d, int G, float norm_eps) {
+    const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const int ds = d / G, nj = d / 32;
+    const bool retained = route[row] != 0;
+    if (dv_in)
+        for (int j = 0; j < nj; ++j) dv[row * d + lane + 32 * j] = from_f32<T>(dv_in[row * d + lane + 32 * j]);
+    for (int which = 0; which < 2; ++which) {
+        const T *src = (which ? k : q) + row * d;
+        const float *gin = (which ? dk_in : dq_la) + row * d;
+        T *gout = (which ? dk : dq) + row * d;
+        float x[4], g[4], ssg[4], xgg[4], out[4], ss_all = 0.f, xg_all = 0.f;
+        for (int j = 0; j < nj; ++j) {
+            x[j] = to_f32(src[lane + 32 * j]);
+            g[j] = gin[lane + 32 * j];
+            out[j] = 0.f;
+        }
+        const bool l2_part = which == 0 || !retained, rms_part = which == 0 || retained;
+        if (l2_part) {
+            for (int j = 0; j < nj; ++j) {
+                ss_all = fmaf(x[j], x[j], ss_all);
+                xg_all = fmaf(x[j], g[j], xg_all);
+            }
+            ss_all = warp_sum(ss_all);
+            xg_all = warp_sum(xg_all);
+            const float r = rsqrtf(ss_all + norm_eps), dot = r * xg_all;
+            for (int j = 0; j < nj; ++j) out[j] = r * (g[j] - x[j] * r * dot);
+        }
+        if (rms_part) {
+            float gs[4];
+            for (int j = 0; j < nj; ++j) {
+                gs[j] = which == 0 ? dq_sm[row * d + lane + 32 * j] : g[j];
+                ssg[j] = warp_sum(x[j] * x[j]);
+                xgg[j] = warp_sum(x[j] * gs[j]);
+            }
+            for (int j = 0; j < nj; ++j) {
+                float ss = 0.f, xg = 0.f;
+                for (int y = 0; y < nj; ++y)
+                    if ((32 * y) / ds == (32 * j) / ds) { ss += ssg[y]; xg += xgg[y]; }
+                const float r = rsqrtf(ss / ds + norm_eps), m = r * xg / ds;
+                out[j] += r * (gs[j] - x[j] * r * m);
+            }
+        }
+        for (int j = 0; j < nj; ++j) gout[lane + 32 * j] = from_f32<T>(out[j]);
     }
 }
 
@@ -540,10 +601,32 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
                    out, o_nla, lse, br, s, st);
 }
 
-cudaError_t launch_qk_norm_f32(const float *q, const float *k, float *q_la, float *k_la, float *q_sm,
+cudaError_t launch_qk_norm_f32(const void *q, const void *k, bool bf16, float *q_la, float *k_la, float *q_sm,
                                float *k_sm, size_t rows, int d, int G, float norm_eps, cudaStream_t st) {
-    qk_norm_f32_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(q, k, q_la, k_la, q_sm, k_sm, rows, d, G,
-                                                                  norm_eps);
+    const unsigned blocks = (unsigned)((rows + 7) / 8);
+    if (bf16)
+        qk_norm_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
+                                                                 q_la, k_la, q_sm, k_sm, rows, d, G, norm_eps);
+    else
+        qk_norm_f32_kernel<float><<<blocks, 256, 0, st>>>((const float *)q, (const float *)k, q_la, k_la, q_sm,
+                                                         k_sm, rows, d, G, norm_eps);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_qk_norm_bwd_f32(const void *q, const void *k, bool bf16, const uint8_t *route,
+                                   const float *dq_la, const float *dq_sm, const float *dk_in,
+                                   const float *dv_in, void *dq, void *dk, void *dv, size_t rows, int d, int G,
+                                   float norm_eps, cudaStream_t st) {
+    const unsigned blocks = (unsigned)((rows + 7) / 8);
+    if (bf16)
+        qk_norm_bwd_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
+            (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, route, dq_la, dq_sm, dk_in, dv_in,
+            (__nv_bfloat16 *)dq, (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, rows, d, G, norm_eps);
+    else
+        qk_norm_bwd_f32_kernel<float><<<blocks, 256, 0, st>>>((const float *)q, (const float *)k, route, dq_la,
+                                                             dq_sm, dk_in, dv_in, (float *)dq, (float *)dk,
+                                                             (float *)dv, rows, d, G, norm_eps);
     count_launch();
     return cudaGetLastError();
 }

@@ -71,8 +71,17 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
 // (G > 1: grouped softmax heads, fp32 storage only; see HeadGroups)
 // fp32 storage: q, k [rows, d] -> L2-normalised rows (q_la, k_la) and rows with each of the G slices
 // RMS-normalised (q_sm, k_sm)
-cudaError_t launch_qk_norm_f32(const float *q, const float *k, float *q_la, float *k_la, float *q_sm,
+cudaError_t launch_qk_norm_f32(const void *q, const void *k, bool bf16, float *q_la, float *k_la, float *q_sm,
                                float *k_sm, size_t rows, int d, int G, float norm_eps, cudaStream_t st);
+// (q, k in fp32 or bf16 storage; q_sm, k_sm may be nullptr)
+// Its backward, in place: dq (gradient w.r.t. the L2 copy) and dq_sm (w.r.t. the RMS copy) -> dq;
+// dk (w.r.t. the L2 copy for a linear token, the RMS copy for a retained one) -> dk.
+cudaError_t launch_qk_norm_bwd_f32(const void *q, const void *k, bool bf16, const uint8_t *route,
+                                   const float *dq_la, const float *dq_sm, const float *dk_in,
+                                   const float *dv_in, void *dq, void *dk, void *dv, size_t rows, int d, int G,
+                                   float norm_eps, cudaStream_t st);
+// (fp32 gradients in: dq_la, dq_sm, dk_in, and dv_in or nullptr; out in the storage type: dq, dk, and dv =
+// dv_in converted when given.  In place is fine for fp32 storage: dq_la == dq, dk_in == dk.)
 
 // softmax_tc.cu -- tensor-core softmax branch + combination (bf16 storage)
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
@@ -101,7 +110,10 @@ cudaError_t launch_softmax_bwd_tc(const void *q, void *Qh, const void *dO16, con
                                   const int32_t *sm_chunk_prefix, const float *lse, const float *Dsm,
                                   float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
                                   float *dmask, bool qh_ready, int32_t *status, Shape s, cudaStream_t st,
-                                  cudaStream_t st_kv);   // st: query-side kernel, st_kv: key-side kernel
+                                  cudaStream_t st_kv,    // st: query-side kernel, st_kv: key-side kernel
+                                  HeadGroups hg = HeadGroups{});
+// (hg.G = 2 at d = 128: softmax heads are column slices, lse / Dsm [B,H,G,L]; hg.norm_eps >= 0: Qh is
+// written here as the slice-wise RMS-normalised q, k16 must hold the normalised keys already)
 
 // gdn_tc.cu -- tensor-core chunkwise Gated DeltaNet (bf16 storage): intermediates in workspace
 struct GdnTcWs {
@@ -177,14 +189,15 @@ cudaError_t launch_to_f32(const void *a, const void *b, const void *c, float *a3
 cudaError_t launch_combine_bwd(const float *o_la, const float *o_nla, const void *dout,
                                const float *w, float eps, float *do_la, float *do_nla, float *dw,
                                float *Dsm, void *do16, void *dola16, void *dolag16, const float *Gd,
-                               float scale_la, const int32_t *gsc, Shape s, cudaStream_t st);
+                               float scale_la, const int32_t *gsc, Shape s, cudaStream_t st, int G = 1);
+// (G > 1: the softmax branch's output was normalised per slice of d / G columns; Dsm is [B,H,G,L])
 // max |dout| (n elements) into word kGradAmaxWord of the status page (zeroed first)
 cudaError_t launch_dout_amax(const void *dout, size_t n, bool bf16, int32_t *status, cudaStream_t st);
 cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const float *v_sm32, int cap,
                                const int32_t *sm_idx, const int32_t *sm_chunk_prefix,
                                const float *do_nla, const float *lse, const float *Dsm,
                                float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm, Shape s,
-                               cudaStream_t st, float *dmask = nullptr);
+                               cudaStream_t st, float *dmask = nullptr, int G = 1);
 // (dmask [B,H,cap] or nullptr: per retained key the sum of the mask gradients of Section 4.2)
 // Block-level routing, fp32: the softmax branch's backward through the own block of the queries of a
 // linear block (adds to dq_sm, writes the dk_x / dv_x rows of the linear blocks).  gsc: gradient

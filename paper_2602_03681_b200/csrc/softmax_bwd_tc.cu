@@ -48,7 +48,10 @@ template <int D> struct QLayout {
     static constexpr int kTmem = D == 64 ? 256 : 512;     // S 64 + dP 64 + dQ D
 };
 
-template <int D>
+// kG softmax heads per linear head (Section 4.3, grouped heads): a CTA's head is then one slice of D
+// columns of rows of kG D columns -- the x coordinate of every copy and the column offset of every
+// store --, the lists of retained tokens are the linear head's, lse and Dsm are [B,H,kG,L].
+template <int D, int kG>
 __global__ void __launch_bounds__(kThreadsB)
 softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B*H*L][D] fp16, box 128
                          const __grid_constant__ CUtensorMap map_do,   // dO16 [B*H*L][D] fp16, box 128
@@ -65,7 +68,7 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NP = (L + 127) / 128, NC = L / kC;
     const int p = NP - 1 - (int)blockIdx.x;
-    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    const int bhg = blockIdx.y, bh = bhg / kG, x0 = (bhg % kG) * D, b = bh / H, h = bh % H;
     const int32_t *pre = sm_chunk_prefix + (size_t)bh * (NC + 1);
     const int n_full = min(pre[2 * p], cap), n_end = min(pre[min(2 * p + 2, NC)], cap);
     const int T = (n_end + 63) / 64;
@@ -101,8 +104,8 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
         if (lane == 0 && T > 0) {      // nothing is loaded for a tile that sees no retained key
             mbar_arrive_expect_tx(&ms.barQ, 2 * SL::kQ);
             for (int kb = 0; kb < KB; ++kb) {
-                tma_load_2d(smem + SL::oQ + kb * 16384, &map_q, &ms.barQ, kb * 64, bh * L + p * 128);
-                tma_load_2d(smem + SL::oDO + kb * 16384, &map_do, &ms.barQ, kb * 64, bh * L + p * 128);
+                tma_load_2d(smem + SL::oQ + kb * 16384, &map_q, &ms.barQ, x0 + kb * 64, bh * L + p * 128);
+                tma_load_2d(smem + SL::oDO + kb * 16384, &map_do, &ms.barQ, x0 + kb * 64, bh * L + p * 128);
             }
             int t = 0;
             for (; t < T; ++t) {
@@ -110,9 +113,9 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
                 if (!mbar_wait(&ms.empty[s], ((t / SL::kStages) & 1) ^ 1, abort_flag)) break;
                 mbar_arrive_expect_tx(&ms.full[s], 2 * SL::kKV);
                 for (int kb = 0; kb < KB; ++kb) {
-                    tma_load_2d(smem + SL::oK + s * SL::kKV + kb * 8192, &map_k, &ms.full[s], kb * 64,
+                    tma_load_2d(smem + SL::oK + s * SL::kKV + kb * 8192, &map_k, &ms.full[s], x0 + kb * 64,
                                 bh * cap + t * 64);
-                    tma_load_2d(smem + SL::oV + s * SL::kKV + kb * 8192, &map_v, &ms.full[s], kb * 64,
+                    tma_load_2d(smem + SL::oV + s * SL::kKV + kb * 8192, &map_v, &ms.full[s], x0 + kb * 64,
                                 bh * cap + t * 64);
                 }
             }
@@ -172,8 +175,8 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
         const bool row_ok = i_abs < L;
         const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
         const float sl2 = scale_sm * kLog2e;
-        const float lse2 = row_ok ? lse[(size_t)bh * L + i_abs] * kLog2e : 0.f;
-        const float Di = row_ok ? Dsm[(size_t)bh * L + i_abs] : 0.f;
+        const float lse2 = row_ok ? lse[(size_t)bhg * L + i_abs] * kLog2e : 0.f;
+        const float Di = row_ok ? Dsm[(size_t)bhg * L + i_abs] : 0.f;
         bool ok = true;
         // The compacted keys are in position order, so row i sees exactly the first `cnt` of them
         // (a per-element look-up of the key's position costs a divergent branch per element).
@@ -225,7 +228,7 @@ softmax_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh  [B
         }
         if (ok) {
             const float gi = grad_scale(status).y;          // dO and Dsm arrive times the gradient scale
-            float4 *dst = reinterpret_cast<float4 *>(dq_sm + (((size_t)b * L + i_abs) * H + h) * D);
+            float4 *dst = reinterpret_cast<float4 *>(dq_sm + (((size_t)b * L + i_abs) * H + h) * (D * kG) + x0);
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t x[32];
@@ -265,7 +268,7 @@ template <int D> struct KLayout {
     static constexpr int kTmem = D == 64 ? 256 : 512;     // S^T 64 + dP^T 64 + dV D + dK D
 };
 
-template <int D, bool kMask>       // kMask: also the per-key sums of the mask gradient (dmask)
+template <int D, bool kMask, int kG>   // kMask: also the per-key sums of the mask gradient (dmask); kG: as above
 __global__ void __launch_bounds__(kThreadsB)
 softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B*H*L][D], box 64
                           const __grid_constant__ CUtensorMap map_do,   // dO16, box 64
@@ -283,7 +286,7 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
     MiscB &ms = *reinterpret_cast<MiscB *>(smem + SL::oMisc);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NC = L / kC;
-    const int kt = blockIdx.x, bh = blockIdx.y;
+    const int kt = blockIdx.x, bhg = blockIdx.y, bh = bhg / kG, x0 = (bhg % kG) * D;
     const int n_sm = min(sm_chunk_prefix[(size_t)bh * (NC + 1) + NC], cap);
     if (kt * 128 >= n_sm) return;                        // uniform: no retained key in this tile
     const int first_pos = sm_idx[(size_t)bh * L + kt * 128];
@@ -317,8 +320,8 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
         if (lane == 0) {
             mbar_arrive_expect_tx(&ms.barQ, 2 * SL::kKV);
             for (int kb = 0; kb < KB; ++kb) {
-                tma_load_2d(smem + SL::oK + kb * 16384, &map_k, &ms.barQ, kb * 64, bh * cap + kt * 128);
-                tma_load_2d(smem + SL::oV + kb * 16384, &map_v, &ms.barQ, kb * 64, bh * cap + kt * 128);
+                tma_load_2d(smem + SL::oK + kb * 16384, &map_k, &ms.barQ, x0 + kb * 64, bh * cap + kt * 128);
+                tma_load_2d(smem + SL::oV + kb * 16384, &map_v, &ms.barQ, x0 + kb * 64, bh * cap + kt * 128);
             }
             int t = 0;
             for (; t < T; ++t) {
@@ -326,9 +329,9 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
                 if (!mbar_wait(&ms.empty[s], ((t >> 1) & 1) ^ 1, abort_flag)) break;
                 mbar_arrive_expect_tx(&ms.full[s], 2 * SL::kQ);
                 for (int kb = 0; kb < KB; ++kb) {
-                    tma_load_2d(smem + SL::oQ + s * SL::kQ + kb * 8192, &map_q, &ms.full[s], kb * 64,
+                    tma_load_2d(smem + SL::oQ + s * SL::kQ + kb * 8192, &map_q, &ms.full[s], x0 + kb * 64,
                                 bh * L + (qt0 + t) * 64);
-                    tma_load_2d(smem + SL::oDO + s * SL::kQ + kb * 8192, &map_do, &ms.full[s], kb * 64,
+                    tma_load_2d(smem + SL::oDO + s * SL::kQ + kb * 8192, &map_do, &ms.full[s], x0 + kb * 64,
                                 bh * L + (qt0 + t) * 64);
                 }
             }
@@ -400,8 +403,8 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
             // the previous tile's values is not overtaken (the barrier below separates t from t + 2)
             float *lse2 = ms.lse2[t & 1], *dsum = ms.dsum[t & 1];
             if (r < 64) {
-                lse2[r] = lse[(size_t)bh * L + i0 + r] * kLog2e;
-                dsum[r] = Dsm[(size_t)bh * L + i0 + r];
+                lse2[r] = lse[(size_t)bhg * L + i0 + r] * kLog2e;
+                dsum[r] = Dsm[(size_t)bhg * L + i0 + r];
             }
             named_barrier_sync(1, kRowsB);
             ok = mbar_wait(&ms.barS, t & 1, abort_flag);
@@ -452,10 +455,10 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
             tc_fence_after_sync();
         }
         if (ok) {      // the TMEM loads are warp-wide: only the stores depend on the key being real
-            float4 *dv_dst = reinterpret_cast<float4 *>(dv_sm + ((size_t)bh * cap + j) * D);
-            float4 *dk_dst = reinterpret_cast<float4 *>(dk_sm + ((size_t)bh * cap + j) * D);
+            float4 *dv_dst = reinterpret_cast<float4 *>(dv_sm + ((size_t)bh * cap + j) * (D * kG) + x0);
+            float4 *dk_dst = reinterpret_cast<float4 *>(dk_sm + ((size_t)bh * cap + j) * (D * kG) + x0);
             const float gi = grad_scale(status).y;          // dO and Dsm arrive times the gradient scale
-            if (kMask && key_ok) dmask[(size_t)bh * cap + j] = gi * msum;
+            if (kMask && key_ok) dmask[(size_t)bhg * cap + j] = gi * msum;
 #pragma unroll
             for (int cb = 0; cb < D / 32; ++cb) {
                 uint32_t x[32], y[32];
@@ -482,10 +485,13 @@ softmax_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap map_q,    // Qh [B
     if (tid == 0 && ms.abort_flag) atomicMin(status, (int)NATSL_ERR_TIMEOUT);
 }
 
-// q (bf16, [B,L,H,d]) -> fp16 [B,H,L,d]; 8 values per thread.
+// q (bf16, [B,L,H,d]) -> fp16 [B,H,L,d]; 8 values per thread.  norm_eps >= 0: each of the `groups` slices
+// of a row RMS-normalised on the way (Section 4.3: the softmax operation's q; a slice's pieces sit in
+// neighbouring lanes).
 template <int D>
 __global__ void __launch_bounds__(256)
-to_f16_bhld_kernel(const __nv_bfloat16 *__restrict__ q, __half *__restrict__ qh, int B, int L, int H) {
+to_f16_bhld_kernel(const __nv_bfloat16 *__restrict__ q, __half *__restrict__ qh, int B, int L, int H,
+                   int groups, float norm_eps) {
     constexpr int kPieces = D / 8;
     const size_t idx = (size_t)blockIdx.x * 256 + threadIdx.x;
     const size_t total = (size_t)B * L * H * kPieces;
@@ -498,47 +504,62 @@ to_f16_bhld_kernel(const __nv_bfloat16 *__restrict__ q, __half *__restrict__ qh,
     const uint4 u = reinterpret_cast<const uint4 *>(q)[idx];
     const uint32_t wv[4] = {u.x, u.y, u.z, u.w};
     uint32_t o[4];
+    float rq = 1.f;
+    if (norm_eps >= 0.f) {         // (the grid covers whole rows, so all lanes of a row are here)
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float lo = __uint_as_float(wv[i] << 16), hi = __uint_as_float(wv[i] & 0xffff0000u);
+            ss = fmaf(lo, lo, fmaf(hi, hi, ss));
+        }
+        const int lanes = kPieces / groups;
+        const unsigned row_mask = ((1u << kPieces) - 1u) << ((threadIdx.x & 31) & ~(kPieces - 1));
+        for (int off = 1; off < lanes; off <<= 1) ss += __shfl_xor_sync(row_mask, ss, off);
+        rq = rsqrtf(ss * groups / D + norm_eps);
+    }
 #pragma unroll
     for (int i = 0; i < 4; ++i)
-        o[i] = pack_half2(__uint_as_float(wv[i] << 16), __uint_as_float(wv[i] & 0xffff0000u));
+        o[i] = pack_half2(__uint_as_float(wv[i] << 16) * rq, __uint_as_float(wv[i] & 0xffff0000u) * rq);
     reinterpret_cast<uint4 *>(qh)[(((size_t)b * H + h) * L + l) * kPieces + pc] =
         make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 }  // namespace
 
-template <int D>
+template <int D, int G>      // D: columns of a softmax head, G of them per linear head (s.d = D G)
 static cudaError_t softmax_bwd_tc_impl(const void *q, void *Qh, const void *dO16, const void *k16,
                                        const void *v16, int cap, const int32_t *sm_idx,
                                        const int32_t *pre, const float *lse, const float *Dsm,
                                        float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
                                        float *dmask, bool qh_ready, int32_t *status, Shape s,
-                                       cudaStream_t st, cudaStream_t st_kv) {
+                                       cudaStream_t st, cudaStream_t st_kv, float norm_eps) {
     const uint64_t BH = (uint64_t)s.B * s.H;
-    if (!qh_ready) {      // (the linear branch's prepare kernel leaves the same fp16 copy of q behind)
-        const size_t pieces = (size_t)s.B * s.L * s.H * (D / 8);
-        to_f16_bhld_kernel<D><<<(unsigned)((pieces + 255) / 256), 256, 0, st>>>(
-            (const __nv_bfloat16 *)q, (__half *)Qh, s.B, s.L, s.H);
+    constexpr int DL = D * G;
+    if (!qh_ready) {      // (the linear branch's prepare kernel leaves the same fp16 copy of q behind --
+                          //  unless q is normalised, differently for the two operations)
+        const size_t pieces = (size_t)s.B * s.L * s.H * (DL / 8);
+        to_f16_bhld_kernel<DL><<<(unsigned)((pieces + 255) / 256), 256, 0, st>>>(
+            (const __nv_bfloat16 *)q, (__half *)Qh, s.B, s.L, s.H, G, norm_eps);
         count_launch();
     }
     CUtensorMap mq128, mdo128, mk64, mv64, mq64, mdo64, mk128, mv128;
-    if (!tch::make_map_2d(&mq128, Qh, BH * s.L, D, 128) || !tch::make_map_2d(&mdo128, dO16, BH * s.L, D, 128) ||
-        !tch::make_map_2d(&mk64, k16, BH * cap, D, 64) || !tch::make_map_2d(&mv64, v16, BH * cap, D, 64) ||
-        !tch::make_map_2d(&mq64, Qh, BH * s.L, D, 64) || !tch::make_map_2d(&mdo64, dO16, BH * s.L, D, 64) ||
-        !tch::make_map_2d(&mk128, k16, BH * cap, D, 128) || !tch::make_map_2d(&mv128, v16, BH * cap, D, 128))
+    if (!tch::make_map_2d(&mq128, Qh, BH * s.L, DL, 128) || !tch::make_map_2d(&mdo128, dO16, BH * s.L, DL, 128) ||
+        !tch::make_map_2d(&mk64, k16, BH * cap, DL, 64) || !tch::make_map_2d(&mv64, v16, BH * cap, DL, 64) ||
+        !tch::make_map_2d(&mq64, Qh, BH * s.L, DL, 64) || !tch::make_map_2d(&mdo64, dO16, BH * s.L, DL, 64) ||
+        !tch::make_map_2d(&mk128, k16, BH * cap, DL, 128) || !tch::make_map_2d(&mv128, v16, BH * cap, DL, 128))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(softmax_bwd_dq_tc_kernel<D>,
+    cudaError_t e = cudaFuncSetAttribute(softmax_bwd_dq_tc_kernel<D, G>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, QLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
-    auto dkv = dmask ? softmax_bwd_dkv_tc_kernel<D, true> : softmax_bwd_dkv_tc_kernel<D, false>;
+    auto dkv = dmask ? softmax_bwd_dkv_tc_kernel<D, true, G> : softmax_bwd_dkv_tc_kernel<D, false, G>;
     e = cudaFuncSetAttribute(dkv, cudaFuncAttributeMaxDynamicSharedMemorySize, KLayout<D>::kTotal);
     if (e != cudaSuccess) return e;
-    dim3 gq((s.L + 127) / 128, s.B * s.H);
-    softmax_bwd_dq_tc_kernel<D><<<gq, kThreadsB, QLayout<D>::kTotal, st>>>(
+    dim3 gq((s.L + 127) / 128, s.B * s.H * G);
+    softmax_bwd_dq_tc_kernel<D, G><<<gq, kThreadsB, QLayout<D>::kTotal, st>>>(
         mq128, mdo128, mk64, mv64, cap, sm_idx, pre, lse, Dsm, scale_sm, dq_sm, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    dim3 gk((s.L + 127) / 128, s.B * s.H);
+    dim3 gk((s.L + 127) / 128, s.B * s.H * G);
     dkv<<<gk, kThreadsB, KLayout<D>::kTotal, st_kv>>>(
         mq64, mdo64, mk128, mv128, cap, sm_idx, pre, lse, Dsm, scale_sm, dk_sm, dv_sm, dmask, status, s.L, s.H, debug_wait_kcycles());
     count_launch();
@@ -550,12 +571,17 @@ cudaError_t launch_softmax_bwd_tc(const void *q, void *Qh, const void *dO16, con
                                   const int32_t *sm_chunk_prefix, const float *lse, const float *Dsm,
                                   float scale_sm, float *dq_sm, float *dk_sm, float *dv_sm,
                                   float *dmask, bool qh_ready, int32_t *status, Shape s,
-                                  cudaStream_t st, cudaStream_t st_kv) {
+                                  cudaStream_t st, cudaStream_t st_kv, HeadGroups hg) {
+    if (hg.norm_eps >= 0.f && qh_ready) return cudaErrorInvalidValue;   // (the copy at hand is the linear operation's)
+    if (hg.G == 2 && s.d == 128)
+        return softmax_bwd_tc_impl<64, 2>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm, scale_sm,
+                                          dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st, st_kv, hg.norm_eps);
+    if (hg.G > 1) return cudaErrorInvalidValue;
     if (s.d == 128)
-        return softmax_bwd_tc_impl<128>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm,
-                                        scale_sm, dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st, st_kv);
-    return softmax_bwd_tc_impl<64>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm,
-                                   scale_sm, dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st, st_kv);
+        return softmax_bwd_tc_impl<128, 1>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm, scale_sm,
+                                           dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st, st_kv, hg.norm_eps);
+    return softmax_bwd_tc_impl<64, 1>(q, Qh, dO16, k16, v16, cap, sm_idx, sm_chunk_prefix, lse, Dsm, scale_sm,
+                                      dq_sm, dk_sm, dv_sm, dmask, qh_ready, status, s, st, st_kv, hg.norm_eps);
 }
 
 }  // namespace natsl

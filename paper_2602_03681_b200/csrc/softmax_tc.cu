@@ -589,7 +589,9 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
                             pack_half2(f[4] * rk, f[5] * rk), pack_half2(f[6] * rk, f[7] * rk));
         }
         reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
-        if (dk16) {
+        if (dk16 && norm_eps >= 0.f) {
+            *dk16 = kk;                                   // already fp16
+        } else if (dk16) {
             const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
             uint32_t ko[4];
 #pragma unroll

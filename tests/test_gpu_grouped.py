@@ -7,6 +7,8 @@ on the same seeded inputs:
 * bf16 storage (tensor-core kernels): d = 128 with G = 2 -- six linear heads with twelve softmax heads,
   the appendix's smaller model -- and G = 1 with normalisation, on shapes that take the one-pass scan,
   and the segmented scan;
+* the backward for fp32 storage and for bf16 storage at d = 128, including the Jacobians of the two
+  normalisations;
 * requests that are not built come back as NATSL_ERR_UNSUPPORTED, before any launch.
 """
 import dataclasses
@@ -98,6 +100,91 @@ def test_bf16_tensor_cores(G, norm, B, H, L, flags):
     check(wl, got, ref, TOL["bf16"], G)
 
 
+@pytest.mark.parametrize("d,G,norm,B,H,L,states", [
+    (64, 2, True, 1, 3, 256, False),
+    (128, 4, True, 1, 2, 192, True),
+    (128, 2, False, 2, 2, 128, False),
+    (64, 1, True, 1, 2, 192, True),
+    (128, 2, True, 1, 2, 256, False),
+])
+def test_fp32_storage_backward(d, G, norm, B, H, L, states):
+    """Backward with grouped heads and the normalisation's Jacobians (fp32 storage) against the gradients
+    of the oracle's definition, with and without a carried state and its gradient."""
+    from paper_2602_03681_b200 import binding
+    from test_gpu_parity import check_bwd
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg0_f32_tiny_fwd"], d=d, seed=51 + d + G)
+    x = make_inputs(wl, B, H, L, norm)
+    scale_sm = (d / G) ** -0.5 if norm else wl.scale_sm
+    r = np.random.default_rng(6)
+    s0 = (0.1 * r.standard_normal((B, H, d, d))).astype(np.float32) if states else None
+    dso = (0.05 * r.standard_normal((B, H, d, d))).astype(np.float32) if states else None
+    p = binding.make_params(B, H, L, d, binding.NATSL_F32, wl.scale_la, scale_sm, w=dev(x["w"]),
+                            flags=binding.QK_NORM if norm else 0, G=G, norm_eps=1e-6)
+    keep = [dev(a) for a in (s0, dso) if a is not None]
+    dstate_in = torch.empty((B, H, d, d), device="cuda")
+    if states:
+        p.state_in, p.dstate_out, p.dstate_in = keep[0].data_ptr(), keep[1].data_ptr(), dstate_in.data_ptr()
+    w_dev = dev(x["w"])
+    p.w = w_dev.data_ptr()
+    ws = binding.alloc_workspace(p, binding.OP_BWD)
+    t = {n: dev(x[n]) for n in ("q", "k", "v", "g", "beta", "route", "dout")}
+    outs = {n: torch.empty_like(t["q"]) for n in ("dq", "dk", "dv")}
+    outs.update(dg=torch.empty_like(t["g"]), dbeta=torch.empty_like(t["g"]),
+                dw=torch.empty((B, L, H, 2), device="cuda"))
+    binding.natsl_hybrid_bwd(t["q"], t["k"], t["v"], t["g"], t["beta"], t["route"], t["dout"], outs["dq"], outs["dk"],
+                             outs["dv"], outs["dg"], outs["dbeta"], outs["dw"], p, ws)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(ws) == 0
+    got = {n: v.cpu().numpy() for n, v in outs.items()}
+    ref = grouped.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"], G=G,
+                             qk_norm=norm, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6,
+                             state_in=s0, dstate_out=dso)
+    check_bwd(wl, got, ref, TOL["f32"])
+    if states:
+        assert rel_err(dstate_in.cpu().numpy(), ref["dstate_in"]) <= TOL["f32"]
+    if norm:      # Euler: a normalised layer's gradient is orthogonal to every q and k row
+        for n in ("q", "k"):
+            dot = np.abs((got["d" + n].astype(np.float64) * x[n]).sum(-1))
+            scale = np.sqrt((got["d" + n].astype(np.float64) ** 2).sum(-1) * (x[n].astype(np.float64) ** 2).sum(-1))
+            assert (dot <= 1e-3 * scale + 1e-9).all()
+
+
+@pytest.mark.parametrize("G,norm,B,H,L", [
+    (2, True, 1, 6, 256),        # six linear heads x two softmax heads
+    (2, False, 2, 2, 320),
+    (1, True, 1, 3, 192),
+    (2, True, 2, 3, 384),
+])
+def test_bf16_tensor_cores_backward(G, norm, B, H, L):
+    """Backward at d = 128 on tensor cores (softmax branch's kernels on column slices, reverse scan on the
+    L2-normalised copies, chunk-level products as tile GEMMs, Jacobians of the normalisations last)."""
+    from test_gpu_parity import check_bwd
+    from paper_2602_03681_b200 import binding
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg1_bf16_prefill"], seed=61 + G + B)
+    x = make_inputs(wl, B, H, L, norm)
+    scale_sm = (wl.d / G) ** -0.5 if norm else wl.scale_sm
+    dt = torch.bfloat16
+    p = binding.make_params(B, H, L, wl.d, binding.NATSL_BF16, wl.scale_la, scale_sm,
+                            flags=binding.QK_NORM if norm else 0, G=G, norm_eps=1e-6)
+    w_dev = dev(x["w"])
+    p.w = w_dev.data_ptr()
+    ws = binding.alloc_workspace(p, binding.OP_BWD)
+    t = {n: dev(x[n], dt) for n in ("q", "k", "v", "dout")}
+    t.update({n: dev(x[n]) for n in ("g", "beta", "route")})
+    outs = {n: torch.empty_like(t["q"]) for n in ("dq", "dk", "dv")}
+    outs.update(dg=torch.empty_like(t["g"]), dbeta=torch.empty_like(t["g"]),
+                dw=torch.empty((B, L, H, 2), device="cuda"))
+    binding.natsl_hybrid_bwd(t["q"], t["k"], t["v"], t["g"], t["beta"], t["route"], t["dout"], outs["dq"], outs["dk"],
+                             outs["dv"], outs["dg"], outs["dbeta"], outs["dw"], p, ws)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(ws) == 0
+    got = {n: v.float().cpu().numpy() for n, v in outs.items()}
+    ref = grouped.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"], G=G,
+                             qk_norm=norm, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6)
+    # (with the normalisation the q, k rows differ in length by up to 16 x, and so do their gradient rows)
+    check_bwd(wl, got, ref, TOL["bf16"], large_only=not norm)
+
+
 def test_normalisation_ignores_row_lengths_on_the_device():
     """Rescaling the q and k rows by powers of two changes no bf16 mantissa, so with norm_eps = 0 the
     normalised layer must return almost the same bits."""
@@ -139,11 +226,16 @@ def test_requests_that_are_not_built_are_refused():
     assert refused(lambda: binding.hybrid_fwd(*args, flags=binding.QK_NORM, want=("cache",), **kw))
     with pytest.raises(binding.NatslError):                                                       # G must divide d
         binding.hybrid_fwd(*args, G=3, **kw)
-    p = binding.make_params(1, 2, 128, 128, binding.NATSL_BF16, wl.scale_la, wl.scale_sm, G=2)
+    # backward: bf16 storage at d = 64 (the fused chunk kernel's path) has no normalisation
+    wl4 = inputs.WORKLOADS["cfg4_bf16_train"]
+    x4 = make_inputs(wl4, 1, 2, 128, False)
+    a4 = [dev(x4[n], torch.bfloat16) for n in ("q", "k", "v")] + [dev(x4["g"]), dev(x4["beta"]), dev(x4["route"])]
+    p = binding.make_params(1, 2, 128, 64, binding.NATSL_BF16, wl4.scale_la, wl4.scale_sm, flags=binding.QK_NORM,
+                            norm_eps=1e-6)
     n = binding.natsl_workspace_size(p, binding.OP_BWD)
     ws = torch.zeros(n, dtype=torch.uint8, device="cuda")
-    outs = [torch.empty_like(args[0]) for _ in range(3)] + [torch.empty_like(args[3]) for _ in range(2)]
+    outs = [torch.empty_like(a4[0]) for _ in range(3)] + [torch.empty_like(a4[3]) for _ in range(2)]
     dw = torch.empty((1, 128, 2, 2), device="cuda")
     with pytest.raises(binding.NatslError) as e:
-        binding.natsl_hybrid_bwd(*args[:6], args[0], *outs, dw, p, ws)
+        binding.natsl_hybrid_bwd(*a4, a4[0], *outs, dw, p, ws)
     assert e.value.status == binding.ERR_UNSUPPORTED

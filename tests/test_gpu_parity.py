@@ -56,12 +56,15 @@ def half_ulp_bf16(x):
     return 2.0 ** (e - 8)
 
 
-def check_stored(got, ref, tol, storage, name="out"):
+def check_stored(got, ref, tol, storage, name="out", large_only=True):
     """A tensor stored in the workload's storage type: the computed value must be within
     tol * RMS of the oracle; storing it in bf16 adds at most half a bf16 ulp on top, which by
     itself already exceeds 2e-2 * RMS for the few elements with |x| >= 4.  Returns how many
     elements needed that allowance; each of them must be a large one, whose half ulp is at least
-    half the plain bound (for the layer output, RMS about 0.77, that means |ref| >= 2)."""
+    half the plain bound (for the layer output, RMS about 0.77, that means |ref| >= 2).
+    large_only=False drops that last requirement, for tensors whose rows differ in scale by an order of
+    magnitude (gradients through a normalisation of rows of very different lengths), where "large" measured
+    against the whole tensor's RMS says nothing about an element of a small row."""
     ref = np.asarray(ref, np.float64)
     err = np.abs(np.asarray(got, np.float64) - ref)
     plain = tol * np.sqrt((ref ** 2).mean())
@@ -69,7 +72,7 @@ def check_stored(got, ref, tol, storage, name="out"):
     worst = (err / bound).max()
     assert worst <= 1.0, (name, worst, rel_err(got, ref))
     needed = err > plain
-    if storage == "bf16" and tol >= 1e-2:     # (a caller with a tighter tolerance lives on the allowance)
+    if storage == "bf16" and tol >= 1e-2 and large_only:     # (a caller with a tighter tolerance lives on the allowance)
         assert np.all(half_ulp_bf16(ref[needed]) >= 0.5 * plain), (name, "allowance used by a small element")
     return int(needed.sum())
 
@@ -252,9 +255,9 @@ def run_bwd(wl, x, w="given", flags=0):
     return {n: t.float().cpu().numpy() for n, t in res.items() if n != "ws"}
 
 
-def check_bwd(wl, got, ref, tol):
+def check_bwd(wl, got, ref, tol, large_only=True):
     for name in ("dq", "dk", "dv"):
-        check_stored(got[name], ref[name], tol, wl.dtype, name)
+        check_stored(got[name], ref[name], tol, wl.dtype, name, large_only)
     for name in ("dg", "dbeta", "dw"):
         e = rel_err(got[name], ref[name])
         assert e <= tol, (name, e)
