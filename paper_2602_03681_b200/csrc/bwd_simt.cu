@@ -154,7 +154,7 @@ dout_amax_kernel(const T *__restrict__ dout, size_t n4, int32_t *status) {
 // G > 1 (grouped softmax heads, Section 4.3): the softmax branch's output is normalised per slice of
 // D / G columns, so its part of the backward (do_nla, dw_nla, D_i = <do_i, o_i>) is formed per slice;
 // Dsm is then [B,H,G,L].
-template <typename T, int D>
+template <typename T, int D, bool kGrouped>     // kGrouped: G > 1 (one reduction per 32-column group instead of per row)
 __global__ void __launch_bounds__(kThreads)
 combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_nla,
                    const T *__restrict__ dout, const float *__restrict__ w, float eps,
@@ -170,51 +170,67 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
     const int h = row % H;
     const size_t bl = row / H;
     const int l = bl % L, b = bl / L;
-    const int ds = D / G;                    // columns per softmax head (a multiple of 32)
-    float ol[kCols], on[kCols], dy[kCols], ssl = 0.f, ssn[kCols];
+    const int ds = kGrouped ? D / G : D;     // columns per softmax head: 32, 64 or 128
+    const int gsh = 26 - __clz(ds);          // 32-column group x belongs to slice x >> gsh
+    // sum over the lanes and over the 32-column groups of x's slice (ungrouped: over the whole row, one reduction)
+    auto slice_sums = [&](const float (&v)[kCols], float (&out)[kCols]) {
+        if (!kGrouped) {
+            float t = 0.f;
+#pragma unroll
+            for (int x = 0; x < kCols; ++x) t += v[x];
+            t = warp_sum(t);
+#pragma unroll
+            for (int x = 0; x < kCols; ++x) out[x] = t;
+        } else {
+            float part[kCols];
+#pragma unroll
+            for (int x = 0; x < kCols; ++x) part[x] = warp_sum(v[x]);
+#pragma unroll
+            for (int x = 0; x < kCols; ++x) {
+                float t = 0.f;
+#pragma unroll
+                for (int y = 0; y < kCols; ++y) t += (y >> gsh) == (x >> gsh) ? part[y] : 0.f;
+                out[x] = t;
+            }
+        }
+    };
+    float ol[kCols], on[kCols], dy[kCols], ssl = 0.f, sq[kCols], ssn[kCols];
 #pragma unroll
     for (int x = 0; x < kCols; ++x) {
         const size_t i = row * D + lane + 32 * x;
         ol[x] = o_la[i]; on[x] = o_nla[i]; dy[x] = to_f32(dout[i]);
         ssl = fmaf(ol[x], ol[x], ssl);
-        ssn[x] = warp_sum(on[x] * on[x]);     // sum of squares of this 32-column group
+        sq[x] = on[x] * on[x];
     }
     ssl = warp_sum(ssl);
+    slice_sums(sq, ssn);
     const float fl = rsqrtf(ssl / D + eps);
     float fn[kCols];                          // RMS factor of the slice a 32-column group belongs to
 #pragma unroll
-    for (int x = 0; x < kCols; ++x) {
-        float t = 0.f;
-#pragma unroll
-        for (int y = 0; y < kCols; ++y) t += (32 * y) / ds == (32 * x) / ds ? ssn[y] : 0.f;
-        fn[x] = rsqrtf(t / ds + eps);
-    }
+    for (int x = 0; x < kCols; ++x) fn[x] = rsqrtf(ssn[x] * (1.f / ds) + eps);
     const float wn = w ? w[row * 2] : 0.5f, wl = w ? w[row * 2 + 1] : 0.5f;
     // scale_la gamma_l of the token (decay from its chunk's entry), for the reverse scan's operand
     const float sg = dolag16 ? scale_la * Gd[((size_t)(b * H + h) * (L / kC) + l / kC) * 128 + l % kC] : 0.f;
-    float dwl = 0.f, dwn_g[kCols];
+    float dwl = 0.f, dyn[kCols], dwn_s[kCols];
 #pragma unroll
     for (int x = 0; x < kCols; ++x) {
         dwl = fmaf(dy[x], ol[x] * fl, dwl);
-        dwn_g[x] = warp_sum(dy[x] * on[x] * fn[x]);
+        dyn[x] = dy[x] * on[x] * fn[x];
     }
     dwl = warp_sum(dwl);
-    float dwn = 0.f, mn[kCols];               // mn: w_nla <dy, y_nla> / ds over the group's slice
+    slice_sums(dyn, dwn_s);                   // <dy, y_nla> over the group's slice
+    float dwn = 0.f;
 #pragma unroll
-    for (int x = 0; x < kCols; ++x) {
-        dwn += dwn_g[x];
-        float t = 0.f;
-#pragma unroll
-        for (int y = 0; y < kCols; ++y) t += (32 * y) / ds == (32 * x) / ds ? dwn_g[y] : 0.f;
-        mn[x] = wn * t / ds;
-    }
+    for (int x = 0; x < kCols; ++x)           // ... and over the row: each slice counted once
+        if (!kGrouped ? x == 0 : (x & ((1 << gsh) - 1)) == 0) dwn += dwn_s[x];
     const float ml = wl * dwl / D;
-    float dsm_g[kCols];
+    float dno[kCols], dsm_s[kCols];
 #pragma unroll
     for (int x = 0; x < kCols; ++x) {
         const size_t i = row * D + lane + 32 * x;
+        const float mn = wn * dwn_s[x] * (1.f / ds);
         const float dl = fl * (wl * dy[x] - ol[x] * fl * ml);
-        const float dn = fn[x] * (wn * dy[x] - on[x] * fn[x] * mn[x]);
+        const float dn = fn[x] * (wn * dy[x] - on[x] * fn[x] * mn);
         do_la[i] = dl;
         if (do_nla) do_nla[i] = dn;   // (the tensor-core softmax backward reads the fp16 copy only)
         const size_t i16 = ((((size_t)b * H + h) * L + l) * D) + lane + 32 * x;
@@ -223,15 +239,20 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
             dola16[i16] = __float2half_rn(gs * dl);
             dolag16[i16] = __float2half_rn(gs * sg * dl);
         }
-        dsm_g[x] = warp_sum(dn * on[x]);
+        dno[x] = dn * on[x];
     }
+    slice_sums(dno, dsm_s);
     if (lane == 0) {
         if (dw) { dw[row * 2] = dwn; dw[row * 2 + 1] = dwl; }
-        for (int g = 0; g < G; ++g) {
-            float t = 0.f;
+        if (!kGrouped) {
+            Dsm[((size_t)b * H + h) * L + l] = gs * dsm_s[0];
+        } else {
+            for (int g = 0; g < G; ++g) {
+                float t = 0.f;
 #pragma unroll
-            for (int x = 0; x < kCols; ++x) t += (32 * x) / ds == g ? dsm_g[x] : 0.f;
-            Dsm[(((size_t)b * H + h) * G + g) * L + l] = gs * t;
+                for (int x = 0; x < kCols; ++x) t = (x >> gsh) == g ? dsm_s[x] : t;
+                Dsm[(((size_t)b * H + h) * G + g) * L + l] = gs * t;
+            }
         }
     }
 }
@@ -863,7 +884,8 @@ static cudaError_t combine_bwd_impl(const float *o_la, const float *o_nla, const
                                     const float *Gd, float scale_la, const int32_t *gsc, Shape s,
                                     cudaStream_t st, int G) {
     const size_t rows = (size_t)s.B * s.L * s.H;
-    combine_bwd_kernel<T, D><<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
+    auto kernel = G > 1 ? combine_bwd_kernel<T, D, true> : combine_bwd_kernel<T, D, false>;
+    kernel<<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
         o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, (__half *)do16, (__half *)dola16,
         (__half *)dolag16, Gd, scale_la, gsc, G, s.B, s.L, s.H);
     count_launch();
