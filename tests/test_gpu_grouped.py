@@ -100,6 +100,14 @@ def test_bf16_tensor_cores(G, norm, B, H, L, flags):
     check(wl, got, ref, TOL["bf16"], G)
 
 
+def test_bf16_tensor_cores_d64_normalisation():
+    """The normalisation alone at d = 64 (one softmax head per linear head, the 64-column kernels)."""
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg4_bf16_train"], seed=47)
+    x = make_inputs(wl, 2, 3, 448, True)
+    got, ref = run_both(wl, x, 1, True, wl.d ** -0.5)
+    check(wl, got, ref, TOL["bf16"], 1)
+
+
 @pytest.mark.parametrize("d,G,norm,B,H,L,states", [
     (64, 2, True, 1, 3, 256, False),
     (128, 4, True, 1, 2, 192, True),
