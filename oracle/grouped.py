@@ -36,7 +36,7 @@ def rms_normalise(x, norm_eps):
     return x / torch.sqrt((x * x).mean(-1, keepdim=True) + norm_eps)
 
 
-def _forward(q, k, v, g, beta, route, w, G, qk_norm, scale_la, scale_sm, eps, norm_eps, state_in):
+def _forward(q, k, v, g, beta, route, w, G, qk_norm, scale_la, scale_sm, eps, norm_eps, state_in, block=None):
     B, L, H, d = q.shape
     ds = d // G
     lin = (route == 0).to(q.dtype)                       # [B,L,H]: 1 for linear tokens
@@ -46,12 +46,24 @@ def _forward(q, k, v, g, beta, route, w, G, qk_norm, scale_la, scale_sm, eps, no
     S = state_in if state_in is not None else q.new_zeros((B, H, d, d))
     o_la = []
     for i in range(L):
+        if block and i % block == 0:
+            S_start, decay = S, torch.ones_like(g[:, i])  # state and decay since the block began
         S = torch.exp(g[:, i])[:, :, None, None] * S     # decay on every token
         ki, vi = k_la[:, i], v[:, i]
         err = vi - torch.einsum("bha,bhac->bhc", ki, S)
-        bt = (beta[:, i] * lin[:, i])[:, :, None, None]  # softmax tokens do not write the state
+        if block:
+            # block-level routing (Section 4.1): the decision is known only at the block's end, so
+            # every token of the block runs the delta rule ...
+            bt = beta[:, i][:, :, None, None]
+            decay = decay * torch.exp(g[:, i])
+        else:
+            bt = (beta[:, i] * lin[:, i])[:, :, None, None]  # softmax tokens do not write the state
         S = S + bt * ki[:, :, :, None] * err[:, :, None, :]
         o_la.append(scale_la * torch.einsum("bha,bhac->bhc", q_la[:, i], S))
+        if block and i % block == block - 1:
+            # ... and a softmax block's update is rolled back: only the decay remains
+            keep = lin[:, i][:, :, None, None]
+            S = keep * S + (1 - keep) * decay[:, :, None, None] * S_start
     o_la = torch.stack(o_la, 1)                          # [B,L,H,d]
     # ---- softmax operation: G heads per linear head, keys = retained tokens j <= i ----
     qs, ks, vs = (x.reshape(B, L, H, G, ds) for x in (q, k, v))
@@ -60,6 +72,9 @@ def _forward(q, k, v, g, beta, route, w, G, qk_norm, scale_la, scale_sm, eps, no
     logits = scale_sm * torch.einsum("blhsa,bmhsa->bhslm", qs, ks)          # [B,H,G,L(query),L(key)]
     causal = torch.tril(torch.ones((L, L), dtype=torch.bool))
     vis = causal[None, None] & (route != 0).permute(0, 2, 1)[:, :, None, :]  # [B,H,L,L]
+    if block:         # both operations read the query's own block
+        blk = torch.arange(L) // block
+        vis = vis | (causal & (blk[:, None] == blk[None, :]))[None, None]
     vis = vis[:, :, None]                                                    # same for every head of the group
     neg = torch.full_like(logits, -np.inf)
     masked = torch.where(vis, logits, neg)
@@ -88,30 +103,35 @@ def _t(a, grad=False):
     return x.requires_grad_(grad)
 
 
-def _check(q, route, G):
+def _check(q, route, G, block=None):
     B, L, H, d = q.shape
     if G < 1 or d % G:
         raise ValueError("G must divide the head dimension")
     if route.shape != (B, L, H):
         raise ValueError("route must be [B,L,H]")
+    if block:
+        r = np.asarray(route).reshape(B, L // block, block, H) if L % block == 0 else None
+        if r is None or (r != r[:, :, :1]).any():
+            raise ValueError("block mode: route must be constant within each block")
 
 
 def hybrid_fwd(q, k, v, g, beta, route, w=None, *, G=1, qk_norm=False, scale_la, scale_sm, eps=1e-5,
-               norm_eps=1e-6, state_in=None):
+               norm_eps=1e-6, state_in=None, block=None):
     """q,k,v [B,L,H,d]; g,beta,route [B,L,H]; w [B,L,H,2] or None; G softmax heads per linear head.
+    block=R: block-level routing (route constant per block of R tokens, Section 4.1).
     Returns dict(out, o_la, o_nla [B,L,H,d]; lse [B,H,G,L]; state_out [B,H,d,d]) as numpy float64."""
-    _check(np.asarray(q), np.asarray(route), G)
+    _check(np.asarray(q), np.asarray(route), G, block)
     with torch.no_grad():
         res = _forward(_t(q), _t(k), _t(v), _t(g), _t(beta), torch.from_numpy(np.asarray(route).astype(np.int64)),
-                       _t(w), G, qk_norm, scale_la, scale_sm, eps, norm_eps, _t(state_in))
+                       _t(w), G, qk_norm, scale_la, scale_sm, eps, norm_eps, _t(state_in), block)
     return {n: x.numpy() for n, x in res.items()}
 
 
 def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, G=1, qk_norm=False, scale_la, scale_sm, eps=1e-5,
-               norm_eps=1e-6, state_in=None, dstate_out=None):
+               norm_eps=1e-6, state_in=None, dstate_out=None, block=None):
     """Gradients of <out, dout> (+ <state_out, dstate_out>) with respect to q, k, v, g, beta, w and
     state_in.  Returns dict(dq, dk, dv, dg, dbeta, dw, dstate_in)."""
-    _check(np.asarray(q), np.asarray(route), G)
+    _check(np.asarray(q), np.asarray(route), G, block)
     B, L, H, d = np.asarray(q).shape
     if w is None:
         w = np.full((B, L, H, 2), 0.5)
@@ -120,7 +140,7 @@ def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, G=1, qk_norm=False, scale_la
     leaves = [_t(x, True) for x in (q, k, v, g, beta, w, state_in)]
     tq, tk, tv, tg, tb, tw, ts = leaves
     res = _forward(tq, tk, tv, tg, tb, torch.from_numpy(np.asarray(route).astype(np.int64)), tw, G, qk_norm,
-                   scale_la, scale_sm, eps, norm_eps, ts)
+                   scale_la, scale_sm, eps, norm_eps, ts, block)
     loss = (res["out"] * _t(dout)).sum()
     if dstate_out is not None:
         loss = loss + (res["state_out"] * _t(dstate_out)).sum()

@@ -173,6 +173,53 @@ def test_backward_finite_differences():
             assert abs(fd - gr[gname][idx]) <= 1e-5 * max(1.0, abs(fd)), (n, idx, fd, gr[gname][idx])
 
 
+def block_route(B, L, H, R, p, seed):
+    r = np.random.default_rng(seed)
+    return np.repeat((r.random((B, L // R, H)) < p).astype(np.uint8), R, axis=1)
+
+
+def test_block_mode_with_one_head_per_group_is_the_c_oracles_block_mode():
+    B, L, H, d, R = 2, 96, 2, 16, 16
+    x = rand_inputs(B, L, H, d, seed=28)
+    x["route"] = block_route(B, L, H, R, 0.4, 1)
+    r = np.random.default_rng(3)
+    s0 = 0.1 * r.standard_normal((B, H, d, d))
+    a = gf(x, G=1, state_in=s0, block=R)
+    b = oracle.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], state_in=s0, block=R, **KW)
+    for n in ("out", "o_la", "o_nla", "state_out"):
+        np.testing.assert_allclose(a[n], b[n], rtol=1e-9, atol=1e-11, err_msg=n)
+    dout = r.standard_normal(x["q"].shape)
+    ds = 0.05 * r.standard_normal(s0.shape)
+    ga = gb(x, dout, G=1, state_in=s0, dstate_out=ds, block=R)
+    gc = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], dout, state_in=s0,
+                           dstate_out=ds, block=R, **KW)
+    for n in ("dq", "dk", "dv", "dg", "dbeta", "dw", "dstate_in"):
+        np.testing.assert_allclose(ga[n], gc[n], rtol=1e-8, atol=1e-10, err_msg=n)
+    # and it is not the token-level layer
+    assert np.abs(a["out"] - gf(x, G=1, state_in=s0)["out"]).max() > 1e-3
+
+
+def test_block_mode_group_heads_are_block_mode_heads_over_column_slices():
+    B, L, H, d, R, G = 1, 64, 2, 16, 16, 2
+    x = rand_inputs(B, L, H, d, seed=29, unit=False)
+    x["route"] = block_route(B, L, H, R, 0.5, 2)
+    a = gf(x, G=G, scale_sm=0.4, block=R)
+    sl = {n: x[n].reshape(B, L, H * G, d // G) for n in ("q", "k", "v")}
+    rep = {n: np.repeat(x[n], G, axis=2) for n in ("g", "beta", "route")}
+    b = oracle.hybrid_fwd(sl["q"], sl["k"], sl["v"], rep["g"], rep["beta"], rep["route"], None, scale_la=0.5,
+                          scale_sm=0.4, block=R)
+    np.testing.assert_allclose(a["o_nla"], b["o_nla"].reshape(B, L, H, d), rtol=1e-10, atol=1e-12)
+    c = oracle.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], scale_la=0.5,
+                          scale_sm=0.4, block=R)
+    np.testing.assert_allclose(a["o_la"], c["o_la"], rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(a["state_out"], c["state_out"], rtol=1e-9, atol=1e-11)
+    with pytest.raises(ValueError):
+        y = dict(x)
+        y["route"] = x["route"].copy()
+        y["route"][0, 3, 0] ^= 1
+        gf(y, G=G, block=R)
+
+
 def test_rejects_group_count_that_does_not_divide():
     x = rand_inputs(1, 8, 1, 8, seed=27)
     with pytest.raises(ValueError):
