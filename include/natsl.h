@@ -178,13 +178,13 @@ typedef struct natsl_params {
                             /*   those columns of the softmax output, which is RMS-normalised per      */
                             /*   slice; the linear operation, its state and the two weights stay per   */
                             /*   head h over all d columns.  p->lse becomes [B,H,G,L].                 */
-                            /*   Built: natsl_hybrid_fwd with token-level routing, for fp32 storage    */
-                            /*   (d / G in {32, 64, 128}) and on the tensor-core path for d = 128,     */
-                            /*   G = 2 (the appendix's two softmax heads per linear head; three would  */
-                            /*   need d = 192); natsl_hybrid_bwd for the same shapes except bf16       */
-                            /*   storage with d = 64 (self-contained call, token-level routing).       */
-                            /*   G > 1 or NATSL_QK_NORM with anything else (decode,                    */
-                            /*   NATSL_BLOCK_ROUTING, NATSL_APPEND_CACHE, NATSL_SAVE_FOR_BWD /         */
+                            /*   Built: natsl_hybrid_fwd with token-level and block-level routing, for */
+                            /*   fp32 storage (d / G in {32, 64, 128}) and on the tensor-core path for */
+                            /*   d = 128, G = 2 (the appendix's two softmax heads per linear head;     */
+                            /*   three would need d = 192); natsl_hybrid_bwd with token-level routing  */
+                            /*   for the same shapes except bf16 storage with d = 64 (self-contained   */
+                            /*   call).  G > 1 or NATSL_QK_NORM with anything else (decode, backward   */
+                            /*   with NATSL_BLOCK_ROUTING, NATSL_APPEND_CACHE, NATSL_SAVE_FOR_BWD /    */
                             /*   NATSL_SAVED_FWD, NATSL_FORCE_SIMT on bf16, NATSL_QK_NORM with         */
                             /*   p->k_sm): NATSL_ERR_UNSUPPORTED.                                      */
     float norm_eps;         /* NATSL_QK_NORM: epsilon under the square roots, >= 0                     */

@@ -471,7 +471,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     if (append && !want_cache) return NATSL_ERR_NULL;
     const HeadGroups hg = head_groups(p);
     if (grouped_or_normed(p)) {
-        if (block || append || (p->flags & NATSL_SAVE_FOR_BWD)) return NATSL_ERR_UNSUPPORTED;
+        if (append || (p->flags & NATSL_SAVE_FOR_BWD)) return NATSL_ERR_UNSUPPORTED;
         if ((p->flags & NATSL_QK_NORM) && want_cache) return NATSL_ERR_UNSUPPORTED;   // (the cache would hold normalised keys)
         if (tensor_cores) {
             if (hg.G > 1 && !(hg.G == 2 && p->d == 128)) return NATSL_ERR_UNSUPPORTED;
@@ -581,8 +581,10 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gdn_scan_simt(q_la, k_la, g, f.W, f.U, f.P, p->scale_la, p->state_in,
                                        p->state_out, nullptr, nullptr, o_la, br.route, s, st));
         NATSL_TRY(mark());
+        // (an own-block tile of block-level routing reads the layer's keys: the softmax operation's copy)
         NATSL_TRY(launch_softmax_combine_simt(q_sm, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
-                                              p->scale_sm, p->eps, out, p->o_nla, p->lse, br, s, st, hg.G));
+                                              p->scale_sm, p->eps, out, p->o_nla, p->lse,
+                                              BlockRouting{br.route, k_nsm, v}, s, st, hg.G));
     }
     NATSL_TRY(mark());
 #undef NATSL_TRY

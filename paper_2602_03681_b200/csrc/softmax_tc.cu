@@ -65,7 +65,7 @@ template <int D> struct SmLayout {
 };
 
 struct Misc {                    // lives in the last kMiscBytes of the CTA's shared memory
-    uint64_t barQ, barQn, fullK[kStages], emptyK[kStages], fullV[kStages], emptyV[kStages], barS[2], barP, barO, barE;
+    uint64_t barQ, barQn, barKn, fullK[kStages], emptyK[kStages], fullV[kStages], emptyV[kStages], barS[2], barP, barO, barE;
     uint32_t tmem_base;
     int abort_flag, wait_kcycles;   // in this order: the waits read the limit as abort_flag[1]
     alignas(16) int pos[kBM];    // positions of the retained tokens inside the CTA's own chunks
@@ -132,6 +132,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     if (tid == 0) {
         mbar_init(&ms.barQ, 1);
         mbar_init(&ms.barQn, kSoftmaxThreads);       // normalised queries written (NATSL_QK_NORM)
+        mbar_init(&ms.barKn, 1);                     // ... and the keys of an own-block tile (one phase per tile)
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ms.fullK[s], 1); mbar_init(&ms.emptyK[s], 1);
             mbar_init(&ms.fullV[s], 1); mbar_init(&ms.emptyV[s], 1);
@@ -241,15 +242,21 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 mma_commit(&ms.emptyK[t % kStages]);
                 mma_commit(&ms.barS[t & 1]);
             };
+            // (normalisation with block-level routing: an own-block tile's keys arrive raw and are
+            // normalised in place by the softmax threads first; barKn completes one phase per such tile)
+            auto own_keys_ready = [&](int t) {
+                return !(kBlock && kNorm) || t < T || mbar_wait(&ms.barKn, (t - T) & 1, abort_flag);
+            };
             bool ok = mbar_wait(&ms.barQ, 0, abort_flag) && (!kNorm || mbar_wait(&ms.barQn, 0, abort_flag)) &&
-                      mbar_wait(&ms.fullK[0], 0, abort_flag);
+                      mbar_wait(&ms.fullK[0], 0, abort_flag) && own_keys_ready(0);
             if (ok) {
                 tc_fence_after_sync();
                 issue_qk(0);
             }
             for (int t = 0; ok && t < T2; ++t) {
                 if (t + 1 < T2) {
-                    ok = mbar_wait(&ms.fullK[(t + 1) % kStages], ((t + 1) / kStages) & 1, abort_flag);
+                    ok = mbar_wait(&ms.fullK[(t + 1) % kStages], ((t + 1) / kStages) & 1, abort_flag) &&
+                         own_keys_ready(t + 1);
                     if (!ok) break;
                     tc_fence_after_sync();
                     issue_qk(t + 1);
@@ -322,7 +329,54 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
         // all n_full earlier ones plus those of the CTA's own chunks at positions <= i.
         int cnt = n_full;
         for (int kq = 0; kq < n_end - n_full; ++kq) cnt += ms.pos[kq] <= i_abs ? 1 : 0;
+        // Keys of own-block tile u (block-level routing with normalisation): raw bf16 rows from the layer's
+        // k; threads 0-63 rewrite one row each as fp16 of the RMS-normalised row.
+        auto normalise_own_keys = [&](int u) -> bool {
+            if (!mbar_wait(&ms.fullK[u % kStages], (u / kStages) & 1, abort_flag)) return false;
+            if (tid < kBN) {
+                uint8_t *rowp = smem + SL::oK + (u % kStages) * SL::kKStage + tid * 128;
+                float ss = 0.f;
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint4 a = *reinterpret_cast<const uint4 *>(rowp + kb * kBN * 128 + ((c ^ (tid & 7)) << 4));
+                        const uint32_t wd[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float lo = __uint_as_float(wd[e] << 16), hi = __uint_as_float(wd[e] & 0xffff0000u);
+                            ss = fmaf(lo, lo, fmaf(hi, hi, ss));
+                        }
+                    }
+                const float rk = rsqrtf(ss / D + norm_eps);
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        uint4 *pp = reinterpret_cast<uint4 *>(rowp + kb * kBN * 128 + ((c ^ (tid & 7)) << 4));
+                        const uint4 a = *pp;
+                        const uint32_t wd[4] = {a.x, a.y, a.z, a.w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            o[e] = pack_half2(__uint_as_float(wd[e] << 16) * rk, __uint_as_float(wd[e] & 0xffff0000u) * rk);
+                        *pp = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+            }
+            // One arrival per tile, after all rows are written.  (With one arrival per thread, the threads
+            // that have no row to write reached the next tile's arrival while the others were still
+            // writing this tile's rows, and completed this tile's phase for them.)
+            fence_proxy_async_smem();
+            named_barrier_sync(2, kSoftmaxThreads);
+            if (tid == 0) mbar_arrive(&ms.barKn);
+            return true;
+        };
+        if (kBlock && kNorm && ok && T2 > 0 && T == 0) ok = normalise_own_keys(0);
         for (int t = 0; ok && t < T2; ++t) {
+            if (kBlock && kNorm && t + 1 < T2 && t + 1 >= T) {      // (before this tile's logits are waited for)
+                ok = normalise_own_keys(t + 1);
+                if (!ok) break;
+            }
             ok = mbar_wait(&ms.barS[t & 1], (t >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after_sync();
@@ -633,13 +687,10 @@ static cudaError_t softmax_tc_impl(const void *q, const void *k_sm, const void *
     if (br.route && (!tch::make_map_blhd(&mkd, br.k, s.B, s.L, s.H * G, D, kBN) ||
                      !tch::make_map_blhd(&mvd, br.v, s.B, s.L, s.H * G, D, kBN)))
         return cudaErrorInvalidValue;
-    // (block-level routing is built without grouping and without normalisation only)
     auto kernel = softmax_combine_tc_kernel<D, false, G, false>;
     if (norm_eps >= 0.f) kernel = softmax_combine_tc_kernel<D, false, G, true>;
-    if (br.route) {
-        if (G > 1 || norm_eps >= 0.f) return cudaErrorInvalidValue;
-        kernel = softmax_combine_tc_kernel<D, true, 1, false>;
-    }
+    if (br.route) kernel = norm_eps >= 0.f ? softmax_combine_tc_kernel<D, true, G, true>
+                                          : softmax_combine_tc_kernel<D, true, G, false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SL::kTotal);
     if (e != cudaSuccess) return e;
     // With emit_flags the kernel is launched as a programmatic dependent of the kernel before it in

@@ -24,8 +24,9 @@ from test_gpu_parity import TOL, check_stored, dev, rel_err, tdtype
 pytestmark = pytest.mark.gpu
 
 
-def make_inputs(wl, B, H, L, unnormalised):
-    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L)
+def make_inputs(wl, B, H, L, unnormalised, block_p=None):
+    route = None if block_p is None else inputs.route_blocks(wl.seed, (B, L, H), block_p)
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L, route=route)
     if unnormalised:      # rows of very different lengths: the normalisation has something to do
         r = np.random.default_rng(wl.seed + 100)
         for n in ("q", "k"):
@@ -35,10 +36,10 @@ def make_inputs(wl, B, H, L, unnormalised):
     return x
 
 
-def run_both(wl, x, G, norm, scale_sm, norm_eps=1e-6, flags=0):
+def run_both(wl, x, G, norm, scale_sm, norm_eps=1e-6, flags=0, block=False):
     from paper_2602_03681_b200 import binding
     dt = tdtype(wl)
-    f = flags | (binding.QK_NORM if norm else 0)
+    f = flags | (binding.QK_NORM if norm else 0) | (binding.BLOCK_ROUTING if block else 0)
     res = binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]), dev(x["beta"]),
                              dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la, scale_sm=scale_sm,
                              want=("o_la", "o_nla", "lse", "state_out"), flags=f, G=G, norm_eps=norm_eps)
@@ -46,7 +47,8 @@ def run_both(wl, x, G, norm, scale_sm, norm_eps=1e-6, flags=0):
     assert binding.natsl_device_status(res["ws"]) == 0
     got = {n: t.float().cpu().numpy() for n, t in res.items() if n != "ws"}
     ref = grouped.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], G=max(G, 1),
-                             qk_norm=norm, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=norm_eps)
+                             qk_norm=norm, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=norm_eps,
+                             block=64 if block else None)
     return got, ref
 
 
@@ -98,6 +100,28 @@ def test_bf16_tensor_cores(G, norm, B, H, L, flags):
     scale_sm = (wl.d / G) ** -0.5 if norm else wl.scale_sm
     got, ref = run_both(wl, x, G, norm, scale_sm, flags=flags)
     check(wl, got, ref, TOL["bf16"], G)
+
+
+@pytest.mark.parametrize("storage,d,G,norm,B,H,L,p", [
+    ("f32", 64, 2, True, 1, 2, 256, 0.4),
+    ("f32", 128, 2, False, 1, 2, 192, 0.5),
+    ("bf16", 128, 2, True, 1, 6, 512, 0.3),      # the paper's mode: one decision per block, grouped heads, normalised q, k
+    ("bf16", 128, 2, True, 2, 3, 320, 0.6),      # ragged last query tile
+    ("bf16", 128, 2, False, 1, 3, 384, 0.4),
+    ("bf16", 128, 1, True, 1, 2, 256, 0.0),      # all blocks linear: every tile is an own-block tile
+    ("bf16", 64, 1, True, 2, 2, 256, 0.4),
+])
+def test_block_level_routing_with_grouped_heads(storage, d, G, norm, B, H, L, p):
+    """Block-level routing (Section 4.1) together with grouped heads and the normalisation: the own-block
+    tile of a linear block reads the layer's own keys, which the kernel normalises in shared memory."""
+    base = "cfg0_f32_tiny_fwd" if storage == "f32" else ("cfg1_bf16_prefill" if d == 128 else "cfg4_bf16_train")
+    wl = dataclasses.replace(inputs.WORKLOADS[base], d=d, seed=71 + d + G)
+    x = make_inputs(wl, B, H, L, norm, block_p=p)
+    if p == 0.0:
+        x["route"][:] = 0
+    scale_sm = (d / G) ** -0.5 if norm else wl.scale_sm
+    got, ref = run_both(wl, x, G, norm, scale_sm, block=True)
+    check(wl, got, ref, TOL[storage], G)
 
 
 def test_bf16_tensor_cores_d64_normalisation():
@@ -229,7 +253,6 @@ def test_requests_that_are_not_built_are_refused():
         return e.value.status == binding.ERR_UNSUPPORTED
 
     assert refused(lambda: binding.hybrid_fwd(*args, G=4, **kw))                                  # d/G = 32 on tensor cores
-    assert refused(lambda: binding.hybrid_fwd(*args, G=2, flags=binding.BLOCK_ROUTING, **kw))
     assert refused(lambda: binding.hybrid_fwd(*args, G=2, flags=binding.FORCE_SIMT, **kw))        # bf16 on CUDA cores
     assert refused(lambda: binding.hybrid_fwd(*args, flags=binding.QK_NORM, want=("cache",), **kw))
     with pytest.raises(binding.NatslError):                                                       # G must divide d
