@@ -181,12 +181,12 @@ typedef struct natsl_params {
                             /*   Built: natsl_hybrid_fwd with token-level and block-level routing, for */
                             /*   fp32 storage (d / G in {32, 64, 128}) and on the tensor-core path for */
                             /*   d = 128, G = 2 (the appendix's two softmax heads per linear head;     */
-                            /*   three would need d = 192); natsl_hybrid_bwd with token-level routing  */
-                            /*   for the same shapes except bf16 storage with d = 64 (self-contained   */
-                            /*   call).  G > 1 or NATSL_QK_NORM with anything else (decode, backward   */
-                            /*   with NATSL_BLOCK_ROUTING, NATSL_APPEND_CACHE, NATSL_SAVE_FOR_BWD /    */
-                            /*   NATSL_SAVED_FWD, NATSL_FORCE_SIMT on bf16, NATSL_QK_NORM with         */
-                            /*   p->k_sm): NATSL_ERR_UNSUPPORTED.                                      */
+                            /*   three would need d = 192); natsl_hybrid_bwd with either routing for   */
+                            /*   the same shapes except bf16 storage with d = 64 (self-contained call, */
+                            /*   no p->dscore).  G > 1 or NATSL_QK_NORM with anything else (decode,    */
+                            /*   NATSL_APPEND_CACHE, NATSL_SAVE_FOR_BWD / NATSL_SAVED_FWD,             */
+                            /*   NATSL_FORCE_SIMT on bf16, NATSL_QK_NORM with p->k_sm):                */
+                            /*   NATSL_ERR_UNSUPPORTED.                                                */
     float norm_eps;         /* NATSL_QK_NORM: epsilon under the square roots, >= 0                     */
 } natsl_params;
 

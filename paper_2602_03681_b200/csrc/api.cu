@@ -188,7 +188,8 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.sm_len = c.take<int32_t>(B * H);
     f.k_sm32 = tm(!tcs); f.v_sm32 = tm(!tcs);
     f.q32 = tm(general); f.k32 = tm(general); f.v32 = tm(general);
-    const bool normed = !tcs && (p->flags & NATSL_QK_NORM);
+    // (needed by the fp32 softmax kernels: all of them for fp32 storage, the own-block one of block-level routing)
+    const bool normed = (p->flags & NATSL_QK_NORM) && (!tcs || (general && block));
     f.qs32 = tm(normed); f.ks32 = tm(normed);
     const size_t Gg = p->G > 1 ? (size_t)p->G : 1;           // softmax heads per linear head: lse, Dsm per softmax head
     f.W = tm(general); f.U = tm(general);
@@ -338,8 +339,9 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
     const HeadGroups hg = head_groups(p);
     const float *qs = f.q32, *ks = f.k32;
     if (hg.norm_eps >= 0.f) {
-        NATSL_TRY(launch_qk_norm_f32(q, k, s.bf16, f.q32, f.k32, tensor_cores ? nullptr : f.qs32,
-                                     tensor_cores ? nullptr : f.ks32, (size_t)(B * L * H), p->d, hg.G,
+        const bool rms_copies = !tensor_cores || block;
+        NATSL_TRY(launch_qk_norm_f32(q, k, s.bf16, f.q32, f.k32, rms_copies ? f.qs32 : nullptr,
+                                     rms_copies ? f.ks32 : nullptr, (size_t)(B * L * H), p->d, hg.G,
                                      hg.norm_eps, st));
         if (!tensor_cores) { qs = f.qs32; ks = f.ks32; }
     }
@@ -375,7 +377,7 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
     else
         NATSL_TRY(launch_softmax_combine_simt(qs, f.k_sm32, f.v_sm32, p->L, f.sm_idx, f.prefix,
                                               f.o_la, p->w, p->scale_sm, p->eps, out, f.o_nla,
-                                              f.lse, BlockRouting{block_route, f.k32, f.v32}, s32, st, hg.G));
+                                              f.lse, BlockRouting{block_route, ks, f.v32}, s32, st, hg.G));
 #undef NATSL_TRY
     return NATSL_OK;
 }
@@ -602,7 +604,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (p->flags & NATSL_APPEND_CACHE) return NATSL_ERR_UNSUPPORTED;
     const HeadGroups hg = head_groups(p);
     if (grouped_or_normed(p)) {      // grouped heads, q/k normalisation: the paths with separate chunk-level products
-        if (p->flags & (NATSL_BLOCK_ROUTING | NATSL_SAVED_FWD)) return NATSL_ERR_UNSUPPORTED;
+        if ((p->flags & NATSL_SAVED_FWD) || p->dscore) return NATSL_ERR_UNSUPPORTED;
         if (use_tensor_cores(p)) {
             if (p->d != 128 || hg.G > 2) return NATSL_ERR_UNSUPPORTED;
         } else {
@@ -728,11 +730,16 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         // Every token has a softmax-branch dk, dv: the retained tokens' from the compacted gradients, the
         // tokens of linear blocks' from their own block (each token is written by exactly one of the
         // two); the assembly adds them to the linear branch's.
+        // (With the normalisation the own-block kernel reads the softmax operation's copies of q and k, and
+        // dk_x -- a gradient with respect to that copy -- stays apart from the linear branch's dk until the
+        // normalisations' backward.)
         NATSL_TRY(launch_gdn_finish(a, f.dk_x, f.dv_x, s32, st, false));
-        NATSL_TRY(launch_softmax_bwd_own_block_simt(f.q32, f.k32, f.v32, f.do_nla, f.lse, f.Dsm, route,
-                                                    p->scale_sm, f.dq_sm, f.dk_x, f.dv_x, gsc, s32, st));
-        a.dk_x = f.dk_x;
+        NATSL_TRY(launch_softmax_bwd_own_block_simt(normed ? f.qs32 : f.q32, normed ? f.ks32 : f.k32, f.v32,
+                                                    f.do_nla, f.lse, f.Dsm, route, p->scale_sm, f.dq_sm, f.dk_x,
+                                                    f.dv_x, gsc, s32, st, hg.G));
+        a.dk_x = normed ? nullptr : f.dk_x;
         a.dv_x = f.dv_x;
+        a.no_scatter = true;
     }
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, s, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, s, st));
@@ -760,12 +767,14 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     } else if (!s.bf16) {
         NATSL_TRY(launch_gdn_assemble(a, dq, dk, dv, s, st));
         NATSL_TRY(launch_qk_norm_bwd_f32(q, k, false, route, (const float *)dq, f.dq_sm, (const float *)dk, nullptr,
-                                         dq, dk, nullptr, (size_t)(B * L * H), p->d, hg.G, hg.norm_eps, st));
+                                         dq, dk, nullptr, (size_t)(B * L * H), p->d, hg.G, hg.norm_eps, st,
+                                         general_block ? f.dk_x : nullptr));
     } else {
         float *dq32 = f.dW, *dk32 = f.W, *dv32 = f.U;
         NATSL_TRY(launch_gdn_assemble(a, dq32, dk32, dv32, s32, st));
         NATSL_TRY(launch_qk_norm_bwd_f32(q, k, true, route, dq32, f.dq_sm, dk32, dv32, dq, dk, dv,
-                                         (size_t)(B * L * H), p->d, hg.G, hg.norm_eps, st));
+                                         (size_t)(B * L * H), p->d, hg.G, hg.norm_eps, st,
+                                         general_block ? f.dk_x : nullptr));
     }
     if (p->dscore)   // softmax blocks: the mask gradients of their keys; linear blocks: the kappa of their tokens
         NATSL_TRY(launch_dscore(route, f.prefix, f.dmask, nullptr, f.kappa, p->L, p->dscore, s, st));

@@ -464,7 +464,9 @@ softmax_bwd_dkv_kernel(const float *__restrict__ q32, const float *__restrict__ 
 //   block have no other softmax-branch gradient).  grid = (L/64, B*H); softmax blocks return.
 // Dsm arrives times the gradient scale of the tensor-core kernels (gsc; 1 without them).
 // ------------------------------------------------------------------------------------------
-template <int D>
+// G softmax heads per linear head: a CTA's head is a slice of D columns of rows of DL = G D columns;
+// lse and Dsm are [B,H,G,L]; q32, k32 are the softmax operation's copies of q and k.
+template <int D, int G>
 __global__ void __launch_bounds__(kThreads)
 softmax_bwd_own_block_simt_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
                                   const float *__restrict__ v32, const float *__restrict__ do_nla,
@@ -479,14 +481,15 @@ softmax_bwd_own_block_simt_kernel(const float *__restrict__ q32, const float *__
     float *dOs = Vs + kC * (D + 1);
     float *Ps = dOs + kC * (D + 1);          // [64][65]
     float *dSs = Ps + kC * (kC + 1);         // [64][65]
-    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
-    const size_t ts = (size_t)H * D;
+    constexpr int DL = D * G;
+    const int c = blockIdx.x, bhg = blockIdx.y, bh = bhg / G, col0 = (bhg % G) * D, b = bh / H, h = bh % H;
+    const size_t ts = (size_t)H * DL;
     const size_t tok0 = ((size_t)b * L + (size_t)c * kC) * H + h;
     if (route[tok0]) return;                 // a softmax block: its tokens are retained ones
     const float ginv = grad_scale(gsc).y;
     for (int idx = threadIdx.x; idx < kC * D / 4; idx += kThreads) {
         const int r = idx / (D / 4), c4 = (idx % (D / 4)) * 4;
-        const size_t src = tok0 * D + (size_t)r * ts + c4;
+        const size_t src = tok0 * DL + (size_t)r * ts + col0 + c4;
         const float4 a = load4(q32 + src), bb = load4(k32 + src), cc = load4(v32 + src), dd = load4(do_nla + src);
         float *p0 = Qs + r * (D + 1) + c4, *p1 = Ks + r * (D + 1) + c4, *p2 = Vs + r * (D + 1) + c4,
               *p3 = dOs + r * (D + 1) + c4;
@@ -507,7 +510,7 @@ softmax_bwd_own_block_simt_kernel(const float *__restrict__ q32, const float *__
                 s = fmaf(qr[x], kr[x], s);
                 dp = fmaf(dor[x], vr[x], dp);
             }
-            const size_t row = (size_t)bh * L + (size_t)c * kC + i;
+            const size_t row = (size_t)bhg * L + (size_t)c * kC + i;
             pj = __expf(s * scale_sm - lse[row]);
             ds = pj * (dp - ginv * Dsm[row]);
         }
@@ -524,7 +527,7 @@ softmax_bwd_own_block_simt_kernel(const float *__restrict__ q32, const float *__
             ak = fmaf(dSs[i * (kC + 1) + r], Qs[i * (D + 1) + x], ak);
             av = fmaf(Ps[i * (kC + 1) + r], dOs[i * (D + 1) + x], av);
         }
-        const size_t dst = tok0 * D + (size_t)r * ts + x;
+        const size_t dst = tok0 * DL + (size_t)r * ts + col0 + x;
         dq_sm[dst] += scale_sm * aq;
         dk_x[dst] = scale_sm * ak;
         dv_x[dst] = av;
@@ -960,16 +963,16 @@ cudaError_t launch_softmax_bwd(const float *q32, const float *k_sm32, const floa
     return softmax_bwd_impl<64>(q32, k_sm32, v_sm32, cap, sm_idx, sm_chunk_prefix, do_nla, lse, Dsm, scale_sm, dq_sm, dk_sm, dv_sm, dmask, s, st);
 }
 
-template <int D>
+template <int D, int G = 1>
 static cudaError_t own_block_impl(const float *q32, const float *k32, const float *v32, const float *do_nla,
                                   const float *lse, const float *Dsm, const uint8_t *route, float scale_sm,
                                   float *dq_sm, float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
                                   cudaStream_t st) {
     const size_t smem = sizeof(float) * (4 * kC * (D + 1) + 2 * kC * (kC + 1));
-    cudaError_t e = set_smem(softmax_bwd_own_block_simt_kernel<D>, smem);
+    cudaError_t e = set_smem(softmax_bwd_own_block_simt_kernel<D, G>, smem);
     if (e != cudaSuccess) return e;
-    dim3 grid(s.L / kC, s.B * s.H);
-    softmax_bwd_own_block_simt_kernel<D><<<grid, kThreads, smem, st>>>(q32, k32, v32, do_nla, lse, Dsm, route,
+    dim3 grid(s.L / kC, s.B * s.H * G);
+    softmax_bwd_own_block_simt_kernel<D, G><<<grid, kThreads, smem, st>>>(q32, k32, v32, do_nla, lse, Dsm, route,
                                                                       scale_sm, dq_sm, dk_x, dv_x, gsc, s.L, s.H);
     count_launch();
     return cudaGetLastError();
@@ -979,7 +982,18 @@ cudaError_t launch_softmax_bwd_own_block_simt(const float *q32, const float *k32
                                               const float *do_nla, const float *lse, const float *Dsm,
                                               const uint8_t *route, float scale_sm, float *dq_sm,
                                               float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
-                                              cudaStream_t st) {
+                                              cudaStream_t st, int G) {
+    if (G > 1) {
+#define NATSL_GROUPED(DS, GG)                                                                               \
+        if (s.d == DS * GG && G == GG)                                                                      \
+            return own_block_impl<DS, GG>(q32, k32, v32, do_nla, lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, \
+                                          gsc, s, st)
+        NATSL_GROUPED(32, 2);
+        NATSL_GROUPED(64, 2);
+        NATSL_GROUPED(32, 4);
+#undef NATSL_GROUPED
+        return cudaErrorInvalidValue;
+    }
     if (s.d == 128) return own_block_impl<128>(q32, k32, v32, do_nla, lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, gsc, s, st);
     return own_block_impl<64>(q32, k32, v32, do_nla, lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, gsc, s, st);
 }
@@ -1047,7 +1061,7 @@ static cudaError_t assemble_impl(const AssembleArgs &a, void *dq, void *dk, void
     dg_kernel<<<(unsigned)((nch + 127) / 128), 128, 0, st>>>(a.dGrow, a.kappa, a.gS, a.Gcum,
                                                             s.d / kDvs, a.dg, s.B, s.L, s.H);
     count_launch();
-    if (a.dk_x) return cudaGetLastError();   // (the retained tokens' gradients came in through dk_x, dv_x)
+    if (a.no_scatter) return cudaGetLastError();   // (the retained tokens' gradients came in through dk_x, dv_x)
     constexpr int kRows = kThreads / (D / 4);
     dim3 grid((a.cap + kRows - 1) / kRows, s.B * s.H);
     scatter_sm_kernel<T, D><<<grid, kThreads, 0, st>>>(a.dk_sm, a.dv_sm, a.cap, a.sm_idx, a.sm_prefix,

@@ -444,7 +444,8 @@ __global__ void __launch_bounds__(256)
 qk_norm_bwd_f32_kernel(const T *__restrict__ q, const T *__restrict__ k,
                        const uint8_t *__restrict__ route, const float *dq_la,
                        const float *__restrict__ dq_sm, const float *dk_in, const float *dv_in,
-                       T *dq, T *dk, T *dv, size_t rows, int d, int G, float norm_eps) {
+                       T *dq, T *dk, T *dv, size_t rows, int d, int G, float norm_eps,
+                       const float *__restrict__ dk_sm) {
     const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= rows) return;
@@ -462,7 +463,8 @@ qk_norm_bwd_f32_kernel(const T *__restrict__ q, const T *__restrict__ k,
             g[j] = gin[lane + 32 * j];
             out[j] = 0.f;
         }
-        const bool l2_part = which == 0 || !retained, rms_part = which == 0 || retained;
+        const float *sm_in = which == 0 ? dq_sm : dk_sm;   // separate softmax-operation gradient, if any
+        const bool l2_part = sm_in || !retained, rms_part = sm_in || retained;
         if (l2_part) {
             for (int j = 0; j < nj; ++j) {
                 ss_all = fmaf(x[j], x[j], ss_all);
@@ -476,7 +478,7 @@ qk_norm_bwd_f32_kernel(const T *__restrict__ q, const T *__restrict__ k,
         if (rms_part) {
             float gs[4];
             for (int j = 0; j < nj; ++j) {
-                gs[j] = which == 0 ? dq_sm[row * d + lane + 32 * j] : g[j];
+                gs[j] = sm_in ? sm_in[row * d + lane + 32 * j] : g[j];
                 ssg[j] = warp_sum(x[j] * x[j]);
                 xgg[j] = warp_sum(x[j] * gs[j]);
             }
@@ -617,16 +619,16 @@ cudaError_t launch_qk_norm_f32(const void *q, const void *k, bool bf16, float *q
 cudaError_t launch_qk_norm_bwd_f32(const void *q, const void *k, bool bf16, const uint8_t *route,
                                    const float *dq_la, const float *dq_sm, const float *dk_in,
                                    const float *dv_in, void *dq, void *dk, void *dv, size_t rows, int d, int G,
-                                   float norm_eps, cudaStream_t st) {
+                                   float norm_eps, cudaStream_t st, const float *dk_sm) {
     const unsigned blocks = (unsigned)((rows + 7) / 8);
     if (bf16)
         qk_norm_bwd_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
             (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, route, dq_la, dq_sm, dk_in, dv_in,
-            (__nv_bfloat16 *)dq, (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, rows, d, G, norm_eps);
+            (__nv_bfloat16 *)dq, (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, rows, d, G, norm_eps, dk_sm);
     else
         qk_norm_bwd_f32_kernel<float><<<blocks, 256, 0, st>>>((const float *)q, (const float *)k, route, dq_la,
                                                              dq_sm, dk_in, dv_in, (float *)dq, (float *)dk,
-                                                             (float *)dv, rows, d, G, norm_eps);
+                                                             (float *)dv, rows, d, G, norm_eps, dk_sm);
     count_launch();
     return cudaGetLastError();
 }

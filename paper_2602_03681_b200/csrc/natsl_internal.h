@@ -79,7 +79,9 @@ cudaError_t launch_qk_norm_f32(const void *q, const void *k, bool bf16, float *q
 cudaError_t launch_qk_norm_bwd_f32(const void *q, const void *k, bool bf16, const uint8_t *route,
                                    const float *dq_la, const float *dq_sm, const float *dk_in,
                                    const float *dv_in, void *dq, void *dk, void *dv, size_t rows, int d, int G,
-                                   float norm_eps, cudaStream_t st);
+                                   float norm_eps, cudaStream_t st, const float *dk_sm = nullptr);
+// (dk_sm given -- block-level routing, where every token's k reaches both operations: dk_in is the gradient
+// w.r.t. the L2 copy and dk_sm the one w.r.t. the RMS copy, for every token, like q)
 // (fp32 gradients in: dq_la, dq_sm, dk_in, and dv_in or nullptr; out in the storage type: dq, dk, and dv =
 // dv_in converted when given.  In place is fine for fp32 storage: dq_la == dq, dk_in == dk.)
 
@@ -206,7 +208,8 @@ cudaError_t launch_softmax_bwd_own_block_simt(const float *q32, const float *k32
                                               const float *do_nla, const float *lse, const float *Dsm,
                                               const uint8_t *route, float scale_sm, float *dq_sm,
                                               float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
-                                              cudaStream_t st);
+                                              cudaStream_t st, int G = 1);
+// (G > 1: slices of d / G columns, lse / Dsm [B,H,G,L]; q32, k32: the softmax operation's copies of q, k)
 // dstate_out [B,H,d,d] (or nullptr: zero): the gradient the scan starts from, at the final state;
 // dstate_in (or nullptr): receives what is left after the first chunk, the initial state's gradient.
 cudaError_t launch_gdn_rscan(const float *q32, const float *k32, const float *Gcum, const float *W,
@@ -237,6 +240,7 @@ struct AssembleArgs {
     // block-level routing on the path with separate chunk-level products: route == nullptr (every token
     // takes part in the delta rule) and the softmax-branch dk, dv of every token, fp32 token-major
     const float *dk_x = nullptr, *dv_x = nullptr;
+    bool no_scatter = false;     // the retained tokens' dk, dv are part of dk_x, dv_x (or handled by the caller)
 };
 // dq (all tokens), dk/dv (linear tokens from the GDN branch, retained tokens scattered from the
 // compacted softmax-branch gradients), dbeta, dg.  Three kernels.

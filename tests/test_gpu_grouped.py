@@ -217,6 +217,47 @@ def test_bf16_tensor_cores_backward(G, norm, B, H, L):
     check_bwd(wl, got, ref, TOL["bf16"], large_only=not norm)
 
 
+@pytest.mark.parametrize("storage,d,G,norm,B,H,L,p", [
+    ("f32", 64, 2, True, 1, 2, 256, 0.4),
+    ("f32", 128, 2, False, 1, 2, 192, 0.5),
+    ("f32", 128, 4, True, 1, 1, 128, 0.0),
+    ("bf16", 128, 2, True, 1, 6, 256, 0.3),      # the paper's mode, trainable: blocks, grouped heads, normalised q, k
+    ("bf16", 128, 2, False, 2, 2, 320, 0.5),
+    ("bf16", 128, 1, True, 1, 2, 256, 0.4),
+])
+def test_block_level_routing_backward_with_grouped_heads(storage, d, G, norm, B, H, L, p):
+    """Backward under block-level routing with grouped heads and the normalisation (every token's k
+    reaches both operations there, through two different normalisations)."""
+    from test_gpu_parity import check_bwd
+    from paper_2602_03681_b200 import binding
+    base = "cfg0_f32_tiny_fwd" if storage == "f32" else "cfg1_bf16_prefill"
+    wl = dataclasses.replace(inputs.WORKLOADS[base], d=d, seed=81 + d + G)
+    x = make_inputs(wl, B, H, L, norm, block_p=p)
+    if p == 0.0:
+        x["route"][:] = 0
+    scale_sm = (d / G) ** -0.5 if norm else wl.scale_sm
+    dt = tdtype(wl)
+    pr = binding.make_params(B, H, L, d, binding.NATSL_F32 if storage == "f32" else binding.NATSL_BF16,
+                             wl.scale_la, scale_sm, G=G, norm_eps=1e-6,
+                             flags=binding.BLOCK_ROUTING | (binding.QK_NORM if norm else 0))
+    w_dev = dev(x["w"])
+    pr.w = w_dev.data_ptr()
+    ws = binding.alloc_workspace(pr, binding.OP_BWD)
+    t = {n: dev(x[n], dt) for n in ("q", "k", "v", "dout")}
+    t.update({n: dev(x[n]) for n in ("g", "beta", "route")})
+    outs = {n: torch.empty_like(t["q"]) for n in ("dq", "dk", "dv")}
+    outs.update(dg=torch.empty_like(t["g"]), dbeta=torch.empty_like(t["g"]),
+                dw=torch.empty((B, L, H, 2), device="cuda"))
+    binding.natsl_hybrid_bwd(t["q"], t["k"], t["v"], t["g"], t["beta"], t["route"], t["dout"], outs["dq"], outs["dk"],
+                             outs["dv"], outs["dg"], outs["dbeta"], outs["dw"], pr, ws)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(ws) == 0
+    got = {n: v.float().cpu().numpy() for n, v in outs.items()}
+    ref = grouped.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"], G=G,
+                             qk_norm=norm, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6, block=64)
+    check_bwd(wl, got, ref, TOL[storage], large_only=not norm)
+
+
 def test_normalisation_ignores_row_lengths_on_the_device():
     """Rescaling the q and k rows by powers of two changes no bf16 mantissa, so with norm_eps = 0 the
     normalised layer must return almost the same bits."""
