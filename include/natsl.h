@@ -182,11 +182,10 @@ typedef struct natsl_params {
                             /*   fp32 storage (d / G in {32, 64, 128}) and on the tensor-core path for */
                             /*   d = 128, G = 2 (the appendix's two softmax heads per linear head;     */
                             /*   three would need d = 192); natsl_hybrid_bwd with either routing for   */
-                            /*   the same shapes except bf16 storage with d = 64 (self-contained call, */
-                            /*   no p->dscore).  G > 1 or NATSL_QK_NORM with anything else (decode,    */
-                            /*   NATSL_APPEND_CACHE, NATSL_SAVE_FOR_BWD / NATSL_SAVED_FWD,             */
-                            /*   NATSL_FORCE_SIMT on bf16, NATSL_QK_NORM with p->k_sm):                */
-                            /*   NATSL_ERR_UNSUPPORTED.                                                */
+                            /*   the same shapes except bf16 storage with d = 64 (self-contained or    */
+                            /*   from a saved forward; no p->dscore).  G > 1 or NATSL_QK_NORM with     */
+                            /*   anything else (decode, NATSL_APPEND_CACHE, NATSL_FORCE_SIMT on bf16,  */
+                            /*   NATSL_QK_NORM with p->k_sm): NATSL_ERR_UNSUPPORTED.                   */
     float norm_eps;         /* NATSL_QK_NORM: epsilon under the square roots, >= 0                     */
 } natsl_params;
 

@@ -473,10 +473,12 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     if (append && !want_cache) return NATSL_ERR_NULL;
     const HeadGroups hg = head_groups(p);
     if (grouped_or_normed(p)) {
-        if (append || (p->flags & NATSL_SAVE_FOR_BWD)) return NATSL_ERR_UNSUPPORTED;
+        if (append) return NATSL_ERR_UNSUPPORTED;
         if ((p->flags & NATSL_QK_NORM) && want_cache) return NATSL_ERR_UNSUPPORTED;   // (the cache would hold normalised keys)
         if (tensor_cores) {
             if (hg.G > 1 && !(hg.G == 2 && p->d == 128)) return NATSL_ERR_UNSUPPORTED;
+            // (the saved forward is the backward's forward part: built where the backward is)
+            if ((p->flags & NATSL_SAVE_FOR_BWD) && p->d != 128) return NATSL_ERR_UNSUPPORTED;
         } else {
             if (p->dtype != NATSL_F32) return NATSL_ERR_UNSUPPORTED;
             if (hg.G > 1 && (hg.G > 4 || p->d / hg.G < 32)) return NATSL_ERR_UNSUPPORTED;
@@ -604,7 +606,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (p->flags & NATSL_APPEND_CACHE) return NATSL_ERR_UNSUPPORTED;
     const HeadGroups hg = head_groups(p);
     if (grouped_or_normed(p)) {      // grouped heads, q/k normalisation: the paths with separate chunk-level products
-        if ((p->flags & NATSL_SAVED_FWD) || p->dscore) return NATSL_ERR_UNSUPPORTED;
+        if (p->dscore) return NATSL_ERR_UNSUPPORTED;
         if (use_tensor_cores(p)) {
             if (p->d != 128 || hg.G > 2) return NATSL_ERR_UNSUPPORTED;
         } else {

@@ -258,6 +258,44 @@ def test_block_level_routing_backward_with_grouped_heads(storage, d, G, norm, B,
     check_bwd(wl, got, ref, TOL[storage], large_only=not norm)
 
 
+@pytest.mark.parametrize("storage,block", [("bf16", False), ("bf16", True), ("f32", False)])
+def test_saved_forward_then_backward_with_grouped_heads(storage, block):
+    """The training step as two calls (NATSL_SAVE_FOR_BWD, then NATSL_SAVED_FWD) with grouped heads and the
+    normalisation: same `out` as the plain forward's oracle, same gradients as the oracle's."""
+    from test_gpu_parity import check_bwd
+    from paper_2602_03681_b200 import binding
+    d, G, B, H, L = 128, 2, 1, 3, 256
+    base = "cfg0_f32_tiny_fwd" if storage == "f32" else "cfg1_bf16_prefill"
+    wl = dataclasses.replace(inputs.WORKLOADS[base], d=d, seed=91)
+    x = make_inputs(wl, B, H, L, True, block_p=0.4 if block else None)
+    scale_sm = (d / G) ** -0.5
+    dt = tdtype(wl)
+    flags = binding.QK_NORM | (binding.BLOCK_ROUTING if block else 0)
+    code = binding.NATSL_F32 if storage == "f32" else binding.NATSL_BF16
+    w_dev = dev(x["w"])
+    pr = binding.make_params(B, H, L, d, code, wl.scale_la, scale_sm, w=w_dev, G=G, norm_eps=1e-6,
+                             flags=flags | binding.SAVE_FOR_BWD)
+    ws = binding.alloc_workspace(pr, binding.OP_BWD)
+    t = {n: dev(x[n], dt) for n in ("q", "k", "v", "dout")}
+    t.update({n: dev(x[n]) for n in ("g", "beta", "route")})
+    out = torch.empty_like(t["q"])
+    binding.natsl_hybrid_fwd(t["q"], t["k"], t["v"], t["g"], t["beta"], t["route"], out, pr, ws)
+    pb = binding.make_params(B, H, L, d, code, wl.scale_la, scale_sm, w=w_dev, G=G, norm_eps=1e-6,
+                             flags=flags | binding.SAVED_FWD)
+    outs = {n: torch.empty_like(t["q"]) for n in ("dq", "dk", "dv")}
+    outs.update(dg=torch.empty_like(t["g"]), dbeta=torch.empty_like(t["g"]),
+                dw=torch.empty((B, L, H, 2), device="cuda"))
+    binding.natsl_hybrid_bwd(t["q"], t["k"], t["v"], t["g"], t["beta"], t["route"], t["dout"], outs["dq"], outs["dk"],
+                             outs["dv"], outs["dg"], outs["dbeta"], outs["dw"], pb, ws)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(ws) == 0
+    kw = dict(G=G, qk_norm=True, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6, block=64 if block else None)
+    ref_f = grouped.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], **kw)
+    check_stored(out.float().cpu().numpy(), ref_f["out"], TOL[storage], wl.dtype)
+    ref_b = grouped.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"], **kw)
+    check_bwd(wl, {n: v.float().cpu().numpy() for n, v in outs.items()}, ref_b, TOL[storage], large_only=False)
+
+
 def test_normalisation_ignores_row_lengths_on_the_device():
     """Rescaling the q and k rows by powers of two changes no bf16 mantissa, so with norm_eps = 0 the
     normalised layer must return almost the same bits."""
