@@ -576,9 +576,54 @@ def bench_grouped_heads(peaks, peak_kind, B=10, H=6, G=2):
         assert binding.natsl_device_status(ws) == 0
         ms[label] = best
     fl = sum(useful_flops(x["route"], wl.d, wl.C).values())
-    return {"B": B, "H_linear": H, "G": G, "L": wl.L, "d": wl.d, "ms": ms,
-            "tokens_per_s": B * wl.L / (ms["grouped_qk_norm"] * 1e-3), "useful_fwd_gflop": fl / 1e9,
-            "roofline": {"fwd": tensor_roofline(fl, ms["grouped_qk_norm"], peaks, peak_kind)}}
+    res = {"B": B, "H_linear": H, "G": G, "L": wl.L, "d": wl.d, "ms": ms,
+           "tokens_per_s": B * wl.L / (ms["grouped_qk_norm"] * 1e-3), "useful_fwd_gflop": fl / 1e9,
+           "roofline": {"fwd": tensor_roofline(fl, ms["grouped_qk_norm"], peaks, peak_kind)}}
+    # The mode the paper's models run in -- one routing decision per block, grouped heads, normalised q, k --
+    # forward and training step (forward saved in the backward's workspace, then the backward; at d = 128
+    # the backward's chunk-level products are CUDA-core tile GEMMs).
+    xb = inputs.make_layer_inputs(wl, route=inputs.route_blocks(wl.seed, (B, wl.L, H), wl.p_softmax))
+    rb = torch.from_numpy(xb["route"]).cuda()
+    dout = torch.from_numpy(xb["dout"]).cuda().to(torch.bfloat16)
+    flags = binding.QK_NORM | binding.BLOCK_ROUTING
+    kw = dict(G=G, norm_eps=1e-6)
+    scale_sm = float(wl.d // G) ** -0.5
+    pf = binding.make_params(B, H, wl.L, wl.d, binding.NATSL_BF16, wl.scale_la, scale_sm, w=d["w"],
+                             flags=flags | binding.SAVE_FOR_BWD, **kw)
+    pb = binding.make_params(B, H, wl.L, wl.d, binding.NATSL_BF16, wl.scale_la, scale_sm, w=d["w"],
+                             flags=flags | binding.SAVED_FWD, **kw)
+    wsb = binding.alloc_workspace(pf, binding.OP_BWD)
+    out = torch.empty_like(d["q"])
+    grads = [torch.empty_like(d["q"]) for _ in range(3)] + [torch.empty_like(d["g"]) for _ in range(2)] + \
+        [torch.empty((B, wl.L, H, 2), device="cuda")]
+    wsf = None
+
+    def fwd_block():
+        nonlocal wsf
+        wsf = binding.hybrid_fwd(d["q"], d["k"], d["v"], d["g"], d["beta"], rb, d["w"], scale_la=wl.scale_la,
+                                 scale_sm=scale_sm, flags=flags, ws=wsf, **kw)["ws"]
+
+    def train_step():
+        binding.natsl_hybrid_fwd(d["q"], d["k"], d["v"], d["g"], d["beta"], rb, out, pf, wsb)
+        binding.natsl_hybrid_bwd(d["q"], d["k"], d["v"], d["g"], d["beta"], rb, dout, *grads, pb, wsb)
+
+    for label, call in (("block_routed_fwd", fwd_block), ("block_routed_fwd_saved+bwd", train_step)):
+        best = float("inf")
+        for it in range(4):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            call()
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= 1:
+                best = min(best, e0.elapsed_time(e1))
+        ms[label] = best
+    assert binding.natsl_device_status(wsb) == 0 and binding.natsl_device_status(wsf) == 0
+    res["bwd_workspace_bytes"] = int(wsb.numel())
+    res["train_tokens_per_s"] = B * wl.L / (ms["block_routed_fwd_saved+bwd"] * 1e-3)
+    del wsb, wsf, out, grads
+    torch.cuda.empty_cache()
+    return res
 
 
 def bench_long_context_serving(L=131072, piece=16384, decode_steps=64):

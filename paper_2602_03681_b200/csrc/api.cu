@@ -736,9 +736,14 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         // dk_x -- a gradient with respect to that copy -- stays apart from the linear branch's dk until the
         // normalisations' backward.)
         NATSL_TRY(launch_gdn_finish(a, f.dk_x, f.dv_x, s32, st, false));
-        NATSL_TRY(launch_softmax_bwd_own_block_simt(normed ? f.qs32 : f.q32, normed ? f.ks32 : f.k32, f.v32,
-                                                    f.do_nla, f.lse, f.Dsm, route, p->scale_sm, f.dq_sm, f.dk_x,
-                                                    f.dv_x, gsc, s32, st, hg.G));
+        if (tensor_cores && p->d == 128 && hg.G == 2)      // softmax heads of 64 columns: warp-level tensor cores
+            NATSL_TRY(launch_softmax_bwd_own_block(q, k, v, f.dO16, f.lse, f.Dsm, route, p->scale_sm, f.dq_sm,
+                                                   f.dk_x, f.dv_x, gsc, s, st, 2, normed ? f.qs32 : nullptr,
+                                                   normed ? f.ks32 : nullptr));
+        else
+            NATSL_TRY(launch_softmax_bwd_own_block_simt(normed ? f.qs32 : f.q32, normed ? f.ks32 : f.k32, f.v32,
+                                                        f.do_nla, f.lse, f.Dsm, route, p->scale_sm, f.dq_sm, f.dk_x,
+                                                        f.dv_x, gsc, s32, st, hg.G));
         a.dk_x = normed ? nullptr : f.dk_x;
         a.dv_x = f.dv_x;
         a.no_scatter = true;

@@ -720,25 +720,30 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
 //   dq += dS K  (added to the query-side result of the compacted kernels)
 //   dk  = dS^T Q,  dv = P^T dO  (written: the tokens of a linear block have no other
 //                                 softmax-branch gradient)
-// with lse_i and D_i = <do_i, o_i> of the whole softmax row.  d = 64.
+// with lse_i and D_i = <do_i, o_i> of the whole softmax row.  Softmax heads of 64 columns: d = 64, or
+// kG = 2 heads per linear head of d = 128 (Section 4.3; the head is then a column slice of rows of 128
+// columns, lse / Dsm are [B,H,kG,L]).  kNormSrc: q and k come from the fp32 copies that hold the softmax
+// operation's normalised rows (qn, kn) instead of the bf16 inputs.
 constexpr int kOwnSmem = 6 * kTileH * 2;
 
+template <int kG, bool kNormSrc>
 __global__ void __launch_bounds__(kCkThreads, 3)
 softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
-                             const __nv_bfloat16 *__restrict__ v, const __half *__restrict__ do16,
+                             const __nv_bfloat16 *__restrict__ v, const float *__restrict__ qn,
+                             const float *__restrict__ kn, const __half *__restrict__ do16,
                              const float *__restrict__ lse, const float *__restrict__ Dsm,
                              const uint8_t *__restrict__ route, float scale_sm,
                              float *__restrict__ dq_sm, float *__restrict__ dk_x,
                              float *__restrict__ dv_x, const int32_t *gsc_status, int L, int H) {
-    constexpr int D = 64;
+    constexpr int D = 64, DL = D * kG;
     const float ginv = grad_scale(gsc_status).y;   // do16 and Dsm arrive times the gradient scale
     extern __shared__ __align__(16) uint8_t smraw[];
     __half *sQ = reinterpret_cast<__half *>(smraw), *sK = sQ + kTileH, *sV = sK + kTileH, *sDO = sV + kTileH,
            *sP = sDO + kTileH, *sDS = sP + kTileH;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H;
-    const size_t ts = (size_t)H * D;
-    const size_t tok0 = (((size_t)b * L + (size_t)c * kC) * H + h) * D;
+    const int c = blockIdx.x, bhg = blockIdx.y, bh = bhg / kG, col0 = (bhg % kG) * D, b = bh / H, h = bh % H;
+    const size_t ts = (size_t)H * DL;
+    const size_t tok0 = (((size_t)b * L + (size_t)c * kC) * H + h) * DL + col0;
     if (route[((size_t)b * L + (size_t)c * kC) * H + h]) return;   // a softmax block: its tokens are retained ones
     {
         const int r0 = tid >> 4, c4 = (tid & 15) * 4;
@@ -749,11 +754,17 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
         for (int it = 0; it < 4; ++it) {
             const int r = r0 + 16 * it;
             const size_t off = tok0 + (size_t)r * ts + c4;
-            const uint2 xq = *reinterpret_cast<const uint2 *>(q + off), xk = *reinterpret_cast<const uint2 *>(k + off),
-                        xv = *reinterpret_cast<const uint2 *>(v + off);
-            const uint2 xo = *reinterpret_cast<const uint2 *>(do16 + ((size_t)bh * L + (size_t)c * kC + r) * D + c4);
-            *reinterpret_cast<uint2 *>(sQ + r * kLdH + c4) = make_uint2(cv(xq.x), cv(xq.y));
-            *reinterpret_cast<uint2 *>(sK + r * kLdH + c4) = make_uint2(cv(xk.x), cv(xk.y));
+            const uint2 xv = *reinterpret_cast<const uint2 *>(v + off);
+            const uint2 xo = *reinterpret_cast<const uint2 *>(do16 + ((size_t)bh * L + (size_t)c * kC + r) * DL + col0 + c4);
+            if (kNormSrc) {
+                const float4 fq = *reinterpret_cast<const float4 *>(qn + off), fk = *reinterpret_cast<const float4 *>(kn + off);
+                *reinterpret_cast<uint2 *>(sQ + r * kLdH + c4) = make_uint2(pack_half2(fq.x, fq.y), pack_half2(fq.z, fq.w));
+                *reinterpret_cast<uint2 *>(sK + r * kLdH + c4) = make_uint2(pack_half2(fk.x, fk.y), pack_half2(fk.z, fk.w));
+            } else {
+                const uint2 xq = *reinterpret_cast<const uint2 *>(q + off), xk = *reinterpret_cast<const uint2 *>(k + off);
+                *reinterpret_cast<uint2 *>(sQ + r * kLdH + c4) = make_uint2(cv(xq.x), cv(xq.y));
+                *reinterpret_cast<uint2 *>(sK + r * kLdH + c4) = make_uint2(cv(xk.x), cv(xk.y));
+            }
             *reinterpret_cast<uint2 *>(sV + r * kLdH + c4) = make_uint2(cv(xv.x), cv(xv.y));
             *reinterpret_cast<uint2 *>(sDO + r * kLdH + c4) = xo;
         }
@@ -761,7 +772,7 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
     __syncthreads();
     const int row0 = 16 * (warp & 3), n0 = 32 * (warp >> 2);
     const int iA = row0 + g, iB = iA + 8;
-    const size_t rowA = (size_t)bh * L + (size_t)c * kC + iA;
+    const size_t rowA = (size_t)bhg * L + (size_t)c * kC + iA;
     const float l2e = 1.4426950408889634f;
     const float lseA = lse[rowA] * l2e, lseB = lse[rowA + 8] * l2e, DA = Dsm[rowA], DB = Dsm[rowA + 8];
     float pr[4][4], acc[4][4];
@@ -928,14 +939,16 @@ cudaError_t launch_softmax_bwd_own_block(const void *q, const void *k, const voi
                                          const void *do16, const float *lse, const float *Dsm,
                                          const uint8_t *route, float scale_sm, float *dq_sm,
                                          float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
-                                         cudaStream_t st) {
-    if (s.d != 64 || !s.bf16) return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(softmax_bwd_own_block_kernel,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kOwnSmem);
+                                         cudaStream_t st, int G, const float *qn, const float *kn) {
+    if (!s.bf16 || !((s.d == 64 && G <= 1) || (s.d == 128 && G == 2))) return cudaErrorInvalidValue;
+    auto kernel = softmax_bwd_own_block_kernel<1, false>;
+    if (G <= 1 && qn) kernel = softmax_bwd_own_block_kernel<1, true>;
+    if (G == 2) kernel = qn ? softmax_bwd_own_block_kernel<2, true> : softmax_bwd_own_block_kernel<2, false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOwnSmem);
     if (e != cudaSuccess) return e;
-    dim3 grid(s.L / kC, s.B * s.H);
-    softmax_bwd_own_block_kernel<<<grid, kCkThreads, kOwnSmem, st>>>(
-        (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, (const __half *)do16,
+    dim3 grid(s.L / kC, s.B * s.H * (G == 2 ? 2 : 1));
+    kernel<<<grid, kCkThreads, kOwnSmem, st>>>(
+        (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, qn, kn, (const __half *)do16,
         lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, gsc, s.L, s.H);
     count_launch();
     return cudaGetLastError();

@@ -270,7 +270,10 @@ cudaError_t launch_softmax_bwd_own_block(const void *q, const void *k, const voi
                                          const void *do16, const float *lse, const float *Dsm,
                                          const uint8_t *route, float scale_sm, float *dq_sm,
                                          float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
-                                         cudaStream_t st);
+                                         cudaStream_t st, int G = 1, const float *qn = nullptr,
+                                         const float *kn = nullptr);
+// (softmax heads of 64 columns: d = 64, or G = 2 at d = 128 with lse / Dsm [B,H,G,L]; qn, kn: fp32 copies
+// holding the softmax operation's normalised q, k [B,L,H,d], read instead of q, k)
 
 // decode.cu
 constexpr int kDecodeParts = 4;   // CTAs that share the retained K/V of one (sequence, head)

@@ -8,6 +8,8 @@ calls of `--op` on the current device and exits.  Nothing is timed or checked he
     python -m paper_2602_03681_b200.profile_case --op bwd --workload cfg4_bf16_train --B 1
     python -m paper_2602_03681_b200.profile_case --op fwd --flags 4        (block-level routing)
     python -m paper_2602_03681_b200.profile_case --op score --iters 6      (attention score layer)
+    python -m paper_2602_03681_b200.profile_case --op train --workload cfg1_bf16_prefill --B 10 --H 6 --G 2 \
+        --qk-norm --flags 4        (six linear x twelve softmax heads, normalised q, k, one route per block)
 """
 from __future__ import annotations
 
@@ -26,6 +28,9 @@ def main():
                     help="default: the workload that belongs to --op")
     ap.add_argument("--B", type=int, default=None, help="batch override (smaller case)")
     ap.add_argument("--L", type=int, default=None, help="sequence length override")
+    ap.add_argument("--H", type=int, default=None, help="(linear) head count override")
+    ap.add_argument("--G", type=int, default=0, help="softmax heads per linear head (fwd, bwd, train)")
+    ap.add_argument("--qk-norm", action="store_true", help="NATSL_QK_NORM with norm_eps 1e-6; scale_sm = (d/G)^-1/2")
     ap.add_argument("--iters", type=int, default=2)
     ap.add_argument("--flags", type=int, default=0)
     ap.add_argument("--report", action="store_true", help="print CUDA-event time of each call")
@@ -99,8 +104,13 @@ def main():
         kw["B"] = args.B
     if args.L:
         kw["L"] = args.L
+    if args.H:
+        kw["H"] = args.H
+    gflags = args.flags | (binding.QK_NORM if args.qk_norm else 0)
+    gkw = dict(G=args.G, norm_eps=1e-6 if args.qk_norm else 0.0)
+    scale_sm = float(wl.d // max(args.G, 1)) ** -0.5 if args.qk_norm else wl.scale_sm
     if args.op in ("fwd", "bwd", "train") and args.flags & binding.BLOCK_ROUTING:   # one route per block of 64 tokens
-        kw["route"] = inputs.route_blocks(wl.seed, (kw.get("B", wl.B), kw.get("L", wl.L), wl.H),
+        kw["route"] = inputs.route_blocks(wl.seed, (kw.get("B", wl.B), kw.get("L", wl.L), kw.get("H", wl.H)),
                                           wl.p_softmax)
     x = inputs.make_layer_inputs(wl, **kw)
     q, k, v = (dev(x[m], dt) for m in ("q", "k", "v"))
@@ -111,20 +121,23 @@ def main():
             def call():
                 nonlocal ws
                 ws = binding.hybrid_fwd(q, k, v, g, beta, route, w, scale_la=wl.scale_la,
-                                        scale_sm=wl.scale_sm, flags=args.flags, ws=ws)["ws"]
+                                        scale_sm=scale_sm, flags=gflags, ws=ws, **gkw)["ws"]
             timed(call)
     elif args.op == "train":
         dout = dev(x["dout"], dt)
         B, L, H, d = q.shape
-        p = binding.make_params(B, H, L, d, code, wl.scale_la, wl.scale_sm, w=w,
-                                flags=args.flags | binding.SAVE_FOR_BWD)
+        p = binding.make_params(B, H, L, d, code, wl.scale_la, scale_sm, w=w,
+                                flags=gflags | binding.SAVE_FOR_BWD, **gkw)
+        pb = binding.make_params(B, H, L, d, code, wl.scale_la, scale_sm, w=w,
+                                 flags=gflags | binding.SAVED_FWD, **gkw)
         ws = binding.alloc_workspace(p, binding.OP_BWD)
         out = torch.empty_like(q)
+        grads = [torch.empty_like(q) for _ in range(3)] + [torch.empty_like(g) for _ in range(2)] + \
+            [torch.empty((B, L, H, 2), dtype=torch.float32, device="cuda")]
         for _ in range(args.iters):
             def call():
                 binding.natsl_hybrid_fwd(q, k, v, g, beta, route, out, p, ws)
-                binding.hybrid_bwd(q, k, v, g, beta, route, w, dout, scale_la=wl.scale_la,
-                                   scale_sm=wl.scale_sm, flags=args.flags | binding.SAVED_FWD, ws=ws)
+                binding.natsl_hybrid_bwd(q, k, v, g, beta, route, dout, *grads, pb, ws)
             timed(call)
     else:
         dout = dev(x["dout"], dt)
