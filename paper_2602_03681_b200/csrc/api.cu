@@ -726,6 +726,9 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(side_join.join());      // the side stream's last kernels
         return NATSL_OK;
     }
+    // (the tile GEMMs run on tf32 tensor cores for bf16 storage -- unless the caller asked for fp32
+    // arithmetic -- and as fp32 FMAs otherwise: launch_bgemm goes by the storage type it is told)
+    const Shape sgemm = tensor_cores ? s : s32;
     // (block-level routing: beta~ = beta for every token, so the kernels below get no route)
     const uint8_t *route_bt = general_block ? nullptr : route;
     if (general_block) {
@@ -748,23 +751,23 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         a.dv_x = f.dv_x;
         a.no_scatter = true;
     }
-    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, s, st));
-    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, s, st));
-    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, s, st));
-    NATSL_TRY(launch_bgemm(false, true, 1, TM(f.do_la), TM(f.Ut), CC(f.N), kC, kC, di, 1.f, false, s, st));
+    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, sgemm, st));
+    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, sgemm, st));
+    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, sgemm, st));
+    NATSL_TRY(launch_bgemm(false, true, 1, TM(f.do_la), TM(f.Ut), CC(f.N), kC, kC, di, 1.f, false, sgemm, st));
     if (tensor_cores) {   // [dKb | dVb] = (I + A)^-T [dW | dU~] with the inverse the forward already formed
-        NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dW), TM(f.dKb), kC, di, kC, 1.f, false, s, st));
-        NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dUt), TM(f.dVb), kC, di, kC, 1.f, false, s, st));
+        NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dW), TM(f.dKb), kC, di, kC, 1.f, false, sgemm, st));
+        NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dUt), TM(f.dVb), kC, di, kC, 1.f, false, sgemm, st));
     } else {
         NATSL_TRY(launch_gdn_tsolve(f.Abar, beta, route_bt, f.dW, f.dUt, f.dKb, f.dVb, s, st));
     }
-    NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dKb), TM(f.W), CC(f.M), kC, kC, di, -1.f, false, s, st));
-    NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dVb), TM(f.U), CC(f.M), kC, kC, di, -1.f, true, s, st));
+    NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dKb), TM(f.W), CC(f.M), kC, kC, di, -1.f, false, sgemm, st));
+    NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dVb), TM(f.U), CC(f.M), kC, kC, di, -1.f, true, sgemm, st));
     NATSL_TRY(launch_mask_scale(f.M, f.N, f.Gcum, beta, route_bt, p->scale_la, f.Mg, f.Ms, f.Ns, s, st));
-    NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Mg), TM(f.k32), TM(f.X1p), kC, di, kC, 1.f, false, s, st));
-    NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ms), TM(f.k32), TM(f.X2), kC, di, kC, 1.f, false, s, st));
-    NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Ns), TM(f.k32), TM(f.X3), kC, di, kC, 1.f, false, s, st));
-    NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ns), TM(f.q32), TM(f.X4), kC, di, kC, 1.f, false, s, st));
+    NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Mg), TM(f.k32), TM(f.X1p), kC, di, kC, 1.f, false, sgemm, st));
+    NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ms), TM(f.k32), TM(f.X2), kC, di, kC, 1.f, false, sgemm, st));
+    NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Ns), TM(f.k32), TM(f.X3), kC, di, kC, 1.f, false, sgemm, st));
+    NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ns), TM(f.q32), TM(f.X4), kC, di, kC, 1.f, false, sgemm, st));
     // With the normalisation the assembly's dq, dk are gradients with respect to the normalised rows; a
     // last kernel applies the two row-local Jacobians.  fp32 storage: in place.  bf16 storage: the
     // assembly writes fp32 (into buffers the chunk-level products are done with) and the last kernel

@@ -34,26 +34,43 @@ constexpr int kThreads = 256;
 
 // ------------------------------------------------------------------------------------------
 // generic batched GEMM: C = alpha * op(A) op(B) (+ C), 64x64 output tiles, fp32
+// kTF32 (bf16 storage, whose tolerance it fits): the products run on the warp-level tensor-core path
+// with tf32 operands (fp32 range, 11 significant bits) and fp32 accumulation -- warp w owns rows
+// 16 (w & 3) .. and columns 32 (w >> 2) .. of the tile, four m16n8k8 products per 8 values of k --;
+// otherwise fp32 FMAs (fp32 storage: 1e-4 tolerance).
 // ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ void mma_tf32_16x8x8(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
 __device__ __forceinline__ const float *mat_base(const BMat &m, int b, int h, int ch) {
     return m.p + (size_t)b * m.sb + (size_t)h * m.sh + (size_t)ch * m.sc;
 }
 
-template <bool TA, bool TB, int MASK>
+template <bool TA, bool TB, int MASK, bool kTF32>
 __global__ void __launch_bounds__(kThreads)
 bgemm_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H, int NC) {
-    __shared__ __align__(16) float As[16][68];
-    __shared__ __align__(16) float Bs[16][68];
+    constexpr int kLd = kTF32 ? 72 : 68;      // (72: the fragment reads of a warp fall on 32 different banks)
+    __shared__ __align__(16) float As[16][kLd];
+    __shared__ __align__(16) float Bs[16][kLd];
     const int z = blockIdx.z, ch = z % NC, bh = z / NC, b = bh / H, h = bh % H;
     const float *Ap = mat_base(A, b, h, ch), *Bp = mat_base(B, b, h, ch);
     float *Cp = const_cast<float *>(mat_base(Cm, b, h, ch));
     const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
     const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
-    float acc[4][4];
+    float acc[4][4];          // fp32 FMAs: rows ty*4 + i, columns tx*4 + j; tf32: n-tile i, fragment element j
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    const int warp = t >> 5, lane = t & 31, fg = lane >> 2, ft = lane & 3;
+    const int wr = (warp & 3) * 16, wc = (warp >> 2) * 32;
 
     for (int k0 = 0; k0 < K; k0 += 16) {
         if (!TA) {   // A[m][k], k contiguous
@@ -75,6 +92,18 @@ bgemm_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H,
             Bs[kk][c] = x.x; Bs[kk + 1][c] = x.y; Bs[kk + 2][c] = x.z; Bs[kk + 3][c] = x.w;
         }
         __syncthreads();
+        if (kTF32) {
+#pragma unroll
+            for (int k8 = 0; k8 < 16; k8 += 8) {
+                const uint32_t a[4] = {to_tf32(As[k8 + ft][wr + fg]), to_tf32(As[k8 + ft][wr + fg + 8]),
+                                       to_tf32(As[k8 + ft + 4][wr + fg]), to_tf32(As[k8 + ft + 4][wr + fg + 8])};
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+                    const uint32_t bfr[2] = {to_tf32(Bs[k8 + ft][wc + 8 * nt + fg]), to_tf32(Bs[k8 + ft + 4][wc + 8 * nt + fg])};
+                    mma_tf32_16x8x8(acc[nt], a, bfr);
+                }
+            }
+        } else
 #pragma unroll
         for (int kk = 0; kk < 16; ++kk) {
             const float4 a = *reinterpret_cast<const float4 *>(&As[kk][ty * 4]);
@@ -86,6 +115,21 @@ bgemm_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H,
                 for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
         }
         __syncthreads();
+    }
+    if (kTF32) {      // fragment layout: elements (0, 1) in row fg, (2, 3) in row fg + 8; columns 2 ft, 2 ft + 1
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int row = m0 + wr + fg + 8 * hh, col = n0 + wc + 8 * nt + 2 * ft;
+                float o0 = alpha * acc[nt][2 * hh], o1 = alpha * acc[nt][2 * hh + 1];
+                if (MASK == 1) { if (col > row) o0 = 0.f; if (col + 1 > row) o1 = 0.f; }
+                if (MASK == 2) { if (col >= row) o0 = 0.f; if (col + 1 >= row) o1 = 0.f; }
+                float2 *cr = reinterpret_cast<float2 *>(Cp + (size_t)row * Cm.ld + col);
+                if (accumulate) { const float2 old = *cr; o0 += old.x; o1 += old.y; }
+                *cr = make_float2(o0, o1);
+            }
+        return;
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -852,8 +896,11 @@ cudaError_t launch_bgemm(bool ta, bool tb, int mask, BMat A, BMat B, BMat C, int
                          float alpha, bool accumulate, Shape s, cudaStream_t st) {
     const int NC = s.L / kC;
     dim3 grid(n / 64, m / 64, s.B * s.H * NC);
-#define NATSL_BG(TA, TB, MK) \
-    bgemm_kernel<TA, TB, MK><<<grid, kThreads, 0, st>>>(A, B, C, k, alpha, accumulate ? 1 : 0, s.H, NC)
+#define NATSL_BG(TA, TB, MK)                                                                                   \
+    do {                                                                                                        \
+        if (s.bf16) bgemm_kernel<TA, TB, MK, true><<<grid, kThreads, 0, st>>>(A, B, C, k, alpha, accumulate ? 1 : 0, s.H, NC); \
+        else bgemm_kernel<TA, TB, MK, false><<<grid, kThreads, 0, st>>>(A, B, C, k, alpha, accumulate ? 1 : 0, s.H, NC);       \
+    } while (0)
     if (!ta && !tb && mask == 0) NATSL_BG(false, false, 0);
     else if (!ta && tb && mask == 0) NATSL_BG(false, true, 0);
     else if (ta && !tb && mask == 0) NATSL_BG(true, false, 0);
