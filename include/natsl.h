@@ -183,9 +183,11 @@ typedef struct natsl_params {
                             /*   d = 128, G = 2 (the appendix's two softmax heads per linear head;     */
                             /*   three would need d = 192); natsl_hybrid_bwd with either routing for   */
                             /*   the same shapes except bf16 storage with d = 64 (self-contained or    */
-                            /*   from a saved forward; no p->dscore).  G > 1 or NATSL_QK_NORM with     */
-                            /*   anything else (decode, NATSL_APPEND_CACHE, NATSL_FORCE_SIMT on bf16,  */
-                            /*   NATSL_QK_NORM with p->k_sm): NATSL_ERR_UNSUPPORTED.                   */
+                            /*   from a saved forward; no p->dscore); natsl_decode_step for d / G in   */
+                            /*   {32, 64, 128}.  A cache returned or read with NATSL_QK_NORM holds the */
+                            /*   keys as given: they are normalised as they are read.  G > 1 or        */
+                            /*   NATSL_QK_NORM with anything else (NATSL_APPEND_CACHE, NATSL_FORCE_SIMT */
+                            /*   on bf16): NATSL_ERR_UNSUPPORTED.                                      */
     float norm_eps;         /* NATSL_QK_NORM: epsilon under the square roots, >= 0                     */
 } natsl_params;
 

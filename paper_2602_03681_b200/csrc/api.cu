@@ -474,7 +474,6 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     const HeadGroups hg = head_groups(p);
     if (grouped_or_normed(p)) {
         if (append) return NATSL_ERR_UNSUPPORTED;
-        if ((p->flags & NATSL_QK_NORM) && want_cache) return NATSL_ERR_UNSUPPORTED;   // (the cache would hold normalised keys)
         if (tensor_cores) {
             if (hg.G > 1 && !(hg.G == 2 && p->d == 128)) return NATSL_ERR_UNSUPPORTED;
             // (the saved forward is the backward's forward part: built where the backward is)
@@ -537,11 +536,20 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
                                      (size_t)p->B * p->L * p->H, p->d, hg.G, hg.norm_eps, st));
         q_la = f.q_la; k_la = f.k_la; q_sm = f.q_sm; k_nsm = f.k_nsm;
     }
-    if (tensor_cores)
+    // A cache the call returns keeps the keys as given (the decode step normalises them as it reads them);
+    // with the normalisation the softmax kernel then reads a normalised copy in the workspace instead.
+    const bool raw_cache = want_cache && hg.norm_eps >= 0.f;
+    const void *k_soft = raw_cache ? f.k_sm : k_sm, *v_soft = raw_cache ? f.v_sm : v_sm;
+    const int32_t cap_soft = raw_cache ? p->L : cap;
+    if (tensor_cores) {
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
-                                      f.v16, nullptr, cap, capv, append, f.status, s, st0, hg));
-    else
-        NATSL_TRY(launch_gather_kv(k_nsm, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
+                                      f.v16, raw_cache ? f.k_sm : nullptr, cap, capv, append, f.status, s, st0,
+                                      hg, raw_cache));
+    } else {
+        if (raw_cache) NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));
+        NATSL_TRY(launch_gather_kv(k_nsm, v, f.sm_idx, f.prefix, raw_cache ? f.k_sm : k_sm,
+                                   raw_cache ? f.v_sm : v_sm, cap_soft, f.status, s, st));
+    }
     NATSL_TRY(mark());
     if (tensor_cores) {
         // block-level routing: every token takes part in the delta rule of its own block
@@ -574,7 +582,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
                                          f.status, s, st));
         }
         NATSL_TRY(mark());
-        NATSL_TRY(launch_softmax_combine_tc(q, k_sm, f.v16, cap, capv, f.sm_idx, f.prefix, f.o_la16,
+        NATSL_TRY(launch_softmax_combine_tc(q, k_soft, f.v16, cap_soft, capv, f.sm_idx, f.prefix, f.o_la16,
                                             flags_softmax, p->w, p->scale_sm, p->eps, out, p->o_nla,
                                             p->lse, br, append, f.status, s, st, hg));
     } else {
@@ -586,7 +594,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
                                        p->state_out, nullptr, nullptr, o_la, br.route, s, st));
         NATSL_TRY(mark());
         // (an own-block tile of block-level routing reads the layer's keys: the softmax operation's copy)
-        NATSL_TRY(launch_softmax_combine_simt(q_sm, k_sm, v_sm, cap, f.sm_idx, f.prefix, o_la, p->w,
+        NATSL_TRY(launch_softmax_combine_simt(q_sm, k_soft, v_soft, cap_soft, f.sm_idx, f.prefix, o_la, p->w,
                                               p->scale_sm, p->eps, out, p->o_nla, p->lse,
                                               BlockRouting{br.route, k_nsm, v}, s, st, hg.G));
     }
@@ -802,7 +810,8 @@ int natsl_decode_step(const void *q, const void *k, const void *v, const float *
         !out)
         return NATSL_ERR_NULL;
     if (cache_cap <= 0) return NATSL_ERR_SHAPE;
-    if (grouped_or_normed(p)) return NATSL_ERR_UNSUPPORTED;
+    const HeadGroups hg = head_groups(p);
+    if (hg.G > 1 && (hg.G > 4 || p->d / hg.G < 32)) return NATSL_ERR_UNSUPPORTED;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(state) ||
         !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(ws))
         return NATSL_ERR_ALIGN;
@@ -810,7 +819,7 @@ int natsl_decode_step(const void *q, const void *k, const void *v, const float *
     cudaError_t e = launch_decode_step(q, k, v, g, beta, route, p->w, state, k_cache, v_cache,
                                        cache_len, cache_cap, out, p->scale_la, p->scale_sm, p->eps,
                                        ws, shape_of(p),
-                                       static_cast<cudaStream_t>(stream));
+                                       static_cast<cudaStream_t>(stream), hg);
     return e == cudaSuccess ? NATSL_OK : NATSL_ERR_CUDA;
 }
 

@@ -14,6 +14,13 @@
 // Whichever CTA of the head finishes last (an atomic ticket, nobody waits) merges the partials,
 // adds the new token's own term, normalises, combines, writes `out`, appends the token to the
 // cache and bumps its length.
+// Grouped softmax heads and per-operation q/k normalisation (Section 4.3; template flag, so that the
+// plain instantiation is unchanged code): the G softmax heads of a linear head are the G slices of d / G
+// columns -- the lanes that share a key row split into G groups, each with its own logit, running
+// maximum and sum --, the state CTAs work on the L2-normalised q and k, and the cache keeps the keys as
+// given: a cached key is RMS-normalised per slice as it is read (its sum of squares rides along with the
+// logit's reduction), because normalised keys rounded to the cache's bf16 would cost 2.8e-2 of the
+// branch output's RMS.
 #include "common.cuh"
 #include "natsl_internal.h"
 #include "tc_common.cuh"
@@ -52,24 +59,28 @@ template <> struct Vec16<__nv_bfloat16> {
     }
 };
 
-// Workspace: [0,256) status word; then tickets [BH] i32; partials [BH][kDecodeParts][D+2] f32
-// (m, z, acc[D]); o_la [BH][D] f32.
+// Workspace: [0,256) status word; then tickets [BH] i32; partials [BH][kDecodeParts][D+8] f32
+// (m[G], z[G] in the first 8 with G <= 4, then acc[D]); o_la [BH][D] f32.
+constexpr int kPartHead = 8;
 __host__ __device__ inline size_t dec_off_tickets() { return 256; }
 __host__ __device__ inline size_t dec_off_partials(size_t BH) {
     return (256 + BH * 4 + 255) / 256 * 256;
 }
 __host__ __device__ inline size_t dec_off_ola(size_t BH, int D) {
-    return dec_off_partials(BH) + (BH * kDecodeParts * (D + 2) * 4 + 255) / 256 * 256;
+    return dec_off_partials(BH) + (BH * kDecodeParts * (D + kPartHead) * 4 + 255) / 256 * 256;
 }
 
-template <typename T, int D>
+template <typename T, int D, bool kGrouped>
 __global__ void __launch_bounds__(kThreads, 3)
 decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__restrict__ v,
                    const float *__restrict__ g, const float *__restrict__ beta,
                    const uint8_t *__restrict__ route, const float *__restrict__ w,
                    float *__restrict__ state, T *__restrict__ k_cache, T *__restrict__ v_cache,
                    int32_t *__restrict__ cache_len, int cap, T *__restrict__ out, float scale_la,
-                   float scale_sm, float eps, uint8_t *__restrict__ ws, int BH) {
+                   float scale_sm, float eps, uint8_t *__restrict__ ws, int BH, int Gin, float norm_eps) {
+    const int G = kGrouped ? Gin : 1;              // softmax heads per linear head
+    const int ds = D / G;                          // columns per softmax head
+    const bool normed = kGrouped && norm_eps >= 0.f;
     constexpr int kE = Vec16<T>::kN;               // elements per 16-byte piece
     constexpr int kRowBytes = D * (int)sizeof(T);
     constexpr int kLpk = kRowBytes / 16;           // lanes per key row
@@ -79,8 +90,9 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
 
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint64_t full[kStages], empty[kStages];
-    __shared__ __align__(16) float qs[D], ks[D], vs[D];
-    __shared__ float sm_m[kTileKeys], sm_z[kTileKeys];
+    __shared__ __align__(16) float qs[D], ks[D], vs[D];     // (normalised: the linear operation's q, k)
+    __shared__ __align__(16) float qsm[kGrouped ? D : 4], ksm[kGrouped ? D : 4];   // the softmax operation's q, k
+    __shared__ float sm_m[kTileKeys * (kGrouped ? 4 : 1)], sm_z[kTileKeys * (kGrouped ? 4 : 1)];
     __shared__ float norm_red[2][kWarps];
     __shared__ int s_last, s_abort[2];   // s_abort[1]: wait limit (see mbar_wait)
 
@@ -89,7 +101,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
     int32_t *status = reinterpret_cast<int32_t *>(ws);
     int32_t *ticket = reinterpret_cast<int32_t *>(ws + dec_off_tickets()) + bh;
     float *partials =
-        reinterpret_cast<float *>(ws + dec_off_partials(BH)) + (size_t)bh * kDecodeParts * (D + 2);
+        reinterpret_cast<float *>(ws + dec_off_partials(BH)) + (size_t)bh * kDecodeParts * (D + kPartHead);
     float *ola_ws = reinterpret_cast<float *>(ws + dec_off_ola(BH, D)) + (size_t)bh * D;
 
     // route 0: linear token (delta rule); 1: softmax token (appended to the cache); 2: token of a
@@ -116,6 +128,29 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
     }
     __syncthreads();
     volatile int *abort_flag = s_abort;
+    if (kGrouped) {
+        // q, k of the two operations: L2 over the row for the linear one (in place in qs, ks), RMS per slice
+        // for the softmax one (qsm, ksm); without the normalisation both are the token's q, k.
+        float sq = 0.f, sk = 0.f;
+        if (tid < D) { sq = qs[tid] * qs[tid]; sk = ks[tid] * ks[tid]; }
+        sq = warp_sum(sq);
+        sk = warp_sum(sk);
+        if (lane == 0 && warp < D / 32) { norm_red[0][warp] = sq; norm_red[1][warp] = sk; }
+        __syncthreads();
+        if (tid < D) {
+            float aq = 0.f, ak = 0.f, gq = 0.f, gk = 0.f;
+            for (int wv = 0; wv < D / 32; ++wv) {
+                aq += norm_red[0][wv];
+                ak += norm_red[1][wv];
+                if ((32 * wv) / ds == tid / ds) { gq += norm_red[0][wv]; gk += norm_red[1][wv]; }
+            }
+            const float qv = qs[tid], kv = ks[tid];
+            qsm[tid] = normed ? qv * rsqrtf(gq / ds + norm_eps) : qv;
+            ksm[tid] = normed ? kv * rsqrtf(gk / ds + norm_eps) : kv;
+            if (normed) { qs[tid] = qv * rsqrtf(aq + norm_eps); ks[tid] = kv * rsqrtf(ak + norm_eps); }
+        }
+        __syncthreads();
+    }
 
     if (part < kDecodeParts) {
         // ---------------- cache CTA: one slice of the retained K/V ----------------
@@ -145,7 +180,8 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
             const int stream = tid / kLpk, piece = tid % kLpk;
             float qf[kE];
 #pragma unroll
-            for (int x = 0; x < kE; ++x) qf[x] = qs[piece * kE + x] * scale_sm;
+            for (int x = 0; x < kE; ++x) qf[x] = (kGrouped ? qsm[piece * kE + x] : qs[piece * kE + x]) * scale_sm;
+            const int lps = kLpk / G;              // lanes per softmax head within a key row
             float m = -INFINITY, z = 0.f, acc[kE];
 #pragma unroll
             for (int x = 0; x < kE; ++x) acc[x] = 0.f;
@@ -163,8 +199,19 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
                     float sc = 0.f;
 #pragma unroll
                     for (int x = 0; x < kE; ++x) sc = fmaf(qf[x], kx[x], sc);
+                    if (!kGrouped) {
 #pragma unroll
-                    for (int o = kLpk / 2; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                        for (int o = kLpk / 2; o > 0; o >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                    } else {                     // per softmax head; the key's sum of squares rides along
+                        float kk = 0.f;
+#pragma unroll
+                        for (int x = 0; x < kE; ++x) kk = fmaf(kx[x], kx[x], kk);
+                        for (int o = lps / 2; o > 0; o >>= 1) {
+                            sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                            kk += __shfl_xor_sync(0xffffffffu, kk, o);
+                        }
+                        if (normed) sc *= rsqrtf(kk / ds + norm_eps);
+                    }
                     if (j < rows) {                            // rows past the slice hold stale bytes
                         const float m_new = fmaxf(m, sc);
                         const float corr = __expf(m - m_new), pj = __expf(sc - m_new);
@@ -179,24 +226,25 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
             // merge the streams of this CTA -> one partial (m, z, acc[D]); the ring is free now
             float *stage_acc = reinterpret_cast<float *>(smem);   // [kStreams][D]
             named_barrier_sync(1, kWorkThreads);
-            if (piece == 0) { sm_m[stream] = m; sm_z[stream] = z; }
+            if (piece % lps == 0) { sm_m[stream * G + piece / lps] = m; sm_z[stream * G + piece / lps] = z; }
 #pragma unroll
             for (int x = 0; x < kE; ++x) stage_acc[stream * D + piece * kE + x] = acc[x];
             named_barrier_sync(1, kWorkThreads);
             if (tid < D) {
+                const int sg = tid / ds;             // this column's softmax head
                 float M = -INFINITY;
-                for (int st = 0; st < kStreams; ++st) M = fmaxf(M, sm_m[st]);
+                for (int st = 0; st < kStreams; ++st) M = fmaxf(M, sm_m[st * G + sg]);
                 float Z = 0.f, o = 0.f;
                 if (M > -INFINITY) {
                     for (int st = 0; st < kStreams; ++st) {
-                        const float f = __expf(sm_m[st] - M);
-                        Z = fmaf(sm_z[st], f, Z);
+                        const float f = __expf(sm_m[st * G + sg] - M);
+                        Z = fmaf(sm_z[st * G + sg], f, Z);
                         o = fmaf(stage_acc[st * D + tid], f, o);
                     }
                 }
-                float *pp = partials + (size_t)part * (D + 2);
-                pp[2 + tid] = o;
-                if (tid == 0) { pp[0] = M; pp[1] = Z; }
+                float *pp = partials + (size_t)part * (D + kPartHead);
+                pp[kPartHead + tid] = o;
+                if (tid % ds == 0) { pp[sg] = M; pp[4 + sg] = Z; }
             }
         }
     } else if (warp < kWarps && !cache_full) {
@@ -282,23 +330,28 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
         return;
     }
     float on = 0.f, ol = 0.f;
+    const int sg = tid < D ? tid / ds : 0;            // this column's softmax head
     if (tid < D) {
         const volatile float *pv = partials;
+        constexpr int kPs = D + kPartHead;
         float M = -INFINITY;
-        for (int pt = 0; pt < kDecodeParts; ++pt) M = fmaxf(M, pv[pt * (D + 2)]);
+        for (int pt = 0; pt < kDecodeParts; ++pt) M = fmaxf(M, pv[pt * kPs + sg]);
         float sc_self = 0.f;
         if (r) {                                       // the token attends to itself
-            for (int x = 0; x < D; ++x) sc_self = fmaf(qs[x] * scale_sm, ks[x], sc_self);
+            if (kGrouped)
+                for (int x = sg * ds; x < (sg + 1) * ds; ++x) sc_self = fmaf(qsm[x] * scale_sm, ksm[x], sc_self);
+            else
+                for (int x = 0; x < D; ++x) sc_self = fmaf(qs[x] * scale_sm, ks[x], sc_self);
             M = fmaxf(M, sc_self);
         }
         float Z = 0.f;
         if (M > -INFINITY) {
             for (int pt = 0; pt < kDecodeParts; ++pt) {
-                const float mp = pv[pt * (D + 2)];
+                const float mp = pv[pt * kPs + sg];
                 if (mp > -INFINITY) {
                     const float f = __expf(mp - M);
-                    Z = fmaf(pv[pt * (D + 2) + 1], f, Z);
-                    on = fmaf(pv[pt * (D + 2) + 2 + tid], f, on);
+                    Z = fmaf(pv[pt * kPs + 4 + sg], f, Z);
+                    on = fmaf(pv[pt * kPs + kPartHead + tid], f, on);
                 }
             }
             if (r) {
@@ -314,10 +367,13 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
     if (lane == 0 && warp < kWarps) { norm_red[0][warp] = ssn; norm_red[1][warp] = ssl; }
     __syncthreads();
     if (tid < D) {
-        float tn = 0.f, tl = 0.f;
+        float tn = 0.f, tl = 0.f;      // softmax output: over this column's softmax head; linear read-out: over the row
 #pragma unroll
-        for (int wv = 0; wv < kWarps; ++wv) { tn += norm_red[0][wv]; tl += norm_red[1][wv]; }
-        const float fn = rsqrtf(tn / D + eps), fl = rsqrtf(tl / D + eps);
+        for (int wv = 0; wv < kWarps; ++wv) {
+            if (!kGrouped || (32 * wv) / ds == sg) tn += norm_red[0][wv];
+            tl += norm_red[1][wv];
+        }
+        const float fn = rsqrtf(tn / ds + eps), fl = rsqrtf(tl / D + eps);
         const float wn = w ? w[(size_t)bh * 2] : 0.5f, wl = w ? w[(size_t)bh * 2 + 1] : 0.5f;
         out[(size_t)bh * D + tid] = from_f32<T>(wn * on * fn + wl * ol * fl);
         if (r) {   // retain the token: every reader of the old length has finished
@@ -378,18 +434,21 @@ static cudaError_t decode_impl(const void *q, const void *k, const void *v, cons
                                const float *beta, const uint8_t *route, const float *w,
                                float *state, void *k_cache, void *v_cache, int32_t *cache_len,
                                int32_t cap, void *out, float scale_la, float scale_sm, float eps,
-                               void *ws, Shape s, cudaStream_t st) {
+                               void *ws, Shape s, cudaStream_t st, HeadGroups hg) {
     constexpr int kTileBytes = kTileKeys * D * (int)sizeof(T);
     constexpr int kRing = 2 * kStages * kTileBytes;
     constexpr int kRed = 32 * D * 4;               // per-stream / per-slot reduction scratch
     constexpr int kSmem = kRing > kRed ? kRing : kRed;
-    cudaError_t e = cudaFuncSetAttribute(decode_step_kernel<T, D>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    const bool grouped = hg.G > 1 || hg.norm_eps >= 0.f;
+    if (grouped && (hg.G > 4 || D % (32 * hg.G) != 0)) return cudaErrorInvalidValue;
+    auto kernel = grouped ? decode_step_kernel<T, D, true> : decode_step_kernel<T, D, false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
     if (e != cudaSuccess) return e;
     dim3 grid(kCtasPerHead, s.B * s.H);
-    decode_step_kernel<T, D><<<grid, kThreads, kSmem, st>>>(
+    kernel<<<grid, kThreads, kSmem, st>>>(
         (const T *)q, (const T *)k, (const T *)v, g, beta, route, w, state, (T *)k_cache,
-        (T *)v_cache, cache_len, cap, (T *)out, scale_la, scale_sm, eps, (uint8_t *)ws, s.B * s.H);
+        (T *)v_cache, cache_len, cap, (T *)out, scale_la, scale_sm, eps, (uint8_t *)ws, s.B * s.H, hg.G,
+        hg.norm_eps);
     count_launch();
     return cudaGetLastError();
 }
@@ -398,9 +457,9 @@ cudaError_t launch_decode_step(const void *q, const void *k, const void *v, cons
                                const float *beta, const uint8_t *route, const float *w,
                                float *state, void *k_cache, void *v_cache, int32_t *cache_len,
                                int32_t cache_cap, void *out, float scale_la, float scale_sm,
-                               float eps, void *ws, Shape s, cudaStream_t st) {
+                               float eps, void *ws, Shape s, cudaStream_t st, HeadGroups hg) {
 #define ARGS q, k, v, g, beta, route, w, state, k_cache, v_cache, cache_len, cache_cap, out, \
-             scale_la, scale_sm, eps, ws, s, st
+             scale_la, scale_sm, eps, ws, s, st, hg
     if (s.bf16) {
         if (s.d == 128) return decode_impl<__nv_bfloat16, 128>(ARGS);
         return decode_impl<__nv_bfloat16, 64>(ARGS);

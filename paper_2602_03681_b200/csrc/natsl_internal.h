@@ -89,7 +89,9 @@ cudaError_t launch_qk_norm_bwd_f32(const void *q, const void *k, bool bf16, cons
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
                                 const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
                                 void *k16, int32_t cap, int32_t capv, bool appending, int32_t *status,
-                                Shape s, cudaStream_t st, HeadGroups hg = HeadGroups{});
+                                Shape s, cudaStream_t st, HeadGroups hg = HeadGroups{}, bool raw_k_sm = false);
+// (hg.norm_eps >= 0: the keys are RMS-normalised per softmax head and stored as fp16 -- in k_sm and k16, or,
+// with raw_k_sm, in k16 only while k_sm, a cache handed on to the decode step, keeps them as given)
 cudaError_t launch_softmax_combine_tc(const void *q, const void *k_sm, const void *v16, int32_t cap,
                                       int32_t capv, const int32_t *sm_idx,
                                       const int32_t *sm_chunk_prefix, const void *o_la16,
@@ -284,7 +286,7 @@ cudaError_t launch_decode_step(const void *q, const void *k, const void *v, cons
                                const float *beta, const uint8_t *route, const float *w,
                                float *state, void *k_cache, void *v_cache, int32_t *cache_len,
                                int32_t cache_cap, void *out, float scale_la, float scale_sm,
-                               float eps, void *ws, Shape s, cudaStream_t st);
+                               float eps, void *ws, Shape s, cudaStream_t st, HeadGroups hg = HeadGroups{});
 cudaError_t launch_decode_block_end(const uint8_t *route_block, const float *g_block, float *state,
                                     float *state_start, int32_t *cache_len, int32_t block_len,
                                     void *ws, Shape s, cudaStream_t st);

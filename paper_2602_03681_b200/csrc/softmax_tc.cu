@@ -588,7 +588,9 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
                     const int32_t *__restrict__ sm_idx, const int32_t *__restrict__ sm_chunk_prefix,
                     __nv_bfloat16 *__restrict__ k_sm, __nv_bfloat16 *__restrict__ v_sm,
                     __half *__restrict__ v16, __half *__restrict__ k16, int cap, int capv, int appending,
-                    int groups, float norm_eps, int32_t *status, int L, int H) {
+                    int groups, float norm_eps, int raw_k_sm, int32_t *status, int L, int H) {
+    // raw_k_sm (with the normalisation): k_sm is a cache that keeps the keys as given; the normalised
+    // fp16 keys then go to k16 only
     constexpr int kVecPerRow = D * 2 / 16;
     constexpr int kRows = 256 / kVecPerRow;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
@@ -622,6 +624,7 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
         const int tok = sm_idx[(size_t)bh * L + row - n_prev];
         const size_t src = (((size_t)b * L + tok) * H + h) * D;
         uint4 kk = reinterpret_cast<const uint4 *>(k + src)[piece];
+        if (norm_eps >= 0.f && raw_k_sm) reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
         if (norm_eps >= 0.f) {
             // RMS-normalised keys of the softmax operation (Section 4.3), per softmax head = per slice of
             // D / groups columns: the slice's pieces sit in neighbouring lanes of the row's lanes
@@ -642,7 +645,7 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
             kk = make_uint4(pack_half2(f[0] * rk, f[1] * rk), pack_half2(f[2] * rk, f[3] * rk),
                             pack_half2(f[4] * rk, f[5] * rk), pack_half2(f[6] * rk, f[7] * rk));
         }
-        reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
+        if (!(norm_eps >= 0.f && raw_k_sm)) reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
         if (dk16 && norm_eps >= 0.f) {
             *dk16 = kk;                                   // already fp16
         } else if (dk16) {
@@ -735,7 +738,7 @@ template <int D>
 static cudaError_t gather_tc_impl(const void *k, const void *v, const int32_t *sm_idx,
                                   const int32_t *pre, void *k_sm, void *v_sm, void *v16, void *k16,
                                   int cap, int capv, bool appending, int32_t *status, Shape s,
-                                  cudaStream_t st, HeadGroups hg) {
+                                  cudaStream_t st, HeadGroups hg, bool raw_k_sm) {
     constexpr int kRows = 256 / (D * 2 / 16);
     const int max_rows = s.L < capv ? s.L : capv;
     const int blocks = (max_rows + kRows - 1) / kRows;
@@ -743,7 +746,7 @@ static cudaError_t gather_tc_impl(const void *k, const void *v, const int32_t *s
     gather_kv_tc_kernel<D><<<grid, 256, 0, st>>>(
         (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, sm_idx, pre, (__nv_bfloat16 *)k_sm,
         (__nv_bfloat16 *)v_sm, (__half *)v16, (__half *)k16, cap, capv, appending ? 1 : 0, hg.G, hg.norm_eps,
-        status, s.L, s.H);
+        raw_k_sm ? 1 : 0, status, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }
@@ -751,10 +754,10 @@ static cudaError_t gather_tc_impl(const void *k, const void *v, const int32_t *s
 cudaError_t launch_gather_kv_tc(const void *k, const void *v, const int32_t *sm_idx,
                                 const int32_t *sm_chunk_prefix, void *k_sm, void *v_sm, void *v16,
                                 void *k16, int32_t cap, int32_t capv, bool appending, int32_t *status,
-                                Shape s, cudaStream_t st, HeadGroups hg) {
+                                Shape s, cudaStream_t st, HeadGroups hg, bool raw_k_sm) {
     if (s.d == 128)
-        return gather_tc_impl<128>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st, hg);
-    return gather_tc_impl<64>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st, hg);
+        return gather_tc_impl<128>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st, hg, raw_k_sm);
+    return gather_tc_impl<64>(k, v, sm_idx, sm_chunk_prefix, k_sm, v_sm, v16, k16, cap, capv, appending, status, s, st, hg, raw_k_sm);
 }
 
 }  // namespace natsl

@@ -9,6 +9,7 @@ on the same seeded inputs:
   and the segmented scan;
 * the backward for fp32 storage and for bf16 storage at d = 128, including the Jacobians of the two
   normalisations;
+* generation: natsl_decode_step (and the block end) with grouped heads and the normalisation;
 * requests that are not built come back as NATSL_ERR_UNSUPPORTED, before any launch.
 """
 import dataclasses
@@ -296,6 +297,103 @@ def test_saved_forward_then_backward_with_grouped_heads(storage, block):
     check_bwd(wl, {n: v.float().cpu().numpy() for n, v in outs.items()}, ref_b, TOL[storage], large_only=False)
 
 
+@pytest.mark.parametrize("storage,d,G,norm,block,B,H,L", [
+    ("bf16", 128, 2, True, True, 2, 3, 192),       # the paper's mode in generation: decision open, roll-back per block
+    ("bf16", 128, 2, True, False, 2, 2, 160),
+    ("bf16", 128, 2, False, False, 1, 2, 96),
+    ("bf16", 64, 1, True, False, 2, 2, 96),
+    ("f32", 128, 4, True, True, 1, 2, 128),
+    ("f32", 64, 2, True, False, 2, 1, 96),
+])
+def test_generation_with_grouped_heads(storage, d, G, norm, block, B, H, L):
+    """natsl_decode_step with grouped heads and the normalisation, from an empty state and cache: step t
+    equals row t of the forward over the whole sequence (oracle/grouped.py); the cache keeps the keys as given."""
+    from paper_2602_03681_b200 import binding
+    base = "cfg0_f32_tiny_fwd" if storage == "f32" else ("cfg1_bf16_prefill" if d == 128 else "cfg4_bf16_train")
+    wl = dataclasses.replace(inputs.WORKLOADS[base], d=d, seed=101 + d + G)
+    x = make_inputs(wl, B, H, L, norm, block_p=0.4 if block else None)
+    scale_sm = (d / G) ** -0.5 if norm else wl.scale_sm
+    ref = grouped.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], G=G, qk_norm=norm,
+                             scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6, block=64 if block else None)
+    dt = tdtype(wl)
+    code = binding.NATSL_F32 if storage == "f32" else binding.NATSL_BF16
+    p = binding.make_params(B, H, 0, d, code, wl.scale_la, scale_sm, flags=binding.QK_NORM if norm else 0, G=G,
+                            norm_eps=1e-6)
+    ws = binding.alloc_workspace(p, binding.OP_DECODE)
+    state = torch.zeros((B, H, d, d), device="cuda")
+    start = state.clone()
+    kc = torch.zeros((B, H, L, d), dtype=dt, device="cuda")
+    vc = torch.zeros_like(kc)
+    n = torch.zeros((B, H), dtype=torch.int32, device="cuda")
+    undecided = torch.full((B, H), 2, dtype=torch.uint8, device="cuda")
+    for t in range(L):
+        w = dev(x["w"][:, t])
+        p.w = w.data_ptr()
+        out = torch.empty((B, H, d), dtype=dt, device="cuda")
+        binding.natsl_decode_step(dev(x["q"][:, t], dt), dev(x["k"][:, t], dt), dev(x["v"][:, t], dt),
+                                  dev(x["g"][:, t]), dev(x["beta"][:, t]),
+                                  undecided if block else dev(x["route"][:, t]), state, kc, vc, n, out, p, ws)
+        check_stored(out.float().cpu().numpy(), ref["out"][:, t], TOL[storage], wl.dtype, f"step{t}")
+        if block and (t + 1) % 64 == 0:
+            g_block = x["g"][:, t - 63:t + 1].astype(np.float64).sum(1).astype(np.float32)
+            binding.natsl_decode_block_end(dev(x["route"][:, t]), dev(g_block), state, start, n, 64, p, ws)
+    assert binding.natsl_device_status(ws) == 0
+    assert rel_err(state.cpu().numpy(), ref["state_out"]) <= max(TOL[storage], 1e-3) * (1 if storage == "f32" else 1)
+    kept = x["route"].sum(1).T if not block else x["route"][:, ::64].sum(1).T * 64      # [H,B] -> compare as [B,H]
+    assert np.array_equal(n.cpu().numpy(), kept.T.astype(np.int32))
+    b0, h0 = 0, H - 1                       # the cache rows are the retained tokens' keys as given
+    rows = np.nonzero(x["route"][b0, :, h0])[0]
+    assert np.array_equal(kc[b0, h0, :len(rows)].float().cpu().numpy(), x["k"][b0, rows, h0])
+
+
+@pytest.mark.parametrize("storage,d,G,block,B,H,L0,L", [
+    ("bf16", 128, 2, True, 2, 3, 256, 384),
+    ("bf16", 128, 2, False, 1, 2, 192, 256),
+    ("f32", 64, 2, True, 1, 2, 128, 192),
+])
+def test_prefill_then_generation_with_grouped_heads(storage, d, G, block, B, H, L0, L):
+    """Prefill L0 tokens with the normalisation on, hand state and cache to natsl_decode_step, generate up to
+    L: every generated step equals its row of the forward over the whole sequence.  The cache the prefill
+    returns holds the keys as given; the prefill's own softmax kernel read a normalised copy."""
+    from paper_2602_03681_b200 import binding
+    base = "cfg0_f32_tiny_fwd" if storage == "f32" else "cfg1_bf16_prefill"
+    wl = dataclasses.replace(inputs.WORKLOADS[base], d=d, seed=111 + d + G)
+    x = make_inputs(wl, B, H, L, True, block_p=0.4 if block else None)
+    scale_sm = (d / G) ** -0.5
+    ref = grouped.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], G=G, qk_norm=True,
+                             scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6, block=64 if block else None)
+    dt = tdtype(wl)
+    flags = binding.QK_NORM | (binding.BLOCK_ROUTING if block else 0)
+    pre = binding.hybrid_fwd(*(dev(x[n][:, :L0], dt) for n in ("q", "k", "v")), dev(x["g"][:, :L0]),
+                             dev(x["beta"][:, :L0]), dev(x["route"][:, :L0]), dev(x["w"][:, :L0]),
+                             scale_la=wl.scale_la, scale_sm=scale_sm, want=("state_out", "cache"), sm_cap=L,
+                             flags=flags, G=G, norm_eps=1e-6)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(pre["ws"]) == 0
+    check_stored(pre["out"].float().cpu().numpy(), ref["out"][:, :L0], TOL[storage], wl.dtype, "prefill")
+    state, kc, vc, n = pre["state_out"], pre["k_sm"], pre["v_sm"], pre["sm_len"]
+    rows = np.nonzero(x["route"][0, :L0, 0])[0]
+    assert np.array_equal(kc[0, 0, :len(rows)].float().cpu().numpy(), x["k"][0, rows, 0])      # as given
+    code = binding.NATSL_F32 if storage == "f32" else binding.NATSL_BF16
+    p = binding.make_params(B, H, 0, d, code, wl.scale_la, scale_sm, flags=binding.QK_NORM, G=G, norm_eps=1e-6)
+    ws = binding.alloc_workspace(p, binding.OP_DECODE)
+    start = state.clone()
+    undecided = torch.full((B, H), 2, dtype=torch.uint8, device="cuda")
+    for t in range(L0, L):
+        w = dev(x["w"][:, t])
+        p.w = w.data_ptr()
+        out = torch.empty((B, H, d), dtype=dt, device="cuda")
+        binding.natsl_decode_step(dev(x["q"][:, t], dt), dev(x["k"][:, t], dt), dev(x["v"][:, t], dt),
+                                  dev(x["g"][:, t]), dev(x["beta"][:, t]),
+                                  undecided if block else dev(x["route"][:, t]), state, kc, vc, n, out, p, ws)
+        check_stored(out.float().cpu().numpy(), ref["out"][:, t], TOL[storage], wl.dtype, f"step{t}")
+        if block and (t + 1) % 64 == 0:
+            g_block = x["g"][:, t - 63:t + 1].astype(np.float64).sum(1).astype(np.float32)
+            binding.natsl_decode_block_end(dev(x["route"][:, t]), dev(g_block), state, start, n, 64, p, ws)
+    assert binding.natsl_device_status(ws) == 0
+    assert rel_err(state.cpu().numpy(), ref["state_out"]) <= max(TOL[storage], 1e-3)
+
+
 def test_normalisation_ignores_row_lengths_on_the_device():
     """Rescaling the q and k rows by powers of two changes no bf16 mantissa, so with norm_eps = 0 the
     normalised layer must return almost the same bits."""
@@ -333,7 +431,8 @@ def test_requests_that_are_not_built_are_refused():
 
     assert refused(lambda: binding.hybrid_fwd(*args, G=4, **kw))                                  # d/G = 32 on tensor cores
     assert refused(lambda: binding.hybrid_fwd(*args, G=2, flags=binding.FORCE_SIMT, **kw))        # bf16 on CUDA cores
-    assert refused(lambda: binding.hybrid_fwd(*args, flags=binding.QK_NORM, want=("cache",), **kw))
+    assert refused(lambda: binding.hybrid_fwd(*args, flags=binding.QK_NORM | binding.APPEND_CACHE,
+                                              want=("cache",), **kw))
     with pytest.raises(binding.NatslError):                                                       # G must divide d
         binding.hybrid_fwd(*args, G=3, **kw)
     # backward: bf16 storage at d = 64 (the fused chunk kernel's path) has no normalisation
