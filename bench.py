@@ -834,8 +834,27 @@ def bench_decode(args, peaks, peak_kind, traffic):
     mean_len = float(x["cache_len"].mean()) + 0.5 * float(x["route"].mean()) * T
     bytes_step = decode_bytes_per_step(B, H, d, mean_len)
     gbs = bytes_step / (ms / T * 1e-3) / 1e9
+    # the same trajectory with two softmax heads per linear head and q, k normalised inside the kernel
+    # (Section 4.3): same bytes, more arithmetic per cached key
+    p = binding.make_params(B, H, 0, d, binding.NATSL_BF16, wl.scale_la, float(d // 2) ** -0.5,
+                            flags=binding.QK_NORM, G=2, norm_eps=1e-6)
+    ms_grouped = float("inf")
+    for rep in range(2):          # (the first repetition loads the kernel)
+        state.copy_(state0)
+        n.copy_(n0)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        trajectory()
+        e1.record()
+        torch.cuda.synchronize()
+        if rep:
+            ms_grouped = e0.elapsed_time(e1)
+    assert binding.natsl_device_status(ws) == 0
     return {"workload": wl.name, "value": B * T / (ms * 1e-3), "unit": "tokens/s",
             "ms_per_step": ms / T, "steps": T,
+            "grouped_heads_G2_qk_norm": {"ms_per_step": ms_grouped / T,
+                                         "frac_of_hbm_peak": bytes_step / (ms_grouped / T * 1e-3) / 1e9 / peaks["hbm_gbs"]},
             "roofline": {"kernel": "decode_step", "bound": "hbm", "achieved": gbs,
                          "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                          "peak_source": peak_kind, "algorithmic_bytes_per_launch": bytes_step,

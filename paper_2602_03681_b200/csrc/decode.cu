@@ -182,6 +182,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
 #pragma unroll
             for (int x = 0; x < kE; ++x) qf[x] = (kGrouped ? qsm[piece * kE + x] : qs[piece * kE + x]) * scale_sm;
             const int lps = kLpk / G;              // lanes per softmax head within a key row
+            const float inv_ds = 1.f / ds;
             float m = -INFINITY, z = 0.f, acc[kE];
 #pragma unroll
             for (int x = 0; x < kE; ++x) acc[x] = 0.f;
@@ -206,11 +207,13 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
                         float kk = 0.f;
 #pragma unroll
                         for (int x = 0; x < kE; ++x) kk = fmaf(kx[x], kx[x], kk);
-                        for (int o = lps / 2; o > 0; o >>= 1) {
-                            sc += __shfl_xor_sync(0xffffffffu, sc, o);
-                            kk += __shfl_xor_sync(0xffffffffu, kk, o);
-                        }
-                        if (normed) sc *= rsqrtf(kk / ds + norm_eps);
+#pragma unroll
+                        for (int o = kLpk / 2; o > 0; o >>= 1)
+                            if (o < lps) {           // (uniform: the group count is the same for every lane)
+                                sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                                kk += __shfl_xor_sync(0xffffffffu, kk, o);
+                            }
+                        if (normed) sc *= rsqrtf(fmaf(kk, inv_ds, norm_eps));
                     }
                     if (j < rows) {                            // rows past the slice hold stale bytes
                         const float m_new = fmaxf(m, sc);
