@@ -185,9 +185,9 @@ typedef struct natsl_params {
                             /*   the same shapes except bf16 storage with d = 64 (self-contained or    */
                             /*   from a saved forward; no p->dscore); natsl_decode_step for d / G in   */
                             /*   {32, 64, 128}.  A cache returned or read with NATSL_QK_NORM holds the */
-                            /*   keys as given: they are normalised as they are read.  G > 1 or        */
-                            /*   NATSL_QK_NORM with anything else (NATSL_APPEND_CACHE, NATSL_FORCE_SIMT */
-                            /*   on bf16): NATSL_ERR_UNSUPPORTED.                                      */
+                            /*   keys as given: they are normalised as they are read                   */
+                            /*   (NATSL_APPEND_CACHE included).  G > 1 or NATSL_QK_NORM with           */
+                            /*   NATSL_FORCE_SIMT on bf16: NATSL_ERR_UNSUPPORTED.                      */
     float norm_eps;         /* NATSL_QK_NORM: epsilon under the square roots, >= 0                     */
 } natsl_params;
 

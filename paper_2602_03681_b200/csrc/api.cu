@@ -66,6 +66,7 @@ struct FwdWs {
     int32_t *status, *emit_flags, *sm_idx, *prefix, *lin_idx, *n_lin, *sm_len;
     size_t head_bytes;          // status page + emit_flags: cleared at the start of every call
     void *k_sm, *v_sm, *v16;
+    void *kn16;                 // prefill in pieces with NATSL_QK_NORM: normalised fp16 keys of the whole cache
     void *o_la16;               // tensor-core path: the linear read-out as fp16 [B,L,H,d]
     float *W, *U, *P, *o_la;    // fp32 CUDA-core path only
     float *q_la, *k_la, *q_sm, *k_nsm;   // fp32 storage with NATSL_QK_NORM: normalised copies of q and k
@@ -108,6 +109,7 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
         // fp16 V of the retained tokens; when the call appends to a cache, of the whole cache
         const size_t capv = (p->flags & NATSL_APPEND_CACHE) && p->sm_cap > 0 ? (size_t)p->sm_cap : L;
         f.v16 = c.take<char>(B * H * capv * d * 2);
+        f.kn16 = c.take<char>((p->flags & NATSL_APPEND_CACHE) && (p->flags & NATSL_QK_NORM) ? B * H * capv * d * 2 : 0);
         f.tc.Qh = c.take<char>(B * H * L * d * 2);
         f.tc.Kh = c.take<char>(B * H * L * d * 2);
         f.tc.Wt = c.take<char>(B * H * L * d * 2);
@@ -123,6 +125,7 @@ FwdWs carve_fwd(const natsl_params *p, void *ws) {
         f.o_la = nullptr;
     } else {
         f.v16 = nullptr;
+        f.kn16 = nullptr;
         f.o_la16 = nullptr;
         f.tc = GdnTcWs{};
         f.seg_incr = f.seg_trans = f.seg_start = nullptr;
@@ -473,7 +476,6 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     if (append && !want_cache) return NATSL_ERR_NULL;
     const HeadGroups hg = head_groups(p);
     if (grouped_or_normed(p)) {
-        if (append) return NATSL_ERR_UNSUPPORTED;
         if (tensor_cores) {
             if (hg.G > 1 && !(hg.G == 2 && p->d == 128)) return NATSL_ERR_UNSUPPORTED;
             // (the saved forward is the backward's forward part: built where the backward is)
@@ -539,11 +541,12 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
     // A cache the call returns keeps the keys as given (the decode step normalises them as it reads them);
     // with the normalisation the softmax kernel then reads a normalised copy in the workspace instead.
     const bool raw_cache = want_cache && hg.norm_eps >= 0.f;
-    const void *k_soft = raw_cache ? f.k_sm : k_sm, *v_soft = raw_cache ? f.v_sm : v_sm;
-    const int32_t cap_soft = raw_cache ? p->L : cap;
+    void *k_norm = append ? f.kn16 : f.k_sm;     // (appending: normalised copies of the whole cache, capv rows per head)
+    const void *k_soft = raw_cache ? k_norm : k_sm, *v_soft = raw_cache ? f.v_sm : v_sm;
+    const int32_t cap_soft = raw_cache ? capv : cap;
     if (tensor_cores) {
         NATSL_TRY(launch_gather_kv_tc(k, v, f.sm_idx, f.prefix, k_sm, want_cache ? v_sm : nullptr,
-                                      f.v16, raw_cache ? f.k_sm : nullptr, cap, capv, append, f.status, s, st0,
+                                      f.v16, raw_cache ? k_norm : nullptr, cap, capv, append, f.status, s, st0,
                                       hg, raw_cache));
     } else {
         if (raw_cache) NATSL_TRY(launch_gather_kv(k, v, f.sm_idx, f.prefix, k_sm, v_sm, cap, f.status, s, st));

@@ -601,6 +601,26 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
     const int n_pad = min((n + 127) / 128 * 128, capv);
     const int n_prev = appending ? sm_chunk_prefix[(size_t)bh * (NC + 1)] : 0;   // rows of earlier calls
     const int piece = threadIdx.x % kVecPerRow;
+    // RMS-normalised keys of the softmax operation (Section 4.3), per softmax head = per slice of D / groups
+    // columns, as fp16 (the softmax kernel's logit product is an fp16 MMA in this mode): the slice's pieces
+    // sit in neighbouring lanes of the row's lanes.  bf16 pieces in, fp16 pieces out.
+    auto rms_fp16 = [&](uint4 kk) {
+        const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
+        float f[8], ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __uint_as_float(kw[i] << 16);
+            f[2 * i + 1] = __uint_as_float(kw[i] & 0xffff0000u);
+            ss = fmaf(f[2 * i], f[2 * i], fmaf(f[2 * i + 1], f[2 * i + 1], ss));
+        }
+        const int lanes = kVecPerRow / groups;            // lanes per slice (a power of two)
+        const unsigned row_mask = (kVecPerRow == 32 ? 0xffffffffu : ((1u << kVecPerRow) - 1u))
+                                  << ((threadIdx.x & 31) & ~(kVecPerRow - 1));
+        for (int o = 1; o < lanes; o <<= 1) ss += __shfl_xor_sync(row_mask, ss, o);
+        const float rk = rsqrtf(ss * groups / D + norm_eps);
+        return make_uint4(pack_half2(f[0] * rk, f[1] * rk), pack_half2(f[2] * rk, f[3] * rk),
+                          pack_half2(f[4] * rk, f[5] * rk), pack_half2(f[6] * rk, f[7] * rk));
+    };
     // the grid is sized for a typical retention rate; each CTA strides over the rows there are
     for (int row = blockIdx.x * kRows + threadIdx.x / kVecPerRow; row < n_pad; row += gridDim.x * kRows) {
         uint4 *dv16 = reinterpret_cast<uint4 *>(v16 + ((size_t)bh * capv + row) * D) + piece;
@@ -619,32 +639,15 @@ gather_kv_tc_kernel(const __nv_bfloat16 *__restrict__ k, const __nv_bfloat16 *__
             for (int i = 0; i < 4; ++i)
                 o[i] = pack_half2(__uint_as_float(wv[i] << 16), __uint_as_float(wv[i] & 0xffff0000u));
             *dv16 = make_uint4(o[0], o[1], o[2], o[3]);
+            // (and, with the normalisation, the normalised copy of its key, which the cache keeps as given)
+            if (dk16 && norm_eps >= 0.f) *dk16 = rms_fp16(reinterpret_cast<const uint4 *>(k_sm + dst)[piece]);
             continue;
         }
         const int tok = sm_idx[(size_t)bh * L + row - n_prev];
         const size_t src = (((size_t)b * L + tok) * H + h) * D;
         uint4 kk = reinterpret_cast<const uint4 *>(k + src)[piece];
         if (norm_eps >= 0.f && raw_k_sm) reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
-        if (norm_eps >= 0.f) {
-            // RMS-normalised keys of the softmax operation (Section 4.3), per softmax head = per slice of
-            // D / groups columns: the slice's pieces sit in neighbouring lanes of the row's lanes
-            const uint32_t kw[4] = {kk.x, kk.y, kk.z, kk.w};
-            float f[8], ss = 0.f;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                f[2 * i] = __uint_as_float(kw[i] << 16);
-                f[2 * i + 1] = __uint_as_float(kw[i] & 0xffff0000u);
-                ss = fmaf(f[2 * i], f[2 * i], fmaf(f[2 * i + 1], f[2 * i + 1], ss));
-            }
-            const int lanes = kVecPerRow / groups;            // lanes per slice (a power of two)
-            const unsigned row_mask = (kVecPerRow == 32 ? 0xffffffffu : ((1u << kVecPerRow) - 1u))
-                                      << ((threadIdx.x & 31) & ~(kVecPerRow - 1));
-            for (int o = 1; o < lanes; o <<= 1) ss += __shfl_xor_sync(row_mask, ss, o);
-            const float rk = rsqrtf(ss * groups / D + norm_eps);
-            // stored as fp16 (the softmax kernel's logit product is an fp16 MMA in this mode)
-            kk = make_uint4(pack_half2(f[0] * rk, f[1] * rk), pack_half2(f[2] * rk, f[3] * rk),
-                            pack_half2(f[4] * rk, f[5] * rk), pack_half2(f[6] * rk, f[7] * rk));
-        }
+        if (norm_eps >= 0.f) kk = rms_fp16(kk);
         if (!(norm_eps >= 0.f && raw_k_sm)) reinterpret_cast<uint4 *>(k_sm + dst)[piece] = kk;
         if (dk16 && norm_eps >= 0.f) {
             *dk16 = kk;                                   // already fp16

@@ -394,6 +394,47 @@ def test_prefill_then_generation_with_grouped_heads(storage, d, G, block, B, H, 
     assert rel_err(state.cpu().numpy(), ref["state_out"]) <= max(TOL[storage], 1e-3)
 
 
+@pytest.mark.parametrize("G,norm,block,B,H,pieces", [
+    (2, True, True, 1, 3, (256, 128, 320)),
+    (2, True, False, 2, 2, (192, 320)),
+    (2, False, False, 1, 2, (128, 256)),
+    (1, True, False, 1, 2, (320, 192)),
+])
+def test_prefill_in_pieces_with_grouped_heads(G, norm, block, B, H, pieces):
+    """NATSL_APPEND_CACHE with grouped heads and the normalisation: the pieces' outputs equal the forward over
+    the whole sequence; the cache holds the keys as given, and a later piece reads normalised copies of the
+    earlier pieces' keys made from it."""
+    from paper_2602_03681_b200 import binding
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg1_bf16_prefill"], seed=121 + G)
+    d, L = wl.d, sum(pieces)
+    x = make_inputs(wl, B, H, L, norm, block_p=0.35 if block else None)
+    scale_sm = (d / G) ** -0.5 if norm else wl.scale_sm
+    ref = grouped.hybrid_fwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], G=G, qk_norm=norm,
+                             scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6, block=64 if block else None)
+    dt = torch.bfloat16
+    flags = binding.APPEND_CACHE | (binding.QK_NORM if norm else 0) | (binding.BLOCK_ROUTING if block else 0)
+    k_sm = torch.zeros((B, H, L, d), dtype=dt, device="cuda")
+    v_sm = torch.zeros_like(k_sm)
+    sm_len = torch.zeros((B, H), dtype=torch.int32, device="cuda")
+    state, outs, t0 = None, [], 0
+    for n in pieces:
+        sl = slice(t0, t0 + n)
+        res = binding.hybrid_fwd(*(dev(x[m][:, sl], dt) for m in ("q", "k", "v")), dev(x["g"][:, sl]),
+                                 dev(x["beta"][:, sl]), dev(x["route"][:, sl]), dev(x["w"][:, sl]),
+                                 scale_la=wl.scale_la, scale_sm=scale_sm, state_in=state, want=("state_out",),
+                                 cache=(k_sm, v_sm, sm_len), flags=flags, G=G, norm_eps=1e-6)
+        torch.cuda.synchronize()
+        assert binding.natsl_device_status(res["ws"]) == 0
+        state = res["state_out"]
+        outs.append(res["out"].float().cpu().numpy())
+        t0 += n
+    check_stored(np.concatenate(outs, 1), ref["out"], TOL["bf16"], "bf16")
+    assert rel_err(state.cpu().numpy(), ref["state_out"]) <= TOL["bf16"]
+    rows = np.nonzero(x["route"][0, :, 0])[0]
+    assert sm_len[0, 0].item() == len(rows)
+    assert np.array_equal(k_sm[0, 0, :len(rows)].float().cpu().numpy(), x["k"][0, rows, 0])
+
+
 def test_normalisation_ignores_row_lengths_on_the_device():
     """Rescaling the q and k rows by powers of two changes no bf16 mantissa, so with norm_eps = 0 the
     normalised layer must return almost the same bits."""
@@ -431,8 +472,6 @@ def test_requests_that_are_not_built_are_refused():
 
     assert refused(lambda: binding.hybrid_fwd(*args, G=4, **kw))                                  # d/G = 32 on tensor cores
     assert refused(lambda: binding.hybrid_fwd(*args, G=2, flags=binding.FORCE_SIMT, **kw))        # bf16 on CUDA cores
-    assert refused(lambda: binding.hybrid_fwd(*args, flags=binding.QK_NORM | binding.APPEND_CACHE,
-                                              want=("cache",), **kw))
     with pytest.raises(binding.NatslError):                                                       # G must divide d
         binding.hybrid_fwd(*args, G=3, **kw)
     # backward: bf16 storage at d = 64 (the fused chunk kernel's path) has no normalisation
