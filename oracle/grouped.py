@@ -36,7 +36,12 @@ def rms_normalise(x, norm_eps):
     return x / torch.sqrt((x * x).mean(-1, keepdim=True) + norm_eps)
 
 
-def _forward(q, k, v, g, beta, route, w, G, qk_norm, scale_la, scale_sm, eps, norm_eps, state_in, block=None):
+def _forward(q, k, v, g, beta, route, w, G, qk_norm, scale_la, scale_sm, eps, norm_eps, state_in, block=None,
+             masks=None):
+    # masks (block mode only): [B, L/block, H, 2] of ones = (linear, softmax) operation masks of the blocks,
+    # present so that their gradients can be taken (Section 4.2): the linear one multiplies the update a
+    # linear block commits to the state, the softmax one multiplies the unnormalised probabilities of a
+    # softmax block's keys.
     B, L, H, d = q.shape
     ds = d // G
     lin = (route == 0).to(q.dtype)                       # [B,L,H]: 1 for linear tokens
@@ -63,7 +68,11 @@ def _forward(q, k, v, g, beta, route, w, G, qk_norm, scale_la, scale_sm, eps, no
         if block and i % block == block - 1:
             # ... and a softmax block's update is rolled back: only the decay remains
             keep = lin[:, i][:, :, None, None]
-            S = keep * S + (1 - keep) * decay[:, :, None, None] * S_start
+            rolled = decay[:, :, None, None] * S_start
+            if masks is not None:        # S_next = decay S_start + m_la U, U = the block's update
+                S = rolled + keep * masks[:, i // block, :, 0][:, :, None, None] * (S - rolled)
+            else:
+                S = keep * S + (1 - keep) * rolled
     o_la = torch.stack(o_la, 1)                          # [B,L,H,d]
     # ---- softmax operation: G heads per linear head, keys = retained tokens j <= i ----
     qs, ks, vs = (x.reshape(B, L, H, G, ds) for x in (q, k, v))
@@ -81,6 +90,12 @@ def _forward(q, k, v, g, beta, route, w, G, qk_norm, scale_la, scale_sm, eps, no
     m = masked.max(-1, keepdim=True).values
     m_safe = torch.where(torch.isfinite(m), m, torch.zeros_like(m))
     p = torch.exp(masked - m_safe)                       # exp(-inf) = 0 at the keys a query does not see
+    if masks is not None:
+        # the softmax mask of key j's block, for every query that sees the key (what it does to the keys of a
+        # linear block, seen inside their own block only, is discarded: that block did not choose softmax)
+        blk = torch.arange(L) // block
+        mk = masks[:, :, :, 1].permute(0, 2, 1)[:, :, blk]                    # [B,H,L(key)]
+        p = p * mk[:, :, None, None, :]
     z = p.sum(-1, keepdim=True)
     any_key = z > 0
     p = p / torch.where(any_key, z, torch.ones_like(z))
@@ -128,7 +143,7 @@ def hybrid_fwd(q, k, v, g, beta, route, w=None, *, G=1, qk_norm=False, scale_la,
 
 
 def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, G=1, qk_norm=False, scale_la, scale_sm, eps=1e-5,
-               norm_eps=1e-6, state_in=None, dstate_out=None, block=None):
+               norm_eps=1e-6, state_in=None, dstate_out=None, block=None, want_dscore=False):
     """Gradients of <out, dout> (+ <state_out, dstate_out>) with respect to q, k, v, g, beta, w and
     state_in.  Returns dict(dq, dk, dv, dg, dbeta, dw, dstate_in)."""
     _check(np.asarray(q), np.asarray(route), G, block)
@@ -139,11 +154,22 @@ def hybrid_bwd(q, k, v, g, beta, route, w, dout, *, G=1, qk_norm=False, scale_la
         state_in = np.zeros((B, H, d, d))
     leaves = [_t(x, True) for x in (q, k, v, g, beta, w, state_in)]
     tq, tk, tv, tg, tb, tw, ts = leaves
+    masks = None
+    if want_dscore:
+        if not block:
+            raise ValueError("score gradients: one decision per block")
+        masks = torch.ones((B, L // block, H, 2), dtype=torch.float64, requires_grad=True)
+        leaves = leaves + [masks]
     res = _forward(tq, tk, tv, tg, tb, torch.from_numpy(np.asarray(route).astype(np.int64)), tw, G, qk_norm,
-                   scale_la, scale_sm, eps, norm_eps, ts, block)
+                   scale_la, scale_sm, eps, norm_eps, ts, block, masks)
     loss = (res["out"] * _t(dout)).sum()
     if dstate_out is not None:
         loss = loss + (res["state_out"] * _t(dstate_out)).sum()
     grads = torch.autograd.grad(loss, leaves, allow_unused=True)
-    names = ("dq", "dk", "dv", "dg", "dbeta", "dw", "dstate_in")
-    return {n: (np.zeros(tuple(x.shape)) if gr is None else gr.numpy()) for n, gr, x in zip(names, grads, leaves)}
+    names = ("dq", "dk", "dv", "dg", "dbeta", "dw", "dstate_in", "dscore")
+    out = {n: (np.zeros(tuple(x.shape)) if gr is None else gr.numpy()) for n, gr, x in zip(names, grads, leaves)}
+    if want_dscore:      # only the operation a block chose has a mask gradient ("d score = 0 if the mask is 0")
+        blocks = np.asarray(route)[:, ::block]                                # [B, L/block, H]
+        out["dscore"][..., 0][blocks != 0] = 0.0
+        out["dscore"][..., 1][blocks == 0] = 0.0
+    return out

@@ -220,6 +220,33 @@ def test_block_mode_group_heads_are_block_mode_heads_over_column_slices():
         gf(y, G=G, block=R)
 
 
+def test_block_mode_score_gradients_equal_the_c_oracles_and_add_over_the_group():
+    B, L, H, d, R = 1, 96, 2, 16, 16
+    x = rand_inputs(B, L, H, d, seed=30)
+    x["route"] = block_route(B, L, H, R, 0.5, 4)
+    r = np.random.default_rng(5)
+    dout = r.standard_normal(x["q"].shape)
+    a = gb(x, dout, G=1, block=R, want_dscore=True)
+    c = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], dout, block=R, **KW)
+    np.testing.assert_allclose(a["dscore"], c["dscore"], rtol=1e-8, atol=1e-10)
+    assert np.abs(c["dscore"][..., 0]).max() > 0 and np.abs(c["dscore"][..., 1]).max() > 0
+    for n in ("dq", "dk", "dg"):                           # the masks leave the other gradients alone
+        np.testing.assert_allclose(a[n], c[n], rtol=1e-8, atol=1e-10, err_msg=n)
+    # grouped heads share their linear head's mask: its gradient is the sum over the group's heads, i.e. what
+    # the C oracle gives for the column slices run as separate heads, added up (softmax operation; weights 1, 0
+    # keep the linear operation out of it)
+    G = 2
+    w1 = np.zeros((B, L, H, 2)); w1[..., 0] = 1.0
+    y = dict(x); y["w"] = w1
+    ag = gb(y, dout, G=G, block=R, want_dscore=True, scale_sm=0.4)
+    sl = {n: x[n].reshape(B, L, H * G, d // G) for n in ("q", "k", "v")}
+    rep = {n: np.repeat(x[n], G, axis=2) for n in ("g", "beta", "route")}
+    cg = oracle.hybrid_bwd(sl["q"], sl["k"], sl["v"], rep["g"], rep["beta"], rep["route"], np.repeat(w1, G, axis=2),
+                           dout.reshape(B, L, H * G, d // G), block=R, scale_la=0.5, scale_sm=0.4)
+    np.testing.assert_allclose(ag["dscore"][..., 1], cg["dscore"][..., 1].reshape(B, L // R, H, G).sum(-1),
+                               rtol=1e-8, atol=1e-10)
+
+
 def test_rejects_group_count_that_does_not_divide():
     x = rand_inputs(1, 8, 1, 8, seed=27)
     with pytest.raises(ValueError):
