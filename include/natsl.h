@@ -183,7 +183,8 @@ typedef struct natsl_params {
                             /*   d = 128, G = 2 (the appendix's two softmax heads per linear head;     */
                             /*   three would need d = 192); natsl_hybrid_bwd with either routing for   */
                             /*   the same shapes except bf16 storage with d = 64 (self-contained or    */
-                            /*   from a saved forward; no p->dscore); natsl_decode_step for d / G in   */
+                            /*   from a saved forward; p->dscore: the softmax heads of a group share   */
+                            /*   the block's mask, their gradients add); natsl_decode_step for d / G in */
                             /*   {32, 64, 128}.  A cache returned or read with NATSL_QK_NORM holds the */
                             /*   keys as given: they are normalised as they are read                   */
                             /*   (NATSL_APPEND_CACHE included).  G > 1 or NATSL_QK_NORM with           */

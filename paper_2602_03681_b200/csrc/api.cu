@@ -218,7 +218,7 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.kappa = c.take<float>(BHL);
     f.gS = c.take<float>(general ? B * H * NC * (d / 32) : 0);
     f.dk_x = tm(general && block); f.dv_x = tm(general && block);
-    f.dmask = c.take<float>(general && block ? BHL : 0);
+    f.dmask = c.take<float>(general && block ? BHL * Gg : 0);
     const size_t h16 = tcs ? TM * 2 : 0;
     f.k_smb = c.take<char>(h16);
     f.k16 = c.take<char>(h16);
@@ -617,7 +617,6 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (p->flags & NATSL_APPEND_CACHE) return NATSL_ERR_UNSUPPORTED;
     const HeadGroups hg = head_groups(p);
     if (grouped_or_normed(p)) {      // grouped heads, q/k normalisation: the paths with separate chunk-level products
-        if (p->dscore) return NATSL_ERR_UNSUPPORTED;
         if (use_tensor_cores(p)) {
             if (p->d != 128 || hg.G > 2) return NATSL_ERR_UNSUPPORTED;
         } else {
@@ -798,7 +797,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
                                          general_block ? f.dk_x : nullptr));
     }
     if (p->dscore)   // softmax blocks: the mask gradients of their keys; linear blocks: the kappa of their tokens
-        NATSL_TRY(launch_dscore(route, f.prefix, f.dmask, nullptr, f.kappa, p->L, p->dscore, s, st));
+        NATSL_TRY(launch_dscore(route, f.prefix, f.dmask, nullptr, f.kappa, p->L, p->dscore, s, st, hg.G));
 #undef NATSL_TRY
     return NATSL_OK;
 }

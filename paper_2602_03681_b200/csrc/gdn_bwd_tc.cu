@@ -902,12 +902,14 @@ namespace {
 __global__ void __launch_bounds__(64)
 dscore_kernel(const uint8_t *__restrict__ route, const int32_t *__restrict__ sm_chunk_prefix,
               const float *__restrict__ dmask, const float *__restrict__ kap_c,
-              const float *__restrict__ kappa_tok, int cap, float *__restrict__ dscore, int L, int H) {
+              const float *__restrict__ kappa_tok, int cap, float *__restrict__ dscore, int L, int H, int G) {
     const int c = blockIdx.x, bh = blockIdx.y, b = bh / H, h = bh % H, NC = L / kC;
     float *dst = dscore + (((size_t)b * NC + c) * H + h) * 2;
     if (route[((size_t)b * L + (size_t)c * kC) * H + h]) {
+        // (grouped heads: dmask is [B,H,G,cap]; the softmax heads of a group share the block's mask)
         const int row = sm_chunk_prefix[(size_t)bh * (NC + 1) + c] + (int)threadIdx.x;
-        float x = row < cap ? dmask[(size_t)bh * cap + row] : 0.f;
+        float x = 0.f;
+        for (int gg = 0; gg < G; ++gg) x += row < cap ? dmask[((size_t)bh * G + gg) * cap + row] : 0.f;
         x = warp_sum(x);
         __shared__ float part[2];
         if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = x;
@@ -928,9 +930,10 @@ dscore_kernel(const uint8_t *__restrict__ route, const int32_t *__restrict__ sm_
 
 cudaError_t launch_dscore(const uint8_t *route, const int32_t *sm_chunk_prefix, const float *dmask,
                           const float *kap_c, const float *kappa_tok, int cap, float *dscore, Shape s,
-                          cudaStream_t st) {
+                          cudaStream_t st, int G) {
     dim3 grid(s.L / kC, s.B * s.H);
-    dscore_kernel<<<grid, 64, 0, st>>>(route, sm_chunk_prefix, dmask, kap_c, kappa_tok, cap, dscore, s.L, s.H);
+    dscore_kernel<<<grid, 64, 0, st>>>(route, sm_chunk_prefix, dmask, kap_c, kappa_tok, cap, dscore, s.L, s.H,
+                                       G > 1 ? G : 1);
     count_launch();
     return cudaGetLastError();
 }

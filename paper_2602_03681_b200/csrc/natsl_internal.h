@@ -264,7 +264,8 @@ cudaError_t launch_gdn_bwd_chunk(const void *q, const void *k, const void *v, co
 // (kap_c [B,H,L/C]: the chunk sums of kappa, or kappa_tok [B,H,L]: kappa per token, summed here)
 cudaError_t launch_dscore(const uint8_t *route, const int32_t *sm_chunk_prefix, const float *dmask,
                           const float *kap_c, const float *kappa_tok, int cap, float *dscore, Shape s,
-                          cudaStream_t st);
+                          cudaStream_t st, int G = 1);
+// (G > 1: dmask is [B,H,G,cap], summed over the group's softmax heads)
 
 // block-level routing: softmax-branch backward through the own block of the queries of a linear
 // block (adds to dq_sm, writes the dk_x / dv_x rows of the linear blocks); do16: fp16 [B,H,L,d]

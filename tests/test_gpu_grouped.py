@@ -243,6 +243,8 @@ def test_block_level_routing_backward_with_grouped_heads(storage, d, G, norm, B,
                              flags=binding.BLOCK_ROUTING | (binding.QK_NORM if norm else 0))
     w_dev = dev(x["w"])
     pr.w = w_dev.data_ptr()
+    dscore = torch.zeros((B, L // 64, H, 2), device="cuda")
+    pr.dscore = dscore.data_ptr()
     ws = binding.alloc_workspace(pr, binding.OP_BWD)
     t = {n: dev(x[n], dt) for n in ("q", "k", "v", "dout")}
     t.update({n: dev(x[n]) for n in ("g", "beta", "route")})
@@ -255,8 +257,16 @@ def test_block_level_routing_backward_with_grouped_heads(storage, d, G, norm, B,
     assert binding.natsl_device_status(ws) == 0
     got = {n: v.float().cpu().numpy() for n, v in outs.items()}
     ref = grouped.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"], G=G,
-                             qk_norm=norm, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6, block=64)
+                             qk_norm=norm, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6, block=64,
+                             want_dscore=True)
     check_bwd(wl, got, ref, TOL[storage], large_only=not norm)
+    # score gradients (Section 4.2): the group's softmax heads share the block's mask
+    gd = dscore.cpu().numpy()
+    blocks = x["route"][:, ::64]
+    assert np.all(gd[..., 0][blocks == 1] == 0) and np.all(gd[..., 1][blocks == 0] == 0)
+    for op in (0, 1):
+        if np.abs(ref["dscore"][..., op]).max() > 0:
+            assert rel_err(gd[..., op], ref["dscore"][..., op]) <= TOL[storage], (op, rel_err(gd[..., op], ref["dscore"][..., op]))
 
 
 @pytest.mark.parametrize("storage,block", [("bf16", False), ("bf16", True), ("f32", False)])
