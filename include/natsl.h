@@ -182,7 +182,7 @@ typedef struct natsl_params {
                             /*   fp32 storage (d / G in {32, 64, 128}) and on the tensor-core path for */
                             /*   d = 128, G = 2 (the appendix's two softmax heads per linear head;     */
                             /*   three would need d = 192); natsl_hybrid_bwd with either routing for   */
-                            /*   the same shapes except bf16 storage with d = 64 (self-contained or    */
+                            /*   the same shapes (self-contained or                                    */
                             /*   from a saved forward; p->dscore: the softmax heads of a group share   */
                             /*   the block's mask, their gradients add); natsl_decode_step for d / G in */
                             /*   {32, 64, 128}.  A cache returned or read with NATSL_QK_NORM holds the */

@@ -79,6 +79,12 @@ bool use_tensor_cores(const natsl_params *p) {
     return p->dtype == NATSL_BF16 && !(p->flags & NATSL_FORCE_SIMT);
 }
 
+// Backward on tensor cores with d = 64: all chunk-level products in one fused kernel per chunk -- unless
+// q and k are normalised, which that kernel does not know; the separate products then serve d = 64 too.
+bool fused_chunk_path(const natsl_params *p) {
+    return use_tensor_cores(p) && p->d == 64 && !grouped_or_normed(p);
+}
+
 // Segments of the forward scan (tensor-core path): the largest power of two that keeps the two
 // runs per segment within ~one CTA per SM, divides the chunk count and leaves >= 8 chunks each.
 int scan_segments(const natsl_params *p) {
@@ -177,7 +183,7 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     BwdWs f;
     const size_t B = p->B, H = p->H, L = p->L, d = p->d, NC = L / kC;
     const size_t TM = B * L * H * d, CC = B * H * NC * kC * kC, ST = B * H * NC * d * d, BHL = B * H * L;
-    const bool tcs = use_tensor_cores(p), fused = tcs && p->d == 64, general = !fused;
+    const bool tcs = use_tensor_cores(p), fused = fused_chunk_path(p), general = !fused;
     const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
     auto tm = [&](bool need) { return c.take<float>(need ? TM : 0); };
     auto cc = [&](bool need) { return c.take<float>(need ? CC : 0); };
@@ -312,7 +318,7 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
     const bool block = (p->flags & NATSL_BLOCK_ROUTING) != 0;
     const uint8_t *block_route = block ? route : nullptr;
     const bool tensor_cores = use_tensor_cores(p);
-    const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
+    const bool fused_chunks = fused_chunk_path(p);          // chunk-level products in one kernel
     int32_t *flags = tensor_cores && !(p->flags & NATSL_SINGLE_STREAM) ? f.emit_flags : nullptr;
 #define NATSL_TRY(call) do { if ((call) != cudaSuccess) return NATSL_ERR_CUDA; } while (0)
     NATSL_TRY(cudaMemsetAsync(f.status, 0, f.head_bytes, st));
@@ -479,7 +485,7 @@ int natsl_hybrid_fwd(const void *q, const void *k, const void *v, const float *g
         if (tensor_cores) {
             if (hg.G > 1 && !(hg.G == 2 && p->d == 128)) return NATSL_ERR_UNSUPPORTED;
             // (the saved forward is the backward's forward part: built where the backward is)
-            if ((p->flags & NATSL_SAVE_FOR_BWD) && p->d != 128) return NATSL_ERR_UNSUPPORTED;
+            if ((p->flags & NATSL_SAVE_FOR_BWD) && hg.G > 1 && p->d != 128) return NATSL_ERR_UNSUPPORTED;
         } else {
             if (p->dtype != NATSL_F32) return NATSL_ERR_UNSUPPORTED;
             if (hg.G > 1 && (hg.G > 4 || p->d / hg.G < 32)) return NATSL_ERR_UNSUPPORTED;
@@ -617,8 +623,8 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (p->flags & NATSL_APPEND_CACHE) return NATSL_ERR_UNSUPPORTED;
     const HeadGroups hg = head_groups(p);
     if (grouped_or_normed(p)) {      // grouped heads, q/k normalisation: the paths with separate chunk-level products
-        if (use_tensor_cores(p)) {
-            if (p->d != 128 || hg.G > 2) return NATSL_ERR_UNSUPPORTED;
+        if (use_tensor_cores(p)) {      // softmax heads of 64 or 128 columns
+            if (!((p->d == 128 && hg.G <= 2) || (p->d == 64 && hg.G == 1))) return NATSL_ERR_UNSUPPORTED;
         } else {
             if (p->dtype != NATSL_F32) return NATSL_ERR_UNSUPPORTED;
             if (hg.G > 1 && (hg.G > 4 || p->d / hg.G < 32)) return NATSL_ERR_UNSUPPORTED;
@@ -643,7 +649,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     const int di = p->d;
     const uint8_t *block_route = block ? route : nullptr;
     const bool tensor_cores = use_tensor_cores(p);
-    const bool fused_chunks = tensor_cores && p->d == 64;   // chunk-level products in one kernel
+    const bool fused_chunks = fused_chunk_path(p);          // chunk-level products in one kernel
 
     // ---- forward, keeping what the backward needs (unless the caller's forward already did) ----
     if (!(p->flags & NATSL_SAVED_FWD)) {

@@ -25,13 +25,13 @@ from test_gpu_parity import TOL, check_stored, dev, rel_err, tdtype
 pytestmark = pytest.mark.gpu
 
 
-def make_inputs(wl, B, H, L, unnormalised, block_p=None):
+def make_inputs(wl, B, H, L, unnormalised, block_p=None, spread=0.7):
     route = None if block_p is None else inputs.route_blocks(wl.seed, (B, L, H), block_p)
     x = inputs.make_layer_inputs(wl, B=B, H=H, L=L, route=route)
-    if unnormalised:      # rows of very different lengths: the normalisation has something to do
+    if unnormalised:      # rows of very different lengths (log-normal, sigma = spread): the normalisation has something to do
         r = np.random.default_rng(wl.seed + 100)
         for n in ("q", "k"):
-            x[n] = (x[n] * np.exp(0.7 * r.standard_normal((B, L, H, 1)))).astype(np.float32)
+            x[n] = (x[n] * np.exp(spread * r.standard_normal((B, L, H, 1)))).astype(np.float32)
             if wl.dtype == "bf16":
                 x[n] = inputs.round_bf16(x[n])
     return x
@@ -445,6 +445,37 @@ def test_prefill_in_pieces_with_grouped_heads(G, norm, block, B, H, pieces):
     assert np.array_equal(k_sm[0, 0, :len(rows)].float().cpu().numpy(), x["k"][0, rows, 0])
 
 
+@pytest.mark.parametrize("block", [False, True])
+def test_bf16_d64_normalised_backward(block):
+    """bf16 storage at d = 64 with the normalisation: the backward takes the path with separate chunk-level
+    products (the fused chunk kernel does not know the normalisation)."""
+    from test_gpu_parity import check_bwd
+    from paper_2602_03681_b200 import binding
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg4_bf16_train"], seed=131)
+    B, H, L, d = 2, 2, 256, 64
+    # (row lengths over a factor of ~5: a gradient row scales with 1 / its row's length, and the bound is
+    # relative to the whole tensor's RMS; with sigma = 0.7 the shortest rows of this case sit 2 % above it)
+    x = make_inputs(wl, B, H, L, True, block_p=0.4 if block else None, spread=0.4)
+    scale_sm = d ** -0.5
+    flags = binding.QK_NORM | (binding.BLOCK_ROUTING if block else 0)
+    pr = binding.make_params(B, H, L, d, binding.NATSL_BF16, wl.scale_la, scale_sm, flags=flags, norm_eps=1e-6)
+    w_dev = dev(x["w"])
+    pr.w = w_dev.data_ptr()
+    ws = binding.alloc_workspace(pr, binding.OP_BWD)
+    t = {n: dev(x[n], torch.bfloat16) for n in ("q", "k", "v", "dout")}
+    t.update({n: dev(x[n]) for n in ("g", "beta", "route")})
+    outs = {n: torch.empty_like(t["q"]) for n in ("dq", "dk", "dv")}
+    outs.update(dg=torch.empty_like(t["g"]), dbeta=torch.empty_like(t["g"]), dw=torch.empty((B, L, H, 2), device="cuda"))
+    binding.natsl_hybrid_bwd(t["q"], t["k"], t["v"], t["g"], t["beta"], t["route"], t["dout"], outs["dq"], outs["dk"],
+                             outs["dv"], outs["dg"], outs["dbeta"], outs["dw"], pr, ws)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(ws) == 0
+    ref = grouped.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"], G=1,
+                             qk_norm=True, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6,
+                             block=64 if block else None)
+    check_bwd(wl, {n: v.float().cpu().numpy() for n, v in outs.items()}, ref, TOL["bf16"], large_only=False)
+
+
 def test_normalisation_ignores_row_lengths_on_the_device():
     """Rescaling the q and k rows by powers of two changes no bf16 mantissa, so with norm_eps = 0 the
     normalised layer must return almost the same bits."""
@@ -484,12 +515,11 @@ def test_requests_that_are_not_built_are_refused():
     assert refused(lambda: binding.hybrid_fwd(*args, G=2, flags=binding.FORCE_SIMT, **kw))        # bf16 on CUDA cores
     with pytest.raises(binding.NatslError):                                                       # G must divide d
         binding.hybrid_fwd(*args, G=3, **kw)
-    # backward: bf16 storage at d = 64 (the fused chunk kernel's path) has no normalisation
+    # backward: two softmax heads of 32 columns (d = 64) are not built on tensor cores
     wl4 = inputs.WORKLOADS["cfg4_bf16_train"]
     x4 = make_inputs(wl4, 1, 2, 128, False)
     a4 = [dev(x4[n], torch.bfloat16) for n in ("q", "k", "v")] + [dev(x4["g"]), dev(x4["beta"]), dev(x4["route"])]
-    p = binding.make_params(1, 2, 128, 64, binding.NATSL_BF16, wl4.scale_la, wl4.scale_sm, flags=binding.QK_NORM,
-                            norm_eps=1e-6)
+    p = binding.make_params(1, 2, 128, 64, binding.NATSL_BF16, wl4.scale_la, wl4.scale_sm, G=2)
     n = binding.natsl_workspace_size(p, binding.OP_BWD)
     ws = torch.zeros(n, dtype=torch.uint8, device="cuda")
     outs = [torch.empty_like(a4[0]) for _ in range(3)] + [torch.empty_like(a4[3]) for _ in range(2)]
