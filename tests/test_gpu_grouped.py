@@ -125,6 +125,15 @@ def test_block_level_routing_with_grouped_heads(storage, d, G, norm, B, H, L, p)
     check(wl, got, ref, TOL[storage], G)
 
 
+def test_bf16_paper_mode_at_length():
+    """Six linear x twelve softmax heads, one decision per block, normalised q, k, L = 2048: 16 query tiles per
+    head with up to ~10 retained tiles and two own-block tiles each, several waves of CTAs."""
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg1_bf16_prefill"], seed=77)
+    x = make_inputs(wl, 1, 6, 2048, True, block_p=0.3)
+    got, ref = run_both(wl, x, 2, True, 64 ** -0.5, block=True)
+    check(wl, got, ref, TOL["bf16"], 2)
+
+
 def test_bf16_tensor_cores_d64_normalisation():
     """The normalisation alone at d = 64 (one softmax head per linear head, the 64-column kernels)."""
     wl = dataclasses.replace(inputs.WORKLOADS["cfg4_bf16_train"], seed=47)
