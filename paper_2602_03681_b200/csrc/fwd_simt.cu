@@ -439,58 +439,89 @@ qk_norm_f32_kernel(const T *__restrict__ q, const T *__restrict__ k, float *__re
 // (a token's k reaches only the operation the token was routed to).  x^ = x r, r = (sum x^2 + e)^-1/2:
 // dx = r (g - x^ <x^, g>);  x~ = x r, r = (mean x^2 + e)^-1/2 over a slice of ds columns:
 // dx = r (g - x~ <x~, g> / ds).
-template <typename T>
+// (One warp per row; a lane owns D / 32 neighbouring columns, moved as one vector.  A slice is an aligned
+// group of 32 / G lanes, so one xor butterfly yields a slice's sum on the way to the row's.)
+template <int N> __device__ __forceinline__ void load_vec(const float *p, float (&x)[N]) {
+    if (N == 4) { const float4 v = *reinterpret_cast<const float4 *>(p); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+    else { const float2 v = *reinterpret_cast<const float2 *>(p); x[0] = v.x; x[1] = v.y; }
+}
+template <int N> __device__ __forceinline__ void load_vec(const __nv_bfloat16 *p, float (&x)[N]) {
+    if (N == 4) {
+        const uint2 v = *reinterpret_cast<const uint2 *>(p);
+        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
+        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
+    } else {
+        const uint32_t v = *reinterpret_cast<const uint32_t *>(p);
+        x[0] = __uint_as_float(v << 16); x[1] = __uint_as_float(v & 0xffff0000u);
+    }
+}
+template <int N> __device__ __forceinline__ void store_vec(float *p, const float (&x)[N]) {
+    if (N == 4) *reinterpret_cast<float4 *>(p) = make_float4(x[0], x[1], x[2], x[3]);
+    else *reinterpret_cast<float2 *>(p) = make_float2(x[0], x[1]);
+}
+template <int N> __device__ __forceinline__ void store_vec(__nv_bfloat16 *p, const float (&x)[N]) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(x[0], x[1]);
+    if (N == 4) {
+        __nv_bfloat162 hi = __floats2bfloat162_rn(x[2], x[3]);
+        *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+    } else {
+        *reinterpret_cast<uint32_t *>(p) = *reinterpret_cast<uint32_t *>(&lo);
+    }
+}
+
+template <typename T, int D>
 __global__ void __launch_bounds__(256)
 qk_norm_bwd_f32_kernel(const T *__restrict__ q, const T *__restrict__ k,
                        const uint8_t *__restrict__ route, const float *dq_la,
                        const float *__restrict__ dq_sm, const float *dk_in, const float *dv_in,
-                       T *dq, T *dk, T *dv, size_t rows, int d, int G, float norm_eps,
+                       T *dq, T *dk, T *dv, size_t rows, int G, float norm_eps,
                        const float *__restrict__ dk_sm) {
+    constexpr int N = D / 32;
     const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= rows) return;
-    const int ds = d / G, nj = d / 32;
+    const int lps = 32 / G;                                  // lanes per slice
+    const float inv_ds = (float)G / D;
     const bool retained = route[row] != 0;
-    if (dv_in)
-        for (int j = 0; j < nj; ++j) dv[row * d + lane + 32 * j] = from_f32<T>(dv_in[row * d + lane + 32 * j]);
+    const size_t at = row * D + (size_t)lane * N;
+    if (dv_in) {
+        float t[N];
+        load_vec<N>(dv_in + at, t);
+        store_vec<N>(dv + at, t);
+    }
+#pragma unroll
     for (int which = 0; which < 2; ++which) {
-        const T *src = (which ? k : q) + row * d;
-        const float *gin = (which ? dk_in : dq_la) + row * d;
-        T *gout = (which ? dk : dq) + row * d;
-        float x[4], g[4], ssg[4], xgg[4], out[4], ss_all = 0.f, xg_all = 0.f;
-        for (int j = 0; j < nj; ++j) {
-            x[j] = to_f32(src[lane + 32 * j]);
-            g[j] = gin[lane + 32 * j];
-            out[j] = 0.f;
-        }
         const float *sm_in = which == 0 ? dq_sm : dk_sm;   // separate softmax-operation gradient, if any
         const bool l2_part = sm_in || !retained, rms_part = sm_in || retained;
-        if (l2_part) {
-            for (int j = 0; j < nj; ++j) {
-                ss_all = fmaf(x[j], x[j], ss_all);
-                xg_all = fmaf(x[j], g[j], xg_all);
-            }
-            ss_all = warp_sum(ss_all);
-            xg_all = warp_sum(xg_all);
-            const float r = rsqrtf(ss_all + norm_eps), dot = r * xg_all;
-            for (int j = 0; j < nj; ++j) out[j] = r * (g[j] - x[j] * r * dot);
+        float x[N], g[N], gs[N], out[N];
+        load_vec<N>((which ? k : q) + at, x);
+        load_vec<N>((which ? dk_in : dq_la) + at, g);
+        if (sm_in) load_vec<N>(sm_in + at, gs);
+        float ss = 0.f, xg = 0.f, xs = 0.f;
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            if (!sm_in) gs[j] = g[j];
+            ss = fmaf(x[j], x[j], ss);
+            xg = fmaf(x[j], g[j], xg);
+            xs = fmaf(x[j], gs[j], xs);
         }
-        if (rms_part) {
-            float gs[4];
-            for (int j = 0; j < nj; ++j) {
-                gs[j] = sm_in ? sm_in[row * d + lane + 32 * j] : g[j];
-                ssg[j] = warp_sum(x[j] * x[j]);
-                xgg[j] = warp_sum(x[j] * gs[j]);
-            }
-            for (int j = 0; j < nj; ++j) {
-                float ss = 0.f, xg = 0.f;
-                for (int y = 0; y < nj; ++y)
-                    if ((32 * y) / ds == (32 * j) / ds) { ss += ssg[y]; xg += xgg[y]; }
-                const float r = rsqrtf(ss / ds + norm_eps), m = r * xg / ds;
-                out[j] += r * (gs[j] - x[j] * r * m);
-            }
+        float ss_s = 0.f, xs_s = 0.f;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            if (o == lps) { ss_s = ss; xs_s = xs; }
+            ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            xg += __shfl_xor_sync(0xffffffffu, xg, o);
+            xs += __shfl_xor_sync(0xffffffffu, xs, o);
         }
-        for (int j = 0; j < nj; ++j) gout[lane + 32 * j] = from_f32<T>(out[j]);
+        if (lps == 32) { ss_s = ss; xs_s = xs; }
+        const float rl = rsqrtf(ss + norm_eps), dot = rl * xg;
+        const float rs = rsqrtf(fmaf(ss_s, inv_ds, norm_eps)), m = rs * xs_s * inv_ds;
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            out[j] = l2_part ? rl * (g[j] - x[j] * rl * dot) : 0.f;
+            if (rms_part) out[j] += rs * (gs[j] - x[j] * rs * m);
+        }
+        store_vec<N>((which ? dk : dq) + at, out);
     }
 }
 
@@ -621,14 +652,14 @@ cudaError_t launch_qk_norm_bwd_f32(const void *q, const void *k, bool bf16, cons
                                    const float *dv_in, void *dq, void *dk, void *dv, size_t rows, int d, int G,
                                    float norm_eps, cudaStream_t st, const float *dk_sm) {
     const unsigned blocks = (unsigned)((rows + 7) / 8);
-    if (bf16)
-        qk_norm_bwd_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
-            (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, route, dq_la, dq_sm, dk_in, dv_in,
-            (__nv_bfloat16 *)dq, (__nv_bfloat16 *)dk, (__nv_bfloat16 *)dv, rows, d, G, norm_eps, dk_sm);
-    else
-        qk_norm_bwd_f32_kernel<float><<<blocks, 256, 0, st>>>((const float *)q, (const float *)k, route, dq_la,
-                                                             dq_sm, dk_in, dv_in, (float *)dq, (float *)dk,
-                                                             (float *)dv, rows, d, G, norm_eps, dk_sm);
+    if ((d != 64 && d != 128) || G < 1 || 32 % G != 0) return cudaErrorInvalidValue;
+#define NATSL_NB(TT, DD)                                                                                      \
+    qk_norm_bwd_f32_kernel<TT, DD><<<blocks, 256, 0, st>>>((const TT *)q, (const TT *)k, route, dq_la, dq_sm,  \
+                                                          dk_in, dv_in, (TT *)dq, (TT *)dk, (TT *)dv, rows, G, \
+                                                          norm_eps, dk_sm)
+    if (bf16) { if (d == 128) NATSL_NB(__nv_bfloat16, 128); else NATSL_NB(__nv_bfloat16, 64); }
+    else { if (d == 128) NATSL_NB(float, 128); else NATSL_NB(float, 64); }
+#undef NATSL_NB
     count_launch();
     return cudaGetLastError();
 }
