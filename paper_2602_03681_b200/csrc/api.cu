@@ -92,6 +92,9 @@ int scan_segments(const natsl_params *p) {
     const int NC = p->L / kC, BH = p->B * p->H;
     int nseg = 1;
     while (2 * BH * (nseg * 2) <= 128 && NC % (nseg * 2) == 0 && NC / (nseg * 2) >= 8) nseg *= 2;
+    // Once the scan is segmented (and so already pays its second run), one more doubling up to one CTA per
+    // SM: the two runs shrink by half again, which outweighs what the softmax kernel loses beside them.
+    if (nseg >= 2 && BH * (nseg * 2) <= 128 && NC % (nseg * 2) == 0 && NC / (nseg * 2) >= 8) nseg *= 2;
     return nseg;
 }
 
