@@ -209,7 +209,7 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.o_la = tm(true);
     f.o_nla = tm(true);
     f.do_la = tm(true);
-    f.do_nla = tm(!tcs || (general && block));     // (fp32 own-block kernel of block-level routing)
+    f.do_nla = tm(!tcs);
     f.dUt = tcs ? f.o_la : tm(true);
     f.dQg = tm(general); f.dW = tm(general); f.dKt = tm(general); f.dKb = tm(general); f.dVb = tm(general);
     f.X1p = tm(general); f.X2 = tm(general);
@@ -678,7 +678,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     const int32_t *gsc = tensor_cores ? f.status : nullptr;
     const bool general_block = block && !fused_chunks;   // block-level routing with separate chunk-level products
     NATSL_TRY(launch_combine_bwd(f.o_la, f.o_nla, dout, p->w, p->eps, f.do_la,
-                                 tensor_cores && !general_block ? nullptr : f.do_nla, dw, f.Dsm,
+                                 tensor_cores ? nullptr : f.do_nla, dw, f.Dsm,
                                  tensor_cores ? f.dO16 : nullptr, tensor_cores ? f.dOla16 : nullptr,
                                  tensor_cores ? f.dOlag16 : nullptr, f.tc.Gd, p->scale_la, gsc, s, st, hg.G));
     // Dependencies from here on: the query-side softmax kernel, the key-side one and the reverse
@@ -758,9 +758,9 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         // dk_x -- a gradient with respect to that copy -- stays apart from the linear branch's dk until the
         // normalisations' backward.)
         NATSL_TRY(launch_gdn_finish(a, f.dk_x, f.dv_x, s32, st, false));
-        if (tensor_cores && p->d == 128 && hg.G == 2)      // softmax heads of 64 columns: warp-level tensor cores
+        if (tensor_cores)      // softmax heads of 64 or 128 columns: warp-level tensor cores
             NATSL_TRY(launch_softmax_bwd_own_block(q, k, v, f.dO16, f.lse, f.Dsm, route, p->scale_sm, f.dq_sm,
-                                                   f.dk_x, f.dv_x, gsc, s, st, 2, normed ? f.qs32 : nullptr,
+                                                   f.dk_x, f.dv_x, gsc, s, st, hg.G, normed ? f.qs32 : nullptr,
                                                    normed ? f.ks32 : nullptr));
         else
             NATSL_TRY(launch_softmax_bwd_own_block_simt(normed ? f.qs32 : f.q32, normed ? f.ks32 : f.k32, f.v32,

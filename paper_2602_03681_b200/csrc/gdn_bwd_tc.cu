@@ -720,14 +720,15 @@ __global__ void __launch_bounds__(kCkThreads, 2) gdn_bwd_chunk_kernel(ChunkBwdAr
 //   dq += dS K  (added to the query-side result of the compacted kernels)
 //   dk  = dS^T Q,  dv = P^T dO  (written: the tokens of a linear block have no other
 //                                 softmax-branch gradient)
-// with lse_i and D_i = <do_i, o_i> of the whole softmax row.  Softmax heads of 64 columns: d = 64, or
-// kG = 2 heads per linear head of d = 128 (Section 4.3; the head is then a column slice of rows of 128
-// columns, lse / Dsm are [B,H,kG,L]).  kNormSrc: q and k come from the fp32 copies that hold the softmax
-// operation's normalised rows (qn, kn) instead of the bf16 inputs.
-constexpr int kOwnSmem = 6 * kTileH * 2;
+// with lse_i and D_i = <do_i, o_i> of the whole softmax row.  Softmax heads of 64 KB columns: KB = 1 for
+// d = 64 or kG = 2 heads per linear head of d = 128 (Section 4.3; the head is then a column slice of rows
+// of 128 columns, lse / Dsm are [B,H,kG,L]), KB = 2 for d = 128 (two tiles per operand: the logit products
+// add over them, the three results are formed half by half).  kNormSrc: q and k come from the fp32 copies
+// that hold the softmax operation's normalised rows (qn, kn) instead of the bf16 inputs.
+template <int KB> constexpr int own_smem() { return (4 * KB + 2) * kTileH * 2; }
 
-template <int kG, bool kNormSrc>
-__global__ void __launch_bounds__(kCkThreads, 3)
+template <int kG, bool kNormSrc, int KB>
+__global__ void __launch_bounds__(kCkThreads, KB == 1 ? 3 : 2)
 softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfloat16 *__restrict__ k,
                              const __nv_bfloat16 *__restrict__ v, const float *__restrict__ qn,
                              const float *__restrict__ kn, const __half *__restrict__ do16,
@@ -735,11 +736,12 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
                              const uint8_t *__restrict__ route, float scale_sm,
                              float *__restrict__ dq_sm, float *__restrict__ dk_x,
                              float *__restrict__ dv_x, const int32_t *gsc_status, int L, int H) {
-    constexpr int D = 64, DL = D * kG;
+    static_assert(KB == 1 || kG == 1, "grouped heads have 64 columns");
+    constexpr int D = 64 * KB, DL = D * kG;
     const float ginv = grad_scale(gsc_status).y;   // do16 and Dsm arrive times the gradient scale
     extern __shared__ __align__(16) uint8_t smraw[];
-    __half *sQ = reinterpret_cast<__half *>(smraw), *sK = sQ + kTileH, *sV = sK + kTileH, *sDO = sV + kTileH,
-           *sP = sDO + kTileH, *sDS = sP + kTileH;
+    __half *sQ = reinterpret_cast<__half *>(smraw), *sK = sQ + KB * kTileH, *sV = sK + KB * kTileH,
+           *sDO = sV + KB * kTileH, *sP = sDO + KB * kTileH, *sDS = sP + kTileH;      // KB tiles per operand
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int c = blockIdx.x, bhg = blockIdx.y, bh = bhg / kG, col0 = (bhg % kG) * D, b = bh / H, h = bh % H;
     const size_t ts = (size_t)H * DL;
@@ -751,22 +753,24 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
             return pack_half2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
         };
 #pragma unroll
+        for (int kb = 0; kb < KB; ++kb)
+#pragma unroll
         for (int it = 0; it < 4; ++it) {
-            const int r = r0 + 16 * it;
-            const size_t off = tok0 + (size_t)r * ts + c4;
+            const int r = r0 + 16 * it, tl = kb * kTileH + r * kLdH + c4;
+            const size_t off = tok0 + (size_t)r * ts + kb * 64 + c4;
             const uint2 xv = *reinterpret_cast<const uint2 *>(v + off);
-            const uint2 xo = *reinterpret_cast<const uint2 *>(do16 + ((size_t)bh * L + (size_t)c * kC + r) * DL + col0 + c4);
+            const uint2 xo = *reinterpret_cast<const uint2 *>(do16 + ((size_t)bh * L + (size_t)c * kC + r) * DL + col0 + kb * 64 + c4);
             if (kNormSrc) {
                 const float4 fq = *reinterpret_cast<const float4 *>(qn + off), fk = *reinterpret_cast<const float4 *>(kn + off);
-                *reinterpret_cast<uint2 *>(sQ + r * kLdH + c4) = make_uint2(pack_half2(fq.x, fq.y), pack_half2(fq.z, fq.w));
-                *reinterpret_cast<uint2 *>(sK + r * kLdH + c4) = make_uint2(pack_half2(fk.x, fk.y), pack_half2(fk.z, fk.w));
+                *reinterpret_cast<uint2 *>(sQ + tl) = make_uint2(pack_half2(fq.x, fq.y), pack_half2(fq.z, fq.w));
+                *reinterpret_cast<uint2 *>(sK + tl) = make_uint2(pack_half2(fk.x, fk.y), pack_half2(fk.z, fk.w));
             } else {
                 const uint2 xq = *reinterpret_cast<const uint2 *>(q + off), xk = *reinterpret_cast<const uint2 *>(k + off);
-                *reinterpret_cast<uint2 *>(sQ + r * kLdH + c4) = make_uint2(cv(xq.x), cv(xq.y));
-                *reinterpret_cast<uint2 *>(sK + r * kLdH + c4) = make_uint2(cv(xk.x), cv(xk.y));
+                *reinterpret_cast<uint2 *>(sQ + tl) = make_uint2(cv(xq.x), cv(xq.y));
+                *reinterpret_cast<uint2 *>(sK + tl) = make_uint2(cv(xk.x), cv(xk.y));
             }
-            *reinterpret_cast<uint2 *>(sV + r * kLdH + c4) = make_uint2(cv(xv.x), cv(xv.y));
-            *reinterpret_cast<uint2 *>(sDO + r * kLdH + c4) = xo;
+            *reinterpret_cast<uint2 *>(sV + tl) = make_uint2(cv(xv.x), cv(xv.y));
+            *reinterpret_cast<uint2 *>(sDO + tl) = xo;
         }
     }
     __syncthreads();
@@ -791,7 +795,8 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
     };
     // p = exp(scale s - lse), causal inside the block (mask on the exponent: no branch per element)
     zero(pr);
-    mma64<false, true>(sQ, sK, row0, n0, lane, pr);
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb) mma64<false, true>(sQ + kb * kTileH, sK + kb * kTileH, row0, n0, lane, pr);
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
@@ -802,18 +807,19 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
     put(sP, pr);
     // ds = scale p (dp - D)
     zero(acc);
-    mma64<false, true>(sDO, sV, row0, n0, lane, acc);
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb) mma64<false, true>(sDO + kb * kTileH, sV + kb * kTileH, row0, n0, lane, acc);
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[nt][e] = scale_sm * pr[nt][e] * (acc[nt][e] - (e < 2 ? DA : DB));
     put(sDS, acc);
     __syncthreads();
-    auto out2 = [&](float *dst, const float (&a)[4][4], bool add) {
+    auto out2 = [&](float *dst, const float (&a)[4][4], bool add, int kb) {
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
-            float2 *pa = reinterpret_cast<float2 *>(dst + tok0 + (size_t)iA * ts + n0 + 8 * nt + 2 * t);
-            float2 *pb = reinterpret_cast<float2 *>(dst + tok0 + (size_t)iB * ts + n0 + 8 * nt + 2 * t);
+            float2 *pa = reinterpret_cast<float2 *>(dst + tok0 + (size_t)iA * ts + kb * 64 + n0 + 8 * nt + 2 * t);
+            float2 *pb = reinterpret_cast<float2 *>(dst + tok0 + (size_t)iB * ts + kb * 64 + n0 + 8 * nt + 2 * t);
             float2 va = make_float2(ginv * a[nt][0], ginv * a[nt][1]), vb = make_float2(ginv * a[nt][2], ginv * a[nt][3]);
             if (add) {
                 const float2 ca = *pa, cb = *pb;
@@ -823,15 +829,18 @@ softmax_bwd_own_block_kernel(const __nv_bfloat16 *__restrict__ q, const __nv_bfl
             *pb = vb;
         }
     };
-    zero(acc);
-    mma64<false, false>(sDS, sK, row0, n0, lane, acc);          // dq += dS K
-    out2(dq_sm, acc, true);
-    zero(acc);
-    mma64<true, false>(sDS, sQ, row0, n0, lane, acc);           // dk = dS^T Q
-    out2(dk_x, acc, false);
-    zero(acc);
-    mma64<true, false>(sP, sDO, row0, n0, lane, acc);           // dv = P^T dO
-    out2(dv_x, acc, false);
+#pragma unroll
+    for (int kb = 0; kb < KB; ++kb) {
+        zero(acc);
+        mma64<false, false>(sDS, sK + kb * kTileH, row0, n0, lane, acc);          // dq += dS K
+        out2(dq_sm, acc, true, kb);
+        zero(acc);
+        mma64<true, false>(sDS, sQ + kb * kTileH, row0, n0, lane, acc);           // dk = dS^T Q
+        out2(dk_x, acc, false, kb);
+        zero(acc);
+        mma64<true, false>(sP, sDO + kb * kTileH, row0, n0, lane, acc);           // dv = P^T dO
+        out2(dv_x, acc, false, kb);
+    }
 }
 
 }  // namespace
@@ -943,14 +952,19 @@ cudaError_t launch_softmax_bwd_own_block(const void *q, const void *k, const voi
                                          const uint8_t *route, float scale_sm, float *dq_sm,
                                          float *dk_x, float *dv_x, const int32_t *gsc, Shape s,
                                          cudaStream_t st, int G, const float *qn, const float *kn) {
-    if (!s.bf16 || !((s.d == 64 && G <= 1) || (s.d == 128 && G == 2))) return cudaErrorInvalidValue;
-    auto kernel = softmax_bwd_own_block_kernel<1, false>;
-    if (G <= 1 && qn) kernel = softmax_bwd_own_block_kernel<1, true>;
-    if (G == 2) kernel = qn ? softmax_bwd_own_block_kernel<2, true> : softmax_bwd_own_block_kernel<2, false>;
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kOwnSmem);
+    if (!s.bf16 || !((s.d == 64 && G <= 1) || (s.d == 128 && G <= 2))) return cudaErrorInvalidValue;
+    auto kernel = softmax_bwd_own_block_kernel<1, false, 1>;
+    int smem = own_smem<1>();
+    if (s.d == 64 && qn) kernel = softmax_bwd_own_block_kernel<1, true, 1>;
+    if (s.d == 128 && G == 2) kernel = qn ? softmax_bwd_own_block_kernel<2, true, 1> : softmax_bwd_own_block_kernel<2, false, 1>;
+    if (s.d == 128 && G <= 1) {
+        kernel = qn ? softmax_bwd_own_block_kernel<1, true, 2> : softmax_bwd_own_block_kernel<1, false, 2>;
+        smem = own_smem<2>();
+    }
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(s.L / kC, s.B * s.H * (G == 2 ? 2 : 1));
-    kernel<<<grid, kCkThreads, kOwnSmem, st>>>(
+    kernel<<<grid, kCkThreads, smem, st>>>(
         (const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k, (const __nv_bfloat16 *)v, qn, kn, (const __half *)do16,
         lse, Dsm, route, scale_sm, dq_sm, dk_x, dv_x, gsc, s.L, s.H);
     count_launch();
