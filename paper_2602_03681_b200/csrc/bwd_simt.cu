@@ -301,6 +301,85 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
     }
 }
 
+// The ungrouped case again with four neighbouring columns per lane (one vector per array and lane; D / 4
+// lanes per row, so a warp takes two rows at D = 64): the kernel sits at the head of the backward's
+// dependency chain and is bound by how many bytes a warp has in flight.
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads)
+combine_bwd_vec_kernel(const float *__restrict__ o_la, const float *__restrict__ o_nla,
+                       const T *__restrict__ dout, const float *__restrict__ w, float eps,
+                       float *__restrict__ do_la, float *__restrict__ do_nla, float *__restrict__ dw,
+                       float *__restrict__ Dsm, __half *__restrict__ do16,
+                       __half *__restrict__ dola16, __half *__restrict__ dolag16,
+                       const float *__restrict__ Gd, float scale_la, const int32_t *gsc, int B, int L, int H) {
+    constexpr int kLpr = D / 4, kRpw = 32 / kLpr;           // lanes per row, rows per warp
+    const float gs = grad_scale(gsc).x;
+    const int lane = threadIdx.x & 31, sub = lane / kLpr, li = lane % kLpr;
+    const size_t row = ((size_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5)) * kRpw + sub;
+    const bool live = row < (size_t)B * L * H;              // (all lanes stay for the shuffles)
+    const size_t rr = live ? row : 0;
+    const int h = rr % H;
+    const size_t bl = rr / H;
+    const int l = bl % L, b = bl / L;
+    const size_t at = rr * D + li * 4;
+    const float4 a = *reinterpret_cast<const float4 *>(o_la + at), n = *reinterpret_cast<const float4 *>(o_nla + at);
+    float dy[4];
+    if (sizeof(T) == 2) {
+        const uint2 u = *reinterpret_cast<const uint2 *>(dout + at);
+        dy[0] = __uint_as_float(u.x << 16); dy[1] = __uint_as_float(u.x & 0xffff0000u);
+        dy[2] = __uint_as_float(u.y << 16); dy[3] = __uint_as_float(u.y & 0xffff0000u);
+    } else {
+        const float4 u = *reinterpret_cast<const float4 *>(dout + at);
+        dy[0] = u.x; dy[1] = u.y; dy[2] = u.z; dy[3] = u.w;
+    }
+    const float ol[4] = {a.x, a.y, a.z, a.w}, on[4] = {n.x, n.y, n.z, n.w};
+    auto row_sum = [&](float v) {
+#pragma unroll
+        for (int o = kLpr / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        return v;
+    };
+    float ssl = 0.f, ssn = 0.f;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) { ssl = fmaf(ol[x], ol[x], ssl); ssn = fmaf(on[x], on[x], ssn); }
+    ssl = row_sum(ssl);
+    ssn = row_sum(ssn);
+    const float fl = rsqrtf(ssl / D + eps), fn = rsqrtf(ssn / D + eps);
+    const float wn = w ? w[rr * 2] : 0.5f, wl = w ? w[rr * 2 + 1] : 0.5f;
+    const float sg = dolag16 ? scale_la * Gd[((size_t)(b * H + h) * (L / kC) + l / kC) * 128 + l % kC] : 0.f;
+    float dwl = 0.f, dwn = 0.f;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) { dwl = fmaf(dy[x], ol[x] * fl, dwl); dwn = fmaf(dy[x], on[x] * fn, dwn); }
+    dwl = row_sum(dwl);
+    dwn = row_sum(dwn);
+    const float ml = wl * dwl / D, mn = wn * dwn / D;
+    float dl[4], dn[4], dsm = 0.f;
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        dl[x] = fl * (wl * dy[x] - ol[x] * fl * ml);
+        dn[x] = fn * (wn * dy[x] - on[x] * fn * mn);
+        dsm = fmaf(dn[x], on[x], dsm);
+    }
+    dsm = row_sum(dsm);
+    if (!live) return;
+    *reinterpret_cast<float4 *>(do_la + at) = make_float4(dl[0], dl[1], dl[2], dl[3]);
+    if (do_nla) *reinterpret_cast<float4 *>(do_nla + at) = make_float4(dn[0], dn[1], dn[2], dn[3]);
+    const size_t at16 = (((size_t)b * H + h) * L + l) * D + li * 4;
+    auto h4 = [](float x0, float x1, float x2, float x3) {
+        const __half2 p = __floats2half2_rn(x0, x1), q2 = __floats2half2_rn(x2, x3);
+        return make_uint2(*reinterpret_cast<const uint32_t *>(&p), *reinterpret_cast<const uint32_t *>(&q2));
+    };
+    if (do16) *reinterpret_cast<uint2 *>(do16 + at16) = h4(gs * dn[0], gs * dn[1], gs * dn[2], gs * dn[3]);
+    if (dolag16) {
+        *reinterpret_cast<uint2 *>(dola16 + at16) = h4(gs * dl[0], gs * dl[1], gs * dl[2], gs * dl[3]);
+        const float gg = gs * sg;
+        *reinterpret_cast<uint2 *>(dolag16 + at16) = h4(gg * dl[0], gg * dl[1], gg * dl[2], gg * dl[3]);
+    }
+    if (li == 0) {
+        if (dw) { dw[rr * 2] = dwn; dw[rr * 2 + 1] = dwl; }
+        Dsm[((size_t)b * H + h) * L + l] = gs * dsm;
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // softmax backward, query side: dq_sm.  grid = (L/64, B*H), same tiling as the forward.
 // ------------------------------------------------------------------------------------------
@@ -934,7 +1013,15 @@ static cudaError_t combine_bwd_impl(const float *o_la, const float *o_nla, const
                                     const float *Gd, float scale_la, const int32_t *gsc, Shape s,
                                     cudaStream_t st, int G) {
     const size_t rows = (size_t)s.B * s.L * s.H;
-    auto kernel = G > 1 ? combine_bwd_kernel<T, D, true> : combine_bwd_kernel<T, D, false>;
+    if (G <= 1) {
+        constexpr int kRowsPerBlock = (kThreads / 32) * (32 / (D / 4));
+        combine_bwd_vec_kernel<T, D><<<(unsigned)((rows + kRowsPerBlock - 1) / kRowsPerBlock), kThreads, 0, st>>>(
+            o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, (__half *)do16, (__half *)dola16,
+            (__half *)dolag16, Gd, scale_la, gsc, s.B, s.L, s.H);
+        count_launch();
+        return cudaGetLastError();
+    }
+    auto kernel = combine_bwd_kernel<T, D, true>;
     kernel<<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
         o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, (__half *)do16, (__half *)dola16,
         (__half *)dolag16, Gd, scale_la, gsc, G, s.B, s.L, s.H);
