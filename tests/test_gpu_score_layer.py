@@ -35,7 +35,11 @@ def run_score_layer(x, w, H, bf16, want_scores=True):
 
 @pytest.mark.parametrize("B,L,Dm,H,bf16", [(2, 256, 512, 4, True), (1, 64, 8, 1, True),
                                            (3, 640, 2048, 16, True), (2, 192, 1032, 3, True),
-                                           (2, 128, 260, 5, False), (1, 4096, 1024, 12, False)])
+                                           (2, 128, 260, 5, False), (1, 4096, 1024, 12, False),
+                                           # several column pieces per thread, the last one ragged; rows too
+                                           # wide for the deep ring of staged rows, and for any ring
+                                           (1, 192, 1544, 3, False), (1, 128, 4616, 2, True),
+                                           (1, 192, 16896, 2, True)])
 def test_score_layer_matches_oracle(B, L, Dm, H, bf16):
     x, w = features(B * L + Dm, B, L, Dm, H, bf16)
     ref = router.score_layer(x, w, 64)
