@@ -342,13 +342,16 @@ static int bwd_forward_part(const void *q, const void *k, const void *v, const f
     }
     NATSL_TRY(launch_route_compact(route, f.sm_idx, f.prefix, f.lin_idx, f.n_lin, f.sm_len, nullptr,
                                    block ? f.status : nullptr, p->L, p->B, p->L, p->H, st0));
-    if (!fused_chunks)
-        NATSL_TRY(launch_to_f32(q, k, v, f.q32, f.k32, f.v32, (size_t)(B * L * H * d), s.bf16, st));
+    const HeadGroups hg = head_groups(p);
+    if (!fused_chunks) {     // (with NATSL_QK_NORM the copies of q, k are the normalised ones, made below)
+        const bool qk = hg.norm_eps < 0.f;
+        NATSL_TRY(launch_to_f32(qk ? q : nullptr, qk ? k : nullptr, v, f.q32, f.k32, f.v32,
+                                (size_t)(B * L * H * d), s.bf16, st));
+    }
     // fp32 storage with NATSL_QK_NORM: q32, k32 become the L2-normalised rows (everything of the linear
     // branch reads those), qs32, ks32 the slice-wise RMS-normalised ones (softmax branch)
     // (tensor cores: the kernels normalise inside; only the fp32 copies the separate chunk-level products
     // of the backward read are made here)
-    const HeadGroups hg = head_groups(p);
     const float *qs = f.q32, *ks = f.k32;
     if (hg.norm_eps >= 0.f) {
         const bool rms_copies = !tensor_cores || block;

@@ -161,15 +161,14 @@ __global__ void to_f32_kernel(const T *__restrict__ a, const T *__restrict__ b, 
                               float *__restrict__ c32, size_t n4) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4;
          i += (size_t)gridDim.x * blockDim.x) {
-        store4(a32 + 4 * i, load4(a + 4 * i));
-        store4(b32 + 4 * i, load4(b + 4 * i));
+        if (a) store4(a32 + 4 * i, load4(a + 4 * i));      // (a, b: optional)
+        if (b) store4(b32 + 4 * i, load4(b + 4 * i));
         store4(c32 + 4 * i, load4(c + 4 * i));
     }
 }
 
 // ------------------------------------------------------------------------------------------
 // combination backward (row-local): do_la, do_nla, dw, Dsm = <do_nla, o_nla>
-// one warp per (token, head) row
 // ------------------------------------------------------------------------------------------
 // max |dout| over the whole tensor, as the bit pattern of a non-negative float (ordered like an
 // integer), into the status page; the word is zeroed by the caller beforehand.
@@ -195,10 +194,14 @@ dout_amax_kernel(const T *__restrict__ dout, size_t n4, int32_t *status) {
     if ((threadIdx.x & 31) == 0 && m > 0.f) atomicMax(status + kGradAmaxWord, __float_as_int(m));
 }
 
+// Four neighbouring columns per lane (one vector per array and lane), D / 4 lanes per row, so a warp takes
+// two rows at D = 64: the kernel sits at the head of the backward's dependency chain and is bound by how
+// many bytes a warp has in flight.
 // G > 1 (grouped softmax heads, Section 4.3): the softmax branch's output is normalised per slice of
 // D / G columns, so its part of the backward (do_nla, dw_nla, D_i = <do_i, o_i>) is formed per slice;
-// Dsm is then [B,H,G,L].
-template <typename T, int D, bool kGrouped>     // kGrouped: G > 1 (one reduction per 32-column group instead of per row)
+// Dsm is then [B,H,G,L].  A slice is an aligned group of D / (4 G) lanes: one xor butterfly gives the
+// slice's sum on its way to the row's.
+template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_nla,
                    const T *__restrict__ dout, const float *__restrict__ w, float eps,
@@ -206,115 +209,11 @@ combine_bwd_kernel(const float *__restrict__ o_la, const float *__restrict__ o_n
                    float *__restrict__ Dsm, __half *__restrict__ do16,
                    __half *__restrict__ dola16, __half *__restrict__ dolag16,
                    const float *__restrict__ Gd, float scale_la, const int32_t *gsc, int G, int B, int L, int H) {
-    constexpr int kCols = D / 32;
-    const float gs = grad_scale(gsc).x;      // scale of the fp16 operand copies (and of Dsm with them)
-    const int lane = threadIdx.x & 31;
-    const size_t row = (size_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
-    if (row >= (size_t)B * L * H) return;
-    const int h = row % H;
-    const size_t bl = row / H;
-    const int l = bl % L, b = bl / L;
-    const int ds = kGrouped ? D / G : D;     // columns per softmax head: 32, 64 or 128
-    const int gsh = 26 - __clz(ds);          // 32-column group x belongs to slice x >> gsh
-    // sum over the lanes and over the 32-column groups of x's slice (ungrouped: over the whole row, one reduction)
-    auto slice_sums = [&](const float (&v)[kCols], float (&out)[kCols]) {
-        if (!kGrouped) {
-            float t = 0.f;
-#pragma unroll
-            for (int x = 0; x < kCols; ++x) t += v[x];
-            t = warp_sum(t);
-#pragma unroll
-            for (int x = 0; x < kCols; ++x) out[x] = t;
-        } else {
-            float part[kCols];
-#pragma unroll
-            for (int x = 0; x < kCols; ++x) part[x] = warp_sum(v[x]);
-#pragma unroll
-            for (int x = 0; x < kCols; ++x) {
-                float t = 0.f;
-#pragma unroll
-                for (int y = 0; y < kCols; ++y) t += (y >> gsh) == (x >> gsh) ? part[y] : 0.f;
-                out[x] = t;
-            }
-        }
-    };
-    float ol[kCols], on[kCols], dy[kCols], ssl = 0.f, sq[kCols], ssn[kCols];
-#pragma unroll
-    for (int x = 0; x < kCols; ++x) {
-        const size_t i = row * D + lane + 32 * x;
-        ol[x] = o_la[i]; on[x] = o_nla[i]; dy[x] = to_f32(dout[i]);
-        ssl = fmaf(ol[x], ol[x], ssl);
-        sq[x] = on[x] * on[x];
-    }
-    ssl = warp_sum(ssl);
-    slice_sums(sq, ssn);
-    const float fl = rsqrtf(ssl / D + eps);
-    float fn[kCols];                          // RMS factor of the slice a 32-column group belongs to
-#pragma unroll
-    for (int x = 0; x < kCols; ++x) fn[x] = rsqrtf(ssn[x] * (1.f / ds) + eps);
-    const float wn = w ? w[row * 2] : 0.5f, wl = w ? w[row * 2 + 1] : 0.5f;
-    // scale_la gamma_l of the token (decay from its chunk's entry), for the reverse scan's operand
-    const float sg = dolag16 ? scale_la * Gd[((size_t)(b * H + h) * (L / kC) + l / kC) * 128 + l % kC] : 0.f;
-    float dwl = 0.f, dyn[kCols], dwn_s[kCols];
-#pragma unroll
-    for (int x = 0; x < kCols; ++x) {
-        dwl = fmaf(dy[x], ol[x] * fl, dwl);
-        dyn[x] = dy[x] * on[x] * fn[x];
-    }
-    dwl = warp_sum(dwl);
-    slice_sums(dyn, dwn_s);                   // <dy, y_nla> over the group's slice
-    float dwn = 0.f;
-#pragma unroll
-    for (int x = 0; x < kCols; ++x)           // ... and over the row: each slice counted once
-        if (!kGrouped ? x == 0 : (x & ((1 << gsh) - 1)) == 0) dwn += dwn_s[x];
-    const float ml = wl * dwl / D;
-    float dno[kCols], dsm_s[kCols];
-#pragma unroll
-    for (int x = 0; x < kCols; ++x) {
-        const size_t i = row * D + lane + 32 * x;
-        const float mn = wn * dwn_s[x] * (1.f / ds);
-        const float dl = fl * (wl * dy[x] - ol[x] * fl * ml);
-        const float dn = fn[x] * (wn * dy[x] - on[x] * fn[x] * mn);
-        do_la[i] = dl;
-        if (do_nla) do_nla[i] = dn;   // (the tensor-core softmax backward reads the fp16 copy only)
-        const size_t i16 = ((((size_t)b * H + h) * L + l) * D) + lane + 32 * x;
-        if (do16) do16[i16] = __float2half_rn(gs * dn);
-        if (dolag16) {
-            dola16[i16] = __float2half_rn(gs * dl);
-            dolag16[i16] = __float2half_rn(gs * sg * dl);
-        }
-        dno[x] = dn * on[x];
-    }
-    slice_sums(dno, dsm_s);
-    if (lane == 0) {
-        if (dw) { dw[row * 2] = dwn; dw[row * 2 + 1] = dwl; }
-        if (!kGrouped) {
-            Dsm[((size_t)b * H + h) * L + l] = gs * dsm_s[0];
-        } else {
-            for (int g = 0; g < G; ++g) {
-                float t = 0.f;
-#pragma unroll
-                for (int x = 0; x < kCols; ++x) t = (x >> gsh) == g ? dsm_s[x] : t;
-                Dsm[(((size_t)b * H + h) * G + g) * L + l] = gs * t;
-            }
-        }
-    }
-}
-
-// The ungrouped case again with four neighbouring columns per lane (one vector per array and lane; D / 4
-// lanes per row, so a warp takes two rows at D = 64): the kernel sits at the head of the backward's
-// dependency chain and is bound by how many bytes a warp has in flight.
-template <typename T, int D>
-__global__ void __launch_bounds__(kThreads)
-combine_bwd_vec_kernel(const float *__restrict__ o_la, const float *__restrict__ o_nla,
-                       const T *__restrict__ dout, const float *__restrict__ w, float eps,
-                       float *__restrict__ do_la, float *__restrict__ do_nla, float *__restrict__ dw,
-                       float *__restrict__ Dsm, __half *__restrict__ do16,
-                       __half *__restrict__ dola16, __half *__restrict__ dolag16,
-                       const float *__restrict__ Gd, float scale_la, const int32_t *gsc, int B, int L, int H) {
     constexpr int kLpr = D / 4, kRpw = 32 / kLpr;           // lanes per row, rows per warp
-    const float gs = grad_scale(gsc).x;
+    const float gs = grad_scale(gsc).x;      // scale of the fp16 operand copies (and of Dsm with them)
     const int lane = threadIdx.x & 31, sub = lane / kLpr, li = lane % kLpr;
+    const int lps = kLpr / G;                               // lanes per slice
+    const float inv_ds = (float)G / D;
     const size_t row = ((size_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5)) * kRpw + sub;
     const bool live = row < (size_t)B * L * H;              // (all lanes stay for the shuffles)
     const size_t rr = live ? row : 0;
@@ -333,35 +232,42 @@ combine_bwd_vec_kernel(const float *__restrict__ o_la, const float *__restrict__
         dy[0] = u.x; dy[1] = u.y; dy[2] = u.z; dy[3] = u.w;
     }
     const float ol[4] = {a.x, a.y, a.z, a.w}, on[4] = {n.x, n.y, n.z, n.w};
-    auto row_sum = [&](float v) {
+    // returns the row's sum; slice = the sum over the lane's slice
+    auto sums = [&](float v, float &slice) {
 #pragma unroll
-        for (int o = kLpr / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        for (int o = 1; o < kLpr; o <<= 1) {
+            if (o == lps) slice = v;
+            v += __shfl_xor_sync(0xffffffffu, v, o);
+        }
+        if (lps == kLpr) slice = v;
         return v;
     };
-    float ssl = 0.f, ssn = 0.f;
+    float ssl = 0.f, ssn = 0.f, ssn_s, unused;
 #pragma unroll
     for (int x = 0; x < 4; ++x) { ssl = fmaf(ol[x], ol[x], ssl); ssn = fmaf(on[x], on[x], ssn); }
-    ssl = row_sum(ssl);
-    ssn = row_sum(ssn);
-    const float fl = rsqrtf(ssl / D + eps), fn = rsqrtf(ssn / D + eps);
+    ssl = sums(ssl, unused);
+    sums(ssn, ssn_s);
+    const float fl = rsqrtf(ssl / D + eps), fn = rsqrtf(ssn_s * inv_ds + eps);   // fn: of the lane's slice
     const float wn = w ? w[rr * 2] : 0.5f, wl = w ? w[rr * 2 + 1] : 0.5f;
+    // scale_la gamma_l of the token (decay from its chunk's entry), for the reverse scan's operand
     const float sg = dolag16 ? scale_la * Gd[((size_t)(b * H + h) * (L / kC) + l / kC) * 128 + l % kC] : 0.f;
-    float dwl = 0.f, dwn = 0.f;
+    float dwl = 0.f, dwn = 0.f, dwn_s;
 #pragma unroll
     for (int x = 0; x < 4; ++x) { dwl = fmaf(dy[x], ol[x] * fl, dwl); dwn = fmaf(dy[x], on[x] * fn, dwn); }
-    dwl = row_sum(dwl);
-    dwn = row_sum(dwn);
-    const float ml = wl * dwl / D, mn = wn * dwn / D;
-    float dl[4], dn[4], dsm = 0.f;
+    dwl = sums(dwl, unused);
+    dwn = sums(dwn, dwn_s);                  // <dy, y_nla> over the row and over the slice
+    const float ml = wl * dwl / D, mn = wn * dwn_s * inv_ds;
+    float dl[4], dn[4], dsm = 0.f, dsm_s;
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
         dl[x] = fl * (wl * dy[x] - ol[x] * fl * ml);
         dn[x] = fn * (wn * dy[x] - on[x] * fn * mn);
         dsm = fmaf(dn[x], on[x], dsm);
     }
-    dsm = row_sum(dsm);
+    sums(dsm, dsm_s);
     if (!live) return;
     *reinterpret_cast<float4 *>(do_la + at) = make_float4(dl[0], dl[1], dl[2], dl[3]);
+    // (the tensor-core softmax backward reads the fp16 copy only)
     if (do_nla) *reinterpret_cast<float4 *>(do_nla + at) = make_float4(dn[0], dn[1], dn[2], dn[3]);
     const size_t at16 = (((size_t)b * H + h) * L + l) * D + li * 4;
     auto h4 = [](float x0, float x1, float x2, float x3) {
@@ -374,10 +280,8 @@ combine_bwd_vec_kernel(const float *__restrict__ o_la, const float *__restrict__
         const float gg = gs * sg;
         *reinterpret_cast<uint2 *>(dolag16 + at16) = h4(gg * dl[0], gg * dl[1], gg * dl[2], gg * dl[3]);
     }
-    if (li == 0) {
-        if (dw) { dw[rr * 2] = dwn; dw[rr * 2 + 1] = dwl; }
-        Dsm[((size_t)b * H + h) * L + l] = gs * dsm;
-    }
+    if (li % lps == 0) Dsm[(((size_t)b * H + h) * G + li / lps) * L + l] = gs * dsm_s;
+    if (li == 0 && dw) { dw[rr * 2] = dwn; dw[rr * 2 + 1] = dwl; }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1013,16 +917,8 @@ static cudaError_t combine_bwd_impl(const float *o_la, const float *o_nla, const
                                     const float *Gd, float scale_la, const int32_t *gsc, Shape s,
                                     cudaStream_t st, int G) {
     const size_t rows = (size_t)s.B * s.L * s.H;
-    if (G <= 1) {
-        constexpr int kRowsPerBlock = (kThreads / 32) * (32 / (D / 4));
-        combine_bwd_vec_kernel<T, D><<<(unsigned)((rows + kRowsPerBlock - 1) / kRowsPerBlock), kThreads, 0, st>>>(
-            o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, (__half *)do16, (__half *)dola16,
-            (__half *)dolag16, Gd, scale_la, gsc, s.B, s.L, s.H);
-        count_launch();
-        return cudaGetLastError();
-    }
-    auto kernel = combine_bwd_kernel<T, D, true>;
-    kernel<<<(unsigned)((rows + 7) / 8), kThreads, 0, st>>>(
+    constexpr int kRowsPerBlock = (kThreads / 32) * (32 / (D / 4));
+    combine_bwd_kernel<T, D><<<(unsigned)((rows + kRowsPerBlock - 1) / kRowsPerBlock), kThreads, 0, st>>>(
         o_la, o_nla, (const T *)dout, w, eps, do_la, do_nla, dw, Dsm, (__half *)do16, (__half *)dola16,
         (__half *)dolag16, Gd, scale_la, gsc, G, s.B, s.L, s.H);
     count_launch();

@@ -469,6 +469,46 @@ template <int N> __device__ __forceinline__ void store_vec(__nv_bfloat16 *p, con
     }
 }
 
+// The forward normalisation with the same layout (d = 64 or 128, a slice an aligned group of 32 / G lanes).
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+qk_norm_f32_vec_kernel(const T *__restrict__ q, const T *__restrict__ k, float *__restrict__ q_la,
+                       float *__restrict__ k_la, float *__restrict__ q_sm, float *__restrict__ k_sm,
+                       size_t rows, int G, float norm_eps) {
+    constexpr int N = D / 32;
+    const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= rows) return;
+    const int lps = 32 / G;
+    const float inv_ds = (float)G / D;
+    const size_t at = row * D + (size_t)lane * N;
+    float x[2][N];
+    load_vec<N>(q + at, x[0]);
+    load_vec<N>(k + at, x[1]);
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+        float ss = 0.f, ss_s = 0.f;
+#pragma unroll
+        for (int j = 0; j < N; ++j) ss = fmaf(x[which][j], x[which][j], ss);
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            if (o == lps) ss_s = ss;
+            ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        }
+        if (lps == 32) ss_s = ss;
+        const float rl = rsqrtf(ss + norm_eps), rs = rsqrtf(fmaf(ss_s, inv_ds, norm_eps));
+        float y[N];
+#pragma unroll
+        for (int j = 0; j < N; ++j) y[j] = x[which][j] * rl;
+        store_vec<N>((which ? k_la : q_la) + at, y);
+        if (q_sm) {
+#pragma unroll
+            for (int j = 0; j < N; ++j) y[j] = x[which][j] * rs;
+            store_vec<N>((which ? k_sm : q_sm) + at, y);
+        }
+    }
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
 qk_norm_bwd_f32_kernel(const T *__restrict__ q, const T *__restrict__ k,
@@ -637,6 +677,16 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
 cudaError_t launch_qk_norm_f32(const void *q, const void *k, bool bf16, float *q_la, float *k_la, float *q_sm,
                                float *k_sm, size_t rows, int d, int G, float norm_eps, cudaStream_t st) {
     const unsigned blocks = (unsigned)((rows + 7) / 8);
+    if ((d == 64 || d == 128) && G >= 1 && 32 % G == 0 && !q_sm == !k_sm) {
+#define NATSL_NF(TT, DD)                                                                                     \
+    qk_norm_f32_vec_kernel<TT, DD><<<blocks, 256, 0, st>>>((const TT *)q, (const TT *)k, q_la, k_la, q_sm, k_sm, \
+                                                          rows, G, norm_eps)
+        if (bf16) { if (d == 128) NATSL_NF(__nv_bfloat16, 128); else NATSL_NF(__nv_bfloat16, 64); }
+        else { if (d == 128) NATSL_NF(float, 128); else NATSL_NF(float, 64); }
+#undef NATSL_NF
+        count_launch();
+        return cudaGetLastError();
+    }
     if (bf16)
         qk_norm_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
                                                                  q_la, k_la, q_sm, k_sm, rows, d, G, norm_eps);
