@@ -33,11 +33,11 @@ namespace {
 constexpr int kThreads = 256;
 
 // ------------------------------------------------------------------------------------------
-// generic batched GEMM: C = alpha * op(A) op(B) (+ C), 64x64 output tiles, fp32
-// kTF32 (bf16 storage, whose tolerance it fits): the products run on the warp-level tensor-core path
-// with tf32 operands (fp32 range, 11 significant bits) and fp32 accumulation -- warp w owns rows
-// 16 (w & 3) .. and columns 32 (w >> 2) .. of the tile, four m16n8k8 products per 8 values of k --;
-// otherwise fp32 FMAs (fp32 storage: 1e-4 tolerance).
+// generic batched GEMM: C = alpha * op(A) op(B) (+ C), 64x64 output tiles, fp32.
+// fp32 storage (1e-4 tolerance): fp32 FMAs (bgemm_kernel).  bf16 storage, whose tolerance it fits:
+// the warp-level tensor-core path with tf32 operands (fp32 range, 11 significant bits) and fp32
+// accumulation (bgemm_tf32_kernel, below) -- warp w owns rows 16 (w & 3) .. and columns 32 (w >> 2) ..
+// of the tile, four m16n8k8 products per 8 values of k.
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t to_tf32(float x) {
     uint32_t r;
@@ -53,10 +53,10 @@ __device__ __forceinline__ const float *mat_base(const BMat &m, int b, int h, in
     return m.p + (size_t)b * m.sb + (size_t)h * m.sh + (size_t)ch * m.sc;
 }
 
-template <bool TA, bool TB, int MASK, bool kTF32>
+template <bool TA, bool TB, int MASK>
 __global__ void __launch_bounds__(kThreads)
 bgemm_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H, int NC) {
-    constexpr int kLd = kTF32 ? 72 : 68;      // (72: the fragment reads of a warp fall on 32 different banks)
+    constexpr int kLd = 68;
     __shared__ __align__(16) float As[16][kLd];
     __shared__ __align__(16) float Bs[16][kLd];
     const int z = blockIdx.z, ch = z % NC, bh = z / NC, b = bh / H, h = bh % H;
@@ -64,13 +64,11 @@ bgemm_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H,
     float *Cp = const_cast<float *>(mat_base(Cm, b, h, ch));
     const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
     const int t = threadIdx.x, ty = t >> 4, tx = t & 15;
-    float acc[4][4];          // fp32 FMAs: rows ty*4 + i, columns tx*4 + j; tf32: n-tile i, fragment element j
+    float acc[4][4];          // rows ty*4 + i, columns tx*4 + j
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-    const int warp = t >> 5, lane = t & 31, fg = lane >> 2, ft = lane & 3;
-    const int wr = (warp & 3) * 16, wc = (warp >> 2) * 32;
 
     for (int k0 = 0; k0 < K; k0 += 16) {
         if (!TA) {   // A[m][k], k contiguous
@@ -92,18 +90,6 @@ bgemm_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H,
             Bs[kk][c] = x.x; Bs[kk + 1][c] = x.y; Bs[kk + 2][c] = x.z; Bs[kk + 3][c] = x.w;
         }
         __syncthreads();
-        if (kTF32) {
-#pragma unroll
-            for (int k8 = 0; k8 < 16; k8 += 8) {
-                const uint32_t a[4] = {to_tf32(As[k8 + ft][wr + fg]), to_tf32(As[k8 + ft][wr + fg + 8]),
-                                       to_tf32(As[k8 + ft + 4][wr + fg]), to_tf32(As[k8 + ft + 4][wr + fg + 8])};
-#pragma unroll
-                for (int nt = 0; nt < 4; ++nt) {
-                    const uint32_t bfr[2] = {to_tf32(Bs[k8 + ft][wc + 8 * nt + fg]), to_tf32(Bs[k8 + ft + 4][wc + 8 * nt + fg])};
-                    mma_tf32_16x8x8(acc[nt], a, bfr);
-                }
-            }
-        } else
 #pragma unroll
         for (int kk = 0; kk < 16; ++kk) {
             const float4 a = *reinterpret_cast<const float4 *>(&As[kk][ty * 4]);
@@ -115,21 +101,6 @@ bgemm_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H,
                 for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
         }
         __syncthreads();
-    }
-    if (kTF32) {      // fragment layout: elements (0, 1) in row fg, (2, 3) in row fg + 8; columns 2 ft, 2 ft + 1
-#pragma unroll
-        for (int nt = 0; nt < 4; ++nt)
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                const int row = m0 + wr + fg + 8 * hh, col = n0 + wc + 8 * nt + 2 * ft;
-                float o0 = alpha * acc[nt][2 * hh], o1 = alpha * acc[nt][2 * hh + 1];
-                if (MASK == 1) { if (col > row) o0 = 0.f; if (col + 1 > row) o1 = 0.f; }
-                if (MASK == 2) { if (col >= row) o0 = 0.f; if (col + 1 >= row) o1 = 0.f; }
-                float2 *cr = reinterpret_cast<float2 *>(Cp + (size_t)row * Cm.ld + col);
-                if (accumulate) { const float2 old = *cr; o0 += old.x; o1 += old.y; }
-                *cr = make_float2(o0, o1);
-            }
-        return;
     }
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -150,6 +121,103 @@ bgemm_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H,
         }
         *reinterpret_cast<float4 *>(cr) = make_float4(o[0], o[1], o[2], o[3]);
     }
+}
+
+// The tf32 case as a pipeline: operands go to shared memory in the layout they have in global memory
+// (16-byte asynchronous copies, three 32-wide steps of k in flight) and the fragment reads adapt to the
+// layout instead -- rows of 36 floats for a k-contiguous operand, of 72 for an m- or n-contiguous one,
+// both free of bank conflicts for the m16n8k8 fragments.  Operands are rounded to tf32 as they are
+// read, products accumulated in fp32; k is a multiple of 32 (64 or the head dimension).
+constexpr int kBgK = 32, kBgStages = 3;
+constexpr int kBgTileFloats = 64 * (kBgK + 4);           // = kBgK * 72: either layout
+constexpr size_t kBgSmem = (size_t)kBgStages * 2 * kBgTileFloats * sizeof(float);
+__device__ __forceinline__ void cp_async16(float *dst, const float *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(
+                     static_cast<uint32_t>(__cvta_generic_to_shared(dst))),
+                 "l"(reinterpret_cast<uint64_t>(src))
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+template <bool TA, bool TB, int MASK>
+__global__ void __launch_bounds__(kThreads)
+bgemm_tf32_kernel(BMat A, BMat B, BMat Cm, int K, float alpha, int accumulate, int H, int NC) {
+    extern __shared__ __align__(16) float bg_smem[];
+    constexpr int kLdK = kBgK + 4, kLdMN = 72;
+    const int z = blockIdx.z, ch = z % NC, bh = z / NC, b = bh / H, h = bh % H;
+    const float *Ap = mat_base(A, b, h, ch), *Bp = mat_base(B, b, h, ch);
+    float *Cp = const_cast<float *>(mat_base(Cm, b, h, ch));
+    const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+    const int t = threadIdx.x, warp = t >> 5, lane = t & 31, fg = lane >> 2, ft = lane & 3;
+    const int wr = (warp & 3) * 16, wc = (warp >> 2) * 32;
+    const int nk = K / kBgK;
+    auto issue = [&](int kt) {
+        if (kt < nk) {
+            float *As = bg_smem + (size_t)(kt % kBgStages) * 2 * kBgTileFloats, *Bs = As + kBgTileFloats;
+            const int k0 = kt * kBgK;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int f = t + kThreads * i;
+                if (!TA) {   // A[m][k], k contiguous
+                    const int r = f / (kBgK / 4), kq = (f % (kBgK / 4)) * 4;
+                    cp_async16(As + r * kLdK + kq, Ap + (size_t)(m0 + r) * A.ld + k0 + kq);
+                } else {     // A[k][m], m contiguous
+                    const int kk = f / 16, r4 = (f % 16) * 4;
+                    cp_async16(As + kk * kLdMN + r4, Ap + (size_t)(k0 + kk) * A.ld + m0 + r4);
+                }
+                if (TB) {    // B[n][k], k contiguous
+                    const int c = f / (kBgK / 4), kq = (f % (kBgK / 4)) * 4;
+                    cp_async16(Bs + c * kLdK + kq, Bp + (size_t)(n0 + c) * B.ld + k0 + kq);
+                } else {     // B[k][n], n contiguous
+                    const int kk = f / 16, c4 = (f % 16) * 4;
+                    cp_async16(Bs + kk * kLdMN + c4, Bp + (size_t)(k0 + kk) * B.ld + n0 + c4);
+                }
+            }
+        }
+        cp_async_commit();       // (an empty group past the end keeps the count uniform)
+    };
+    float acc[4][4];             // n-tile i, fragment element j
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll
+    for (int kt = 0; kt < kBgStages - 1; ++kt) issue(kt);
+    for (int kt = 0; kt < nk; ++kt) {
+        cp_async_wait<kBgStages - 2>();          // step kt has landed (this thread's copies) ...
+        __syncthreads();                         // ... and everyone's; step kt - 1 has been read by all
+        issue(kt + kBgStages - 1);               // into the slot of step kt - 1
+        const float *As = bg_smem + (size_t)(kt % kBgStages) * 2 * kBgTileFloats, *Bs = As + kBgTileFloats;
+        auto a_at = [&](int m, int k) { return to_tf32(TA ? As[k * kLdMN + m] : As[m * kLdK + k]); };
+        auto b_at = [&](int k, int n) { return to_tf32(TB ? Bs[n * kLdK + k] : Bs[k * kLdMN + n]); };
+#pragma unroll
+        for (int k8 = 0; k8 < kBgK; k8 += 8) {
+            const uint32_t a[4] = {a_at(wr + fg, k8 + ft), a_at(wr + fg + 8, k8 + ft),
+                                   a_at(wr + fg, k8 + ft + 4), a_at(wr + fg + 8, k8 + ft + 4)};
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const uint32_t bfr[2] = {b_at(k8 + ft, wc + 8 * nt + fg), b_at(k8 + ft + 4, wc + 8 * nt + fg)};
+                mma_tf32_16x8x8(acc[nt], a, bfr);
+            }
+        }
+    }
+    cp_async_wait<0>();
+    // fragment layout: elements (0, 1) in row fg, (2, 3) in row fg + 8; columns 2 ft, 2 ft + 1
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int row = m0 + wr + fg + 8 * hh, col = n0 + wc + 8 * nt + 2 * ft;
+            float o0 = alpha * acc[nt][2 * hh], o1 = alpha * acc[nt][2 * hh + 1];
+            if (MASK == 1) { if (col > row) o0 = 0.f; if (col + 1 > row) o1 = 0.f; }
+            if (MASK == 2) { if (col >= row) o0 = 0.f; if (col + 1 >= row) o1 = 0.f; }
+            float2 *cr = reinterpret_cast<float2 *>(Cp + (size_t)row * Cm.ld + col);
+            if (accumulate) { const float2 old = *cr; o0 += old.x; o1 += old.y; }
+            *cr = make_float2(o0, o1);
+        }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -878,11 +946,16 @@ cudaError_t set_smem(Kn kernel, size_t bytes) {
 cudaError_t launch_bgemm(bool ta, bool tb, int mask, BMat A, BMat B, BMat C, int m, int n, int k,
                          float alpha, bool accumulate, Shape s, cudaStream_t st) {
     const int NC = s.L / kC;
+    if (m % 64 || n % 64 || k % kBgK) return cudaErrorInvalidValue;
     dim3 grid(n / 64, m / 64, s.B * s.H * NC);
 #define NATSL_BG(TA, TB, MK)                                                                                   \
     do {                                                                                                        \
-        if (s.bf16) bgemm_kernel<TA, TB, MK, true><<<grid, kThreads, 0, st>>>(A, B, C, k, alpha, accumulate ? 1 : 0, s.H, NC); \
-        else bgemm_kernel<TA, TB, MK, false><<<grid, kThreads, 0, st>>>(A, B, C, k, alpha, accumulate ? 1 : 0, s.H, NC);       \
+        if (s.bf16) {                                                                                           \
+            cudaError_t e = cudaFuncSetAttribute(bgemm_tf32_kernel<TA, TB, MK>,                                 \
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBgSmem);    \
+            if (e != cudaSuccess) return e;                                                                     \
+            bgemm_tf32_kernel<TA, TB, MK><<<grid, kThreads, kBgSmem, st>>>(A, B, C, k, alpha, accumulate ? 1 : 0, s.H, NC); \
+        } else bgemm_kernel<TA, TB, MK><<<grid, kThreads, 0, st>>>(A, B, C, k, alpha, accumulate ? 1 : 0, s.H, NC); \
     } while (0)
     if (!ta && !tb && mask == 0) NATSL_BG(false, false, 0);
     else if (!ta && tb && mask == 0) NATSL_BG(false, true, 0);
