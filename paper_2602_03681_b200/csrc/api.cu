@@ -93,8 +93,12 @@ int scan_segments(const natsl_params *p) {
     int nseg = 1;
     while (2 * BH * (nseg * 2) <= 128 && NC % (nseg * 2) == 0 && NC / (nseg * 2) >= 8) nseg *= 2;
     // Once the scan is segmented (and so already pays its second run), one more doubling up to one CTA per
-    // SM: the two runs shrink by half again, which outweighs what the softmax kernel loses beside them.
-    if (nseg >= 2 && BH * (nseg * 2) <= 128 && NC % (nseg * 2) == 0 && NC / (nseg * 2) >= 8) nseg *= 2;
+    // SM: the two runs shrink by half again, which outweighs what the softmax kernel loses beside them --
+    // unless the call appends to a cache: the softmax kernel then also reads the earlier pieces' keys, is
+    // the longer of the two and needs the multiprocessors (a long prompt in pieces was 14 % slower with it).
+    if (!(p->flags & NATSL_APPEND_CACHE) && nseg >= 2 && BH * (nseg * 2) <= 128 && NC % (nseg * 2) == 0 &&
+        NC / (nseg * 2) >= 8)
+        nseg *= 2;
     return nseg;
 }
 
