@@ -790,24 +790,32 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dKb), TM(f.W), CC(f.M), kC, kC, di, -1.f, false, sgemm, st));
     NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dVb), TM(f.U), CC(f.M), kC, kC, di, -1.f, true, sgemm, st));
     NATSL_TRY(launch_mask_scale(f.M, f.N, f.Gcum, beta, route_bt, p->scale_la, f.Mg, f.Ms, f.Ns, s, st));
-    NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Mg), TM(f.k32), TM(f.X1p), kC, di, kC, 1.f, false, sgemm, st));
-    NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ms), TM(f.k32), TM(f.X2), kC, di, kC, 1.f, false, sgemm, st));
-    NATSL_TRY(launch_bgemm(false, false, 0, CC(f.Ns), TM(f.k32), TM(f.X3), kC, di, kC, 1.f, false, sgemm, st));
-    NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Ns), TM(f.q32), TM(f.X4), kC, di, kC, 1.f, false, sgemm, st));
+    // The last four products (X1 = Mg K, X2 = Ms^T K, X3 = Ns K, X4 = Ns^T Q) and the assembly: on tensor
+    // cores one kernel per chunk that keeps the products in its accumulators; otherwise four tile GEMMs
+    // and the row-local assembly.
+    auto assemble = [&](void *dq_o, void *dk_o, void *dv_o, Shape so) -> cudaError_t {
+        if (tensor_cores) return launch_gdn_xassemble(a, f.Mg, f.Ms, f.Ns, dq_o, dk_o, dv_o, so, st);
+        cudaError_t e;
+        if ((e = launch_bgemm(false, false, 0, CC(f.Mg), TM(f.k32), TM(f.X1p), kC, di, kC, 1.f, false, sgemm, st)) != cudaSuccess) return e;
+        if ((e = launch_bgemm(true, false, 0, CC(f.Ms), TM(f.k32), TM(f.X2), kC, di, kC, 1.f, false, sgemm, st)) != cudaSuccess) return e;
+        if ((e = launch_bgemm(false, false, 0, CC(f.Ns), TM(f.k32), TM(f.X3), kC, di, kC, 1.f, false, sgemm, st)) != cudaSuccess) return e;
+        if ((e = launch_bgemm(true, false, 0, CC(f.Ns), TM(f.q32), TM(f.X4), kC, di, kC, 1.f, false, sgemm, st)) != cudaSuccess) return e;
+        return launch_gdn_assemble(a, dq_o, dk_o, dv_o, so, st);
+    };
     // With the normalisation the assembly's dq, dk are gradients with respect to the normalised rows; a
     // last kernel applies the two row-local Jacobians.  fp32 storage: in place.  bf16 storage: the
     // assembly writes fp32 (into buffers the chunk-level products are done with) and the last kernel
     // rounds once.
     if (!normed) {
-        NATSL_TRY(launch_gdn_assemble(a, dq, dk, dv, s, st));
+        NATSL_TRY(assemble(dq, dk, dv, s));
     } else if (!s.bf16) {
-        NATSL_TRY(launch_gdn_assemble(a, dq, dk, dv, s, st));
+        NATSL_TRY(assemble(dq, dk, dv, s));
         NATSL_TRY(launch_qk_norm_bwd_f32(q, k, false, route, (const float *)dq, f.dq_sm, (const float *)dk, nullptr,
                                          dq, dk, nullptr, (size_t)(B * L * H), p->d, hg.G, hg.norm_eps, st,
                                          general_block ? f.dk_x : nullptr));
     } else {
         float *dq32 = f.dW, *dk32 = f.W, *dv32 = f.U;
-        NATSL_TRY(launch_gdn_assemble(a, dq32, dk32, dv32, s32, st));
+        NATSL_TRY(assemble(dq32, dk32, dv32, s32));
         NATSL_TRY(launch_qk_norm_bwd_f32(q, k, true, route, dq32, f.dq_sm, dk32, dv32, dq, dk, dv,
                                          (size_t)(B * L * H), p->d, hg.G, hg.norm_eps, st,
                                          general_block ? f.dk_x : nullptr));

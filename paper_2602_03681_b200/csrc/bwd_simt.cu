@@ -49,6 +49,10 @@ __device__ __forceinline__ void mma_tf32_16x8x8(float (&c)[4], const uint32_t (&
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
+__device__ __forceinline__ void store2(float *p, float a, float b) { *reinterpret_cast<float2 *>(p) = make_float2(a, b); }
+__device__ __forceinline__ void store2(__nv_bfloat16 *p, float a, float b) {
+    *reinterpret_cast<__nv_bfloat162 *>(p) = __floats2bfloat162_rn(a, b);
+}
 __device__ __forceinline__ const float *mat_base(const BMat &m, int b, int h, int ch) {
     return m.p + (size_t)b * m.sb + (size_t)h * m.sh + (size_t)ch * m.sc;
 }
@@ -891,6 +895,167 @@ gdn_assemble_kernel(const float *__restrict__ q32, const float *__restrict__ k32
     }
 }
 
+// The last four chunk-level products and the assembly in one kernel per chunk (bf16 storage, tf32
+// products as in bgemm_tf32_kernel): X1 = Mg K, X2 = Ms^T K, X3 = Ns K, X4 = Ns^T Q stay in the
+// accumulator fragments and meet the other terms of dq, dk, dv there, so the four [B,L,H,d] fp32
+// arrays are neither written nor read back.  One CTA per chunk, 64 columns at a time; warp w owns rows
+// 16 (w & 3) .. and columns 32 (w >> 2) .. of the 64; the eight per-row dot products are summed over a
+// thread's columns, then over the four lanes that share a row, then over the two warps that do.
+constexpr int kXaLdA = 68, kXaLdT = 72;                  // rows read along k / read transposed (and K, Q)
+constexpr size_t kXaSmem = sizeof(float) * (2 * kC * kXaLdA + 3 * kC * kXaLdT + 4 * kC + 2 * kC * 8);
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads, 2)
+gdn_xassemble_kernel(const float *__restrict__ q32, const float *__restrict__ k32,
+                     const float *__restrict__ v32, const float *__restrict__ Gcum,
+                     const float *__restrict__ beta, const uint8_t *__restrict__ route,
+                     const float *__restrict__ dQg, const float *__restrict__ dKb,
+                     const float *__restrict__ dVb, const float *__restrict__ dKt,
+                     const float *__restrict__ Mg, const float *__restrict__ Ms,
+                     const float *__restrict__ Ns, const float *__restrict__ dq_sm,
+                     const float *__restrict__ dk_x, const float *__restrict__ dv_x, float scale_la,
+                     T *__restrict__ dq, T *__restrict__ dk, T *__restrict__ dv, float *__restrict__ dGrow,
+                     float *__restrict__ kappa, float *__restrict__ dbeta, int L, int H) {
+    extern __shared__ __align__(16) float xa_smem[];
+    float *sMg = xa_smem;                        // [i][j], ld 68
+    float *sNs = sMg + kC * kXaLdA;              // [i][j], ld 68
+    float *sMs = sNs + kC * kXaLdA;              // [i][j], ld 72 (read transposed only)
+    float *sK = sMs + kC * kXaLdT;               // [token][64 columns], ld 72
+    float *sQ = sK + kC * kXaLdT;
+    float *sGam = sQ + kC * kXaLdT, *sKt = sGam + kC, *sBt = sKt + kC, *sLin = sBt + kC;
+    float *sSum = sLin + kC;                     // [2 column warps][64 rows][8]
+    const int NC = L / kC, ch = blockIdx.x % NC, bh = blockIdx.x / NC, b = bh / H, h = bh % H;
+    const int t = threadIdx.x, warp = t >> 5, lane = t & 31, fg = lane >> 2, ft = lane & 3;
+    const int wr = (warp & 3) * 16, wcw = warp >> 2, wc = wcw * 32;
+    const size_t tok0 = ((size_t)b * L + (size_t)ch * kC) * H + h;         // the chunk's first token (stride H)
+    const size_t bhl = (size_t)bh * L + (size_t)ch * kC;
+    {
+        const float *mg = Mg + (size_t)blockIdx.x * kC * kC, *msrc = Ms + (size_t)blockIdx.x * kC * kC,
+                    *ns = Ns + (size_t)blockIdx.x * kC * kC;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int f = t + kThreads * i, r = f >> 4, c4 = (f & 15) * 4;
+            cp_async16(sMg + r * kXaLdA + c4, mg + r * kC + c4);
+            cp_async16(sNs + r * kXaLdA + c4, ns + r * kC + c4);
+            cp_async16(sMs + r * kXaLdT + c4, msrc + r * kC + c4);
+        }
+    }
+    if (t < kC) {
+        const size_t tok = tok0 + (size_t)t * H;
+        const float Gi = Gcum[bhl + t], GC = Gcum[bhl + kC - 1];
+        const bool lin = !route || route[tok] == 0;
+        sGam[t] = __expf(Gi);
+        sKt[t] = __expf(GC - Gi);
+        sBt[t] = lin ? beta[tok] : 0.f;
+        sLin[t] = lin ? 1.f : 0.f;
+    }
+    float sums[2][8];            // per row half: kdKb, qdQg, kdKt, kX1, kX2, qX3, kX4, vdVb
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sums[hh][j] = 0.f;
+
+    for (int n0 = 0; n0 < D; n0 += 64) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int f = t + kThreads * i, r = f >> 4, c4 = (f & 15) * 4;
+            cp_async16(sK + r * kXaLdT + c4, k32 + (tok0 + (size_t)r * H) * D + n0 + c4);
+            cp_async16(sQ + r * kXaLdT + c4, q32 + (tok0 + (size_t)r * H) * D + n0 + c4);
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+        float x1[4][4], x2[4][4], x3[4][4], x4[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { x1[i][j] = 0.f; x2[i][j] = 0.f; x3[i][j] = 0.f; x4[i][j] = 0.f; }
+#pragma unroll 2
+        for (int k8 = 0; k8 < kC; k8 += 8) {
+            const int m0 = wr + fg, m1 = wr + fg + 8, ka = k8 + ft, kb = k8 + ft + 4;
+            const uint32_t a1[4] = {to_tf32(sMg[m0 * kXaLdA + ka]), to_tf32(sMg[m1 * kXaLdA + ka]),
+                                    to_tf32(sMg[m0 * kXaLdA + kb]), to_tf32(sMg[m1 * kXaLdA + kb])};
+            const uint32_t a2[4] = {to_tf32(sMs[ka * kXaLdT + m0]), to_tf32(sMs[ka * kXaLdT + m1]),
+                                    to_tf32(sMs[kb * kXaLdT + m0]), to_tf32(sMs[kb * kXaLdT + m1])};
+            const uint32_t a3[4] = {to_tf32(sNs[m0 * kXaLdA + ka]), to_tf32(sNs[m1 * kXaLdA + ka]),
+                                    to_tf32(sNs[m0 * kXaLdA + kb]), to_tf32(sNs[m1 * kXaLdA + kb])};
+            const uint32_t a4[4] = {to_tf32(sNs[ka * kXaLdA + m0]), to_tf32(sNs[ka * kXaLdA + m1]),
+                                    to_tf32(sNs[kb * kXaLdA + m0]), to_tf32(sNs[kb * kXaLdA + m1])};
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int n = wc + 8 * nt + fg;
+                const uint32_t bk[2] = {to_tf32(sK[ka * kXaLdT + n]), to_tf32(sK[kb * kXaLdT + n])};
+                const uint32_t bq[2] = {to_tf32(sQ[ka * kXaLdT + n]), to_tf32(sQ[kb * kXaLdT + n])};
+                mma_tf32_16x8x8(x1[nt], a1, bk);
+                mma_tf32_16x8x8(x2[nt], a2, bk);
+                mma_tf32_16x8x8(x3[nt], a3, bk);
+                mma_tf32_16x8x8(x4[nt], a4, bq);
+            }
+        }
+        // fragment layout: elements (0, 1) in row fg, (2, 3) in row fg + 8; columns 2 ft, 2 ft + 1
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int row = wr + fg + 8 * hh;
+            const float gam = sGam[row], kt = sKt[row], bt = sBt[row];
+            const bool lin = sLin[row] != 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int cl = wc + 8 * nt + 2 * ft;                     // column within the 64
+                const size_t i = (tok0 + (size_t)row * H) * D + n0 + cl;
+                const float2 a_dQg = *reinterpret_cast<const float2 *>(dQg + i), a_dKb = *reinterpret_cast<const float2 *>(dKb + i);
+                const float2 a_dVb = *reinterpret_cast<const float2 *>(dVb + i), a_dKt = *reinterpret_cast<const float2 *>(dKt + i);
+                const float2 vv = *reinterpret_cast<const float2 *>(v32 + i);
+                const float2 qv = *reinterpret_cast<const float2 *>(sQ + row * kXaLdT + cl);
+                const float2 kv = *reinterpret_cast<const float2 *>(sK + row * kXaLdT + cl);
+                float2 e_dq = dq_sm ? *reinterpret_cast<const float2 *>(dq_sm + i) : make_float2(0.f, 0.f);
+                float2 e_dk = dk_x ? *reinterpret_cast<const float2 *>(dk_x + i) : make_float2(0.f, 0.f);
+                float2 e_dv = dv_x ? *reinterpret_cast<const float2 *>(dv_x + i) : make_float2(0.f, 0.f);
+                const float x1a = x1[nt][2 * hh], x1b = x1[nt][2 * hh + 1], x2a = x2[nt][2 * hh], x2b = x2[nt][2 * hh + 1];
+                const float x3a = x3[nt][2 * hh], x3b = x3[nt][2 * hh + 1], x4a = x4[nt][2 * hh], x4b = x4[nt][2 * hh + 1];
+                float *sm = sums[hh];
+                sm[0] = fmaf(kv.x, a_dKb.x, fmaf(kv.y, a_dKb.y, sm[0]));
+                sm[1] = fmaf(qv.x, a_dQg.x, fmaf(qv.y, a_dQg.y, sm[1]));
+                sm[2] = fmaf(kv.x, a_dKt.x, fmaf(kv.y, a_dKt.y, sm[2]));
+                sm[3] = fmaf(kv.x, x1a, fmaf(kv.y, x1b, sm[3]));
+                sm[4] = fmaf(kv.x, x2a, fmaf(kv.y, x2b, sm[4]));
+                sm[5] = fmaf(qv.x, x3a, fmaf(qv.y, x3b, sm[5]));
+                sm[6] = fmaf(kv.x, x4a, fmaf(kv.y, x4b, sm[6]));
+                sm[7] = fmaf(vv.x, a_dVb.x, fmaf(vv.y, a_dVb.y, sm[7]));
+                const float sgm = scale_la * gam;
+                store2(dq + i, sgm * a_dQg.x + x3a + e_dq.x, sgm * a_dQg.y + x3b + e_dq.y);
+                if (lin) {
+                    const float bg = bt * gam;
+                    store2(dk + i, bg * a_dKb.x + kt * a_dKt.x + bt * x1a + x2a + x4a + e_dk.x,
+                           bg * a_dKb.y + kt * a_dKt.y + bt * x1b + x2b + x4b + e_dk.y);
+                    store2(dv + i, bt * a_dVb.x + e_dv.x, bt * a_dVb.y + e_dv.y);
+                }
+            }
+        }
+        __syncthreads();         // K, Q of these columns have been read by all
+    }
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float v = sums[hh][j];
+            v += __shfl_xor_sync(0xffffffffu, v, 1);
+            v += __shfl_xor_sync(0xffffffffu, v, 2);
+            if (ft == 0) sSum[(wcw * kC + wr + fg + 8 * hh) * 8 + j] = v;
+        }
+    __syncthreads();
+    if (t < kC) {
+        float r[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r[j] = sSum[t * 8 + j] + sSum[(kC + t) * 8 + j];
+        const float gam = sGam[t], kt = sKt[t], bt = sBt[t];
+        const bool lin = sLin[t] != 0.f;
+        const float kap = kt * r[2];
+        dGrow[bhl + t] = bt * gam * r[0] + scale_la * gam * r[1] - kap + bt * r[3] - r[4] + r[5] - r[6];
+        kappa[bhl + t] = kap;
+        dbeta[tok0 + (size_t)t * H] = lin ? gam * r[0] + r[7] + r[3] : 0.f;
+    }
+}
+
 // dg_j = sum_{i>=j in chunk} dG_i, with the chunk-end extras added to the last row.
 __global__ void dg_kernel(const float *__restrict__ dGrow, const float *__restrict__ kappa,
                           const float *__restrict__ gS, const float *__restrict__ Gcum, int n_slices,
@@ -1189,6 +1354,40 @@ static cudaError_t finish_impl(const AssembleArgs &a, void *dk, void *dv, Shape 
                                                        (T *)dk, (T *)dv, s.L, s.H);
     count_launch();
     return cudaGetLastError();
+}
+
+template <typename T, int D>
+static cudaError_t xassemble_impl(const AssembleArgs &a, const float *Mg, const float *Ms, const float *Ns,
+                                  void *dq, void *dk, void *dv, Shape s, cudaStream_t st) {
+    const int NC = s.L / kC;
+    const size_t nch = (size_t)s.B * s.H * NC;
+    cudaError_t e = cudaFuncSetAttribute(gdn_xassemble_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)kXaSmem);
+    if (e != cudaSuccess) return e;
+    gdn_xassemble_kernel<T, D><<<(unsigned)nch, kThreads, kXaSmem, st>>>(
+        a.q32, a.k32, a.v32, a.Gcum, a.beta, a.route, a.dQg, a.dKb, a.dVb, a.dKt, Mg, Ms, Ns, a.dq_sm, a.dk_x,
+        a.dv_x, a.scale_la, (T *)dq, (T *)dk, (T *)dv, a.dGrow, a.kappa, a.dbeta, s.L, s.H);
+    count_launch();
+    dg_kernel<<<(unsigned)((nch + 127) / 128), 128, 0, st>>>(a.dGrow, a.kappa, a.gS, a.Gcum,
+                                                            s.d / kDvs, a.dg, s.B, s.L, s.H);
+    count_launch();
+    if (a.no_scatter) return cudaGetLastError();
+    constexpr int kRows = kThreads / (D / 4);
+    dim3 grid((a.cap + kRows - 1) / kRows, s.B * s.H);
+    scatter_sm_kernel<T, D><<<grid, kThreads, 0, st>>>(a.dk_sm, a.dv_sm, a.cap, a.sm_idx, a.sm_prefix,
+                                                       (T *)dk, (T *)dv, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gdn_xassemble(const AssembleArgs &a, const float *Mg, const float *Ms, const float *Ns,
+                                 void *dq, void *dk, void *dv, Shape s, cudaStream_t st) {
+    if (s.bf16) {
+        if (s.d == 128) return xassemble_impl<__nv_bfloat16, 128>(a, Mg, Ms, Ns, dq, dk, dv, s, st);
+        return xassemble_impl<__nv_bfloat16, 64>(a, Mg, Ms, Ns, dq, dk, dv, s, st);
+    }
+    if (s.d == 128) return xassemble_impl<float, 128>(a, Mg, Ms, Ns, dq, dk, dv, s, st);
+    return xassemble_impl<float, 64>(a, Mg, Ms, Ns, dq, dk, dv, s, st);
 }
 
 cudaError_t launch_gdn_finish(const AssembleArgs &a, void *dk, void *dv, Shape s, cudaStream_t st,

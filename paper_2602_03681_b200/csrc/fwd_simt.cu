@@ -402,35 +402,7 @@ softmax_combine_simt_kernel(const T *__restrict__ q, const T *__restrict__ k_sm,
 // Per-operation normalisation of q and k for fp32 storage (Section 4.3): one warp per row of d
 // columns writes the L2-normalised row (linear operation) and the row with each of its G slices
 // RMS-normalised (softmax operation).  The tensor-core path does both inside its kernels instead.
-template <typename T>
-__global__ void __launch_bounds__(256)
-qk_norm_f32_kernel(const T *__restrict__ q, const T *__restrict__ k, float *__restrict__ q_la,
-                   float *__restrict__ k_la, float *__restrict__ q_sm, float *__restrict__ k_sm,
-                   size_t rows, int d, int G, float norm_eps) {
-    const size_t row = (size_t)blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= rows) return;
-    const int ds = d / G;                                // 32, 64 or 128: a multiple of the warp size
-    for (int which = 0; which < 2; ++which) {
-        const T *src = (which ? k : q) + row * d;
-        float *la = (which ? k_la : q_la) + row * d, *sm = (which ? k_sm : q_sm);
-        float x[4], ss_all = 0.f;
-        for (int j = 0; j < d / 32; ++j) {
-            x[j] = to_f32(src[lane + 32 * j]);
-            ss_all = fmaf(x[j], x[j], ss_all);
-        }
-        ss_all = warp_sum(ss_all);
-        const float rl = rsqrtf(ss_all + norm_eps);
-        for (int sg = 0; sm && sg < G; ++sg) {
-            float ss = 0.f;
-            for (int j = sg * ds / 32; j < (sg + 1) * ds / 32; ++j) ss = fmaf(x[j], x[j], ss);
-            ss = warp_sum(ss);
-            const float rs = rsqrtf(ss / ds + norm_eps);
-            for (int j = sg * ds / 32; j < (sg + 1) * ds / 32; ++j) sm[row * d + lane + 32 * j] = x[j] * rs;
-        }
-        for (int j = 0; j < d / 32; ++j) la[lane + 32 * j] = x[j] * rl;
-    }
-}
+// (qk_norm_f32_kernel, below the vector helpers.)
 
 // Backward of that normalisation, in place on fp32 gradients, one warp per row.  On entry dq holds the
 // gradient with respect to the L2-normalised q (linear operation) and dq_sm the one with respect to the
@@ -472,7 +444,7 @@ template <int N> __device__ __forceinline__ void store_vec(__nv_bfloat16 *p, con
 // The forward normalisation with the same layout (d = 64 or 128, a slice an aligned group of 32 / G lanes).
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
-qk_norm_f32_vec_kernel(const T *__restrict__ q, const T *__restrict__ k, float *__restrict__ q_la,
+qk_norm_f32_kernel(const T *__restrict__ q, const T *__restrict__ k, float *__restrict__ q_la,
                        float *__restrict__ k_la, float *__restrict__ q_sm, float *__restrict__ k_sm,
                        size_t rows, int G, float norm_eps) {
     constexpr int N = D / 32;
@@ -677,22 +649,13 @@ cudaError_t launch_softmax_combine_simt(const void *q, const void *k_sm, const v
 cudaError_t launch_qk_norm_f32(const void *q, const void *k, bool bf16, float *q_la, float *k_la, float *q_sm,
                                float *k_sm, size_t rows, int d, int G, float norm_eps, cudaStream_t st) {
     const unsigned blocks = (unsigned)((rows + 7) / 8);
-    if ((d == 64 || d == 128) && G >= 1 && 32 % G == 0 && !q_sm == !k_sm) {
-#define NATSL_NF(TT, DD)                                                                                     \
-    qk_norm_f32_vec_kernel<TT, DD><<<blocks, 256, 0, st>>>((const TT *)q, (const TT *)k, q_la, k_la, q_sm, k_sm, \
-                                                          rows, G, norm_eps)
-        if (bf16) { if (d == 128) NATSL_NF(__nv_bfloat16, 128); else NATSL_NF(__nv_bfloat16, 64); }
-        else { if (d == 128) NATSL_NF(float, 128); else NATSL_NF(float, 64); }
+    if ((d != 64 && d != 128) || G < 1 || 32 % G != 0 || !q_sm != !k_sm) return cudaErrorInvalidValue;
+#define NATSL_NF(TT, DD)                                                                                  \
+    qk_norm_f32_kernel<TT, DD><<<blocks, 256, 0, st>>>((const TT *)q, (const TT *)k, q_la, k_la, q_sm, k_sm, \
+                                                      rows, G, norm_eps)
+    if (bf16) { if (d == 128) NATSL_NF(__nv_bfloat16, 128); else NATSL_NF(__nv_bfloat16, 64); }
+    else { if (d == 128) NATSL_NF(float, 128); else NATSL_NF(float, 64); }
 #undef NATSL_NF
-        count_launch();
-        return cudaGetLastError();
-    }
-    if (bf16)
-        qk_norm_f32_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16 *)q, (const __nv_bfloat16 *)k,
-                                                                 q_la, k_la, q_sm, k_sm, rows, d, G, norm_eps);
-    else
-        qk_norm_f32_kernel<float><<<blocks, 256, 0, st>>>((const float *)q, (const float *)k, q_la, k_la, q_sm,
-                                                         k_sm, rows, d, G, norm_eps);
     count_launch();
     return cudaGetLastError();
 }

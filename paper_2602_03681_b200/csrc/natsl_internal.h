@@ -248,6 +248,10 @@ struct AssembleArgs {
 // compacted softmax-branch gradients), dbeta, dg.  Three kernels.
 cudaError_t launch_gdn_assemble(const AssembleArgs &a, void *dq, void *dk, void *dv, Shape s,
                                 cudaStream_t st);
+// The same with the four products X1 = Mg K, X2 = Ms^T K, X3 = Ns K, X4 = Ns^T Q formed inside (tf32
+// tensor-core products; a.X1p .. a.X4 are not read); s.bf16 says what dq, dk, dv are stored as.
+cudaError_t launch_gdn_xassemble(const AssembleArgs &a, const float *Mg, const float *Ms, const float *Ns,
+                                 void *dq, void *dk, void *dv, Shape s, cudaStream_t st);
 // The last two of those kernels only (dg from the per-token sums, scatter of the retained tokens'
 // dk, dv), for callers that formed dq, dk, dv of the linear tokens and the sums themselves.
 cudaError_t launch_gdn_finish(const AssembleArgs &a, void *dk, void *dv, Shape s, cudaStream_t st,
