@@ -780,16 +780,17 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, sgemm, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, sgemm, st));
     NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, sgemm, st));
-    NATSL_TRY(launch_bgemm(false, true, 1, TM(f.do_la), TM(f.Ut), CC(f.N), kC, kC, di, 1.f, false, sgemm, st));
-    if (tensor_cores) {   // [dKb | dVb] = (I + A)^-T [dW | dU~] with the inverse the forward already formed
-        NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dW), TM(f.dKb), kC, di, kC, 1.f, false, sgemm, st));
-        NATSL_TRY(launch_bgemm(true, false, 0, CC(f.Tinv), TM(f.dUt), TM(f.dVb), kC, di, kC, 1.f, false, sgemm, st));
+    if (tensor_cores) {   // [dKb | dVb] = (I + A)^-T [dW | dU~] with the inverse the forward already formed, M, N and
+                          // their masked, scaled forms: one kernel per chunk
+        NATSL_TRY(launch_gdn_tm(f.Tinv, f.dW, f.dUt, f.W, f.U, f.do_la, f.Ut, f.Gcum, beta, route_bt, p->scale_la,
+                                f.dKb, f.dVb, f.Mg, f.Ms, f.Ns, s, st));
     } else {
+        NATSL_TRY(launch_bgemm(false, true, 1, TM(f.do_la), TM(f.Ut), CC(f.N), kC, kC, di, 1.f, false, sgemm, st));
         NATSL_TRY(launch_gdn_tsolve(f.Abar, beta, route_bt, f.dW, f.dUt, f.dKb, f.dVb, s, st));
+        NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dKb), TM(f.W), CC(f.M), kC, kC, di, -1.f, false, sgemm, st));
+        NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dVb), TM(f.U), CC(f.M), kC, kC, di, -1.f, true, sgemm, st));
+        NATSL_TRY(launch_mask_scale(f.M, f.N, f.Gcum, beta, route_bt, p->scale_la, f.Mg, f.Ms, f.Ns, s, st));
     }
-    NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dKb), TM(f.W), CC(f.M), kC, kC, di, -1.f, false, sgemm, st));
-    NATSL_TRY(launch_bgemm(false, true, 2, TM(f.dVb), TM(f.U), CC(f.M), kC, kC, di, -1.f, true, sgemm, st));
-    NATSL_TRY(launch_mask_scale(f.M, f.N, f.Gcum, beta, route_bt, p->scale_la, f.Mg, f.Ms, f.Ns, s, st));
     // The last four products (X1 = Mg K, X2 = Ms^T K, X3 = Ns K, X4 = Ns^T Q) and the assembly: on tensor
     // cores one kernel per chunk that keeps the products in its accumulators; otherwise four tile GEMMs
     // and the row-local assembly.

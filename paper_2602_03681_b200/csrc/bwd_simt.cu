@@ -895,6 +895,151 @@ gdn_assemble_kernel(const float *__restrict__ q32, const float *__restrict__ k32
     }
 }
 
+// The middle of the chunk-level chain in one kernel per chunk (bf16 storage, tf32 products):
+//   dKb = Tinv^T dW, dVb = Tinv^T dU~   (written out: the assembly reads them)
+//   M = -strictly_lower(dKb W^T + dVb U^T),  N = lower(dO U~^T)
+//   Mg = M . Gamma, Ms = diag(beta~) Mg, Ns = scale_la N . Gamma
+// 64 columns of the head at a time: dKb, dVb of those columns go from the accumulators to shared memory as
+// the next products' operands, and M, N add up in accumulators over the column blocks; the two 64 x 64
+// intermediates never reach global memory.  Warp w owns rows 16 (w & 3) .. and columns 32 (w >> 2) ..
+// of every 64 x 64 result.  Operand rows are 72 floats when read along the row index and 68 when read
+// along k (both free of bank conflicts for the fragments).
+constexpr size_t kTmSmem = sizeof(float) * (5 * kC * 72 + 2 * kC);
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 2)
+gdn_tm_kernel(const float *__restrict__ Tinv, const float *__restrict__ dW, const float *__restrict__ dUt,
+              const float *__restrict__ W, const float *__restrict__ U, const float *__restrict__ dO,
+              const float *__restrict__ Ut, const float *__restrict__ Gcum, const float *__restrict__ beta,
+              const uint8_t *__restrict__ route, float scale_la, float *__restrict__ dKb,
+              float *__restrict__ dVb, float *__restrict__ Mg, float *__restrict__ Ms, float *__restrict__ Ns,
+              int L, int H) {
+    extern __shared__ __align__(16) float tm_smem[];
+    float *sT = tm_smem, *bufA = sT + kC * 72, *bufB = bufA + kC * 72, *bufC = bufB + kC * 72, *bufD = bufC + kC * 72;
+    float *Gs = bufD + kC * 72, *bts = Gs + kC;
+    const int NC = L / kC, ch = blockIdx.x % NC, bh = blockIdx.x / NC, b = bh / H, h = bh % H;
+    const int t = threadIdx.x, warp = t >> 5, lane = t & 31, fg = lane >> 2, ft = lane & 3;
+    const int wr = (warp & 3) * 16, wc = (warp >> 2) * 32;
+    const size_t tok0 = ((size_t)b * L + (size_t)ch * kC) * H + h;         // the chunk's first token (stride H)
+    // 64 tokens x 64 columns [n0, n0 + 64) of a token-major array into rows of `ld` floats
+    auto load_tile = [&](float *dst, int ld, const float *src, int n0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int f = t + kThreads * i, r = f >> 4, c4 = (f & 15) * 4;
+            cp_async16(dst + r * ld + c4, src + (tok0 + (size_t)r * H) * D + n0 + c4);
+        }
+    };
+    {
+        const float *ti = Tinv + (size_t)blockIdx.x * kC * kC;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int f = t + kThreads * i, r = f >> 4, c4 = (f & 15) * 4;
+            cp_async16(sT + r * 72 + c4, ti + r * kC + c4);
+        }
+    }
+    if (t < kC) {
+        const size_t tok = tok0 + (size_t)t * H;
+        bts[t] = route && route[tok] ? 0.f : beta[tok];
+        Gs[t] = Gcum[(size_t)bh * L + (size_t)ch * kC + t];
+    }
+    float Macc[4][4], Nacc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { Macc[i][j] = 0.f; Nacc[i][j] = 0.f; }
+    const int m0 = wr + fg, m1 = wr + fg + 8;
+    // acc += A B^T with both operands stored [row][k] in rows of 68 floats
+    auto mma_abt = [&](float (&acc)[4][4], const float *A, const float *Bm) {
+#pragma unroll 2
+        for (int k8 = 0; k8 < kC; k8 += 8) {
+            const int ka = k8 + ft, kb = k8 + ft + 4;
+            const uint32_t a[4] = {to_tf32(A[m0 * 68 + ka]), to_tf32(A[m1 * 68 + ka]),
+                                   to_tf32(A[m0 * 68 + kb]), to_tf32(A[m1 * 68 + kb])};
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int n = wc + 8 * nt + fg;
+                const uint32_t bb[2] = {to_tf32(Bm[n * 68 + ka]), to_tf32(Bm[n * 68 + kb])};
+                mma_tf32_16x8x8(acc[nt], a, bb);
+            }
+        }
+    };
+    for (int n0 = 0; n0 < D; n0 += 64) {
+        load_tile(bufA, 72, dW, n0);
+        load_tile(bufB, 72, dUt, n0);
+        cp_async_commit();
+        load_tile(bufC, 68, W, n0);
+        load_tile(bufD, 68, U, n0);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();
+        float kb_[4][4], vb_[4][4];          // dKb, dVb of these 64 columns
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { kb_[i][j] = 0.f; vb_[i][j] = 0.f; }
+#pragma unroll 2
+        for (int k8 = 0; k8 < kC; k8 += 8) {
+            const int ka = k8 + ft, kb = k8 + ft + 4;
+            const uint32_t a[4] = {to_tf32(sT[ka * 72 + m0]), to_tf32(sT[ka * 72 + m1]),
+                                   to_tf32(sT[kb * 72 + m0]), to_tf32(sT[kb * 72 + m1])};
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int n = wc + 8 * nt + fg;
+                const uint32_t b1[2] = {to_tf32(bufA[ka * 72 + n]), to_tf32(bufA[kb * 72 + n])};
+                const uint32_t b2[2] = {to_tf32(bufB[ka * 72 + n]), to_tf32(bufB[kb * 72 + n])};
+                mma_tf32_16x8x8(kb_[nt], a, b1);
+                mma_tf32_16x8x8(vb_[nt], a, b2);
+            }
+        }
+        __syncthreads();                     // dW, dU~ of these columns have been read by all
+        // fragment layout: elements (0, 1) in row fg, (2, 3) in row fg + 8; columns 2 ft, 2 ft + 1
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int row = wr + fg + 8 * hh, cl = wc + 8 * nt + 2 * ft;
+                const size_t i = (tok0 + (size_t)row * H) * D + n0 + cl;
+                const float2 kv = make_float2(kb_[nt][2 * hh], kb_[nt][2 * hh + 1]);
+                const float2 vv = make_float2(vb_[nt][2 * hh], vb_[nt][2 * hh + 1]);
+                *reinterpret_cast<float2 *>(dKb + i) = kv;
+                *reinterpret_cast<float2 *>(dVb + i) = vv;
+                *reinterpret_cast<float2 *>(bufA + row * 68 + cl) = kv;
+                *reinterpret_cast<float2 *>(bufB + row * 68 + cl) = vv;
+            }
+        cp_async_wait<0>();
+        __syncthreads();
+        mma_abt(Macc, bufA, bufC);           // dKb W^T
+        mma_abt(Macc, bufB, bufD);           // + dVb U^T
+        __syncthreads();
+        load_tile(bufA, 68, dO, n0);
+        load_tile(bufC, 68, Ut, n0);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+        mma_abt(Nacc, bufA, bufC);           // dO U~^T
+        __syncthreads();
+    }
+    const size_t base = (size_t)blockIdx.x * kC * kC;
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int row = wr + fg + 8 * hh, col = wc + 8 * nt + 2 * ft;
+            float mg[2], ns[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int j = col + e;
+                const float gam = j <= row ? __expf(Gs[row] - Gs[j]) : 0.f;
+                mg[e] = j < row ? -Macc[nt][2 * hh + e] * gam : 0.f;
+                ns[e] = scale_la * Nacc[nt][2 * hh + e] * gam;
+            }
+            const size_t o = base + (size_t)row * kC + col;
+            *reinterpret_cast<float2 *>(Mg + o) = make_float2(mg[0], mg[1]);
+            *reinterpret_cast<float2 *>(Ms + o) = make_float2(bts[row] * mg[0], bts[row] * mg[1]);
+            *reinterpret_cast<float2 *>(Ns + o) = make_float2(ns[0], ns[1]);
+        }
+}
+
 // The last four chunk-level products and the assembly in one kernel per chunk (bf16 storage, tf32
 // products as in bgemm_tf32_kernel): X1 = Mg K, X2 = Ms^T K, X3 = Ns K, X4 = Ns^T Q stay in the
 // accumulator fragments and meet the other terms of dq, dk, dv there, so the four [B,L,H,d] fp32
@@ -1352,6 +1497,20 @@ static cudaError_t finish_impl(const AssembleArgs &a, void *dk, void *dv, Shape 
     dim3 grid((a.cap + kRows - 1) / kRows, s.B * s.H);
     scatter_sm_kernel<T, D><<<grid, kThreads, 0, st>>>(a.dk_sm, a.dv_sm, a.cap, a.sm_idx, a.sm_prefix,
                                                        (T *)dk, (T *)dv, s.L, s.H);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gdn_tm(const float *Tinv, const float *dW, const float *dUt, const float *W, const float *U,
+                          const float *dO, const float *Ut, const float *Gcum, const float *beta,
+                          const uint8_t *route, float scale_la, float *dKb, float *dVb, float *Mg, float *Ms,
+                          float *Ns, Shape s, cudaStream_t st) {
+    const unsigned nch = (unsigned)(s.B * s.H * (s.L / kC));
+    auto kernel = s.d == 128 ? gdn_tm_kernel<128> : gdn_tm_kernel<64>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTmSmem);
+    if (e != cudaSuccess) return e;
+    kernel<<<nch, kThreads, kTmSmem, st>>>(Tinv, dW, dUt, W, U, dO, Ut, Gcum, beta, route, scale_la, dKb, dVb, Mg,
+                                          Ms, Ns, s.L, s.H);
     count_launch();
     return cudaGetLastError();
 }

@@ -248,6 +248,12 @@ struct AssembleArgs {
 // compacted softmax-branch gradients), dbeta, dg.  Three kernels.
 cudaError_t launch_gdn_assemble(const AssembleArgs &a, void *dq, void *dk, void *dv, Shape s,
                                 cudaStream_t st);
+// Tensor-core path (tf32 products), one kernel per chunk: dKb = Tinv^T dW, dVb = Tinv^T dU~ (written out),
+// M = -strictly_lower(dKb W^T + dVb U^T), N = lower(dO U~^T), then Mg, Ms, Ns as launch_mask_scale forms them.
+cudaError_t launch_gdn_tm(const float *Tinv, const float *dW, const float *dUt, const float *W, const float *U,
+                          const float *dO, const float *Ut, const float *Gcum, const float *beta,
+                          const uint8_t *route, float scale_la, float *dKb, float *dVb, float *Mg, float *Ms,
+                          float *Ns, Shape s, cudaStream_t st);
 // The same with the four products X1 = Mg K, X2 = Ms^T K, X3 = Ns K, X4 = Ns^T Q formed inside (tf32
 // tensor-core products; a.X1p .. a.X4 are not read); s.bf16 says what dq, dk, dv are stored as.
 cudaError_t launch_gdn_xassemble(const AssembleArgs &a, const float *Mg, const float *Ms, const float *Ns,

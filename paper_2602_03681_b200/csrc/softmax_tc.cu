@@ -65,7 +65,7 @@ template <int D> struct SmLayout {
 };
 
 struct Misc {                    // lives in the last kMiscBytes of the CTA's shared memory
-    uint64_t barQ, barQn, barKn, fullK[kStages], emptyK[kStages], fullV[kStages], emptyV[kStages], barS[2], barP, barO, barE;
+    uint64_t barQ, barQn, barKn[2], fullK[kStages], emptyK[kStages], fullV[kStages], emptyV[kStages], barS[2], barP, barO, barE;
     uint32_t tmem_base;
     int abort_flag, wait_kcycles;   // in this order: the waits read the limit as abort_flag[1]
     alignas(16) int pos[kBM];    // positions of the retained tokens inside the CTA's own chunks
@@ -132,7 +132,8 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
     if (tid == 0) {
         mbar_init(&ms.barQ, 1);
         mbar_init(&ms.barQn, kSoftmaxThreads);       // normalised queries written (NATSL_QK_NORM)
-        mbar_init(&ms.barKn, 1);                     // ... and the keys of an own-block tile (one phase per tile)
+        mbar_init(&ms.barKn[0], 1);                  // ... and the keys of an own-block tile: one barrier per tile,
+        mbar_init(&ms.barKn[1], 1);                  //     each completing once
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&ms.fullK[s], 1); mbar_init(&ms.emptyK[s], 1);
             mbar_init(&ms.fullV[s], 1); mbar_init(&ms.emptyV[s], 1);
@@ -243,9 +244,13 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
                 mma_commit(&ms.barS[t & 1]);
             };
             // (normalisation with block-level routing: an own-block tile's keys arrive raw and are
-            // normalised in place by the softmax threads first; barKn completes one phase per such tile)
+            // normalised in place by the softmax threads first.  One single-phase barrier per own-block
+            // tile, of which a CTA has at most two: with one barrier and a phase per tile, nothing kept the
+            // softmax threads from completing the second phase before this thread had looked at the
+            // first -- a parity wait then never returns -- and a late enough start of this thread, as in
+            // the first wave of a launch, did let that happen.)
             auto own_keys_ready = [&](int t) {
-                return !(kBlock && kNorm) || t < T || mbar_wait(&ms.barKn, (t - T) & 1, abort_flag);
+                return !(kBlock && kNorm) || t < T || mbar_wait(&ms.barKn[t - T], 0, abort_flag);
             };
             bool ok = mbar_wait(&ms.barQ, 0, abort_flag) && (!kNorm || mbar_wait(&ms.barQn, 0, abort_flag)) &&
                       mbar_wait(&ms.fullK[0], 0, abort_flag) && own_keys_ready(0);
@@ -368,7 +373,7 @@ softmax_combine_tc_kernel(const __grid_constant__ CUtensorMap map_q,
             // writing this tile's rows, and completed this tile's phase for them.)
             fence_proxy_async_smem();
             named_barrier_sync(2, kSoftmaxThreads);
-            if (tid == 0) mbar_arrive(&ms.barKn);
+            if (tid == 0) mbar_arrive(&ms.barKn[u - T]);
             return true;
         };
         if (kBlock && kNorm && ok && T2 > 0 && T == 0) ok = normalise_own_keys(0);
