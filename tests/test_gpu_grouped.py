@@ -134,6 +134,35 @@ def test_bf16_paper_mode_at_length():
     check(wl, got, ref, TOL["bf16"], 2)
 
 
+def test_paper_mode_forward_repeated_calls_complete_and_agree():
+    """Many back-to-back calls on shapes whose second query tile has two own-block tiles in most heads (the
+    case in which the MMA thread waits for two rounds of in-kernel key normalisation): every call ends
+    without a device-side time-out and returns the same bits.  With a short bound on the waits, so that a
+    missed hand-over shows as a status, not as a two-second stall."""
+    from paper_2602_03681_b200 import binding
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg1_bf16_prefill"], seed=83)
+    B, H, L, G = 8, 6, 512, 2
+    x = make_inputs(wl, B, H, L, True, block_p=0.15)
+    dt = tdtype(wl)
+    args = [dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]), dev(x["beta"]), dev(x["route"]), dev(x["w"])]
+    f = binding.QK_NORM | binding.BLOCK_ROUTING
+    binding.natsl_debug_set_wait_limit(100000)           # ~0.05 s
+    try:
+        first, ws = None, None
+        for it in range(60):
+            res = binding.hybrid_fwd(*args, scale_la=wl.scale_la, scale_sm=64 ** -0.5, flags=f, G=G, norm_eps=1e-6, ws=ws)
+            ws = res["ws"]
+            if it % 10 == 9 or it == 0:
+                torch.cuda.synchronize()
+                assert binding.natsl_device_status(ws) == 0, it
+                out = res["out"].clone()
+                if first is None:
+                    first = out
+                assert torch.equal(out, first), it
+    finally:
+        binding.natsl_debug_set_wait_limit(0)
+
+
 def test_bf16_tensor_cores_d64_normalisation():
     """The normalisation alone at d = 64 (one softmax head per linear head, the 64-column kernels)."""
     wl = dataclasses.replace(inputs.WORKLOADS["cfg4_bf16_train"], seed=47)
