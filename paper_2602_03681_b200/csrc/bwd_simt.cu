@@ -963,14 +963,22 @@ gdn_tm_kernel(const float *__restrict__ Tinv, const float *__restrict__ dW, cons
             }
         }
     };
+    // Per 64 columns: every group of loads is in flight while the previous product runs.
     for (int n0 = 0; n0 < D; n0 += 64) {
-        load_tile(bufA, 72, dW, n0);
-        load_tile(bufB, 72, dUt, n0);
+        load_tile(bufA, 68, dO, n0);
+        load_tile(bufC, 68, Ut, n0);
         cp_async_commit();
-        load_tile(bufC, 68, W, n0);
-        load_tile(bufD, 68, U, n0);
+        load_tile(bufB, 72, dW, n0);
+        load_tile(bufD, 72, dUt, n0);
         cp_async_commit();
         cp_async_wait<1>();
+        __syncthreads();
+        mma_abt(Nacc, bufA, bufC);           // dO U~^T
+        __syncthreads();                     // dO, U~ of these columns have been read by all
+        load_tile(bufA, 68, W, n0);
+        load_tile(bufC, 68, U, n0);
+        cp_async_commit();
+        cp_async_wait<1>();                  // dW, dU~ (and Tinv) have landed
         __syncthreads();
         float kb_[4][4], vb_[4][4];          // dKb, dVb of these 64 columns
 #pragma unroll
@@ -985,8 +993,8 @@ gdn_tm_kernel(const float *__restrict__ Tinv, const float *__restrict__ dW, cons
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt) {
                 const int n = wc + 8 * nt + fg;
-                const uint32_t b1[2] = {to_tf32(bufA[ka * 72 + n]), to_tf32(bufA[kb * 72 + n])};
-                const uint32_t b2[2] = {to_tf32(bufB[ka * 72 + n]), to_tf32(bufB[kb * 72 + n])};
+                const uint32_t b1[2] = {to_tf32(bufB[ka * 72 + n]), to_tf32(bufB[kb * 72 + n])};
+                const uint32_t b2[2] = {to_tf32(bufD[ka * 72 + n]), to_tf32(bufD[kb * 72 + n])};
                 mma_tf32_16x8x8(kb_[nt], a, b1);
                 mma_tf32_16x8x8(vb_[nt], a, b2);
             }
@@ -1003,20 +1011,13 @@ gdn_tm_kernel(const float *__restrict__ Tinv, const float *__restrict__ dW, cons
                 const float2 vv = make_float2(vb_[nt][2 * hh], vb_[nt][2 * hh + 1]);
                 *reinterpret_cast<float2 *>(dKb + i) = kv;
                 *reinterpret_cast<float2 *>(dVb + i) = vv;
-                *reinterpret_cast<float2 *>(bufA + row * 68 + cl) = kv;
-                *reinterpret_cast<float2 *>(bufB + row * 68 + cl) = vv;
+                *reinterpret_cast<float2 *>(bufB + row * 68 + cl) = kv;
+                *reinterpret_cast<float2 *>(bufD + row * 68 + cl) = vv;
             }
-        cp_async_wait<0>();
+        cp_async_wait<0>();                  // W, U
         __syncthreads();
-        mma_abt(Macc, bufA, bufC);           // dKb W^T
-        mma_abt(Macc, bufB, bufD);           // + dVb U^T
-        __syncthreads();
-        load_tile(bufA, 68, dO, n0);
-        load_tile(bufC, 68, Ut, n0);
-        cp_async_commit();
-        cp_async_wait<0>();
-        __syncthreads();
-        mma_abt(Nacc, bufA, bufC);           // dO U~^T
+        mma_abt(Macc, bufB, bufA);           // dKb W^T
+        mma_abt(Macc, bufD, bufC);           // + dVb U^T
         __syncthreads();
     }
     const size_t base = (size_t)blockIdx.x * kC * kC;
