@@ -216,12 +216,16 @@ BwdWs carve_bwd(const natsl_params *p, void *ws) {
     f.do_nla = tm(!tcs);
     f.dUt = tcs ? f.o_la : tm(true);
     f.dQg = tm(general); f.dW = tm(general); f.dKt = tm(general); f.dKb = tm(general); f.dVb = tm(general);
-    f.X1p = tm(general); f.X2 = tm(general);
-    f.X3 = tm(general || block); f.X4 = tm(general || block);
+    // (the last four products' results: only the fp32 path stores them, the tensor-core path keeps them in
+    // the accumulators of its assembly kernel; X3, X4 also serve the fused chunk kernel's block-routed call
+    // as its side buffers)
+    f.X1p = tm(general && !tcs); f.X2 = tm(general && !tcs);
+    f.X3 = tm((general && !tcs) || (fused && block)); f.X4 = tm((general && !tcs) || (fused && block));
     f.dq_sm = tcs ? f.o_nla : tm(true);
     f.dk_sm = tm(true); f.dv_sm = tm(true);
     f.P = cc(!tcs); f.Abar = cc(!tcs);
-    f.M = cc(general); f.N = cc(general); f.Mg = cc(general); f.Ms = cc(general); f.Ns = cc(general);
+    f.M = cc(general && !tcs); f.N = cc(general && !tcs);     // (tensor cores: M, N stay in gdn_tm_kernel's accumulators)
+    f.Mg = cc(general); f.Ms = cc(general); f.Ns = cc(general);
     f.S_c = c.take<float>(ST);
     f.dS_c = c.take<float>(ST);
     f.Gcum = c.take<float>(BHL);
