@@ -676,7 +676,11 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     std::unique_lock<std::mutex> side_lock;
     SideStream *side = nullptr;
     SideJoin side_join;
-    if (fused_chunks && !(p->flags & NATSL_SINGLE_STREAM)) {
+    // (tensor cores with separate chunk-level kernels: the whole linear branch -- reverse scan, the products
+    // with the states, the middle of the chain -- runs on the side stream beside the softmax branch's
+    // backward, and the two meet at the assembly)
+    const bool side_general = tensor_cores && !fused_chunks;
+    if ((fused_chunks || side_general) && !(p->flags & NATSL_SINGLE_STREAM)) {
         side_lock = std::unique_lock<std::mutex>(g_side_mu);
         side = side_stream_locked();
         if (!side) side_lock.unlock();
@@ -699,7 +703,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     // kernel, scatter; caller's stream = query-side kernel, chunk kernel.  (Block-level routing:
     // the chunk kernel adds the scattered gradients and so waits for the side stream, but the
     // own-block kernel, which needs the query-side kernel only, still runs beside the key-side one.)
-    const bool kv_aside = side != nullptr;
+    const bool kv_aside = side != nullptr && fused_chunks;
     if (side) {
         NATSL_TRY(cudaEventRecord(side->fork, st));
         NATSL_TRY(cudaStreamWaitEvent(st0, side->fork, 0));
@@ -710,10 +714,13 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         NATSL_TRY(launch_gdn_rscan_tc(f.dOla16, f.dOlag16, f.tc, f.S_c, f.dUt, f.dS_c,
                                       fused_chunks ? nullptr : f.gS, p->dstate_out, p->dstate_in,
                                       block_route, f.status, s, st0));
-    if (side) NATSL_TRY(cudaEventRecord(side->join, st0));
+    if (side && fused_chunks) NATSL_TRY(cudaEventRecord(side->join, st0));
     if (tensor_cores)   // (d = 64: the prepare kernel has left the fp16 copy of q in f.Qh, and the reverse
                         //  scan on the side stream reads it, so it is not written again)
-        NATSL_TRY(launch_softmax_bwd_tc(q, f.Qh, f.dO16, f.k16, f.v16, p->L, f.sm_idx, f.prefix, f.lse,
+        // (separate chunk-level kernels: the softmax branch writes its own fp16 copy of q -- raw, or RMS-
+        //  normalised -- while the reverse scan beside it reads the linear operation's copy in f.Qh; the copy
+        //  goes where the forward's softmax kernel had its gathered keys, which nothing reads any more)
+        NATSL_TRY(launch_softmax_bwd_tc(q, fused_chunks ? f.Qh : f.k_smb, f.dO16, f.k16, f.v16, p->L, f.sm_idx, f.prefix, f.lse,
                                         f.Dsm, p->scale_sm, f.dq_sm, f.dk_sm, f.dv_sm,
                                         p->dscore ? (general_block ? f.dmask : f.dGrow) : nullptr, fused_chunks,
                                         f.status, s, st, kv_aside ? st0 : st, hg));
@@ -724,7 +731,7 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
     if (!tensor_cores)
         NATSL_TRY(launch_gdn_rscan(f.q32, f.k32, f.Gcum, f.W, f.P, f.do_la, f.S_c, p->scale_la, f.dUt,
                                    f.dS_c, f.gS, p->dstate_out, p->dstate_in, s, st, block_route));
-    if (side) NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));     // the reverse scan has finished
+    if (side && fused_chunks) NATSL_TRY(cudaStreamWaitEvent(st, side->join, 0));     // the reverse scan has finished
     // (with the normalisation the two operations' dq stay apart until its backward at the very end)
     const bool normed = hg.norm_eps >= 0.f;
     AssembleArgs a{f.q32, f.k32, f.v32, f.Gcum, beta, general_block ? nullptr : route, f.dQg, f.dKb, f.dVb, f.dKt, f.X1p, f.X2,
@@ -781,13 +788,15 @@ int natsl_hybrid_bwd(const void *q, const void *k, const void *v, const float *g
         a.dv_x = f.dv_x;
         a.no_scatter = true;
     }
-    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, sgemm, st));
-    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, sgemm, st));
-    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, sgemm, st));
+    cudaStream_t stl = side ? st0 : st;     // the linear branch's stream (behind the reverse scan)
+    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.do_la), ST(f.S_c), TM(f.dQg), kC, di, di, 1.f, false, sgemm, stl));
+    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.dUt), ST(f.S_c), TM(f.dW), kC, di, di, -1.f, false, sgemm, stl));
+    NATSL_TRY(launch_bgemm(false, true, 0, TM(f.Ut), ST(f.dS_c), TM(f.dKt), kC, di, di, 1.f, false, sgemm, stl));
     if (tensor_cores) {   // [dKb | dVb] = (I + A)^-T [dW | dU~] with the inverse the forward already formed, M, N and
                           // their masked, scaled forms: one kernel per chunk
         NATSL_TRY(launch_gdn_tm(f.Tinv, f.dW, f.dUt, f.W, f.U, f.do_la, f.Ut, f.Gcum, beta, route_bt, p->scale_la,
-                                f.dKb, f.dVb, f.Mg, f.Ms, f.Ns, s, st));
+                                f.dKb, f.dVb, f.Mg, f.Ms, f.Ns, s, stl));
+        NATSL_TRY(side_join.join());      // the two branches meet at the assembly
     } else {
         NATSL_TRY(launch_bgemm(false, true, 1, TM(f.do_la), TM(f.Ut), CC(f.N), kC, kC, di, 1.f, false, sgemm, st));
         NATSL_TRY(launch_gdn_tsolve(f.Abar, beta, route_bt, f.dW, f.dUt, f.dKb, f.dVb, s, st));
