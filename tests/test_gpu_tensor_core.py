@@ -184,6 +184,11 @@ def test_fwd_tensor_core_is_deterministic():
 @pytest.mark.parametrize("name,B,H,L,route", [("cfg4_bf16_train", 2, 3, 320, None),
                                               ("cfg4_bf16_train", 1, 2, 64, None),
                                               ("cfg1_bf16_prefill", 1, 2, 448, None),
+                                              # d = 128 (separate chunk-level kernels, two streams): one chunk;
+                                              # odd batch and head counts; all tokens retained
+                                              ("cfg1_bf16_prefill", 3, 1, 64, None),
+                                              ("cfg1_bf16_prefill", 3, 5, 128, None),
+                                              ("cfg1_bf16_prefill", 1, 3, 192, "all_softmax"),
                                               ("cfg4_bf16_train", 1, 2, 384, "all_softmax"),
                                               ("cfg1_bf16_prefill", 1, 2, 256, "all_linear"),
                                               ("cfg4_bf16_train", 1, 1, 256, "late")])
@@ -229,8 +234,9 @@ def test_bwd_tensor_core_is_linear_in_the_incoming_gradient(scale, name, block):
     check_bwd(wl, got, ref, TOL["bf16"])
 
 
-def test_bwd_tensor_core_many_chunks():
-    wl = inputs.WORKLOADS["cfg4_bf16_train"]
+@pytest.mark.parametrize("name", ["cfg4_bf16_train", "cfg1_bf16_prefill"])
+def test_bwd_tensor_core_many_chunks(name):
+    wl = inputs.WORKLOADS[name]
     x = inputs.make_layer_inputs(wl, B=1, H=2, L=1024)
     got = run_bwd(wl, x)
     ref = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
