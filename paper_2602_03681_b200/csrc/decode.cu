@@ -128,7 +128,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
     }
     __syncthreads();
     volatile int *abort_flag = s_abort;
-    if (kGrouped) {
+    if (kGrouped && warp < kWarps) {     // (the work threads only: the copy warp goes straight to its ring)
         // q, k of the two operations: L2 over the row for the linear one (in place in qs, ks), RMS per slice
         // for the softmax one (qsm, ksm); without the normalisation both are the token's q, k.
         float sq = 0.f, sk = 0.f;
@@ -136,7 +136,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
         sq = warp_sum(sq);
         sk = warp_sum(sk);
         if (lane == 0 && warp < D / 32) { norm_red[0][warp] = sq; norm_red[1][warp] = sk; }
-        __syncthreads();
+        named_barrier_sync(1, kWorkThreads);
         if (tid < D) {
             float aq = 0.f, ak = 0.f, gq = 0.f, gk = 0.f;
             for (int wv = 0; wv < D / 32; ++wv) {
@@ -149,7 +149,7 @@ decode_step_kernel(const T *__restrict__ q, const T *__restrict__ k, const T *__
             ksm[tid] = normed ? kv * rsqrtf(gk / ds + norm_eps) : kv;
             if (normed) { qs[tid] = qv * rsqrtf(aq + norm_eps); ks[tid] = kv * rsqrtf(ak + norm_eps); }
         }
-        __syncthreads();
+        named_barrier_sync(1, kWorkThreads);
     }
 
     if (part < kDecodeParts) {
