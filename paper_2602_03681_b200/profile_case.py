@@ -86,7 +86,10 @@ def main():
         x = inputs.make_decode_inputs(wl, B=B, steps=args.iters)
         state, n = dev(x["state"]), dev(x["cache_len"])
         kc, vc = dev(x["k_cache"], dt), dev(x["v_cache"], dt)
-        p = binding.make_params(B, wl.H, 0, wl.d, code, wl.scale_la, wl.scale_sm, flags=args.flags)
+        p = binding.make_params(B, wl.H, 0, wl.d, code, wl.scale_la,
+                                float(wl.d // max(args.G, 1)) ** -0.5 if args.qk_norm else wl.scale_sm,
+                                flags=args.flags | (binding.QK_NORM if args.qk_norm else 0), G=args.G,
+                                norm_eps=1e-6 if args.qk_norm else 0.0)
         ws = binding.alloc_workspace(p, binding.OP_DECODE)
         out = torch.empty((B, wl.H, wl.d), dtype=dt, device="cuda")
         tok = {m: dev(x[m], dt if m in ("q", "k", "v") else None)
