@@ -78,6 +78,86 @@ def test_fwd_bwd_full_size_training_workload_block_routing():
     check_bwd(wl, gb, rb, TOL[wl.dtype])
 
 
+@pytest.mark.parametrize("block", [False, True])
+def test_bwd_full_size_prefill_shapes(block):
+    """The backward at d = 128 (separate chunk-level kernels on two streams) on the prefill workload's full
+    shapes, token-level and with one decision per block: every element of every gradient."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS["cfg1_bf16_prefill"]
+    route = inputs.route_blocks(wl.seed, (wl.B, wl.L, wl.H), wl.p_softmax) if block else None
+    x = inputs.make_layer_inputs(wl, route=route)
+    gb = run_bwd(wl, x, flags=binding.BLOCK_ROUTING if block else 0)
+    rb = oracle.hybrid_bwd(x["q"], x["k"], x["v"], x["g"], x["beta"], x["route"], x["w"], x["dout"],
+                           scale_la=wl.scale_la, scale_sm=wl.scale_sm, block=64 if block else None)
+    check_bwd(wl, gb, rb, TOL[wl.dtype])
+    if not block:
+        assert np.all(gb["dbeta"][x["route"] != 0] == 0)
+
+
+def test_paper_mode_training_step_full_size_sampled_heads():
+    """The paper's mode at the size bench.py times it (six linear heads of 128 columns with two softmax heads
+    each, q and k normalised per operation, one decision per block, B = 10, L = 4096; saved forward, then
+    backward with score gradients).  Every (batch, head) is independent, so the oracle -- plain fp64
+    statements differentiated in reverse mode, far too slow for all sixty -- recomputes two of them at full
+    length, and their slices of `out` and of every gradient are compared element by element."""
+    import dataclasses
+    from oracle import grouped
+    from paper_2602_03681_b200 import binding
+    from test_gpu_grouped import make_inputs
+    from test_gpu_parity import rel_err
+    B, H, G, L, d = 10, 6, 2, 4096, 128
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg1_bf16_prefill"], seed=29)
+    # (row lengths of q, k log-normal with sigma 0.4: the gradients through the normalisation go with the
+    # inverse row length, and the tolerance is relative to the RMS of the whole tensor -- with the wider
+    # spread of the small cases, over 245 760 rows, single rows of dk reach 50 x RMS, where the error the
+    # 11-bit operands leave on such a row alone exceeds 2 % of the RMS)
+    x = make_inputs(wl, B, H, L, True, block_p=wl.p_softmax, spread=0.4)
+    scale_sm = (d / G) ** -0.5
+    dt = torch.bfloat16
+    flags = binding.QK_NORM | binding.BLOCK_ROUTING
+    w_dev = dev(x["w"])
+    pf = binding.make_params(B, H, L, d, binding.NATSL_BF16, wl.scale_la, scale_sm, w=w_dev, G=G, norm_eps=1e-6,
+                             flags=flags | binding.SAVE_FOR_BWD)
+    ws = binding.alloc_workspace(pf, binding.OP_BWD)
+    t = {n: dev(x[n], dt) for n in ("q", "k", "v", "dout")}
+    t.update({n: dev(x[n]) for n in ("g", "beta", "route")})
+    out = torch.empty_like(t["q"])
+    binding.natsl_hybrid_fwd(t["q"], t["k"], t["v"], t["g"], t["beta"], t["route"], out, pf, ws)
+    pb = binding.make_params(B, H, L, d, binding.NATSL_BF16, wl.scale_la, scale_sm, w=w_dev, G=G, norm_eps=1e-6,
+                             flags=flags | binding.SAVED_FWD)
+    dscore = torch.zeros((B, L // 64, H, 2), device="cuda")
+    pb.dscore = dscore.data_ptr()
+    outs = {n: torch.empty_like(t["q"]) for n in ("dq", "dk", "dv")}
+    outs.update(dg=torch.empty_like(t["g"]), dbeta=torch.empty_like(t["g"]),
+                dw=torch.empty((B, L, H, 2), device="cuda"))
+    binding.natsl_hybrid_bwd(t["q"], t["k"], t["v"], t["g"], t["beta"], t["route"], t["dout"], outs["dq"], outs["dk"],
+                             outs["dv"], outs["dg"], outs["dbeta"], outs["dw"], pb, ws)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(ws) == 0
+    got = {n: v.float().cpu().numpy() for n, v in outs.items()}
+    got["out"] = out.float().cpu().numpy()
+    got["dscore"] = dscore.cpu().numpy()
+    tol = TOL["bf16"]
+    kw = dict(G=G, qk_norm=True, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6, block=64)
+    for b, h in ((0, 0), (7, 4)):
+        sl = lambda a: a[b:b + 1, :, h:h + 1]
+        xs = {n: np.ascontiguousarray(sl(x[n])) for n in ("q", "k", "v", "g", "beta", "route", "w", "dout")}
+        ref_f = grouped.hybrid_fwd(xs["q"], xs["k"], xs["v"], xs["g"], xs["beta"], xs["route"], xs["w"], **kw)
+        check_stored(sl(got["out"]), ref_f["out"], tol, "bf16")
+        ref = grouped.hybrid_bwd(xs["q"], xs["k"], xs["v"], xs["g"], xs["beta"], xs["route"], xs["w"], xs["dout"],
+                                 want_dscore=True, **kw)
+        for n in ("dq", "dk", "dv"):
+            check_stored(sl(got[n]), ref[n], tol, "bf16", n, large_only=False)
+        for n in ("dg", "dbeta", "dw"):
+            e = rel_err(sl(got[n]), ref[n])
+            assert e <= tol, (b, h, n, e)
+        for op in (0, 1):
+            r = ref["dscore"][..., op]
+            if np.abs(r).max() > 0:
+                e = rel_err(got["dscore"][b:b + 1, :, h:h + 1, op], r)
+                assert e <= tol, (b, h, "dscore", op, e)
+
+
 def test_decode_full_size_sampled_sequences():
     from paper_2602_03681_b200 import binding
     wl = inputs.WORKLOADS["cfg3_bf16_decode"]
