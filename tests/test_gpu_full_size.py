@@ -94,6 +94,41 @@ def test_bwd_full_size_prefill_shapes(block):
         assert np.all(gb["dbeta"][x["route"] != 0] == 0)
 
 
+def test_grouped_forward_full_size_sampled_heads():
+    """Token-level routing with two softmax heads per linear head and q, k normalised inside the kernels, at
+    the size bench.py times it (B = 10, H = 6, L = 4096, d = 128): two (batch, head) pairs recomputed by the
+    oracle at full length, every element of their slices of out, the branch outputs, lse and the final state."""
+    import dataclasses
+    from oracle import grouped
+    from paper_2602_03681_b200 import binding
+    from test_gpu_grouped import make_inputs
+    from test_gpu_parity import rel_err
+    B, H, G, L, d = 10, 6, 2, 4096, 128
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg1_bf16_prefill"], seed=31)
+    x = make_inputs(wl, B, H, L, True)
+    scale_sm = (d / G) ** -0.5
+    dt = torch.bfloat16
+    res = binding.hybrid_fwd(dev(x["q"], dt), dev(x["k"], dt), dev(x["v"], dt), dev(x["g"]), dev(x["beta"]),
+                             dev(x["route"]), dev(x["w"]), scale_la=wl.scale_la, scale_sm=scale_sm,
+                             want=("o_la", "o_nla", "lse", "state_out"), flags=binding.QK_NORM, G=G, norm_eps=1e-6)
+    torch.cuda.synchronize()
+    assert binding.natsl_device_status(res["ws"]) == 0
+    got = {n: t.float().cpu().numpy() for n, t in res.items() if n != "ws"}
+    tol = TOL["bf16"]
+    for b, h in ((2, 5), (9, 0)):
+        sl = lambda a: np.ascontiguousarray(a[b:b + 1, :, h:h + 1])
+        ref = grouped.hybrid_fwd(sl(x["q"]), sl(x["k"]), sl(x["v"]), sl(x["g"]), sl(x["beta"]), sl(x["route"]),
+                                 sl(x["w"]), G=G, qk_norm=True, scale_la=wl.scale_la, scale_sm=scale_sm, norm_eps=1e-6)
+        check_stored(sl(got["out"]), ref["out"], tol, "bf16")
+        for n in ("o_la", "o_nla"):
+            assert rel_err(sl(got[n]), ref[n]) <= tol, (b, h, n)
+        assert rel_err(got["state_out"][b:b + 1, h:h + 1], ref["state_out"]) <= tol, (b, h)
+        lse = got["lse"].reshape(B, H, G, L)[b:b + 1, h:h + 1]
+        fin = np.isfinite(ref["lse"])
+        assert np.array_equal(np.isneginf(lse), ~fin)
+        assert np.abs(lse[fin] - ref["lse"][fin]).max() <= 2 * tol
+
+
 def test_paper_mode_training_step_full_size_sampled_heads():
     """The paper's mode at the size bench.py times it (six linear heads of 128 columns with two softmax heads
     each, q and k normalised per operation, one decision per block, B = 10, L = 4096; saved forward, then
