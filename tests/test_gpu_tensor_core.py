@@ -235,6 +235,25 @@ def test_bwd_tensor_core_is_linear_in_the_incoming_gradient(scale, name, block):
 
 
 @pytest.mark.parametrize("name", ["cfg4_bf16_train", "cfg1_bf16_prefill"])
+@pytest.mark.parametrize("block", [False, True])
+def test_bwd_on_one_stream_gives_the_same_bits(name, block):
+    """NATSL_SINGLE_STREAM puts every kernel of the backward on the caller's stream; by default independent
+    stages run on a second stream beside it (d = 64: reverse scan and key-side softmax kernel beside the
+    query-side and chunk kernels; d = 128: the whole linear branch beside the softmax branch).  Same kernels,
+    same inputs: the gradients must agree bit for bit, or two stages share a buffer they should not."""
+    from paper_2602_03681_b200 import binding
+    wl = inputs.WORKLOADS[name]
+    B, H, L = 2, 3, 512
+    route = inputs.route_blocks(wl.seed, (B, L, H), wl.p_softmax) if block else None
+    x = inputs.make_layer_inputs(wl, B=B, H=H, L=L, route=route)
+    f = binding.BLOCK_ROUTING if block else 0
+    a = run_bwd(wl, x, flags=f)
+    b = run_bwd(wl, x, flags=f | binding.SINGLE_STREAM)
+    for n in ("dq", "dk", "dv", "dg", "dbeta", "dw"):
+        assert np.array_equal(a[n], b[n]), n
+
+
+@pytest.mark.parametrize("name", ["cfg4_bf16_train", "cfg1_bf16_prefill"])
 def test_bwd_tensor_core_many_chunks(name):
     wl = inputs.WORKLOADS[name]
     x = inputs.make_layer_inputs(wl, B=1, H=2, L=1024)
