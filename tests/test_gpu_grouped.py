@@ -307,6 +307,37 @@ def test_block_level_routing_backward_with_grouped_heads(storage, d, G, norm, B,
             assert rel_err(gd[..., op], ref["dscore"][..., op]) <= TOL[storage], (op, rel_err(gd[..., op], ref["dscore"][..., op]))
 
 
+def test_paper_mode_backward_on_one_stream_gives_the_same_bits():
+    """Grouped heads, normalised q and k, one decision per block: the backward with every kernel on the caller's
+    stream (NATSL_SINGLE_STREAM) and the default one, whose linear branch runs on a second stream beside the
+    softmax branch, agree bit for bit (they would not if the two branches shared a buffer)."""
+    from paper_2602_03681_b200 import binding
+    d, G, B, H, L = 128, 2, 2, 3, 512
+    wl = dataclasses.replace(inputs.WORKLOADS["cfg1_bf16_prefill"], seed=97)
+    x = make_inputs(wl, B, H, L, True, block_p=0.3)
+    dt = tdtype(wl)
+    t = {n: dev(x[n], dt) for n in ("q", "k", "v", "dout")}
+    t.update({n: dev(x[n]) for n in ("g", "beta", "route")})
+    w_dev = dev(x["w"])
+    results = []
+    for extra in (0, binding.SINGLE_STREAM):
+        pr = binding.make_params(B, H, L, d, binding.NATSL_BF16, wl.scale_la, (d / G) ** -0.5, w=w_dev, G=G,
+                                 norm_eps=1e-6, flags=binding.BLOCK_ROUTING | binding.QK_NORM | extra)
+        dscore = torch.zeros((B, L // 64, H, 2), device="cuda")
+        pr.dscore = dscore.data_ptr()
+        ws = binding.alloc_workspace(pr, binding.OP_BWD)
+        outs = {n: torch.empty_like(t["q"]) for n in ("dq", "dk", "dv")}
+        outs.update(dg=torch.empty_like(t["g"]), dbeta=torch.empty_like(t["g"]),
+                    dw=torch.empty((B, L, H, 2), device="cuda"), dscore=dscore)
+        binding.natsl_hybrid_bwd(t["q"], t["k"], t["v"], t["g"], t["beta"], t["route"], t["dout"], outs["dq"],
+                                 outs["dk"], outs["dv"], outs["dg"], outs["dbeta"], outs["dw"], pr, ws)
+        torch.cuda.synchronize()
+        assert binding.natsl_device_status(ws) == 0
+        results.append(outs)
+    for n in results[0]:
+        assert torch.equal(results[0][n], results[1][n]), n
+
+
 @pytest.mark.parametrize("storage,block", [("bf16", False), ("bf16", True), ("f32", False)])
 def test_saved_forward_then_backward_with_grouped_heads(storage, block):
     """The training step as two calls (NATSL_SAVE_FOR_BWD, then NATSL_SAVED_FWD) with grouped heads and the
